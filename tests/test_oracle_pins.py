@@ -1,0 +1,354 @@
+"""Pins for the fp64 oracle: things the paper and the mathematics fix, none of which
+re-types the oracle's own formula.  CPU only."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import kata_oracle as ko
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def golden(name):
+    out = {}
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, *vals = line.split()
+            out[key] = float(vals[0])
+    return out
+
+
+def rng(seed):
+    return np.random.default_rng(seed)
+
+
+def rand_qkv(seed, T, d, dv):
+    r = rng(seed)
+    return r.standard_normal((T, d)), r.standard_normal((T, d)), r.standard_normal((T, dv))
+
+
+# ---------------------------------------------------------------------------
+# printed numbers
+# ---------------------------------------------------------------------------
+
+def test_rope_worked_example_weight():
+    g = golden("rope_kernel_ratio.txt")
+    ang = g["omega_delta"]
+    q = np.array([[1.0, 0.0]])
+    k = np.array([[math.cos(ang), math.sin(ang)]])
+    w = ko.causal_weights(3.7 * q, 0.2 * k)[0, 0]       # scale must not matter
+    assert round(w, 4) == g["r_kata"]
+    assert abs(w - math.cos(ang) ** 2) < 1e-15
+    # the companion softmax number, to check the fixture was read in the right way
+    assert round(math.exp((math.cos(ang) - 1.0) / g["tau"]), 4) == g["r_softmax"]
+
+
+def test_feature_widths_printed():
+    g = golden("feature_widths.txt")
+    d = int(g["d"])
+    u = rng(0).standard_normal((3, d))
+    assert ko.psi_direct(u).shape[-1] == g["direct"] == ko.feature_dim(d, "psd_direct")
+    assert ko.psi_packed(u).shape[-1] == g["packed"] == ko.feature_dim(d, "psd_packed")
+
+
+def test_state_entries_table():
+    g = golden("state_entries_kata_m1.txt")
+    d, dv = int(g["d"]), int(g["d_v"])
+    k, v = rng(1).standard_normal((5, d)), rng(2).standard_normal((5, dv))
+    S_loc, Z_loc = ko.chunk_local_states(k, v, 5, "psd_packed")
+    assert g["layers"] * S_loc[0].size == g["state_entries"]
+    assert Z_loc[0].size == d * (d + 1) // 2
+
+
+def test_scan_rounds_printed():
+    g = golden("scan_rounds.txt")
+    NC = -(-int(g["T"]) // int(g["C"]))
+    assert NC == g["n_chunks"]
+    assert ko.scan_rounds(NC) == g["rounds"]
+    x = rng(3).standard_normal((NC, 4, 3))
+    pre, rounds = ko.exclusive_prefix_doubling(x)
+    assert rounds == g["rounds"]
+    assert np.all(pre[0] == 0)
+    for n, r in [(1, 0), (2, 1), (3, 2), (5, 3), (128, 7), (512, 9), (2048, 11), (2049, 12)]:
+        assert ko.scan_rounds(n) == r
+        assert ko.exclusive_prefix_doubling(np.ones((n, 1)))[1] == r
+
+
+def test_psnr_simplex_closed_form():
+    g = golden("psnr_welch.txt")
+    p, T = int(g["p"]), int(g["T"])
+    # regular simplex: centre the T standard basis vectors of R^T, express in the (T-1)-dim span
+    E = np.eye(T) - 1.0 / T
+    U, s, _ = np.linalg.svd(E)
+    keys = (U[:, :p] * s[:p])
+    keys /= np.linalg.norm(keys, axis=1, keepdims=True)
+    G = keys @ keys.T
+    assert np.allclose(G[~np.eye(T, dtype=bool)], -1.0 / p, atol=1e-12)
+    v = np.eye(T)                       # orthonormal values: coefficients are read off directly
+    for j in range(T):
+        q = np.tile(keys[j], (T, 1))
+        o, _, _ = ko.kata_quadratic(q, keys, v)
+        coef = o[T - 1]                 # a_i at the last position
+        expected = np.full(T, p ** -2.0) / (1 + (T - 1) * p ** -2.0)
+        expected[j] = 1.0 / (1 + (T - 1) * p ** -2.0)
+        assert np.allclose(coef, expected, atol=1e-14)
+        psnr = coef[j] ** 2 / np.sum(np.delete(coef, j) ** 2)
+        assert abs(psnr - g["psnr"]) < 1e-9
+        assert abs(psnr - p ** 2 * (T - 1) / (T - p) ** 2) < 1e-9
+
+
+# ---------------------------------------------------------------------------
+# kernel identity and packing
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("d", [1, 2, 3, 16, 64])
+def test_kernel_identity(d):
+    r = rng(d)
+    u = ko.normalize_rows(r.standard_normal((7, d)))
+    w = ko.normalize_rows(r.standard_normal((9, d)))
+    ref = (u @ w.T) ** 2
+    assert np.allclose(ko.psi_direct(u) @ ko.psi_direct(w).T, ref, atol=1e-14)
+    assert np.allclose(ko.psi_packed(u) @ ko.psi_packed(w).T, ref, atol=1e-14)
+    # unit Frobenius norm of the lift
+    assert np.allclose(np.linalg.norm(ko.psi_direct(u), axis=1), 1.0, atol=1e-14)
+    assert np.allclose(np.linalg.norm(ko.psi_packed(u), axis=1), 1.0, atol=1e-14)
+
+
+def test_direct_layout_is_row_major_outer_product():
+    u = np.array([2.0, 3.0, 5.0])
+    f = ko.psi_direct(u)
+    assert f.tolist() == [4, 6, 10, 6, 9, 15, 10, 15, 25]
+    p = ko.psi_packed(u)
+    s = math.sqrt(2.0)
+    assert np.allclose(p, [4, 6 * s, 10 * s, 9, 15 * s, 25])
+
+
+def test_normalize_zero_row():
+    x = np.array([[0.0, 0.0], [3.0, 4.0]])
+    assert ko.normalize_rows(x).tolist() == [[0.0, 0.0], [0.6, 0.8]]
+
+
+# ---------------------------------------------------------------------------
+# the forms agree
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("feature", ["psd_direct", "psd_packed", "identity"])
+@pytest.mark.parametrize("T,d,dv", [(37, 5, 3), (64, 8, 8), (130, 4, 6)])
+def test_forms_agree(feature, T, d, dv):
+    q, k, v = rand_qkv(T * 100 + d, T, d, dv)
+    if feature == "identity":
+        q, k = np.abs(q), np.abs(k)
+    oq, _, _ = ko.kata_quadratic(q, k, v, feature)
+    orr = ko.kata_recurrent(q, k, v, feature)
+    assert np.max(np.abs(oq - orr)) < 1e-10
+    for C in (1, 2, 7, 64, T, T + 5):
+        oc = ko.kata_chunked(q, k, v, C, feature)
+        assert oc.shape == oq.shape
+        assert np.max(np.abs(oq - oc)) < 1e-10, C
+        for prefix in ("running", "doubling"):
+            os_, S_pre, Z_pre = ko.kata_scan(q, k, v, C, feature, prefix)
+            assert np.max(np.abs(oq - os_)) < 1e-10, (C, prefix)
+            assert np.all(S_pre[0] == 0) and np.all(Z_pre[0] == 0)
+    rows = [0, 1, T // 2, T - 1]
+    assert np.max(np.abs(ko.kata_rows(q, k, v, rows, feature) - oq[rows])) < 1e-12
+
+
+def test_config1_forms_agree_full_size():
+    """B=1,H=2,T=512,d=16,C=64 (the tiny config), all forms."""
+    from paper_2607_17419_b200 import inputs
+    w = inputs.config(1)
+    for h in range(w.H):
+        q, k, v = w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h]
+        oq, _, _ = ko.kata_quadratic(q, k, v)
+        assert np.max(np.abs(ko.kata_recurrent(q, k, v, "psd_packed") - oq)) < 1e-10
+        assert np.max(np.abs(ko.kata_chunked(q, k, v, w.C, "psd_direct") - oq)) < 1e-10
+        assert np.max(np.abs(ko.kata_scan(q, k, v, w.C, "psd_packed")[0] - oq)) < 1e-10
+
+
+def test_prefix_two_ways_and_against_cumsum():
+    x = rng(5).standard_normal((37, 6, 2))
+    a = ko.exclusive_prefix_running(x)
+    b, _ = ko.exclusive_prefix_doubling(x)
+    c = np.concatenate([np.zeros((1, 6, 2)), np.cumsum(x, axis=0)[:-1]])
+    assert np.allclose(a, c, atol=1e-12) and np.allclose(b, c, atol=1e-12)
+
+
+def test_scan_states_match_running_state():
+    q, k, v = rand_qkv(11, 50, 4, 3)
+    C = 8
+    _, S_pre, Z_pre = ko.kata_scan(q, k, v, C, "psd_direct")
+    fk = ko.psi_direct(ko.normalize_rows(k))
+    for c in range(S_pre.shape[0]):
+        S = sum((np.outer(fk[i], v[i]) for i in range(c * C)), np.zeros((16, 3)))
+        assert np.allclose(S_pre[c], S, atol=1e-12)
+        assert np.allclose(Z_pre[c], fk[: c * C].sum(axis=0), atol=1e-12)
+
+
+# ---------------------------------------------------------------------------
+# brute force, written independently (scalar loops straight from the sums)
+# ---------------------------------------------------------------------------
+
+def brute(q, k, v):
+    T, d, dv = len(q), len(q[0]), len(v[0])
+    out = [[0.0] * dv for _ in range(T)]
+    for t in range(T):
+        nq = math.sqrt(sum(x * x for x in q[t]))
+        num = [0.0] * dv
+        den = 0.0
+        for i in range(t + 1):
+            nk = math.sqrt(sum(x * x for x in k[i]))
+            if nq == 0 or nk == 0:
+                w = 0.0
+            else:
+                w = (sum(q[t][a] * k[i][a] for a in range(d)) / (nq * nk)) ** 2
+            den += w
+            for j in range(dv):
+                num[j] += w * v[i][j]
+        if den != 0:
+            out[t] = [x / den for x in num]
+    return np.array(out)
+
+
+@pytest.mark.parametrize("T,d,dv", [(1, 1, 1), (5, 2, 3), (8, 3, 2)])
+def test_brute_force_tiny(T, d, dv):
+    q, k, v = rand_qkv(T + 10 * d, T, d, dv)
+    ref = brute(q.tolist(), k.tolist(), v.tolist())
+    for feature in ("psd_direct", "psd_packed"):
+        assert np.allclose(ko.kata_quadratic(q, k, v, feature)[0], ref, atol=1e-13)
+        assert np.allclose(ko.kata_recurrent(q, k, v, feature), ref, atol=1e-13)
+        assert np.allclose(ko.kata_chunked(q, k, v, 3, feature), ref, atol=1e-13)
+        assert np.allclose(ko.kata_scan(q, k, v, 3, feature)[0], ref, atol=1e-13)
+
+
+def test_zero_rows_and_zero_denominator():
+    # first key zero -> D_0 = 0 -> o_0 = 0; orthogonal query/keys -> 0; zero query -> 0
+    k = np.array([[0.0, 0.0], [1.0, 0.0], [1.0, 0.0], [0.0, 2.0]])
+    q = np.array([[1.0, 1.0], [0.0, 1.0], [0.0, 0.0], [1.0, 1.0]])
+    v = np.array([[1.0], [2.0], [4.0], [8.0]])
+    ref = brute(q.tolist(), k.tolist(), v.tolist())
+    assert ref[:3].tolist() == [[0.0], [0.0], [0.0]]
+    assert abs(ref[3, 0] - (0.5 * 2 + 0.5 * 4 + 0.5 * 8) / 1.5) < 1e-15
+    for C in (1, 2, 3, 4):
+        assert np.allclose(ko.kata_chunked(q, k, v, C), ref, atol=1e-15)
+        assert np.allclose(ko.kata_scan(q, k, v, C, "psd_packed")[0], ref, atol=1e-15)
+    assert np.allclose(ko.kata_quadratic(q, k, v)[0], ref, atol=1e-15)
+    assert np.allclose(ko.kata_recurrent(q, k, v), ref, atol=1e-15)
+
+
+# ---------------------------------------------------------------------------
+# textbook reductions and invariances
+# ---------------------------------------------------------------------------
+
+def test_dk1_is_running_mean():
+    T = 40
+    r = rng(7)
+    q, k = r.standard_normal((T, 1)), r.standard_normal((T, 1))
+    v = r.standard_normal((T, 3))
+    mean = np.cumsum(v, axis=0) / np.arange(1, T + 1)[:, None]
+    for o in (ko.kata_quadratic(q, k, v)[0], ko.kata_recurrent(q, k, v), ko.kata_chunked(q, k, v, 8),
+              ko.kata_scan(q, k, v, 8)[0]):
+        assert np.allclose(o, mean, atol=1e-13)
+
+
+def test_orthonormal_keys_exact_retrieval():
+    d = 6
+    k = np.eye(d)
+    v = rng(8).standard_normal((d, 4))
+    for j in range(d):
+        q = np.tile(k[j], (d, 1))
+        o = ko.kata_chunked(q, k, v, 4)
+        for t in range(j, d):
+            assert np.allclose(o[t], v[j], atol=1e-15)
+        assert np.all(o[:j] == 0)          # key j not yet seen: all weights 0 -> D = 0 -> 0
+
+
+def test_first_row_is_first_value_and_constant_values():
+    q, k, v = rand_qkv(9, 30, 5, 4)
+    o, _, _ = ko.kata_quadratic(q, k, v)
+    assert np.allclose(o[0], v[0], atol=1e-15)
+    vc = np.tile(np.array([[1.5, -2.0]]), (30, 1))
+    assert np.allclose(ko.kata_chunked(q, k, vc, 7), vc, atol=1e-13)
+
+
+def test_convex_hull_and_nonnegative_weights():
+    q, k, v = rand_qkv(10, 60, 4, 3)
+    w = ko.causal_weights(q, k)
+    assert np.all(w >= 0) and np.all(np.triu(w, 1) == 0)
+    o = ko.kata_scan(q, k, v, 16)[0]
+    lo = np.minimum.accumulate(v, axis=0)
+    hi = np.maximum.accumulate(v, axis=0)
+    assert np.all(o >= lo - 1e-12) and np.all(o <= hi + 1e-12)
+
+
+def test_invariances():
+    T, d, dv = 33, 6, 4
+    q, k, v = rand_qkv(12, T, d, dv)
+    r = rng(13)
+    base = ko.kata_chunked(q, k, v, 8)
+    cq = r.uniform(0.1, 5.0, (T, 1)) * r.choice([-1.0, 1.0], (T, 1))
+    ck = r.uniform(0.1, 5.0, (T, 1)) * r.choice([-1.0, 1.0], (T, 1))
+    assert np.allclose(ko.kata_chunked(q * cq, k * ck, v, 8), base, atol=1e-12)
+    R, _ = np.linalg.qr(r.standard_normal((d, d)))
+    assert np.allclose(ko.kata_chunked(q @ R, k @ R, v, 8), base, atol=1e-12)
+    A, b = r.standard_normal((dv, 2)), r.standard_normal(2)
+    assert np.allclose(ko.kata_chunked(q, k, v @ A + b, 8), base @ A + b, atol=1e-12)
+
+
+def test_dense_matmul_definition():
+    """tril((Q K^T)^2) V / rowsum with library matmuls on independently normalised rows."""
+    q, k, v = rand_qkv(14, 48, 8, 5)
+    qh = q / np.linalg.norm(q, axis=1, keepdims=True)
+    kh = k / np.linalg.norm(k, axis=1, keepdims=True)
+    W = np.tril(np.square(qh @ kh.T))
+    ref = (W @ v) / W.sum(axis=1, keepdims=True)
+    assert np.allclose(ko.kata_recurrent(q, k, v, "psd_packed"), ref, atol=1e-12)
+    assert np.allclose(ko.kata_chunked(q, k, v, 16), ref, atol=1e-12)
+
+
+def test_identity_feature_is_plain_linear_attention():
+    q, k, v = rand_qkv(15, 40, 6, 3)
+    q, k = np.abs(q), np.abs(k)
+    W = np.tril(q @ k.T)
+    ref = (W @ v) / W.sum(axis=1, keepdims=True)
+    assert np.allclose(ko.kata_scan(q, k, v, 8, "identity")[0], ref, atol=1e-12)
+    S_loc, Z_loc = ko.chunk_local_states(k, v, 8, "identity")
+    assert np.allclose(S_loc[1], k[8:16].T @ v[8:16], atol=1e-13)
+    assert np.allclose(Z_loc[4], k[32:40].sum(axis=0), atol=1e-13)
+
+
+# ---------------------------------------------------------------------------
+# Proposition 1: the normaliser is a convex gate
+# ---------------------------------------------------------------------------
+
+def test_gate_decomposition():
+    q, k, v = rand_qkv(16, 45, 5, 3)
+    k[0] = 0.0                                   # D_0 = 0 and D_1 = c_1 only
+    g = ko.gate_decomposition(q, k, v)
+    o = ko.kata_quadratic(q, k, v)[0]
+    assert np.all(g["alpha"] >= 0) and np.all(g["beta"] >= 0)
+    live = (g["D_prev"] + g["c"]) > 0
+    assert np.allclose((g["alpha"] + g["beta"])[live], 1.0, atol=1e-14)
+    assert np.allclose(g["o"], o, atol=1e-12)
+    assert g["alpha"][1] == 0.0 and g["beta"][1] == 1.0 and np.allclose(o[1], v[1])
+    assert np.all(o[0] == 0)
+    # D_{t-1} uses the *current* query against the previous state
+    w = ko.causal_weights(q, k)
+    assert np.allclose(g["D_prev"], w.sum(axis=1) - np.diag(w), atol=1e-13)
+    assert np.allclose(g["c"], np.diag(w), atol=1e-15)
+
+
+def test_batched_wrapper():
+    r = rng(17)
+    q, k = r.standard_normal((2, 3, 20, 4)), r.standard_normal((2, 3, 20, 4))
+    v = r.standard_normal((2, 3, 20, 5))
+    ob = ko.batched(ko.kata_chunked, q, k, v, 8)
+    for b, h in itertools.product(range(2), range(3)):
+        assert np.array_equal(ob[b, h], ko.kata_chunked(q[b, h], k[b, h], v[b, h], 8))
+    ob2 = ko.batched(ko.kata_quadratic, q, k, v)
+    assert np.allclose(ob, ob2, atol=1e-12)
