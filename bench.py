@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the KATA chunked forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one ``kata_fwd_chunked`` call (rows a0-a6 of the hot path: normalise, feature
+products, state update, inter-chunk read, intra-chunk scores and apply, gate/normalise epilogue)
+on the long-context workload B=1, H=16, T=131072, d_k=d_v=64, C=64, bf16, q,k,v iid N(0,1) from
+seed 3.  The metric is tokens/s (B*T per step).  With N > 1 every rank runs its own copy of the
+workload (heads and batches are independent, no collective in the data path): weak scaling.
+
+The JSON line also carries: ``roofline`` for the dominant kernel, ``e2e`` (the same call through
+``kata_fwd_host`` with pinned host buffers, copies inside the timed region), ``cpu_baseline`` (the
+fp64 oracle timed on a bounded sample on the host cores), ``clocks`` sampled during the timed
+region, and ``extra`` with separately timed figures for the quadratic form and the scan forms.
+
+``--impl reference`` times the oracle itself (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "kata_chunked_fwd_tokens_per_s_T131072_d64"
+UNIT = "tokens/s"
+WORKLOAD = dict(B=1, H=16, T=131072, d_k=64, d_v=64, C=64)
+
+# Algorithmic work per (b,h,t) of the chunked form with the packed symmetric feature
+# n = d(d+1)/2 = 2080: state update 2*n*d_v + inter-chunk read 2*n*d_v + intra-chunk
+# (C+1)/2 * 2*(d + d_v) + normaliser via the d x d Gram 3*d^2.
+def chunked_flops_per_head_token(d=64, dv=64, C=64):
+    n = d * (d + 1) // 2
+    return 4 * n * dv + (C + 1) * (d + dv) + 3 * d * d
+
+
+def quadratic_flops(B, H, T, d=64, dv=64):
+    return B * H * (T * (T + 1) // 2) * (2 * d + 2 * dv)
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons in the background."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+def time_oracle_sample(heads: int = 1, tokens: int = 8192):
+    """The fp64 oracle's chunked form on `heads` heads x `tokens` tokens of the benchmark workload."""
+    import numpy as np
+    from oracle import kata_oracle as ko
+    from paper_2607_17419_b200 import inputs
+    w = inputs.gaussian_workload("cpu_sample", "bf16", 1, heads, tokens, 64, 64, 64, 3)
+    t0 = time.perf_counter()
+    for h in range(heads):
+        o = ko.kata_chunked(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h], 64, "psd_direct")
+    dt = time.perf_counter() - t0
+    assert np.all(np.isfinite(o))
+    # whole-job tokens/s: a token counts once its H heads are done
+    per_head_token = dt / (heads * tokens)
+    return 1.0 / (per_head_token * WORKLOAD["H"]), dt
+
+
+def host_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy  # noqa: F401  (loads BLAS so that host_threads sees it)
+    heads, tokens = 1, 4096
+    for _ in range(args.warmup):
+        time_oracle_sample(heads, 1024)
+    times, vals = [], []
+    for _ in range(args.steps):
+        v, dt = time_oracle_sample(heads, tokens)
+        times.append(dt)
+        vals.append(v)
+    value = statistics.mean(vals)
+    ms = 1e3 * statistics.mean(times)
+    sample = (f"fp64 numpy oracle, Algorithm-1 chunked form (direct d^2 feature), {heads} head x {tokens} tokens "
+              f"of the workload per step; tokens/s extrapolated to H={WORKLOAD['H']} heads (linear in T and H)")
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic",
+                config=dict(workload="c4 long-context chunked forward B=1 H=16 T=131072 d_k=d_v=64 C=64 bf16 inputs",
+                            **WORKLOAD),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=host_threads(), kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_17419_b200 import binding as kb
+    from paper_2607_17419_b200 import build as kbuild
+    from paper_2607_17419_b200 import inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        kbuild.build()
+    if world > 1:
+        dist.barrier()
+    kb.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    W = WORKLOAD
+    w = inputs.gaussian_workload("c4_long_bf16", "bf16", W["B"], W["H"], W["T"], W["d_k"], W["d_v"], W["C"], 3)
+
+    def tt(a):
+        return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    hq, hk, hv = (tt(a).pin_memory() for a in (w.q_dev, w.k_dev, w.v_dev))
+    ho = torch.empty_like(hv).pin_memory()
+    q, k, v = hq.to(dev), hk.to(dev), hv.to(dev)
+    out = torch.empty_like(v)
+    stream = torch.cuda.current_stream(dev)
+    inter = kb.KATA_SCAN if args.mode == "scan" else kb.KATA_SEQUENTIAL
+
+    def step():
+        kb.kata_fwd_chunked(q, k, v, out, inter_chunk=inter)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    launches_per_step = kb.kata_last_launch_count()
+    impl = "tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt"
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end: pinned host buffers through kata_fwd_host, copies inside the timed region ----
+    ws = kb.Workspace()
+    for _ in range(2):
+        kb.kata_fwd_host(kb.KATA_FN_CHUNKED, hq, hk, hv, ho, inter_chunk=inter, workspace=ws)
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(2, min(args.steps, 5))
+    f0.record(stream)
+    for _ in range(e2e_steps):
+        kb.kata_fwd_host(kb.KATA_FN_CHUNKED, hq, hk, hv, ho, inter_chunk=inter, workspace=ws)
+        stream.synchronize()          # the caller reads the result of each step
+    f1.record(stream)
+    barrier()
+    e2e_ms_total = f0.elapsed_time(f1)
+    assert torch.equal(ho.to(dev), out)
+
+    t = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms_total = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peaks = load_peaks()
+        tokens = W["B"] * W["T"]
+        ms_step = ms_total / args.steps
+        value = world * tokens / (ms_step * 1e-3)
+        e2e_value = world * tokens / (e2e_ms_total / e2e_steps * 1e-3)
+        flops = chunked_flops_per_head_token() * W["B"] * W["H"] * W["T"]
+        achieved = flops / (ms_step * 1e-3) / 1e12
+        if impl == "tensor":
+            sustained = ms_total > 1000.0
+            peak = peaks["bf16_sustained"] if sustained else peaks["bf16_burst"]
+            roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
+                        traffic=None, kernel="kata chunked forward (tcgen05)",
+                        note=f"algorithmic flops (packed feature n=2080) / CUDA-event time; peak = "
+                             f"{'sustained' if sustained else 'burst'} bf16 cuBLAS of {peaks['source']}")
+        else:
+            alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12      # SMs x fp32 lanes x FMA x max clock
+            roof = dict(bound="alu", achieved=achieved, peak=alu_peak, unit="TFLOP/s", frac=achieved / alu_peak,
+                        traffic=None, kernel="chunk_simt_kernel (fp32 FMA path)",
+                        note="algorithmic flops / CUDA-event time; peak = 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz")
+        extra = measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks) if args.extra else None
+        cpu_val, cpu_dt = time_oracle_sample(1, 8192)
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+                    ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                    data="synthetic",
+                    config=dict(workload="c4 long-context chunked forward B=1 H=16 T=131072 d_k=d_v=64 C=64 bf16 "
+                                         "(per GPU; q,k,v iid N(0,1), seed 3)",
+                                inter_chunk=args.mode, impl=impl, l2="inputs (805 MB) larger than L2", **W),
+                    e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=int(3 * q.numel() * 2),
+                             d2h_bytes_per_step=int(out.numel() * 2), ms_per_step=e2e_ms_total / e2e_steps),
+                    gpu_launches=int(launches_per_step * args.steps),
+                    roofline=roof,
+                    cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=host_threads(), kind="oracle",
+                                      sample=f"fp64 numpy oracle, Algorithm-1 chunked form, 1 head x 8192 tokens "
+                                             f"({cpu_dt:.1f} s), extrapolated linearly to H=16"),
+                    clocks=clocks, extra=extra)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
+    """Separately timed secondary figures: scan forms on the same workload, quadratic form on config 2."""
+    import numpy as np
+    import torch
+
+    def timed(fn, reps=5, warm=2):
+        for _ in range(warm):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    res = {}
+    T = q.shape[2]
+    for name, fn in (("chunked_seq", lambda: kb.kata_fwd_chunked(q, k, v, out, inter_chunk=kb.KATA_SEQUENTIAL)),
+                     ("chunked_scan", lambda: kb.kata_fwd_chunked(q, k, v, out, inter_chunk=kb.KATA_SCAN)),
+                     ("chunk_state_scan", lambda: kb.kata_chunk_state_scan(q, k, v, out))):
+        ms = timed(fn)
+        res[name] = dict(ms=ms, tokens_per_s=T / (ms * 1e-3), launches=kb.kata_last_launch_count())
+    w2 = inputs.config(2)
+    q2, k2, v2 = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).to(dev) for a in (w2.q_dev, w2.k_dev, w2.v_dev))
+    o2 = torch.empty_like(v2)
+    ms = timed(lambda: kb.kata_fwd_quadratic(q2, k2, v2, o2))
+    fl = quadratic_flops(w2.B, w2.H, w2.T)
+    res["quadratic_c2"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=fl / (ms * 1e-3) / 1e12,
+                               frac_of_bf16_burst=fl / (ms * 1e-3) / 1e12 / peaks["bf16_burst"],
+                               impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="sequential", choices=["sequential", "scan"])
+    ap.add_argument("--no-extra", dest="extra", action="store_false")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

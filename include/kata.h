@@ -1,0 +1,176 @@
+/*
+ * kata.h -- C ABI of the KATA forward pass for NVIDIA B200 (sm_100a).
+ *
+ * KATA is causal linear attention whose feature map is the rank-one PSD lift of the
+ * l2-normalised query/key, psi(u) = u_hat u_hat^T, so that the attention weight is
+ * <psi(q_t), psi(k_i)> = (q_hat_t . k_hat_i)^2, with the normalised readout
+ *
+ *     o_t = sum_{i<=t} w_ti v_i / sum_{i<=t} w_ti            (paper Eq. (2), "linearized form")
+ *
+ * whose denominator acts as the parameter-free convex output gate of Proposition 1
+ * ("Output-level gating").  o_t = 0 where the denominator is 0.  There is no temperature,
+ * no epsilon in the normalisation (a zero row has a zero feature) and the causal mask
+ * includes the diagonal.
+ *
+ * Problem statement (Algorithm 1, Require/Return): per head Q,K in R^{T x d_k},
+ * V in R^{T x d_v}, chunk size C; returns O in R^{T x d_v}.  Batch and heads are independent.
+ *
+ * Conventions common to every entry point
+ *   - q, k: [B,H,T,d_k]; v, out: [B,H,T,d_v]; row-major, contiguous, 16-byte aligned,
+ *     DEVICE pointers (except in kata_fwd_host), element type opts->dtype (fp32 or bf16).
+ *   - All accumulation, the running state (S,Z) and the normaliser are fp32; out is rounded
+ *     to the element type (round-to-nearest-even).
+ *   - The caller owns every buffer.  The library allocates nothing, frees nothing and never
+ *     synchronises; all work is enqueued on opts->stream.  q,k,v are read-only; out and the
+ *     workspace are fully overwritten (no pre-zeroing needed).
+ *   - Supported shapes: d_k, d_v in {16,32,64}; C = 64 (the chunked/scan forms); T >= 1
+ *     (any; the last chunk is zero-padded as in Algorithm 1 and truncated on output);
+ *     B,H >= 1.  The tensor-core (tcgen05) kernels cover bf16 with d_k = d_v = 64; everything
+ *     else runs on the fp32 SIMT kernels.
+ *   - Return value: KATA_OK (0) or a negative kata_status.  Errors detectable on the host
+ *     launch nothing.  No exceptions, no abort, no device trap.  A bounded device-side wait
+ *     that expires writes KATA_ERR_DEVICE_TIMEOUT to *opts->device_status (if non-null),
+ *     visible after the caller synchronises the stream; the kernel still terminates.
+ */
+#ifndef KATA_H_
+#define KATA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KATA_VERSION 100
+
+typedef enum kata_status {
+  KATA_OK = 0,
+  KATA_ERR_INVALID_ARG = -1,        /* null pointer, non-positive size, bad enum, bad struct_size */
+  KATA_ERR_UNSUPPORTED_SHAPE = -2,  /* d_k/d_v/C outside the supported set                        */
+  KATA_ERR_ALIGNMENT = -3,          /* a tensor or workspace pointer is not 16-byte aligned        */
+  KATA_ERR_WORKSPACE_TOO_SMALL = -4,
+  KATA_ERR_ARCH = -5,               /* current device is not compute capability 10.x              */
+  KATA_ERR_CUDA = -6,               /* a CUDA runtime call or a launch failed                      */
+  KATA_ERR_DEVICE_TIMEOUT = -7      /* only ever written to *device_status                         */
+} kata_status;
+
+enum { KATA_F32 = 0, KATA_BF16 = 1 };                 /* kata_opts.dtype          */
+enum { KATA_LAYOUT_DIRECT = 0, KATA_LAYOUT_PACKED = 1 }; /* kata_opts.state_layout */
+enum { KATA_SEQUENTIAL = 0, KATA_SCAN = 1 };          /* kata_opts.inter_chunk    */
+enum { KATA_IMPL_AUTO = 0, KATA_IMPL_SIMT = 1, KATA_IMPL_TENSOR = 2 }; /* kata_opts.impl */
+enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2 };
+
+/*
+ * Options (plain data; zero-initialise, then set struct_size = sizeof(kata_opts)).
+ *
+ *  dtype          element type of q,k,v,out.
+ *  feature_order  2: rank-one PSD lift of the normalised rows (default when 0 is passed).
+ *                 1: rows of q,k are already-mapped features used as they are (no
+ *                    normalisation, no lift; state d_k x d_v) -- the setting of the paper's
+ *                    associative-scan appendix ("already-feature-mapped inputs").
+ *  state_layout   layout of the exported prefix states for feature_order 2:
+ *                 DIRECT  n_psi = d_k^2, row a*d_k+b holds the (a,b) entry of sum k_hat k_hat^T (x) v;
+ *                 PACKED  n_psi = d_k(d_k+1)/2, upper triangle a<=b in row-major order, diagonal
+ *                         entries as they are and off-diagonal entries times sqrt(2) (the isometric
+ *                         packing, so packed features keep the inner product (q_hat.k_hat)^2).
+ *                 Ignored for feature_order 1 (n_psi = d_k).
+ *  inter_chunk    kata_fwd_chunked only: SEQUENTIAL walks the chunks of a head in order
+ *                 (Algorithm 1); SCAN splits the chunk axis into groups, reduces each group,
+ *                 runs a log-depth exclusive scan over the group states and finishes every
+ *                 group in parallel (section "Tree-scan inter-chunk reduction").
+ *  impl           AUTO picks the tensor-core kernels where they exist; SIMT / TENSOR force one
+ *                 (TENSOR returns KATA_ERR_UNSUPPORTED_SHAPE where it does not exist).
+ *  scan_group     chunks per scan group; 0 = library's choice (kata_chunk_state_scan: 1, i.e.
+ *                 the paper's per-chunk pipeline, whenever s_pre/z_pre are requested).
+ *  workspace      device scratch of at least kata_workspace_bytes(...) bytes, 256-byte aligned;
+ *                 may be null when that size is 0.
+ *  s_pre, z_pre   optional device outputs of kata_chunk_state_scan (fp32):
+ *                 s_pre [B,H,N_C,n_psi,d_v], z_pre [B,H,N_C,n_psi], N_C = ceil(T/C), the exclusive
+ *                 prefix chunk states, entry 0 along N_C being zero.  Both null or both non-null.
+ *  device_status  optional device int, written only on a device-side timeout.
+ *  stream         cudaStream_t as void* (null = the legacy default stream).
+ */
+typedef struct kata_opts {
+  uint32_t struct_size;
+  int32_t dtype;
+  int32_t feature_order;
+  int32_t state_layout;
+  int32_t inter_chunk;
+  int32_t impl;
+  int32_t scan_group;
+  int32_t reserved0;
+  void* workspace;
+  size_t workspace_bytes;
+  float* s_pre;
+  float* z_pre;
+  int* device_status;
+  void* stream;
+} kata_opts;
+
+/*
+ * Quadratic ("flash-style") forward: the definition evaluated tile by tile, never forming
+ * the d_k^2-wide state (section "Why the PSD feature keeps to O(T) or O(T^2)"; weights from
+ * the rank-one lift identity <uu^T,vv^T>_F = (u^T v)^2).  O(T^2) work.  C is ignored.
+ * Needs no workspace.
+ */
+int kata_fwd_quadratic(const void* q, const void* k, const void* v, void* out,
+                       int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
+
+/*
+ * Chunked-state forward: Algorithm 1 with the chunk equations
+ *   S_[c+1] = S_[c] + Psi(K_[c])^T V_[c],  Z_[c+1] = Z_[c] + Psi(K_[c])^T 1,
+ *   P = (Psi(Q_[c]) Psi(K_[c])^T) o M,  N = Psi(Q_[c]) S_[c] + P V_[c],
+ *   D = Psi(Q_[c]) Z_[c] + P 1,  O_[c] = diag(D)^-1 N
+ * (section "Chunkwise forward").  O(T) work, fp32 state.  opts->inter_chunk selects how
+ * the inter-chunk recurrence is traversed; both give the same result up to fp32
+ * re-association.  Workspace: kata_workspace_bytes(KATA_FN_CHUNKED, ...).
+ */
+int kata_fwd_chunked(const void* q, const void* k, const void* v, void* out,
+                     int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
+
+/*
+ * Three-stage pipeline of the appendix "Associative-scan kernel": (i) chunk-local states
+ * S_loc = Psi(K_[c])^T V_[c], Z_loc = 1^T Psi(K_[c]) for all (b,h,c) in parallel; (ii) exclusive
+ * prefix along the chunk axis in ceil(log2 N) rounds; (iii) chunk output from the prefix and
+ * the local C x C causal term.  Writes out; if opts->s_pre/z_pre are set it also writes the
+ * exclusive-prefix chunk states there (which forces scan_group = 1).
+ * Workspace: kata_workspace_bytes(KATA_FN_CHUNK_STATE_SCAN, ...).
+ */
+int kata_chunk_state_scan(const void* q, const void* k, const void* v, void* out,
+                          int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
+
+/*
+ * Same computation as entry point `fn` (a KATA_FN_* value) but q,k,v,out are HOST pointers
+ * (pinned memory recommended).  The inputs are copied to a staging area inside the workspace,
+ * the kernels run, and out is copied back, all enqueued on opts->stream; the caller synchronises
+ * the stream before reading out.  Workspace: kata_workspace_bytes(fn | KATA_FN_HOST_IO, ...).
+ * The paper has no counterpart; this is the end-to-end path measured by the benchmark.
+ */
+#define KATA_FN_HOST_IO 0x100
+int kata_fwd_host(int fn, const void* q_host, const void* k_host, const void* v_host, void* out_host,
+                  int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
+
+/*
+ * Bytes of device workspace entry point `fn` needs for these sizes and options (0 if none);
+ * returns 0 also for invalid arguments (the entry point itself reports the error).
+ */
+size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
+
+/* Number of scan groups / chunks per group the library would use (for reporting and tests). */
+int kata_scan_plan(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts,
+                   int* n_groups, int* chunks_per_group, int* scan_rounds);
+
+/* Number of kernels the last successful call on this host thread enqueued. */
+int kata_last_launch_count(void);
+
+/* Which kernels the last successful call on this host thread used: KATA_IMPL_SIMT or KATA_IMPL_TENSOR. */
+int kata_last_impl(void);
+
+const char* kata_status_string(int status);
+int kata_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KATA_H_ */

@@ -1,0 +1,217 @@
+"""Thin ctypes binding over libkata.so (argument marshalling only; every step runs in the CUDA
+library).  Function names mirror the C ABI of include/kata.h.
+
+Tensors are torch CUDA tensors (or pinned host tensors for ``kata_fwd_host``); torch is used for
+device memory and streams only.  There is no CPU fallback: if the library is missing or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libkata.so")
+
+KATA_F32, KATA_BF16 = 0, 1
+KATA_LAYOUT_DIRECT, KATA_LAYOUT_PACKED = 0, 1
+KATA_SEQUENTIAL, KATA_SCAN = 0, 1
+KATA_IMPL_AUTO, KATA_IMPL_SIMT, KATA_IMPL_TENSOR = 0, 1, 2
+KATA_FN_QUADRATIC, KATA_FN_CHUNKED, KATA_FN_CHUNK_STATE_SCAN = 0, 1, 2
+KATA_FN_HOST_IO = 0x100
+
+EXPORTS = ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan", "kata_fwd_host",
+           "kata_workspace_bytes", "kata_scan_plan", "kata_last_launch_count", "kata_last_impl",
+           "kata_status_string",
+           "kata_version")
+
+
+class KataOpts(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("dtype", ctypes.c_int32),
+        ("feature_order", ctypes.c_int32),
+        ("state_layout", ctypes.c_int32),
+        ("inter_chunk", ctypes.c_int32),
+        ("impl", ctypes.c_int32),
+        ("scan_group", ctypes.c_int32),
+        ("reserved0", ctypes.c_int32),
+        ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t),
+        ("s_pre", ctypes.c_void_p),
+        ("z_pre", ctypes.c_void_p),
+        ("device_status", ctypes.c_void_p),
+        ("stream", ctypes.c_void_p),
+    ]
+
+
+class KataError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libkata.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2607_17419_b200.build`")
+    L = ctypes.CDLL(LIB_PATH)
+    ptr, i = ctypes.c_void_p, ctypes.c_int
+    fwd_args = [ptr, ptr, ptr, ptr, i, i, i, i, i, i, ctypes.POINTER(KataOpts)]
+    for name in ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan"):
+        getattr(L, name).argtypes = fwd_args
+        getattr(L, name).restype = i
+    L.kata_fwd_host.argtypes = [i] + fwd_args
+    L.kata_fwd_host.restype = i
+    L.kata_workspace_bytes.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(KataOpts)]
+    L.kata_workspace_bytes.restype = ctypes.c_size_t
+    L.kata_scan_plan.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(KataOpts)] + [ctypes.POINTER(i)] * 3
+    L.kata_scan_plan.restype = i
+    L.kata_last_launch_count.argtypes = []
+    L.kata_last_launch_count.restype = i
+    L.kata_last_impl.argtypes = []
+    L.kata_last_impl.restype = i
+    L.kata_status_string.argtypes = [i]
+    L.kata_status_string.restype = ctypes.c_char_p
+    L.kata_version.argtypes = []
+    L.kata_version.restype = i
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().kata_status_string(status).decode()
+
+
+def make_opts(dtype: int, *, feature_order: int = 2, state_layout: int = KATA_LAYOUT_DIRECT,
+              inter_chunk: int = KATA_SEQUENTIAL, impl: int = KATA_IMPL_AUTO, scan_group: int = 0,
+              workspace: int = 0, workspace_bytes: int = 0, s_pre: int = 0, z_pre: int = 0,
+              device_status: int = 0, stream: int = 0) -> KataOpts:
+    o = KataOpts()
+    o.struct_size = ctypes.sizeof(KataOpts)
+    o.dtype, o.feature_order, o.state_layout = dtype, feature_order, state_layout
+    o.inter_chunk, o.impl, o.scan_group = inter_chunk, impl, scan_group
+    o.workspace, o.workspace_bytes = workspace or None, workspace_bytes
+    o.s_pre, o.z_pre = s_pre or None, z_pre or None
+    o.device_status, o.stream = device_status or None, stream or None
+    return o
+
+
+def kata_workspace_bytes(fn: int, B, H, T, d_k, d_v, C, opts: KataOpts) -> int:
+    return int(lib().kata_workspace_bytes(fn, B, H, T, d_k, d_v, C, ctypes.byref(opts)))
+
+
+def kata_scan_plan(fn: int, B, H, T, d_k, d_v, C, opts: KataOpts):
+    """(n_groups, chunks_per_group, scan_rounds) the library would use."""
+    a, b, c = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    st = lib().kata_scan_plan(fn, B, H, T, d_k, d_v, C, ctypes.byref(opts), ctypes.byref(a), ctypes.byref(b),
+                              ctypes.byref(c))
+    if st != 0:
+        raise KataError(st, "kata_scan_plan")
+    return a.value, b.value, c.value
+
+
+def kata_last_launch_count() -> int:
+    return int(lib().kata_last_launch_count())
+
+
+def kata_last_impl() -> int:
+    return int(lib().kata_last_impl())
+
+
+def kata_version() -> int:
+    return int(lib().kata_version())
+
+
+# ---------------------------------------------------------------------------
+# tensor-level wrappers
+# ---------------------------------------------------------------------------
+
+_FN_NAMES = {KATA_FN_QUADRATIC: "kata_fwd_quadratic", KATA_FN_CHUNKED: "kata_fwd_chunked",
+             KATA_FN_CHUNK_STATE_SCAN: "kata_chunk_state_scan"}
+
+
+def _dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.float32:
+        return KATA_F32
+    if t.dtype == torch.bfloat16:
+        return KATA_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+class Workspace:
+    """A reusable device scratch buffer (torch allocation, grown on demand)."""
+
+    def __init__(self):
+        self.buf = None
+
+    def get(self, nbytes: int, device):
+        import torch
+        if nbytes == 0:
+            return 0, 0
+        if self.buf is None or self.buf.numel() < nbytes or self.buf.device != device:
+            self.buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        return self.buf.data_ptr(), self.buf.numel()
+
+
+_default_ws = Workspace()
+
+
+def _call(fn: int, q, k, v, out, C: int, *, host_io: bool = False, workspace: Optional[Workspace] = None,
+          s_pre=None, z_pre=None, device_status=None, stream=None, **opt_kw):
+    import torch
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+        raise ValueError("q, k, v must be contiguous [B,H,T,d]")
+    B, H, T, d_k = q.shape
+    d_v = v.shape[-1]
+    if out is None:
+        out = torch.empty_like(v)
+    dev = torch.device("cuda", torch.cuda.current_device()) if host_io else q.device
+    if stream is None:
+        stream = torch.cuda.current_stream(dev).cuda_stream
+    opts = make_opts(_dtype_code(q), stream=stream,
+                     s_pre=s_pre.data_ptr() if s_pre is not None else 0,
+                     z_pre=z_pre.data_ptr() if z_pre is not None else 0,
+                     device_status=device_status.data_ptr() if device_status is not None else 0, **opt_kw)
+    need = kata_workspace_bytes(fn | (KATA_FN_HOST_IO if host_io else 0), B, H, T, d_k, d_v, C, opts)
+    ws = workspace if workspace is not None else _default_ws
+    ptr, size = ws.get(need, dev)
+    opts.workspace, opts.workspace_bytes = ptr or None, size
+    args = (q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), B, H, T, d_k, d_v, C, ctypes.byref(opts))
+    if host_io:
+        st = lib().kata_fwd_host(fn, *args)
+        name = "kata_fwd_host"
+    else:
+        name = _FN_NAMES[fn]
+        st = getattr(lib(), name)(*args)
+    if st != 0:
+        raise KataError(st, name)
+    return out
+
+
+def kata_fwd_quadratic(q, k, v, out=None, C: int = 64, **kw):
+    """Quadratic forward; q,k [B,H,T,d_k], v [B,H,T,d_v] CUDA tensors (fp32 or bf16)."""
+    return _call(KATA_FN_QUADRATIC, q, k, v, out, C, **kw)
+
+
+def kata_fwd_chunked(q, k, v, out=None, C: int = 64, **kw):
+    """Chunked-state forward; inter_chunk=KATA_SEQUENTIAL (default) or KATA_SCAN."""
+    return _call(KATA_FN_CHUNKED, q, k, v, out, C, **kw)
+
+
+def kata_chunk_state_scan(q, k, v, out=None, C: int = 64, **kw):
+    """Chunk-state -> log-depth scan -> chunk-output pipeline; optional s_pre/z_pre export."""
+    return _call(KATA_FN_CHUNK_STATE_SCAN, q, k, v, out, C, **kw)
+
+
+def kata_fwd_host(fn: int, q, k, v, out, C: int = 64, **kw):
+    """Same as entry point ``fn`` with (pinned) host tensors; copies ride the current CUDA stream."""
+    return _call(fn, q, k, v, out, C, host_io=True, **kw)

@@ -1,0 +1,329 @@
+// C ABI of the KATA forward library: argument validation, scan planning, workspace carve-up and
+// dispatch to the SIMT (fp32) or tensor-core (tcgen05) kernels.  Declarations and the contract of
+// every entry point are in include/kata.h.
+#include <cstring>
+
+#include "kata_common.cuh"
+
+namespace kata {
+namespace {
+
+thread_local int g_last_launches = 0;
+thread_local int g_last_impl = KATA_IMPL_SIMT;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool dim_ok(int d) { return d == 16 || d == 32 || d == 64; }
+inline int ceil_log2(int n) {
+  int r = 0;
+  while ((1 << r) < n) ++r;
+  return r;
+}
+
+struct Opts {
+  int dtype, feature_order, state_layout, inter_chunk, impl, scan_group;
+  void* workspace;
+  size_t workspace_bytes;
+  float* s_pre;
+  float* z_pre;
+  int* device_status;
+  cudaStream_t stream;
+};
+
+int read_opts(const kata_opts* o, Opts& out) {
+  if (o == nullptr || o->struct_size != sizeof(kata_opts)) return KATA_ERR_INVALID_ARG;
+  out.dtype = o->dtype;
+  out.feature_order = o->feature_order == 0 ? 2 : o->feature_order;
+  out.state_layout = o->state_layout;
+  out.inter_chunk = o->inter_chunk;
+  out.impl = o->impl;
+  out.scan_group = o->scan_group;
+  out.workspace = o->workspace;
+  out.workspace_bytes = o->workspace_bytes;
+  out.s_pre = o->s_pre;
+  out.z_pre = o->z_pre;
+  out.device_status = o->device_status;
+  out.stream = static_cast<cudaStream_t>(o->stream);
+  if (out.dtype != KATA_F32 && out.dtype != KATA_BF16) return KATA_ERR_INVALID_ARG;
+  if (out.feature_order != 1 && out.feature_order != 2) return KATA_ERR_INVALID_ARG;
+  if (out.state_layout != KATA_LAYOUT_DIRECT && out.state_layout != KATA_LAYOUT_PACKED) return KATA_ERR_INVALID_ARG;
+  if (out.inter_chunk != KATA_SEQUENTIAL && out.inter_chunk != KATA_SCAN) return KATA_ERR_INVALID_ARG;
+  if (out.impl < KATA_IMPL_AUTO || out.impl > KATA_IMPL_TENSOR) return KATA_ERR_INVALID_ARG;
+  if (out.scan_group < 0) return KATA_ERR_INVALID_ARG;
+  if ((out.s_pre == nullptr) != (out.z_pre == nullptr)) return KATA_ERR_INVALID_ARG;
+  return KATA_OK;
+}
+
+int check_shape(int fn, int B, int H, int T, int d_k, int d_v, int C) {
+  if (fn < KATA_FN_QUADRATIC || fn > KATA_FN_CHUNK_STATE_SCAN) return KATA_ERR_INVALID_ARG;
+  if (B < 1 || H < 1 || T < 1 || d_k < 1 || d_v < 1) return KATA_ERR_INVALID_ARG;
+  if ((long long)B * H > 65535) return KATA_ERR_UNSUPPORTED_SHAPE;
+  if (!dim_ok(d_k) || !dim_ok(d_v)) return KATA_ERR_UNSUPPORTED_SHAPE;
+  if (fn != KATA_FN_QUADRATIC) {
+    if (C < 1) return KATA_ERR_INVALID_ARG;
+    if (C != kChunk) return KATA_ERR_UNSUPPORTED_SHAPE;
+  }
+  return KATA_OK;
+}
+
+bool want_tensor(const Problem& p, const Opts& o) {
+  return o.impl != KATA_IMPL_SIMT && tc_supported(p);
+}
+
+// How the chunk axis is cut into scan groups, and how many floats one group state takes.
+int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, ScanPlan& plan, size_t& state_elems) {
+  plan.n_chunks = (p.T + kChunk - 1) / kChunk;
+  const int NC = plan.n_chunks;
+  const int BH = p.B * p.H;
+  int slices;
+  if (tensor) {
+    state_elems = tc_chunked_state_elems();
+    slices = tc_chunked_slices();
+  } else if (p.feature_order == 1) {
+    state_elems = order1_state_elems(p.d_k, p.d_v);
+    slices = 1;
+  } else {
+    state_elems = simt_chunked_state_elems(p.d_k, p.d_v);
+    slices = simt_chunked_slices(p.d_k, p.d_v);
+  }
+  int G;
+  if (fn == KATA_FN_CHUNKED) {
+    if (o.inter_chunk == KATA_SEQUENTIAL) {
+      G = NC;
+    } else if (o.scan_group > 0) {
+      G = o.scan_group < NC ? o.scan_group : NC;
+    } else {
+      // enough groups for about two CTAs per SM, at least two groups
+      int ng = (2 * 148 + slices * BH - 1) / (slices * BH);
+      if (ng < 2) ng = 2;
+      if (ng > NC) ng = NC;
+      G = (NC + ng - 1) / ng;
+    }
+  } else {
+    if (o.s_pre != nullptr && o.scan_group > 1) return KATA_ERR_INVALID_ARG;
+    if (o.s_pre != nullptr) {
+      G = 1;
+    } else if (o.scan_group > 0) {
+      G = o.scan_group < NC ? o.scan_group : NC;
+    } else {
+      // the paper's per-chunk pipeline while the two state buffers stay below 2 GiB
+      const double cap = 2.0 * 1024 * 1024 * 1024;
+      G = 1;
+      while (G < NC && 2.0 * BH * ((NC + G - 1) / G) * (double)state_elems * 4.0 > cap) G *= 2;
+      if (G > NC) G = NC;
+    }
+  }
+  plan.chunks_per_group = G;
+  plan.n_groups = (NC + G - 1) / G;
+  plan.rounds = plan.n_groups > 2 ? ceil_log2(plan.n_groups - 1) : 0;
+  return KATA_OK;
+}
+
+size_t inner_workspace(int fn, const ScanPlan& plan, const Problem& p, size_t state_elems) {
+  if (fn == KATA_FN_QUADRATIC) return 0;
+  if (fn == KATA_FN_CHUNKED && plan.n_groups == 1) return 0;
+  return 2 * align_up((size_t)p.B * p.H * plan.n_groups * state_elems * sizeof(float));
+}
+
+size_t elem_bytes(int dtype) { return dtype == KATA_F32 ? 4 : 2; }
+
+struct Staging {
+  size_t q, k, v, out, inner, total;
+};
+
+Staging staging_layout(const Problem& p, size_t inner_bytes) {
+  const size_t eb = elem_bytes(p.dtype);
+  const size_t nqk = (size_t)p.B * p.H * p.T * p.d_k * eb;
+  const size_t nv = (size_t)p.B * p.H * p.T * p.d_v * eb;
+  Staging s;
+  s.q = 0;
+  s.k = s.q + align_up(nqk);
+  s.v = s.k + align_up(nqk);
+  s.out = s.v + align_up(nv);
+  s.inner = s.out + align_up(nv);
+  s.total = s.inner + inner_bytes;
+  return s;
+}
+
+int check_arch() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return KATA_ERR_CUDA;
+  }
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return KATA_ERR_CUDA;
+  }
+  return major == 10 ? KATA_OK : KATA_ERR_ARCH;
+}
+
+// Validation shared by every entry point; fills the problem, the plan and the workspace need.
+struct Prepared {
+  Problem p;
+  Opts o;
+  ScanPlan plan;
+  size_t state_elems;
+  size_t inner_bytes;
+  bool tensor;
+};
+
+int prepare(int fn, const void* q, const void* k, const void* v, void* out, int B, int H, int T, int d_k,
+            int d_v, int C, const kata_opts* opts, bool need_ptrs, Prepared& r) {
+  int st = read_opts(opts, r.o);
+  if (st != KATA_OK) return st;
+  st = check_shape(fn, B, H, T, d_k, d_v, C);
+  if (st != KATA_OK) return st;
+  if (need_ptrs && (q == nullptr || k == nullptr || v == nullptr || out == nullptr)) return KATA_ERR_INVALID_ARG;
+  if (fn != KATA_FN_CHUNK_STATE_SCAN && r.o.s_pre != nullptr) return KATA_ERR_INVALID_ARG;
+  r.p = Problem{q, k, v, out, B, H, T, d_k, d_v, r.o.dtype, r.o.feature_order};
+  r.tensor = want_tensor(r.p, r.o);
+  if (r.o.impl == KATA_IMPL_TENSOR && !r.tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
+  r.plan = ScanPlan{(T + kChunk - 1) / kChunk, 0, 1, 0};
+  r.state_elems = 0;
+  r.inner_bytes = 0;
+  if (fn != KATA_FN_QUADRATIC) {
+    if (r.tensor && r.o.s_pre != nullptr) r.tensor = false;   // state export lives on the SIMT pipeline
+    st = make_plan(fn, r.p, r.o, r.tensor, r.plan, r.state_elems);
+    if (st != KATA_OK) return st;
+    r.inner_bytes = inner_workspace(fn, r.plan, r.p, r.state_elems);
+  }
+  return KATA_OK;
+}
+
+int run_device(int fn, Prepared& r, void* ws) {
+  LaunchCtx ctx{r.o.stream, 0, KATA_OK};
+  float* wsf = static_cast<float*>(ws);
+  if (fn == KATA_FN_QUADRATIC) {
+    if (r.tensor) tc_quadratic(r.p, r.o.device_status, ctx);
+    else simt_quadratic(r.p, ctx);
+  } else {
+    const bool use_scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || r.plan.n_groups > 1;
+    if (r.tensor) tc_chunked(r.p, r.plan, use_scan, wsf, r.o.device_status, ctx);
+    else if (r.p.feature_order == 1) order1_chunked(r.p, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, ctx);
+    else simt_chunked(r.p, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, r.o.state_layout, ctx);
+  }
+  if (ctx.status == KATA_OK) {
+    g_last_launches = ctx.launches;
+    g_last_impl = r.tensor ? KATA_IMPL_TENSOR : KATA_IMPL_SIMT;
+  }
+  return ctx.status;
+}
+
+int entry(int fn, const void* q, const void* k, const void* v, void* out, int B, int H, int T, int d_k,
+          int d_v, int C, const kata_opts* opts) {
+  Prepared r;
+  int st = prepare(fn, q, k, v, out, B, H, T, d_k, d_v, C, opts, true, r);
+  if (st != KATA_OK) return st;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return KATA_ERR_ALIGNMENT;
+  if (r.o.s_pre != nullptr && (!aligned16(r.o.s_pre) || !aligned16(r.o.z_pre))) return KATA_ERR_ALIGNMENT;
+  if (r.inner_bytes > 0) {
+    if (r.o.workspace == nullptr || r.o.workspace_bytes < r.inner_bytes) return KATA_ERR_WORKSPACE_TOO_SMALL;
+    if ((reinterpret_cast<uintptr_t>(r.o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;
+  }
+  st = check_arch();
+  if (st != KATA_OK) return st;
+  return run_device(fn, r, r.o.workspace);
+}
+
+}  // namespace
+}  // namespace kata
+
+using namespace kata;
+
+extern "C" {
+
+int kata_fwd_quadratic(const void* q, const void* k, const void* v, void* out, int B, int H, int T, int d_k,
+                       int d_v, int C, const kata_opts* opts) {
+  return entry(KATA_FN_QUADRATIC, q, k, v, out, B, H, T, d_k, d_v, C, opts);
+}
+
+int kata_fwd_chunked(const void* q, const void* k, const void* v, void* out, int B, int H, int T, int d_k,
+                     int d_v, int C, const kata_opts* opts) {
+  return entry(KATA_FN_CHUNKED, q, k, v, out, B, H, T, d_k, d_v, C, opts);
+}
+
+int kata_chunk_state_scan(const void* q, const void* k, const void* v, void* out, int B, int H, int T,
+                          int d_k, int d_v, int C, const kata_opts* opts) {
+  return entry(KATA_FN_CHUNK_STATE_SCAN, q, k, v, out, B, H, T, d_k, d_v, C, opts);
+}
+
+int kata_fwd_host(int fn, const void* q_host, const void* k_host, const void* v_host, void* out_host, int B,
+                  int H, int T, int d_k, int d_v, int C, const kata_opts* opts) {
+  Prepared r;
+  int st = prepare(fn, q_host, k_host, v_host, out_host, B, H, T, d_k, d_v, C, opts, true, r);
+  if (st != KATA_OK) return st;
+  if (r.o.s_pre != nullptr && (!aligned16(r.o.s_pre) || !aligned16(r.o.z_pre))) return KATA_ERR_ALIGNMENT;
+  const Staging s = staging_layout(r.p, r.inner_bytes);
+  if (r.o.workspace == nullptr || r.o.workspace_bytes < s.total) return KATA_ERR_WORKSPACE_TOO_SMALL;
+  if ((reinterpret_cast<uintptr_t>(r.o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;
+  st = check_arch();
+  if (st != KATA_OK) return st;
+  char* ws = static_cast<char*>(r.o.workspace);
+  const size_t eb = elem_bytes(r.p.dtype);
+  const size_t nqk = (size_t)B * H * T * d_k * eb, nv = (size_t)B * H * T * d_v * eb;
+  cudaStream_t stream = r.o.stream;
+  bool ok = cudaMemcpyAsync(ws + s.q, q_host, nqk, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(ws + s.k, k_host, nqk, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(ws + s.v, v_host, nv, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return KATA_ERR_CUDA;
+  }
+  r.p.q = ws + s.q;
+  r.p.k = ws + s.k;
+  r.p.v = ws + s.v;
+  r.p.out = ws + s.out;
+  st = run_device(fn, r, ws + s.inner);
+  if (st != KATA_OK) return st;
+  if (cudaMemcpyAsync(out_host, ws + s.out, nv, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
+    cudaGetLastError();
+    return KATA_ERR_CUDA;
+  }
+  return KATA_OK;
+}
+
+size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts) {
+  const bool host_io = (fn & KATA_FN_HOST_IO) != 0;
+  fn &= ~KATA_FN_HOST_IO;
+  Prepared r;
+  if (prepare(fn, nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, C, opts, false, r) != KATA_OK) return 0;
+  if (!host_io) return r.inner_bytes;
+  return staging_layout(r.p, r.inner_bytes).total;
+}
+
+int kata_scan_plan(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts, int* n_groups,
+                   int* chunks_per_group, int* scan_rounds) {
+  Prepared r;
+  const int st = prepare(fn & ~KATA_FN_HOST_IO, nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, C, opts,
+                         false, r);
+  if (st != KATA_OK) return st;
+  if (n_groups) *n_groups = r.plan.n_groups;
+  if (chunks_per_group) *chunks_per_group = r.plan.chunks_per_group;
+  if (scan_rounds) *scan_rounds = r.plan.rounds;
+  return KATA_OK;
+}
+
+int kata_last_launch_count(void) { return g_last_launches; }
+
+int kata_last_impl(void) { return g_last_impl; }
+
+const char* kata_status_string(int status) {
+  switch (status) {
+    case KATA_OK: return "ok";
+    case KATA_ERR_INVALID_ARG: return "invalid argument";
+    case KATA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case KATA_ERR_ALIGNMENT: return "pointer not sufficiently aligned";
+    case KATA_ERR_WORKSPACE_TOO_SMALL: return "workspace missing or too small";
+    case KATA_ERR_ARCH: return "device is not compute capability 10.x (B200)";
+    case KATA_ERR_CUDA: return "CUDA runtime error";
+    case KATA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int kata_version(void) { return KATA_VERSION; }
+
+}  // extern "C"

@@ -1,0 +1,84 @@
+// Shared device/host helpers of the KATA kernels (element-type access, status plumbing).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/kata.h"
+
+namespace kata {
+
+constexpr int kChunk = 64;  // chunk size C of the chunked and scan forms
+
+// ---- element access: global element -> fp32 and back (round-to-nearest-even) -------------
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// 1/||x||^2-style scale with the zero-row reading: a zero row has a zero feature.
+__device__ __forceinline__ float inv_or_zero(float s) { return s > 0.f ? 1.f / s : 0.f; }
+__device__ __forceinline__ float rsqrt_or_zero(float s) { return s > 0.f ? rsqrtf(s) : 0.f; }
+
+// ---- launch bookkeeping (host) --------------------------------------------------------------
+struct LaunchCtx {
+  cudaStream_t stream;
+  int launches;
+  int status;
+};
+
+inline void note_launch(LaunchCtx& ctx) {
+  ctx.launches++;
+  if (ctx.status == KATA_OK && cudaPeekAtLastError() != cudaSuccess) {
+    cudaGetLastError();
+    ctx.status = KATA_ERR_CUDA;
+  }
+}
+
+struct Problem {
+  const void* q;
+  const void* k;
+  const void* v;
+  void* out;
+  int B, H, T, d_k, d_v;
+  int dtype;
+  int feature_order;
+};
+
+// Scan/group plan of the chunked forms.
+struct ScanPlan {
+  int n_chunks;          // N_C = ceil(T / C)
+  int chunks_per_group;  // G
+  int n_groups;          // ceil(N_C / G)
+  int rounds;            // ceil(log2 n_groups)
+};
+
+// SIMT kernels (fp32 arithmetic; any supported shape and element type)
+void simt_quadratic(const Problem& p, LaunchCtx& ctx);
+size_t simt_chunked_state_elems(int d_k, int d_v);  // floats of internal state per (b,h,group)
+int simt_chunked_slices(int d_k, int d_v);          // CTAs per (b,h,group)
+// Inclusive Hillis-Steele scan over the first g_used of n_groups group states x[BH][n_groups][E]
+// (E a multiple of 4), ping-ponging between bufA (input) and bufB; returns the buffer holding the result.
+const float* scan_group_states(float* bufA, float* bufB, int BH, int n_groups, int g_used, size_t E,
+                               LaunchCtx& ctx);
+void simt_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre,
+                  float* z_pre, int state_layout, LaunchCtx& ctx);
+
+// feature_order = 1: rows of q,k are the features (plain normalised linear attention, state d_k x d_v)
+size_t order1_state_elems(int d_k, int d_v);
+void order1_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre,
+                    float* z_pre, LaunchCtx& ctx);
+
+// Tensor-core kernels (tcgen05/TMEM; bf16, d_k = d_v = 64)
+bool tc_supported(const Problem& p);
+void tc_quadratic(const Problem& p, int* device_status, LaunchCtx& ctx);
+size_t tc_chunked_state_elems();
+int tc_chunked_slices();
+void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, int* device_status,
+                LaunchCtx& ctx);
+
+}  // namespace kata

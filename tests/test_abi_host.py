@@ -1,0 +1,113 @@
+"""Host-side checks of the C ABI (no GPU): the library loads, exports what include/kata.h
+declares, and rejects bad arguments with the documented status codes before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2607_17419_b200 import binding as kb
+from paper_2607_17419_b200 import build as kbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    kbuild.build()
+    return kb.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "kata.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(kata_[a-z_]+)\s*\(", text)))
+
+
+def test_exports_match_header(L):
+    names = declared_functions()
+    assert set(names) == set(kb.EXPORTS)
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_version_and_status_strings(L):
+    assert kb.kata_version() == 100
+    seen = {kb.status_string(s) for s in range(0, -8, -1)}
+    assert len(seen) == 8 and "unknown status" not in seen
+    assert kb.status_string(-99) == "unknown status"
+
+
+def test_opts_struct_layout():
+    assert ctypes.sizeof(kb.KataOpts) == 80
+    assert kb.KataOpts.workspace.offset == 32 and kb.KataOpts.stream.offset == 72
+
+
+def call(L, fn, q=256, k=512, v=768, out=1024, B=1, H=1, T=64, d_k=64, d_v=64, C=64, opts=None):
+    opts = opts if opts is not None else kb.make_opts(kb.KATA_BF16)
+    return getattr(L, fn)(q, k, v, out, B, H, T, d_k, d_v, C, ctypes.byref(opts))
+
+
+@pytest.mark.parametrize("fn", ["kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan"])
+def test_invalid_arguments(L, fn):
+    INV, SHAPE, ALIGN, WS = -1, -2, -3, -4
+    assert getattr(L, fn)(256, 512, 768, 1024, 1, 1, 64, 64, 64, 64, None) == INV
+    bad = kb.make_opts(kb.KATA_BF16)
+    bad.struct_size = 12
+    assert call(L, fn, opts=bad) == INV
+    assert call(L, fn, q=None) == INV
+    assert call(L, fn, out=None) == INV
+    assert call(L, fn, B=0) == INV
+    assert call(L, fn, T=0) == INV
+    assert call(L, fn, opts=kb.make_opts(7)) == INV
+    assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, feature_order=3)) == INV
+    assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, scan_group=-1)) == INV
+    assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096)) == INV       # z_pre missing
+    assert call(L, fn, d_k=48) == SHAPE
+    assert call(L, fn, d_v=128) == SHAPE
+    assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, impl=kb.KATA_IMPL_TENSOR)) == SHAPE
+    assert call(L, fn, q=260) == ALIGN
+    assert call(L, fn, out=1032) == ALIGN
+    if fn != "kata_fwd_quadratic":
+        assert call(L, fn, C=32) == SHAPE
+        assert call(L, fn, C=0) == INV
+    if fn == "kata_chunk_state_scan":
+        assert call(L, fn, T=640) == WS                                        # needs a workspace
+        o = kb.make_opts(kb.KATA_F32, workspace=4096 + 8, workspace_bytes=1 << 40)
+        assert call(L, fn, T=640, opts=o) == ALIGN
+        o = kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192, scan_group=4)
+        assert call(L, fn, T=640, opts=o) == INV
+    else:
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192)) == INV
+
+
+def test_scan_workspace_and_plan(L):
+    o = kb.make_opts(kb.KATA_BF16)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 4, 16, 4096, 64, 64, 64, o) == 0
+    assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 8, 16, 4096, 64, 64, 64, o) == 0   # sequential
+    assert kb.kata_scan_plan(kb.KATA_FN_CHUNKED, 8, 16, 4096, 64, 64, 64, o)[0] == 1
+    o = kb.make_opts(kb.KATA_BF16, inter_chunk=kb.KATA_SCAN, scan_group=16, impl=kb.KATA_IMPL_SIMT)
+    ng, g, rounds = kb.kata_scan_plan(kb.KATA_FN_CHUNKED, 1, 16, 8192, 64, 64, 64, o)
+    assert (ng, g, rounds) == (8, 16, 3)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 16, 8192, 64, 64, 64, o) > 0
+    # per-chunk pipeline: T=2048, C=64 -> 32 chunks; the exclusive prefix needs the inclusive scan of
+    # the first 31 chunk states: ceil(log2 31) = 5 rounds
+    o = kb.make_opts(kb.KATA_F32, impl=kb.KATA_IMPL_SIMT)
+    assert kb.kata_scan_plan(kb.KATA_FN_CHUNK_STATE_SCAN, 1, 2, 2048, 16, 16, 64, o) == (32, 1, 5)
+    assert kb.kata_scan_plan(kb.KATA_FN_CHUNK_STATE_SCAN, 1, 2, 4160, 16, 16, 64, o) == (65, 1, 6)
+    # host-I/O variant adds the staging area
+    a = kb.kata_workspace_bytes(kb.KATA_FN_CHUNK_STATE_SCAN, 1, 2, 2048, 16, 16, 64, o)
+    b = kb.kata_workspace_bytes(kb.KATA_FN_CHUNK_STATE_SCAN | kb.KATA_FN_HOST_IO, 1, 2, 2048, 16, 16, 64, o)
+    assert b >= a + 4 * 2 * 2048 * 16 * 4
+    assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 1, 64, 48, 64, 64, o) == 0      # invalid -> 0
+
+
+def test_no_oracle_in_product_path():
+    """The package must not import or reference the oracle."""
+    pkg = os.path.join(ROOT, "paper_2607_17419_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert not re.search(r"^\s*(from|import)\s+\S*oracle", text, flags=re.M), f
+                assert "kata_oracle" not in text and "oracle/" not in text, f
