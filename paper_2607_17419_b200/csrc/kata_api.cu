@@ -67,8 +67,9 @@ int check_shape(int fn, int B, int H, int T, int d_k, int d_v, int C) {
   return KATA_OK;
 }
 
-bool want_tensor(const Problem& p, const Opts& o) {
-  return o.impl != KATA_IMPL_SIMT && tc_supported(p);
+bool want_tensor(int fn, const Problem& p, const Opts& o) {
+  const bool scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || (fn == KATA_FN_CHUNKED && o.inter_chunk == KATA_SCAN);
+  return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn, scan);
 }
 
 // How the chunk axis is cut into scan groups, and how many floats one group state takes.
@@ -179,7 +180,7 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   if (need_ptrs && (q == nullptr || k == nullptr || v == nullptr || out == nullptr)) return KATA_ERR_INVALID_ARG;
   if (fn != KATA_FN_CHUNK_STATE_SCAN && r.o.s_pre != nullptr) return KATA_ERR_INVALID_ARG;
   r.p = Problem{q, k, v, out, B, H, T, d_k, d_v, r.o.dtype, r.o.feature_order};
-  r.tensor = want_tensor(r.p, r.o);
+  r.tensor = want_tensor(fn, r.p, r.o);
   if (r.o.impl == KATA_IMPL_TENSOR && !r.tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
   r.plan = ScanPlan{(T + kChunk - 1) / kChunk, 0, 1, 0};
   r.state_elems = 0;

@@ -1,12 +1,14 @@
-// Tensor-core (tcgen05/TMEM) kernels: placeholder until the first version lands.
+// Which problems the tensor-core (tcgen05/TMEM) kernels cover.
 #include "kata_common.cuh"
 
 namespace kata {
-bool tc_supported(const Problem&) { return false; }
-void tc_quadratic(const Problem&, int*, LaunchCtx& ctx) { ctx.status = KATA_ERR_UNSUPPORTED_SHAPE; }
-size_t tc_chunked_state_elems() { return 0; }
-int tc_chunked_slices() { return 1; }
-void tc_chunked(const Problem&, const ScanPlan&, bool, float*, int*, LaunchCtx& ctx) {
-  ctx.status = KATA_ERR_UNSUPPORTED_SHAPE;
+
+bool tc_supported(const Problem& p, int fn, bool scan) {
+  if (p.dtype != KATA_BF16 || p.d_k != 64 || p.d_v != 64 || p.feature_order != 2) return false;
+  if (fn == KATA_FN_CHUNKED) return !scan;
+  return false;
 }
+
+void tc_quadratic(const Problem&, int*, LaunchCtx& ctx) { ctx.status = KATA_ERR_UNSUPPORTED_SHAPE; }
+
 }  // namespace kata
