@@ -6,18 +6,23 @@
 // re-associated so that no feature matrix Psi is ever built:
 //
 //   state update   S[(b,v), a] += sum_t W[(b,v), t] * k[t, a],   W[(b,v), t] = k[t,b] v[t,v] / ||k_t||^2
-//                  (tcgen05 kind::f16: A = W from shared memory, built on the fly; B = the TMA-loaded
+//                  (tcgen05 kind::f16: A = W, built in registers and stored to TMEM; B = the TMA-loaded
 //                   key tile used MN-major; D = fp32 accumulators resident in TMEM for the whole head)
 //   inter-chunk    Y[(b,v), t] = sum_a S[(b,v), a] * q[t, a]     (tcgen05 kind::tf32: A = the fp32
 //   read           accumulators of the update, read straight from TMEM; B = the query tile as tf32)
 //                  N_inter[t, v] = sum_b q[t,b] * Y[(b,v), t]    (fp32 FMAs on the TMEM read-back)
 //   normaliser     the same two steps with the "ones" value column: rows (b) of a fifth tile hold Z
-//   intra-chunk    P = (Q K^T)^2 / ||k||^2 o M from one d-dimensional bf16 MMA, squared in fp32;
-//                  N_intra = P V, D_intra = P 1 on fp32 FMAs
+//   intra-chunk    scores s = Q K^T from one d-dimensional bf16 MMA; P = s^2 / ||k||^2 o M in fp32,
+//                  rounded to bf16 into TMEM; [N_intra | D_intra] = P [V | 1] as one more MMA, so the
+//                  normaliser is the row sum of exactly the P that multiplies V
 //   epilogue       O = (N_inter + N_intra) / (D_inter + D_intra)   (gate + normalise), bf16 store
 //
 // The query norm is a common factor of numerator and denominator and is never applied.  Rows (b,v) of a
 // 128-row MMA tile are b = 16*tile + row/8, v = row%8; four tiles cover b = 0..63, the fifth holds Z.
+//
+// Scan form: grid.z cuts the chunk axis into groups.  A first launch (write_out = 0) only accumulates
+// the group-local states and stores them; after the log-depth scan over groups a second launch restarts
+// every group from the prefix before it.
 //
 // Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 operand builders
 // (norms, tf32 query tile, transposes, W tiles), warps 6-9 TMEM readers (Y reduction, scores, epilogue).
@@ -37,45 +42,51 @@ constexpr int C = kChunk;        // 64 tokens per chunk
 constexpr int D = 64;            // d_k = d_v
 constexpr int VS = 8;            // value columns per CTA
 constexpr int NSLICE = D / VS;   // CTAs per head
-constexpr int NT = 5;            // MMA tiles per chunk: 4 state tiles + the normaliser tile
+constexpr int NT = 5;            // state tiles: 4 x S + the normaliser tile
+constexpr int NI = 6;            // ring items per chunk: 5 reads + the score/intra item
 constexpr int NTHREADS = 320;
+constexpr size_t STATE_PER_SLICE = (size_t)NT * 128 * 64;   // floats
 
-// TMEM columns (fp32 accumulators, 128 lanes each)
-constexpr uint32_t COL_S = 0;      // 5 tiles x 64 columns: S tiles 0..3, Z tile 4
-constexpr uint32_t COL_Y = 320;    // 2 x 64: ring of read results
-constexpr uint32_t COL_P = 448;    // 64: intra-chunk scores (rows 0..63 valid)
+// TMEM columns (128 lanes each)
+constexpr uint32_t COL_S = 0;      // 5 x 64 fp32: S tiles 0..3, Z tile 4
+constexpr uint32_t COL_R = 320;    // 2 x 64: ring (read results; scores -> P bf16 [0,32) -> P[V|1] at [32,48))
+constexpr uint32_t COL_W = 448;    // 2 x 32: W tiles (bf16 pairs), A operand of the update
 constexpr uint32_t TMEM_COLS = 512;
 
 // shared memory map (bytes from a 1024-aligned base)
+constexpr uint32_t KT_STRIDE = 68;                // floats per kT / vT row (16-byte aligned, conflict-free LDS.128)
 constexpr uint32_t OFF_QK = 0;                    // 2 stages x (Q tile 8 KB, K tile 8 KB), TMA, 128B swizzle
-constexpr uint32_t OFF_V = 32768;                 // 2 stages x 64 x 8 bf16
-constexpr uint32_t OFF_QF = 34816;                // 2 x 16 KB: query tile as tf32, K-major, 128B swizzle, 2 atoms
-constexpr uint32_t OFF_W = 67584;                 // 2 x 16 KB: W tile, bf16, K-major, 128B swizzle
-constexpr uint32_t OFF_KT = 100352;               // kT[b][t] fp32 (builders only)
-constexpr uint32_t OFF_VT = 116736;               // vT[v][t] = v / ||k||^2, fp32 (builders only)
-constexpr uint32_t OFF_QT = 118784;               // 2 x qT[b][t] fp32 (readers)
-constexpr uint32_t OFF_VS = 151552;               // 2 x vS[t][v] fp32 raw values (readers)
-constexpr uint32_t OFF_R2 = 155648;               // 2 x r2[t] = 1/||k_t||^2
-constexpr uint32_t OFF_RED = 156160;              // red[128][68] fp32 cross-lane reduction scratch
+constexpr uint32_t OFF_V = 32768;                 // 2 stages x 64 x 8 bf16 (TMA, dense 16-byte rows)
+constexpr uint32_t OFF_ONES = 34816;              // 64 x 8 bf16 rows (1,0,..,0): the "ones" column group
+constexpr uint32_t OFF_QF = 35840;                // 2 x 16 KB: query tile as tf32, K-major, 128B swizzle, 2 atoms
+constexpr uint32_t OFF_KT = 68608;                // kT[b][t] fp32, stride 68 (builders only)
+constexpr uint32_t OFF_VT = 86016;                // vT[v][t] = v / ||k||^2, fp32, stride 68 (builders only)
+constexpr uint32_t OFF_QT = 88192;                // 2 x qT[b][t] fp32 (readers)
+constexpr uint32_t OFF_R2 = 120960;               // 2 x r2[t] = 1/||k_t||^2
+constexpr uint32_t OFF_RED = 121472;              // red[128][68] fp32 cross-lane reduction scratch
 constexpr uint32_t RED_STRIDE = 68;
-constexpr uint32_t OFF_NINTRA = 190976;           // [64][9]
-constexpr uint32_t OFF_NINTER = 193280;           // [64][9]
-constexpr uint32_t OFF_BAR = 195584;              // mbarriers
-constexpr uint32_t SMEM_BYTES = 195584 + 256;
+constexpr uint32_t OFF_NINTRA = 156288;           // [64][9]
+constexpr uint32_t OFF_NINTER = 158592;           // [64][9]
+constexpr uint32_t OFF_BAR = 160896;              // mbarriers
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;  // slack for the 1024-byte alignment
+static_assert(OFF_QF % 1024 == 0 && OFF_QK % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+static_assert(SMEM_ALLOC > 116 * 1024, "one CTA per SM is assumed (the CTA allocates all of TMEM)");
 
 enum {
   BAR_FULL = 0,     // [2] TMA landed
   BAR_EMPTY = 2,    // [2] stage free (128 builders + MMA commit)
   BAR_PREP = 4,     // [2] operands of the chunk built (128 builders)
-  BAR_WFULL = 6,    // [2] W tile built
+  BAR_WFULL = 6,    // [2] W tile stored to TMEM
   BAR_WEMPTY = 8,   // [2] W tile consumed by the MMA
-  BAR_YFULL = 10,   // [2] read result in TMEM
-  BAR_YEMPTY = 12,  // [2] read result drained (128 readers)
-  BAR_PFULL = 14,
-  BAR_PEMPTY = 15,
+  BAR_RFULL = 10,   // [2] ring item produced by the MMA
+  BAR_REMPTY = 12,  // [2] ring item drained (128 readers)
+  BAR_PREADY = 14,  // P (bf16) stored to TMEM (128 readers)
+  BAR_PVFULL = 15,  // P [V|1] complete
   BAR_U = 16,       // [5] update of state tile i complete
-  BAR_COUNT = 21
+  BAR_DRAIN = 21,
+  BAR_DONE = 22,    // every update of this CTA has completed
+  BAR_COUNT = 23
 };
 
 struct Shared {
@@ -83,12 +94,11 @@ struct Shared {
   __device__ unsigned char* qtile(int s) const { return base + OFF_QK + s * 16384; }
   __device__ unsigned char* ktile(int s) const { return base + OFF_QK + s * 16384 + 8192; }
   __device__ unsigned char* vtile(int s) const { return base + OFF_V + s * 1024; }
+  __device__ unsigned char* ones() const { return base + OFF_ONES; }
   __device__ unsigned char* qf(int s) const { return base + OFF_QF + s * 16384; }
-  __device__ unsigned char* w(int s) const { return base + OFF_W + s * 16384; }
   __device__ float* kT() const { return reinterpret_cast<float*>(base + OFF_KT); }
   __device__ float* vT() const { return reinterpret_cast<float*>(base + OFF_VT); }
   __device__ float* qT(int s) const { return reinterpret_cast<float*>(base + OFF_QT + s * 16384); }
-  __device__ float* vS(int s) const { return reinterpret_cast<float*>(base + OFF_VS + s * 2048); }
   __device__ float* r2(int s) const { return reinterpret_cast<float*>(base + OFF_R2 + s * 256); }
   __device__ float* red() const { return reinterpret_cast<float*>(base + OFF_RED); }
   __device__ float* nintra() const { return reinterpret_cast<float*>(base + OFF_NINTRA); }
@@ -113,10 +123,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+struct KernelArgs {
+  __nv_bfloat16* out;
+  const float* init_state;   // inclusive group scan [BH][n_groups][NSLICE][5][128][64]; group g starts from entry g-1
+  float* final_state;        // same layout; group g stores entry g
+  int* device_status;
+  int Tlen, n_chunks, chunks_per_group, n_groups, write_out;
+};
+
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ out, int Tlen, int n_chunks,
-                int* __restrict__ device_status) {
+                const __grid_constant__ CUtensorMap tmV, const KernelArgs args) {
   extern __shared__ unsigned char smem_raw[];
   Shared sm;
   sm.base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -125,29 +142,39 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   volatile int* abort_flag = &abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int slice = blockIdx.x;
-  const int bh = blockIdx.y;
+  const int slice = blockIdx.x, bh = blockIdx.y, grp = blockIdx.z;
+  const int c_begin = grp * args.chunks_per_group;
+  const int c_end = min(args.n_chunks, c_begin + args.chunks_per_group);
+  const int nloc = c_end - c_begin;                  // chunks handled by this CTA
+  const bool write_out = args.write_out != 0;
+  const bool have_init = args.init_state != nullptr && grp > 0;
+  const size_t state_off = (((size_t)bh * args.n_groups + grp) * NSLICE + slice) * STATE_PER_SLICE;
 
   if (tid == 0) {
     abort_s = 0;
-    mbar_init(sm.bar(BAR_FULL + 0), 1);
-    mbar_init(sm.bar(BAR_FULL + 1), 1);
-    mbar_init(sm.bar(BAR_EMPTY + 0), 129);
-    mbar_init(sm.bar(BAR_EMPTY + 1), 129);
     for (int i = 0; i < 2; ++i) {
+      mbar_init(sm.bar(BAR_FULL + i), 1);
+      mbar_init(sm.bar(BAR_EMPTY + i), 129);
       mbar_init(sm.bar(BAR_PREP + i), 128);
       mbar_init(sm.bar(BAR_WFULL + i), 128);
       mbar_init(sm.bar(BAR_WEMPTY + i), 1);
-      mbar_init(sm.bar(BAR_YFULL + i), 1);
-      mbar_init(sm.bar(BAR_YEMPTY + i), 128);
+      mbar_init(sm.bar(BAR_RFULL + i), 1);
+      mbar_init(sm.bar(BAR_REMPTY + i), 128);
     }
-    mbar_init(sm.bar(BAR_PFULL), 1);
-    mbar_init(sm.bar(BAR_PEMPTY), 128);
+    mbar_init(sm.bar(BAR_PREADY), 128);
+    mbar_init(sm.bar(BAR_PVFULL), 1);
     for (int i = 0; i < NT; ++i) mbar_init(sm.bar(BAR_U + i), 1);
+    mbar_init(sm.bar(BAR_DRAIN), 1);
+    mbar_init(sm.bar(BAR_DONE), 1);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmV);
+  }
+  // constant "ones" column group for the intra-chunk MMA: row t = (1, 0, 0, 0, 0, 0, 0, 0) in bf16
+  if (tid >= 64 && tid < 128) {
+    *reinterpret_cast<uint4*>(sm.ones() + (tid - 64) * 16) = make_uint4(0x00003F80u, 0u, 0u, 0u);
+    fence_async_smem();
   }
   if (warp == 0) {
     tmem_alloc(&tmem_base_s, TMEM_COLS);
@@ -158,13 +185,29 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
 
-  // zero the state accumulators (readers own the TMEM lanes)
+  // initial state: zero, or the prefix of the groups before this one (readers own the TMEM lanes)
   if (warp >= 6) {
     const uint32_t q4 = warp & 3;
+    const int rowl = q4 * 32 + lane;
     uint32_t z[32];
+    for (int cblk = 0; cblk < (NT * 64) / 32; ++cblk) {
+      if (have_init) {
+        const float* src = args.init_state + (state_off - (size_t)NSLICE * STATE_PER_SLICE) +
+                           ((size_t)(cblk >> 1) * 128 + rowl) * 64 + (cblk & 1) * 32;
 #pragma unroll
-    for (int j = 0; j < 32; ++j) z[j] = 0u;
-    for (int cblk = 0; cblk < (NT * 64) / 32; ++cblk) tmem_st32(tmem_addr(tb, q4 * 32, COL_S + cblk * 32), z);
+        for (int j = 0; j < 32; j += 4) {
+          const float4 f = *reinterpret_cast<const float4*>(src + j);
+          z[j] = __float_as_uint(f.x);
+          z[j + 1] = __float_as_uint(f.y);
+          z[j + 2] = __float_as_uint(f.z);
+          z[j + 3] = __float_as_uint(f.w);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) z[j] = 0u;
+      }
+      tmem_st32(tmem_addr(tb, q4 * 32, COL_S + cblk * 32), z);
+    }
     tmem_wait_st();
   }
   tc_fence_before();
@@ -176,81 +219,114 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (warp == 0) {
     // =========================== TMA producer ===========================
     if (lane == 0) {
-      for (int c = 0; c < n_chunks && ok; ++c) {
+      for (int c = 0; c < nloc && ok; ++c) {
         const int s = c & 1;
         ok = wait_or_abort(sm.bar(BAR_EMPTY + s), ((c >> 1) & 1) ^ 1, abort_flag);
         if (!ok) break;
+        const int t0 = (c_begin + c) * C;
         mbar_arrive_expect_tx(sm.bar(BAR_FULL + s), 8192 + 8192 + 1024);
-        tma_load_3d(sm.qtile(s), &tmQ, sm.bar(BAR_FULL + s), 0, c * C, bh);
-        tma_load_3d(sm.ktile(s), &tmK, sm.bar(BAR_FULL + s), 0, c * C, bh);
-        tma_load_3d(sm.vtile(s), &tmV, sm.bar(BAR_FULL + s), slice * VS, c * C, bh);
+        tma_load_3d(sm.qtile(s), &tmQ, sm.bar(BAR_FULL + s), 0, t0, bh);
+        tma_load_3d(sm.ktile(s), &tmK, sm.bar(BAR_FULL + s), 0, t0, bh);
+        tma_load_3d(sm.vtile(s), &tmV, sm.bar(BAR_FULL + s), slice * VS, t0, bh);
       }
     }
   } else if (warp == 1) {
     // =========================== MMA issuer ===========================
     if (lane == 0) {
-      const uint32_t id_read = instr_desc(kFmtTF32, kFmtTF32, 0, 0, 128, 64);    // A tmem, B K-major
-      const uint32_t id_qk = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 64);      // both K-major
-      const uint32_t id_upd = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 64);     // B MN-major
-      for (int c = 0; c < n_chunks && ok; ++c) {
+      const uint32_t id_read = instr_desc(kFmtTF32, kFmtTF32, 0, 0, 128, 64);    // A tmem (fp32 as tf32), B K-major
+      const uint32_t id_qk = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 64);      // both K-major from smem
+      const uint32_t id_upd = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 64);     // A tmem, B MN-major
+      const uint32_t id_pv = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 16);      // A tmem, B MN-major, N = 16
+      // descriptors that depend only on the stage
+      uint64_t d_qf[2][8], d_q[2][4], d_k[2][4], d_kmn[2][4], d_v[2][4];
+#pragma unroll
+      for (int s = 0; s < 2; ++s) {
+        const uint32_t qf = smem_u32(sm.qf(s)), qa = smem_u32(sm.qtile(s)), ka = smem_u32(sm.ktile(s));
+        const uint32_t va = smem_u32(sm.vtile(s));
+        const uint32_t ones_off = smem_u32(sm.ones()) - va;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          d_qf[s][ks] = smem_desc(qf + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, kSwizzle128B);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          d_q[s][ks] = smem_desc(qa + ks * 32, 16, 1024, kSwizzle128B);
+          d_k[s][ks] = smem_desc(ka + ks * 32, 16, 1024, kSwizzle128B);
+          d_kmn[s][ks] = smem_desc(ka + ks * 2048, 8192, 1024, kSwizzle128B);
+          // [V | ones]: MN-major, no swizzle: 8 k-rows x 16 bytes per core matrix, next 8 k at +128 (LBO),
+          // second group of 8 columns (the ones group) at +ones_off (SBO)
+          d_v[s][ks] = smem_desc(va + ks * 256, 128, ones_off, kSwizzleNone);
+        }
+      }
+      for (int c = 0; c < nloc && ok; ++c) {
         const int s = c & 1;
         const uint32_t ph = (c >> 1) & 1;
         ok = wait_or_abort(sm.bar(BAR_FULL + s), ph, abort_flag) &&
              wait_or_abort(sm.bar(BAR_PREP + s), ph, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        // ---- inter-chunk reads Y_i = S_i * Q^T (tf32, A from TMEM) ----
-        for (int i = 0; i < NT && ok; ++i) {
-          const int g = c * NT + i;
-          ok = wait_or_abort(sm.bar(BAR_YEMPTY + (g & 1)), ((g >> 1) & 1) ^ 1, abort_flag);
-          if (ok && c > 0) ok = wait_or_abort(sm.bar(BAR_U + i), (c - 1) & 1, abort_flag);
+        if (write_out) {
+          // ---- inter-chunk reads Y_i = S_i * Q^T (tf32, A = accumulators in TMEM) ----
+          for (int i = 0; i < NT && ok; ++i) {
+            const int g = c * NI + i;
+            ok = wait_or_abort(sm.bar(BAR_REMPTY + (g & 1)), ((g >> 1) & 1) ^ 1, abort_flag);
+            if (ok && c > 0) ok = wait_or_abort(sm.bar(BAR_U + i), (c - 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+              mma_tf32_ts(tb + COL_R + (g & 1) * 64, tb + COL_S + i * 64 + ks * 8, d_qf[s][ks], id_read, ks > 0);
+            mma_commit(sm.bar(BAR_RFULL + (g & 1)));
+          }
           if (!ok) break;
-          tc_fence_after();
-          const uint32_t qf = smem_u32(sm.qf(s));
+          // ---- intra-chunk scores [Q;K] K^T (rows 0..63 used) ----
+          {
+            const int g = c * NI + 5;
+            ok = wait_or_abort(sm.bar(BAR_REMPTY + (g & 1)), ((g >> 1) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            mma_tf32_ts(tb + COL_Y + (g & 1) * 64, tb + COL_S + i * 64 + ks * 8,
-                        smem_desc(qf + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, kSwizzle128B), id_read, ks > 0);
-          mma_commit(sm.bar(BAR_YFULL + (g & 1)));
+            for (int ks = 0; ks < 4; ++ks)
+              mma_f16_ss(tb + COL_R + (g & 1) * 64, d_q[s][ks], d_k[s][ks], id_qk, ks > 0);
+            mma_commit(sm.bar(BAR_RFULL + (g & 1)));
+          }
         }
-        if (!ok) break;
-        // ---- intra-chunk scores [Q;K] K^T (rows 0..63 used) ----
-        ok = wait_or_abort(sm.bar(BAR_PEMPTY), (c & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        {
-          const uint32_t qa = smem_u32(sm.qtile(s)), ka = smem_u32(sm.ktile(s));
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            mma_f16_ss(tb + COL_P, smem_desc(qa + ks * 32, 16, 1024, kSwizzle128B),
-                       smem_desc(ka + ks * 32, 16, 1024, kSwizzle128B), id_qk, ks > 0);
-          mma_commit(sm.bar(BAR_PFULL));
-        }
-        // ---- state updates S_i += W_i * K ----
+        // ---- state updates S_i += W_i * K (A = W in TMEM) ----
         for (int i = 0; i < NT && ok; ++i) {
           const int g = c * NT + i;
           ok = wait_or_abort(sm.bar(BAR_WFULL + (g & 1)), (g >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t wa = smem_u32(sm.w(g & 1)), ka = smem_u32(sm.ktile(s));
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
-            mma_f16_ss(tb + COL_S + i * 64, smem_desc(wa + ks * 32, 16, 1024, kSwizzle128B),
-                       smem_desc(ka + ks * 2048, 8192, 1024, kSwizzle128B), id_upd, 1u);
+            mma_f16_ts(tb + COL_S + i * 64, tb + COL_W + (g & 1) * 32 + ks * 8, d_kmn[s][ks], id_upd, 1u);
           mma_commit(sm.bar(BAR_WEMPTY + (g & 1)));
           mma_commit(sm.bar(BAR_U + i));
         }
         if (!ok) break;
+        if (write_out) {
+          // ---- [N_intra | D_intra] = P [V | 1] (A = P bf16 in the ring slot) ----
+          const int g = c * NI + 5;
+          ok = wait_or_abort(sm.bar(BAR_PREADY), c & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            mma_f16_ts(tb + COL_R + (g & 1) * 64 + 32, tb + COL_R + (g & 1) * 64 + ks * 8, d_v[s][ks], id_pv, ks > 0);
+          mma_commit(sm.bar(BAR_PVFULL));
+        }
         mma_commit(sm.bar(BAR_EMPTY + s));
       }
+      if (ok) mma_commit(sm.bar(BAR_DONE));
     }
   } else if (warp < 6) {
     // =========================== operand builders (128 threads) ===========================
     const int ta = tid - 64;
     const int row = ta >> 1, hf = ta & 1;          // prep mapping: two threads per token row
+    const uint32_t q4 = warp & 3;                  // TMEM lane quadrant of this warp
+    const int rowl = q4 * 32 + lane;               // W-tile row owned by this thread
     float* kT = sm.kT();
     float* vT = sm.vT();
-    for (int c = 0; c < n_chunks && ok; ++c) {
+    for (int c = 0; c < nloc && ok; ++c) {
       const int s = c & 1;
       ok = wait_or_abort(sm.bar(BAR_FULL + s), (c >> 1) & 1, abort_flag);
       if (!ok) break;
@@ -267,76 +343,94 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int j = 0; j < 4; ++j) {
           const int chunk = hf * 4 + j;
           const uint4 kraw = *reinterpret_cast<const uint4*>(kt + sw128_offset(row, chunk));
-          const uint4 qraw = *reinterpret_cast<const uint4*>(qt + sw128_offset(row, chunk));
           const uint32_t kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
-          const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
-          float kf[8], qv[8];
+          float kf[8];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             kf[2 * e] = __uint_as_float(kw[e] << 16);
             kf[2 * e + 1] = __uint_as_float(kw[e] & 0xFFFF0000u);
-            qv[2 * e] = __uint_as_float(qw[e] << 16);
-            qv[2 * e + 1] = __uint_as_float(qw[e] & 0xFFFF0000u);
           }
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             ss = fmaf(kf[e], kf[e], ss);
-            kT[(chunk * 8 + e) * C + row] = kf[e];
-            qT[(chunk * 8 + e) * C + row] = qv[e];
+            kT[(chunk * 8 + e) * KT_STRIDE + row] = kf[e];
           }
-          // tf32 query tile: 32 fp32 per 128-byte row, this thread's half-row is atom `hf`
-          *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j)) = make_float4(qv[0], qv[1], qv[2], qv[3]);
-          *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j + 1)) = make_float4(qv[4], qv[5], qv[6], qv[7]);
+          if (write_out) {
+            const uint4 qraw = *reinterpret_cast<const uint4*>(qt + sw128_offset(row, chunk));
+            const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
+            float qv[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              qv[2 * e] = __uint_as_float(qw[e] << 16);
+              qv[2 * e + 1] = __uint_as_float(qw[e] & 0xFFFF0000u);
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) qT[(chunk * 8 + e) * C + row] = qv[e];
+            // tf32 query tile: 32 fp32 per 128-byte row, this thread's half-row is atom `hf`
+            *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j)) = make_float4(qv[0], qv[1], qv[2], qv[3]);
+            *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j + 1)) = make_float4(qv[4], qv[5], qv[6], qv[7]);
+          }
         }
         ss += __shfl_xor_sync(0xffffffffu, ss, 1);
         if (hf == 0) r2[row] = inv_or_zero(ss);
       }
       group_sync(2);
-      // ---- phase 2: values: raw copy for the readers, scaled transposed copy for the W tiles ----
+      // ---- phase 2: scaled transposed values for the W tiles ----
       if (ta < C) {
         const uint4 vraw = *reinterpret_cast<const uint4*>(sm.vtile(s) + ta * 16);
         const uint32_t vw[4] = {vraw.x, vraw.y, vraw.z, vraw.w};
         const float rr = r2[ta];
-        float* vS = sm.vS(s);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float lo = __uint_as_float(vw[e] << 16), hi = __uint_as_float(vw[e] & 0xFFFF0000u);
-          vS[ta * VS + 2 * e] = lo;
-          vS[ta * VS + 2 * e + 1] = hi;
-          vT[(2 * e) * C + ta] = lo * rr;
-          vT[(2 * e + 1) * C + ta] = hi * rr;
+          vT[(2 * e) * KT_STRIDE + ta] = __uint_as_float(vw[e] << 16) * rr;
+          vT[(2 * e + 1) * KT_STRIDE + ta] = __uint_as_float(vw[e] & 0xFFFF0000u) * rr;
         }
       }
       fence_async_smem();
       group_sync(2);
       mbar_arrive(sm.bar(BAR_PREP + s));
-      mbar_arrive(sm.bar(BAR_EMPTY + s));     // done with the raw tiles (the MMA adds its own arrival)
-      // ---- W tiles: row ta <-> (b = 16 i + ta/8, v = ta%8); fifth tile: rows < 64 hold k[t,b]/||k||^2 ----
+      // the value row of this thread (v = rowl % 8), scaled by 1/||k||^2, for all 64 tokens
+      float vr[C];
+      {
+        const float* vrow = vT + (rowl & 7) * KT_STRIDE;
+#pragma unroll
+        for (int t4 = 0; t4 < C; t4 += 4) {
+          const float4 f = *reinterpret_cast<const float4*>(vrow + t4);
+          vr[t4] = f.x; vr[t4 + 1] = f.y; vr[t4 + 2] = f.z; vr[t4 + 3] = f.w;
+        }
+      }
+      // ---- W tiles: row rowl <-> (b = 16 i + rowl/8, v = rowl%8); fifth tile: rows < 64 hold k[t,b]/||k||^2 ----
       for (int i = 0; i < NT && ok; ++i) {
         const int g = c * NT + i;
         ok = wait_or_abort(sm.bar(BAR_WEMPTY + (g & 1)), ((g >> 1) & 1) ^ 1, abort_flag);
         if (!ok) break;
-        unsigned char* wt = sm.w(g & 1);
-        const float* krow = kT + ((i < 4) ? (16 * i + (ta >> 3)) : (ta & 63)) * C;
-        const float* vrow = (i < 4) ? (vT + (ta & 7) * C) : r2;
-        const bool zero = (i == 4) && (ta >= 64);
+        tc_fence_after();
+        const float* krow = kT + ((i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63)) * KT_STRIDE;
+        uint32_t pk[32];
+        if (i < 4) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float4 k0 = *reinterpret_cast<const float4*>(krow + 8 * j);
-          const float4 k1 = *reinterpret_cast<const float4*>(krow + 8 * j + 4);
-          const float4 v0 = *reinterpret_cast<const float4*>(vrow + 8 * j);
-          const float4 v1 = *reinterpret_cast<const float4*>(vrow + 8 * j + 4);
-          uint4 pk;
-          pk.x = pack_bf16(k0.x * v0.x, k0.y * v0.y);
-          pk.y = pack_bf16(k0.z * v0.z, k0.w * v0.w);
-          pk.z = pack_bf16(k1.x * v1.x, k1.y * v1.y);
-          pk.w = pack_bf16(k1.z * v1.z, k1.w * v1.w);
-          if (zero) pk = make_uint4(0u, 0u, 0u, 0u);
-          *reinterpret_cast<uint4*>(wt + sw128_offset(ta, j)) = pk;
+          for (int t4 = 0; t4 < C; t4 += 4) {
+            const float4 kk = *reinterpret_cast<const float4*>(krow + t4);
+            pk[t4 / 2] = pack_bf16(kk.x * vr[t4], kk.y * vr[t4 + 1]);
+            pk[t4 / 2 + 1] = pack_bf16(kk.z * vr[t4 + 2], kk.w * vr[t4 + 3]);
+          }
+        } else {
+          const bool live = rowl < 64;
+#pragma unroll
+          for (int t4 = 0; t4 < C; t4 += 4) {
+            const float4 kk = *reinterpret_cast<const float4*>(krow + t4);
+            const float4 rr = *reinterpret_cast<const float4*>(r2 + t4);
+            pk[t4 / 2] = live ? pack_bf16(kk.x * rr.x, kk.y * rr.y) : 0u;
+            pk[t4 / 2 + 1] = live ? pack_bf16(kk.z * rr.z, kk.w * rr.w) : 0u;
+          }
         }
-        fence_async_smem();
+        tmem_st32(tmem_addr(tb, q4 * 32, COL_W + (g & 1) * 32), pk);
+        tmem_wait_st();
+        tc_fence_before();
         mbar_arrive(sm.bar(BAR_WFULL + (g & 1)));
       }
+      if (!ok) break;
+      mbar_arrive(sm.bar(BAR_EMPTY + s));     // done with the stage (the MMA adds its own arrival)
     }
   } else {
     // =========================== TMEM readers (128 threads) ===========================
@@ -346,22 +440,28 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     float* red = sm.red();
     float* nintra = sm.nintra();
     float* ninter = sm.ninter();
-    __nv_bfloat16* oh = out + (size_t)bh * Tlen * D + slice * VS;
-    for (int c = 0; c < n_chunks && ok; ++c) {
+    __nv_bfloat16* oh = args.out + (size_t)bh * args.Tlen * D + slice * VS;
+    for (int c = 0; c < nloc && ok && write_out; ++c) {
       const int s = c & 1;
       ok = wait_or_abort(sm.bar(BAR_PREP + s), (c >> 1) & 1, abort_flag);
       if (!ok) break;
       const float* qT = sm.qT(s);
-      const float* vS = sm.vS(s);
       const float* r2 = sm.r2(s);
       float acc[C];
 #pragma unroll
       for (int t = 0; t < C; ++t) acc[t] = 0.f;
       for (int i = 0; i < NT && ok; ++i) {
-        const int g = c * NT + i;
-        ok = wait_or_abort(sm.bar(BAR_YFULL + (g & 1)), (g >> 1) & 1, abort_flag);
+        const int g = c * NI + i;
+        ok = wait_or_abort(sm.bar(BAR_RFULL + (g & 1)), (g >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
+        uint32_t y[C];
+        {
+          uint32_t(&y0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&y[0]);
+          uint32_t(&y1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&y[32]);
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (g & 1) * 64), y0);
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (g & 1) * 64 + 32), y1);
+        }
         if (i == 4) {
           // the four state tiles are in acc: reduce over b within the CTA -> ninter[t][v]
 #pragma unroll
@@ -386,22 +486,17 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         const int b = (i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63);
         const float* qrow = qT + b * C;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t y[32];
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_Y + (g & 1) * 64 + half * 32), y);
-          tmem_wait_ld();
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 qq = *reinterpret_cast<const float4*>(qrow + half * 32 + j);
-            acc[half * 32 + j] = fmaf(qq.x, __uint_as_float(y[j]), acc[half * 32 + j]);
-            acc[half * 32 + j + 1] = fmaf(qq.y, __uint_as_float(y[j + 1]), acc[half * 32 + j + 1]);
-            acc[half * 32 + j + 2] = fmaf(qq.z, __uint_as_float(y[j + 2]), acc[half * 32 + j + 2]);
-            acc[half * 32 + j + 3] = fmaf(qq.w, __uint_as_float(y[j + 3]), acc[half * 32 + j + 3]);
-          }
-        }
+        tmem_wait_ld();
         tc_fence_before();
-        mbar_arrive(sm.bar(BAR_YEMPTY + (g & 1)));
+        mbar_arrive(sm.bar(BAR_REMPTY + (g & 1)));      // the slot is in registers now
+#pragma unroll
+        for (int j = 0; j < C; j += 4) {
+          const float4 qq = *reinterpret_cast<const float4*>(qrow + j);
+          acc[j] = fmaf(qq.x, __uint_as_float(y[j]), acc[j]);
+          acc[j + 1] = fmaf(qq.y, __uint_as_float(y[j + 1]), acc[j + 1]);
+          acc[j + 2] = fmaf(qq.z, __uint_as_float(y[j + 2]), acc[j + 2]);
+          acc[j + 3] = fmaf(qq.w, __uint_as_float(y[j + 3]), acc[j + 3]);
+        }
       }
       if (!ok) break;
       // normaliser tile: rows 0..63 hold b, reduce over them -> ninter[t][8]
@@ -411,59 +506,64 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           *reinterpret_cast<float4*>(red + rowl * RED_STRIDE + t4) =
               make_float4(acc[t4], acc[t4 + 1], acc[t4 + 2], acc[t4 + 3]);
       }
-      group_sync(3);
+      // ---- intra-chunk: P = s^2 / ||k||^2 (causal) -> bf16 into the ring slot ----
+      const int gp = c * NI + 5;
+      ok = wait_or_abort(sm.bar(BAR_RFULL + (gp & 1)), (gp >> 1) & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      if (rowl < 64) {
+        uint32_t sc[C];
+        {
+          uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sc[0]);
+          uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sc[32]);
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64), s0);
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64 + 32), s1);
+          tmem_wait_ld();
+        }
+        uint32_t pk[32];
+#pragma unroll
+        for (int j = 0; j < C; j += 4) {
+          const float4 rr = *reinterpret_cast<const float4*>(r2 + j);
+          const float s0 = __uint_as_float(sc[j]), s1 = __uint_as_float(sc[j + 1]);
+          const float s2 = __uint_as_float(sc[j + 2]), s3 = __uint_as_float(sc[j + 3]);
+          const float w0 = (j <= rowl) ? s0 * s0 * rr.x : 0.f;
+          const float w1 = (j + 1 <= rowl) ? s1 * s1 * rr.y : 0.f;
+          const float w2 = (j + 2 <= rowl) ? s2 * s2 * rr.z : 0.f;
+          const float w3 = (j + 3 <= rowl) ? s3 * s3 * rr.w : 0.f;
+          pk[j / 2] = pack_bf16(w0, w1);
+          pk[j / 2 + 1] = pack_bf16(w2, w3);
+        }
+        tmem_st32(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64), pk);
+        tmem_wait_st();
+      }
+      tc_fence_before();
+      mbar_arrive(sm.bar(BAR_PREADY));
+      group_sync(3);                      // red rows 0..63 (normaliser partials) are complete
       if (tr < C) {
         float sum = 0.f;
 #pragma unroll 16
         for (int r = 0; r < 64; ++r) sum += red[r * RED_STRIDE + tr];
         ninter[tr * 9 + 8] = sum;
       }
-      // ---- intra-chunk: P = s^2 / ||k||^2 (causal), N_intra = P V, D_intra = P 1 ----
-      ok = wait_or_abort(sm.bar(BAR_PFULL), c & 1, abort_flag);
+      // ---- [N_intra | D_intra] from the MMA ----
+      ok = wait_or_abort(sm.bar(BAR_PVFULL), c & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       if (rowl < 64) {
-        float nacc[VS];
+        uint32_t pv[16];
+        tmem_ld16(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64 + 32), pv);
+        tmem_wait_ld();
 #pragma unroll
-        for (int v = 0; v < VS; ++v) nacc[v] = 0.f;
-        float dacc = 0.f;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t sc[32];
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_P + half * 32), sc);
-          tmem_wait_ld();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int i2 = half * 32 + j;
-            const float sv = __uint_as_float(sc[j]);
-            const float w = (i2 <= rowl) ? sv * sv * r2[i2] : 0.f;
-            dacc += w;
-            const float4 va = *reinterpret_cast<const float4*>(vS + i2 * VS);
-            const float4 vb = *reinterpret_cast<const float4*>(vS + i2 * VS + 4);
-            nacc[0] = fmaf(w, va.x, nacc[0]);
-            nacc[1] = fmaf(w, va.y, nacc[1]);
-            nacc[2] = fmaf(w, va.z, nacc[2]);
-            nacc[3] = fmaf(w, va.w, nacc[3]);
-            nacc[4] = fmaf(w, vb.x, nacc[4]);
-            nacc[5] = fmaf(w, vb.y, nacc[5]);
-            nacc[6] = fmaf(w, vb.z, nacc[6]);
-            nacc[7] = fmaf(w, vb.w, nacc[7]);
-          }
-        }
-#pragma unroll
-        for (int v = 0; v < VS; ++v) nintra[rowl * 9 + v] = nacc[v];
-        nintra[rowl * 9 + 8] = dacc;
-      } else {
-        // lanes 64..127 of the score tile are not used; still order the TMEM access for the arrive below
+        for (int v = 0; v < 9; ++v) nintra[rowl * 9 + v] = __uint_as_float(pv[v]);
       }
       tc_fence_before();
-      mbar_arrive(sm.bar(BAR_PEMPTY));
+      mbar_arrive(sm.bar(BAR_REMPTY + (gp & 1)));
       group_sync(3);
       // ---- gate + normalise epilogue ----
       {
         const int t = tr >> 1, vq = (tr & 1) * 4;
-        const int tg = c * C + t;
-        if (tg < Tlen) {
+        const int tg = (c_begin + c) * C + t;
+        if (tg < args.Tlen) {
           const float den = ninter[t * 9 + 8] + nintra[t * 9 + 8];
           const float inv = den > 0.f ? 1.f / den : 0.f;
           float o[4];
@@ -477,19 +577,35 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       group_sync(3);   // ninter / nintra / red are rewritten in the next chunk
     }
+    // ---- final state of this group (scan pass 1) ----
+    if (ok && args.final_state != nullptr) {
+      ok = wait_or_abort(sm.bar(BAR_DONE), 0, abort_flag);
+      tc_fence_after();
+      if (ok) {
+        float* dst = args.final_state + state_off;
+        for (int cblk = 0; cblk < (NT * 64) / 32; ++cblk) {
+          uint32_t z[32];
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + cblk * 32), z);
+          tmem_wait_ld();
+          float* d = dst + ((size_t)(cblk >> 1) * 128 + rowl) * 64 + (cblk & 1) * 32;
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            *reinterpret_cast<float4*>(d + j) = make_float4(__uint_as_float(z[j]), __uint_as_float(z[j + 1]),
+                                                            __uint_as_float(z[j + 2]), __uint_as_float(z[j + 3]));
+        }
+      }
+    }
   }
 
   // ---------------- teardown ----------------
-  if (!ok && device_status != nullptr) atomicExch(device_status, (int)KATA_ERR_DEVICE_TIMEOUT);
+  if (!ok && args.device_status != nullptr) atomicExch(args.device_status, (int)KATA_ERR_DEVICE_TIMEOUT);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   if (warp == 1 && lane == 0) {
     // make sure no MMA is still in flight before TMEM is released
-    mbar_init(sm.bar(BAR_COUNT), 1);
-    fence_mbar_init();
-    mma_commit(sm.bar(BAR_COUNT));
-    mbar_wait(sm.bar(BAR_COUNT), 0);
+    mma_commit(sm.bar(BAR_DRAIN));
+    mbar_wait(sm.bar(BAR_DRAIN), 0);
   }
   __syncthreads();
   if (warp == 0) tmem_dealloc(tb, TMEM_COLS);
@@ -530,13 +646,11 @@ bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T, int box_cols, boo
 
 }  // namespace
 
-size_t tc_chunked_state_elems() { return (size_t)NSLICE * NT * 128 * 64; }
+size_t tc_chunked_state_elems() { return (size_t)NSLICE * STATE_PER_SLICE; }
 int tc_chunked_slices() { return NSLICE; }
 
 void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, int* device_status,
                 LaunchCtx& ctx) {
-  (void)use_scan;
-  (void)ws;
   const int BH = p.B * p.H;
   CUtensorMap tmQ, tmK, tmV;
   if (!make_map(&tmQ, p.q, BH, p.T, 64, true) || !make_map(&tmK, p.k, BH, p.T, 64, true) ||
@@ -550,8 +664,40 @@ void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-  tc_chunk_kernel<<<dim3(NSLICE, BH), NTHREADS, SMEM_ALLOC, ctx.stream>>>(
-      tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.out), p.T, plan.n_chunks, device_status);
+  KernelArgs a;
+  a.out = static_cast<__nv_bfloat16*>(p.out);
+  a.device_status = device_status;
+  a.Tlen = p.T;
+  a.n_chunks = plan.n_chunks;
+  if (!use_scan) {
+    a.init_state = nullptr;
+    a.final_state = nullptr;
+    a.chunks_per_group = plan.n_chunks;
+    a.n_groups = 1;
+    a.write_out = 1;
+    tc_chunk_kernel<<<dim3(NSLICE, BH, 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
+    note_launch(ctx);
+    return;
+  }
+  const int NG = plan.n_groups;
+  const size_t E = tc_chunked_state_elems();
+  float* bufA = ws;
+  float* bufB = ws + (size_t)BH * NG * E;
+  const float* incl = bufA;
+  a.chunks_per_group = plan.chunks_per_group;
+  a.n_groups = NG;
+  if (NG > 1) {
+    a.init_state = nullptr;
+    a.final_state = bufA;
+    a.write_out = 0;
+    tc_chunk_kernel<<<dim3(NSLICE, BH, NG - 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
+    note_launch(ctx);
+    incl = scan_group_states(bufA, bufB, BH, NG, NG - 1, E, ctx);
+  }
+  a.init_state = incl;
+  a.final_state = nullptr;
+  a.write_out = 1;
+  tc_chunk_kernel<<<dim3(NSLICE, BH, NG), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
   note_launch(ctx);
 }
 
