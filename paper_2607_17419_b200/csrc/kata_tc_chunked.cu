@@ -24,8 +24,12 @@
 // the group-local states and stores them; after the log-depth scan over groups a second launch restarts
 // every group from the prefix before it.
 //
-// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 operand builders
-// (norms, tf32 query tile, transposes, W tiles), warps 6-9 TMEM readers (Y reduction, scores, epilogue).
+// Warp roles (384 threads): warp 0 TMA producer; warps 1-3 MMA issuers (one elected lane each; issuer j
+// owns state tiles j and j+3: the read of a tile and then its update, so the write-after-read on the tile
+// is ordered by issue order; issuer 2 also issues the score MMA and the P[V|1] MMA); warps 4-7 operand
+// builders (norms, tf32 query tile, transposes, W tiles); warps 8-11 TMEM readers (Y reduction, scores,
+// epilogue).  Several issuing warps are needed because a thread that has MMAs in flight stalls on its next
+// barrier wait until they drain; with three issuers the tensor pipe stays fed.
 // All hand-offs go through mbarriers with bounded waits; on a timeout the CTA records
 // KATA_ERR_DEVICE_TIMEOUT in *device_status, drains and returns.
 #include <cuda.h>
@@ -44,7 +48,9 @@ constexpr int VS = 8;            // value columns per CTA
 constexpr int NSLICE = D / VS;   // CTAs per head
 constexpr int NT = 5;            // state tiles: 4 x S + the normaliser tile
 constexpr int NI = 6;            // ring items per chunk: 5 reads + the score/intra item
-constexpr int NTHREADS = 320;
+constexpr int NTHREADS = 384;   // 12 warps = 3 per scheduler, which leaves 168 registers per thread
+constexpr int WARP_ISS0 = 1, WARP_BLD0 = 4, WARP_RD0 = 8;   // first warp of each role
+constexpr int NISSUER = 3;
 constexpr size_t STATE_PER_SLICE = (size_t)NT * 128 * 64;   // floats
 
 // TMEM columns (128 lanes each)
@@ -68,25 +74,28 @@ constexpr uint32_t RED_STRIDE = 68;
 constexpr uint32_t OFF_NINTRA = 156288;           // [64][9]
 constexpr uint32_t OFF_NINTER = 158592;           // [64][9]
 constexpr uint32_t OFF_BAR = 160896;              // mbarriers
-constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;  // slack for the 1024-byte alignment
 static_assert(OFF_QF % 1024 == 0 && OFF_QK % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 static_assert(SMEM_ALLOC > 116 * 1024, "one CTA per SM is assumed (the CTA allocates all of TMEM)");
 
+// Barriers are indexed per tile / per ring item, never per buffer: roles run at different speeds, and a
+// buffer-indexed barrier shared by several waiters lets a waiter observe the parity of a phase that is
+// two completions away from the one it means (phase aliasing).  Every barrier below completes exactly
+// once per chunk (stage barriers: once per two chunks) and each waiter waits for every phase in order.
 enum {
   BAR_FULL = 0,     // [2] TMA landed
-  BAR_EMPTY = 2,    // [2] stage free (128 builders + MMA commit)
+  BAR_EMPTY = 2,    // [2] stage free (128 builders + one commit per issuer)
   BAR_PREP = 4,     // [2] operands of the chunk built (128 builders)
-  BAR_WFULL = 6,    // [2] W tile stored to TMEM
-  BAR_WEMPTY = 8,   // [2] W tile consumed by the MMA
-  BAR_RFULL = 10,   // [2] ring item produced by the MMA
-  BAR_REMPTY = 12,  // [2] ring item drained (128 readers)
-  BAR_PREADY = 14,  // P (bf16) stored to TMEM (128 readers)
-  BAR_PVFULL = 15,  // P [V|1] complete
-  BAR_U = 16,       // [5] update of state tile i complete
-  BAR_DRAIN = 21,
-  BAR_DONE = 22,    // every update of this CTA has completed
-  BAR_COUNT = 23
+  BAR_WFULL = 6,    // [5] W tile i stored to TMEM (128 builders)
+  BAR_RFULL = 11,   // [6] ring item i produced by the MMA
+  BAR_REMPTY = 17,  // [6] ring item i drained (128 readers)
+  BAR_PREADY = 23,  // P (bf16) stored to TMEM (128 readers)
+  BAR_PVFULL = 24,  // P [V|1] complete
+  BAR_U = 25,       // [5] update of state tile i complete (frees the W buffer, allows the next read)
+  BAR_DRAIN = 30,
+  BAR_DONE = 31,    // every update of this CTA has completed
+  BAR_COUNT = 32
 };
 
 struct Shared {
@@ -154,26 +163,29 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     abort_s = 0;
     for (int i = 0; i < 2; ++i) {
       mbar_init(sm.bar(BAR_FULL + i), 1);
-      mbar_init(sm.bar(BAR_EMPTY + i), 129);
+      mbar_init(sm.bar(BAR_EMPTY + i), 128 + NISSUER);
       mbar_init(sm.bar(BAR_PREP + i), 128);
+    }
+    for (int i = 0; i < NT; ++i) {
       mbar_init(sm.bar(BAR_WFULL + i), 128);
-      mbar_init(sm.bar(BAR_WEMPTY + i), 1);
+      mbar_init(sm.bar(BAR_U + i), 1);
+    }
+    for (int i = 0; i < NI; ++i) {
       mbar_init(sm.bar(BAR_RFULL + i), 1);
       mbar_init(sm.bar(BAR_REMPTY + i), 128);
     }
     mbar_init(sm.bar(BAR_PREADY), 128);
     mbar_init(sm.bar(BAR_PVFULL), 1);
-    for (int i = 0; i < NT; ++i) mbar_init(sm.bar(BAR_U + i), 1);
-    mbar_init(sm.bar(BAR_DRAIN), 1);
-    mbar_init(sm.bar(BAR_DONE), 1);
+    mbar_init(sm.bar(BAR_DRAIN), NISSUER);
+    mbar_init(sm.bar(BAR_DONE), NISSUER);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmV);
   }
   // constant "ones" column group for the intra-chunk MMA: row t = (1, 0, 0, 0, 0, 0, 0, 0) in bf16
-  if (tid >= 64 && tid < 128) {
-    *reinterpret_cast<uint4*>(sm.ones() + (tid - 64) * 16) = make_uint4(0x00003F80u, 0u, 0u, 0u);
+  if (tid < 64) {
+    *reinterpret_cast<uint4*>(sm.ones() + tid * 16) = make_uint4(0x00003F80u, 0u, 0u, 0u);
     fence_async_smem();
   }
   if (warp == 0) {
@@ -186,7 +198,7 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t tb = tmem_base_s;
 
   // initial state: zero, or the prefix of the groups before this one (readers own the TMEM lanes)
-  if (warp >= 6) {
+  if (warp >= WARP_RD0) {
     const uint32_t q4 = warp & 3;
     const int rowl = q4 * 32 + lane;
     uint32_t z[32];
@@ -230,33 +242,74 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tma_load_3d(sm.vtile(s), &tmV, sm.bar(BAR_FULL + s), slice * VS, t0, bh);
       }
     }
-  } else if (warp == 1) {
-    // =========================== MMA issuer ===========================
+  } else if (warp < WARP_BLD0) {
+    // =========================== MMA issuers ===========================
     if (lane == 0) {
+      const int j = warp - WARP_ISS0;            // issuer index = state tile it owns
       const uint32_t id_read = instr_desc(kFmtTF32, kFmtTF32, 0, 0, 128, 64);    // A tmem (fp32 as tf32), B K-major
       const uint32_t id_qk = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 64);      // both K-major from smem
       const uint32_t id_upd = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 64);     // A tmem, B MN-major
       const uint32_t id_pv = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 16);      // A tmem, B MN-major, N = 16
-      // descriptors that depend only on the stage
-      uint64_t d_qf[2][8], d_q[2][4], d_k[2][4], d_kmn[2][4], d_v[2][4];
-#pragma unroll
-      for (int s = 0; s < 2; ++s) {
-        const uint32_t qf = smem_u32(sm.qf(s)), qa = smem_u32(sm.qtile(s)), ka = smem_u32(sm.ktile(s));
-        const uint32_t va = smem_u32(sm.vtile(s));
-        const uint32_t ones_off = smem_u32(sm.ones()) - va;
+      const uint64_t d_k128 = smem_desc(0, 16, 1024, kSwizzle128B);              // K-major, 128B swizzle
+      const uint64_t d_mn128 = smem_desc(0, 8192, 1024, kSwizzle128B);           // MN-major, 128B swizzle
+      auto at = [](uint64_t d, uint32_t addr) { return d + (uint64_t)((addr >> 4) & 0x3FFF); };
+
+      // Y_i = S_i * Q^T (tf32, A = accumulators in TMEM) into ring item (c, i)
+      auto issue_read = [&](int c, int i) {
+        const int g = c * NI + i;
+        // the ring slot (g & 1) is free once its previous occupant, item g - 2, has been drained
+        if (g >= 2) ok = wait_or_abort(sm.bar(BAR_REMPTY + (g - 2) % NI), ((g - 2) / NI) & 1, abort_flag);
+        if (ok && c > 0) ok = wait_or_abort(sm.bar(BAR_U + i), (c - 1) & 1, abort_flag);
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t qf = smem_u32(sm.qf(c & 1));
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          d_qf[s][ks] = smem_desc(qf + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, kSwizzle128B);
+          mma_tf32_ts(tb + COL_R + (g & 1) * 64, tb + COL_S + i * 64 + ks * 8,
+                      at(d_k128, qf + (ks >> 2) * 8192 + (ks & 3) * 32), id_read, ks > 0);
+        mma_commit(sm.bar(BAR_RFULL + i));
+      };
+      // S_i += W_i * K (A = W in TMEM, B = key tile MN-major)
+      auto issue_update = [&](int c, int i) {
+        const int g = c * NT + i;
+        ok = wait_or_abort(sm.bar(BAR_WFULL + i), c & 1, abort_flag);
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t ka = smem_u32(sm.ktile(c & 1));
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          d_q[s][ks] = smem_desc(qa + ks * 32, 16, 1024, kSwizzle128B);
-          d_k[s][ks] = smem_desc(ka + ks * 32, 16, 1024, kSwizzle128B);
-          d_kmn[s][ks] = smem_desc(ka + ks * 2048, 8192, 1024, kSwizzle128B);
-          // [V | ones]: MN-major, no swizzle: 8 k-rows x 16 bytes per core matrix, next 8 k at +128 (LBO),
-          // second group of 8 columns (the ones group) at +ones_off (SBO)
-          d_v[s][ks] = smem_desc(va + ks * 256, 128, ones_off, kSwizzleNone);
-        }
-      }
+        for (int ks = 0; ks < 4; ++ks)
+          mma_f16_ts(tb + COL_S + i * 64, tb + COL_W + (g & 1) * 32 + ks * 8, at(d_mn128, ka + ks * 2048), id_upd, 1u);
+        mma_commit(sm.bar(BAR_U + i));
+      };
+      // intra-chunk scores [Q;K] K^T into ring item (c, 5) (rows 0..63 used)
+      auto issue_qk = [&](int c) {
+        const int g = c * NI + 5;
+        ok = wait_or_abort(sm.bar(BAR_REMPTY + 3), c & 1, abort_flag);     // item (c, 3) shared the slot
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t qa = smem_u32(sm.qtile(c & 1)), ka = smem_u32(sm.ktile(c & 1));
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          mma_f16_ss(tb + COL_R + (g & 1) * 64, at(d_k128, qa + ks * 32), at(d_k128, ka + ks * 32), id_qk, ks > 0);
+        mma_commit(sm.bar(BAR_RFULL + 5));
+      };
+      // [N_intra | D_intra] = P [V | 1] (A = P bf16 in the ring slot; B = the value tile and the ones group)
+      auto issue_pv = [&](int c) {
+        const int g = c * NI + 5;
+        ok = wait_or_abort(sm.bar(BAR_PREADY), c & 1, abort_flag);
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t va = smem_u32(sm.vtile(c & 1));
+        const uint32_t ones_off = smem_u32(sm.ones()) - va;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          // MN-major, no swizzle: 8 k-rows x 16 bytes per core matrix, next 8 k at +128 (LBO), the second
+          // group of 8 columns (the ones group) at +ones_off (SBO)
+          mma_f16_ts(tb + COL_R + (g & 1) * 64 + 32, tb + COL_R + (g & 1) * 64 + ks * 8,
+                     smem_desc(va + ks * 256, 128, ones_off, kSwizzleNone), id_pv, ks > 0);
+        mma_commit(sm.bar(BAR_PVFULL));
+      };
+
       for (int c = 0; c < nloc && ok; ++c) {
         const int s = c & 1;
         const uint32_t ph = (c >> 1) & 1;
@@ -264,63 +317,23 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
              wait_or_abort(sm.bar(BAR_PREP + s), ph, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        if (write_out) {
-          // ---- inter-chunk reads Y_i = S_i * Q^T (tf32, A = accumulators in TMEM) ----
-          for (int i = 0; i < NT && ok; ++i) {
-            const int g = c * NI + i;
-            ok = wait_or_abort(sm.bar(BAR_REMPTY + (g & 1)), ((g >> 1) & 1) ^ 1, abort_flag);
-            if (ok && c > 0) ok = wait_or_abort(sm.bar(BAR_U + i), (c - 1) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-              mma_tf32_ts(tb + COL_R + (g & 1) * 64, tb + COL_S + i * 64 + ks * 8, d_qf[s][ks], id_read, ks > 0);
-            mma_commit(sm.bar(BAR_RFULL + (g & 1)));
-          }
-          if (!ok) break;
-          // ---- intra-chunk scores [Q;K] K^T (rows 0..63 used) ----
-          {
-            const int g = c * NI + 5;
-            ok = wait_or_abort(sm.bar(BAR_REMPTY + (g & 1)), ((g >> 1) & 1) ^ 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              mma_f16_ss(tb + COL_R + (g & 1) * 64, d_q[s][ks], d_k[s][ks], id_qk, ks > 0);
-            mma_commit(sm.bar(BAR_RFULL + (g & 1)));
-          }
-        }
-        // ---- state updates S_i += W_i * K (A = W in TMEM) ----
-        for (int i = 0; i < NT && ok; ++i) {
-          const int g = c * NT + i;
-          ok = wait_or_abort(sm.bar(BAR_WFULL + (g & 1)), (g >> 1) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            mma_f16_ts(tb + COL_S + i * 64, tb + COL_W + (g & 1) * 32 + ks * 8, d_kmn[s][ks], id_upd, 1u);
-          mma_commit(sm.bar(BAR_WEMPTY + (g & 1)));
-          mma_commit(sm.bar(BAR_U + i));
+        if (write_out) issue_read(c, j);
+        if (ok) issue_update(c, j);
+        if (j < 2) {
+          if (ok && write_out) issue_read(c, j + 3);
+          if (ok) issue_update(c, j + 3);
+        } else if (write_out) {
+          if (ok) issue_qk(c);
+          if (ok) issue_pv(c);
         }
         if (!ok) break;
-        if (write_out) {
-          // ---- [N_intra | D_intra] = P [V | 1] (A = P bf16 in the ring slot) ----
-          const int g = c * NI + 5;
-          ok = wait_or_abort(sm.bar(BAR_PREADY), c & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            mma_f16_ts(tb + COL_R + (g & 1) * 64 + 32, tb + COL_R + (g & 1) * 64 + ks * 8, d_v[s][ks], id_pv, ks > 0);
-          mma_commit(sm.bar(BAR_PVFULL));
-        }
         mma_commit(sm.bar(BAR_EMPTY + s));
       }
       if (ok) mma_commit(sm.bar(BAR_DONE));
     }
-  } else if (warp < 6) {
+  } else if (warp < WARP_RD0) {
     // =========================== operand builders (128 threads) ===========================
-    const int ta = tid - 64;
+    const int ta = tid - WARP_BLD0 * 32;
     const int row = ta >> 1, hf = ta & 1;          // prep mapping: two threads per token row
     const uint32_t q4 = warp & 3;                  // TMEM lane quadrant of this warp
     const int rowl = q4 * 32 + lane;               // W-tile row owned by this thread
@@ -402,9 +415,12 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // ---- W tiles: row rowl <-> (b = 16 i + rowl/8, v = rowl%8); fifth tile: rows < 64 hold k[t,b]/||k||^2 ----
       for (int i = 0; i < NT && ok; ++i) {
         const int g = c * NT + i;
-        ok = wait_or_abort(sm.bar(BAR_WEMPTY + (g & 1)), ((g >> 1) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
+        if (g >= 2) {   // the W buffer is free once the update two tiles back has completed
+          const int gp = g - 2;
+          ok = wait_or_abort(sm.bar(BAR_U + gp % NT), (gp / NT) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+        }
         const float* krow = kT + ((i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63)) * KT_STRIDE;
         uint32_t pk[32];
         if (i < 4) {
@@ -427,14 +443,14 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tmem_st32(tmem_addr(tb, q4 * 32, COL_W + (g & 1) * 32), pk);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(sm.bar(BAR_WFULL + (g & 1)));
+        mbar_arrive(sm.bar(BAR_WFULL + i));
       }
       if (!ok) break;
       mbar_arrive(sm.bar(BAR_EMPTY + s));     // done with the stage (the MMA adds its own arrival)
     }
   } else {
     // =========================== TMEM readers (128 threads) ===========================
-    const int tr = tid - 192;                  // 0..127
+    const int tr = tid - WARP_RD0 * 32;        // 0..127
     const uint32_t q4 = warp & 3;              // TMEM lane quadrant this warp may access
     const int rowl = q4 * 32 + lane;           // tile row (= TMEM lane) of this thread
     float* red = sm.red();
@@ -452,16 +468,9 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       for (int t = 0; t < C; ++t) acc[t] = 0.f;
       for (int i = 0; i < NT && ok; ++i) {
         const int g = c * NI + i;
-        ok = wait_or_abort(sm.bar(BAR_RFULL + (g & 1)), (g >> 1) & 1, abort_flag);
+        ok = wait_or_abort(sm.bar(BAR_RFULL + i), c & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        uint32_t y[C];
-        {
-          uint32_t(&y0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&y[0]);
-          uint32_t(&y1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&y[32]);
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (g & 1) * 64), y0);
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (g & 1) * 64 + 32), y1);
-        }
         if (i == 4) {
           // the four state tiles are in acc: reduce over b within the CTA -> ninter[t][v]
 #pragma unroll
@@ -486,16 +495,23 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         const int b = (i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63);
         const float* qrow = qT + b * C;
-        tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(sm.bar(BAR_REMPTY + (g & 1)));      // the slot is in registers now
 #pragma unroll
-        for (int j = 0; j < C; j += 4) {
-          const float4 qq = *reinterpret_cast<const float4*>(qrow + j);
-          acc[j] = fmaf(qq.x, __uint_as_float(y[j]), acc[j]);
-          acc[j + 1] = fmaf(qq.y, __uint_as_float(y[j + 1]), acc[j + 1]);
-          acc[j + 2] = fmaf(qq.z, __uint_as_float(y[j + 2]), acc[j + 2]);
-          acc[j + 3] = fmaf(qq.w, __uint_as_float(y[j + 3]), acc[j + 3]);
+        for (int half = 0; half < 2; ++half) {
+          uint32_t y[32];
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (g & 1) * 64 + half * 32), y);
+          tmem_wait_ld();
+          if (half == 1) {
+            tc_fence_before();
+            mbar_arrive(sm.bar(BAR_REMPTY + i));      // the slot is in registers now
+          }
+#pragma unroll
+          for (int jj = 0; jj < 32; jj += 4) {
+            const float4 qq = *reinterpret_cast<const float4*>(qrow + half * 32 + jj);
+            acc[half * 32 + jj] = fmaf(qq.x, __uint_as_float(y[jj]), acc[half * 32 + jj]);
+            acc[half * 32 + jj + 1] = fmaf(qq.y, __uint_as_float(y[jj + 1]), acc[half * 32 + jj + 1]);
+            acc[half * 32 + jj + 2] = fmaf(qq.z, __uint_as_float(y[jj + 2]), acc[half * 32 + jj + 2]);
+            acc[half * 32 + jj + 3] = fmaf(qq.w, __uint_as_float(y[jj + 3]), acc[half * 32 + jj + 3]);
+          }
         }
       }
       if (!ok) break;
@@ -508,30 +524,30 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       // ---- intra-chunk: P = s^2 / ||k||^2 (causal) -> bf16 into the ring slot ----
       const int gp = c * NI + 5;
-      ok = wait_or_abort(sm.bar(BAR_RFULL + (gp & 1)), (gp >> 1) & 1, abort_flag);
+      ok = wait_or_abort(sm.bar(BAR_RFULL + 5), c & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       if (rowl < 64) {
-        uint32_t sc[C];
-        {
-          uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sc[0]);
-          uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sc[32]);
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64), s0);
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64 + 32), s1);
-          tmem_wait_ld();
-        }
+        // scores of both halves are read before the packed P overwrites columns [0,32) of the slot
         uint32_t pk[32];
 #pragma unroll
-        for (int j = 0; j < C; j += 4) {
-          const float4 rr = *reinterpret_cast<const float4*>(r2 + j);
-          const float s0 = __uint_as_float(sc[j]), s1 = __uint_as_float(sc[j + 1]);
-          const float s2 = __uint_as_float(sc[j + 2]), s3 = __uint_as_float(sc[j + 3]);
-          const float w0 = (j <= rowl) ? s0 * s0 * rr.x : 0.f;
-          const float w1 = (j + 1 <= rowl) ? s1 * s1 * rr.y : 0.f;
-          const float w2 = (j + 2 <= rowl) ? s2 * s2 * rr.z : 0.f;
-          const float w3 = (j + 3 <= rowl) ? s3 * s3 * rr.w : 0.f;
-          pk[j / 2] = pack_bf16(w0, w1);
-          pk[j / 2 + 1] = pack_bf16(w2, w3);
+        for (int half = 0; half < 2; ++half) {
+          uint32_t sc[32];
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64 + half * 32), sc);
+          tmem_wait_ld();
+#pragma unroll
+          for (int jj = 0; jj < 32; jj += 4) {
+            const int j = half * 32 + jj;
+            const float4 rr = *reinterpret_cast<const float4*>(r2 + j);
+            const float s0 = __uint_as_float(sc[jj]), s1 = __uint_as_float(sc[jj + 1]);
+            const float s2 = __uint_as_float(sc[jj + 2]), s3 = __uint_as_float(sc[jj + 3]);
+            const float w0 = (j <= rowl) ? s0 * s0 * rr.x : 0.f;
+            const float w1 = (j + 1 <= rowl) ? s1 * s1 * rr.y : 0.f;
+            const float w2 = (j + 2 <= rowl) ? s2 * s2 * rr.z : 0.f;
+            const float w3 = (j + 3 <= rowl) ? s3 * s3 * rr.w : 0.f;
+            pk[j / 2] = pack_bf16(w0, w1);
+            pk[j / 2 + 1] = pack_bf16(w2, w3);
+          }
         }
         tmem_st32(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64), pk);
         tmem_wait_st();
@@ -557,7 +573,7 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int v = 0; v < 9; ++v) nintra[rowl * 9 + v] = __uint_as_float(pv[v]);
       }
       tc_fence_before();
-      mbar_arrive(sm.bar(BAR_REMPTY + (gp & 1)));
+      mbar_arrive(sm.bar(BAR_REMPTY + 5));
       group_sync(3);
       // ---- gate + normalise epilogue ----
       {
@@ -602,7 +618,7 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (warp == 1 && lane == 0) {
+  if (warp >= WARP_ISS0 && warp < WARP_BLD0 && lane == 0) {
     // make sure no MMA is still in flight before TMEM is released
     mma_commit(sm.bar(BAR_DRAIN));
     mbar_wait(sm.bar(BAR_DRAIN), 0);

@@ -13,7 +13,7 @@
 namespace kata {
 namespace umma {
 
-constexpr uint32_t kSpinLimit = 1u << 24;   // polls of ~20-40 ns each before a wait gives up
+constexpr uint32_t kSpinLimit = 1u << 22;   // polls of ~20-40 ns each (~0.1 s) before a wait gives up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
