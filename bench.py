@@ -288,6 +288,31 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_small(args):
+    """Profiler case: the chunked forward on B=1, H=16, T=32768 (inputs 201 MB > L2, well under a GB)."""
+    import numpy as np
+    import torch
+    from paper_2607_17419_b200 import binding as kb, build as kbuild, inputs
+    kbuild.build()
+    torch.cuda.set_device(0)
+    w = inputs.gaussian_workload("c4_T32768", "bf16", 1, 16, 32768, 64, 64, 64, 3)
+    q, k, v = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda() for a in (w.q_dev, w.k_dev, w.v_dev))
+    out = torch.empty_like(v)
+    inter = kb.KATA_SCAN if args.mode == "scan" else kb.KATA_SEQUENTIAL
+    for _ in range(args.warmup):
+        kb.kata_fwd_chunked(q, k, v, out, inter_chunk=inter)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        kb.kata_fwd_chunked(q, k, v, out, inter_chunk=inter)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    print(json.dumps(dict(case="small", T=32768, ms_per_step=ms, tokens_per_s=32768 / (ms * 1e-3),
+                          impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")))
+
+
 def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
     """Separately timed secondary figures: scan forms on the same workload, quadratic form on config 2."""
     import numpy as np
@@ -331,8 +356,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="sequential", choices=["sequential", "scan"])
     ap.add_argument("--no-extra", dest="extra", action="store_false")
+    ap.add_argument("--case", default="full", choices=["full", "small"],
+                    help="small: the same kernel on T=32768 only (for profiler captures); prints a short line")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.case == "small":
+        run_small(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -24,11 +24,11 @@
 // the group-local states and stores them; after the log-depth scan over groups a second launch restarts
 // every group from the prefix before it.
 //
-// Warp roles (384 threads): warp 0 TMA producer; warps 1-3 MMA issuers (one elected lane each; issuer j
+// Warp roles (512 threads): warp 0 TMA producer; warps 1-3 MMA issuers (one elected lane each; issuer j
 // owns state tiles j and j+3: the read of a tile and then its update, so the write-after-read on the tile
 // is ordered by issue order; issuer 2 also issues the score MMA and the P[V|1] MMA); warps 4-7 operand
-// builders (norms, tf32 query tile, transposes, W tiles); warps 8-11 TMEM readers (Y reduction, scores,
-// epilogue).  Several issuing warps are needed because a thread that has MMAs in flight stalls on its next
+// builders (norms, tf32 query tile, transposes, W tiles); warps 8-15 TMEM readers in two groups (Y
+// reduction, scores, epilogue).  Several issuing warps are needed because a thread that has MMAs in flight stalls on its next
 // barrier wait until they drain; with three issuers the tensor pipe stays fed.
 // All hand-offs go through mbarriers with bounded waits; on a timeout the CTA records
 // KATA_ERR_DEVICE_TIMEOUT in *device_status, drains and returns.
@@ -48,7 +48,7 @@ constexpr int VS = 8;            // value columns per CTA
 constexpr int NSLICE = D / VS;   // CTAs per head
 constexpr int NT = 5;            // state tiles: 4 x S + the normaliser tile
 constexpr int NI = 6;            // ring items per chunk: 5 reads + the score/intra item
-constexpr int NTHREADS = 384;   // 12 warps = 3 per scheduler, which leaves 168 registers per thread
+constexpr int NTHREADS = 512;   // 16 warps = 4 per scheduler: 128 registers per thread
 constexpr int WARP_ISS0 = 1, WARP_BLD0 = 4, WARP_RD0 = 8;   // first warp of each role
 constexpr int NISSUER = 3;
 constexpr size_t STATE_PER_SLICE = (size_t)NT * 128 * 64;   // floats
@@ -60,20 +60,19 @@ constexpr uint32_t COL_W = 448;    // 2 x 32: W tiles (bf16 pairs), A operand of
 constexpr uint32_t TMEM_COLS = 512;
 
 // shared memory map (bytes from a 1024-aligned base)
-constexpr uint32_t KT_STRIDE = 68;                // floats per kT / vT row (16-byte aligned, conflict-free LDS.128)
+constexpr uint32_t KT_STRIDE = 144;               // bytes per kT / vT row: 64 bf16 + 16 pad (conflict-free LDS.128)
 constexpr uint32_t OFF_QK = 0;                    // 2 stages x (Q tile 8 KB, K tile 8 KB), TMA, 128B swizzle
 constexpr uint32_t OFF_V = 32768;                 // 2 stages x 64 x 8 bf16 (TMA, dense 16-byte rows)
 constexpr uint32_t OFF_ONES = 34816;              // 64 x 8 bf16 rows (1,0,..,0): the "ones" column group
 constexpr uint32_t OFF_QF = 35840;                // 2 x 16 KB: query tile as tf32, K-major, 128B swizzle, 2 atoms
-constexpr uint32_t OFF_KT = 68608;                // kT[b][t] fp32, stride 68 (builders only)
-constexpr uint32_t OFF_VT = 86016;                // vT[v][t] = v / ||k||^2, fp32, stride 68 (builders only)
+constexpr uint32_t OFF_KT = 68608;                // kT[b][t] bf16, 64 rows (builders only)
+constexpr uint32_t OFF_VT = 86016;                // vT[v][t] = bf16(v / ||k||^2), row 8 = bf16(1 / ||k||^2) (builders only)
 constexpr uint32_t OFF_QT = 88192;                // 2 x qT[b][t] fp32 (readers)
 constexpr uint32_t OFF_R2 = 120960;               // 2 x r2[t] = 1/||k_t||^2
-constexpr uint32_t OFF_RED = 121472;              // red[128][68] fp32 cross-lane reduction scratch
+constexpr uint32_t OFF_RED = 121472;              // red[128+128+64][68] fp32: per-group state partials, normaliser partials
 constexpr uint32_t RED_STRIDE = 68;
-constexpr uint32_t OFF_NINTRA = 156288;           // [64][9]
-constexpr uint32_t OFF_NINTER = 158592;           // [64][9]
-constexpr uint32_t OFF_BAR = 160896;              // mbarriers
+constexpr uint32_t OFF_NINTRA = 208512;           // [64][9]
+constexpr uint32_t OFF_BAR = 210816;              // mbarriers
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;  // slack for the 1024-byte alignment
 static_assert(OFF_QF % 1024 == 0 && OFF_QK % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -105,17 +104,17 @@ struct Shared {
   __device__ unsigned char* vtile(int s) const { return base + OFF_V + s * 1024; }
   __device__ unsigned char* ones() const { return base + OFF_ONES; }
   __device__ unsigned char* qf(int s) const { return base + OFF_QF + s * 16384; }
-  __device__ float* kT() const { return reinterpret_cast<float*>(base + OFF_KT); }
-  __device__ float* vT() const { return reinterpret_cast<float*>(base + OFF_VT); }
+  __device__ unsigned char* kT() const { return base + OFF_KT; }
+  __device__ unsigned char* vT() const { return base + OFF_VT; }
   __device__ float* qT(int s) const { return reinterpret_cast<float*>(base + OFF_QT + s * 16384); }
   __device__ float* r2(int s) const { return reinterpret_cast<float*>(base + OFF_R2 + s * 256); }
   __device__ float* red() const { return reinterpret_cast<float*>(base + OFF_RED); }
   __device__ float* nintra() const { return reinterpret_cast<float*>(base + OFF_NINTRA); }
-  __device__ float* ninter() const { return reinterpret_cast<float*>(base + OFF_NINTER); }
   __device__ uint64_t* bar(int i) const { return reinterpret_cast<uint64_t*>(base + OFF_BAR) + i; }
 };
 
 __device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+__device__ __forceinline__ void reader_sync() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
 
 // Bounded wait that also gives up as soon as another role has flagged an abort.
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -125,6 +124,12 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
   }
   *abort_flag = 1;
   return false;
+}
+
+// element-wise product of two packed bf16 pairs (one HMUL2.BF16)
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+  const __nv_bfloat162 r = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+  return *reinterpret_cast<const uint32_t*>(&r);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -198,7 +203,7 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t tb = tmem_base_s;
 
   // initial state: zero, or the prefix of the groups before this one (readers own the TMEM lanes)
-  if (warp >= WARP_RD0) {
+  if (warp >= WARP_RD0 && warp < WARP_RD0 + 4) {
     const uint32_t q4 = warp & 3;
     const int rowl = q4 * 32 + lane;
     uint32_t z[32];
@@ -337,8 +342,8 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int row = ta >> 1, hf = ta & 1;          // prep mapping: two threads per token row
     const uint32_t q4 = warp & 3;                  // TMEM lane quadrant of this warp
     const int rowl = q4 * 32 + lane;               // W-tile row owned by this thread
-    float* kT = sm.kT();
-    float* vT = sm.vT();
+    unsigned char* kT = sm.kT();
+    unsigned char* vT = sm.vT();
     for (int c = 0; c < nloc && ok; ++c) {
       const int s = c & 1;
       ok = wait_or_abort(sm.bar(BAR_FULL + s), (c >> 1) & 1, abort_flag);
@@ -346,7 +351,7 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       group_sync(2);   // every builder is done with kT / vT of the previous chunk
       float* qT = sm.qT(s);
       float* r2 = sm.r2(s);
-      // ---- phase 1: key norms, kT, tf32 query tile, qT ----
+      // ---- phase 1: key norms, kT (bf16), tf32 query tile, qT ----
       {
         const unsigned char* kt = sm.ktile(s);
         const unsigned char* qt = sm.qtile(s);
@@ -357,16 +362,13 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const int chunk = hf * 4 + j;
           const uint4 kraw = *reinterpret_cast<const uint4*>(kt + sw128_offset(row, chunk));
           const uint32_t kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
-          float kf[8];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            kf[2 * e] = __uint_as_float(kw[e] << 16);
-            kf[2 * e + 1] = __uint_as_float(kw[e] & 0xFFFF0000u);
-          }
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            ss = fmaf(kf[e], kf[e], ss);
-            kT[(chunk * 8 + e) * KT_STRIDE + row] = kf[e];
+            const float lo = __uint_as_float(kw[e] << 16), hi = __uint_as_float(kw[e] & 0xFFFF0000u);
+            ss = fmaf(lo, lo, ss);
+            ss = fmaf(hi, hi, ss);
+            *reinterpret_cast<uint16_t*>(kT + (chunk * 8 + 2 * e) * KT_STRIDE + row * 2) = (uint16_t)(kw[e] & 0xFFFFu);
+            *reinterpret_cast<uint16_t*>(kT + (chunk * 8 + 2 * e + 1) * KT_STRIDE + row * 2) = (uint16_t)(kw[e] >> 16);
           }
           if (write_out) {
             const uint4 qraw = *reinterpret_cast<const uint4*>(qt + sw128_offset(row, chunk));
@@ -388,31 +390,34 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (hf == 0) r2[row] = inv_or_zero(ss);
       }
       group_sync(2);
-      // ---- phase 2: scaled transposed values for the W tiles ----
+      // ---- phase 2: transposed values scaled by 1/||k||^2 (bf16); row 8 is the scale itself ----
       if (ta < C) {
         const uint4 vraw = *reinterpret_cast<const uint4*>(sm.vtile(s) + ta * 16);
         const uint32_t vw[4] = {vraw.x, vraw.y, vraw.z, vraw.w};
         const float rr = r2[ta];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          vT[(2 * e) * KT_STRIDE + ta] = __uint_as_float(vw[e] << 16) * rr;
-          vT[(2 * e + 1) * KT_STRIDE + ta] = __uint_as_float(vw[e] & 0xFFFF0000u) * rr;
+          const uint32_t p2 = pack_bf16(__uint_as_float(vw[e] << 16) * rr, __uint_as_float(vw[e] & 0xFFFF0000u) * rr);
+          *reinterpret_cast<uint16_t*>(vT + (2 * e) * KT_STRIDE + ta * 2) = (uint16_t)(p2 & 0xFFFFu);
+          *reinterpret_cast<uint16_t*>(vT + (2 * e + 1) * KT_STRIDE + ta * 2) = (uint16_t)(p2 >> 16);
         }
+        *reinterpret_cast<uint16_t*>(vT + 8 * KT_STRIDE + ta * 2) = (uint16_t)(pack_bf16(rr, 0.f) & 0xFFFFu);
       }
       fence_async_smem();
       group_sync(2);
       mbar_arrive(sm.bar(BAR_PREP + s));
-      // the value row of this thread (v = rowl % 8), scaled by 1/||k||^2, for all 64 tokens
-      float vr[C];
+      // the scaled value row of this thread (v = rowl % 8) as 32 bf16 pairs
+      uint32_t vr[32];
       {
-        const float* vrow = vT + (rowl & 7) * KT_STRIDE;
+        const unsigned char* vrow = vT + (rowl & 7) * KT_STRIDE;
 #pragma unroll
-        for (int t4 = 0; t4 < C; t4 += 4) {
-          const float4 f = *reinterpret_cast<const float4*>(vrow + t4);
-          vr[t4] = f.x; vr[t4 + 1] = f.y; vr[t4 + 2] = f.z; vr[t4 + 3] = f.w;
+        for (int j = 0; j < 8; ++j) {
+          const uint4 f = *reinterpret_cast<const uint4*>(vrow + j * 16);
+          vr[4 * j] = f.x; vr[4 * j + 1] = f.y; vr[4 * j + 2] = f.z; vr[4 * j + 3] = f.w;
         }
       }
-      // ---- W tiles: row rowl <-> (b = 16 i + rowl/8, v = rowl%8); fifth tile: rows < 64 hold k[t,b]/||k||^2 ----
+      // ---- W tiles: row rowl <-> (b = 16 i + rowl/8, v = rowl%8); fifth tile: rows < 64 hold k[t,b]/||k||^2.
+      //      One packed bf16 multiply per token pair; the products go straight to TMEM. ----
       for (int i = 0; i < NT && ok; ++i) {
         const int g = c * NT + i;
         if (g >= 2) {   // the W buffer is free once the update two tiles back has completed
@@ -421,23 +426,28 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (!ok) break;
           tc_fence_after();
         }
-        const float* krow = kT + ((i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63)) * KT_STRIDE;
+        const unsigned char* krow = kT + ((i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63)) * KT_STRIDE;
         uint32_t pk[32];
         if (i < 4) {
 #pragma unroll
-          for (int t4 = 0; t4 < C; t4 += 4) {
-            const float4 kk = *reinterpret_cast<const float4*>(krow + t4);
-            pk[t4 / 2] = pack_bf16(kk.x * vr[t4], kk.y * vr[t4 + 1]);
-            pk[t4 / 2 + 1] = pack_bf16(kk.z * vr[t4 + 2], kk.w * vr[t4 + 3]);
+          for (int j = 0; j < 8; ++j) {
+            const uint4 kk = *reinterpret_cast<const uint4*>(krow + j * 16);
+            pk[4 * j] = mul_bf16x2(kk.x, vr[4 * j]);
+            pk[4 * j + 1] = mul_bf16x2(kk.y, vr[4 * j + 1]);
+            pk[4 * j + 2] = mul_bf16x2(kk.z, vr[4 * j + 2]);
+            pk[4 * j + 3] = mul_bf16x2(kk.w, vr[4 * j + 3]);
           }
         } else {
           const bool live = rowl < 64;
+          const unsigned char* srow = vT + 8 * KT_STRIDE;
 #pragma unroll
-          for (int t4 = 0; t4 < C; t4 += 4) {
-            const float4 kk = *reinterpret_cast<const float4*>(krow + t4);
-            const float4 rr = *reinterpret_cast<const float4*>(r2 + t4);
-            pk[t4 / 2] = live ? pack_bf16(kk.x * rr.x, kk.y * rr.y) : 0u;
-            pk[t4 / 2 + 1] = live ? pack_bf16(kk.z * rr.z, kk.w * rr.w) : 0u;
+          for (int j = 0; j < 8; ++j) {
+            const uint4 kk = *reinterpret_cast<const uint4*>(krow + j * 16);
+            const uint4 rr = *reinterpret_cast<const uint4*>(srow + j * 16);
+            pk[4 * j] = live ? mul_bf16x2(kk.x, rr.x) : 0u;
+            pk[4 * j + 1] = live ? mul_bf16x2(kk.y, rr.y) : 0u;
+            pk[4 * j + 2] = live ? mul_bf16x2(kk.z, rr.z) : 0u;
+            pk[4 * j + 3] = live ? mul_bf16x2(kk.w, rr.w) : 0u;
           }
         }
         tmem_st32(tmem_addr(tb, q4 * 32, COL_W + (g & 1) * 32), pk);
@@ -446,16 +456,21 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mbar_arrive(sm.bar(BAR_WFULL + i));
       }
       if (!ok) break;
-      mbar_arrive(sm.bar(BAR_EMPTY + s));     // done with the stage (the MMA adds its own arrival)
+      mbar_arrive(sm.bar(BAR_EMPTY + s));     // done with the stage (each issuer adds its own arrival)
     }
   } else {
-    // =========================== TMEM readers (128 threads) ===========================
-    const int tr = tid - WARP_RD0 * 32;        // 0..127
+    // =========================== TMEM readers (2 groups x 128 threads) ===========================
+    // group 0 drains ring items 0, 2 and 4 (state tiles 0, 2 and the normaliser tile), group 1 drains
+    // items 1, 3 and 5 (state tiles 1, 3 and the intra-chunk scores); both meet in the epilogue.
+    const int rgrp = (warp - WARP_RD0) >> 2;
+    const int tr = tid - WARP_RD0 * 32;        // 0..255
     const uint32_t q4 = warp & 3;              // TMEM lane quadrant this warp may access
     const int rowl = q4 * 32 + lane;           // tile row (= TMEM lane) of this thread
-    float* red = sm.red();
+    float* redS = sm.red() + rgrp * 128 * RED_STRIDE;     // per-group partial sums over its state tiles
+    float* redA = sm.red();
+    float* redB = sm.red() + 128 * RED_STRIDE;
+    float* redZ = sm.red() + 256 * RED_STRIDE;            // 64 rows: normaliser partials
     float* nintra = sm.nintra();
-    float* ninter = sm.ninter();
     __nv_bfloat16* oh = args.out + (size_t)bh * args.Tlen * D + slice * VS;
     for (int c = 0; c < nloc && ok && write_out; ++c) {
       const int s = c & 1;
@@ -466,135 +481,132 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       float acc[C];
 #pragma unroll
       for (int t = 0; t < C; ++t) acc[t] = 0.f;
-      for (int i = 0; i < NT && ok; ++i) {
-        const int g = c * NI + i;
+      // acc[t] += q[t,b] * Y[row, t] for ring item i (b = the feature index of this row in that tile)
+      auto drain_item = [&](int i) {
         ok = wait_or_abort(sm.bar(BAR_RFULL + i), c & 1, abort_flag);
-        if (!ok) break;
+        if (!ok) return;
         tc_fence_after();
-        if (i == 4) {
-          // the four state tiles are in acc: reduce over b within the CTA -> ninter[t][v]
-#pragma unroll
-          for (int t4 = 0; t4 < C; t4 += 4)
-            *reinterpret_cast<float4*>(red + rowl * RED_STRIDE + t4) =
-                make_float4(acc[t4], acc[t4 + 1], acc[t4 + 2], acc[t4 + 3]);
-          group_sync(3);
-          {
-            const int t = tr & 63, vh = tr >> 6;
-#pragma unroll
-            for (int vv = 0; vv < 4; ++vv) {
-              const int v = vh * 4 + vv;
-              float sum = 0.f;
-#pragma unroll
-              for (int bl = 0; bl < 16; ++bl) sum += red[(bl * 8 + v) * RED_STRIDE + t];
-              ninter[t * 9 + v] = sum;
-            }
-          }
-          group_sync(3);
-#pragma unroll
-          for (int t = 0; t < C; ++t) acc[t] = 0.f;
-        }
         const int b = (i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63);
         const float* qrow = qT + b * C;
+        const uint32_t col = COL_R + (i & 1) * 64;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t y[32];
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (g & 1) * 64 + half * 32), y);
+        for (int qtr = 0; qtr < 4; ++qtr) {
+          uint32_t y[16];
+          tmem_ld16(tmem_addr(tb, q4 * 32, col + qtr * 16), y);
+          float4 qq[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) qq[e] = *reinterpret_cast<const float4*>(qrow + qtr * 16 + e * 4);
           tmem_wait_ld();
-          if (half == 1) {
+          if (qtr == 3) {
             tc_fence_before();
-            mbar_arrive(sm.bar(BAR_REMPTY + i));      // the slot is in registers now
+            mbar_arrive(sm.bar(BAR_REMPTY + i));      // the item is in registers now
           }
 #pragma unroll
-          for (int jj = 0; jj < 32; jj += 4) {
-            const float4 qq = *reinterpret_cast<const float4*>(qrow + half * 32 + jj);
-            acc[half * 32 + jj] = fmaf(qq.x, __uint_as_float(y[jj]), acc[half * 32 + jj]);
-            acc[half * 32 + jj + 1] = fmaf(qq.y, __uint_as_float(y[jj + 1]), acc[half * 32 + jj + 1]);
-            acc[half * 32 + jj + 2] = fmaf(qq.z, __uint_as_float(y[jj + 2]), acc[half * 32 + jj + 2]);
-            acc[half * 32 + jj + 3] = fmaf(qq.w, __uint_as_float(y[jj + 3]), acc[half * 32 + jj + 3]);
+          for (int e = 0; e < 4; ++e) {
+            const int t = qtr * 16 + e * 4;
+            const float2 a0 = __ffma2_rn(make_float2(qq[e].x, qq[e].y),
+                                         make_float2(__uint_as_float(y[e * 4]), __uint_as_float(y[e * 4 + 1])),
+                                         make_float2(acc[t], acc[t + 1]));
+            const float2 a1 = __ffma2_rn(make_float2(qq[e].z, qq[e].w),
+                                         make_float2(__uint_as_float(y[e * 4 + 2]), __uint_as_float(y[e * 4 + 3])),
+                                         make_float2(acc[t + 2], acc[t + 3]));
+            acc[t] = a0.x; acc[t + 1] = a0.y; acc[t + 2] = a1.x; acc[t + 3] = a1.y;
           }
         }
-      }
+      };
+      drain_item(rgrp);
+      if (ok) drain_item(2 + rgrp);
       if (!ok) break;
-      // normaliser tile: rows 0..63 hold b, reduce over them -> ninter[t][8]
-      if (rowl < 64) {
 #pragma unroll
-        for (int t4 = 0; t4 < C; t4 += 4)
-          *reinterpret_cast<float4*>(red + rowl * RED_STRIDE + t4) =
-              make_float4(acc[t4], acc[t4 + 1], acc[t4 + 2], acc[t4 + 3]);
-      }
-      // ---- intra-chunk: P = s^2 / ||k||^2 (causal) -> bf16 into the ring slot ----
-      const int gp = c * NI + 5;
-      ok = wait_or_abort(sm.bar(BAR_RFULL + 5), c & 1, abort_flag);
-      if (!ok) break;
-      tc_fence_after();
-      if (rowl < 64) {
-        // scores of both halves are read before the packed P overwrites columns [0,32) of the slot
-        uint32_t pk[32];
+      for (int t4 = 0; t4 < C; t4 += 4)
+        *reinterpret_cast<float4*>(redS + rowl * RED_STRIDE + t4) =
+            make_float4(acc[t4], acc[t4 + 1], acc[t4 + 2], acc[t4 + 3]);
+      if (rgrp == 0) {
+        // normaliser tile: rows 0..63 hold b
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t sc[32];
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64 + half * 32), sc);
+        for (int t = 0; t < C; ++t) acc[t] = 0.f;
+        drain_item(4);
+        if (!ok) break;
+        if (rowl < 64) {
+#pragma unroll
+          for (int t4 = 0; t4 < C; t4 += 4)
+            *reinterpret_cast<float4*>(redZ + rowl * RED_STRIDE + t4) =
+                make_float4(acc[t4], acc[t4 + 1], acc[t4 + 2], acc[t4 + 3]);
+        }
+      } else {
+        // ---- intra-chunk: P = s^2 / ||k||^2 (causal) -> bf16 into the ring slot ----
+        ok = wait_or_abort(sm.bar(BAR_RFULL + 5), c & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        if (rowl < 64) {
+          // scores of both halves are read before the packed P overwrites columns [0,32) of the slot
+          uint32_t pk[32];
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t sc[32];
+            tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + 64 + half * 32), sc);
+            tmem_wait_ld();
+#pragma unroll
+            for (int jj = 0; jj < 32; jj += 4) {
+              const int j = half * 32 + jj;
+              const float4 rr = *reinterpret_cast<const float4*>(r2 + j);
+              const float s0 = __uint_as_float(sc[jj]), s1 = __uint_as_float(sc[jj + 1]);
+              const float s2 = __uint_as_float(sc[jj + 2]), s3 = __uint_as_float(sc[jj + 3]);
+              const float w0 = (j <= rowl) ? s0 * s0 * rr.x : 0.f;
+              const float w1 = (j + 1 <= rowl) ? s1 * s1 * rr.y : 0.f;
+              const float w2 = (j + 2 <= rowl) ? s2 * s2 * rr.z : 0.f;
+              const float w3 = (j + 3 <= rowl) ? s3 * s3 * rr.w : 0.f;
+              pk[j / 2] = pack_bf16(w0, w1);
+              pk[j / 2 + 1] = pack_bf16(w2, w3);
+            }
+          }
+          tmem_st32(tmem_addr(tb, q4 * 32, COL_R + 64), pk);
+          tmem_wait_st();
+        }
+        tc_fence_before();
+        mbar_arrive(sm.bar(BAR_PREADY));
+        // ---- [N_intra | D_intra] from the MMA ----
+        ok = wait_or_abort(sm.bar(BAR_PVFULL), c & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        if (rowl < 64) {
+          uint32_t pv[16];
+          tmem_ld16(tmem_addr(tb, q4 * 32, COL_R + 64 + 32), pv);
           tmem_wait_ld();
 #pragma unroll
-          for (int jj = 0; jj < 32; jj += 4) {
-            const int j = half * 32 + jj;
-            const float4 rr = *reinterpret_cast<const float4*>(r2 + j);
-            const float s0 = __uint_as_float(sc[jj]), s1 = __uint_as_float(sc[jj + 1]);
-            const float s2 = __uint_as_float(sc[jj + 2]), s3 = __uint_as_float(sc[jj + 3]);
-            const float w0 = (j <= rowl) ? s0 * s0 * rr.x : 0.f;
-            const float w1 = (j + 1 <= rowl) ? s1 * s1 * rr.y : 0.f;
-            const float w2 = (j + 2 <= rowl) ? s2 * s2 * rr.z : 0.f;
-            const float w3 = (j + 3 <= rowl) ? s3 * s3 * rr.w : 0.f;
-            pk[j / 2] = pack_bf16(w0, w1);
-            pk[j / 2 + 1] = pack_bf16(w2, w3);
-          }
+          for (int v = 0; v < 9; ++v) nintra[rowl * 9 + v] = __uint_as_float(pv[v]);
         }
-        tmem_st32(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64), pk);
-        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(sm.bar(BAR_REMPTY + 5));
       }
-      tc_fence_before();
-      mbar_arrive(sm.bar(BAR_PREADY));
-      group_sync(3);                      // red rows 0..63 (normaliser partials) are complete
-      if (tr < C) {
-        float sum = 0.f;
-#pragma unroll 16
-        for (int r = 0; r < 64; ++r) sum += red[r * RED_STRIDE + tr];
-        ninter[tr * 9 + 8] = sum;
-      }
-      // ---- [N_intra | D_intra] from the MMA ----
-      ok = wait_or_abort(sm.bar(BAR_PVFULL), c & 1, abort_flag);
-      if (!ok) break;
-      tc_fence_after();
-      if (rowl < 64) {
-        uint32_t pv[16];
-        tmem_ld16(tmem_addr(tb, q4 * 32, COL_R + (gp & 1) * 64 + 32), pv);
-        tmem_wait_ld();
-#pragma unroll
-        for (int v = 0; v < 9; ++v) nintra[rowl * 9 + v] = __uint_as_float(pv[v]);
-      }
-      tc_fence_before();
-      mbar_arrive(sm.bar(BAR_REMPTY + 5));
-      group_sync(3);
-      // ---- gate + normalise epilogue ----
+      reader_sync();      // partial sums of both groups are in shared memory
+      // ---- reduce over b, gate + normalise epilogue: thread <-> (t, two value columns) ----
       {
-        const int t = tr >> 1, vq = (tr & 1) * 4;
+        const int t = tr >> 2, sub = tr & 3;
+        float zp = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) zp += redZ[(4 * kk + sub) * RED_STRIDE + t];
+        zp += __shfl_xor_sync(0xffffffffu, zp, 1);
+        zp += __shfl_xor_sync(0xffffffffu, zp, 2);
+        float n0 = 0.f, n1 = 0.f;
+#pragma unroll
+        for (int bl = 0; bl < 16; ++bl) {
+          const int r0 = (bl * 8 + 2 * sub) * RED_STRIDE + t;
+          n0 += redA[r0] + redB[r0];
+          n1 += redA[r0 + RED_STRIDE] + redB[r0 + RED_STRIDE];
+        }
         const int tg = (c_begin + c) * C + t;
         if (tg < args.Tlen) {
-          const float den = ninter[t * 9 + 8] + nintra[t * 9 + 8];
+          const float den = zp + nintra[t * 9 + 8];
           const float inv = den > 0.f ? 1.f / den : 0.f;
-          float o[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) o[e] = (ninter[t * 9 + vq + e] + nintra[t * 9 + vq + e]) * inv;
-          uint2 pk;
-          pk.x = pack_bf16(o[0], o[1]);
-          pk.y = pack_bf16(o[2], o[3]);
-          *reinterpret_cast<uint2*>(oh + (size_t)tg * D + vq) = pk;
+          const uint32_t pk = pack_bf16((n0 + nintra[t * 9 + 2 * sub]) * inv, (n1 + nintra[t * 9 + 2 * sub + 1]) * inv);
+          *reinterpret_cast<uint32_t*>(oh + (size_t)tg * D + 2 * sub) = pk;
         }
       }
-      group_sync(3);   // ninter / nintra / red are rewritten in the next chunk
+      reader_sync();      // the scratch is rewritten in the next chunk
     }
     // ---- final state of this group (scan pass 1) ----
-    if (ok && args.final_state != nullptr) {
+    if (ok && args.final_state != nullptr && rgrp == 0) {
       ok = wait_or_abort(sm.bar(BAR_DONE), 0, abort_flag);
       tc_fence_after();
       if (ok) {
