@@ -67,7 +67,7 @@ constexpr uint32_t OFF_ONES = 34816;              // 64 x 8 bf16 rows (1,0,..,0)
 constexpr uint32_t OFF_QF = 35840;                // 2 x 16 KB: query tile as tf32, K-major, 128B swizzle, 2 atoms
 constexpr uint32_t OFF_KT = 68608;                // kT[b][t] bf16, 64 rows (builders only)
 constexpr uint32_t OFF_VT = 86016;                // vT[v][t] = bf16(v / ||k||^2), row 8 = bf16(1 / ||k||^2) (builders only)
-constexpr uint32_t OFF_QT = 88192;                // 2 x qT[b][t] fp32 (readers)
+constexpr uint32_t OFF_QT = 88192;                // 2 x qT[b][t] bf16, 144-byte rows (readers)
 constexpr uint32_t OFF_R2 = 120960;               // 2 x r2[t] = 1/||k_t||^2
 constexpr uint32_t OFF_RED = 121472;              // red[128+128+64][68] fp32: per-group state partials, normaliser partials
 constexpr uint32_t RED_STRIDE = 68;
@@ -106,7 +106,7 @@ struct Shared {
   __device__ unsigned char* qf(int s) const { return base + OFF_QF + s * 16384; }
   __device__ unsigned char* kT() const { return base + OFF_KT; }
   __device__ unsigned char* vT() const { return base + OFF_VT; }
-  __device__ float* qT(int s) const { return reinterpret_cast<float*>(base + OFF_QT + s * 16384); }
+  __device__ unsigned char* qT(int s) const { return base + OFF_QT + s * 16384; }
   __device__ float* r2(int s) const { return reinterpret_cast<float*>(base + OFF_R2 + s * 256); }
   __device__ float* red() const { return reinterpret_cast<float*>(base + OFF_RED); }
   __device__ float* nintra() const { return reinterpret_cast<float*>(base + OFF_NINTRA); }
@@ -349,9 +349,9 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       ok = wait_or_abort(sm.bar(BAR_FULL + s), (c >> 1) & 1, abort_flag);
       if (!ok) break;
       group_sync(2);   // every builder is done with kT / vT of the previous chunk
-      float* qT = sm.qT(s);
+      unsigned char* qT = sm.qT(s);
       float* r2 = sm.r2(s);
-      // ---- phase 1: key norms, kT (bf16), tf32 query tile, qT ----
+      // ---- phase 1: key norms, kT (bf16), tf32 query tile, qT (bf16) ----
       {
         const unsigned char* kt = sm.ktile(s);
         const unsigned char* qt = sm.qtile(s);
@@ -380,7 +380,10 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
               qv[2 * e + 1] = __uint_as_float(qw[e] & 0xFFFF0000u);
             }
 #pragma unroll
-            for (int e = 0; e < 8; ++e) qT[(chunk * 8 + e) * C + row] = qv[e];
+            for (int e = 0; e < 4; ++e) {
+              *reinterpret_cast<uint16_t*>(qT + (chunk * 8 + 2 * e) * KT_STRIDE + row * 2) = (uint16_t)(qw[e] & 0xFFFFu);
+              *reinterpret_cast<uint16_t*>(qT + (chunk * 8 + 2 * e + 1) * KT_STRIDE + row * 2) = (uint16_t)(qw[e] >> 16);
+            }
             // tf32 query tile: 32 fp32 per 128-byte row, this thread's half-row is atom `hf`
             *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j)) = make_float4(qv[0], qv[1], qv[2], qv[3]);
             *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j + 1)) = make_float4(qv[4], qv[5], qv[6], qv[7]);
@@ -476,43 +479,49 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int s = c & 1;
       ok = wait_or_abort(sm.bar(BAR_PREP + s), (c >> 1) & 1, abort_flag);
       if (!ok) break;
-      const float* qT = sm.qT(s);
+      const unsigned char* qT = sm.qT(s);
       const float* r2 = sm.r2(s);
       float acc[C];
 #pragma unroll
       for (int t = 0; t < C; ++t) acc[t] = 0.f;
-      // acc[t] += q[t,b] * Y[row, t] for ring item i (b = the feature index of this row in that tile)
+      // acc[t] += q[t,b] * Y[row, t] for ring item i (b = the feature index of this row in that tile).
+      // The TMEM read of the next 16 columns is in flight while the current 16 are multiplied in.
+      auto fma16 = [&](const uint32_t (&y)[16], const unsigned char* qrow, int qtr) {
+        const uint4 qa = *reinterpret_cast<const uint4*>(qrow + qtr * 32);
+        const uint4 qb = *reinterpret_cast<const uint4*>(qrow + qtr * 32 + 16);
+        const uint32_t qw[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int t = qtr * 16 + 2 * e;
+          const float2 r = __ffma2_rn(make_float2(__uint_as_float(qw[e] << 16), __uint_as_float(qw[e] & 0xFFFF0000u)),
+                                      make_float2(__uint_as_float(y[2 * e]), __uint_as_float(y[2 * e + 1])),
+                                      make_float2(acc[t], acc[t + 1]));
+          acc[t] = r.x;
+          acc[t + 1] = r.y;
+        }
+      };
       auto drain_item = [&](int i) {
         ok = wait_or_abort(sm.bar(BAR_RFULL + i), c & 1, abort_flag);
         if (!ok) return;
         tc_fence_after();
         const int b = (i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63);
-        const float* qrow = qT + b * C;
-        const uint32_t col = COL_R + (i & 1) * 64;
-#pragma unroll
-        for (int qtr = 0; qtr < 4; ++qtr) {
-          uint32_t y[16];
-          tmem_ld16(tmem_addr(tb, q4 * 32, col + qtr * 16), y);
-          float4 qq[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) qq[e] = *reinterpret_cast<const float4*>(qrow + qtr * 16 + e * 4);
-          tmem_wait_ld();
-          if (qtr == 3) {
-            tc_fence_before();
-            mbar_arrive(sm.bar(BAR_REMPTY + i));      // the item is in registers now
-          }
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int t = qtr * 16 + e * 4;
-            const float2 a0 = __ffma2_rn(make_float2(qq[e].x, qq[e].y),
-                                         make_float2(__uint_as_float(y[e * 4]), __uint_as_float(y[e * 4 + 1])),
-                                         make_float2(acc[t], acc[t + 1]));
-            const float2 a1 = __ffma2_rn(make_float2(qq[e].z, qq[e].w),
-                                         make_float2(__uint_as_float(y[e * 4 + 2]), __uint_as_float(y[e * 4 + 3])),
-                                         make_float2(acc[t + 2], acc[t + 3]));
-            acc[t] = a0.x; acc[t + 1] = a0.y; acc[t + 2] = a1.x; acc[t + 3] = a1.y;
-          }
-        }
+        const unsigned char* qrow = qT + b * KT_STRIDE;
+        const uint32_t ta0 = tmem_addr(tb, q4 * 32, COL_R + (i & 1) * 64);
+        uint32_t ya[16], yb[16];
+        tmem_ld16(ta0, ya);
+        tmem_wait_ld(ya);
+        tmem_ld16(ta0 + 16, yb);
+        fma16(ya, qrow, 0);
+        tmem_wait_ld(yb);
+        tmem_ld16(ta0 + 32, ya);
+        fma16(yb, qrow, 1);
+        tmem_wait_ld(ya);
+        tmem_ld16(ta0 + 48, yb);
+        fma16(ya, qrow, 2);
+        tmem_wait_ld(yb);
+        tc_fence_before();
+        mbar_arrive(sm.bar(BAR_REMPTY + i));      // the item is in registers now
+        fma16(yb, qrow, 3);
       };
       drain_item(rgrp);
       if (ok) drain_item(2 + rgrp);
@@ -545,7 +554,7 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           for (int half = 0; half < 2; ++half) {
             uint32_t sc[32];
             tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + 64 + half * 32), sc);
-            tmem_wait_ld();
+            tmem_wait_ld(sc);
 #pragma unroll
             for (int jj = 0; jj < 32; jj += 4) {
               const int j = half * 32 + jj;
@@ -572,7 +581,7 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (rowl < 64) {
           uint32_t pv[16];
           tmem_ld16(tmem_addr(tb, q4 * 32, COL_R + 64 + 32), pv);
-          tmem_wait_ld();
+          tmem_wait_ld(pv);
 #pragma unroll
           for (int v = 0; v < 9; ++v) nintra[rowl * 9 + v] = __uint_as_float(pv[v]);
         }
@@ -614,7 +623,7 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int cblk = 0; cblk < (NT * 64) / 32; ++cblk) {
           uint32_t z[32];
           tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + cblk * 32), z);
-          tmem_wait_ld();
+          tmem_wait_ld(z);
           float* d = dst + ((size_t)(cblk >> 1) * 128 + rowl) * 64 + (cblk & 1) * 32;
 #pragma unroll
           for (int j = 0; j < 32; j += 4)
