@@ -69,10 +69,10 @@ constexpr uint32_t OFF_KT = 68608;                // kT[b][t] bf16, 64 rows (bui
 constexpr uint32_t OFF_VT = 86016;                // vT[v][t] = bf16(v / ||k||^2), row 8 = bf16(1 / ||k||^2) (builders only)
 constexpr uint32_t OFF_QT = 88192;                // 2 x qT[b][t] bf16, 144-byte rows (readers)
 constexpr uint32_t OFF_R2 = 120960;               // 2 x r2[t] = 1/||k_t||^2
-constexpr uint32_t OFF_RED = 121472;              // red[128+128+64][68] fp32: per-group state partials, normaliser partials
+constexpr uint32_t OFF_RED = 121472;              // red[128+64][68] fp32: state partials, normaliser partials
 constexpr uint32_t RED_STRIDE = 68;
-constexpr uint32_t OFF_NINTRA = 208512;           // [64][9]
-constexpr uint32_t OFF_BAR = 210816;              // mbarriers
+constexpr uint32_t OFF_NINTRA = 173696;           // [64][9]
+constexpr uint32_t OFF_BAR = 176000;              // mbarriers
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;  // slack for the 1024-byte alignment
 static_assert(OFF_QF % 1024 == 0 && OFF_QK % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -88,8 +88,8 @@ enum {
   BAR_PREP = 4,     // [2] operands of the chunk built (128 builders)
   BAR_WFULL = 6,    // [5] W tile i stored to TMEM (128 builders)
   BAR_RFULL = 11,   // [6] ring item i produced by the MMA
-  BAR_REMPTY = 17,  // [6] ring item i drained (128 readers)
-  BAR_PREADY = 23,  // P (bf16) stored to TMEM (128 readers)
+  BAR_REMPTY = 17,  // [6] ring item i drained (256 readers)
+  BAR_PREADY = 23,  // P (bf16) stored to TMEM (256 readers)
   BAR_PVFULL = 24,  // P [V|1] complete
   BAR_U = 25,       // [5] update of state tile i complete (frees the W buffer, allows the next read)
   BAR_DRAIN = 30,
@@ -115,6 +115,8 @@ struct Shared {
 
 __device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 __device__ __forceinline__ void reader_sync() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
+// the two reader warps (one per group) that share TMEM lane quadrant q
+__device__ __forceinline__ void group_pair_sync(uint32_t q) { asm volatile("bar.sync %0, 64;" ::"r"(4 + q) : "memory"); }
 
 // Bounded wait that also gives up as soon as another role has flagged an abort.
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -177,9 +179,9 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     for (int i = 0; i < NI; ++i) {
       mbar_init(sm.bar(BAR_RFULL + i), 1);
-      mbar_init(sm.bar(BAR_REMPTY + i), 128);
+      mbar_init(sm.bar(BAR_REMPTY + i), 256);
     }
-    mbar_init(sm.bar(BAR_PREADY), 128);
+    mbar_init(sm.bar(BAR_PREADY), 256);
     mbar_init(sm.bar(BAR_PVFULL), 1);
     mbar_init(sm.bar(BAR_DRAIN), NISSUER);
     mbar_init(sm.bar(BAR_DONE), NISSUER);
@@ -351,7 +353,7 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       group_sync(2);   // every builder is done with kT / vT of the previous chunk
       unsigned char* qT = sm.qT(s);
       float* r2 = sm.r2(s);
-      // ---- phase 1: key norms, kT (bf16), tf32 query tile, qT (bf16) ----
+      // ---- phase 1: key norms, tf32 query tile; kT and qT (bf16 transposes) via ldmatrix / stmatrix.trans ----
       {
         const unsigned char* kt = sm.ktile(s);
         const unsigned char* qt = sm.qtile(s);
@@ -367,30 +369,40 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const float lo = __uint_as_float(kw[e] << 16), hi = __uint_as_float(kw[e] & 0xFFFF0000u);
             ss = fmaf(lo, lo, ss);
             ss = fmaf(hi, hi, ss);
-            *reinterpret_cast<uint16_t*>(kT + (chunk * 8 + 2 * e) * KT_STRIDE + row * 2) = (uint16_t)(kw[e] & 0xFFFFu);
-            *reinterpret_cast<uint16_t*>(kT + (chunk * 8 + 2 * e + 1) * KT_STRIDE + row * 2) = (uint16_t)(kw[e] >> 16);
           }
           if (write_out) {
             const uint4 qraw = *reinterpret_cast<const uint4*>(qt + sw128_offset(row, chunk));
             const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
-            float qv[8];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              qv[2 * e] = __uint_as_float(qw[e] << 16);
-              qv[2 * e + 1] = __uint_as_float(qw[e] & 0xFFFF0000u);
-            }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              *reinterpret_cast<uint16_t*>(qT + (chunk * 8 + 2 * e) * KT_STRIDE + row * 2) = (uint16_t)(qw[e] & 0xFFFFu);
-              *reinterpret_cast<uint16_t*>(qT + (chunk * 8 + 2 * e + 1) * KT_STRIDE + row * 2) = (uint16_t)(qw[e] >> 16);
-            }
             // tf32 query tile: 32 fp32 per 128-byte row, this thread's half-row is atom `hf`
-            *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j)) = make_float4(qv[0], qv[1], qv[2], qv[3]);
-            *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j + 1)) = make_float4(qv[4], qv[5], qv[6], qv[7]);
+            *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j)) =
+                make_float4(__uint_as_float(qw[0] << 16), __uint_as_float(qw[0] & 0xFFFF0000u),
+                            __uint_as_float(qw[1] << 16), __uint_as_float(qw[1] & 0xFFFF0000u));
+            *reinterpret_cast<float4*>(qf + sw128_offset(row, 2 * j + 1)) =
+                make_float4(__uint_as_float(qw[2] << 16), __uint_as_float(qw[2] & 0xFFFF0000u),
+                            __uint_as_float(qw[3] << 16), __uint_as_float(qw[3] & 0xFFFF0000u));
           }
         }
         ss += __shfl_xor_sync(0xffffffffu, ss, 1);
         if (hf == 0) r2[row] = inv_or_zero(ss);
+        // transposes: this warp owns feature blocks 2*wb and 2*wb+1 (8 features each) for all 64 tokens.
+        // One ldmatrix.x4 reads four 8-token x 8-feature blocks, stmatrix.x4.trans writes their transposes.
+        const int wb = warp - WARP_BLD0;
+        const int mj = lane >> 3, mr = lane & 7;      // matrix index and row this lane addresses
+#pragma unroll
+        for (int ab = 0; ab < 2; ++ab) {
+          const int A = 2 * wb + ab;                  // feature block = 16-byte chunk index of a tile row
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int tblk = 4 * h + mj;              // token block of the matrix this lane addresses
+            uint32_t frag[4];
+            ldmatrix_x4(frag, smem_u32(kt + sw128_offset(tblk * 8 + mr, A)));
+            stmatrix_x4_trans(smem_u32(kT + (A * 8 + mr) * KT_STRIDE + tblk * 16), frag);
+            if (write_out) {
+              ldmatrix_x4(frag, smem_u32(qt + sw128_offset(tblk * 8 + mr, A)));
+              stmatrix_x4_trans(smem_u32(qT + (A * 8 + mr) * KT_STRIDE + tblk * 16), frag);
+            }
+          }
+        }
       }
       group_sync(2);
       // ---- phase 2: transposed values scaled by 1/||k||^2 (bf16); row 8 is the scale itself ----
@@ -420,40 +432,45 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
       }
       // ---- W tiles: row rowl <-> (b = 16 i + rowl/8, v = rowl%8); fifth tile: rows < 64 hold k[t,b]/||k||^2.
-      //      One packed bf16 multiply per token pair; the products go straight to TMEM. ----
+      //      One packed bf16 multiply per token pair; the products go straight to TMEM.  The key row of
+      //      the next tile is fetched while the TMEM store of the current one is in flight. ----
+      uint32_t kk[32];
+      auto load_krow = [&](int i) {
+        const unsigned char* krow = kT + ((i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63)) * KT_STRIDE;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint4 f = *reinterpret_cast<const uint4*>(krow + j * 16);
+          kk[4 * j] = f.x; kk[4 * j + 1] = f.y; kk[4 * j + 2] = f.z; kk[4 * j + 3] = f.w;
+        }
+      };
+      load_krow(0);
       for (int i = 0; i < NT && ok; ++i) {
         const int g = c * NT + i;
+        uint32_t pk[32];
+        if (i == 4) {
+          // normaliser tile: the value row is the scale 1/||k||^2 itself; rows 64..127 are not used
+          const unsigned char* srow = vT + 8 * KT_STRIDE;
+          const bool live = rowl < 64;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 rr = *reinterpret_cast<const uint4*>(srow + j * 16);
+            pk[4 * j] = live ? mul_bf16x2(kk[4 * j], rr.x) : 0u;
+            pk[4 * j + 1] = live ? mul_bf16x2(kk[4 * j + 1], rr.y) : 0u;
+            pk[4 * j + 2] = live ? mul_bf16x2(kk[4 * j + 2], rr.z) : 0u;
+            pk[4 * j + 3] = live ? mul_bf16x2(kk[4 * j + 3], rr.w) : 0u;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) pk[j] = mul_bf16x2(kk[j], vr[j]);
+        }
         if (g >= 2) {   // the W buffer is free once the update two tiles back has completed
           const int gp = g - 2;
           ok = wait_or_abort(sm.bar(BAR_U + gp % NT), (gp / NT) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
         }
-        const unsigned char* krow = kT + ((i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63)) * KT_STRIDE;
-        uint32_t pk[32];
-        if (i < 4) {
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint4 kk = *reinterpret_cast<const uint4*>(krow + j * 16);
-            pk[4 * j] = mul_bf16x2(kk.x, vr[4 * j]);
-            pk[4 * j + 1] = mul_bf16x2(kk.y, vr[4 * j + 1]);
-            pk[4 * j + 2] = mul_bf16x2(kk.z, vr[4 * j + 2]);
-            pk[4 * j + 3] = mul_bf16x2(kk.w, vr[4 * j + 3]);
-          }
-        } else {
-          const bool live = rowl < 64;
-          const unsigned char* srow = vT + 8 * KT_STRIDE;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint4 kk = *reinterpret_cast<const uint4*>(krow + j * 16);
-            const uint4 rr = *reinterpret_cast<const uint4*>(srow + j * 16);
-            pk[4 * j] = live ? mul_bf16x2(kk.x, rr.x) : 0u;
-            pk[4 * j + 1] = live ? mul_bf16x2(kk.y, rr.y) : 0u;
-            pk[4 * j + 2] = live ? mul_bf16x2(kk.z, rr.z) : 0u;
-            pk[4 * j + 3] = live ? mul_bf16x2(kk.w, rr.w) : 0u;
-          }
-        }
         tmem_st32(tmem_addr(tb, q4 * 32, COL_W + (g & 1) * 32), pk);
+        if (i + 1 < NT) load_krow(i + 1);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(sm.bar(BAR_WFULL + i));
@@ -463,16 +480,16 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   } else {
     // =========================== TMEM readers (2 groups x 128 threads) ===========================
-    // group 0 drains ring items 0, 2 and 4 (state tiles 0, 2 and the normaliser tile), group 1 drains
-    // items 1, 3 and 5 (state tiles 1, 3 and the intra-chunk scores); both meet in the epilogue.
-    const int rgrp = (warp - WARP_RD0) >> 2;
+    // Both groups drain every ring item; group g owns the token columns [32 g, 32 g + 32) of it, so a
+    // thread keeps 32 accumulators and one TMEM load of 32 columns covers its share of an item.  The
+    // load of an item is in flight while the previous item is multiplied in.
+    const int rgrp = (warp - WARP_RD0) >> 2;   // column half
     const int tr = tid - WARP_RD0 * 32;        // 0..255
     const uint32_t q4 = warp & 3;              // TMEM lane quadrant this warp may access
     const int rowl = q4 * 32 + lane;           // tile row (= TMEM lane) of this thread
-    float* redS = sm.red() + rgrp * 128 * RED_STRIDE;     // per-group partial sums over its state tiles
-    float* redA = sm.red();
-    float* redB = sm.red() + 128 * RED_STRIDE;
-    float* redZ = sm.red() + 256 * RED_STRIDE;            // 64 rows: normaliser partials
+    const int t0h = rgrp * 32;                 // first token column of this group
+    float* redS = sm.red();                               // [128][68]: partial sums over the four state tiles
+    float* redZ = sm.red() + 128 * RED_STRIDE;            // [64][68]: normaliser partials
     float* nintra = sm.nintra();
     __nv_bfloat16* oh = args.out + (size_t)bh * args.Tlen * D + slice * VS;
     for (int c = 0; c < nloc && ok && write_out; ++c) {
@@ -481,129 +498,137 @@ tc_chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (!ok) break;
       const unsigned char* qT = sm.qT(s);
       const float* r2 = sm.r2(s);
-      float acc[C];
+      float acc[32];
 #pragma unroll
-      for (int t = 0; t < C; ++t) acc[t] = 0.f;
-      // acc[t] += q[t,b] * Y[row, t] for ring item i (b = the feature index of this row in that tile).
-      // The TMEM read of the next 16 columns is in flight while the current 16 are multiplied in.
-      auto fma16 = [&](const uint32_t (&y)[16], const unsigned char* qrow, int qtr) {
-        const uint4 qa = *reinterpret_cast<const uint4*>(qrow + qtr * 32);
-        const uint4 qb = *reinterpret_cast<const uint4*>(qrow + qtr * 32 + 16);
-        const uint32_t qw[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+      for (int t = 0; t < 32; ++t) acc[t] = 0.f;
+      // acc[t] += q[t,b] * Y[row, t] over this group's 32 token columns (b = feature index of the row)
+      auto fma32 = [&](const uint32_t (&y)[32], int i) {
+        const int b = (i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63);
+        const unsigned char* qrow = qT + b * KT_STRIDE + t0h * 2;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int t = qtr * 16 + 2 * e;
-          const float2 r = __ffma2_rn(make_float2(__uint_as_float(qw[e] << 16), __uint_as_float(qw[e] & 0xFFFF0000u)),
-                                      make_float2(__uint_as_float(y[2 * e]), __uint_as_float(y[2 * e + 1])),
-                                      make_float2(acc[t], acc[t + 1]));
-          acc[t] = r.x;
-          acc[t + 1] = r.y;
+        for (int j = 0; j < 4; ++j) {
+          const uint4 qa = *reinterpret_cast<const uint4*>(qrow + j * 16);
+          const uint32_t qw[4] = {qa.x, qa.y, qa.z, qa.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int t = j * 8 + 2 * e;
+            const float2 r = __ffma2_rn(make_float2(__uint_as_float(qw[e] << 16), __uint_as_float(qw[e] & 0xFFFF0000u)),
+                                        make_float2(__uint_as_float(y[t]), __uint_as_float(y[t + 1])),
+                                        make_float2(acc[t], acc[t + 1]));
+            acc[t] = r.x;
+            acc[t + 1] = r.y;
+          }
         }
       };
-      auto drain_item = [&](int i) {
+      auto start_item = [&](uint32_t (&y)[32], int i) {
         ok = wait_or_abort(sm.bar(BAR_RFULL + i), c & 1, abort_flag);
         if (!ok) return;
         tc_fence_after();
-        const int b = (i < 4) ? (16 * i + (rowl >> 3)) : (rowl & 63);
-        const unsigned char* qrow = qT + b * KT_STRIDE;
-        const uint32_t ta0 = tmem_addr(tb, q4 * 32, COL_R + (i & 1) * 64);
-        uint32_t ya[16], yb[16];
-        tmem_ld16(ta0, ya);
-        tmem_wait_ld(ya);
-        tmem_ld16(ta0 + 16, yb);
-        fma16(ya, qrow, 0);
-        tmem_wait_ld(yb);
-        tmem_ld16(ta0 + 32, ya);
-        fma16(yb, qrow, 1);
-        tmem_wait_ld(ya);
-        tmem_ld16(ta0 + 48, yb);
-        fma16(ya, qrow, 2);
-        tmem_wait_ld(yb);
-        tc_fence_before();
-        mbar_arrive(sm.bar(BAR_REMPTY + i));      // the item is in registers now
-        fma16(yb, qrow, 3);
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + (i & 1) * 64 + t0h), y);
       };
-      drain_item(rgrp);
-      if (ok) drain_item(2 + rgrp);
+      auto finish_item = [&](uint32_t (&y)[32], int i) {
+        tmem_wait_ld(y);
+        tc_fence_before();
+        mbar_arrive(sm.bar(BAR_REMPTY + i));      // this group's share of the item is in registers now
+      };
+      auto store_acc = [&](float* dst) {
+#pragma unroll
+        for (int t4 = 0; t4 < 32; t4 += 4)
+          *reinterpret_cast<float4*>(dst + rowl * RED_STRIDE + t0h + t4) =
+              make_float4(acc[t4], acc[t4 + 1], acc[t4 + 2], acc[t4 + 3]);
+      };
+      uint32_t ya[32], yb[32];
+      start_item(ya, 0);
       if (!ok) break;
+      finish_item(ya, 0);
+      start_item(yb, 1);
+      if (!ok) break;
+      fma32(ya, 0);
+      finish_item(yb, 1);
+      start_item(ya, 2);
+      if (!ok) break;
+      fma32(yb, 1);
+      finish_item(ya, 2);
+      start_item(yb, 3);
+      if (!ok) break;
+      fma32(ya, 2);
+      finish_item(yb, 3);
+      start_item(ya, 4);
+      if (!ok) break;
+      fma32(yb, 3);
+      store_acc(redS);            // the four state tiles
 #pragma unroll
-      for (int t4 = 0; t4 < C; t4 += 4)
-        *reinterpret_cast<float4*>(redS + rowl * RED_STRIDE + t4) =
-            make_float4(acc[t4], acc[t4 + 1], acc[t4 + 2], acc[t4 + 3]);
-      if (rgrp == 0) {
-        // normaliser tile: rows 0..63 hold b
+      for (int t = 0; t < 32; ++t) acc[t] = 0.f;
+      finish_item(ya, 4);
+      // ---- intra-chunk scores (item 5): start the load, finish the normaliser tile meanwhile ----
+      ok = wait_or_abort(sm.bar(BAR_RFULL + 5), c & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      if (rowl < 64) tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + 64 + t0h), yb);
+      fma32(ya, 4);
+      if (rowl < 64) {
+        store_acc(redZ);          // normaliser tile: rows 0..63 hold b
+        // P = s^2 / ||k||^2 (causal) -> bf16 into columns [16 g, 16 g + 16) of the slot.  Every lane's
+        // scores are read (by both groups) before PREADY completes, and the MMA that overwrites the
+        // slot waits for PREADY.
+        tmem_wait_ld(yb);
+        uint32_t pk[16];
 #pragma unroll
-        for (int t = 0; t < C; ++t) acc[t] = 0.f;
-        drain_item(4);
-        if (!ok) break;
-        if (rowl < 64) {
-#pragma unroll
-          for (int t4 = 0; t4 < C; t4 += 4)
-            *reinterpret_cast<float4*>(redZ + rowl * RED_STRIDE + t4) =
-                make_float4(acc[t4], acc[t4 + 1], acc[t4 + 2], acc[t4 + 3]);
-        }
-      } else {
-        // ---- intra-chunk: P = s^2 / ||k||^2 (causal) -> bf16 into the ring slot ----
-        ok = wait_or_abort(sm.bar(BAR_RFULL + 5), c & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        if (rowl < 64) {
-          // scores of both halves are read before the packed P overwrites columns [0,32) of the slot
-          uint32_t pk[32];
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            uint32_t sc[32];
-            tmem_ld32(tmem_addr(tb, q4 * 32, COL_R + 64 + half * 32), sc);
-            tmem_wait_ld(sc);
-#pragma unroll
-            for (int jj = 0; jj < 32; jj += 4) {
-              const int j = half * 32 + jj;
-              const float4 rr = *reinterpret_cast<const float4*>(r2 + j);
-              const float s0 = __uint_as_float(sc[jj]), s1 = __uint_as_float(sc[jj + 1]);
-              const float s2 = __uint_as_float(sc[jj + 2]), s3 = __uint_as_float(sc[jj + 3]);
-              const float w0 = (j <= rowl) ? s0 * s0 * rr.x : 0.f;
-              const float w1 = (j + 1 <= rowl) ? s1 * s1 * rr.y : 0.f;
-              const float w2 = (j + 2 <= rowl) ? s2 * s2 * rr.z : 0.f;
-              const float w3 = (j + 3 <= rowl) ? s3 * s3 * rr.w : 0.f;
-              pk[j / 2] = pack_bf16(w0, w1);
-              pk[j / 2 + 1] = pack_bf16(w2, w3);
-            }
-          }
-          tmem_st32(tmem_addr(tb, q4 * 32, COL_R + 64), pk);
-          tmem_wait_st();
-        }
-        tc_fence_before();
-        mbar_arrive(sm.bar(BAR_PREADY));
-        // ---- [N_intra | D_intra] from the MMA ----
-        ok = wait_or_abort(sm.bar(BAR_PVFULL), c & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        if (rowl < 64) {
-          uint32_t pv[16];
-          tmem_ld16(tmem_addr(tb, q4 * 32, COL_R + 64 + 32), pv);
-          tmem_wait_ld(pv);
-#pragma unroll
-          for (int v = 0; v < 9; ++v) nintra[rowl * 9 + v] = __uint_as_float(pv[v]);
+        for (int jj = 0; jj < 32; jj += 4) {
+          const int j = t0h + jj;
+          const float4 rr = *reinterpret_cast<const float4*>(r2 + j);
+          const float s0 = __uint_as_float(yb[jj]), s1 = __uint_as_float(yb[jj + 1]);
+          const float s2 = __uint_as_float(yb[jj + 2]), s3 = __uint_as_float(yb[jj + 3]);
+          const float w0 = (j <= rowl) ? s0 * s0 * rr.x : 0.f;
+          const float w1 = (j + 1 <= rowl) ? s1 * s1 * rr.y : 0.f;
+          const float w2 = (j + 2 <= rowl) ? s2 * s2 * rr.z : 0.f;
+          const float w3 = (j + 3 <= rowl) ? s3 * s3 * rr.w : 0.f;
+          pk[jj / 2] = pack_bf16(w0, w1);
+          pk[jj / 2 + 1] = pack_bf16(w2, w3);
         }
         tc_fence_before();
-        mbar_arrive(sm.bar(BAR_REMPTY + 5));
+        group_pair_sync(q4);      // both groups have read their scores of these 32 lanes
+        tc_fence_after();
+        tmem_st16(tmem_addr(tb, q4 * 32, COL_R + 64 + rgrp * 16), pk);
+        tmem_wait_st();
       }
-      reader_sync();      // partial sums of both groups are in shared memory
+      tc_fence_before();
+      mbar_arrive(sm.bar(BAR_PREADY));
+      // ---- [N_intra | D_intra] from the MMA ----
+      ok = wait_or_abort(sm.bar(BAR_PVFULL), c & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      if (rowl < 64 && rgrp == 0) {
+        uint32_t pv[16];
+        tmem_ld16(tmem_addr(tb, q4 * 32, COL_R + 64 + 32), pv);
+        tmem_wait_ld(pv);
+#pragma unroll
+        for (int v = 0; v < 9; ++v) nintra[rowl * 9 + v] = __uint_as_float(pv[v]);
+      }
+      tc_fence_before();
+      mbar_arrive(sm.bar(BAR_REMPTY + 5));
+      reader_sync();      // partial sums are in shared memory
       // ---- reduce over b, gate + normalise epilogue: thread <-> (t, two value columns) ----
       {
         const int t = tr >> 2, sub = tr & 3;
-        float zp = 0.f;
+        float zv[16], nv[32];
 #pragma unroll
-        for (int kk = 0; kk < 16; ++kk) zp += redZ[(4 * kk + sub) * RED_STRIDE + t];
-        zp += __shfl_xor_sync(0xffffffffu, zp, 1);
-        zp += __shfl_xor_sync(0xffffffffu, zp, 2);
-        float n0 = 0.f, n1 = 0.f;
+        for (int kk = 0; kk < 16; ++kk) zv[kk] = redZ[(4 * kk + sub) * RED_STRIDE + t];
 #pragma unroll
         for (int bl = 0; bl < 16; ++bl) {
-          const int r0 = (bl * 8 + 2 * sub) * RED_STRIDE + t;
-          n0 += redA[r0] + redB[r0];
-          n1 += redA[r0 + RED_STRIDE] + redB[r0 + RED_STRIDE];
+          nv[2 * bl] = redS[(bl * 8 + 2 * sub) * RED_STRIDE + t];
+          nv[2 * bl + 1] = redS[(bl * 8 + 2 * sub + 1) * RED_STRIDE + t];
         }
+        float zp = 0.f, n0 = 0.f, n1 = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) zp += zv[kk];
+#pragma unroll
+        for (int bl = 0; bl < 16; ++bl) {
+          n0 += nv[2 * bl];
+          n1 += nv[2 * bl + 1];
+        }
+        zp += __shfl_xor_sync(0xffffffffu, zp, 1);
+        zp += __shfl_xor_sync(0xffffffffu, zp, 2);
         const int tg = (c_begin + c) * C + t;
         if (tg < args.Tlen) {
           const float den = zp + nintra[t * 9 + 8];

@@ -227,6 +227,23 @@ __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
 
+// Four 8x8 b16 matrices from shared memory in MMA fragment layout: lane i supplies the address of row
+// i%8 of matrix i/8 (16 bytes per row); afterwards lane i holds elements [i/4][2(i%4)], [i/4][2(i%4)+1]
+// of matrix j in r[j].
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(saddr)
+               : "memory");
+}
+// The inverse with a transpose: the four fragments are written as the transposes of the matrices they
+// were loaded from; lane i supplies the address of row i%8 of (transposed) matrix i/8.
+__device__ __forceinline__ void stmatrix_x4_trans(uint32_t saddr, const uint32_t (&r)[4]) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1,%2,%3,%4};"
+               ::"r"(saddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3])
+               : "memory");
+}
+
 // Byte offset of element (row, 16-byte chunk) inside a tile whose rows are 128 bytes and which is
 // stored with the 128-byte swizzle (as TMA SWIZZLE_128B writes it and the MMA descriptors read it):
 // chunk index XOR (row mod 8).  The tile base must be 1024-byte aligned.
