@@ -152,6 +152,37 @@ int kata_fwd_host(int fn, const void* q_host, const void* k_host, const void* v_
                   int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
 
 /*
+ * kata_chunk_state_scan for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this entry point exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a framework whose allocator
+ * owns all device memory and hands out no scratch, in a plugin called under a "no allocation after
+ * initialisation" rule, or on a serving path that must not touch the allocator because an
+ * allocation may synchronise the device.  Such callers still pass q, k, v and out; only the scan
+ * scratch (group states and the ping-pong buffer of the log-depth scan) is supplied by the library,
+ * from a fixed device array of KATA_STATIC_SCRATCH_BYTES bytes that is part of the library image.
+ * Every GPU context that loads the library holds that array until it exits.
+ *
+ *  - Same arguments, layouts, results and status codes as kata_chunk_state_scan, except:
+ *    opts->workspace / workspace_bytes are ignored; opts->s_pre / z_pre must be null
+ *    (KATA_ERR_INVALID_ARG otherwise); if opts->scan_group is 0 the library picks the smallest
+ *    power-of-two group size whose scratch fits the array.
+ *  - If the scratch needed exceeds KATA_STATIC_SCRATCH_BYTES (large B*H with a small scan_group, or
+ *    simply too many heads), nothing is launched and KATA_ERR_WORKSPACE_TOO_SMALL is returned.
+ *  - The call allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ *  - The first call on each device looks up the device address of the array (one
+ *    cudaGetSymbolAddress, with that device current).  Make that first call outside any stream
+ *    capture; later calls on the same device do no set-up.
+ *  - All calls on a device share the one array, and it keeps whatever the last call left in it.
+ *    Nothing in it has to start at zero: every word a call reads, the same call has written first.
+ *    Two calls that overlap on the GPU (different streams, or different host threads without
+ *    ordering between their streams) race on the array and give wrong results; serialise them.
+ */
+#define KATA_STATIC_SCRATCH_BYTES (32u << 20)
+int kata_chunk_state_scan_static(const void* q, const void* k, const void* v, void* out,
+                                 int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
+
+/*
  * Bytes of device workspace entry point `fn` needs for these sizes and options (0 if none);
  * returns 0 also for invalid arguments (the entry point itself reports the error).
  */

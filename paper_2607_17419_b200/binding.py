@@ -21,7 +21,8 @@ KATA_IMPL_AUTO, KATA_IMPL_SIMT, KATA_IMPL_TENSOR = 0, 1, 2
 KATA_FN_QUADRATIC, KATA_FN_CHUNKED, KATA_FN_CHUNK_STATE_SCAN = 0, 1, 2
 KATA_FN_HOST_IO = 0x100
 
-EXPORTS = ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan", "kata_fwd_host",
+EXPORTS = ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan", "kata_chunk_state_scan_static",
+           "kata_fwd_host",
            "kata_workspace_bytes", "kata_scan_plan", "kata_last_launch_count", "kata_last_impl",
            "kata_status_string",
            "kata_version")
@@ -65,7 +66,7 @@ def lib() -> ctypes.CDLL:
     L = ctypes.CDLL(LIB_PATH)
     ptr, i = ctypes.c_void_p, ctypes.c_int
     fwd_args = [ptr, ptr, ptr, ptr, i, i, i, i, i, i, ctypes.POINTER(KataOpts)]
-    for name in ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan"):
+    for name in ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan", "kata_chunk_state_scan_static"):
         getattr(L, name).argtypes = fwd_args
         getattr(L, name).restype = i
     L.kata_fwd_host.argtypes = [i] + fwd_args
@@ -215,3 +216,26 @@ def kata_chunk_state_scan(q, k, v, out=None, C: int = 64, **kw):
 def kata_fwd_host(fn: int, q, k, v, out, C: int = 64, **kw):
     """Same as entry point ``fn`` with (pinned) host tensors; copies ride the current CUDA stream."""
     return _call(fn, q, k, v, out, C, host_io=True, **kw)
+
+
+KATA_STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def kata_chunk_state_scan_static(q, k, v, out, C: int = 64, *, scan_group: int = 0, impl: int = KATA_IMPL_AUTO,
+                                 feature_order: int = 2, stream=None):
+    """The scan pipeline with the library's built-in scratch: for callers that must not allocate.
+
+    Unlike the other wrappers this one never touches torch's allocator: ``out`` must be passed in, and
+    no workspace is requested.  Calls that overlap on the GPU share (and race on) the one scratch array.
+    """
+    import torch
+    B, H, T, d_k = q.shape
+    d_v = v.shape[-1]
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    opts = make_opts(_dtype_code(q), stream=stream, scan_group=scan_group, impl=impl, feature_order=feature_order)
+    st = lib().kata_chunk_state_scan_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), B, H, T, d_k, d_v,
+                                            C, ctypes.byref(opts))
+    if st != 0:
+        raise KataError(st, "kata_chunk_state_scan_static")
+    return out
