@@ -255,8 +255,10 @@ def run_ours(args):
         if impl == "tensor":
             sustained = ms_total > 1000.0
             peak = peaks["bf16_sustained"] if sustained else peaks["bf16_burst"]
+            # DRAM bytes per launch: ncu on the T=32768 case (202.1 MB read + 47.9 MB written), times 4 (linear in T)
+            traffic = 4 * (202.1e6 + 47.9e6)
             roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
-                        traffic=None, kernel="kata chunked forward (tcgen05)",
+                        traffic=traffic, kernel="kata::tc_chunk_kernel (tcgen05 chunked forward)",
                         note=f"algorithmic flops (packed feature n=2080) / CUDA-event time; peak = "
                              f"{'sustained' if sustained else 'burst'} bf16 cuBLAS of {peaks['source']}")
         else:
