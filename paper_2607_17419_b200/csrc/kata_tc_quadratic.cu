@@ -3,14 +3,16 @@
 // One CTA = one head x one tile of 128 queries; it walks the key tiles j <= i of 128 keys:
 //   scores   S = Q K_j^T                      tcgen05 kind::f16, both operands from TMA-loaded 128B-swizzled tiles,
 //                                             fp32 result in TMEM (two buffers)
-//   weights  P = S^2 / ||k||^2 (causal mask   fp32 on the TMEM read-back; rounded to bf16 and stored back to TMEM;
-//            on the diagonal tile)            the normaliser D accumulates the rounded weights per row
-//   apply    O += P V_j                       tcgen05 kind::f16, A = P from TMEM, B = the value tile MN-major
+//   weights  P = S^2 (causal mask on the      packed fp32x2 multiplies on the TMEM read-back; rounded to bf16 and
+//            diagonal tile)                   stored back to TMEM
+//   apply    [O | D] += P [V/||k||^2 | 1/||k||^2]   tcgen05 kind::f16, A = P from TMEM, B = the value tile (scaled in
+//                                             place by the norm warps) plus one extra column group, MN-major, N = 80:
+//                                             the normaliser is column 64 of the same accumulator
 //   epilogue out = O / D (0 where D = 0)      the gate/normalise step of the readout
 // There is no running maximum and no rescaling: the weights are polynomial.  The query norm cancels between
 // numerator and denominator and is never applied.  The d^2-wide feature state is never formed.
 //
-// Warps (512 threads): 0 TMA producer, 1 score-MMA issuer, 2 apply-MMA issuer, 4-7 key norms, 8-15 weight
+// Warps (512 threads): 0 TMA producer, 1 score-MMA issuer, 2 apply-MMA issuer, 4-7 key norms + value scaling, 8-15 weight
 // builders (TMEM lane quadrant = warp % 4, column half = (warp - 8) / 4).  All waits are bounded.
 #include <cuda.h>
 
@@ -25,19 +27,18 @@ using namespace umma;
 constexpr int D = 64;
 constexpr int QT = 128;          // queries per CTA
 constexpr int KTILE = 128;       // keys per tile
-constexpr int NSTAGE = 4;
+constexpr int NSTAGE = 3;
 constexpr int NTHREADS = 512;
 
 constexpr uint32_t COL_S = 0;    // 2 x 128 fp32 score buffers
 constexpr uint32_t COL_P = 256;  // 2 x 64: bf16 weights (128 keys packed in 64 columns)
-constexpr uint32_t COL_O = 384;  // 64 fp32 output accumulators
+constexpr uint32_t COL_O = 384;  // 80 fp32 accumulators: 64 outputs, column 64 = normaliser
 constexpr uint32_t TMEM_COLS = 512;
 
 constexpr uint32_t OFF_Q = 0;                       // 128 x 64 bf16, 128B swizzle
-constexpr uint32_t OFF_KV = 16384;                  // NSTAGE x (K tile 16 KB, V tile 16 KB)
-constexpr uint32_t OFF_R2 = OFF_KV + NSTAGE * 32768;   // NSTAGE x 128 floats: 1/||k||^2
-constexpr uint32_t OFF_DPART = OFF_R2 + NSTAGE * 512;  // 2 x 128 floats: row sums of the two column halves
-constexpr uint32_t OFF_BAR = OFF_DPART + 1024;
+constexpr uint32_t STAGE_BYTES = 49152;             // K tile 16 KB, V tile 16 KB, scale-column tile 16 KB
+constexpr uint32_t OFF_KV = 16384;                  // NSTAGE stages
+constexpr uint32_t OFF_BAR = OFF_KV + NSTAGE * STAGE_BYTES;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
 static_assert(SMEM_ALLOC > 116 * 1024, "one CTA per SM is assumed (the CTA allocates all of TMEM)");
@@ -47,7 +48,7 @@ enum {
   BAR_QFULL = 0,
   BAR_FULL = 1,      // [4] K and V tiles landed
   BAR_EMPTY = 5,     // [4] stage free: both issuers' commits + 128 norm threads
-  BAR_R2FULL = 9,    // [4] key norms of the stage written (128 norm threads)
+  BAR_R2FULL = 9,    // [4] values scaled by 1/||k||^2 and the scale column written (128 norm threads)
   BAR_SFULL = 13,    // [2] scores in TMEM
   BAR_SEMPTY = 15,   // [2] scores read (256 builders)
   BAR_PFULL = 17,    // [2] weights stored (256 builders)
@@ -83,10 +84,9 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   auto bar = [&](int i) { return reinterpret_cast<uint64_t*>(base + OFF_BAR) + i; };
-  auto ktile = [&](int s) { return base + OFF_KV + s * 32768; };
-  auto vtile = [&](int s) { return base + OFF_KV + s * 32768 + 16384; };
-  auto r2buf = [&](int s) { return reinterpret_cast<float*>(base + OFF_R2 + s * 512); };
-  float* dpart = reinterpret_cast<float*>(base + OFF_DPART);
+  auto ktile = [&](int s) { return base + OFF_KV + s * STAGE_BYTES; };
+  auto vtile = [&](int s) { return base + OFF_KV + s * STAGE_BYTES + 16384; };
+  auto rtile = [&](int s) { return base + OFF_KV + s * STAGE_BYTES + 32768; };   // column group 64..127 of the B operand
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
   volatile int* abort_flag = &abort_s;
@@ -118,6 +118,10 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmV);
   }
+  // the scale-column tiles are zero except for one bf16 per key row, rewritten for every key tile
+  for (int i = tid; i < NSTAGE * 1024; i += NTHREADS)
+    *reinterpret_cast<uint4*>(rtile(i >> 10) + (i & 1023) * 16) = make_uint4(0u, 0u, 0u, 0u);
+  fence_async_smem();
   if (warp == 0) {
     tmem_alloc(&tmem_base_s, TMEM_COLS);
     tmem_relinquish();
@@ -167,11 +171,12 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   } else if (warp == 2) {
     // =========================== apply MMA issuer: O += P V ===========================
     if (lane == 0) {
-      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 64);     // A tmem, B MN-major
-      const uint64_t dmn = smem_desc(0, 8192, 1024, kSwizzle128B);
+      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);     // A tmem, B MN-major, N = 64 + 16
+      // MN-major, 128B swizzle: 8 key rows per 1024-byte atom (SBO), second group of 64 columns 16 KB on (LBO)
+      const uint64_t dmn = smem_desc(0, 16384, 1024, kSwizzle128B);
       for (int j = 0; j < ntiles && ok; ++j) {
         const int s = j % NSTAGE, b = j & 1;
-        ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
+        ok = wait_or_abort(bar(BAR_R2FULL + s), (j / NSTAGE) & 1, abort_flag) &&
              wait_or_abort(bar(BAR_PFULL + b), (j >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -205,7 +210,22 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           ss1 = fmaf(hi, hi, ss1);
         }
       }
-      r2buf(s)[kr] = inv_or_zero(ss0 + ss1);
+      const float r2 = inv_or_zero(ss0 + ss1);
+      unsigned char* vt = vtile(s);
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        uint4* pv = reinterpret_cast<uint4*>(vt + sw128_offset(kr, ch));
+        const uint4 raw = *pv;
+        uint4 sc;
+        sc.x = pack_bf16(__uint_as_float(raw.x << 16) * r2, __uint_as_float(raw.x & 0xFFFF0000u) * r2);
+        sc.y = pack_bf16(__uint_as_float(raw.y << 16) * r2, __uint_as_float(raw.y & 0xFFFF0000u) * r2);
+        sc.z = pack_bf16(__uint_as_float(raw.z << 16) * r2, __uint_as_float(raw.z & 0xFFFF0000u) * r2);
+        sc.w = pack_bf16(__uint_as_float(raw.w << 16) * r2, __uint_as_float(raw.w & 0xFFFF0000u) * r2);
+        *pv = sc;
+      }
+      // column 64 of the B operand: the scale itself (element 0 of 16-byte chunk 0 of this key row)
+      *reinterpret_cast<uint16_t*>(rtile(s) + sw128_offset(kr, 0)) = (uint16_t)(pack_bf16(r2, 0.f) & 0xFFFFu);
+      fence_async_smem();
       mbar_arrive(bar(BAR_R2FULL + s));
       mbar_arrive(bar(BAR_EMPTY + s));
     }
@@ -215,38 +235,26 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int ch = (warp - 8) >> 2;              // column half: keys [64 ch, 64 ch + 64) of the tile
     const int rowl = q4 * 32 + lane;             // query row inside the tile (= TMEM lane)
     const int qrow = q0 + rowl;
-    float dsum = 0.f;
     for (int j = 0; j < ntiles && ok; ++j) {
-      const int s = j % NSTAGE, b = j & 1;
-      ok = wait_or_abort(bar(BAR_SFULL + b), (j >> 1) & 1, abort_flag) &&
-           wait_or_abort(bar(BAR_R2FULL + s), (j / NSTAGE) & 1, abort_flag);
+      const int b = j & 1;
+      ok = wait_or_abort(bar(BAR_SFULL + b), (j >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      const float* r2 = r2buf(s) + ch * 64;
       const uint32_t scol = tmem_addr(tb, q4 * 32, COL_S + b * 128 + ch * 64);
       const bool diag = (j == ntiles - 1);
       const int key0 = j * KTILE + ch * 64;
       uint32_t ya[32], yb[32], pk[32];
       auto weigh = [&](const uint32_t (&y)[32], int half) {
 #pragma unroll
-        for (int jj = 0; jj < 32; jj += 4) {
+        for (int jj = 0; jj < 32; jj += 2) {
           const int c = half * 32 + jj;
-          const float4 rr = *reinterpret_cast<const float4*>(r2 + c);
-          float w0 = __uint_as_float(y[jj]), w1 = __uint_as_float(y[jj + 1]);
-          float w2 = __uint_as_float(y[jj + 2]), w3 = __uint_as_float(y[jj + 3]);
-          w0 = w0 * w0 * rr.x; w1 = w1 * w1 * rr.y; w2 = w2 * w2 * rr.z; w3 = w3 * w3 * rr.w;
+          const float2 sv = make_float2(__uint_as_float(y[jj]), __uint_as_float(y[jj + 1]));
+          float2 w = __fmul2_rn(sv, sv);
           if (diag) {
-            if (key0 + c > qrow) w0 = 0.f;
-            if (key0 + c + 1 > qrow) w1 = 0.f;
-            if (key0 + c + 2 > qrow) w2 = 0.f;
-            if (key0 + c + 3 > qrow) w3 = 0.f;
+            if (key0 + c > qrow) w.x = 0.f;
+            if (key0 + c + 1 > qrow) w.y = 0.f;
           }
-          const uint32_t p0 = pack_bf16(w0, w1), p1 = pack_bf16(w2, w3);
-          pk[c / 2] = p0;
-          pk[c / 2 + 1] = p1;
-          // the normaliser sums the rounded weights, the same numbers the apply MMA multiplies with V
-          dsum += (__uint_as_float(p0 << 16) + __uint_as_float(p0 & 0xFFFF0000u)) +
-                  (__uint_as_float(p1 << 16) + __uint_as_float(p1 & 0xFFFF0000u));
+          pk[c / 2] = pack_bf16(w.x, w.y);
         }
       };
       tmem_ld32(scol, ya);
@@ -267,15 +275,15 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
     // ---- epilogue: out = O / D ----
     if (ok) ok = wait_or_abort(bar(BAR_ODONE), 0, abort_flag);
-    dpart[ch * 128 + rowl] = dsum;
-    asm volatile("bar.sync 1, 256;" ::: "memory");
     if (ok) {
       tc_fence_after();
-      const float den = dpart[rowl] + dpart[128 + rowl];
-      const float inv = den > 0.f ? 1.f / den : 0.f;
-      uint32_t o[32];
+      uint32_t o[32], dn[16];
       tmem_ld32(tmem_addr(tb, q4 * 32, COL_O + ch * 32), o);
+      tmem_ld16(tmem_addr(tb, q4 * 32, COL_O + 64), dn);
       tmem_wait_ld(o);
+      tmem_wait_ld(dn);
+      const float den = __uint_as_float(dn[0]);
+      const float inv = den > 0.f ? 1.f / den : 0.f;
       if (qrow < args.Tlen) {
         __nv_bfloat16* dst = args.out + ((size_t)bh * args.Tlen + qrow) * D + ch * 32;
 #pragma unroll
