@@ -112,7 +112,8 @@ typedef struct kata_opts {
  * Quadratic ("flash-style") forward: the definition evaluated tile by tile, never forming
  * the d_k^2-wide state (section "Why the PSD feature keeps to O(T) or O(T^2)"; weights from
  * the rank-one lift identity <uu^T,vv^T>_F = (u^T v)^2).  O(T^2) work.  C is ignored.
- * Needs no workspace.
+ * Workspace: kata_workspace_bytes(KATA_FN_QUADRATIC, ...) -- the tensor-core path keeps the values scaled
+ * by 1/||k||^2 there (about the size of v); the fp32 path needs none.
  */
 int kata_fwd_quadratic(const void* q, const void* k, const void* v, void* out,
                        int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);

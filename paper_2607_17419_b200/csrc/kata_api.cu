@@ -184,7 +184,7 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   if (r.o.impl == KATA_IMPL_TENSOR && !r.tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
   r.plan = ScanPlan{(T + kChunk - 1) / kChunk, 0, 1, 0};
   r.state_elems = 0;
-  r.inner_bytes = 0;
+  r.inner_bytes = (fn == KATA_FN_QUADRATIC && r.tensor) ? tc_quadratic_workspace_bytes(r.p) : 0;
   if (fn != KATA_FN_QUADRATIC) {
     if (r.tensor && r.o.s_pre != nullptr) r.tensor = false;   // state export lives on the SIMT pipeline
     st = make_plan(fn, r.p, r.o, r.tensor, r.plan, r.state_elems);
@@ -198,7 +198,7 @@ int run_device(int fn, Prepared& r, void* ws) {
   LaunchCtx ctx{r.o.stream, 0, KATA_OK};
   float* wsf = static_cast<float*>(ws);
   if (fn == KATA_FN_QUADRATIC) {
-    if (r.tensor) tc_quadratic(r.p, r.o.device_status, ctx);
+    if (r.tensor) tc_quadratic(r.p, ws, r.o.device_status, ctx);
     else simt_quadratic(r.p, ctx);
   } else {
     const bool use_scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || r.plan.n_groups > 1;

@@ -75,7 +75,8 @@ void order1_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float
 
 // Tensor-core kernels (tcgen05/TMEM; bf16, d_k = d_v = 64)
 bool tc_supported(const Problem& p, int fn, bool scan);
-void tc_quadratic(const Problem& p, int* device_status, LaunchCtx& ctx);
+size_t tc_quadratic_workspace_bytes(const Problem& p);
+void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx);
 size_t tc_chunked_state_elems();
 int tc_chunked_slices();
 void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, int* device_status,

@@ -1,19 +1,23 @@
 // Quadratic ("flash-style") KATA forward on the Blackwell tensor cores (tcgen05 + TMEM), bf16, d_k = d_v = 64.
 //
-// One CTA = one head x one tile of 128 queries; it walks the key tiles j <= i of 128 keys:
-//   scores   S = Q K_j^T                      tcgen05 kind::f16, both operands from TMA-loaded 128B-swizzled tiles,
-//                                             fp32 result in TMEM (two buffers)
-//   weights  P = S^2 (causal mask on the      packed fp32x2 multiplies on the TMEM read-back; rounded to bf16 and
-//            diagonal tile)                   stored back to TMEM
-//   apply    [O | D] += P [V/||k||^2 | 1/||k||^2]   tcgen05 kind::f16, A = P from TMEM, B = the value tile (scaled in
-//                                             place by the norm warps) plus one extra column group, MN-major, N = 80:
-//                                             the normaliser is column 64 of the same accumulator
+// Pre-pass (one light kernel per call): V'[i] = v_i / ||k_i||^2 (bf16) and r[i] = 1 / ||k_i||^2 (bf16) into
+// the workspace, so that the key scale never touches the 128 x 128 weight tiles.
+//
+// Main kernel: one CTA = one head x one tile of 128 queries; it walks the key tiles j <= i of 128 keys:
+//   scores   S = Q K_j^T            tcgen05 kind::f16; A = the query tile, copied once into TMEM; B = the
+//                                   TMA-loaded 128B-swizzled key tile; fp32 result in one of three TMEM buffers
+//   weights  P = S^2 (causal mask   packed fp32x2 multiplies on the TMEM read-back, rounded to bf16 and stored
+//            on the diagonal tile)  back over the first 64 columns of the same buffer
+//   apply    [O | D] += P [V' | r]  tcgen05 kind::f16, A = P from TMEM, B = the V' tile plus one extra column
+//                                   group holding r, MN-major, N = 80: the normaliser is column 64 of the
+//                                   same accumulator
 //   epilogue out = O / D (0 where D = 0)      the gate/normalise step of the readout
 // There is no running maximum and no rescaling: the weights are polynomial.  The query norm cancels between
 // numerator and denominator and is never applied.  The d^2-wide feature state is never formed.
 //
-// Warps (512 threads): 0 TMA producer, 1 score-MMA issuer, 2 apply-MMA issuer, 4-7 key norms + value scaling, 8-15 weight
-// builders (TMEM lane quadrant = warp % 4, column half = (warp - 8) / 4).  All waits are bounded.
+// Warps (384 threads): 0 TMA producer (its lanes also place r into the extra column group), 1 score-MMA
+// issuer, 2 apply-MMA issuer, 3 idle, 4-11 weight builders (TMEM lane quadrant = warp % 4, column half =
+// (warp - 4) / 4).  All waits are bounded.
 #include <cuda.h>
 
 #include "kata_common.cuh"
@@ -27,16 +31,18 @@ using namespace umma;
 constexpr int D = 64;
 constexpr int QT = 128;          // queries per CTA
 constexpr int KTILE = 128;       // keys per tile
-constexpr int NSTAGE = 3;
-constexpr int NTHREADS = 512;
+constexpr int NSTAGE = 3;        // shared-memory stages of (K, V', r) tiles
+constexpr int NBUF = 3;          // TMEM score / weight buffers
+constexpr int NTHREADS = 384;
+constexpr int WARP_BLD0 = 4;
 
-constexpr uint32_t COL_S = 0;    // 2 x 128 fp32 score buffers
-constexpr uint32_t COL_P = 256;  // 2 x 64: bf16 weights (128 keys packed in 64 columns)
+constexpr uint32_t COL_S = 0;    // 3 x 128 fp32 score buffers; the bf16 weights overwrite columns [0,64) of a buffer
 constexpr uint32_t COL_O = 384;  // 80 fp32 accumulators: 64 outputs, column 64 = normaliser
+constexpr uint32_t COL_Q = 464;  // 32: the query tile as bf16 pairs (A operand of the score MMA)
 constexpr uint32_t TMEM_COLS = 512;
 
-constexpr uint32_t OFF_Q = 0;                       // 128 x 64 bf16, 128B swizzle
-constexpr uint32_t STAGE_BYTES = 49152;             // K tile 16 KB, V tile 16 KB, scale-column tile 16 KB
+constexpr uint32_t OFF_Q = 0;                       // 128 x 64 bf16, 128B swizzle (staging for the TMEM copy)
+constexpr uint32_t STAGE_BYTES = 49152;             // K tile 16 KB, V' tile 16 KB, scale-column tile 16 KB
 constexpr uint32_t OFF_KV = 16384;                  // NSTAGE stages
 constexpr uint32_t OFF_BAR = OFF_KV + NSTAGE * STAGE_BYTES;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
@@ -45,21 +51,21 @@ static_assert(SMEM_ALLOC > 116 * 1024, "one CTA per SM is assumed (the CTA alloc
 
 // Every barrier has waiters that consume each of its phases in order (no waiter skips a phase).
 enum {
-  BAR_QFULL = 0,
-  BAR_FULL = 1,      // [4] K and V tiles landed
-  BAR_EMPTY = 5,     // [4] stage free: both issuers' commits + 128 norm threads
-  BAR_R2FULL = 9,    // [4] values scaled by 1/||k||^2 and the scale column written (128 norm threads)
-  BAR_SFULL = 13,    // [2] scores in TMEM
-  BAR_SEMPTY = 15,   // [2] scores read (256 builders)
-  BAR_PFULL = 17,    // [2] weights stored (256 builders)
-  BAR_PEMPTY = 19,   // [2] weights consumed by the apply MMA
-  BAR_ODONE = 21,
-  BAR_DRAIN = 22,
-  BAR_COUNT = 23
+  BAR_QFULL = 0,     // query tile landed in shared memory
+  BAR_QTMEM = 1,     // query tile copied to TMEM (256 builders)
+  BAR_FULL = 2,      // [3] K and V' tiles landed and the scale column written (TMA bytes + 32 producer lanes)
+  BAR_EMPTY = 5,     // [3] stage free: both issuers' commits
+  BAR_SFULL = 8,     // [3] scores in TMEM
+  BAR_PFULL = 11,    // [3] weights stored (256 builders)
+  BAR_PEMPTY = 14,   // [3] weights consumed by the apply MMA: the buffer may take new scores
+  BAR_ODONE = 17,
+  BAR_DRAIN = 18,
+  BAR_COUNT = 19
 };
 
 struct QArgs {
   __nv_bfloat16* out;
+  const __nv_bfloat16* rscale;   // [BH][T] bf16: 1 / ||k||^2
   int* device_status;
   int Tlen;
 };
@@ -76,6 +82,37 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Pre-pass: one warp per 4 key rows (8 lanes x 16 bytes per row).  V' = v / ||k||^2, r = 1 / ||k||^2.
+__global__ void __launch_bounds__(256) quad_prescale_kernel(const __nv_bfloat16* __restrict__ k,
+                                                            const __nv_bfloat16* __restrict__ v,
+                                                            __nv_bfloat16* __restrict__ vs,
+                                                            __nv_bfloat16* __restrict__ rscale, size_t n_rows) {
+  const size_t row = (size_t)blockIdx.x * 32 + (threadIdx.x >> 3);
+  const int part = threadIdx.x & 7;
+  if (row >= n_rows) return;
+  const uint4 kraw = *reinterpret_cast<const uint4*>(k + row * D + part * 8);
+  const uint32_t kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
+  float ss = 0.f;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float lo = __uint_as_float(kw[e] << 16), hi = __uint_as_float(kw[e] & 0xFFFF0000u);
+    ss = fmaf(lo, lo, ss);
+    ss = fmaf(hi, hi, ss);
+  }
+  ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+  ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+  ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+  const float r2 = inv_or_zero(ss);
+  const uint4 vraw = *reinterpret_cast<const uint4*>(v + row * D + part * 8);
+  uint4 sc;
+  sc.x = pack_bf16(__uint_as_float(vraw.x << 16) * r2, __uint_as_float(vraw.x & 0xFFFF0000u) * r2);
+  sc.y = pack_bf16(__uint_as_float(vraw.y << 16) * r2, __uint_as_float(vraw.y & 0xFFFF0000u) * r2);
+  sc.z = pack_bf16(__uint_as_float(vraw.z << 16) * r2, __uint_as_float(vraw.z & 0xFFFF0000u) * r2);
+  sc.w = pack_bf16(__uint_as_float(vraw.w << 16) * r2, __uint_as_float(vraw.w & 0xFFFF0000u) * r2);
+  *reinterpret_cast<uint4*>(vs + row * D + part * 8) = sc;
+  if (part == 0) rscale[row] = __float2bfloat16_rn(r2);
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -100,14 +137,13 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   if (tid == 0) {
     abort_s = 0;
     mbar_init(bar(BAR_QFULL), 1);
+    mbar_init(bar(BAR_QTMEM), 256);
     for (int i = 0; i < NSTAGE; ++i) {
-      mbar_init(bar(BAR_FULL + i), 1);
-      mbar_init(bar(BAR_EMPTY + i), 2 + 128);
-      mbar_init(bar(BAR_R2FULL + i), 128);
+      mbar_init(bar(BAR_FULL + i), 1 + 32);
+      mbar_init(bar(BAR_EMPTY + i), 2);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < NBUF; ++i) {
       mbar_init(bar(BAR_SFULL + i), 1);
-      mbar_init(bar(BAR_SEMPTY + i), 256);
       mbar_init(bar(BAR_PFULL + i), 256);
       mbar_init(bar(BAR_PEMPTY + i), 1);
     }
@@ -133,111 +169,98 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   bool ok = true;
 
   if (warp == 0) {
-    // =========================== TMA producer ===========================
+    // =========================== TMA producer (+ scale column) ===========================
     if (lane == 0) {
       mbar_arrive_expect_tx(bar(BAR_QFULL), 16384);
       tma_load_3d(base + OFF_Q, &tmQ, bar(BAR_QFULL), 0, q0, bh);
-      for (int j = 0; j < ntiles && ok; ++j) {
-        const int s = j % NSTAGE;
-        ok = wait_or_abort(bar(BAR_EMPTY + s), ((j / NSTAGE) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar(BAR_FULL + s), 32768);
+    }
+    const __nv_bfloat16* rs = args.rscale + (size_t)bh * args.Tlen;
+    for (int j = 0; j < ntiles && ok; ++j) {
+      const int s = j % NSTAGE;
+      ok = wait_or_abort(bar(BAR_EMPTY + s), ((j / NSTAGE) & 1) ^ 1, abort_flag);
+      if (!ok) break;
+      if (lane == 0) {
+        mbar_arrive_expect_tx(bar(BAR_FULL + s), 32768);   // K and V' tiles
         tma_load_3d(ktile(s), &tmK, bar(BAR_FULL + s), 0, j * KTILE, bh);
         tma_load_3d(vtile(s), &tmV, bar(BAR_FULL + s), 0, j * KTILE, bh);
       }
+      // column 64 of the B operand: r for the 128 keys of the tile (element 0 of chunk 0 of each key row)
+      unsigned char* rt = rtile(s);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int kr = lane * 4 + e, key = j * KTILE + kr;
+        const unsigned short rv = key < args.Tlen ? __bfloat16_as_ushort(rs[key]) : (unsigned short)0;
+        *reinterpret_cast<uint16_t*>(rt + sw128_offset(kr, 0)) = rv;
+      }
+      fence_async_smem();
+      mbar_arrive(bar(BAR_FULL + s));
     }
   } else if (warp == 1) {
     // =========================== score MMA issuer: S = Q K^T ===========================
     if (lane == 0) {
       const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 128);
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
-      const uint32_t qa = smem_u32(base + OFF_Q);
-      ok = wait_or_abort(bar(BAR_QFULL), 0, abort_flag);
+      ok = wait_or_abort(bar(BAR_QTMEM), 0, abort_flag);
       for (int j = 0; j < ntiles && ok; ++j) {
-        const int s = j % NSTAGE, b = j & 1;
+        const int s = j % NSTAGE, b = j % NBUF;
         ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_SEMPTY + b), ((j >> 1) & 1) ^ 1, abort_flag);
+             wait_or_abort(bar(BAR_PEMPTY + b), ((j / NBUF) & 1) ^ 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         const uint32_t ka = smem_u32(ktile(s));
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          mma_f16_ss(tb + COL_S + b * 128, dk + (uint64_t)(((qa + ks * 32) >> 4) & 0x3FFF),
-                     dk + (uint64_t)(((ka + ks * 32) >> 4) & 0x3FFF), idesc, ks > 0);
+          mma_f16_ts(tb + COL_S + b * 128, tb + COL_Q + ks * 8, dk + (uint64_t)(((ka + ks * 32) >> 4) & 0x3FFF),
+                     idesc, ks > 0);
         mma_commit(bar(BAR_SFULL + b));
         mma_commit(bar(BAR_EMPTY + s));
       }
     }
   } else if (warp == 2) {
-    // =========================== apply MMA issuer: O += P V ===========================
+    // =========================== apply MMA issuer: [O | D] += P [V' | r] ===========================
     if (lane == 0) {
       const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);     // A tmem, B MN-major, N = 64 + 16
       // MN-major, 128B swizzle: 8 key rows per 1024-byte atom (SBO), second group of 64 columns 16 KB on (LBO)
       const uint64_t dmn = smem_desc(0, 16384, 1024, kSwizzle128B);
       for (int j = 0; j < ntiles && ok; ++j) {
-        const int s = j % NSTAGE, b = j & 1;
-        ok = wait_or_abort(bar(BAR_R2FULL + s), (j / NSTAGE) & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_PFULL + b), (j >> 1) & 1, abort_flag);
+        const int s = j % NSTAGE, b = j % NBUF;
+        ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
+             wait_or_abort(bar(BAR_PFULL + b), (j / NBUF) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         const uint32_t va = smem_u32(vtile(s));
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          mma_f16_ts(tb + COL_O, tb + COL_P + b * 64 + ks * 8, dmn + (uint64_t)(((va + ks * 2048) >> 4) & 0x3FFF),
+          mma_f16_ts(tb + COL_O, tb + COL_S + b * 128 + ks * 8, dmn + (uint64_t)(((va + ks * 2048) >> 4) & 0x3FFF),
                      idesc, (j > 0 || ks > 0) ? 1u : 0u);
         mma_commit(bar(BAR_PEMPTY + b));
         mma_commit(bar(BAR_EMPTY + s));
       }
       if (ok) mma_commit(bar(BAR_ODONE));
     }
-  } else if (warp >= 4 && warp < 8) {
-    // =========================== key norms (128 threads, one key each) ===========================
-    const int kr = tid - 128;
-    for (int j = 0; j < ntiles && ok; ++j) {
-      const int s = j % NSTAGE;
-      ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag);
-      if (!ok) break;
-      const unsigned char* kt = ktile(s);
-      float ss0 = 0.f, ss1 = 0.f;
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(kt + sw128_offset(kr, ch));
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xFFFF0000u);
-          ss0 = fmaf(lo, lo, ss0);
-          ss1 = fmaf(hi, hi, ss1);
-        }
-      }
-      const float r2 = inv_or_zero(ss0 + ss1);
-      unsigned char* vt = vtile(s);
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        uint4* pv = reinterpret_cast<uint4*>(vt + sw128_offset(kr, ch));
-        const uint4 raw = *pv;
-        uint4 sc;
-        sc.x = pack_bf16(__uint_as_float(raw.x << 16) * r2, __uint_as_float(raw.x & 0xFFFF0000u) * r2);
-        sc.y = pack_bf16(__uint_as_float(raw.y << 16) * r2, __uint_as_float(raw.y & 0xFFFF0000u) * r2);
-        sc.z = pack_bf16(__uint_as_float(raw.z << 16) * r2, __uint_as_float(raw.z & 0xFFFF0000u) * r2);
-        sc.w = pack_bf16(__uint_as_float(raw.w << 16) * r2, __uint_as_float(raw.w & 0xFFFF0000u) * r2);
-        *pv = sc;
-      }
-      // column 64 of the B operand: the scale itself (element 0 of 16-byte chunk 0 of this key row)
-      *reinterpret_cast<uint16_t*>(rtile(s) + sw128_offset(kr, 0)) = (uint16_t)(pack_bf16(r2, 0.f) & 0xFFFFu);
-      fence_async_smem();
-      mbar_arrive(bar(BAR_R2FULL + s));
-      mbar_arrive(bar(BAR_EMPTY + s));
-    }
-  } else if (warp >= 8) {
+  } else if (warp >= WARP_BLD0) {
     // =========================== weight builders (256 threads) ===========================
     const uint32_t q4 = warp & 3;
-    const int ch = (warp - 8) >> 2;              // column half: keys [64 ch, 64 ch + 64) of the tile
+    const int ch = (warp - WARP_BLD0) >> 2;      // column half: keys [64 ch, 64 ch + 64) of the tile
     const int rowl = q4 * 32 + lane;             // query row inside the tile (= TMEM lane)
     const int qrow = q0 + rowl;
+    // the query tile goes to TMEM once: this thread copies features [32 ch, 32 ch + 32) of its row
+    ok = wait_or_abort(bar(BAR_QFULL), 0, abort_flag);
+    if (ok) {
+      uint32_t qw[16];
+#pragma unroll
+      for (int cix = 0; cix < 4; ++cix) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(base + OFF_Q + sw128_offset(rowl, ch * 4 + cix));
+        qw[4 * cix] = raw.x; qw[4 * cix + 1] = raw.y; qw[4 * cix + 2] = raw.z; qw[4 * cix + 3] = raw.w;
+      }
+      tmem_st16(tmem_addr(tb, q4 * 32, COL_Q + ch * 16), qw);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(BAR_QTMEM));
+    }
     for (int j = 0; j < ntiles && ok; ++j) {
-      const int b = j & 1;
-      ok = wait_or_abort(bar(BAR_SFULL + b), (j >> 1) & 1, abort_flag);
+      const int b = j % NBUF;
+      ok = wait_or_abort(bar(BAR_SFULL + b), (j / NBUF) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       const uint32_t scol = tmem_addr(tb, q4 * 32, COL_S + b * 128 + ch * 64);
@@ -262,13 +285,13 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       tmem_ld32(scol + 32, yb);
       weigh(ya, 0);
       tmem_wait_ld(yb);
-      tc_fence_before();
-      mbar_arrive(bar(BAR_SEMPTY + b));          // this thread's scores are in registers
       weigh(yb, 1);
-      ok = wait_or_abort(bar(BAR_PEMPTY + b), ((j >> 1) & 1) ^ 1, abort_flag);
-      if (!ok) break;
+      // the weights overwrite score columns [0,64) of the buffer, which the column-half-0 warp of this
+      // quadrant reads: both warps of the quadrant must have their scores in registers first
+      tc_fence_before();
+      asm volatile("bar.sync %0, 64;" ::"r"(1 + (int)q4) : "memory");
       tc_fence_after();
-      tmem_st32(tmem_addr(tb, q4 * 32, COL_P + b * 64 + ch * 32), pk);
+      tmem_st32(tmem_addr(tb, q4 * 32, COL_S + b * 128 + ch * 32), pk);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_PFULL + b));
@@ -344,10 +367,23 @@ bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T) {
 
 }  // namespace
 
-void tc_quadratic(const Problem& p, int* device_status, LaunchCtx& ctx) {
+// workspace: V' [BH][T][64] bf16, then r [BH][T] bf16
+static size_t vs_bytes(const Problem& p) { return ((size_t)p.B * p.H * p.T * D * 2 + 255) / 256 * 256; }
+
+size_t tc_quadratic_workspace_bytes(const Problem& p) {
+  return vs_bytes(p) + ((size_t)p.B * p.H * p.T * 2 + 255) / 256 * 256;
+}
+
+void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx) {
   const int BH = p.B * p.H;
+  __nv_bfloat16* vs = static_cast<__nv_bfloat16*>(workspace);
+  __nv_bfloat16* rscale = reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(workspace) + vs_bytes(p));
+  const size_t n_rows = (size_t)BH * p.T;
+  quad_prescale_kernel<<<(unsigned)((n_rows + 31) / 32), 256, 0, ctx.stream>>>(
+      static_cast<const __nv_bfloat16*>(p.k), static_cast<const __nv_bfloat16*>(p.v), vs, rscale, n_rows);
+  note_launch(ctx);
   CUtensorMap tmQ, tmK, tmV;
-  if (!make_map(&tmQ, p.q, BH, p.T) || !make_map(&tmK, p.k, BH, p.T) || !make_map(&tmV, p.v, BH, p.T)) {
+  if (!make_map(&tmQ, p.q, BH, p.T) || !make_map(&tmK, p.k, BH, p.T) || !make_map(&tmV, vs, BH, p.T)) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }
@@ -357,7 +393,7 @@ void tc_quadratic(const Problem& p, int* device_status, LaunchCtx& ctx) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-  QArgs a{static_cast<__nv_bfloat16*>(p.out), device_status, p.T};
+  QArgs a{static_cast<__nv_bfloat16*>(p.out), rscale, device_status, p.T};
   tc_quad_kernel<<<dim3((p.T + QT - 1) / QT, BH), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
   note_launch(ctx);
 }
