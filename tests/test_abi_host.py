@@ -83,7 +83,10 @@ def test_invalid_arguments(L, fn):
 
 def test_scan_workspace_and_plan(L):
     o = kb.make_opts(kb.KATA_BF16)
-    assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 4, 16, 4096, 64, 64, 64, o) == 0
+    # tensor-core quadratic path: scaled values (bf16, size of v) + one bf16 scale per key
+    assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 4, 16, 4096, 64, 64, 64, o) == 4 * 16 * 4096 * (64 + 1) * 2
+    o32 = kb.make_opts(kb.KATA_F32)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 4, 16, 4096, 64, 64, 64, o32) == 0
     assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 8, 16, 4096, 64, 64, 64, o) == 0   # sequential
     assert kb.kata_scan_plan(kb.KATA_FN_CHUNKED, 8, 16, 4096, 64, 64, 64, o)[0] == 1
     o = kb.make_opts(kb.KATA_BF16, inter_chunk=kb.KATA_SCAN, scan_group=16, impl=kb.KATA_IMPL_SIMT)
