@@ -713,6 +713,10 @@ int tc_chunked_slices() { return NSLICE; }
 
 void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, int* device_status,
                 LaunchCtx& ctx) {
+  if (!use_scan) {   // whole sequence in one pass: the token-major streaming kernel
+    tc_chunked_stream(p, device_status, ctx);
+    return;
+  }
   const int BH = p.B * p.H;
   CUtensorMap tmQ, tmK, tmV;
   if (!make_map(&tmQ, p.q, BH, p.T, 64, true) || !make_map(&tmK, p.k, BH, p.T, 64, true) ||
@@ -731,16 +735,6 @@ void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws
   a.device_status = device_status;
   a.Tlen = p.T;
   a.n_chunks = plan.n_chunks;
-  if (!use_scan) {
-    a.init_state = nullptr;
-    a.final_state = nullptr;
-    a.chunks_per_group = plan.n_chunks;
-    a.n_groups = 1;
-    a.write_out = 1;
-    tc_chunk_kernel<<<dim3(NSLICE, BH, 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
-    note_launch(ctx);
-    return;
-  }
   const int NG = plan.n_groups;
   const size_t E = tc_chunked_state_elems();
   float* bufA = ws;

@@ -1,0 +1,630 @@
+// Chunked (linear-state) KATA forward on the Blackwell tensor cores, token-major, bf16, d_k = d_v = 64,
+// whole sequence in one pass (the sequential inter-chunk recurrence of the chunked form).
+//
+// One CTA owns one head and a slice of 8 value columns and walks the sequence in tiles of 128 tokens.
+// The feature state is never expanded: with k' = k / ||k||^2 the state of the slice is
+//   S[(b,v), a] = sum_t k'[t,b] v[t,v] k[t,a]   and   Z[b, a] = sum_t k'[t,b] k[t,a]       (a, b < 64, v < 8)
+// which is the rank-one lift <psi(q), psi(k)> = (q.k)^2 contracted in two stages.  S and Z are symmetric in
+// (a, b), so only the 16 x 16 blocks with a-block <= b-block are kept (160 + 64 accumulator columns in TMEM).
+// Per tile of 128 tokens:
+//   update   S += W^T K          W[t,(b,v)] = k[t,b] v'[t,v] (v' = v / ||k||^2), one bf16 row per token, built
+//                                by token threads in shared memory (MN-major A operand); B = the TMA-loaded
+//                                key tile as it is; fp32 accumulators stay in TMEM for the whole sequence
+//   snapshot S' = bf16(S)        after each update the accumulators are copied to shared memory as the B operand
+//                                of the read (off-diagonal blocks doubled, which stands for the dropped half)
+//   read     Y[t,(b,v)] = sum_a q[t,a] S'[(b,v),a]     tokens on the TMEM lanes, 8 pieces of 80 columns;
+//            N_inter[t,v] = sum_b q[t,b] Y[t,(b,v)]    then is a dot product inside one thread
+//   intra    P = (Q K^T)^2 masked causally, [O | D] += P [V' | 1/||k||^2]   as in the quadratic form
+//   out      (N_inter + O) / (D_inter + D)             (0 where the denominator is 0)
+// The query norm cancels and is never applied.
+//
+// Warps (512 threads): 0 TMA producer; 1 update-MMA issuer; 2 read-MMA issuer; 3 intra-tile MMA issuer;
+// 4-7 W builders (warp = b-block, lane = token of a 32-token sub-tile); 8-11 readers and epilogue (thread =
+// token); 12-15 key scales, query tile to TMEM, weights P, state snapshot.  All waits are bounded.
+#include <cuda.h>
+
+#include "kata_common.cuh"
+#include "kata_umma.cuh"
+
+namespace kata {
+namespace {
+
+using namespace umma;
+
+constexpr int D = 64;
+constexpr int CT = 128;          // tokens per tile
+constexpr int VS = 8;            // value columns per CTA
+constexpr int NSLICE = D / VS;
+constexpr int NTHREADS = 512;
+constexpr int WARP_U = 1, WARP_R = 2, WARP_I = 3, WARP_BLD0 = 4, WARP_RD0 = 8, WARP_AUX0 = 12;
+
+// ---- TMEM columns ----
+constexpr uint32_t COL_S = 0;     // b-block beta at 8 beta (beta + 1): 16 (beta + 1) columns (a < 16 (beta + 1))
+constexpr uint32_t COL_Z = 160;   // 64 columns, lanes 0..63 = b
+constexpr uint32_t COL_Y = 224;   // 2 x 80: read pieces
+constexpr uint32_t COL_P = 384;   // 64 fp32 scores; the bf16 weights overwrite columns [0,32)
+constexpr uint32_t COL_O = 448;   // 16: intra-tile numerator (8) and denominator (column 8)
+constexpr uint32_t COL_Q = 464;   // 32: the query tile as bf16 pairs
+constexpr uint32_t TMEM_COLS = 512;
+
+// ---- shared memory ----
+constexpr uint32_t OFF_KQ = 0;            // 2 stages x (Q tile 16 KB | K tile 16 KB), 128B swizzle
+constexpr uint32_t OFF_VP = 65536;        // 2 stages x 4 KB: [128 keys][8 bf16] v', then [128 keys][8 bf16] (1/||k||^2, 0..)
+constexpr uint32_t OFF_W = 73728;         // 2 x 40 KB: [5 tiles][2 M-atoms][4 groups of 8 tokens][1 KB], MN-major 128B swizzle
+constexpr uint32_t W_BYTES = 40960;
+constexpr uint32_t OFF_SP = 155648;       // 5 blocks x 80 rows x 128 B: the snapshot, K-major 128B swizzle
+constexpr uint32_t SP_BLOCK = 10240;
+constexpr uint32_t OFF_R2 = 206848;       // 2 stages x 128 x (bf16 1/||k||^2 twice)
+constexpr uint32_t OFF_BAR = 207872;
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
+constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
+
+// Every barrier has waiters that consume each of its phases in order.
+enum {
+  BAR_KQ_FULL = 0,    // [2] query and key tiles landed
+  BAR_KQ_EMPTY = 2,   // [2] stage free: update and intra commits + the 128 readers' query rows
+  BAR_PREP = 4,       // [2] key scales and v' of the tile written
+  BAR_QT_FULL = 6,    // query tile copied to TMEM
+  BAR_W_FULL = 7,     // [2] W sub-tile built
+  BAR_W_EMPTY = 9,    // [2] W sub-tile consumed
+  BAR_U_DONE = 11,    // update of the tile complete
+  BAR_R_DONE = 12,    // all read pieces of the tile complete
+  BAR_SNAP_LD = 13,   // accumulators copied out of TMEM: the next update may run
+  BAR_SNAP_ST = 14,   // snapshot stored: the next read may run
+  BAR_Y_FULL = 15,    // [2]
+  BAR_Y_EMPTY = 17,   // [2]
+  BAR_S_FULL = 19,    // scores of a 64-key half in TMEM
+  BAR_P_FULL = 20,    // weights of the half stored
+  BAR_PV0 = 21,       // first half applied (its weights may be overwritten)
+  BAR_O_FULL = 22,    // intra-tile result complete
+  BAR_O_EMPTY = 23,   // intra-tile result read
+  BAR_DRAIN = 24,
+  BAR_COUNT = 25
+};
+
+struct SArgs {
+  const __nv_bfloat16* v;
+  __nv_bfloat16* out;
+  int* device_status;
+  int Tlen;
+};
+
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+  const __nv_bfloat162 r = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+  return *reinterpret_cast<const uint32_t*>(&r);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint64_t at(uint64_t desc, uint32_t saddr) { return desc + (uint64_t)((saddr >> 4) & 0x3FFF); }
+
+// Snapshot placement of read piece p (8 values of b, b-block p / 2): block and byte offset inside the 128-byte rows.
+// Pieces of the b-blocks 0 and 2 share rows (32 + 96 bytes), the two pieces of b-block 1 share rows (64 + 64).
+__device__ __forceinline__ uint32_t sp_block(int p) { return (0x43102210u >> (4 * p)) & 0xFu; }   // 0,1,2,2,0,1,3,4
+__device__ __forceinline__ uint32_t sp_koff(int p) { return p == 3 ? 64u : (p == 4 || p == 5) ? 32u : 0u; }
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const SArgs args) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  auto bar = [&](int i) { return reinterpret_cast<uint64_t*>(base + OFF_BAR) + i; };
+  auto qtile = [&](int s) { return base + OFF_KQ + s * 32768; };
+  auto ktile = [&](int s) { return base + OFF_KQ + s * 32768 + 16384; };
+  auto vptile = [&](int s) { return base + OFF_VP + s * 4096; };
+  auto wbuf = [&](int b) { return base + OFF_W + b * W_BYTES; };
+  auto r2pair = [&](int s) { return reinterpret_cast<uint32_t*>(base + OFF_R2) + s * CT; };
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int slice = blockIdx.x, bh = blockIdx.y;
+  const int v0 = slice * VS;
+  const int nch = (args.Tlen + CT - 1) / CT;
+
+  if (tid == 0) {
+    abort_s = 0;
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(BAR_KQ_FULL + s), 1);
+      mbar_init(bar(BAR_KQ_EMPTY + s), 2 + 128);
+      mbar_init(bar(BAR_PREP + s), 128);
+      mbar_init(bar(BAR_W_FULL + s), 128);
+      mbar_init(bar(BAR_W_EMPTY + s), 1);
+      mbar_init(bar(BAR_Y_FULL + s), 1);
+      mbar_init(bar(BAR_Y_EMPTY + s), 128);
+    }
+    mbar_init(bar(BAR_QT_FULL), 128);
+    mbar_init(bar(BAR_U_DONE), 1);
+    mbar_init(bar(BAR_R_DONE), 1);
+    mbar_init(bar(BAR_SNAP_LD), 128);
+    mbar_init(bar(BAR_SNAP_ST), 128);
+    mbar_init(bar(BAR_S_FULL), 1);
+    mbar_init(bar(BAR_P_FULL), 128);
+    mbar_init(bar(BAR_PV0), 1);
+    mbar_init(bar(BAR_O_FULL), 1);
+    mbar_init(bar(BAR_O_EMPTY), 128);
+    mbar_init(bar(BAR_DRAIN), 3);
+    fence_mbar_init();
+    tma_prefetch_desc(&tmQ);
+    tma_prefetch_desc(&tmK);
+  }
+  // zero: the W buffers (the second M-atom of the Z tile is never written) and the snapshot (state 0, pad rows)
+  for (uint32_t i = tid; i < (2 * W_BYTES + 5 * SP_BLOCK) / 16; i += NTHREADS)
+    *reinterpret_cast<uint4*>(base + OFF_W + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+  static_assert(OFF_W + 2 * W_BYTES == OFF_SP, "the zero fill runs over both regions");
+  fence_async_smem();
+  if (warp == 0) {
+    tmem_alloc(&tmem_base_s, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tb = tmem_base_s;
+  bool ok = true;
+
+  if (warp == 0) {
+    // =========================== TMA producer ===========================
+    if (lane == 0) {
+      for (int j = 0; j < nch && ok; ++j) {
+        const int s = j & 1;
+        ok = wait_or_abort(bar(BAR_KQ_EMPTY + s), ((j >> 1) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar(BAR_KQ_FULL + s), 32768);
+        tma_load_3d(qtile(s), &tmQ, bar(BAR_KQ_FULL + s), 0, j * CT, bh);
+        tma_load_3d(ktile(s), &tmK, bar(BAR_KQ_FULL + s), 0, j * CT, bh);
+      }
+    }
+  } else if (warp == WARP_U) {
+    // =========================== update issuer: S += W^T K ===========================
+    if (lane == 0) {
+      const uint32_t idU[5] = {instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 16), instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 32),
+                               instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 48), instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64),
+                               instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64)};
+      const uint32_t colU[5] = {COL_S + 0, COL_S + 16, COL_S + 48, COL_S + 96, COL_Z};
+      // A: MN-major, 128B swizzle: 64 rows x 8 tokens per 1 KB atom; next 8 tokens +1 KB (SBO), next 64 rows +4 KB (LBO)
+      const uint64_t dA = smem_desc(0, 4096, 1024, kSwizzle128B);
+      // B: the key tile read MN-major (N = feature a, K = token): one atom of 64 features x 8 tokens per 1 KB
+      const uint64_t dB = smem_desc(0, 16384, 1024, kSwizzle128B);
+      for (int j = 0; j < nch && ok; ++j) {
+        const int s = j & 1;
+        ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag);
+        if (ok && j > 0) ok = wait_or_abort(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
+        for (int sc = 0; sc < 4 && ok; ++sc) {
+          const int g = 4 * j + sc, wb = g & 1;
+          ok = wait_or_abort(bar(BAR_W_FULL + wb), (g >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t wa = smem_u32(wbuf(wb)), ka = smem_u32(ktile(s)) + sc * 4096;
+#pragma unroll
+          for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+            for (int tl = 0; tl < 5; ++tl)
+              mma_f16_ss(tb + colU[tl], at(dA, wa + tl * 8192 + ks * 2048), at(dB, ka + ks * 2048), idU[tl],
+                         (g > 0 || ks > 0) ? 1u : 0u);
+          mma_commit(bar(BAR_W_EMPTY + wb));
+        }
+        if (!ok) break;
+        mma_commit(bar(BAR_U_DONE));
+        mma_commit(bar(BAR_KQ_EMPTY + s));
+      }
+    }
+  } else if (warp == WARP_R) {
+    // =========================== read issuer: Y = Q S'^T, 8 pieces ===========================
+    if (lane == 0) {
+      const uint32_t idR = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 80);
+      const uint64_t dS = smem_desc(0, 16, 1024, kSwizzle128B);
+      const uint32_t spa = smem_u32(base + OFF_SP);
+      for (int j = 0; j < nch && ok; ++j) {
+        ok = wait_or_abort(bar(BAR_QT_FULL), j & 1, abort_flag);
+        if (ok && j > 0) ok = wait_or_abort(bar(BAR_SNAP_ST), (j - 1) & 1, abort_flag);
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+          if (!ok) break;
+          const int g = 8 * j + p, yb = g & 1;
+          ok = wait_or_abort(bar(BAR_Y_EMPTY + yb), ((g >> 1) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sbase = spa + sp_block(p) * SP_BLOCK + sp_koff(p);
+#pragma unroll
+          for (int al = 0; al <= (p >> 1); ++al)
+            mma_f16_ts(tb + COL_Y + yb * 80, tb + COL_Q + al * 8, at(dS, sbase + al * 32), idR, al > 0);
+          mma_commit(bar(BAR_Y_FULL + yb));
+        }
+        if (!ok) break;
+        mma_commit(bar(BAR_R_DONE));
+      }
+    }
+  } else if (warp == WARP_I) {
+    // =========================== intra-tile issuer: scores and [O | D] ===========================
+    if (lane == 0) {
+      const uint32_t idQK = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 64);
+      const uint32_t idPV = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 16);
+      const uint64_t dK = smem_desc(0, 16, 1024, kSwizzle128B);
+      for (int j = 0; j < nch && ok; ++j) {
+        const int s = j & 1;
+        ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag) &&
+             wait_or_abort(bar(BAR_QT_FULL), j & 1, abort_flag) &&
+             wait_or_abort(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
+        // the weights of the previous tile's second half are read by its last apply MMAs
+        if (ok && j > 0) ok = wait_or_abort(bar(BAR_O_FULL), (j - 1) & 1, abort_flag);
+        const uint32_t ka = smem_u32(ktile(s)), va = smem_u32(vptile(s));
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (!ok) break;
+          if (h == 1) ok = wait_or_abort(bar(BAR_PV0), j & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            mma_f16_ts(tb + COL_P, tb + COL_Q + ks * 8, at(dK, ka + h * 8192 + ks * 32), idQK, ks > 0);
+          mma_commit(bar(BAR_S_FULL));
+          ok = wait_or_abort(bar(BAR_P_FULL), h, abort_flag);
+          if (ok && h == 0 && j > 0) ok = wait_or_abort(bar(BAR_O_EMPTY), (j - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            // MN-major, no swizzle: 8 keys x 16 bytes per core matrix, next 8 keys +128 (LBO), columns 8..15 +2048 (SBO)
+            mma_f16_ts(tb + COL_O, tb + COL_P + ks * 8, smem_desc(va + h * 1024 + ks * 256, 128, 2048, kSwizzleNone), idPV,
+                       (h > 0 || ks > 0) ? 1u : 0u);
+          if (h == 0) mma_commit(bar(BAR_PV0));
+        }
+        if (!ok) break;
+        mma_commit(bar(BAR_O_FULL));
+        mma_commit(bar(BAR_KQ_EMPTY + s));
+      }
+    }
+  } else if (warp < WARP_RD0) {
+    // =========================== W builders ===========================
+    const int beta = warp - WARP_BLD0;
+    for (int j = 0; j < nch && ok; ++j) {
+      const int s = j & 1;
+      ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag) &&
+           wait_or_abort(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
+      for (int sc = 0; sc < 4 && ok; ++sc) {
+        const int g = 4 * j + sc, wb = g & 1;
+        const int t = sc * 32 + lane;
+        const uint4 k0 = *reinterpret_cast<const uint4*>(ktile(s) + sw128_offset(t, 2 * beta));
+        const uint4 k1 = *reinterpret_cast<const uint4*>(ktile(s) + sw128_offset(t, 2 * beta + 1));
+        const uint4 vp = *reinterpret_cast<const uint4*>(vptile(s) + t * 16);
+        const uint32_t rr = r2pair(s)[t];
+        const uint32_t kw[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
+        ok = wait_or_abort(bar(BAR_W_EMPTY + wb), ((g >> 1) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        unsigned char* wrow = wbuf(wb) + (lane >> 3) * 1024 + (lane & 7) * 128;
+#pragma unroll
+        for (int bl = 0; bl < 16; ++bl) {
+          const uint32_t kbb = __byte_perm(kw[bl >> 1], 0u, (bl & 1) ? 0x3232 : 0x1010);
+          uint4 w;
+          w.x = mul_bf16x2(kbb, vp.x);
+          w.y = mul_bf16x2(kbb, vp.y);
+          w.z = mul_bf16x2(kbb, vp.z);
+          w.w = mul_bf16x2(kbb, vp.w);
+          *reinterpret_cast<uint4*>(wrow + beta * 8192 + (bl >> 3) * 4096 + (((bl & 7) ^ (lane & 7)) << 4)) = w;
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          uint4 w;
+          w.x = mul_bf16x2(kw[4 * h], rr);
+          w.y = mul_bf16x2(kw[4 * h + 1], rr);
+          w.z = mul_bf16x2(kw[4 * h + 2], rr);
+          w.w = mul_bf16x2(kw[4 * h + 3], rr);
+          *reinterpret_cast<uint4*>(wrow + 4 * 8192 + (((2 * beta + h) ^ (lane & 7)) << 4)) = w;
+        }
+        fence_async_smem();
+        mbar_arrive(bar(BAR_W_FULL + wb));
+      }
+    }
+  } else if (warp < WARP_AUX0) {
+    // =========================== readers and epilogue (thread = token) ===========================
+    const uint32_t q4 = warp & 3;
+    const int t = q4 * 32 + lane;
+    for (int j = 0; j < nch && ok; ++j) {
+      const int s = j & 1;
+      ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag);
+      if (!ok) break;
+      uint32_t qw[32];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(qtile(s) + sw128_offset(t, c));
+        qw[4 * c] = raw.x; qw[4 * c + 1] = raw.y; qw[4 * c + 2] = raw.z; qw[4 * c + 3] = raw.w;
+      }
+      mbar_arrive(bar(BAR_KQ_EMPTY + s));
+      float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      float accz = 0.f;
+#pragma unroll
+      for (int p = 0; p < 8; ++p) {
+        if (!ok) break;
+        const int g = 8 * j + p, yb = g & 1;
+        ok = wait_or_abort(bar(BAR_Y_FULL + yb), (g >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t ycol = tmem_addr(tb, q4 * 32, COL_Y + yb * 80);
+        uint32_t ya[32], yb2[32], yz[16];
+        tmem_ld32(ycol, ya);
+        tmem_ld32(ycol + 32, yb2);
+        tmem_ld16(ycol + 64, yz);
+        tmem_wait_ld(ya);
+        auto fold = [&](const uint32_t (&y)[32], int i0) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int b = 8 * p + i0 + i;
+            const float qb = (b & 1) ? bf_hi(qw[b >> 1]) : bf_lo(qw[b >> 1]);
+            const float2 qq = make_float2(qb, qb);
+#pragma unroll
+            for (int vv = 0; vv < 4; ++vv)
+              acc[vv] = __ffma2_rn(qq, make_float2(__uint_as_float(y[8 * i + 2 * vv]), __uint_as_float(y[8 * i + 2 * vv + 1])),
+                                   acc[vv]);
+          }
+        };
+        fold(ya, 0);
+        tmem_wait_ld(yb2);
+        fold(yb2, 4);
+        tmem_wait_ld(yz);
+        tc_fence_before();
+        mbar_arrive(bar(BAR_Y_EMPTY + yb));
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int b = 8 * p + i;
+          const float qb = (b & 1) ? bf_hi(qw[b >> 1]) : bf_lo(qw[b >> 1]);
+          accz = fmaf(qb, __uint_as_float(yz[i]), accz);
+        }
+      }
+      if (!ok) break;
+      ok = wait_or_abort(bar(BAR_O_FULL), j & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t o[16];
+      tmem_ld16(tmem_addr(tb, q4 * 32, COL_O), o);
+      tmem_wait_ld(o);
+      tc_fence_before();
+      mbar_arrive(bar(BAR_O_EMPTY));
+      const float den = accz + __uint_as_float(o[8]);
+      const float inv = den > 0.f ? 1.f / den : 0.f;
+      const int tok = j * CT + t;
+      if (tok < args.Tlen) {
+        uint4 pkt;
+        pkt.x = pack_bf16((acc[0].x + __uint_as_float(o[0])) * inv, (acc[0].y + __uint_as_float(o[1])) * inv);
+        pkt.y = pack_bf16((acc[1].x + __uint_as_float(o[2])) * inv, (acc[1].y + __uint_as_float(o[3])) * inv);
+        pkt.z = pack_bf16((acc[2].x + __uint_as_float(o[4])) * inv, (acc[2].y + __uint_as_float(o[5])) * inv);
+        pkt.w = pack_bf16((acc[3].x + __uint_as_float(o[6])) * inv, (acc[3].y + __uint_as_float(o[7])) * inv);
+        *reinterpret_cast<uint4*>(args.out + ((size_t)bh * args.Tlen + tok) * D + v0) = pkt;
+      }
+    }
+  } else {
+    // =========================== key scales, query tile, weights, snapshot ===========================
+    const uint32_t q4 = warp & 3;
+    const int t = q4 * 32 + lane;       // token of the tile, and TMEM lane
+    auto load_v = [&](int j) -> uint4 {
+      const int tok = j * CT + t;
+      if (j < nch && tok < args.Tlen)
+        return *reinterpret_cast<const uint4*>(args.v + ((size_t)bh * args.Tlen + tok) * D + v0);
+      return make_uint4(0u, 0u, 0u, 0u);
+    };
+    // key scales and v' of tile j (the value slice was fetched one tile earlier)
+    auto prep = [&](int j, const uint4& vraw) -> bool {
+      const int s = j & 1;
+      if (!wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag)) return false;
+      float ss = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(ktile(s) + sw128_offset(t, c));
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          ss = fmaf(bf_lo(w[e]), bf_lo(w[e]), ss);
+          ss = fmaf(bf_hi(w[e]), bf_hi(w[e]), ss);
+        }
+      }
+      const float r2 = inv_or_zero(ss);
+      uint4 vp;
+      vp.x = pack_bf16(bf_lo(vraw.x) * r2, bf_hi(vraw.x) * r2);
+      vp.y = pack_bf16(bf_lo(vraw.y) * r2, bf_hi(vraw.y) * r2);
+      vp.z = pack_bf16(bf_lo(vraw.z) * r2, bf_hi(vraw.z) * r2);
+      vp.w = pack_bf16(bf_lo(vraw.w) * r2, bf_hi(vraw.w) * r2);
+      *reinterpret_cast<uint4*>(vptile(s) + t * 16) = vp;
+      const uint32_t rb = pack_bf16(r2, r2);
+      *reinterpret_cast<uint4*>(vptile(s) + 2048 + t * 16) = make_uint4(rb & 0xFFFFu, 0u, 0u, 0u);
+      r2pair(s)[t] = rb;
+      fence_async_smem();
+      mbar_arrive(bar(BAR_PREP + s));
+      return true;
+    };
+    uint4 vnext = load_v(0);
+    ok = prep(0, vnext);
+    vnext = load_v(1);
+    for (int j = 0; j < nch && ok; ++j) {
+      const int s = j & 1;
+      // ---- query tile to TMEM (the previous tile's reads and scores are complete: see the end of the loop) ----
+      {
+        uint32_t qw[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint4 raw = *reinterpret_cast<const uint4*>(qtile(s) + sw128_offset(t, c));
+          qw[4 * c] = raw.x; qw[4 * c + 1] = raw.y; qw[4 * c + 2] = raw.z; qw[4 * c + 3] = raw.w;
+        }
+        tmem_st32(tmem_addr(tb, q4 * 32, COL_Q), qw);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_QT_FULL));
+      }
+      // ---- scales of the next tile, so that its W rows can be built during this tile's update ----
+      if (j + 1 < nch) {
+        ok = prep(j + 1, vnext);
+        if (!ok) break;
+        vnext = load_v(j + 2);
+      }
+      // ---- weights P = (q.k)^2, causal, two halves of 64 keys ----
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        ok = wait_or_abort(bar(BAR_S_FULL), h, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t scol = tmem_addr(tb, q4 * 32, COL_P);
+        uint32_t ya[32], yb2[32], pk[32];
+        tmem_ld32(scol, ya);
+        tmem_ld32(scol + 32, yb2);
+        auto weigh = [&](const uint32_t (&y)[32], int half) {
+#pragma unroll
+          for (int jj = 0; jj < 32; jj += 2) {
+            const int c = h * 64 + half * 32 + jj;
+            const float2 sv = make_float2(__uint_as_float(y[jj]), __uint_as_float(y[jj + 1]));
+            float2 w = __fmul2_rn(sv, sv);
+            if (c > t) w.x = 0.f;
+            if (c + 1 > t) w.y = 0.f;
+            pk[(half * 32 + jj) / 2] = pack_bf16(w.x, w.y);
+          }
+        };
+        tmem_wait_ld(ya);
+        weigh(ya, 0);
+        tmem_wait_ld(yb2);
+        weigh(yb2, 1);
+        tmem_st32(scol, pk);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_P_FULL));
+      }
+      if (!ok) break;
+      // ---- snapshot of the state after this tile's update ----
+      ok = wait_or_abort(bar(BAR_U_DONE), j & 1, abort_flag) && wait_or_abort(bar(BAR_R_DONE), j & 1, abort_flag);
+      if (!ok) break;
+      if (j + 1 < nch) {
+        tc_fence_after();
+        const int bloc = t >> 3, vv = t & 7;          // row of a state tile = 8 * (b within the block) + v
+        unsigned char* sp = base + OFF_SP;
+#pragma unroll
+        for (int be = 0; be < 4; ++be) {
+          const int p = 2 * be + (bloc >> 3);
+          unsigned char* row = sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
+          const uint32_t c0 = sp_koff(p) >> 4;
+#pragma unroll
+          for (int al = 0; al <= be; ++al) {
+            uint32_t z[16];
+            tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 8 * be * (be + 1) + 16 * al), z);
+            tmem_wait_ld(z);
+            const float sc = al < be ? 2.f : 1.f;
+#pragma unroll
+            for (int h8 = 0; h8 < 2; ++h8) {
+              uint4 w;
+              w.x = pack_bf16(__uint_as_float(z[8 * h8]) * sc, __uint_as_float(z[8 * h8 + 1]) * sc);
+              w.y = pack_bf16(__uint_as_float(z[8 * h8 + 2]) * sc, __uint_as_float(z[8 * h8 + 3]) * sc);
+              w.z = pack_bf16(__uint_as_float(z[8 * h8 + 4]) * sc, __uint_as_float(z[8 * h8 + 5]) * sc);
+              w.w = pack_bf16(__uint_as_float(z[8 * h8 + 6]) * sc, __uint_as_float(z[8 * h8 + 7]) * sc);
+              *reinterpret_cast<uint4*>(row + (((c0 + 2 * al + h8) ^ (uint32_t)vv) << 4)) = w;
+            }
+          }
+        }
+        if (q4 < 2) {
+          // Z rows: lane = b; row 64 + (b % 8) of piece b / 8, features a < 16 (b / 16 + 1)
+          const int b = t, be = b >> 4, p = b >> 3;
+          unsigned char* row = sp + sp_block(p) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
+          const uint32_t c0 = sp_koff(p) >> 4;
+#pragma unroll
+          for (int al = 0; al < 4; ++al) {
+            uint32_t z[16];
+            tmem_ld16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
+            tmem_wait_ld(z);
+            if (al <= be) {
+              const float sc = al < be ? 2.f : 1.f;
+#pragma unroll
+              for (int h8 = 0; h8 < 2; ++h8) {
+                uint4 w;
+                w.x = pack_bf16(__uint_as_float(z[8 * h8]) * sc, __uint_as_float(z[8 * h8 + 1]) * sc);
+                w.y = pack_bf16(__uint_as_float(z[8 * h8 + 2]) * sc, __uint_as_float(z[8 * h8 + 3]) * sc);
+                w.z = pack_bf16(__uint_as_float(z[8 * h8 + 4]) * sc, __uint_as_float(z[8 * h8 + 5]) * sc);
+                w.w = pack_bf16(__uint_as_float(z[8 * h8 + 6]) * sc, __uint_as_float(z[8 * h8 + 7]) * sc);
+                *reinterpret_cast<uint4*>(row + (((c0 + 2 * al + h8) ^ (uint32_t)(b & 7)) << 4)) = w;
+              }
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar(BAR_SNAP_LD));
+        fence_async_smem();
+        mbar_arrive(bar(BAR_SNAP_ST));
+      }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  if (!ok && args.device_status != nullptr) atomicExch(args.device_status, (int)KATA_ERR_DEVICE_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp >= WARP_U && warp <= WARP_I && lane == 0) {
+    mma_commit(bar(BAR_DRAIN));
+    mbar_wait(bar(BAR_DRAIN), 0);
+  }
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tb, TMEM_COLS);
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// [BH][T][64] bf16 tensor, box = 64 features x 128 tokens x 1 head, 128B swizzle; rows beyond T read as zero.
+bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)BH};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
+  cuuint32_t box[3] = {(cuuint32_t)D, (cuuint32_t)CT, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
+  const int BH = p.B * p.H;
+  CUtensorMap tmQ, tmK;
+  if (!make_map(&tmQ, p.q, BH, p.T) || !make_map(&tmK, p.k, BH, p.T)) {
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  if (cudaFuncSetAttribute(tc_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
+    cudaGetLastError();
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T};
+  tc_stream_kernel<<<dim3(NSLICE, BH, 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, a);
+  note_launch(ctx);
+}
+
+}  // namespace kata
