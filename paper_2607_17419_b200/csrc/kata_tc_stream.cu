@@ -89,7 +89,7 @@ struct SArgs {
   int Tlen;
 };
 
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __noinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023u) == 1023u && *abort_flag) return false;
@@ -233,7 +233,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       for (int j = 0; j < nch && ok; ++j) {
         ok = wait_or_abort(bar(BAR_QT_FULL), j & 1, abort_flag);
         if (ok && j > 0) ok = wait_or_abort(bar(BAR_SNAP_ST), (j - 1) & 1, abort_flag);
-#pragma unroll
+#pragma unroll 1
         for (int p = 0; p < 8; ++p) {
           if (!ok) break;
           const int g = 8 * j + p, yb = g & 1;
@@ -241,7 +241,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (!ok) break;
           tc_fence_after();
           const uint32_t sbase = spa + sp_block(p) * SP_BLOCK + sp_koff(p);
-#pragma unroll
+#pragma unroll 1
           for (int al = 0; al <= (p >> 1); ++al)
             mma_f16_ts(tb + COL_Y + yb * 80, tb + COL_Q + al * 8, at(dS, sbase + al * 32), idR, al > 0);
           mma_commit(bar(BAR_Y_FULL + yb));
@@ -339,19 +339,14 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const int s = j & 1;
       ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag);
       if (!ok) break;
-      uint32_t qw[32];
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(qtile(s) + sw128_offset(t, c));
-        qw[4 * c] = raw.x; qw[4 * c + 1] = raw.y; qw[4 * c + 2] = raw.z; qw[4 * c + 3] = raw.w;
-      }
-      mbar_arrive(bar(BAR_KQ_EMPTY + s));
       float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       float accz = 0.f;
-#pragma unroll
+#pragma unroll 1
       for (int p = 0; p < 8; ++p) {
-        if (!ok) break;
         const int g = 8 * j + p, yb = g & 1;
+        // q[t, 8p .. 8p+7]: the multipliers of this piece
+        const uint4 qraw = *reinterpret_cast<const uint4*>(qtile(s) + sw128_offset(t, p));
+        const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
         ok = wait_or_abort(bar(BAR_Y_FULL + yb), (g >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -364,7 +359,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         auto fold = [&](const uint32_t (&y)[32], int i0) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const int b = 8 * p + i0 + i;
+            const int b = i0 + i;
             const float qb = (b & 1) ? bf_hi(qw[b >> 1]) : bf_lo(qw[b >> 1]);
             const float2 qq = make_float2(qb, qb);
 #pragma unroll
@@ -381,12 +376,12 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         mbar_arrive(bar(BAR_Y_EMPTY + yb));
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const int b = 8 * p + i;
-          const float qb = (b & 1) ? bf_hi(qw[b >> 1]) : bf_lo(qw[b >> 1]);
+          const float qb = (i & 1) ? bf_hi(qw[i >> 1]) : bf_lo(qw[i >> 1]);
           accz = fmaf(qb, __uint_as_float(yz[i]), accz);
         }
       }
       if (!ok) break;
+      mbar_arrive(bar(BAR_KQ_EMPTY + s));
       ok = wait_or_abort(bar(BAR_O_FULL), j & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
@@ -447,12 +442,10 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       return true;
     };
     uint4 vnext = load_v(0);
-    ok = prep(0, vnext);
-    vnext = load_v(1);
-    for (int j = 0; j < nch && ok; ++j) {
+    for (int j = -1; j < nch && ok; ++j) {
       const int s = j & 1;
       // ---- query tile to TMEM (the previous tile's reads and scores are complete: see the end of the loop) ----
-      {
+      if (j >= 0) {
         uint32_t qw[32];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -470,8 +463,9 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (!ok) break;
         vnext = load_v(j + 2);
       }
+      if (j < 0) continue;
       // ---- weights P = (q.k)^2, causal, two halves of 64 keys ----
-#pragma unroll
+#pragma unroll 1
       for (int h = 0; h < 2; ++h) {
         ok = wait_or_abort(bar(BAR_S_FULL), h, abort_flag);
         if (!ok) break;
@@ -508,15 +502,16 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tc_fence_after();
         const int bloc = t >> 3, vv = t & 7;          // row of a state tile = 8 * (b within the block) + v
         unsigned char* sp = base + OFF_SP;
-#pragma unroll
+        uint32_t scol = tmem_addr(tb, q4 * 32, COL_S);
+#pragma unroll 1
         for (int be = 0; be < 4; ++be) {
           const int p = 2 * be + (bloc >> 3);
           unsigned char* row = sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
           const uint32_t c0 = sp_koff(p) >> 4;
-#pragma unroll
-          for (int al = 0; al <= be; ++al) {
+#pragma unroll 1
+          for (int al = 0; al <= be; ++al, scol += 16) {
             uint32_t z[16];
-            tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 8 * be * (be + 1) + 16 * al), z);
+            tmem_ld16(scol, z);
             tmem_wait_ld(z);
             const float sc = al < be ? 2.f : 1.f;
 #pragma unroll
@@ -535,7 +530,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           const int b = t, be = b >> 4, p = b >> 3;
           unsigned char* row = sp + sp_block(p) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
           const uint32_t c0 = sp_koff(p) >> 4;
-#pragma unroll
+#pragma unroll 1
           for (int al = 0; al < 4; ++al) {
             uint32_t z[16];
             tmem_ld16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
