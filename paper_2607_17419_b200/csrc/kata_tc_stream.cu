@@ -18,9 +18,12 @@
 //   out      (N_inter + O) / (D_inter + D)             (0 where the denominator is 0)
 // The query norm cancels and is never applied.
 //
-// Warps (512 threads): 0 TMA producer; 1 update-MMA issuer; 2 read-MMA issuer; 3 intra-tile MMA issuer;
-// 4-7 W builders (warp = b-block, lane = token of a 32-token sub-tile); 8-11 readers and epilogue (thread =
-// token); 12-15 key scales, query tile to TMEM, weights P, state snapshot.  All waits are bounded.
+// Warps (512 threads): 0 TMA producer and update-MMA issuer (b-block 3, Z); 1 update-MMA issuer (b-blocks 0-2);
+// 2 read-MMA issuer; 3 intra-tile MMA issuer; 4-7 W builders (warp = b-block, lanes = 16 tokens x 2 halves of
+// the block) and a share of the snapshot; 8-11 readers and epilogue (thread = token); 12-15 key scales, query
+// tile to TMEM, weights P, the rest of the snapshot.  The snapshot is double-buffered, so the reads of tile
+// j + 1 overlap the update of tile j + 1; only the copy out of TMEM sits between two updates.  All waits are
+// bounded.
 #include <cuda.h>
 
 #include "kata_common.cuh"
@@ -36,7 +39,7 @@ constexpr int CT = 128;          // tokens per tile
 constexpr int VS = 8;            // value columns per CTA
 constexpr int NSLICE = D / VS;
 constexpr int NTHREADS = 512;
-constexpr int WARP_U = 1, WARP_R = 2, WARP_I = 3, WARP_BLD0 = 4, WARP_RD0 = 8, WARP_AUX0 = 12;
+constexpr int WARP_UB = 0, WARP_U = 1, WARP_R = 2, WARP_I = 3, WARP_BLD0 = 4, WARP_RD0 = 8, WARP_AUX0 = 12;
 
 // ---- TMEM columns ----
 constexpr uint32_t COL_S = 0;     // b-block beta at 8 beta (beta + 1): 16 (beta + 1) columns (a < 16 (beta + 1))
@@ -50,12 +53,13 @@ constexpr uint32_t TMEM_COLS = 512;
 // ---- shared memory ----
 constexpr uint32_t OFF_KQ = 0;            // 2 stages x (Q tile 16 KB | K tile 16 KB), 128B swizzle
 constexpr uint32_t OFF_VP = 65536;        // 2 stages x 4 KB: [128 keys][8 bf16] v', then [128 keys][8 bf16] (1/||k||^2, 0..)
-constexpr uint32_t OFF_W = 73728;         // 2 x 40 KB: [5 tiles][2 M-atoms][4 groups of 8 tokens][1 KB], MN-major 128B swizzle
-constexpr uint32_t W_BYTES = 40960;
-constexpr uint32_t OFF_SP = 155648;       // 5 blocks x 80 rows x 128 B: the snapshot, K-major 128B swizzle
+constexpr uint32_t OFF_W = 73728;         // 2 x 20 KB: [5 tiles][2 M-atoms][2 groups of 8 tokens][1 KB], MN-major 128B swizzle
+constexpr uint32_t W_BYTES = 20480;
+constexpr uint32_t OFF_SP = 114688;       // 2 x (5 blocks x 80 rows x 128 B): the snapshots, K-major 128B swizzle
 constexpr uint32_t SP_BLOCK = 10240;
-constexpr uint32_t OFF_R2 = 206848;       // 2 stages x 128 x (bf16 1/||k||^2 twice)
-constexpr uint32_t OFF_BAR = 207872;
+constexpr uint32_t SP_BYTES = 5 * SP_BLOCK;
+constexpr uint32_t OFF_R2 = 217088;       // 2 stages x 128 x (bf16 1/||k||^2 twice)
+constexpr uint32_t OFF_BAR = 218112;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
 
@@ -113,6 +117,20 @@ __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 
 
 __device__ __forceinline__ uint64_t at(uint64_t desc, uint32_t saddr) { return desc + (uint64_t)((saddr >> 4) & 0x3FFF); }
 
+// Rounds 16 fp32 accumulator columns (scaled by sc) to bf16 and stores them as the 16-byte chunks c and c + 1 of a
+// 128-byte snapshot row (128B swizzle: chunk index xor row-in-atom rx).
+__device__ __forceinline__ void snap_store16(unsigned char* row, uint32_t c, uint32_t rx, const uint32_t* z, float sc) {
+#pragma unroll
+  for (int h8 = 0; h8 < 2; ++h8) {
+    uint4 w;
+    w.x = pack_bf16(__uint_as_float(z[8 * h8]) * sc, __uint_as_float(z[8 * h8 + 1]) * sc);
+    w.y = pack_bf16(__uint_as_float(z[8 * h8 + 2]) * sc, __uint_as_float(z[8 * h8 + 3]) * sc);
+    w.z = pack_bf16(__uint_as_float(z[8 * h8 + 4]) * sc, __uint_as_float(z[8 * h8 + 5]) * sc);
+    w.w = pack_bf16(__uint_as_float(z[8 * h8 + 6]) * sc, __uint_as_float(z[8 * h8 + 7]) * sc);
+    *reinterpret_cast<uint4*>(row + (((c + h8) ^ rx) << 4)) = w;
+  }
+}
+
 // Snapshot placement of read piece p (8 values of b, b-block p / 2): block and byte offset inside the 128-byte rows.
 // Pieces of the b-blocks 0 and 2 share rows (32 + 96 bytes), the two pieces of b-block 1 share rows (64 + 64).
 __device__ __forceinline__ uint32_t sp_block(int p) { return (0x43102210u >> (4 * p)) & 0xFu; }   // 0,1,2,2,0,1,3,4
@@ -141,30 +159,30 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     abort_s = 0;
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(BAR_KQ_FULL + s), 1);
-      mbar_init(bar(BAR_KQ_EMPTY + s), 2 + 128);
+      mbar_init(bar(BAR_KQ_EMPTY + s), 3 + 128);
       mbar_init(bar(BAR_PREP + s), 128);
       mbar_init(bar(BAR_W_FULL + s), 128);
-      mbar_init(bar(BAR_W_EMPTY + s), 1);
+      mbar_init(bar(BAR_W_EMPTY + s), 2);
       mbar_init(bar(BAR_Y_FULL + s), 1);
       mbar_init(bar(BAR_Y_EMPTY + s), 128);
     }
     mbar_init(bar(BAR_QT_FULL), 128);
-    mbar_init(bar(BAR_U_DONE), 1);
+    mbar_init(bar(BAR_U_DONE), 2);
     mbar_init(bar(BAR_R_DONE), 1);
-    mbar_init(bar(BAR_SNAP_LD), 128);
-    mbar_init(bar(BAR_SNAP_ST), 128);
+    mbar_init(bar(BAR_SNAP_LD), 256);
+    mbar_init(bar(BAR_SNAP_ST), 256);
     mbar_init(bar(BAR_S_FULL), 1);
     mbar_init(bar(BAR_P_FULL), 128);
     mbar_init(bar(BAR_PV0), 1);
     mbar_init(bar(BAR_O_FULL), 1);
     mbar_init(bar(BAR_O_EMPTY), 128);
-    mbar_init(bar(BAR_DRAIN), 3);
+    mbar_init(bar(BAR_DRAIN), 4);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
   }
   // zero: the W buffers (the second M-atom of the Z tile is never written) and the snapshot (state 0, pad rows)
-  for (uint32_t i = tid; i < (2 * W_BYTES + 5 * SP_BLOCK) / 16; i += NTHREADS)
+  for (uint32_t i = tid; i < (2 * W_BYTES + 2 * SP_BYTES) / 16; i += NTHREADS)
     *reinterpret_cast<uint4*>(base + OFF_W + i * 16) = make_uint4(0u, 0u, 0u, 0u);
   static_assert(OFF_W + 2 * W_BYTES == OFF_SP, "the zero fill runs over both regions");
   fence_async_smem();
@@ -178,45 +196,51 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const uint32_t tb = tmem_base_s;
   bool ok = true;
 
-  if (warp == 0) {
-    // =========================== TMA producer ===========================
+  if (warp == WARP_UB || warp == WARP_U) {
+    // =========================== update issuers: S += W^T K ===========================
+    // Two threads share the MMAs of one 16-token step (their accumulators are disjoint): warp 1 the b-blocks
+    // 0..2, warp 0 b-block 3 and Z.  Warp 0 is also the TMA producer of the query and key tiles.
     if (lane == 0) {
-      for (int j = 0; j < nch && ok; ++j) {
+      // A: MN-major, 128B swizzle: 64 rows x 8 tokens per 1 KB atom; next 8 tokens +1 KB (SBO), next 64 rows +2 KB (LBO)
+      const uint64_t dA = smem_desc(0, 2048, 1024, kSwizzle128B);
+      // B: the key tile read MN-major (N = feature a, K = token): one atom of 64 features x 8 tokens per 1 KB
+      const uint64_t dB = smem_desc(0, 16384, 1024, kSwizzle128B);
+      const bool producer = (warp == WARP_UB);
+      auto load_tiles = [&](int j) -> bool {
         const int s = j & 1;
-        ok = wait_or_abort(bar(BAR_KQ_EMPTY + s), ((j >> 1) & 1) ^ 1, abort_flag);
-        if (!ok) break;
+        if (!wait_or_abort(bar(BAR_KQ_EMPTY + s), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
         mbar_arrive_expect_tx(bar(BAR_KQ_FULL + s), 32768);
         tma_load_3d(qtile(s), &tmQ, bar(BAR_KQ_FULL + s), 0, j * CT, bh);
         tma_load_3d(ktile(s), &tmK, bar(BAR_KQ_FULL + s), 0, j * CT, bh);
+        return true;
+      };
+      if (producer) {
+        ok = load_tiles(0);
+        if (ok && nch > 1) ok = load_tiles(1);
       }
-    }
-  } else if (warp == WARP_U) {
-    // =========================== update issuer: S += W^T K ===========================
-    if (lane == 0) {
-      const uint32_t idU[5] = {instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 16), instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 32),
-                               instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 48), instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64),
-                               instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64)};
-      const uint32_t colU[5] = {COL_S + 0, COL_S + 16, COL_S + 48, COL_S + 96, COL_Z};
-      // A: MN-major, 128B swizzle: 64 rows x 8 tokens per 1 KB atom; next 8 tokens +1 KB (SBO), next 64 rows +4 KB (LBO)
-      const uint64_t dA = smem_desc(0, 4096, 1024, kSwizzle128B);
-      // B: the key tile read MN-major (N = feature a, K = token): one atom of 64 features x 8 tokens per 1 KB
-      const uint64_t dB = smem_desc(0, 16384, 1024, kSwizzle128B);
       for (int j = 0; j < nch && ok; ++j) {
         const int s = j & 1;
         ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag);
         if (ok && j > 0) ok = wait_or_abort(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
-        for (int sc = 0; sc < 4 && ok; ++sc) {
-          const int g = 4 * j + sc, wb = g & 1;
+        // the stage of tile j - 1 is free once that tile's consumers are through: refill it with tile j + 1
+        if (ok && producer && j > 0 && j + 1 < nch) ok = load_tiles(j + 1);
+#pragma unroll 1
+        for (int sc = 0; sc < 8 && ok; ++sc) {
+          const int g = 8 * j + sc, wb = g & 1;
           ok = wait_or_abort(bar(BAR_W_FULL + wb), (g >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t wa = smem_u32(wbuf(wb)), ka = smem_u32(ktile(s)) + sc * 4096;
-#pragma unroll
-          for (int ks = 0; ks < 2; ++ks)
-#pragma unroll
-            for (int tl = 0; tl < 5; ++tl)
-              mma_f16_ss(tb + colU[tl], at(dA, wa + tl * 8192 + ks * 2048), at(dB, ka + ks * 2048), idU[tl],
-                         (g > 0 || ks > 0) ? 1u : 0u);
+          const uint32_t wa = smem_u32(wbuf(wb)), ka = smem_u32(ktile(s)) + sc * 2048;
+          const uint64_t db = at(dB, ka);
+          const uint32_t acc = g > 0 ? 1u : 0u;
+          if (producer) {
+            mma_f16_ss(tb + COL_S + 96, at(dA, wa + 3 * 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64), acc);
+            mma_f16_ss(tb + COL_Z, at(dA, wa + 4 * 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64), acc);
+          } else {
+            mma_f16_ss(tb + COL_S + 0, at(dA, wa), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 16), acc);
+            mma_f16_ss(tb + COL_S + 16, at(dA, wa + 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 32), acc);
+            mma_f16_ss(tb + COL_S + 48, at(dA, wa + 2 * 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 48), acc);
+          }
           mma_commit(bar(BAR_W_EMPTY + wb));
         }
         if (!ok) break;
@@ -240,7 +264,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           ok = wait_or_abort(bar(BAR_Y_EMPTY + yb), ((g >> 1) & 1) ^ 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t sbase = spa + sp_block(p) * SP_BLOCK + sp_koff(p);
+          const uint32_t sbase = spa + (j & 1) * SP_BYTES + sp_block(p) * SP_BLOCK + sp_koff(p);
 #pragma unroll 1
           for (int al = 0; al <= (p >> 1); ++al)
             mma_f16_ts(tb + COL_Y + yb * 80, tb + COL_Q + al * 8, at(dS, sbase + al * 32), idR, al > 0);
@@ -291,44 +315,94 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     }
   } else if (warp < WARP_RD0) {
-    // =========================== W builders ===========================
+    // =========================== W builders (+ a share of the snapshot) ===========================
     const int beta = warp - WARP_BLD0;
+    const uint32_t q4 = warp & 3;
+    const int tk = lane & 15, half = lane >> 4;          // token of the 16-token step, half of the b-block
     for (int j = 0; j < nch && ok; ++j) {
       const int s = j & 1;
       ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag) &&
            wait_or_abort(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
-      for (int sc = 0; sc < 4 && ok; ++sc) {
-        const int g = 4 * j + sc, wb = g & 1;
-        const int t = sc * 32 + lane;
-        const uint4 k0 = *reinterpret_cast<const uint4*>(ktile(s) + sw128_offset(t, 2 * beta));
-        const uint4 k1 = *reinterpret_cast<const uint4*>(ktile(s) + sw128_offset(t, 2 * beta + 1));
+#pragma unroll 1
+      for (int sc = 0; sc < 8 && ok; ++sc) {
+        const int g = 8 * j + sc, wb = g & 1;
+        const int t = sc * 16 + tk;
+        const uint4 kraw = *reinterpret_cast<const uint4*>(ktile(s) + sw128_offset(t, 2 * beta + half));
         const uint4 vp = *reinterpret_cast<const uint4*>(vptile(s) + t * 16);
         const uint32_t rr = r2pair(s)[t];
-        const uint32_t kw[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
+        const uint32_t kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
         ok = wait_or_abort(bar(BAR_W_EMPTY + wb), ((g >> 1) & 1) ^ 1, abort_flag);
         if (!ok) break;
-        unsigned char* wrow = wbuf(wb) + (lane >> 3) * 1024 + (lane & 7) * 128;
+        unsigned char* wrow = wbuf(wb) + (tk >> 3) * 1024 + (tk & 7) * 128;
 #pragma unroll
-        for (int bl = 0; bl < 16; ++bl) {
-          const uint32_t kbb = __byte_perm(kw[bl >> 1], 0u, (bl & 1) ? 0x3232 : 0x1010);
+        for (int i = 0; i < 8; ++i) {
+          const uint32_t kbb = __byte_perm(kw[i >> 1], 0u, (i & 1) ? 0x3232 : 0x1010);
           uint4 w;
           w.x = mul_bf16x2(kbb, vp.x);
           w.y = mul_bf16x2(kbb, vp.y);
           w.z = mul_bf16x2(kbb, vp.z);
           w.w = mul_bf16x2(kbb, vp.w);
-          *reinterpret_cast<uint4*>(wrow + beta * 8192 + (bl >> 3) * 4096 + (((bl & 7) ^ (lane & 7)) << 4)) = w;
+          *reinterpret_cast<uint4*>(wrow + beta * 4096 + half * 2048 + ((i ^ (tk & 7)) << 4)) = w;
         }
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        {
           uint4 w;
-          w.x = mul_bf16x2(kw[4 * h], rr);
-          w.y = mul_bf16x2(kw[4 * h + 1], rr);
-          w.z = mul_bf16x2(kw[4 * h + 2], rr);
-          w.w = mul_bf16x2(kw[4 * h + 3], rr);
-          *reinterpret_cast<uint4*>(wrow + 4 * 8192 + (((2 * beta + h) ^ (lane & 7)) << 4)) = w;
+          w.x = mul_bf16x2(kw[0], rr);
+          w.y = mul_bf16x2(kw[1], rr);
+          w.z = mul_bf16x2(kw[2], rr);
+          w.w = mul_bf16x2(kw[3], rr);
+          *reinterpret_cast<uint4*>(wrow + 4 * 4096 + (((2 * beta + half) ^ (tk & 7)) << 4)) = w;
         }
         fence_async_smem();
         mbar_arrive(bar(BAR_W_FULL + wb));
+        if (sc == 1 && j > 0) {
+          // ---- snapshot of the state after tile j - 1: b-block 2 and the Z rows (the other blocks: warps 12-15) ----
+          // The first two steps of this tile are built; the update that consumes them waits for this copy.
+          const int jp = j - 1;
+          // The buffer written here was read by the reads of tile jp - 1.  They are complete: warps 12-15 wait
+          // for them before they scale tile jp + 1, and this warp has waited for those scales (BAR_PREP).
+          ok = wait_or_abort(bar(BAR_U_DONE), jp & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const int row_t = q4 * 32 + lane, bloc = row_t >> 3, vv = row_t & 7;
+          unsigned char* sp = base + OFF_SP + ((jp + 1) & 1) * SP_BYTES;
+          uint32_t e[32], f[16];
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 48), e);
+          tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 80), f);
+          const int p2 = 4 + (bloc >> 3);
+          unsigned char* row2 = sp + sp_block(p2) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
+          const uint32_t c2 = sp_koff(p2) >> 4;
+          tmem_wait_ld(e);
+          tmem_wait_ld(f);
+          if (q4 < 2) {
+            // Z rows: lane = b; row 64 + (b % 8) of piece b / 8, features a < 16 (b / 16 + 1)
+            uint32_t z0[32], z1[32];
+            tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z), z0);
+            tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z + 32), z1);
+            snap_store16(row2, c2, vv, e, 2.f);
+            snap_store16(row2, c2 + 2, vv, e + 16, 2.f);
+            snap_store16(row2, c2 + 4, vv, f, 1.f);
+            tmem_wait_ld(z0);
+            tmem_wait_ld(z1);
+            tc_fence_before();
+            mbar_arrive(bar(BAR_SNAP_LD));
+            const int b = row_t, bz = b >> 4, pz = b >> 3;
+            unsigned char* rowz = sp + sp_block(pz) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
+            const uint32_t cz = sp_koff(pz) >> 4;
+            const uint32_t rz = (uint32_t)(b & 7);
+            if (0 <= bz) snap_store16(rowz, cz, rz, z0, 0 < bz ? 2.f : 1.f);
+            if (1 <= bz) snap_store16(rowz, cz + 2, rz, z0 + 16, 1 < bz ? 2.f : 1.f);
+            if (2 <= bz) snap_store16(rowz, cz + 4, rz, z1, 2 < bz ? 2.f : 1.f);
+            if (3 <= bz) snap_store16(rowz, cz + 6, rz, z1 + 16, 1.f);
+          } else {
+            tc_fence_before();
+            mbar_arrive(bar(BAR_SNAP_LD));
+            snap_store16(row2, c2, vv, e, 2.f);
+            snap_store16(row2, c2 + 2, vv, e + 16, 2.f);
+            snap_store16(row2, c2 + 4, vv, f, 1.f);
+          }
+          fence_async_smem();
+          mbar_arrive(bar(BAR_SNAP_ST));
+        }
       }
     }
   } else if (warp < WARP_AUX0) {
@@ -443,116 +517,96 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     };
     uint4 vnext = load_v(0);
     for (int j = -1; j < nch && ok; ++j) {
-      const int s = j & 1;
-      // ---- query tile to TMEM (the previous tile's reads and scores are complete: see the end of the loop) ----
-      if (j >= 0) {
-        uint32_t qw[32];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint4 raw = *reinterpret_cast<const uint4*>(qtile(s) + sw128_offset(t, c));
-          qw[4 * c] = raw.x; qw[4 * c + 1] = raw.y; qw[4 * c + 2] = raw.z; qw[4 * c + 3] = raw.w;
-        }
-        tmem_st32(tmem_addr(tb, q4 * 32, COL_Q), qw);
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar(BAR_QT_FULL));
-      }
       // ---- scales of the next tile, so that its W rows can be built during this tile's update ----
       if (j + 1 < nch) {
         ok = prep(j + 1, vnext);
         if (!ok) break;
         vnext = load_v(j + 2);
       }
-      if (j < 0) continue;
       // ---- weights P = (q.k)^2, causal, two halves of 64 keys ----
+      if (j >= 0) {
 #pragma unroll 1
-      for (int h = 0; h < 2; ++h) {
-        ok = wait_or_abort(bar(BAR_S_FULL), h, abort_flag);
+        for (int h = 0; h < 2; ++h) {
+          ok = wait_or_abort(bar(BAR_S_FULL), h, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t scol = tmem_addr(tb, q4 * 32, COL_P);
+          uint32_t ya[32], yb2[32], pk[32];
+          tmem_ld32(scol, ya);
+          tmem_ld32(scol + 32, yb2);
+          auto weigh = [&](const uint32_t (&y)[32], int half) {
+#pragma unroll
+            for (int jj = 0; jj < 32; jj += 2) {
+              const int c = h * 64 + half * 32 + jj;
+              const float2 sv = make_float2(__uint_as_float(y[jj]), __uint_as_float(y[jj + 1]));
+              float2 w = __fmul2_rn(sv, sv);
+              if (c > t) w.x = 0.f;
+              if (c + 1 > t) w.y = 0.f;
+              pk[(half * 32 + jj) / 2] = pack_bf16(w.x, w.y);
+            }
+          };
+          tmem_wait_ld(ya);
+          weigh(ya, 0);
+          tmem_wait_ld(yb2);
+          weigh(yb2, 1);
+          tmem_st32(scol, pk);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar(BAR_P_FULL));
+        }
+        if (!ok) break;
+      }
+      if (j + 1 >= nch) break;
+      // ---- snapshot of the state after tile j: b-blocks 3, 1 and 0 (b-block 2 and Z: warps 4-7) ----
+      if (j >= 0) {
+        ok = wait_or_abort(bar(BAR_U_DONE), j & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t scol = tmem_addr(tb, q4 * 32, COL_P);
-        uint32_t ya[32], yb2[32], pk[32];
-        tmem_ld32(scol, ya);
-        tmem_ld32(scol + 32, yb2);
-        auto weigh = [&](const uint32_t (&y)[32], int half) {
-#pragma unroll
-          for (int jj = 0; jj < 32; jj += 2) {
-            const int c = h * 64 + half * 32 + jj;
-            const float2 sv = make_float2(__uint_as_float(y[jj]), __uint_as_float(y[jj + 1]));
-            float2 w = __fmul2_rn(sv, sv);
-            if (c > t) w.x = 0.f;
-            if (c + 1 > t) w.y = 0.f;
-            pk[(half * 32 + jj) / 2] = pack_bf16(w.x, w.y);
-          }
-        };
-        tmem_wait_ld(ya);
-        weigh(ya, 0);
-        tmem_wait_ld(yb2);
-        weigh(yb2, 1);
-        tmem_st32(scol, pk);
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar(BAR_P_FULL));
-      }
-      if (!ok) break;
-      // ---- snapshot of the state after this tile's update ----
-      ok = wait_or_abort(bar(BAR_U_DONE), j & 1, abort_flag) && wait_or_abort(bar(BAR_R_DONE), j & 1, abort_flag);
-      if (!ok) break;
-      if (j + 1 < nch) {
-        tc_fence_after();
         const int bloc = t >> 3, vv = t & 7;          // row of a state tile = 8 * (b within the block) + v
-        unsigned char* sp = base + OFF_SP;
-        uint32_t scol = tmem_addr(tb, q4 * 32, COL_S);
-#pragma unroll 1
-        for (int be = 0; be < 4; ++be) {
-          const int p = 2 * be + (bloc >> 3);
-          unsigned char* row = sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
-          const uint32_t c0 = sp_koff(p) >> 4;
-#pragma unroll 1
-          for (int al = 0; al <= be; ++al, scol += 16) {
-            uint32_t z[16];
-            tmem_ld16(scol, z);
-            tmem_wait_ld(z);
-            const float sc = al < be ? 2.f : 1.f;
-#pragma unroll
-            for (int h8 = 0; h8 < 2; ++h8) {
-              uint4 w;
-              w.x = pack_bf16(__uint_as_float(z[8 * h8]) * sc, __uint_as_float(z[8 * h8 + 1]) * sc);
-              w.y = pack_bf16(__uint_as_float(z[8 * h8 + 2]) * sc, __uint_as_float(z[8 * h8 + 3]) * sc);
-              w.z = pack_bf16(__uint_as_float(z[8 * h8 + 4]) * sc, __uint_as_float(z[8 * h8 + 5]) * sc);
-              w.w = pack_bf16(__uint_as_float(z[8 * h8 + 6]) * sc, __uint_as_float(z[8 * h8 + 7]) * sc);
-              *reinterpret_cast<uint4*>(row + (((c0 + 2 * al + h8) ^ (uint32_t)vv) << 4)) = w;
-            }
-          }
-        }
-        if (q4 < 2) {
-          // Z rows: lane = b; row 64 + (b % 8) of piece b / 8, features a < 16 (b / 16 + 1)
-          const int b = t, be = b >> 4, p = b >> 3;
-          unsigned char* row = sp + sp_block(p) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
-          const uint32_t c0 = sp_koff(p) >> 4;
-#pragma unroll 1
-          for (int al = 0; al < 4; ++al) {
-            uint32_t z[16];
-            tmem_ld16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
-            tmem_wait_ld(z);
-            if (al <= be) {
-              const float sc = al < be ? 2.f : 1.f;
-#pragma unroll
-              for (int h8 = 0; h8 < 2; ++h8) {
-                uint4 w;
-                w.x = pack_bf16(__uint_as_float(z[8 * h8]) * sc, __uint_as_float(z[8 * h8 + 1]) * sc);
-                w.y = pack_bf16(__uint_as_float(z[8 * h8 + 2]) * sc, __uint_as_float(z[8 * h8 + 3]) * sc);
-                w.z = pack_bf16(__uint_as_float(z[8 * h8 + 4]) * sc, __uint_as_float(z[8 * h8 + 5]) * sc);
-                w.w = pack_bf16(__uint_as_float(z[8 * h8 + 6]) * sc, __uint_as_float(z[8 * h8 + 7]) * sc);
-                *reinterpret_cast<uint4*>(row + (((c0 + 2 * al + h8) ^ (uint32_t)(b & 7)) << 4)) = w;
-              }
-            }
-          }
-        }
+        unsigned char* sp = base + OFF_SP + ((j + 1) & 1) * SP_BYTES;
+        auto rowp = [&](int p) { return sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128; };
+        const int p3 = 6 + (bloc >> 3), p1 = 2 + (bloc >> 3), p0 = bloc >> 3;
+        uint32_t a0[32], a1[32];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 96), a0);
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 128), a1);
+        tmem_wait_ld(a0);
+        tmem_wait_ld(a1);
+        uint32_t c1[32], c0[16];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 16), c1);
+        tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 0), c0);
+        unsigned char* r3 = rowp(p3);
+        snap_store16(r3, 0, vv, a0, 2.f);
+        snap_store16(r3, 2, vv, a0 + 16, 2.f);
+        snap_store16(r3, 4, vv, a1, 2.f);
+        snap_store16(r3, 6, vv, a1 + 16, 1.f);
+        tmem_wait_ld(c1);
+        tmem_wait_ld(c0);
         tc_fence_before();
         mbar_arrive(bar(BAR_SNAP_LD));
+        unsigned char* r1 = rowp(p1);
+        const uint32_t k1 = sp_koff(p1) >> 4;
+        snap_store16(r1, k1, vv, c1, 2.f);
+        snap_store16(r1, k1 + 2, vv, c1 + 16, 1.f);
+        snap_store16(rowp(p0), sp_koff(p0) >> 4, vv, c0, 1.f);
         fence_async_smem();
         mbar_arrive(bar(BAR_SNAP_ST));
+      }
+      // ---- query tile j + 1 to TMEM, once the reads and scores of tile j are complete (the scores: see above) ----
+      {
+        if (j >= 0) ok = wait_or_abort(bar(BAR_R_DONE), j & 1, abort_flag);
+        if (!ok) break;
+        const int s1 = (j + 1) & 1;
+        uint32_t qw[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint4 raw = *reinterpret_cast<const uint4*>(qtile(s1) + sw128_offset(t, c));
+          qw[4 * c] = raw.x; qw[4 * c + 1] = raw.y; qw[4 * c + 2] = raw.z; qw[4 * c + 3] = raw.w;
+        }
+        tc_fence_after();
+        tmem_st32(tmem_addr(tb, q4 * 32, COL_Q), qw);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_QT_FULL));
       }
     }
   }
@@ -562,7 +616,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (warp >= WARP_U && warp <= WARP_I && lane == 0) {
+  if (warp <= WARP_I && lane == 0) {
     mma_commit(bar(BAR_DRAIN));
     mbar_wait(bar(BAR_DRAIN), 0);
   }
