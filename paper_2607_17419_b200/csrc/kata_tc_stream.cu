@@ -18,12 +18,13 @@
 //   out      (N_inter + O) / (D_inter + D)             (0 where the denominator is 0)
 // The query norm cancels and is never applied.
 //
-// Warps (512 threads): 0 TMA producer and update-MMA issuer (b-block 3, Z); 1 update-MMA issuer (b-blocks 0-2);
-// 2 read-MMA issuer; 3 intra-tile MMA issuer; 4-7 W builders (warp = b-block, lanes = 16 tokens x 2 halves of
-// the block) and a share of the snapshot; 8-11 readers and epilogue (thread = token); 12-15 key scales, query
-// tile to TMEM, weights P, the rest of the snapshot.  The snapshot is double-buffered, so the reads of tile
-// j + 1 overlap the update of tile j + 1; only the copy out of TMEM sits between two updates.  All waits are
-// bounded.
+// Warps (768 threads, 80 registers each): 0 TMA producer and update-MMA issuer (b-block 3, Z); 1 update-MMA
+// issuer (b-blocks 0-2); 2 read-MMA issuer; 3 intra-tile MMA issuer; 4-11 W builders in two teams (even / odd
+// 16-token steps; warp = b-block, lanes = 16 tokens x 2 halves of the block), the second team also copies a
+// share of the snapshot; 12-19 readers in two teams (even / odd read pieces, thread = token), the first team
+// writes the output; 20-23 key scales, query tile to TMEM, weights P, the rest of the snapshot.  The snapshot is
+// double-buffered, so the reads of tile j + 1 overlap the update of tile j + 1; only the copy out of TMEM sits
+// between two updates.  All waits are bounded.
 #include <cuda.h>
 
 #include "kata_common.cuh"
@@ -38,8 +39,8 @@ constexpr int D = 64;
 constexpr int CT = 128;          // tokens per tile
 constexpr int VS = 8;            // value columns per CTA
 constexpr int NSLICE = D / VS;
-constexpr int NTHREADS = 512;
-constexpr int WARP_UB = 0, WARP_U = 1, WARP_R = 2, WARP_I = 3, WARP_BLD0 = 4, WARP_RD0 = 8, WARP_AUX0 = 12;
+constexpr int NTHREADS = 768;
+constexpr int WARP_UB = 0, WARP_U = 1, WARP_R = 2, WARP_I = 3, WARP_BLD0 = 4, WARP_RD0 = 12, WARP_AUX0 = 20;
 
 // ---- TMEM columns ----
 constexpr uint32_t COL_S = 0;     // b-block beta at 8 beta (beta + 1): 16 (beta + 1) columns (a < 16 (beta + 1))
@@ -59,7 +60,8 @@ constexpr uint32_t OFF_SP = 114688;       // 2 x (5 blocks x 80 rows x 128 B): t
 constexpr uint32_t SP_BLOCK = 10240;
 constexpr uint32_t SP_BYTES = 5 * SP_BLOCK;
 constexpr uint32_t OFF_R2 = 217088;       // 2 stages x 128 x (bf16 1/||k||^2 twice)
-constexpr uint32_t OFF_BAR = 218112;
+constexpr uint32_t OFF_PART = 218112;     // 9 x 128 fp32: partial sums of the second reader team
+constexpr uint32_t OFF_BAR = 222720;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
 
@@ -82,8 +84,10 @@ enum {
   BAR_PV0 = 21,       // first half applied (its weights may be overwritten)
   BAR_O_FULL = 22,    // intra-tile result complete
   BAR_O_EMPTY = 23,   // intra-tile result read
-  BAR_DRAIN = 24,
-  BAR_COUNT = 25
+  BAR_PART_FULL = 24,   // partial sums of the second reader team written
+  BAR_PART_EMPTY = 25,  // ... and read
+  BAR_DRAIN = 26,
+  BAR_COUNT = 27
 };
 
 struct SArgs {
@@ -159,7 +163,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     abort_s = 0;
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(BAR_KQ_FULL + s), 1);
-      mbar_init(bar(BAR_KQ_EMPTY + s), 3 + 128);
+      mbar_init(bar(BAR_KQ_EMPTY + s), 3 + 256);
       mbar_init(bar(BAR_PREP + s), 128);
       mbar_init(bar(BAR_W_FULL + s), 128);
       mbar_init(bar(BAR_W_EMPTY + s), 2);
@@ -176,6 +180,8 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_init(bar(BAR_PV0), 1);
     mbar_init(bar(BAR_O_FULL), 1);
     mbar_init(bar(BAR_O_EMPTY), 128);
+    mbar_init(bar(BAR_PART_FULL), 128);
+    mbar_init(bar(BAR_PART_EMPTY), 128);
     mbar_init(bar(BAR_DRAIN), 4);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
@@ -316,24 +322,27 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
   } else if (warp < WARP_RD0) {
     // =========================== W builders (+ a share of the snapshot) ===========================
-    const int beta = warp - WARP_BLD0;
+    // Two teams of four warps: team 0 (warps 4-7) builds the even 16-token steps into buffer 0, team 1 the odd
+    // steps into buffer 1.  Warp = b-block, lanes = 16 tokens x 2 halves of the block.
+    const int beta = warp & 3;
+    const int team = (warp - WARP_BLD0) >> 2;
     const uint32_t q4 = warp & 3;
-    const int tk = lane & 15, half = lane >> 4;          // token of the 16-token step, half of the b-block
+    const int tk = lane & 15, half = lane >> 4;
     for (int j = 0; j < nch && ok; ++j) {
       const int s = j & 1;
       ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag) &&
            wait_or_abort(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
 #pragma unroll 1
-      for (int sc = 0; sc < 8 && ok; ++sc) {
-        const int g = 8 * j + sc, wb = g & 1;
+      for (int sc = team; sc < 8 && ok; sc += 2) {
+        const int g = 8 * j + sc;
         const int t = sc * 16 + tk;
         const uint4 kraw = *reinterpret_cast<const uint4*>(ktile(s) + sw128_offset(t, 2 * beta + half));
         const uint4 vp = *reinterpret_cast<const uint4*>(vptile(s) + t * 16);
         const uint32_t rr = r2pair(s)[t];
         const uint32_t kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
-        ok = wait_or_abort(bar(BAR_W_EMPTY + wb), ((g >> 1) & 1) ^ 1, abort_flag);
+        ok = wait_or_abort(bar(BAR_W_EMPTY + team), ((g >> 1) & 1) ^ 1, abort_flag);
         if (!ok) break;
-        unsigned char* wrow = wbuf(wb) + (tk >> 3) * 1024 + (tk & 7) * 128;
+        unsigned char* wrow = wbuf(team) + (tk >> 3) * 1024 + (tk & 7) * 128;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const uint32_t kbb = __byte_perm(kw[i >> 1], 0u, (i & 1) ? 0x3232 : 0x1010);
@@ -353,62 +362,70 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           *reinterpret_cast<uint4*>(wrow + 4 * 4096 + (((2 * beta + half) ^ (tk & 7)) << 4)) = w;
         }
         fence_async_smem();
-        mbar_arrive(bar(BAR_W_FULL + wb));
-        if (sc == 1 && j > 0) {
-          // ---- snapshot of the state after tile j - 1: b-block 2 and the Z rows (the other blocks: warps 12-15) ----
-          // The first two steps of this tile are built; the update that consumes them waits for this copy.
-          const int jp = j - 1;
-          // The buffer written here was read by the reads of tile jp - 1.  They are complete: warps 12-15 wait
-          // for them before they scale tile jp + 1, and this warp has waited for those scales (BAR_PREP).
-          ok = wait_or_abort(bar(BAR_U_DONE), jp & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const int row_t = q4 * 32 + lane, bloc = row_t >> 3, vv = row_t & 7;
-          unsigned char* sp = base + OFF_SP + ((jp + 1) & 1) * SP_BYTES;
-          uint32_t e[32], f[16];
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 48), e);
-          tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 80), f);
-          const int p2 = 4 + (bloc >> 3);
-          unsigned char* row2 = sp + sp_block(p2) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
-          const uint32_t c2 = sp_koff(p2) >> 4;
-          tmem_wait_ld(e);
-          tmem_wait_ld(f);
-          if (q4 < 2) {
-            // Z rows: lane = b; row 64 + (b % 8) of piece b / 8, features a < 16 (b / 16 + 1)
-            uint32_t z0[32], z1[32];
-            tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z), z0);
-            tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z + 32), z1);
-            snap_store16(row2, c2, vv, e, 2.f);
-            snap_store16(row2, c2 + 2, vv, e + 16, 2.f);
-            snap_store16(row2, c2 + 4, vv, f, 1.f);
-            tmem_wait_ld(z0);
-            tmem_wait_ld(z1);
-            tc_fence_before();
-            mbar_arrive(bar(BAR_SNAP_LD));
-            const int b = row_t, bz = b >> 4, pz = b >> 3;
-            unsigned char* rowz = sp + sp_block(pz) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
-            const uint32_t cz = sp_koff(pz) >> 4;
-            const uint32_t rz = (uint32_t)(b & 7);
-            if (0 <= bz) snap_store16(rowz, cz, rz, z0, 0 < bz ? 2.f : 1.f);
-            if (1 <= bz) snap_store16(rowz, cz + 2, rz, z0 + 16, 1 < bz ? 2.f : 1.f);
-            if (2 <= bz) snap_store16(rowz, cz + 4, rz, z1, 2 < bz ? 2.f : 1.f);
-            if (3 <= bz) snap_store16(rowz, cz + 6, rz, z1 + 16, 1.f);
-          } else {
-            tc_fence_before();
-            mbar_arrive(bar(BAR_SNAP_LD));
-            snap_store16(row2, c2, vv, e, 2.f);
-            snap_store16(row2, c2 + 2, vv, e + 16, 2.f);
-            snap_store16(row2, c2 + 4, vv, f, 1.f);
-          }
-          fence_async_smem();
-          mbar_arrive(bar(BAR_SNAP_ST));
+        mbar_arrive(bar(BAR_W_FULL + team));
+      }
+      if (!ok) break;
+      if (team == 1 && j + 1 < nch) {
+        // ---- snapshot of the state after tile j: b-block 2 and the Z rows (the other blocks: warps 20-23) ----
+        // The buffer written here was read by the reads of tile j - 1.  They are complete: warps 20-23 wait for
+        // them before they scale tile j + 1, and this warp waits for those scales first.
+        const int s1 = (j + 1) & 1;
+        ok = wait_or_abort(bar(BAR_KQ_FULL + s1), ((j + 1) >> 1) & 1, abort_flag) &&
+             wait_or_abort(bar(BAR_PREP + s1), ((j + 1) >> 1) & 1, abort_flag) &&
+             wait_or_abort(bar(BAR_U_DONE), j & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const int row_t = q4 * 32 + lane, bloc = row_t >> 3, vv = row_t & 7;
+        unsigned char* sp = base + OFF_SP + ((j + 1) & 1) * SP_BYTES;
+        uint32_t e[32], f[16];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 48), e);
+        tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 80), f);
+        const int p2 = 4 + (bloc >> 3);
+        unsigned char* row2 = sp + sp_block(p2) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
+        const uint32_t c2 = sp_koff(p2) >> 4;
+        tmem_wait_ld(e);
+        tmem_wait_ld(f);
+        if (q4 < 2) {
+          // Z rows: lane = b; row 64 + (b % 8) of piece b / 8, features a < 16 (b / 16 + 1)
+          uint32_t z0[32];
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z), z0);
+          snap_store16(row2, c2, vv, e, 2.f);
+          snap_store16(row2, c2 + 2, vv, e + 16, 2.f);
+          snap_store16(row2, c2 + 4, vv, f, 1.f);
+          uint32_t z1[32];
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z + 32), z1);
+          tmem_wait_ld(z0);
+          tmem_wait_ld(z1);
+          tc_fence_before();
+          mbar_arrive(bar(BAR_SNAP_LD));
+          const int b = row_t, bz = b >> 4, pz = b >> 3;
+          unsigned char* rowz = sp + sp_block(pz) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
+          const uint32_t cz = sp_koff(pz) >> 4;
+          const uint32_t rz = (uint32_t)(b & 7);
+          snap_store16(rowz, cz, rz, z0, 0 < bz ? 2.f : 1.f);
+          if (1 <= bz) snap_store16(rowz, cz + 2, rz, z0 + 16, 1 < bz ? 2.f : 1.f);
+          if (2 <= bz) snap_store16(rowz, cz + 4, rz, z1, 2 < bz ? 2.f : 1.f);
+          if (3 <= bz) snap_store16(rowz, cz + 6, rz, z1 + 16, 1.f);
+        } else {
+          tc_fence_before();
+          mbar_arrive(bar(BAR_SNAP_LD));
+          snap_store16(row2, c2, vv, e, 2.f);
+          snap_store16(row2, c2 + 2, vv, e + 16, 2.f);
+          snap_store16(row2, c2 + 4, vv, f, 1.f);
         }
+        fence_async_smem();
+        mbar_arrive(bar(BAR_SNAP_ST));
       }
     }
   } else if (warp < WARP_AUX0) {
     // =========================== readers and epilogue (thread = token) ===========================
+    // Two teams: team 0 (warps 12-15) folds the even pieces (TMEM buffer 0), team 1 the odd pieces (buffer 1)
+    // and hands its partial sums to team 0 through shared memory; team 0 writes the output.
     const uint32_t q4 = warp & 3;
+    const int team = (warp - WARP_RD0) >> 2;
     const int t = q4 * 32 + lane;
+    float* part = reinterpret_cast<float*>(base + OFF_PART);
+    const uint32_t ycol = tmem_addr(tb, q4 * 32, COL_Y + team * 80);
     for (int j = 0; j < nch && ok; ++j) {
       const int s = j & 1;
       ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag);
@@ -416,23 +433,21 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       float accz = 0.f;
 #pragma unroll 1
-      for (int p = 0; p < 8; ++p) {
-        const int g = 8 * j + p, yb = g & 1;
+      for (int p = team; p < 8; p += 2) {
+        const int g = 8 * j + p;
         // q[t, 8p .. 8p+7]: the multipliers of this piece
         const uint4 qraw = *reinterpret_cast<const uint4*>(qtile(s) + sw128_offset(t, p));
         const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
-        ok = wait_or_abort(bar(BAR_Y_FULL + yb), (g >> 1) & 1, abort_flag);
+        ok = wait_or_abort(bar(BAR_Y_FULL + team), (g >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t ycol = tmem_addr(tb, q4 * 32, COL_Y + yb * 80);
-        uint32_t ya[32], yb2[32], yz[16];
-        tmem_ld32(ycol, ya);
-        tmem_ld32(ycol + 32, yb2);
-        tmem_ld16(ycol + 64, yz);
-        tmem_wait_ld(ya);
-        auto fold = [&](const uint32_t (&y)[32], int i0) {
+        uint32_t y0[16], y1[16], y2[16];
+        tmem_ld16(ycol, y0);
+        tmem_ld16(ycol + 16, y1);
+        tmem_ld16(ycol + 32, y2);
+        auto fold = [&](const uint32_t (&y)[16], int i0) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
+          for (int i = 0; i < 2; ++i) {
             const int b = i0 + i;
             const float qb = (b & 1) ? bf_hi(qw[b >> 1]) : bf_lo(qw[b >> 1]);
             const float2 qq = make_float2(qb, qb);
@@ -442,20 +457,46 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                    acc[vv]);
           }
         };
-        fold(ya, 0);
-        tmem_wait_ld(yb2);
-        fold(yb2, 4);
-        tmem_wait_ld(yz);
+        tmem_wait_ld(y0);
+        fold(y0, 0);
+        tmem_ld16(ycol + 48, y0);
+        tmem_wait_ld(y1);
+        fold(y1, 2);
+        tmem_ld16(ycol + 64, y1);
+        tmem_wait_ld(y2);
+        fold(y2, 4);
+        tmem_wait_ld(y0);
+        fold(y0, 6);
+        tmem_wait_ld(y1);
         tc_fence_before();
-        mbar_arrive(bar(BAR_Y_EMPTY + yb));
+        mbar_arrive(bar(BAR_Y_EMPTY + team));
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const float qb = (i & 1) ? bf_hi(qw[i >> 1]) : bf_lo(qw[i >> 1]);
-          accz = fmaf(qb, __uint_as_float(yz[i]), accz);
+          accz = fmaf(qb, __uint_as_float(y1[i]), accz);
         }
       }
       if (!ok) break;
       mbar_arrive(bar(BAR_KQ_EMPTY + s));
+      if (team == 1) {
+        ok = wait_or_abort(bar(BAR_PART_EMPTY), (j & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        part[0 * CT + t] = acc[0].x; part[1 * CT + t] = acc[0].y;
+        part[2 * CT + t] = acc[1].x; part[3 * CT + t] = acc[1].y;
+        part[4 * CT + t] = acc[2].x; part[5 * CT + t] = acc[2].y;
+        part[6 * CT + t] = acc[3].x; part[7 * CT + t] = acc[3].y;
+        part[8 * CT + t] = accz;
+        mbar_arrive(bar(BAR_PART_FULL));
+        continue;
+      }
+      ok = wait_or_abort(bar(BAR_PART_FULL), j & 1, abort_flag);
+      if (!ok) break;
+      acc[0].x += part[0 * CT + t]; acc[0].y += part[1 * CT + t];
+      acc[1].x += part[2 * CT + t]; acc[1].y += part[3 * CT + t];
+      acc[2].x += part[4 * CT + t]; acc[2].y += part[5 * CT + t];
+      acc[3].x += part[6 * CT + t]; acc[3].y += part[7 * CT + t];
+      accz += part[8 * CT + t];
+      mbar_arrive(bar(BAR_PART_EMPTY));
       ok = wait_or_abort(bar(BAR_O_FULL), j & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
@@ -531,10 +572,12 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (!ok) break;
           tc_fence_after();
           const uint32_t scol = tmem_addr(tb, q4 * 32, COL_P);
-          uint32_t ya[32], yb2[32], pk[32];
-          tmem_ld32(scol, ya);
-          tmem_ld32(scol + 32, yb2);
-          auto weigh = [&](const uint32_t (&y)[32], int half) {
+          // 32 scores at a time; the bf16 weights go back over columns this thread has already read
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t y[32], pk[16];
+            tmem_ld32(scol + half * 32, y);
+            tmem_wait_ld(y);
 #pragma unroll
             for (int jj = 0; jj < 32; jj += 2) {
               const int c = h * 64 + half * 32 + jj;
@@ -542,14 +585,10 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
               float2 w = __fmul2_rn(sv, sv);
               if (c > t) w.x = 0.f;
               if (c + 1 > t) w.y = 0.f;
-              pk[(half * 32 + jj) / 2] = pack_bf16(w.x, w.y);
+              pk[jj / 2] = pack_bf16(w.x, w.y);
             }
-          };
-          tmem_wait_ld(ya);
-          weigh(ya, 0);
-          tmem_wait_ld(yb2);
-          weigh(yb2, 1);
-          tmem_st32(scol, pk);
+            tmem_st16(scol + half * 16, pk);
+          }
           tmem_wait_st();
           tc_fence_before();
           mbar_arrive(bar(BAR_P_FULL));
@@ -569,24 +608,24 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         uint32_t a0[32], a1[32];
         tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 96), a0);
         tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 128), a1);
-        tmem_wait_ld(a0);
-        tmem_wait_ld(a1);
-        uint32_t c1[32], c0[16];
-        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 16), c1);
-        tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 0), c0);
         unsigned char* r3 = rowp(p3);
+        tmem_wait_ld(a0);
         snap_store16(r3, 0, vv, a0, 2.f);
         snap_store16(r3, 2, vv, a0 + 16, 2.f);
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 16), a0);      // b-block 1
+        tmem_wait_ld(a1);
         snap_store16(r3, 4, vv, a1, 2.f);
         snap_store16(r3, 6, vv, a1 + 16, 1.f);
-        tmem_wait_ld(c1);
+        uint32_t c0[16];
+        tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 0), c0);       // b-block 0
+        tmem_wait_ld(a0);
         tmem_wait_ld(c0);
         tc_fence_before();
         mbar_arrive(bar(BAR_SNAP_LD));
         unsigned char* r1 = rowp(p1);
         const uint32_t k1 = sp_koff(p1) >> 4;
-        snap_store16(r1, k1, vv, c1, 2.f);
-        snap_store16(r1, k1 + 2, vv, c1 + 16, 1.f);
+        snap_store16(r1, k1, vv, a0, 2.f);
+        snap_store16(r1, k1 + 2, vv, a0 + 16, 1.f);
         snap_store16(rowp(p0), sp_koff(p0) >> 4, vv, c0, 1.f);
         fence_async_smem();
         mbar_arrive(bar(BAR_SNAP_ST));
