@@ -20,11 +20,11 @@
 //
 // Warps (768 threads, 80 registers each): 0 TMA producer and update-MMA issuer (b-block 3, Z); 1 update-MMA
 // issuer (b-blocks 0-2); 2 read-MMA issuer; 3 intra-tile MMA issuer; 4-11 W builders in two teams (even / odd
-// 16-token steps; warp = b-block, lanes = 16 tokens x 2 halves of the block), the second team also copies a
-// share of the snapshot; 12-19 readers in two teams (even / odd read pieces, thread = token), the first team
-// writes the output; 20-23 key scales, query tile to TMEM, weights P, the rest of the snapshot.  The snapshot is
-// double-buffered, so the reads of tile j + 1 overlap the update of tile j + 1; only the copy out of TMEM sits
-// between two updates.  All waits are bounded.
+// 16-token steps into a ring of three buffers; warp = b-block, lanes = 16 tokens x 2 halves of the block), which
+// also copy shares of the snapshot; 12-19 readers in two teams (even / odd read pieces, thread = token), the
+// first team writes the output; 20-23 key scales, query tile to TMEM, weights P, the last share of the snapshot.
+// The snapshot is double-buffered, so the reads of tile j + 1 overlap the update of tile j + 1; only the copy
+// out of TMEM (twelve warps, at most 64 columns each) sits between two updates.  All waits are bounded.
 #include <cuda.h>
 
 #include "kata_common.cuh"
@@ -52,10 +52,13 @@ constexpr uint32_t COL_Q = 464;   // 32: the query tile as bf16 pairs
 constexpr uint32_t TMEM_COLS = 512;
 
 // ---- shared memory ----
-constexpr uint32_t OFF_KQ = 0;            // 2 stages x (Q tile 16 KB | K tile 16 KB), 128B swizzle
-constexpr uint32_t OFF_VP = 65536;        // 2 stages x 4 KB: [128 keys][8 bf16] v', then [128 keys][8 bf16] (1/||k||^2, 0..)
-constexpr uint32_t OFF_W = 73728;         // 2 x 20 KB: [5 tiles][2 M-atoms][2 groups of 8 tokens][1 KB], MN-major 128B swizzle
-constexpr uint32_t W_BYTES = 20480;
+constexpr uint32_t OFF_K = 0;             // 2 stages x K tile 16 KB, 128B swizzle
+constexpr uint32_t OFF_Q = 32768;         // Q tile 16 KB (staging for the copy to TMEM)
+constexpr uint32_t OFF_VP = 49152;        // 2 stages x 4 KB: [128 keys][8 bf16] v', then [128 keys][8 bf16] (1/||k||^2, 0..)
+constexpr uint32_t OFF_W = 57344;         // 3 x 18 KB: [4 tiles][2 M-atoms][2 groups of 8 tokens][1 KB], then the Z rows
+constexpr uint32_t W_BYTES = 18432;       //   [2 groups of 8 tokens][1 KB]; MN-major 128B swizzle
+constexpr int NWBUF = 3;
+constexpr uint32_t OFF_ZERO = 112640;     // 2 KB of zeros: the missing second M-atom of the Z tile
 constexpr uint32_t OFF_SP = 114688;       // 2 x (5 blocks x 80 rows x 128 B): the snapshots, K-major 128B swizzle
 constexpr uint32_t SP_BLOCK = 10240;
 constexpr uint32_t SP_BYTES = 5 * SP_BLOCK;
@@ -64,30 +67,34 @@ constexpr uint32_t OFF_PART = 218112;     // 9 x 128 fp32: partial sums of the s
 constexpr uint32_t OFF_BAR = 222720;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
+static_assert(OFF_W + NWBUF * W_BYTES == OFF_ZERO && OFF_ZERO + 2048 == OFF_SP, "layout");
 
 // Every barrier has waiters that consume each of its phases in order.
 enum {
-  BAR_KQ_FULL = 0,    // [2] query and key tiles landed
-  BAR_KQ_EMPTY = 2,   // [2] stage free: update and intra commits + the 128 readers' query rows
+  BAR_K_FULL = 0,     // [2] key tile landed
+  BAR_K_EMPTY = 2,    // [2] stage free: the two update issuers' and the intra issuer's commits
   BAR_PREP = 4,       // [2] key scales and v' of the tile written
   BAR_QT_FULL = 6,    // query tile copied to TMEM
-  BAR_W_FULL = 7,     // [2] W sub-tile built
-  BAR_W_EMPTY = 9,    // [2] W sub-tile consumed
-  BAR_U_DONE = 11,    // update of the tile complete
-  BAR_R_DONE = 12,    // all read pieces of the tile complete
-  BAR_SNAP_LD = 13,   // accumulators copied out of TMEM: the next update may run
-  BAR_SNAP_ST = 14,   // snapshot stored: the next read may run
-  BAR_Y_FULL = 15,    // [2]
-  BAR_Y_EMPTY = 17,   // [2]
-  BAR_S_FULL = 19,    // scores of a 64-key half in TMEM
-  BAR_P_FULL = 20,    // weights of the half stored
-  BAR_PV0 = 21,       // first half applied (its weights may be overwritten)
-  BAR_O_FULL = 22,    // intra-tile result complete
-  BAR_O_EMPTY = 23,   // intra-tile result read
-  BAR_PART_FULL = 24,   // partial sums of the second reader team written
-  BAR_PART_EMPTY = 25,  // ... and read
-  BAR_DRAIN = 26,
-  BAR_COUNT = 27
+  BAR_W_FULL = 7,     // [3] W step built
+  BAR_W_EMPTY = 10,   // [3] W step consumed
+  BAR_U_DONE = 13,    // update of the tile complete
+  BAR_R_DONE = 14,    // all read pieces of the tile complete
+  BAR_SNAP_LD = 15,   // accumulators copied out of TMEM: the next update may run
+  BAR_SNAP_ST = 16,   // snapshot stored: the next read may run
+  BAR_Y_FULL = 17,    // [2]
+  BAR_Y_EMPTY = 19,   // [2]
+  BAR_S_FULL = 21,    // scores of a 64-key half in TMEM
+  BAR_P_FULL = 22,    // weights of the half stored
+  BAR_PV0 = 23,       // first half applied (its weights may be overwritten)
+  BAR_O_FULL = 24,    // intra-tile result complete
+  BAR_O_EMPTY = 25,   // intra-tile result read
+  BAR_PART_FULL = 26, // partial sums of the second reader team written
+  BAR_PART_EMPTY = 27,// ... and read
+  BAR_Q_FULL = 28,    // query tile landed in shared memory
+  BAR_QS_EMPTY = 29,  // ... and copied out of it
+  BAR_Q_FREE = 30,    // the readers hold all their multipliers of the tile: the TMEM copy may be replaced
+  BAR_DRAIN = 31,
+  BAR_COUNT = 32
 };
 
 struct SArgs {
@@ -100,6 +107,7 @@ struct SArgs {
 __device__ __noinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(32);
     if ((i & 1023u) == 1023u && *abort_flag) return false;
   }
   *abort_flag = 1;
@@ -145,8 +153,8 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   auto bar = [&](int i) { return reinterpret_cast<uint64_t*>(base + OFF_BAR) + i; };
-  auto qtile = [&](int s) { return base + OFF_KQ + s * 32768; };
-  auto ktile = [&](int s) { return base + OFF_KQ + s * 32768 + 16384; };
+  unsigned char* const qtile = base + OFF_Q;
+  auto ktile = [&](int s) { return base + OFF_K + s * 16384; };
   auto vptile = [&](int s) { return base + OFF_VP + s * 4096; };
   auto wbuf = [&](int b) { return base + OFF_W + b * W_BYTES; };
   auto r2pair = [&](int s) { return reinterpret_cast<uint32_t*>(base + OFF_R2) + s * CT; };
@@ -162,19 +170,21 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (tid == 0) {
     abort_s = 0;
     for (int s = 0; s < 2; ++s) {
-      mbar_init(bar(BAR_KQ_FULL + s), 1);
-      mbar_init(bar(BAR_KQ_EMPTY + s), 3 + 256);
+      mbar_init(bar(BAR_K_FULL + s), 1);
+      mbar_init(bar(BAR_K_EMPTY + s), 3);
       mbar_init(bar(BAR_PREP + s), 128);
-      mbar_init(bar(BAR_W_FULL + s), 128);
-      mbar_init(bar(BAR_W_EMPTY + s), 2);
       mbar_init(bar(BAR_Y_FULL + s), 1);
       mbar_init(bar(BAR_Y_EMPTY + s), 128);
+    }
+    for (int s = 0; s < NWBUF; ++s) {
+      mbar_init(bar(BAR_W_FULL + s), 128);
+      mbar_init(bar(BAR_W_EMPTY + s), 2);
     }
     mbar_init(bar(BAR_QT_FULL), 128);
     mbar_init(bar(BAR_U_DONE), 2);
     mbar_init(bar(BAR_R_DONE), 1);
-    mbar_init(bar(BAR_SNAP_LD), 256);
-    mbar_init(bar(BAR_SNAP_ST), 256);
+    mbar_init(bar(BAR_SNAP_LD), 384);
+    mbar_init(bar(BAR_SNAP_ST), 384);
     mbar_init(bar(BAR_S_FULL), 1);
     mbar_init(bar(BAR_P_FULL), 128);
     mbar_init(bar(BAR_PV0), 1);
@@ -182,15 +192,17 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_init(bar(BAR_O_EMPTY), 128);
     mbar_init(bar(BAR_PART_FULL), 128);
     mbar_init(bar(BAR_PART_EMPTY), 128);
+    mbar_init(bar(BAR_Q_FULL), 1);
+    mbar_init(bar(BAR_QS_EMPTY), 128);
+    mbar_init(bar(BAR_Q_FREE), 256);
     mbar_init(bar(BAR_DRAIN), 4);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
   }
-  // zero: the W buffers (the second M-atom of the Z tile is never written) and the snapshot (state 0, pad rows)
-  for (uint32_t i = tid; i < (2 * W_BYTES + 2 * SP_BYTES) / 16; i += NTHREADS)
-    *reinterpret_cast<uint4*>(base + OFF_W + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-  static_assert(OFF_W + 2 * W_BYTES == OFF_SP, "the zero fill runs over both regions");
+  // zero: the zero atom of the Z tile and the snapshots (state 0, pad rows)
+  for (uint32_t i = tid; i < (2048 + 2 * SP_BYTES) / 16; i += NTHREADS)
+    *reinterpret_cast<uint4*>(base + OFF_ZERO + i * 16) = make_uint4(0u, 0u, 0u, 0u);
   fence_async_smem();
   if (warp == 0) {
     tmem_alloc(&tmem_base_s, TMEM_COLS);
@@ -212,46 +224,56 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       // B: the key tile read MN-major (N = feature a, K = token): one atom of 64 features x 8 tokens per 1 KB
       const uint64_t dB = smem_desc(0, 16384, 1024, kSwizzle128B);
       const bool producer = (warp == WARP_UB);
-      auto load_tiles = [&](int j) -> bool {
+      auto load_k = [&](int j) -> bool {
         const int s = j & 1;
-        if (!wait_or_abort(bar(BAR_KQ_EMPTY + s), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
-        mbar_arrive_expect_tx(bar(BAR_KQ_FULL + s), 32768);
-        tma_load_3d(qtile(s), &tmQ, bar(BAR_KQ_FULL + s), 0, j * CT, bh);
-        tma_load_3d(ktile(s), &tmK, bar(BAR_KQ_FULL + s), 0, j * CT, bh);
+        if (!wait_or_abort(bar(BAR_K_EMPTY + s), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
+        mbar_arrive_expect_tx(bar(BAR_K_FULL + s), 16384);
+        tma_load_3d(ktile(s), &tmK, bar(BAR_K_FULL + s), 0, j * CT, bh);
+        return true;
+      };
+      auto load_q = [&](int j) -> bool {     // one staging buffer: free once the previous tile was copied to TMEM
+        if (!wait_or_abort(bar(BAR_QS_EMPTY), (j & 1) ^ 1, abort_flag)) return false;
+        mbar_arrive_expect_tx(bar(BAR_Q_FULL), 16384);
+        tma_load_3d(qtile, &tmQ, bar(BAR_Q_FULL), 0, j * CT, bh);
         return true;
       };
       if (producer) {
-        ok = load_tiles(0);
-        if (ok && nch > 1) ok = load_tiles(1);
+        ok = load_k(0) && load_q(0);
+        if (ok && nch > 1) ok = load_k(1);
       }
+      uint32_t wbi = 0, wph = 0;             // W buffer of the step and the parity of its phase
       for (int j = 0; j < nch && ok; ++j) {
         const int s = j & 1;
-        ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag);
+        ok = wait_or_abort(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag);
         if (ok && j > 0) ok = wait_or_abort(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
-        // the stage of tile j - 1 is free once that tile's consumers are through: refill it with tile j + 1
-        if (ok && producer && j > 0 && j + 1 < nch) ok = load_tiles(j + 1);
+        // the key stage of tile j - 1 is free once that tile's consumers are through: refill it with tile j + 1
+        if (ok && producer && j > 0 && j + 1 < nch) ok = load_k(j + 1);
 #pragma unroll 1
         for (int sc = 0; sc < 8 && ok; ++sc) {
-          const int g = 8 * j + sc, wb = g & 1;
-          ok = wait_or_abort(bar(BAR_W_FULL + wb), (g >> 1) & 1, abort_flag);
+          ok = wait_or_abort(bar(BAR_W_FULL + wbi), wph, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t wa = smem_u32(wbuf(wb)), ka = smem_u32(ktile(s)) + sc * 2048;
+          const uint32_t wa = smem_u32(wbuf(wbi)), ka = smem_u32(ktile(s)) + sc * 2048;
           const uint64_t db = at(dB, ka);
-          const uint32_t acc = g > 0 ? 1u : 0u;
+          const uint32_t acc = (j > 0 || sc > 0) ? 1u : 0u;
           if (producer) {
             mma_f16_ss(tb + COL_S + 96, at(dA, wa + 3 * 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64), acc);
-            mma_f16_ss(tb + COL_Z, at(dA, wa + 4 * 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64), acc);
+            // Z rows: 64 rows of this buffer, the other 64 rows of the tile read the zero atom (LBO reaches it)
+            mma_f16_ss(tb + COL_Z, smem_desc(wa + 16384, smem_u32(base + OFF_ZERO) - (wa + 16384), 1024, kSwizzle128B), db,
+                       instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64), acc);
           } else {
             mma_f16_ss(tb + COL_S + 0, at(dA, wa), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 16), acc);
             mma_f16_ss(tb + COL_S + 16, at(dA, wa + 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 32), acc);
             mma_f16_ss(tb + COL_S + 48, at(dA, wa + 2 * 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 48), acc);
           }
-          mma_commit(bar(BAR_W_EMPTY + wb));
+          mma_commit(bar(BAR_W_EMPTY + wbi));
+          if (++wbi == NWBUF) { wbi = 0; wph ^= 1; }
         }
         if (!ok) break;
         mma_commit(bar(BAR_U_DONE));
-        mma_commit(bar(BAR_KQ_EMPTY + s));
+        mma_commit(bar(BAR_K_EMPTY + s));
+        // the query staging buffer is free once tile j was copied to TMEM (at the end of tile j - 1)
+        if (producer && j + 1 < nch) ok = load_q(j + 1);
       }
     }
   } else if (warp == WARP_R) {
@@ -288,7 +310,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const uint64_t dK = smem_desc(0, 16, 1024, kSwizzle128B);
       for (int j = 0; j < nch && ok; ++j) {
         const int s = j & 1;
-        ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag) &&
+        ok = wait_or_abort(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag) &&
              wait_or_abort(bar(BAR_QT_FULL), j & 1, abort_flag) &&
              wait_or_abort(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
         // the weights of the previous tile's second half are read by its last apply MMAs
@@ -317,32 +339,99 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         if (!ok) break;
         mma_commit(bar(BAR_O_FULL));
-        mma_commit(bar(BAR_KQ_EMPTY + s));
+        mma_commit(bar(BAR_K_EMPTY + s));
       }
     }
   } else if (warp < WARP_RD0) {
-    // =========================== W builders (+ a share of the snapshot) ===========================
-    // Two teams of four warps: team 0 (warps 4-7) builds the even 16-token steps into buffer 0, team 1 the odd
-    // steps into buffer 1.  Warp = b-block, lanes = 16 tokens x 2 halves of the block.
+    // =========================== W builders (+ shares of the snapshot) ===========================
+    // Two teams of four warps: team 0 (warps 4-7) builds the even 16-token steps, team 1 the odd steps, into a
+    // ring of three buffers.  Warp = b-block, lanes = 16 tokens x 2 halves of the block.
     const int beta = warp & 3;
     const int team = (warp - WARP_BLD0) >> 2;
     const uint32_t q4 = warp & 3;
     const int tk = lane & 15, half = lane >> 4;
+    const int row_t = q4 * 32 + lane, bloc = row_t >> 3, vv = row_t & 7;    // snapshot: row of a state tile
+    uint32_t wbi = team, wph = 0;                                           // buffer and phase parity of the next step
+    // snapshot share of team 0: b-block 1 and the Z rows; of team 1: b-blocks 2 and 0 (b-block 3: warps 20-23).
+    // The buffer written was read by the reads of tile jp - 1.  They are complete: warps 20-23 wait for them
+    // before they scale tile jp + 1, and the callers have waited for those scales (BAR_PREP).
+    auto snapshot_share = [&](int jp) -> bool {
+      if (!wait_or_abort(bar(BAR_U_DONE), jp & 1, abort_flag)) return false;
+      tc_fence_after();
+      unsigned char* sp = base + OFF_SP + ((jp + 1) & 1) * SP_BYTES;
+      auto rowp = [&](int p) { return sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128; };
+      if (team == 1) {
+        uint32_t e[32], f[16], c0[16];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 48), e);
+        tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 80), f);
+        tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 0), c0);
+        const int p2 = 4 + (bloc >> 3), p0 = bloc >> 3;
+        unsigned char* row2 = rowp(p2);
+        const uint32_t c2 = sp_koff(p2) >> 4;
+        tmem_wait_ld(e);
+        tmem_wait_ld(f);
+        tmem_wait_ld(c0);
+        tc_fence_before();
+        mbar_arrive(bar(BAR_SNAP_LD));
+        snap_store16(row2, c2, vv, e, 2.f);
+        snap_store16(row2, c2 + 2, vv, e + 16, 2.f);
+        snap_store16(row2, c2 + 4, vv, f, 1.f);
+        snap_store16(rowp(p0), sp_koff(p0) >> 4, vv, c0, 1.f);
+      } else {
+        uint32_t c1[32];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 16), c1);
+        const int p1 = 2 + (bloc >> 3);
+        unsigned char* r1 = rowp(p1);
+        const uint32_t k1 = sp_koff(p1) >> 4;
+        if (q4 < 2) {
+          // Z rows: lane = b; row 64 + (b % 8) of piece b / 8, features a < 16 (b / 16 + 1)
+          uint32_t z0[32];
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z), z0);
+          tmem_wait_ld(c1);
+          snap_store16(r1, k1, vv, c1, 2.f);
+          snap_store16(r1, k1 + 2, vv, c1 + 16, 1.f);
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z + 32), c1);
+          tmem_wait_ld(z0);
+          tmem_wait_ld(c1);
+          tc_fence_before();
+          mbar_arrive(bar(BAR_SNAP_LD));
+          const int b = row_t, bz = b >> 4, pz = b >> 3;
+          unsigned char* rowz = sp + sp_block(pz) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
+          const uint32_t cz = sp_koff(pz) >> 4;
+          const uint32_t rz = (uint32_t)(b & 7);
+          snap_store16(rowz, cz, rz, z0, 0 < bz ? 2.f : 1.f);
+          if (1 <= bz) snap_store16(rowz, cz + 2, rz, z0 + 16, 1 < bz ? 2.f : 1.f);
+          if (2 <= bz) snap_store16(rowz, cz + 4, rz, c1, 2 < bz ? 2.f : 1.f);
+          if (3 <= bz) snap_store16(rowz, cz + 6, rz, c1 + 16, 1.f);
+        } else {
+          tmem_wait_ld(c1);
+          tc_fence_before();
+          mbar_arrive(bar(BAR_SNAP_LD));
+          snap_store16(r1, k1, vv, c1, 2.f);
+          snap_store16(r1, k1 + 2, vv, c1 + 16, 1.f);
+        }
+      }
+      fence_async_smem();
+      mbar_arrive(bar(BAR_SNAP_ST));
+      return true;
+    };
     for (int j = 0; j < nch && ok; ++j) {
       const int s = j & 1;
-      ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag) &&
+      ok = wait_or_abort(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag) &&
            wait_or_abort(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
+      // team 1 copies its share of the state after tile j - 1 before its first step of tile j, team 0 after
+      // its first step: either way right when the update of tile j - 1 completes
+      if (ok && team == 1 && j > 0) ok = snapshot_share(j - 1);
 #pragma unroll 1
       for (int sc = team; sc < 8 && ok; sc += 2) {
-        const int g = 8 * j + sc;
         const int t = sc * 16 + tk;
         const uint4 kraw = *reinterpret_cast<const uint4*>(ktile(s) + sw128_offset(t, 2 * beta + half));
         const uint4 vp = *reinterpret_cast<const uint4*>(vptile(s) + t * 16);
         const uint32_t rr = r2pair(s)[t];
         const uint32_t kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
-        ok = wait_or_abort(bar(BAR_W_EMPTY + team), ((g >> 1) & 1) ^ 1, abort_flag);
+        ok = wait_or_abort(bar(BAR_W_EMPTY + wbi), wph ^ 1, abort_flag);
         if (!ok) break;
-        unsigned char* wrow = wbuf(team) + (tk >> 3) * 1024 + (tk & 7) * 128;
+        unsigned char* wrow = wbuf(wbi) + (tk >> 3) * 1024 + (tk & 7) * 128;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const uint32_t kbb = __byte_perm(kw[i >> 1], 0u, (i & 1) ? 0x3232 : 0x1010);
@@ -359,62 +448,14 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           w.y = mul_bf16x2(kw[1], rr);
           w.z = mul_bf16x2(kw[2], rr);
           w.w = mul_bf16x2(kw[3], rr);
-          *reinterpret_cast<uint4*>(wrow + 4 * 4096 + (((2 * beta + half) ^ (tk & 7)) << 4)) = w;
+          *reinterpret_cast<uint4*>(wrow + 16384 + (((2 * beta + half) ^ (tk & 7)) << 4)) = w;
         }
         fence_async_smem();
-        mbar_arrive(bar(BAR_W_FULL + team));
-      }
-      if (!ok) break;
-      if (team == 1 && j + 1 < nch) {
-        // ---- snapshot of the state after tile j: b-block 2 and the Z rows (the other blocks: warps 20-23) ----
-        // The buffer written here was read by the reads of tile j - 1.  They are complete: warps 20-23 wait for
-        // them before they scale tile j + 1, and this warp waits for those scales first.
-        const int s1 = (j + 1) & 1;
-        ok = wait_or_abort(bar(BAR_KQ_FULL + s1), ((j + 1) >> 1) & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_PREP + s1), ((j + 1) >> 1) & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_U_DONE), j & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const int row_t = q4 * 32 + lane, bloc = row_t >> 3, vv = row_t & 7;
-        unsigned char* sp = base + OFF_SP + ((j + 1) & 1) * SP_BYTES;
-        uint32_t e[32], f[16];
-        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 48), e);
-        tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 80), f);
-        const int p2 = 4 + (bloc >> 3);
-        unsigned char* row2 = sp + sp_block(p2) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
-        const uint32_t c2 = sp_koff(p2) >> 4;
-        tmem_wait_ld(e);
-        tmem_wait_ld(f);
-        if (q4 < 2) {
-          // Z rows: lane = b; row 64 + (b % 8) of piece b / 8, features a < 16 (b / 16 + 1)
-          uint32_t z0[32];
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z), z0);
-          snap_store16(row2, c2, vv, e, 2.f);
-          snap_store16(row2, c2 + 2, vv, e + 16, 2.f);
-          snap_store16(row2, c2 + 4, vv, f, 1.f);
-          uint32_t z1[32];
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z + 32), z1);
-          tmem_wait_ld(z0);
-          tmem_wait_ld(z1);
-          tc_fence_before();
-          mbar_arrive(bar(BAR_SNAP_LD));
-          const int b = row_t, bz = b >> 4, pz = b >> 3;
-          unsigned char* rowz = sp + sp_block(pz) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
-          const uint32_t cz = sp_koff(pz) >> 4;
-          const uint32_t rz = (uint32_t)(b & 7);
-          snap_store16(rowz, cz, rz, z0, 0 < bz ? 2.f : 1.f);
-          if (1 <= bz) snap_store16(rowz, cz + 2, rz, z0 + 16, 1 < bz ? 2.f : 1.f);
-          if (2 <= bz) snap_store16(rowz, cz + 4, rz, z1, 2 < bz ? 2.f : 1.f);
-          if (3 <= bz) snap_store16(rowz, cz + 6, rz, z1 + 16, 1.f);
-        } else {
-          tc_fence_before();
-          mbar_arrive(bar(BAR_SNAP_LD));
-          snap_store16(row2, c2, vv, e, 2.f);
-          snap_store16(row2, c2 + 2, vv, e + 16, 2.f);
-          snap_store16(row2, c2 + 4, vv, f, 1.f);
-        }
-        fence_async_smem();
-        mbar_arrive(bar(BAR_SNAP_ST));
+        mbar_arrive(bar(BAR_W_FULL + wbi));
+        // this team's next step is two steps on: two buffers further in the ring of three
+        wbi += 2;
+        if (wbi >= NWBUF) { wbi -= NWBUF; wph ^= 1; }
+        if (sc == 0 && j > 0) ok = snapshot_share(j - 1);
       }
     }
   } else if (warp < WARP_AUX0) {
@@ -427,17 +468,22 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     float* part = reinterpret_cast<float*>(base + OFF_PART);
     const uint32_t ycol = tmem_addr(tb, q4 * 32, COL_Y + team * 80);
     for (int j = 0; j < nch && ok; ++j) {
-      const int s = j & 1;
-      ok = wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag);
+      ok = wait_or_abort(bar(BAR_QT_FULL), j & 1, abort_flag);    // the multipliers come from the TMEM copy of the query tile
       if (!ok) break;
+      tc_fence_after();
       float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       float accz = 0.f;
 #pragma unroll 1
       for (int p = team; p < 8; p += 2) {
         const int g = 8 * j + p;
         // q[t, 8p .. 8p+7]: the multipliers of this piece
-        const uint4 qraw = *reinterpret_cast<const uint4*>(qtile(s) + sw128_offset(t, p));
-        const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
+        uint32_t qw[4];
+        tmem_ld4(tmem_addr(tb, q4 * 32, COL_Q + 4 * p), qw);
+        tmem_wait_ld(qw);
+        if (p >= 6) {          // last piece of this team: the query tile in TMEM may be replaced
+          tc_fence_before();
+          mbar_arrive(bar(BAR_Q_FREE));
+        }
         ok = wait_or_abort(bar(BAR_Y_FULL + team), (g >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -477,7 +523,6 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
       }
       if (!ok) break;
-      mbar_arrive(bar(BAR_KQ_EMPTY + s));
       if (team == 1) {
         ok = wait_or_abort(bar(BAR_PART_EMPTY), (j & 1) ^ 1, abort_flag);
         if (!ok) break;
@@ -530,7 +575,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // key scales and v' of tile j (the value slice was fetched one tile earlier)
     auto prep = [&](int j, const uint4& vraw) -> bool {
       const int s = j & 1;
-      if (!wait_or_abort(bar(BAR_KQ_FULL + s), (j >> 1) & 1, abort_flag)) return false;
+      if (!wait_or_abort(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag)) return false;
       float ss = 0.f;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
@@ -556,6 +601,28 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       mbar_arrive(bar(BAR_PREP + s));
       return true;
     };
+    // this warp's share of the snapshot of the state after tile j (b-block 3; the other blocks and Z: warps 4-11);
+    // the update of tile j is complete (BAR_U_DONE observed by the caller)
+    auto snapshot_share = [&](int j) {
+      tc_fence_after();
+      const int bloc = t >> 3, vv = t & 7;          // row of a state tile = 8 * (b within the block) + v
+      unsigned char* sp = base + OFF_SP + ((j + 1) & 1) * SP_BYTES;
+      const int p3 = 6 + (bloc >> 3);
+      unsigned char* r3 = sp + sp_block(p3) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
+      uint32_t a0[32], a1[32];
+      tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 96), a0);
+      tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 128), a1);
+      tmem_wait_ld(a0);
+      tmem_wait_ld(a1);
+      tc_fence_before();
+      mbar_arrive(bar(BAR_SNAP_LD));
+      snap_store16(r3, 0, vv, a0, 2.f);
+      snap_store16(r3, 2, vv, a0 + 16, 2.f);
+      snap_store16(r3, 4, vv, a1, 2.f);
+      snap_store16(r3, 6, vv, a1 + 16, 1.f);
+      fence_async_smem();
+      mbar_arrive(bar(BAR_SNAP_ST));
+    };
     uint4 vnext = load_v(0);
     for (int j = -1; j < nch && ok; ++j) {
       // ---- scales of the next tile, so that its W rows can be built during this tile's update ----
@@ -564,12 +631,20 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (!ok) break;
         vnext = load_v(j + 2);
       }
+      bool snapped = (j < 0) || (j + 1 >= nch);      // nothing to copy before the first and after the last tile
       // ---- weights P = (q.k)^2, causal, two halves of 64 keys ----
       if (j >= 0) {
 #pragma unroll 1
         for (int h = 0; h < 2; ++h) {
-          ok = wait_or_abort(bar(BAR_S_FULL), h, abort_flag);
-          if (!ok) break;
+          // The copy of the state out of TMEM sits between two updates: serve it first when the update
+          // completes while this warp waits for scores.
+          ok = false;
+          for (uint32_t i = 0; i < kSpinLimit; ++i) {
+            if (mbar_test_wait(bar(BAR_S_FULL), h)) { ok = true; break; }
+            if (!snapped && mbar_test_wait(bar(BAR_U_DONE), j & 1)) { snapshot_share(j); snapped = true; }
+            if ((i & 1023u) == 1023u && *abort_flag) break;
+          }
+          if (!ok) { *abort_flag = 1; break; }
           tc_fence_after();
           const uint32_t scol = tmem_addr(tb, q4 * 32, COL_P);
           // 32 scores at a time; the bf16 weights go back over columns this thread has already read
@@ -596,51 +671,24 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (!ok) break;
       }
       if (j + 1 >= nch) break;
-      // ---- snapshot of the state after tile j: b-blocks 3, 1 and 0 (b-block 2 and Z: warps 4-7) ----
-      if (j >= 0) {
+      if (!snapped) {
         ok = wait_or_abort(bar(BAR_U_DONE), j & 1, abort_flag);
         if (!ok) break;
-        tc_fence_after();
-        const int bloc = t >> 3, vv = t & 7;          // row of a state tile = 8 * (b within the block) + v
-        unsigned char* sp = base + OFF_SP + ((j + 1) & 1) * SP_BYTES;
-        auto rowp = [&](int p) { return sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128; };
-        const int p3 = 6 + (bloc >> 3), p1 = 2 + (bloc >> 3), p0 = bloc >> 3;
-        uint32_t a0[32], a1[32];
-        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 96), a0);
-        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 128), a1);
-        unsigned char* r3 = rowp(p3);
-        tmem_wait_ld(a0);
-        snap_store16(r3, 0, vv, a0, 2.f);
-        snap_store16(r3, 2, vv, a0 + 16, 2.f);
-        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 16), a0);      // b-block 1
-        tmem_wait_ld(a1);
-        snap_store16(r3, 4, vv, a1, 2.f);
-        snap_store16(r3, 6, vv, a1 + 16, 1.f);
-        uint32_t c0[16];
-        tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 0), c0);       // b-block 0
-        tmem_wait_ld(a0);
-        tmem_wait_ld(c0);
-        tc_fence_before();
-        mbar_arrive(bar(BAR_SNAP_LD));
-        unsigned char* r1 = rowp(p1);
-        const uint32_t k1 = sp_koff(p1) >> 4;
-        snap_store16(r1, k1, vv, a0, 2.f);
-        snap_store16(r1, k1 + 2, vv, a0 + 16, 1.f);
-        snap_store16(rowp(p0), sp_koff(p0) >> 4, vv, c0, 1.f);
-        fence_async_smem();
-        mbar_arrive(bar(BAR_SNAP_ST));
+        snapshot_share(j);
       }
-      // ---- query tile j + 1 to TMEM, once the reads and scores of tile j are complete (the scores: see above) ----
+      // ---- query tile j + 1 to TMEM, once the reads of tile j are complete, the readers hold their multipliers
+      //      (the scores of tile j are complete: see above) and the tile has landed ----
       {
-        if (j >= 0) ok = wait_or_abort(bar(BAR_R_DONE), j & 1, abort_flag);
+        if (j >= 0) ok = wait_or_abort(bar(BAR_R_DONE), j & 1, abort_flag) && wait_or_abort(bar(BAR_Q_FREE), j & 1, abort_flag);
+        if (ok) ok = wait_or_abort(bar(BAR_Q_FULL), (j + 1) & 1, abort_flag);
         if (!ok) break;
-        const int s1 = (j + 1) & 1;
         uint32_t qw[32];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-          const uint4 raw = *reinterpret_cast<const uint4*>(qtile(s1) + sw128_offset(t, c));
+          const uint4 raw = *reinterpret_cast<const uint4*>(qtile + sw128_offset(t, c));
           qw[4 * c] = raw.x; qw[4 * c + 1] = raw.y; qw[4 * c + 2] = raw.z; qw[4 * c + 3] = raw.w;
         }
+        mbar_arrive(bar(BAR_QS_EMPTY));
         tc_fence_after();
         tmem_st32(tmem_addr(tb, q4 * 32, COL_Q), qw);
         tmem_wait_st();
