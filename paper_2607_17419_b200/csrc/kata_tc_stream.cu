@@ -107,7 +107,8 @@ struct SArgs {
 __device__ __noinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    __nanosleep(32);
+    __nanosleep(64);
+
     if ((i & 1023u) == 1023u && *abort_flag) return false;
   }
   *abort_flag = 1;
