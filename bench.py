@@ -258,7 +258,7 @@ def run_ours(args):
             # DRAM bytes per launch: ncu on the T=32768 case (202.1 MB read + 47.9 MB written), times 4 (linear in T)
             traffic = 4 * (202.1e6 + 47.9e6)
             roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
-                        traffic=traffic, kernel="kata::tc_chunk_kernel (tcgen05 chunked forward)",
+                        traffic=traffic, kernel="kata::tc_stream_kernel (tcgen05 token-major chunked forward)",
                         note=f"algorithmic flops (packed feature n=2080) / CUDA-event time; peak = "
                              f"{'sustained' if sustained else 'burst'} bf16 cuBLAS of {peaks['source']}")
         else:
