@@ -175,8 +175,20 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       tma_load_3d(base + OFF_Q, &tmQ, bar(BAR_QFULL), 0, q0, bh);
     }
     const __nv_bfloat16* rs = args.rscale + (size_t)bh * args.Tlen;
+    // r of this lane's 4 keys of a tile, fetched one tile ahead (the global-load latency stays off the ring)
+    auto load_r = [&](int j, unsigned short (&rv)[4]) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int key = j * KTILE + lane * 4 + e;
+        rv[e] = (j < ntiles && key < args.Tlen) ? __bfloat16_as_ushort(rs[key]) : (unsigned short)0;
+      }
+    };
+    unsigned short rv[4];
+    load_r(0, rv);
     for (int j = 0; j < ntiles && ok; ++j) {
       const int s = j % NSTAGE;
+      unsigned short rn[4];
+      load_r(j + 1, rn);
       ok = wait_or_abort(bar(BAR_EMPTY + s), ((j / NSTAGE) & 1) ^ 1, abort_flag);
       if (!ok) break;
       if (lane == 0) {
@@ -188,9 +200,8 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       unsigned char* rt = rtile(s);
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const int kr = lane * 4 + e, key = j * KTILE + kr;
-        const unsigned short rv = key < args.Tlen ? __bfloat16_as_ushort(rs[key]) : (unsigned short)0;
-        *reinterpret_cast<uint16_t*>(rt + sw128_offset(kr, 0)) = rv;
+        *reinterpret_cast<uint16_t*>(rt + sw128_offset(lane * 4 + e, 0)) = rv[e];
+        rv[e] = rn[e];
       }
       fence_async_smem();
       mbar_arrive(bar(BAR_FULL + s));
