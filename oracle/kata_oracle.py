@@ -168,6 +168,22 @@ def kata_recurrent(q, k, v, feature: str = "psd_direct"):
     return o
 
 
+def kata_decode_step(S, Z, q, k, v, feature: str = "psd_direct"):
+    """One token of the recurrent form ("Linear attention as a recurrence": S_t = S_{t-1} + psi(k_t) v_t^T,
+    Z_t = Z_{t-1} + psi(k_t), readout psi(q_t)^T S_t / psi(q_t)^T Z_t; 0 where the denominator is 0).
+
+    S [n_psi, d_v], Z [n_psi], q, k [d_k], v [d_v].  Returns (o, S_new, Z_new); the inputs are not modified.
+    """
+    fq = apply_feature(np.asarray(q, dtype=np.float64)[None, :], feature)[0]
+    fk = apply_feature(np.asarray(k, dtype=np.float64)[None, :], feature)[0]
+    v = np.asarray(v, dtype=np.float64)
+    S_new = np.asarray(S, dtype=np.float64) + np.outer(fk, v)
+    Z_new = np.asarray(Z, dtype=np.float64) + fk
+    den = fq @ Z_new
+    o = (fq @ S_new) / den if den != 0 else np.zeros_like(v)
+    return o, S_new, Z_new
+
+
 # ---------------------------------------------------------------------------
 # form C: Algorithm 1 (chunkwise forward)
 # ---------------------------------------------------------------------------

@@ -643,6 +643,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           for (uint32_t i = 0; i < kSpinLimit; ++i) {
             if (mbar_test_wait(bar(BAR_S_FULL), h)) { ok = true; break; }
             if (!snapped && mbar_test_wait(bar(BAR_U_DONE), j & 1)) { snapshot_share(j); snapped = true; }
+            __nanosleep(64);
             if ((i & 1023u) == 1023u && *abort_flag) break;
           }
           if (!ok) { *abort_flag = 1; break; }

@@ -352,3 +352,57 @@ def test_batched_wrapper():
         assert np.array_equal(ob[b, h], ko.kata_chunked(q[b, h], k[b, h], v[b, h], 8))
     ob2 = ko.batched(ko.kata_quadratic, q, k, v)
     assert np.allclose(ob, ob2, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------
+# decode step (the recurrence taken one token at a time)
+# ---------------------------------------------------------------------------
+
+def _decode_all(q, k, v, feature):
+    n = ko.feature_dim(q.shape[1], feature)
+    S, Z = np.zeros((n, v.shape[1])), np.zeros(n)
+    out = []
+    for t in range(q.shape[0]):
+        o, S, Z = ko.kata_decode_step(S, Z, q[t], k[t], v[t], feature)
+        out.append(o)
+    return np.array(out), S, Z
+
+
+@pytest.mark.parametrize("feature", ["psd_direct", "psd_packed", "identity"])
+def test_decode_steps_from_zero_state_give_the_definition(feature):
+    # brute force (pure Python loops over the definition) for the PSD features; for the identity feature the
+    # weights are plain dot products, checked against a dense masked matmul
+    q, k, v = rand_qkv(31, 7, 3, 2)
+    o, S, Z = _decode_all(q, k, v, feature)
+    if feature == "identity":
+        w = np.tril(q @ k.T)
+        ref = (w @ v) / w.sum(axis=1, keepdims=True)
+    else:
+        ref = brute(q.tolist(), k.tolist(), v.tolist())
+    assert np.allclose(o, ref, atol=1e-12)
+    # the state is the plain sum of feature-value outer products; its row sums against ones give Z
+    fk = ko.apply_feature(k, feature)
+    assert np.allclose(S, fk.T @ v, atol=1e-13) and np.allclose(Z, fk.sum(axis=0), atol=1e-13)
+
+
+def test_decode_step_special_cases():
+    # d_k = 1: every weight is 1, so the outputs are the running mean of v
+    r = rng(33)
+    q, k, v = r.standard_normal((9, 1)), r.standard_normal((9, 1)), r.standard_normal((9, 3))
+    o, _, Z = _decode_all(q, k, v, "psd_direct")
+    assert np.allclose(o, np.cumsum(v, axis=0) / np.arange(1, 10)[:, None], atol=1e-13)
+    assert np.allclose(Z, [9.0])
+    # zero key leaves the state unchanged; zero query reads 0; the inputs are not modified
+    S0, Z0 = np.ones((4, 2)), np.ones(4)
+    o, S1, Z1 = ko.kata_decode_step(S0, Z0, [1.0, 2.0], [0.0, 0.0], [5.0, 6.0])
+    assert np.array_equal(S1, S0) and np.array_equal(Z1, Z0) and np.all(S0 == 1)
+    o, _, _ = ko.kata_decode_step(S0, Z0, [0.0, 0.0], [1.0, 0.0], [5.0, 6.0])
+    assert np.all(o == 0)
+    # resuming from the exclusive-prefix state of a chunk reproduces the rest of the sequence
+    q, k, v = rand_qkv(35, 12, 3, 2)
+    full = ko.kata_quadratic(q, k, v)[0]
+    _, S_pre, Z_pre = ko.kata_scan(q, k, v, 4)
+    S, Z = S_pre[2], Z_pre[2]
+    for t in range(8, 12):
+        o, S, Z = ko.kata_decode_step(S, Z, q[t], k[t], v[t])
+        assert np.allclose(o, full[t], atol=1e-12)
