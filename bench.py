@@ -344,6 +344,20 @@ def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
     res["quadratic_c2"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=fl / (ms * 1e-3) / 1e12,
                                frac_of_bf16_burst=fl / (ms * 1e-3) / 1e12 / peaks["bf16_burst"],
                                impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
+    # decode step: B=16, H=16, d=64, bf16 tokens, fp32 state in the direct layout (285 MB of state > L2);
+    # HBM-bound: the state is read and written once per token
+    Bd, Hd, d = 16, 16, 64
+    g = torch.Generator(device="cpu").manual_seed(5)
+    qd, kd, vd = (torch.randn(Bd, Hd, d, generator=g).to(torch.bfloat16).to(dev) for _ in range(3))
+    n_psi = kb.decode_n_psi(d)
+    S = torch.zeros(Bd, Hd, n_psi, d, device=dev)
+    Z = torch.zeros(Bd, Hd, n_psi, device=dev)
+    od = torch.empty_like(vd)
+    ms = timed(lambda: kb.kata_decode_step(qd, kd, vd, S, Z, od), reps=20, warm=3)
+    nbytes = 2 * Bd * Hd * n_psi * (d + 1) * 4
+    res["decode_step"] = dict(ms=ms, tokens_per_s=Bd / (ms * 1e-3), heads=Bd * Hd, state_bytes_per_step=nbytes,
+                              gbs=nbytes / (ms * 1e-3) / 1e9, frac_of_hbm=nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                              launches=kb.kata_last_launch_count())
     return res
 
 

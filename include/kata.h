@@ -59,7 +59,7 @@ enum { KATA_F32 = 0, KATA_BF16 = 1 };                 /* kata_opts.dtype        
 enum { KATA_LAYOUT_DIRECT = 0, KATA_LAYOUT_PACKED = 1 }; /* kata_opts.state_layout */
 enum { KATA_SEQUENTIAL = 0, KATA_SCAN = 1 };          /* kata_opts.inter_chunk    */
 enum { KATA_IMPL_AUTO = 0, KATA_IMPL_SIMT = 1, KATA_IMPL_TENSOR = 2 }; /* kata_opts.impl */
-enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2 };
+enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2, KATA_FN_DECODE_STEP = 3 };
 
 /*
  * Options (plain data; zero-initialise, then set struct_size = sizeof(kata_opts)).
@@ -140,6 +140,22 @@ int kata_fwd_chunked(const void* q, const void* k, const void* v, void* out,
  */
 int kata_chunk_state_scan(const void* q, const void* k, const void* v, void* out,
                           int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
+
+/*
+ * One token of the recurrent form (section "Linear attention as a recurrence": S_t = S_{t-1} + psi(k_t) v_t^T,
+ * Z_t = Z_{t-1} + psi(k_t), readout psi(q_t)^T S_t / psi(q_t)^T Z_t), for every (b,h): the constant-time decode
+ * step that follows a prefill.
+ *   q, k [B,H,d_k]; v, out [B,H,d_v] (element type opts->dtype, device pointers, 16-byte aligned);
+ *   S [B,H,n_psi,d_v], Z [B,H,n_psi]: fp32 device state, updated IN PLACE (read and written once per call),
+ *   in the layout of the exported prefix states (opts->state_layout / feature_order, see kata_opts): the
+ *   s_pre/z_pre slice of a chunk written by kata_chunk_state_scan is a valid state to resume from, and an
+ *   all-zero state starts a sequence.  out = 0 where the denominator is 0.
+ * The state of a head is reduced in a fixed order: results are bit-reproducible.  opts->inter_chunk, impl,
+ * scan_group are ignored; opts->s_pre/z_pre must be null.
+ * Workspace: kata_workspace_bytes(KATA_FN_DECODE_STEP, B, H, 1, d_k, d_v, 0, opts).
+ */
+int kata_decode_step(const void* q, const void* k, const void* v, void* out, float* S, float* Z,
+                     int B, int H, int d_k, int d_v, const kata_opts* opts);
 
 /*
  * Same computation as entry point `fn` (a KATA_FN_* value) but q,k,v,out are HOST pointers

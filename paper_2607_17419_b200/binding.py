@@ -18,11 +18,11 @@ KATA_F32, KATA_BF16 = 0, 1
 KATA_LAYOUT_DIRECT, KATA_LAYOUT_PACKED = 0, 1
 KATA_SEQUENTIAL, KATA_SCAN = 0, 1
 KATA_IMPL_AUTO, KATA_IMPL_SIMT, KATA_IMPL_TENSOR = 0, 1, 2
-KATA_FN_QUADRATIC, KATA_FN_CHUNKED, KATA_FN_CHUNK_STATE_SCAN = 0, 1, 2
+KATA_FN_QUADRATIC, KATA_FN_CHUNKED, KATA_FN_CHUNK_STATE_SCAN, KATA_FN_DECODE_STEP = 0, 1, 2, 3
 KATA_FN_HOST_IO = 0x100
 
 EXPORTS = ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan", "kata_chunk_state_scan_static",
-           "kata_fwd_host",
+           "kata_fwd_host", "kata_decode_step",
            "kata_workspace_bytes", "kata_scan_plan", "kata_last_launch_count", "kata_last_impl",
            "kata_status_string",
            "kata_version")
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         getattr(L, name).restype = i
     L.kata_fwd_host.argtypes = [i] + fwd_args
     L.kata_fwd_host.restype = i
+    L.kata_decode_step.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, i, i, i, i, ctypes.POINTER(KataOpts)]
+    L.kata_decode_step.restype = i
     L.kata_workspace_bytes.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(KataOpts)]
     L.kata_workspace_bytes.restype = ctypes.c_size_t
     L.kata_scan_plan.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(KataOpts)] + [ctypes.POINTER(i)] * 3
@@ -216,6 +218,42 @@ def kata_chunk_state_scan(q, k, v, out=None, C: int = 64, **kw):
 def kata_fwd_host(fn: int, q, k, v, out, C: int = 64, **kw):
     """Same as entry point ``fn`` with (pinned) host tensors; copies ride the current CUDA stream."""
     return _call(fn, q, k, v, out, C, host_io=True, **kw)
+
+
+def decode_n_psi(d_k: int, feature_order: int = 2, state_layout: int = KATA_LAYOUT_DIRECT) -> int:
+    """Feature rows of the decode state: d_k (order 1), d_k^2 (direct) or d_k(d_k+1)/2 (packed)."""
+    if feature_order == 1:
+        return d_k
+    return d_k * (d_k + 1) // 2 if state_layout == KATA_LAYOUT_PACKED else d_k * d_k
+
+
+def kata_decode_step(q, k, v, S, Z, out=None, *, workspace: Optional[Workspace] = None, stream=None, **opt_kw):
+    """One decode token per (b,h): q,k [B,H,d_k], v [B,H,d_v]; fp32 state S [B,H,n_psi,d_v], Z [B,H,n_psi] is
+    updated in place.  Returns out [B,H,d_v]."""
+    import torch
+    B, H, d_k = q.shape
+    d_v = v.shape[-1]
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and S.is_contiguous() and Z.is_contiguous()):
+        raise ValueError("q, k, v, S, Z must be contiguous")
+    if S.dtype != torch.float32 or Z.dtype != torch.float32:
+        raise ValueError("the state is fp32")
+    if out is None:
+        out = torch.empty_like(v)
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    opts = make_opts(_dtype_code(q), stream=stream, **opt_kw)
+    n_psi = decode_n_psi(d_k, opts.feature_order, opts.state_layout)
+    if tuple(S.shape) != (B, H, n_psi, d_v) or tuple(Z.shape) != (B, H, n_psi):
+        raise ValueError(f"state shapes must be {(B, H, n_psi, d_v)} and {(B, H, n_psi)}")
+    need = kata_workspace_bytes(KATA_FN_DECODE_STEP, B, H, 1, d_k, d_v, 0, opts)
+    ws = workspace if workspace is not None else _default_ws
+    ptr, size = ws.get(need, q.device)
+    opts.workspace, opts.workspace_bytes = ptr or None, size
+    st = lib().kata_decode_step(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), S.data_ptr(), Z.data_ptr(),
+                                B, H, d_k, d_v, ctypes.byref(opts))
+    if st != 0:
+        raise KataError(st, "kata_decode_step")
+    return out
 
 
 KATA_STATIC_SCRATCH_BYTES = 32 << 20

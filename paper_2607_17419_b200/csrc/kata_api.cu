@@ -251,6 +251,33 @@ int kata_chunk_state_scan(const void* q, const void* k, const void* v, void* out
   return entry(KATA_FN_CHUNK_STATE_SCAN, q, k, v, out, B, H, T, d_k, d_v, C, opts);
 }
 
+int kata_decode_step(const void* q, const void* k, const void* v, void* out, float* S, float* Z, int B, int H,
+                     int d_k, int d_v, const kata_opts* opts) {
+  Opts o;
+  int st = read_opts(opts, o);
+  if (st != KATA_OK) return st;
+  if (B < 1 || H < 1 || d_k < 1 || d_v < 1) return KATA_ERR_INVALID_ARG;
+  if ((long long)B * H > 65535) return KATA_ERR_UNSUPPORTED_SHAPE;
+  if (!dim_ok(d_k) || !dim_ok(d_v)) return KATA_ERR_UNSUPPORTED_SHAPE;
+  if (o.s_pre != nullptr) return KATA_ERR_INVALID_ARG;
+  if (q == nullptr || k == nullptr || v == nullptr || out == nullptr || S == nullptr || Z == nullptr) return KATA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(S) || !aligned16(Z)) return KATA_ERR_ALIGNMENT;
+  const int n_psi = decode_n_psi(d_k, o.state_layout, o.feature_order);
+  const size_t need = align_up(decode_workspace_elems(B * H, n_psi, d_v) * sizeof(float));
+  if (o.workspace == nullptr || o.workspace_bytes < need) return KATA_ERR_WORKSPACE_TOO_SMALL;
+  if ((reinterpret_cast<uintptr_t>(o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;
+  st = check_arch();
+  if (st != KATA_OK) return st;
+  LaunchCtx ctx{o.stream, 0, KATA_OK};
+  decode_step(q, k, v, out, S, Z, static_cast<float*>(o.workspace), B * H, d_k, d_v, o.dtype, o.state_layout,
+              o.feature_order, ctx);
+  if (ctx.status == KATA_OK) {
+    g_last_launches = ctx.launches;
+    g_last_impl = KATA_IMPL_SIMT;
+  }
+  return ctx.status;
+}
+
 int kata_fwd_host(int fn, const void* q_host, const void* k_host, const void* v_host, void* out_host, int B,
                   int H, int T, int d_k, int d_v, int C, const kata_opts* opts) {
   Prepared r;
@@ -289,6 +316,11 @@ int kata_fwd_host(int fn, const void* q_host, const void* k_host, const void* v_
 size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts) {
   const bool host_io = (fn & KATA_FN_HOST_IO) != 0;
   fn &= ~KATA_FN_HOST_IO;
+  if (fn == KATA_FN_DECODE_STEP) {      // T and C are ignored
+    Opts o;
+    if (host_io || read_opts(opts, o) != KATA_OK || B < 1 || H < 1 || !dim_ok(d_k) || !dim_ok(d_v)) return 0;
+    return align_up(decode_workspace_elems(B * H, decode_n_psi(d_k, o.state_layout, o.feature_order), d_v) * sizeof(float));
+  }
   Prepared r;
   if (prepare(fn, nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, C, opts, false, r) != KATA_OK) return 0;
   if (!host_io) return r.inner_bytes;

@@ -114,3 +114,27 @@ def test_no_oracle_in_product_path():
                 text = open(os.path.join(dirpath, f)).read()
                 assert not re.search(r"^\s*(from|import)\s+\S*oracle", text, flags=re.M), f
                 assert "kata_oracle" not in text and "oracle/" not in text, f
+
+
+def test_decode_step_argument_checks(L):
+    INV, SHAPE, ALIGN, WS = -1, -2, -3, -4
+    def dec(q=4096, k=4096, v=4096, out=4096, S=4096, Z=4096, B=2, H=2, dk=64, dv=64, opts=None):
+        o = opts if opts is not None else kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 30)
+        return L.kata_decode_step(q, k, v, out, S, Z, B, H, dk, dv, ctypes.byref(o))
+
+    assert dec(q=0) == INV and dec(S=0) == INV and dec(Z=0) == INV and dec(B=0) == INV
+    assert dec(dk=48) == SHAPE and dec(dv=8) == SHAPE
+    assert dec(S=4100) == ALIGN and dec(out=4104) == ALIGN
+    assert dec(opts=kb.make_opts(kb.KATA_F32)) == WS                                     # needs a workspace
+    assert dec(opts=kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=64)) == WS
+    assert dec(opts=kb.make_opts(kb.KATA_F32, workspace=4096 + 8, workspace_bytes=1 << 30)) == ALIGN
+    assert dec(opts=kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 30, s_pre=4096, z_pre=8192)) == INV
+    # workspace: one partial numerator row and denominator per 256 feature rows of every head, rounded up to 256 B
+    up = lambda n: (n + 255) // 256 * 256
+    o = kb.make_opts(kb.KATA_BF16)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_DECODE_STEP, 2, 3, 1, 64, 64, 0, o) == up(2 * 3 * 16 * 65 * 4)
+    o = kb.make_opts(kb.KATA_BF16, state_layout=kb.KATA_LAYOUT_PACKED)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_DECODE_STEP, 2, 3, 1, 64, 32, 0, o) == up(2 * 3 * 9 * 33 * 4)
+    o = kb.make_opts(kb.KATA_F32, feature_order=1)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_DECODE_STEP, 1, 1, 1, 16, 16, 0, o) == 256   # 17 floats, rounded up
+    assert kb.decode_n_psi(64) == 4096 and kb.decode_n_psi(64, 2, kb.KATA_LAYOUT_PACKED) == 2080 and kb.decode_n_psi(64, 1) == 64
