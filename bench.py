@@ -312,6 +312,34 @@ def run_small(args):
                           impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")))
 
 
+def run_decode(args):
+    """Profiler case of the decode step: B=16, H=16, d=64, bf16 tokens, fp32 state (273 MB > L2); short line."""
+    import torch
+    from paper_2607_17419_b200 import binding as kb, build as kbuild
+    kbuild.build()
+    torch.cuda.set_device(0)
+    Bd, Hd, d = 16, 16, 64
+    g = torch.Generator(device="cpu").manual_seed(5)
+    qd, kd, vd = (torch.randn(Bd, Hd, d, generator=g).to(torch.bfloat16).cuda() for _ in range(3))
+    n_psi = kb.decode_n_psi(d)
+    S = torch.zeros(Bd, Hd, n_psi, d, device="cuda")
+    Z = torch.zeros(Bd, Hd, n_psi, device="cuda")
+    od = torch.empty_like(vd)
+    for _ in range(args.warmup):
+        kb.kata_decode_step(qd, kd, vd, S, Z, od)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        kb.kata_decode_step(qd, kd, vd, S, Z, od)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    nbytes = 2 * Bd * Hd * n_psi * (d + 1) * 4
+    print(json.dumps(dict(case="decode", heads=Bd * Hd, ms_per_step=ms, state_bytes_per_step=nbytes,
+                          gbs=nbytes / (ms * 1e-3) / 1e9)))
+
+
 def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
     """Separately timed secondary figures: scan forms on the same workload, quadratic form on config 2."""
     import numpy as np
@@ -369,11 +397,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="sequential", choices=["sequential", "scan"])
     ap.add_argument("--no-extra", dest="extra", action="store_false")
-    ap.add_argument("--case", default="full", choices=["full", "small"],
-                    help="small: the same kernel on T=32768 only (for profiler captures); prints a short line")
+    ap.add_argument("--case", default="full", choices=["full", "small", "decode"],
+                    help="small: the same kernel on T=32768 only; decode: the decode step only (both for profiler "
+                         "captures; they print a short line)")
     args = ap.parse_args()
     if args.case == "small":
         run_small(args)
+    elif args.case == "decode":
+        run_decode(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
