@@ -85,9 +85,12 @@ enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2,
  *                 the paper's per-chunk pipeline, whenever s_pre/z_pre are requested).
  *  workspace      device scratch of at least kata_workspace_bytes(...) bytes, 256-byte aligned;
  *                 may be null when that size is 0.
- *  s_pre, z_pre   optional device outputs of kata_chunk_state_scan (fp32):
- *                 s_pre [B,H,N_C,n_psi,d_v], z_pre [B,H,N_C,n_psi], N_C = ceil(T/C), the exclusive
- *                 prefix chunk states, entry 0 along N_C being zero.  Both null or both non-null.
+ *  s_pre, z_pre   optional device outputs (fp32), both null or both non-null.
+ *                 kata_chunk_state_scan: s_pre [B,H,N_C,n_psi,d_v], z_pre [B,H,N_C,n_psi], N_C = ceil(T/C),
+ *                 the exclusive prefix chunk states, entry 0 along N_C being zero.
+ *                 kata_fwd_chunked with inter_chunk = SEQUENTIAL (feature_order 2): s_pre [B,H,n_psi,d_v],
+ *                 z_pre [B,H,n_psi], the state after the last token -- the state kata_decode_step
+ *                 continues from (prefill -> decode).  Any other entry point: KATA_ERR_INVALID_ARG.
  *  device_status  optional device int, written only on a device-side timeout.
  *  stream         cudaStream_t as void* (null = the legacy default stream).
  */

@@ -178,7 +178,10 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   st = check_shape(fn, B, H, T, d_k, d_v, C);
   if (st != KATA_OK) return st;
   if (need_ptrs && (q == nullptr || k == nullptr || v == nullptr || out == nullptr)) return KATA_ERR_INVALID_ARG;
-  if (fn != KATA_FN_CHUNK_STATE_SCAN && r.o.s_pre != nullptr) return KATA_ERR_INVALID_ARG;
+  // s_pre/z_pre: prefix chunk states of the scan pipeline, or the final state of the sequential chunked forward
+  if (r.o.s_pre != nullptr && !(fn == KATA_FN_CHUNK_STATE_SCAN ||
+                                (fn == KATA_FN_CHUNKED && r.o.inter_chunk == KATA_SEQUENTIAL))) return KATA_ERR_INVALID_ARG;
+  if (r.o.s_pre != nullptr && fn == KATA_FN_CHUNKED && r.o.feature_order != 2) return KATA_ERR_UNSUPPORTED_SHAPE;
   r.p = Problem{q, k, v, out, B, H, T, d_k, d_v, r.o.dtype, r.o.feature_order};
   r.tensor = want_tensor(fn, r.p, r.o);
   if (r.o.impl == KATA_IMPL_TENSOR && !r.tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
@@ -186,10 +189,13 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   r.state_elems = 0;
   r.inner_bytes = (fn == KATA_FN_QUADRATIC && r.tensor) ? tc_quadratic_workspace_bytes(r.p) : 0;
   if (fn != KATA_FN_QUADRATIC) {
-    if (r.tensor && r.o.s_pre != nullptr) r.tensor = false;   // state export lives on the SIMT pipeline
+    if (r.tensor && r.o.s_pre != nullptr && fn == KATA_FN_CHUNK_STATE_SCAN) r.tensor = false;   // per-chunk export: SIMT pipeline
     st = make_plan(fn, r.p, r.o, r.tensor, r.plan, r.state_elems);
     if (st != KATA_OK) return st;
     r.inner_bytes = inner_workspace(fn, r.plan, r.p, r.state_elems);
+    // final-state export of the fp32 path goes through one internal state per head
+    if (fn == KATA_FN_CHUNKED && r.o.s_pre != nullptr && !r.tensor)
+      r.inner_bytes = align_up((size_t)B * H * r.state_elems * sizeof(float));
   }
   return KATA_OK;
 }
@@ -202,7 +208,7 @@ int run_device(int fn, Prepared& r, void* ws) {
     else simt_quadratic(r.p, ctx);
   } else {
     const bool use_scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || r.plan.n_groups > 1;
-    if (r.tensor) tc_chunked(r.p, r.plan, use_scan, wsf, r.o.device_status, ctx);
+    if (r.tensor) tc_chunked(r.p, r.plan, use_scan, wsf, r.o.device_status, r.o.s_pre, r.o.z_pre, r.o.state_layout, ctx);
     else if (r.p.feature_order == 1) order1_chunked(r.p, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, ctx);
     else simt_chunked(r.p, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, r.o.state_layout, ctx);
   }

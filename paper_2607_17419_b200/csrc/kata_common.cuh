@@ -85,9 +85,11 @@ bool tc_supported(const Problem& p, int fn, bool scan);
 size_t tc_quadratic_workspace_bytes(const Problem& p);
 void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx);
 void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx);
+void tc_chunked_stream_export(const Problem& p, int* device_status, float* s_final, float* z_final, int state_layout,
+                              LaunchCtx& ctx);
 size_t tc_chunked_state_elems();
 int tc_chunked_slices();
 void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, int* device_status,
-                LaunchCtx& ctx);
+                float* s_final, float* z_final, int state_layout, LaunchCtx& ctx);
 
 }  // namespace kata

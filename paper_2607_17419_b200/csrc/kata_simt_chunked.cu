@@ -354,6 +354,44 @@ __global__ void export_states_kernel(const float* __restrict__ incl, float* __re
   }
 }
 
+// State after the last token in the public layouts, from the internal state [BH][NSLICE][slot] of a
+// whole-sequence pass.
+template <int D, int DV>
+__global__ void export_final_kernel(const float* __restrict__ fin, float* __restrict__ s_out, float* __restrict__ z_out,
+                                    int layout) {
+  using G = Cfg<D, DV>;
+  constexpr int BLK = G::BLK, VS = G::VS;
+  const size_t bh = blockIdx.y;
+  const int n_psi = (layout == KATA_LAYOUT_PACKED) ? D * (D + 1) / 2 : D * D;
+  const size_t slot = (size_t)G::NREG * NTHR;
+  float* sp = s_out + bh * (size_t)n_psi * DV;
+  float* zp = z_out + bh * (size_t)n_psi;
+  for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < n_psi * (DV + 1); item += gridDim.x * blockDim.x) {
+    const int row = item / (DV + 1), col = item % (DV + 1);
+    int a, b;
+    float scale = 1.f;
+    if (layout == KATA_LAYOUT_PACKED) {
+      a = 0;
+      int r = row;
+      while (r >= D - a) { r -= D - a; ++a; }
+      b = a + r;
+      if (a != b) scale = 1.41421356237309504880f;
+    } else {
+      a = row / D;
+      b = row % D;
+    }
+    const int lo = min(a, b), hi = max(a, b);
+    const int Ab = lo / BLK, Bb = hi / BLK, i = lo % BLK, j = hi % BLK;
+    const int tid = Ab * NB - Ab * (Ab - 1) / 2 + (Bb - Ab);
+    const int slice = (col < DV) ? col / VS : 0;
+    const int cc = (col < DV) ? col % VS : VS;
+    const float* src = fin + (bh * G::NSLICE + slice) * slot;
+    const float val = scale * src[(size_t)((i * BLK + j) * (VS + 1) + cc) * NTHR + tid];
+    if (col < DV) sp[(size_t)row * DV + col] = val;
+    else zp[row] = val;
+  }
+}
+
 template <typename T, int D, int DV>
 void run(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre, float* z_pre,
          int state_layout, LaunchCtx& ctx) {
@@ -371,9 +409,15 @@ void run(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float
   T* o = static_cast<T*>(p.out);
   const int BH = p.B * p.H;
   if (!use_scan) {
+    // whole sequence in one pass; with s_pre/z_pre the state after the last token is exported
+    float* fin = (s_pre != nullptr) ? ws : nullptr;
     kern<<<dim3(G::NSLICE, BH, 1), NTHR, smem, ctx.stream>>>(q, k, v, o, p.T, plan.n_chunks, plan.n_chunks,
-                                                            1, nullptr, nullptr, 1);
+                                                            1, nullptr, fin, 1);
     note_launch(ctx);
+    if (fin != nullptr) {
+      export_final_kernel<D, DV><<<dim3(16, BH), 256, 0, ctx.stream>>>(fin, s_pre, z_pre, state_layout);
+      note_launch(ctx);
+    }
     return;
   }
   const int NG = plan.n_groups;

@@ -712,9 +712,10 @@ size_t tc_chunked_state_elems() { return (size_t)NSLICE * STATE_PER_SLICE; }
 int tc_chunked_slices() { return NSLICE; }
 
 void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, int* device_status,
-                LaunchCtx& ctx) {
+                float* s_final, float* z_final, int state_layout, LaunchCtx& ctx) {
   if (!use_scan) {   // whole sequence in one pass: the token-major streaming kernel
-    tc_chunked_stream(p, device_status, ctx);
+    if (s_final != nullptr) tc_chunked_stream_export(p, device_status, s_final, z_final, state_layout, ctx);
+    else tc_chunked_stream(p, device_status, ctx);
     return;
   }
   const int BH = p.B * p.H;

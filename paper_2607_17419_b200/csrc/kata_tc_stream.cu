@@ -17,6 +17,8 @@
 //   intra    P = (Q K^T)^2 masked causally, [O | D] += P [V' | 1/||k||^2]   as in the quadratic form
 //   out      (N_inter + O) / (D_inter + D)             (0 where the denominator is 0)
 // The query norm cancels and is never applied.
+// Compiled a second time with KATA_STREAM_EXPORT (kata_tc_stream_export.cu): the same kernel plus the export of
+// the state after the last token; kept as a separate build so that the plain kernel's code stays as it is.
 //
 // Warps (768 threads, 80 registers each): 0 TMA producer and update-MMA issuer (b-block 3, Z); 1 update-MMA
 // issuer (b-blocks 0-2); 2 read-MMA issuer; 3 intra-tile MMA issuer; 4-11 W builders in two teams (even / odd
@@ -102,6 +104,11 @@ struct SArgs {
   __nv_bfloat16* out;
   int* device_status;
   int Tlen;
+#ifdef KATA_STREAM_EXPORT
+  int layout;          // KATA_LAYOUT_DIRECT / KATA_LAYOUT_PACKED
+  float* s_final;      // state after the last token, [BH][n_psi][64] in the public layout
+  float* z_final;      // [BH][n_psi]
+#endif
 };
 
 __device__ __noinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -148,6 +155,62 @@ __device__ __forceinline__ void snap_store16(unsigned char* row, uint32_t c, uin
 // Pieces of the b-blocks 0 and 2 share rows (32 + 96 bytes), the two pieces of b-block 1 share rows (64 + 64).
 __device__ __forceinline__ uint32_t sp_block(int p) { return (0x43102210u >> (4 * p)) & 0xFu; }   // 0,1,2,2,0,1,3,4
 __device__ __forceinline__ uint32_t sp_koff(int p) { return p == 3 ? 64u : (p == 4 || p == 5) ? 32u : 0u; }
+
+#ifdef KATA_STREAM_EXPORT
+// The state after the last token, from the TMEM accumulators to the public layout (one call per thread of the
+// four auxiliary warps; kept out of line so that it does not weigh on the register allocation of the main loop).
+__device__ __noinline__ void export_state(uint32_t tb, uint32_t q4, int t, float* s_final, float* z_final, int layout,
+                                          int bh, int v0, int slice) {
+  tc_fence_after();
+  const bool packed = layout == KATA_LAYOUT_PACKED;
+  const int n_psi = packed ? D * (D + 1) / 2 : D * D;
+  float* sf = s_final + (size_t)bh * n_psi * D + v0;
+  auto prow = [&](int a, int b) { return a * D - a * (a - 1) / 2 + (b - a); };   // packed row of a <= b
+  const int vv = t & 7;
+  uint32_t scol = tmem_addr(tb, q4 * 32, COL_S);
+#pragma unroll 1
+  for (int be = 0; be < 4; ++be) {
+    const int b = 16 * be + (t >> 3);
+#pragma unroll 1
+    for (int al = 0; al <= be; ++al, scol += 16) {
+      uint32_t z[16];
+      tmem_ld16(scol, z);
+      tmem_wait_ld(z);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int a = 16 * al + i;
+        const float val = __uint_as_float(z[i]);
+        if (packed) {
+          if (a <= b) sf[(size_t)prow(a, b) * D + vv] = (a == b) ? val : val * 1.41421356237309504880f;
+        } else {
+          sf[(size_t)(a * D + b) * D + vv] = val;
+          if (al < be) sf[(size_t)(b * D + a) * D + vv] = val;     // the dropped half of the symmetric state
+        }
+      }
+    }
+  }
+  if (slice == 0 && q4 < 2) {
+    float* zf = z_final + (size_t)bh * n_psi;
+    const int b = t;
+#pragma unroll 1
+    for (int al = 0; al < 4; ++al) {
+      uint32_t z[16];
+      tmem_ld16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
+      tmem_wait_ld(z);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int a = 16 * al + i;
+        const float val = __uint_as_float(z[i]);
+        if (packed) {
+          if (a <= b) zf[prow(a, b)] = (a == b) ? val : val * 1.41421356237309504880f;
+        } else {
+          zf[a * D + b] = val;
+        }
+      }
+    }
+  }
+}
+#endif
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const SArgs args) {
@@ -698,6 +761,13 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         mbar_arrive(bar(BAR_QT_FULL));
       }
     }
+#ifdef KATA_STREAM_EXPORT
+    // ---- the state after the last token, from the accumulators to the public layout ----
+    if (ok) {
+      ok = wait_or_abort(bar(BAR_U_DONE), (nch - 1) & 1, abort_flag);
+      if (ok) export_state(tb, q4, t, args.s_final, args.z_final, args.layout, bh, v0, slice);
+    }
+#endif
   }
 
   // ---------------- teardown ----------------
@@ -748,7 +818,12 @@ bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T) {
 
 }  // namespace
 
+#ifdef KATA_STREAM_EXPORT
+void tc_chunked_stream_export(const Problem& p, int* device_status, float* s_final, float* z_final, int state_layout,
+                              LaunchCtx& ctx) {
+#else
 void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
+#endif
   const int BH = p.B * p.H;
   CUtensorMap tmQ, tmK;
   if (!make_map(&tmQ, p.q, BH, p.T) || !make_map(&tmK, p.k, BH, p.T)) {
@@ -760,7 +835,12 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }
+#ifdef KATA_STREAM_EXPORT
+  SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T, state_layout,
+          s_final, z_final};
+#else
   SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T};
+#endif
   tc_stream_kernel<<<dim3(NSLICE, BH, 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, a);
   note_launch(ctx);
 }

@@ -77,6 +77,12 @@ def test_invalid_arguments(L, fn):
         assert call(L, fn, T=640, opts=o) == ALIGN
         o = kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192, scan_group=4)
         assert call(L, fn, T=640, opts=o) == INV
+    elif fn == "kata_fwd_chunked":
+        # final-state export: sequential form and the PSD feature only
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192, inter_chunk=kb.KATA_SCAN)) == INV
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192, feature_order=1)) == SHAPE
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096)) == INV
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192)) == WS          # fp32 path: one internal state per head
     else:
         assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192)) == INV
 

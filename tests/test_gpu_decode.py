@@ -95,3 +95,39 @@ def test_decode_zero_rows_and_determinism():
     oa, ob = kb.kata_decode_step(q, k, v, Sa, Za), kb.kata_decode_step(q, k, v, Sb, Zb)
     torch.cuda.synchronize()
     assert torch.equal(oa, ob) and torch.equal(Sa, Sb) and torch.equal(Za, Zb)
+
+
+@pytest.mark.parametrize("dtype,impl", [("f32", "simt"), ("bf16", "tensor"), ("bf16", "simt")])
+@pytest.mark.parametrize("layout", ["psd_direct", "psd_packed"])
+def test_final_state_of_the_chunked_forward(dtype, impl, layout):
+    """kata_fwd_chunked (sequential) exports the state after the last token; decoding on from it gives the
+    forward pass over the longer sequence."""
+    import torch
+    B, H, T, Tp, d = 1, 2, 300, 270, 64           # prefill 270 tokens (ragged: 2 tiles + 14), decode 30 more
+    w = inputs.gaussian_workload("prefill", dtype, B, H, T, d, d, 64, 91)
+    q, k, v = dev_tensors(w)
+    n = kb.decode_n_psi(d, **FEATURES[layout])
+    S = torch.full((B, H, n, d), float("nan"), device="cuda")
+    Z = torch.full((B, H, n), float("nan"), device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    o = kb.kata_fwd_chunked(q[:, :, :Tp].contiguous(), k[:, :, :Tp].contiguous(), v[:, :, :Tp].contiguous(),
+                            s_pre=S, z_pre=Z, state_layout=FEATURES[layout]["state_layout"], device_status=st,
+                            impl=kb.KATA_IMPL_SIMT if impl == "simt" else kb.KATA_IMPL_TENSOR)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    assert (kb.kata_last_impl() == kb.KATA_IMPL_TENSOR) == (impl == "tensor")
+    g_pre = to_numpy64(o)
+    # bf16 W rows on the tensor path: the state carries the rounding of the per-token products
+    tol_state = 1e-4 if dtype == "f32" else 1e-2
+    for h in range(H):
+        ref = ko.kata_quadratic(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h])[0]
+        check(g_pre[0, h], ref[:Tp], dtype, f"prefill {impl}/{layout}")
+        fk = ko.apply_feature(w.k_ref[0, h, :Tp], layout)
+        Sr, Zr = fk.T @ w.v_ref[0, h, :Tp], fk.sum(axis=0)
+        assert np.all(np.isfinite(to_numpy64(S[0, h]))) and np.all(np.isfinite(to_numpy64(Z[0, h])))
+        assert np.max(np.abs(to_numpy64(S[0, h]) - Sr)) <= tol_state * max(1.0, np.abs(Sr).max())
+        assert np.max(np.abs(to_numpy64(Z[0, h]) - Zr)) <= tol_state * max(1.0, np.abs(Zr).max())
+    g = decode_all(q, k, v, S, Z, Tp, T, **FEATURES[layout])
+    for h in range(H):
+        ref = ko.kata_quadratic(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h])[0]
+        check(g[0, h], ref[Tp:], dtype, f"decode after prefill {impl}/{layout}")
