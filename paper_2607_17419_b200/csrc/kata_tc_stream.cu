@@ -111,15 +111,30 @@ struct SArgs {
 #endif
 };
 
-__device__ __noinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    __nanosleep(64);
-
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
+// Bounded wait, as few instructions per poll as possible (24 warps poll most of the time and share the issue
+// slots with the warps that work): try_wait, exit branch, counter, loop branch.  A wait that gives up raises the
+// abort flag; the other waiters give up on their own limits.
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u32 i;\n\t"
+      "mov.u32 i, 0;\n\t"
+      "KATA_WAIT_%=:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra KATA_DONE_%=;\n\t"
+      "add.u32 i, i, 1;\n\t"
+      "setp.lt.u32 q, i, %3;\n\t"
+      "@q bra KATA_WAIT_%=;\n\t"
+      "KATA_DONE_%=:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSpinLimit)
+      : "memory");
+  if (ok == 0) *abort_flag = 1;
+  return ok != 0;
 }
 
 __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
