@@ -119,13 +119,30 @@ __device__ __forceinline__ void reader_sync() { asm volatile("bar.sync 3, 256;" 
 __device__ __forceinline__ void group_pair_sync(uint32_t q) { asm volatile("bar.sync %0, 64;" ::"r"(4 + q) : "memory"); }
 
 // Bounded wait that also gives up as soon as another role has flagged an abort.
+// Bounded wait, as few instructions per poll as possible (the polling warps share the issue slots with the warps
+// that work): try_wait, exit branch, counter, loop branch.  A wait that gives up raises the abort flag; the other
+// waiters give up on their own limits.
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u32 i;\n\t"
+      "mov.u32 i, 0;\n\t"
+      "KATA_WAIT_%=:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra KATA_DONE_%=;\n\t"
+      "add.u32 i, i, 1;\n\t"
+      "setp.lt.u32 q, i, %3;\n\t"
+      "@q bra KATA_WAIT_%=;\n\t"
+      "KATA_DONE_%=:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSpinLimit)
+      : "memory");
+  if (ok == 0) *abort_flag = 1;
+  return ok != 0;
 }
 
 // element-wise product of two packed bf16 pairs (one HMUL2.BF16)
