@@ -79,25 +79,48 @@ def psi_packed(u: np.ndarray) -> np.ndarray:
     return u[..., a] * u[..., b] * scale
 
 
+def split_feature(feature: str):
+    """'psd_direct', 'psd_packed', 'identity', or a PSD name with a block suffix ':g2' / ':g4' (KATA-Mg).
+
+    Returns (base name, g)."""
+    base, _, suf = feature.partition(":")
+    g = 1
+    if suf:
+        if not (suf.startswith("g") and suf[1:].isdigit()):
+            raise ValueError(feature)
+        g = int(suf[1:])
+    if base not in FEATURES or (g != 1 and base == "identity") or g < 1:
+        raise ValueError(feature)
+    return base, g
+
+
 def feature_dim(d: int, feature: str) -> int:
-    if feature == "psd_direct":
-        return d * d
-    if feature == "psd_packed":
-        return d * (d + 1) // 2
-    if feature == "identity":
-        return d
-    raise ValueError(feature)
+    base, g = split_feature(feature)
+    if d % g != 0:
+        raise ValueError(f"d={d} is not divisible by g={g}")
+    m = d // g
+    if base == "psd_direct":
+        return g * m * m
+    if base == "psd_packed":
+        return g * (m * (m + 1) // 2)
+    return d
 
 
 def apply_feature(x: np.ndarray, feature: str) -> np.ndarray:
-    """Row-wise Psi(X) for one of FEATURES."""
-    if feature == "psd_direct":
-        return psi_direct(normalize_rows(x))
-    if feature == "psd_packed":
-        return psi_packed(normalize_rows(x))
-    if feature == "identity":
+    """Row-wise Psi(X).  PSD features: the row is l2-normalised, then lifted; with a ':g' suffix the
+    normalised row is cut into g blocks of d/g entries and each block is lifted on its own (the blockwise PSD
+    map psi_Mg(u) = (u_1 u_1^T, ..., u_g u_g^T), whose inner product is sum_a (q_a . k_a)^2), blocks
+    concatenated in order."""
+    base, g = split_feature(feature)
+    if base == "identity":
         return np.asarray(x, dtype=np.float64)
-    raise ValueError(feature)
+    u = normalize_rows(x)
+    d = u.shape[-1]
+    if d % g != 0:
+        raise ValueError(f"d={d} is not divisible by g={g}")
+    m = d // g
+    lift = psi_direct if base == "psd_direct" else psi_packed
+    return np.concatenate([lift(u[..., a * m:(a + 1) * m]) for a in range(g)], axis=-1)
 
 
 def _safe_div(n: np.ndarray, d: np.ndarray) -> np.ndarray:
@@ -111,12 +134,28 @@ def _safe_div(n: np.ndarray, d: np.ndarray) -> np.ndarray:
 # form Q: the definition
 # ---------------------------------------------------------------------------
 
+def _block_kernel(qh: np.ndarray, kh: np.ndarray, g: int) -> np.ndarray:
+    """sum over the g blocks of (q_a . k_a)^2 for normalised rows qh [Tq,d], kh [Tk,d]  ->  [Tq,Tk].
+
+    g = 1 is the full rank-one lift (q_hat . k_hat)^2; g > 1 the blockwise PSD map of KATA-Mg."""
+    d = qh.shape[-1]
+    if d % g != 0:
+        raise ValueError(f"d={d} is not divisible by g={g}")
+    m = d // g
+    out = np.zeros((qh.shape[0], kh.shape[0]))
+    for a in range(g):
+        out += (qh[:, a * m:(a + 1) * m] @ kh[:, a * m:(a + 1) * m].T) ** 2
+    return out
+
+
 def causal_weights(q: np.ndarray, k: np.ndarray, feature: str = "psd_direct") -> np.ndarray:
-    """w[t,i] = <psi(q_t), psi(k_i)> for i<=t, else 0.  [T,T]."""
-    if feature == "identity":
+    """w[t,i] = <psi(q_t), psi(k_i)> for i<=t, else 0, from the closed form of the inner product
+    (dot products of the rows, never the lifted features).  [T,T]."""
+    base, g = split_feature(feature)
+    if base == "identity":
         s = np.asarray(q, np.float64) @ np.asarray(k, np.float64).T
     else:
-        s = (normalize_rows(q) @ normalize_rows(k).T) ** 2
+        s = _block_kernel(normalize_rows(q), normalize_rows(k), g)
     return np.tril(s)
 
 
@@ -135,11 +174,13 @@ def kata_rows(q, k, v, rows, feature: str = "psd_direct") -> np.ndarray:
     k = np.asarray(k, np.float64)
     v = np.asarray(v, np.float64)
     out = np.zeros((len(rows), v.shape[1]))
-    kh = k if feature == "identity" else normalize_rows(k)
+    base, g = split_feature(feature)
+    kh = k if base == "identity" else normalize_rows(k)
     for j, t in enumerate(rows):
-        qt = q[t] if feature == "identity" else normalize_rows(q[t][None])[0]
-        s = kh[: t + 1] @ qt
-        w = s if feature == "identity" else s * s
+        if base == "identity":
+            w = kh[: t + 1] @ q[t]
+        else:
+            w = _block_kernel(normalize_rows(q[t][None]), kh[: t + 1], g)[0]
         D = w.sum()
         if D != 0:
             out[j] = (w @ v[: t + 1]) / D

@@ -406,3 +406,72 @@ def test_decode_step_special_cases():
     for t in range(8, 12):
         o, S, Z = ko.kata_decode_step(S, Z, q[t], k[t], v[t])
         assert np.allclose(o, full[t], atol=1e-12)
+
+
+# ---------------------------------------------------------------------------
+# blockwise PSD map (KATA-Mg)
+# ---------------------------------------------------------------------------
+
+def brute_mg(q, k, v, g):
+    """Definition with the blockwise kernel sum_a (q_hat_a . k_hat_a)^2, plain Python loops."""
+    T, d, dv = len(q), len(q[0]), len(v[0])
+    m = d // g
+
+    def unit(x):
+        n = math.sqrt(sum(t * t for t in x))
+        return [t / n for t in x] if n > 0 else [0.0] * len(x)
+
+    qh, kh = [unit(r) for r in q], [unit(r) for r in k]
+    out = []
+    for t in range(T):
+        num, den = [0.0] * dv, 0.0
+        for i in range(t + 1):
+            w = 0.0
+            for a in range(g):
+                dot = sum(qh[t][a * m + e] * kh[i][a * m + e] for e in range(m))
+                w += dot * dot
+            den += w
+            for c in range(dv):
+                num[c] += w * v[i][c]
+        out.append([x / den if den != 0 else 0.0 for x in num])
+    return np.array(out)
+
+
+@pytest.mark.parametrize("g", [1, 2, 4])
+def test_blockwise_feature_against_brute_force(g):
+    q, k, v = rand_qkv(60 + g, 9, 4, 3)
+    ref = brute_mg(q.tolist(), k.tolist(), v.tolist(), g)
+    if g == 1:
+        assert np.allclose(ref, brute(q.tolist(), k.tolist(), v.tolist()), atol=1e-14)
+    for base in ("psd_direct", "psd_packed"):
+        f = f"{base}:g{g}"
+        assert np.allclose(ko.kata_quadratic(q, k, v, f)[0], ref, atol=1e-13)
+        assert np.allclose(ko.kata_recurrent(q, k, v, f), ref, atol=1e-13)
+        assert np.allclose(ko.kata_chunked(q, k, v, 4, f), ref, atol=1e-13)
+        assert np.allclose(ko.kata_scan(q, k, v, 4, f)[0], ref, atol=1e-13)
+    # g = 1 with the suffix is the plain feature
+    assert np.array_equal(ko.apply_feature(q, "psd_direct:g1"), ko.apply_feature(q, "psd_direct"))
+
+
+def test_blockwise_feature_sizes_and_kernel():
+    # state entries d (d/g + 1) / 2 * d_v: the paper's 266,240 (M1) and 135,168 (M2) at d = 64, d_v = 128
+    assert ko.feature_dim(64, "psd_packed") * 128 == 266240
+    assert ko.feature_dim(64, "psd_packed:g2") * 128 == 135168
+    assert ko.feature_dim(64, "psd_direct:g4") == 4 * 16 * 16
+    # kernel identity <psi(q), psi(k)> = sum_a (q_a . k_a)^2 on the normalised rows, both packings
+    r = rng(71)
+    q, k = r.standard_normal((5, 8)), r.standard_normal((6, 8))
+    qh, kh = ko.normalize_rows(q), ko.normalize_rows(k)
+    for g in (2, 4):
+        m = 8 // g
+        want = sum((qh[:, a * m:(a + 1) * m] @ kh[:, a * m:(a + 1) * m].T) ** 2 for a in range(g))
+        for base in ("psd_direct", "psd_packed"):
+            got = ko.apply_feature(q, f"{base}:g{g}") @ ko.apply_feature(k, f"{base}:g{g}").T
+            assert np.allclose(got, want, atol=1e-14)
+    # g = d: every block is one coordinate, the kernel is sum_a q_a^2 k_a^2
+    got = ko.apply_feature(q, "psd_direct:g8") @ ko.apply_feature(k, "psd_direct:g8").T
+    assert np.allclose(got, (qh ** 2) @ (kh ** 2).T, atol=1e-14)
+    with pytest.raises(ValueError):
+        ko.apply_feature(q, "psd_direct:g3")
+    with pytest.raises(ValueError):
+        ko.apply_feature(q, "identity:g2")
