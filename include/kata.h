@@ -69,6 +69,11 @@ enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2,
  *                 1: rows of q,k are already-mapped features used as they are (no
  *                    normalisation, no lift; state d_k x d_v) -- the setting of the paper's
  *                    associative-scan appendix ("already-feature-mapped inputs").
+ *  feature_groups 0 or 1: the full rank-one lift.  g = 2 or 4 (feature_order 2 only): the blockwise PSD map
+ *                 psi_Mg(u) = (u_1 u_1^T, ..., u_g u_g^T) of the normalised row cut into g blocks of d_k/g
+ *                 entries ("KATA-Mg"), with <psi(q),psi(k)> = sum_a (q_a . k_a)^2.  The state layouts then hold
+ *                 the g blocks one after the other: DIRECT n_psi = g (d_k/g)^2, PACKED n_psi = g m(m+1)/2 with
+ *                 m = d_k/g.  Runs on the fp32 kernels.
  *  state_layout   layout of the exported prefix states for feature_order 2:
  *                 DIRECT  n_psi = d_k^2, row a*d_k+b holds the (a,b) entry of sum k_hat k_hat^T (x) v;
  *                 PACKED  n_psi = d_k(d_k+1)/2, upper triangle a<=b in row-major order, diagonal
@@ -102,7 +107,7 @@ typedef struct kata_opts {
   int32_t inter_chunk;
   int32_t impl;
   int32_t scan_group;
-  int32_t reserved0;
+  int32_t feature_groups;
   void* workspace;
   size_t workspace_bytes;
   float* s_pre;

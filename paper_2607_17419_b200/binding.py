@@ -37,7 +37,7 @@ class KataOpts(ctypes.Structure):
         ("inter_chunk", ctypes.c_int32),
         ("impl", ctypes.c_int32),
         ("scan_group", ctypes.c_int32),
-        ("reserved0", ctypes.c_int32),
+        ("feature_groups", ctypes.c_int32),
         ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t),
         ("s_pre", ctypes.c_void_p),
@@ -95,12 +95,14 @@ def status_string(status: int) -> str:
 
 def make_opts(dtype: int, *, feature_order: int = 2, state_layout: int = KATA_LAYOUT_DIRECT,
               inter_chunk: int = KATA_SEQUENTIAL, impl: int = KATA_IMPL_AUTO, scan_group: int = 0,
+              feature_groups: int = 0,
               workspace: int = 0, workspace_bytes: int = 0, s_pre: int = 0, z_pre: int = 0,
               device_status: int = 0, stream: int = 0) -> KataOpts:
     o = KataOpts()
     o.struct_size = ctypes.sizeof(KataOpts)
     o.dtype, o.feature_order, o.state_layout = dtype, feature_order, state_layout
     o.inter_chunk, o.impl, o.scan_group = inter_chunk, impl, scan_group
+    o.feature_groups = feature_groups
     o.workspace, o.workspace_bytes = workspace or None, workspace_bytes
     o.s_pre, o.z_pre = s_pre or None, z_pre or None
     o.device_status, o.stream = device_status or None, stream or None
@@ -220,11 +222,14 @@ def kata_fwd_host(fn: int, q, k, v, out, C: int = 64, **kw):
     return _call(fn, q, k, v, out, C, host_io=True, **kw)
 
 
-def decode_n_psi(d_k: int, feature_order: int = 2, state_layout: int = KATA_LAYOUT_DIRECT) -> int:
-    """Feature rows of the decode state: d_k (order 1), d_k^2 (direct) or d_k(d_k+1)/2 (packed)."""
+def decode_n_psi(d_k: int, feature_order: int = 2, state_layout: int = KATA_LAYOUT_DIRECT, feature_groups: int = 0) -> int:
+    """Feature rows of the state: d_k (order 1); g m^2 (direct) or g m(m+1)/2 (packed) with m = d_k / g for the
+    PSD lift in g blocks (g = 1: the full lift)."""
     if feature_order == 1:
         return d_k
-    return d_k * (d_k + 1) // 2 if state_layout == KATA_LAYOUT_PACKED else d_k * d_k
+    g = max(1, feature_groups)
+    m = d_k // g
+    return g * (m * (m + 1) // 2 if state_layout == KATA_LAYOUT_PACKED else m * m)
 
 
 def kata_decode_step(q, k, v, S, Z, out=None, *, workspace: Optional[Workspace] = None, stream=None, **opt_kw):
@@ -242,7 +247,7 @@ def kata_decode_step(q, k, v, S, Z, out=None, *, workspace: Optional[Workspace] 
     if stream is None:
         stream = torch.cuda.current_stream(q.device).cuda_stream
     opts = make_opts(_dtype_code(q), stream=stream, **opt_kw)
-    n_psi = decode_n_psi(d_k, opts.feature_order, opts.state_layout)
+    n_psi = decode_n_psi(d_k, opts.feature_order, opts.state_layout, opts.feature_groups)
     if tuple(S.shape) != (B, H, n_psi, d_v) or tuple(Z.shape) != (B, H, n_psi):
         raise ValueError(f"state shapes must be {(B, H, n_psi, d_v)} and {(B, H, n_psi)}")
     need = kata_workspace_bytes(KATA_FN_DECODE_STEP, B, H, 1, d_k, d_v, 0, opts)

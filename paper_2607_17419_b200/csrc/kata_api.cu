@@ -22,7 +22,7 @@ inline int ceil_log2(int n) {
 }
 
 struct Opts {
-  int dtype, feature_order, state_layout, inter_chunk, impl, scan_group;
+  int dtype, feature_order, state_layout, inter_chunk, impl, scan_group, groups;
   void* workspace;
   size_t workspace_bytes;
   float* s_pre;
@@ -39,6 +39,7 @@ int read_opts(const kata_opts* o, Opts& out) {
   out.inter_chunk = o->inter_chunk;
   out.impl = o->impl;
   out.scan_group = o->scan_group;
+  out.groups = o->feature_groups == 0 ? 1 : o->feature_groups;
   out.workspace = o->workspace;
   out.workspace_bytes = o->workspace_bytes;
   out.s_pre = o->s_pre;
@@ -51,6 +52,8 @@ int read_opts(const kata_opts* o, Opts& out) {
   if (out.inter_chunk != KATA_SEQUENTIAL && out.inter_chunk != KATA_SCAN) return KATA_ERR_INVALID_ARG;
   if (out.impl < KATA_IMPL_AUTO || out.impl > KATA_IMPL_TENSOR) return KATA_ERR_INVALID_ARG;
   if (out.scan_group < 0) return KATA_ERR_INVALID_ARG;
+  if (out.groups != 1 && out.groups != 2 && out.groups != 4) return KATA_ERR_INVALID_ARG;
+  if (out.groups != 1 && out.feature_order != 2) return KATA_ERR_INVALID_ARG;
   if ((out.s_pre == nullptr) != (out.z_pre == nullptr)) return KATA_ERR_INVALID_ARG;
   return KATA_OK;
 }
@@ -182,7 +185,7 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   if (r.o.s_pre != nullptr && !(fn == KATA_FN_CHUNK_STATE_SCAN ||
                                 (fn == KATA_FN_CHUNKED && r.o.inter_chunk == KATA_SEQUENTIAL))) return KATA_ERR_INVALID_ARG;
   if (r.o.s_pre != nullptr && fn == KATA_FN_CHUNKED && r.o.feature_order != 2) return KATA_ERR_UNSUPPORTED_SHAPE;
-  r.p = Problem{q, k, v, out, B, H, T, d_k, d_v, r.o.dtype, r.o.feature_order};
+  r.p = Problem{q, k, v, out, B, H, T, d_k, d_v, r.o.dtype, r.o.feature_order, r.o.groups};
   r.tensor = want_tensor(fn, r.p, r.o);
   if (r.o.impl == KATA_IMPL_TENSOR && !r.tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
   r.plan = ScanPlan{(T + kChunk - 1) / kChunk, 0, 1, 0};
@@ -268,7 +271,7 @@ int kata_decode_step(const void* q, const void* k, const void* v, void* out, flo
   if (o.s_pre != nullptr) return KATA_ERR_INVALID_ARG;
   if (q == nullptr || k == nullptr || v == nullptr || out == nullptr || S == nullptr || Z == nullptr) return KATA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(S) || !aligned16(Z)) return KATA_ERR_ALIGNMENT;
-  const int n_psi = decode_n_psi(d_k, o.state_layout, o.feature_order);
+  const int n_psi = decode_n_psi(d_k, o.state_layout, o.feature_order, o.groups);
   const size_t need = align_up(decode_workspace_elems(B * H, n_psi, d_v) * sizeof(float));
   if (o.workspace == nullptr || o.workspace_bytes < need) return KATA_ERR_WORKSPACE_TOO_SMALL;
   if ((reinterpret_cast<uintptr_t>(o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;
@@ -276,7 +279,7 @@ int kata_decode_step(const void* q, const void* k, const void* v, void* out, flo
   if (st != KATA_OK) return st;
   LaunchCtx ctx{o.stream, 0, KATA_OK};
   decode_step(q, k, v, out, S, Z, static_cast<float*>(o.workspace), B * H, d_k, d_v, o.dtype, o.state_layout,
-              o.feature_order, ctx);
+              o.feature_order, o.groups, ctx);
   if (ctx.status == KATA_OK) {
     g_last_launches = ctx.launches;
     g_last_impl = KATA_IMPL_SIMT;
@@ -325,7 +328,7 @@ size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C
   if (fn == KATA_FN_DECODE_STEP) {      // T and C are ignored
     Opts o;
     if (host_io || read_opts(opts, o) != KATA_OK || B < 1 || H < 1 || !dim_ok(d_k) || !dim_ok(d_v)) return 0;
-    return align_up(decode_workspace_elems(B * H, decode_n_psi(d_k, o.state_layout, o.feature_order), d_v) * sizeof(float));
+    return align_up(decode_workspace_elems(B * H, decode_n_psi(d_k, o.state_layout, o.feature_order, o.groups), d_v) * sizeof(float));
   }
   Prepared r;
   if (prepare(fn, nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, C, opts, false, r) != KATA_OK) return 0;

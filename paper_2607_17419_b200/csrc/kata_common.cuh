@@ -47,6 +47,7 @@ struct Problem {
   int B, H, T, d_k, d_v;
   int dtype;
   int feature_order;
+  int groups;            // blocks of the blockwise PSD map (1 = full lift)
 };
 
 // Scan/group plan of the chunked forms.
@@ -74,11 +75,11 @@ void order1_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float
                     float* z_pre, LaunchCtx& ctx);
 
 // Decode step (fp32 state in the exported layout; any supported shape and element type)
-int decode_n_psi(int d_k, int layout, int order);
+int decode_n_psi(int d_k, int layout, int order, int groups);
 int decode_slabs(int n_psi);
 size_t decode_workspace_elems(int BH, int n_psi, int d_v);
 void decode_step(const void* q, const void* k, const void* v, void* out, float* S, float* Z, float* part, int BH,
-                 int d_k, int d_v, int dtype, int layout, int order, LaunchCtx& ctx);
+                 int d_k, int d_v, int dtype, int layout, int order, int groups, LaunchCtx& ctx);
 
 // Tensor-core kernels (tcgen05/TMEM; bf16, d_k = d_v = 64)
 bool tc_supported(const Problem& p, int fn, bool scan);

@@ -18,29 +18,38 @@ namespace {
 constexpr int DEC_THREADS = 256;
 constexpr int DEC_ROWS = 256;     // feature rows per CTA
 
-// feature pair (a,b) and scale of row r
-__device__ __forceinline__ void feature_pair(int r, int d, int layout, int order, int& a, int& b, float& scale) {
+// feature pair (a,b) and scale of row r.  With g feature blocks (blockwise PSD map) the rows of the blocks follow
+// one another and (a,b) stay inside one block of m = d / g features.
+__device__ __forceinline__ void feature_pair(int r, int d, int layout, int order, int groups, int& a, int& b, float& scale) {
   if (order == 1) {
     a = r; b = -1; scale = 1.f;
-  } else if (layout == KATA_LAYOUT_DIRECT) {
-    a = r / d; b = r - a * d; scale = 1.f;
+    return;
+  }
+  const int m = d / groups;
+  const int per = (layout == KATA_LAYOUT_PACKED) ? m * (m + 1) / 2 : m * m;
+  const int gb = r / per;
+  r -= gb * per;
+  if (layout == KATA_LAYOUT_DIRECT) {
+    a = r / m; b = r - a * m; scale = 1.f;
   } else {
-    // upper triangle a <= b in row-major order: row a starts at a d - a (a - 1) / 2
-    int aa = (int)((2.f * d + 1.f - sqrtf((2.f * d + 1.f) * (2.f * d + 1.f) - 8.f * (float)r)) * 0.5f);
+    // upper triangle a <= b in row-major order: row a starts at a m - a (a - 1) / 2
+    int aa = (int)((2.f * m + 1.f - sqrtf((2.f * m + 1.f) * (2.f * m + 1.f) - 8.f * (float)r)) * 0.5f);
     if (aa < 0) aa = 0;
-    if (aa > d - 1) aa = d - 1;
-    while (aa > 0 && aa * d - aa * (aa - 1) / 2 > r) --aa;
-    while (aa + 1 < d && (aa + 1) * d - (aa + 1) * aa / 2 <= r) ++aa;
-    a = aa; b = aa + (r - (aa * d - aa * (aa - 1) / 2));
+    if (aa > m - 1) aa = m - 1;
+    while (aa > 0 && aa * m - aa * (aa - 1) / 2 > r) --aa;
+    while (aa + 1 < m && (aa + 1) * m - (aa + 1) * aa / 2 <= r) ++aa;
+    a = aa; b = aa + (r - (aa * m - aa * (aa - 1) / 2));
     scale = (a == b) ? 1.f : 1.41421356237309504880f;
   }
+  a += gb * m;
+  b += gb * m;
 }
 
 template <typename T, int DV>
 __global__ void __launch_bounds__(DEC_THREADS) decode_update_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                                     const T* __restrict__ v, float* __restrict__ S,
                                                                     float* __restrict__ Z, float* __restrict__ part,
-                                                                    int d_k, int n_psi, int layout, int order) {
+                                                                    int d_k, int n_psi, int layout, int order, int groups) {
   constexpr int TPR = DV / 4;                  // threads per state row
   constexpr int RPI = DEC_THREADS / TPR;       // rows per iteration
   __shared__ float kh[64], qs[64], red[DEC_THREADS / 32][DV + 1];
@@ -92,7 +101,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_update_kernel(const T* __r
       const int r = r0 + u * RPI;
       int a, b;
       float scale;
-      feature_pair(r < r_end ? r : 0, d_k, layout, order, a, b, scale);
+      feature_pair(r < r_end ? r : 0, d_k, layout, order, groups, a, b, scale);
       fk[u] = (b < 0) ? kh[a] : kh[a] * kh[b] * scale;
       fq[u] = (b < 0) ? qs[a] : qs[a] * qs[b] * scale;
     }
@@ -145,15 +154,21 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_update_kernel(const T* __r
 // <psi(q), psi(k)> formed directly from the dot product (exact where the feature-space sum would cancel).
 template <typename T, int DV>
 __global__ void decode_finish_kernel(const float* __restrict__ part, const T* __restrict__ q, const T* __restrict__ k,
-                                     const T* __restrict__ v, T* __restrict__ out, int n_slabs, int d_k, int order) {
+                                     const T* __restrict__ v, T* __restrict__ out, int n_slabs, int d_k, int order,
+                                     int groups) {
   const int bh = blockIdx.x, c = threadIdx.x;
-  float qk = 0.f, kk = 0.f;
-  for (int a = 0; a < d_k; ++a) {
-    const float qa = to_f32<T>(q[(size_t)bh * d_k + a]), ka = to_f32<T>(k[(size_t)bh * d_k + a]);
-    qk = fmaf(qa, ka, qk);
-    kk = fmaf(ka, ka, kk);
+  float kk = 0.f, w = 0.f;
+  const int m = d_k / groups;
+  for (int gb = 0; gb < groups; ++gb) {
+    float qk = 0.f;
+    for (int a = gb * m; a < (gb + 1) * m; ++a) {
+      const float qa = to_f32<T>(q[(size_t)bh * d_k + a]), ka = to_f32<T>(k[(size_t)bh * d_k + a]);
+      qk = fmaf(qa, ka, qk);
+      kk = fmaf(ka, ka, kk);
+    }
+    w += (order == 1) ? qk : qk * qk;
   }
-  const float w = order == 1 ? qk : qk * qk * inv_or_zero(kk);     // raw q: the query norm cancels in the ratio
+  if (order != 1) w *= inv_or_zero(kk);     // raw q: the query norm cancels in the ratio
   if (c >= DV) return;
   float num = 0.f, den = 0.f;
   for (int s = 0; s < n_slabs; ++s) {
@@ -167,21 +182,22 @@ __global__ void decode_finish_kernel(const float* __restrict__ part, const T* __
 
 template <typename T, int DV>
 void launch(const void* q, const void* k, const void* v, void* out, float* S, float* Z, float* part, int BH, int d_k,
-            int n_psi, int layout, int order, LaunchCtx& ctx) {
+            int n_psi, int layout, int order, int groups, LaunchCtx& ctx) {
   const int n_slabs = decode_slabs(n_psi);
   decode_update_kernel<T, DV><<<dim3(n_slabs, BH), DEC_THREADS, 0, ctx.stream>>>(
-      static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), S, Z, part, d_k, n_psi, layout, order);
+      static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), S, Z, part, d_k, n_psi, layout, order, groups);
   note_launch(ctx);
   decode_finish_kernel<T, DV><<<BH, 64, 0, ctx.stream>>>(part, static_cast<const T*>(q), static_cast<const T*>(k),
-                                                         static_cast<const T*>(v), static_cast<T*>(out), n_slabs, d_k, order);
+                                                         static_cast<const T*>(v), static_cast<T*>(out), n_slabs, d_k, order, groups);
   note_launch(ctx);
 }
 
 }  // namespace
 
-int decode_n_psi(int d_k, int layout, int order) {
+int decode_n_psi(int d_k, int layout, int order, int groups) {
   if (order == 1) return d_k;
-  return layout == KATA_LAYOUT_PACKED ? d_k * (d_k + 1) / 2 : d_k * d_k;
+  const int m = d_k / groups;
+  return groups * (layout == KATA_LAYOUT_PACKED ? m * (m + 1) / 2 : m * m);
 }
 
 int decode_slabs(int n_psi) { return (n_psi + DEC_ROWS - 1) / DEC_ROWS; }
@@ -189,9 +205,9 @@ int decode_slabs(int n_psi) { return (n_psi + DEC_ROWS - 1) / DEC_ROWS; }
 size_t decode_workspace_elems(int BH, int n_psi, int d_v) { return (size_t)BH * decode_slabs(n_psi) * (d_v + 1); }
 
 void decode_step(const void* q, const void* k, const void* v, void* out, float* S, float* Z, float* part, int BH,
-                 int d_k, int d_v, int dtype, int layout, int order, LaunchCtx& ctx) {
-  const int n_psi = decode_n_psi(d_k, layout, order);
-#define KATA_DEC(T, DV) launch<T, DV>(q, k, v, out, S, Z, part, BH, d_k, n_psi, layout, order, ctx)
+                 int d_k, int d_v, int dtype, int layout, int order, int groups, LaunchCtx& ctx) {
+  const int n_psi = decode_n_psi(d_k, layout, order, groups);
+#define KATA_DEC(T, DV) launch<T, DV>(q, k, v, out, S, Z, part, BH, d_k, n_psi, layout, order, groups, ctx)
   if (dtype == KATA_F32) {
     if (d_v == 64) KATA_DEC(float, 64); else if (d_v == 32) KATA_DEC(float, 32); else KATA_DEC(float, 16);
   } else {

@@ -69,7 +69,8 @@ __global__ void __launch_bounds__(NTHR) chunk_simt_kernel(const T* __restrict__ 
                                                            int Tlen, int n_chunks, int chunks_per_group,
                                                            int n_groups,
                                                            const float* __restrict__ init_state,
-                                                           float* __restrict__ final_state, int write_out) {
+                                                           float* __restrict__ final_state, int write_out,
+                                                           int groups) {
   using G = Cfg<D, DV>;
   constexpr int BLK = G::BLK, VS = G::VS, RS = G::RS;
   extern __shared__ __align__(16) float smem[];
@@ -94,13 +95,15 @@ __global__ void __launch_bounds__(NTHR) chunk_simt_kernel(const T* __restrict__ 
     while (t >= NB - A) { t -= NB - A; ++A; }
     Bq = A + t;
   }
-  float wgt[BLK][BLK];   // 2 above the diagonal, 1 on it, 0 below (and for idle threads)
+  // blockwise PSD map: only pairs (a,b) of the same feature group carry state (NB / groups blocks per group)
+  const bool same_group = (A / (NB / groups)) == (Bq / (NB / groups));
+  float wgt[BLK][BLK];   // 2 above the diagonal, 1 on it, 0 below (and for idle threads and other groups)
 #pragma unroll
   for (int i = 0; i < BLK; ++i)
 #pragma unroll
     for (int j = 0; j < BLK; ++j) {
       const int a = A * BLK + i, b = Bq * BLK + j;
-      wgt[i][j] = !active ? 0.f : (a < b ? 2.f : (a == b ? 1.f : 0.f));
+      wgt[i][j] = (!active || !same_group) ? 0.f : (a < b ? 2.f : (a == b ? 1.f : 0.f));
     }
 
   float S[BLK][BLK][VS];
@@ -174,28 +177,39 @@ __global__ void __launch_bounds__(NTHR) chunk_simt_kernel(const T* __restrict__ 
       // ---- intra-chunk scores, one 4x4 tile per thread on or below the block diagonal ----
       if (active) {
         const int tb = Bq, ib = A;
-        float s[4][4];
+        float s[4][4], w2[4][4];
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
-          for (int j = 0; j < 4; ++j) s[i][j] = 0.f;
-#pragma unroll 4
-        for (int a = 0; a < D; ++a) {
-          const float4 qa = *reinterpret_cast<const float4*>(&qT[a][tb * 4]);
-          const float4 ka = *reinterpret_cast<const float4*>(&kT[a][ib * 4]);
-          const float qq[4] = {qa.x, qa.y, qa.z, qa.w};
-          const float kk[4] = {ka.x, ka.y, ka.z, ka.w};
+          for (int j = 0; j < 4; ++j) w2[i][j] = 0.f;
+        const int mblk = D / groups;
+        for (int gb = 0; gb < groups; ++gb) {
 #pragma unroll
           for (int i = 0; i < 4; ++i)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) s[i][j] = fmaf(qq[i], kk[j], s[i][j]);
+            for (int j = 0; j < 4; ++j) s[i][j] = 0.f;
+#pragma unroll 4
+          for (int a = gb * mblk; a < (gb + 1) * mblk; ++a) {
+            const float4 qa = *reinterpret_cast<const float4*>(&qT[a][tb * 4]);
+            const float4 ka = *reinterpret_cast<const float4*>(&kT[a][ib * 4]);
+            const float qq[4] = {qa.x, qa.y, qa.z, qa.w};
+            const float kk[4] = {ka.x, ka.y, ka.z, ka.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) s[i][j] = fmaf(qq[i], kk[j], s[i][j]);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) w2[i][j] = fmaf(s[i][j], s[i][j], w2[i][j]);
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const int t = tb * 4 + i, i2 = ib * 4 + j;
-            P[t][i2] = (i2 <= t) ? s[i][j] * s[i][j] : 0.f;
+            P[t][i2] = (i2 <= t) ? w2[i][j] : 0.f;
           }
       }
       __syncthreads();
@@ -316,12 +330,12 @@ __global__ void scan_round_kernel(const float4* __restrict__ src, float4* __rest
 // Exclusive-prefix chunk states in the public layouts, from the inclusive scan of per-chunk states.
 template <int D, int DV>
 __global__ void export_states_kernel(const float* __restrict__ incl, float* __restrict__ s_pre,
-                                     float* __restrict__ z_pre, int n_chunks, int layout) {
+                                     float* __restrict__ z_pre, int n_chunks, int layout, int groups) {
   using G = Cfg<D, DV>;
   constexpr int BLK = G::BLK, VS = G::VS;
   const int c = blockIdx.x;
   const size_t bh = blockIdx.y;
-  const int n_psi = (layout == KATA_LAYOUT_PACKED) ? D * (D + 1) / 2 : D * D;
+  const int n_psi = groups * ((layout == KATA_LAYOUT_PACKED) ? (D / groups) * (D / groups + 1) / 2 : (D / groups) * (D / groups));
   const size_t slot = (size_t)G::NREG * NTHR;
   float* sp = s_pre + (bh * n_chunks + c) * (size_t)n_psi * DV;
   float* zp = z_pre + (bh * n_chunks + c) * (size_t)n_psi;
@@ -329,15 +343,24 @@ __global__ void export_states_kernel(const float* __restrict__ incl, float* __re
     const int row = item / (DV + 1), col = item % (DV + 1);
     int a, b;
     float scale = 1.f;
-    if (layout == KATA_LAYOUT_PACKED) {
-      a = 0;
-      int r = row;
-      while (r >= D - a) { r -= D - a; ++a; }
-      b = a + r;
-      if (a != b) scale = 1.41421356237309504880f;
-    } else {
-      a = row / D;
-      b = row % D;
+    {
+      // rows of the g feature blocks follow one another; inside a block of m = D / g features the layout is
+      // the direct m x m or the packed upper triangle
+      const int m = D / groups;
+      const int per = (layout == KATA_LAYOUT_PACKED) ? m * (m + 1) / 2 : m * m;
+      const int gb = row / per;
+      int r = row - gb * per;
+      if (layout == KATA_LAYOUT_PACKED) {
+        a = 0;
+        while (r >= m - a) { r -= m - a; ++a; }
+        b = a + r;
+        if (a != b) scale = 1.41421356237309504880f;
+      } else {
+        a = r / m;
+        b = r % m;
+      }
+      a += gb * m;
+      b += gb * m;
     }
     float val = 0.f;
     if (c > 0) {
@@ -358,11 +381,11 @@ __global__ void export_states_kernel(const float* __restrict__ incl, float* __re
 // whole-sequence pass.
 template <int D, int DV>
 __global__ void export_final_kernel(const float* __restrict__ fin, float* __restrict__ s_out, float* __restrict__ z_out,
-                                    int layout) {
+                                    int layout, int groups) {
   using G = Cfg<D, DV>;
   constexpr int BLK = G::BLK, VS = G::VS;
   const size_t bh = blockIdx.y;
-  const int n_psi = (layout == KATA_LAYOUT_PACKED) ? D * (D + 1) / 2 : D * D;
+  const int n_psi = groups * ((layout == KATA_LAYOUT_PACKED) ? (D / groups) * (D / groups + 1) / 2 : (D / groups) * (D / groups));
   const size_t slot = (size_t)G::NREG * NTHR;
   float* sp = s_out + bh * (size_t)n_psi * DV;
   float* zp = z_out + bh * (size_t)n_psi;
@@ -370,15 +393,24 @@ __global__ void export_final_kernel(const float* __restrict__ fin, float* __rest
     const int row = item / (DV + 1), col = item % (DV + 1);
     int a, b;
     float scale = 1.f;
-    if (layout == KATA_LAYOUT_PACKED) {
-      a = 0;
-      int r = row;
-      while (r >= D - a) { r -= D - a; ++a; }
-      b = a + r;
-      if (a != b) scale = 1.41421356237309504880f;
-    } else {
-      a = row / D;
-      b = row % D;
+    {
+      // rows of the g feature blocks follow one another; inside a block of m = D / g features the layout is
+      // the direct m x m or the packed upper triangle
+      const int m = D / groups;
+      const int per = (layout == KATA_LAYOUT_PACKED) ? m * (m + 1) / 2 : m * m;
+      const int gb = row / per;
+      int r = row - gb * per;
+      if (layout == KATA_LAYOUT_PACKED) {
+        a = 0;
+        while (r >= m - a) { r -= m - a; ++a; }
+        b = a + r;
+        if (a != b) scale = 1.41421356237309504880f;
+      } else {
+        a = r / m;
+        b = r % m;
+      }
+      a += gb * m;
+      b += gb * m;
     }
     const int lo = min(a, b), hi = max(a, b);
     const int Ab = lo / BLK, Bb = hi / BLK, i = lo % BLK, j = hi % BLK;
@@ -412,10 +444,10 @@ void run(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float
     // whole sequence in one pass; with s_pre/z_pre the state after the last token is exported
     float* fin = (s_pre != nullptr) ? ws : nullptr;
     kern<<<dim3(G::NSLICE, BH, 1), NTHR, smem, ctx.stream>>>(q, k, v, o, p.T, plan.n_chunks, plan.n_chunks,
-                                                            1, nullptr, fin, 1);
+                                                            1, nullptr, fin, 1, p.groups);
     note_launch(ctx);
     if (fin != nullptr) {
-      export_final_kernel<D, DV><<<dim3(16, BH), 256, 0, ctx.stream>>>(fin, s_pre, z_pre, state_layout);
+      export_final_kernel<D, DV><<<dim3(16, BH), 256, 0, ctx.stream>>>(fin, s_pre, z_pre, state_layout, p.groups);
       note_launch(ctx);
     }
     return;
@@ -428,18 +460,18 @@ void run(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float
   if (NG > 1) {
     // pass 1: local states of all groups but the last (its state is never read)
     kern<<<dim3(G::NSLICE, BH, NG - 1), NTHR, smem, ctx.stream>>>(q, k, v, o, p.T, plan.n_chunks,
-                                                                 plan.chunks_per_group, NG, nullptr, bufA, 0);
+                                                                 plan.chunks_per_group, NG, nullptr, bufA, 0, p.groups);
     note_launch(ctx);
     // pass 2: inclusive scan over the first NG-1 group states, ceil(log2(NG-1)) rounds
     incl = scan_group_states(bufA, bufB, BH, NG, NG - 1, E, ctx);
   }
   // pass 3: every group restarts from the prefix before it
   kern<<<dim3(G::NSLICE, BH, NG), NTHR, smem, ctx.stream>>>(q, k, v, o, p.T, plan.n_chunks,
-                                                           plan.chunks_per_group, NG, incl, nullptr, 1);
+                                                           plan.chunks_per_group, NG, incl, nullptr, 1, p.groups);
   note_launch(ctx);
   if (s_pre != nullptr && z_pre != nullptr) {
     export_states_kernel<D, DV><<<dim3(plan.n_chunks, BH), 256, 0, ctx.stream>>>(incl, s_pre, z_pre,
-                                                                               plan.n_chunks, state_layout);
+                                                                               plan.n_chunks, state_layout, p.groups);
     note_launch(ctx);
   }
 }

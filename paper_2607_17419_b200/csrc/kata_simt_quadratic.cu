@@ -18,7 +18,7 @@ constexpr int TS = 68;   // row stride of the transposed q/k tiles in shared mem
 template <typename T, int D, int DV>
 __global__ void __launch_bounds__(NTHR) quad_simt_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                           const T* __restrict__ v, T* __restrict__ out,
-                                                          int Tlen, int order) {
+                                                          int Tlen, int order, int groups) {
   extern __shared__ __align__(16) float smem[];
   // transposed tiles, row stride TS (=68 floats: 16-byte aligned rows, few bank conflicts on the fill)
   float (*qT)[TS] = reinterpret_cast<float (*)[TS]>(smem);
@@ -70,23 +70,36 @@ __global__ void __launch_bounds__(NTHR) quad_simt_kernel(const T* __restrict__ q
       for (int a = 0; a < D; ++a) s = fmaf(kT[a][tid], kT[a][tid], s);
       rk2[tid] = (order == 2) ? inv_or_zero(s) : 1.f;
     }
-    // scores: 4 x 8 micro-tile per thread
-    float s[4][8];
+    // scores: 4 x 8 micro-tile per thread; with g feature blocks the weight is the sum of the squared block dots
+    float s[4][8], w2[4][8];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-      for (int j = 0; j < 8; ++j) s[i][j] = 0.f;
-#pragma unroll 4
-    for (int a = 0; a < D; ++a) {
-      const float4 qa = *reinterpret_cast<const float4*>(&qT[a][ty * 4]);
-      const float4 k0v = *reinterpret_cast<const float4*>(&kT[a][tx * 8]);
-      const float4 k1v = *reinterpret_cast<const float4*>(&kT[a][tx * 8 + 4]);
-      const float qq[4] = {qa.x, qa.y, qa.z, qa.w};
-      const float kk[8] = {k0v.x, k0v.y, k0v.z, k0v.w, k1v.x, k1v.y, k1v.z, k1v.w};
+      for (int j = 0; j < 8; ++j) w2[i][j] = 0.f;
+    const int mblk = D / groups;
+    for (int gb = 0; gb < groups; ++gb) {
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) s[i][j] = fmaf(qq[i], kk[j], s[i][j]);
+        for (int j = 0; j < 8; ++j) s[i][j] = 0.f;
+#pragma unroll 4
+      for (int a = gb * mblk; a < (gb + 1) * mblk; ++a) {
+        const float4 qa = *reinterpret_cast<const float4*>(&qT[a][ty * 4]);
+        const float4 k0v = *reinterpret_cast<const float4*>(&kT[a][tx * 8]);
+        const float4 k1v = *reinterpret_cast<const float4*>(&kT[a][tx * 8 + 4]);
+        const float qq[4] = {qa.x, qa.y, qa.z, qa.w};
+        const float kk[8] = {k0v.x, k0v.y, k0v.z, k0v.w, k1v.x, k1v.y, k1v.z, k1v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 8; ++j) s[i][j] = fmaf(qq[i], kk[j], s[i][j]);
+      }
+      if (groups > 1) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 8; ++j) w2[i][j] = fmaf(s[i][j], s[i][j], w2[i][j]);
+      }
     }
     __syncthreads();   // rk2 visible
 #pragma unroll
@@ -95,7 +108,7 @@ __global__ void __launch_bounds__(NTHR) quad_simt_kernel(const T* __restrict__ q
       for (int j = 0; j < 8; ++j) {
         const int r = ty * 4 + i, c = tx * 8 + j;
         const bool live = (k0 + c <= q0 + r) && (k0 + c < Tlen);
-        float w = (order == 2) ? s[i][j] * s[i][j] * rk2[c] : s[i][j];
+        float w = (order == 2) ? (groups > 1 ? w2[i][j] : s[i][j] * s[i][j]) * rk2[c] : s[i][j];
         W[r][c] = live ? w : 0.f;
       }
     __syncthreads();
@@ -137,7 +150,7 @@ void launch_one(const Problem& p, LaunchCtx& ctx) {
   }
   kern<<<grid, NTHR, smem, ctx.stream>>>(static_cast<const T*>(p.q), static_cast<const T*>(p.k),
                                          static_cast<const T*>(p.v), static_cast<T*>(p.out), p.T,
-                                         p.feature_order);
+                                         p.feature_order, p.groups);
   note_launch(ctx);
 }
 

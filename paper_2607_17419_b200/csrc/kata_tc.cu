@@ -4,7 +4,7 @@
 namespace kata {
 
 bool tc_supported(const Problem& p, int fn, bool scan) {
-  if (p.dtype != KATA_BF16 || p.d_k != 64 || p.d_v != 64 || p.feature_order != 2) return false;
+  if (p.dtype != KATA_BF16 || p.d_k != 64 || p.d_v != 64 || p.feature_order != 2 || p.groups != 1) return false;
   (void)scan;
   return fn == KATA_FN_QUADRATIC || fn == KATA_FN_CHUNKED || fn == KATA_FN_CHUNK_STATE_SCAN;
 }

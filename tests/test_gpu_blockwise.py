@@ -1,0 +1,93 @@
+"""GPU parity of the blockwise PSD map (KATA-Mg, g = 2 or 4) against the fp64 oracle: every form, the exported
+prefix states, the final state and the decode step."""
+import numpy as np
+import pytest
+
+from oracle import kata_oracle as ko
+from paper_2607_17419_b200 import binding as kb
+from paper_2607_17419_b200 import inputs
+
+from helpers import check, dev_tensors, to_numpy64
+
+pytestmark = pytest.mark.gpu
+
+FORMS = {
+    "quadratic": lambda q, k, v, **kw: kb.kata_fwd_quadratic(q, k, v, **kw),
+    "chunked_seq": lambda q, k, v, **kw: kb.kata_fwd_chunked(q, k, v, inter_chunk=kb.KATA_SEQUENTIAL, **kw),
+    "chunked_scan": lambda q, k, v, **kw: kb.kata_fwd_chunked(q, k, v, inter_chunk=kb.KATA_SCAN, **kw),
+    "state_scan": lambda q, k, v, **kw: kb.kata_chunk_state_scan(q, k, v, **kw),
+}
+CASES = [("f32", 16, 16, 2), ("f32", 16, 32, 4), ("f32", 32, 16, 4), ("f32", 64, 64, 2), ("bf16", 64, 64, 2),
+         ("bf16", 64, 64, 4), ("bf16", 32, 64, 2)]
+
+
+@pytest.mark.parametrize("form", list(FORMS))
+@pytest.mark.parametrize("dtype,dk,dv,g", CASES)
+def test_blockwise_forms(form, dtype, dk, dv, g):
+    import torch
+    w = inputs.gaussian_workload(f"mg_{dtype}_{dk}_{dv}_{g}", dtype, 2, 2, 333, dk, dv, 64, 300 + dk + g)
+    o = FORMS[form](*dev_tensors(w), feature_groups=g)
+    torch.cuda.synchronize()
+    assert kb.kata_last_impl() == kb.KATA_IMPL_SIMT        # the blockwise map runs on the fp32 kernels
+    gpu = to_numpy64(o)
+    for b in range(w.B):
+        for h in range(w.H):
+            ref = ko.kata_quadratic(w.q_ref[b, h], w.k_ref[b, h], w.v_ref[b, h], f"psd_direct:g{g}")[0]
+            check(gpu[b, h], ref, dtype, f"M{g}/{form} ({b},{h})")
+    # g = 1 given explicitly is the plain feature
+    o1, o0 = FORMS[form](*dev_tensors(w), feature_groups=1), FORMS[form](*dev_tensors(w))
+    torch.cuda.synchronize()
+    assert torch.equal(o1, o0)
+
+
+@pytest.mark.parametrize("layout", ["psd_direct", "psd_packed"])
+@pytest.mark.parametrize("g", [2, 4])
+def test_blockwise_states_and_decode(layout, g):
+    """Exported prefix states, the final state of the sequential form, and decoding on from it."""
+    import torch
+    B, H, T, Tp, d, dv = 1, 2, 200, 150, 32, 16
+    w = inputs.gaussian_workload("mg_state", "f32", B, H, T, d, dv, 64, 400 + g)
+    q, k, v = dev_tensors(w)
+    code = kb.KATA_LAYOUT_PACKED if layout == "psd_packed" else kb.KATA_LAYOUT_DIRECT
+    feat = f"{layout}:g{g}"
+    n = kb.decode_n_psi(d, 2, code, g)
+    assert n == ko.feature_dim(d, feat)
+    NC = (T + 63) // 64
+    s_pre = torch.empty(B, H, NC, n, dv, device="cuda")
+    z_pre = torch.empty(B, H, NC, n, device="cuda")
+    kb.kata_chunk_state_scan(q, k, v, s_pre=s_pre, z_pre=z_pre, state_layout=code, feature_groups=g)
+    S = torch.empty(B, H, n, dv, device="cuda")
+    Z = torch.empty(B, H, n, device="cuda")
+    kb.kata_fwd_chunked(q[:, :, :Tp].contiguous(), k[:, :, :Tp].contiguous(), v[:, :, :Tp].contiguous(),
+                        s_pre=S, z_pre=Z, state_layout=code, feature_groups=g)
+    torch.cuda.synchronize()
+    for h in range(H):
+        _, rs, rz = ko.kata_scan(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h], 64, feat)
+        assert np.max(np.abs(to_numpy64(s_pre[0, h]) - rs)) <= 1e-5 * max(1.0, np.abs(rs).max())
+        assert np.max(np.abs(to_numpy64(z_pre[0, h]) - rz)) <= 1e-5 * max(1.0, np.abs(rz).max())
+        fk = ko.apply_feature(w.k_ref[0, h, :Tp], feat)
+        Sr, Zr = fk.T @ w.v_ref[0, h, :Tp], fk.sum(axis=0)
+        assert np.max(np.abs(to_numpy64(S[0, h]) - Sr)) <= 1e-4 * max(1.0, np.abs(Sr).max())
+        assert np.max(np.abs(to_numpy64(Z[0, h]) - Zr)) <= 1e-4 * max(1.0, np.abs(Zr).max())
+    outs = []
+    for t in range(Tp, T):
+        outs.append(kb.kata_decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(), S, Z,
+                                        state_layout=code, feature_groups=g).float())
+    torch.cuda.synchronize()
+    gdec = torch.stack(outs, dim=2).cpu().numpy().astype(np.float64)
+    for h in range(H):
+        ref = ko.kata_quadratic(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h], feat)[0][Tp:]
+        check(gdec[0, h], ref, "f32", f"M{g} decode after prefill/{layout}")
+
+
+def test_blockwise_argument_checks():
+    import torch
+    w = inputs.gaussian_workload("mg_args", "f32", 1, 1, 64, 16, 16, 64, 1)
+    q, k, v = dev_tensors(w)
+    with pytest.raises(kb.KataError):
+        kb.kata_fwd_quadratic(q, k, v, feature_groups=3)
+    with pytest.raises(kb.KataError):
+        kb.kata_fwd_quadratic(q, k, v, feature_groups=2, feature_order=1)
+    wb = inputs.gaussian_workload("mg_args_bf16", "bf16", 1, 1, 64, 64, 64, 64, 1)
+    with pytest.raises(kb.KataError):
+        kb.kata_fwd_chunked(*dev_tensors(wb), feature_groups=2, impl=kb.KATA_IMPL_TENSOR)
