@@ -132,6 +132,10 @@ __global__ void __launch_bounds__(256) quad_prescale_kernel(const __nv_bfloat16*
   if (part == 0) rscale[row] = __float2bfloat16_rn(r2);
 }
 
+// G = feature groups of the blockwise map (Section 3.3): a key tile holds KT = 128 / G keys, and the 128 score
+// columns of a buffer hold the G per-group score blocks Q_a K_a^T side by side (group a in columns [a KT, a KT + KT));
+// the weight of a key is the sum over the groups of the squared scores.
+template <int G>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const QArgs args) {
@@ -149,7 +153,9 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   const int qtile = gridDim.x - 1 - blockIdx.x;   // heaviest tiles first
   const int bh = blockIdx.y;
   const int q0 = qtile * QT;
-  const int ntiles = qtile + 1;                   // key tiles 0..qtile
+  constexpr int KT = KTILE / G;                   // keys per tile
+  constexpr int KPL = KT / 32;                    // keys per producer lane
+  const int ntiles = (qtile + 1) * G;             // key tiles covering keys 0 .. q0 + 127
 
   if (tid == 0) {
     abort_s = 0;
@@ -193,31 +199,31 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
     const __nv_bfloat16* rs = args.rscale + (size_t)bh * args.Tlen;
     // r of this lane's 4 keys of a tile, fetched one tile ahead (the global-load latency stays off the ring)
-    auto load_r = [&](int j, unsigned short (&rv)[4]) {
+    auto load_r = [&](int j, unsigned short (&rv)[KPL]) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int key = j * KTILE + lane * 4 + e;
+      for (int e = 0; e < KPL; ++e) {
+        const int key = j * KT + lane * KPL + e;
         rv[e] = (j < ntiles && key < args.Tlen) ? __bfloat16_as_ushort(rs[key]) : (unsigned short)0;
       }
     };
-    unsigned short rv[4];
+    unsigned short rv[KPL];
     load_r(0, rv);
     for (int j = 0; j < ntiles && ok; ++j) {
       const int s = j % NSTAGE;
-      unsigned short rn[4];
+      unsigned short rn[KPL];
       load_r(j + 1, rn);
       ok = wait_or_abort(bar(BAR_EMPTY + s), ((j / NSTAGE) & 1) ^ 1, abort_flag);
       if (!ok) break;
       if (lane == 0) {
-        mbar_arrive_expect_tx(bar(BAR_FULL + s), 32768);   // K and V' tiles
-        tma_load_3d(ktile(s), &tmK, bar(BAR_FULL + s), 0, j * KTILE, bh);
-        tma_load_3d(vtile(s), &tmV, bar(BAR_FULL + s), 0, j * KTILE, bh);
+        mbar_arrive_expect_tx(bar(BAR_FULL + s), 2 * KT * 128);   // K and V' tiles
+        tma_load_3d(ktile(s), &tmK, bar(BAR_FULL + s), 0, j * KT, bh);
+        tma_load_3d(vtile(s), &tmV, bar(BAR_FULL + s), 0, j * KT, bh);
       }
-      // column 64 of the B operand: r for the 128 keys of the tile (element 0 of chunk 0 of each key row)
+      // column 64 of the B operand: r for the keys of the tile (element 0 of chunk 0 of each key row)
       unsigned char* rt = rtile(s);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        *reinterpret_cast<uint16_t*>(rt + sw128_offset(lane * 4 + e, 0)) = rv[e];
+      for (int e = 0; e < KPL; ++e) {
+        *reinterpret_cast<uint16_t*>(rt + sw128_offset(lane * KPL + e, 0)) = rv[e];
         rv[e] = rn[e];
       }
       fence_async_smem();
@@ -226,7 +232,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   } else if (warp == 1) {
     // =========================== score MMA issuer: S = Q K^T ===========================
     if (lane == 0) {
-      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 128);
+      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, KT);
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
       ok = wait_or_abort(bar(BAR_QTMEM), 0, abort_flag);
       for (int j = 0; j < ntiles && ok; ++j) {
@@ -237,9 +243,9 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         tc_fence_after();
         const uint32_t ka = smem_u32(ktile(s));
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          mma_f16_ts(tb + COL_S + b * 128, tb + COL_Q + ks * 8, dk + (uint64_t)(((ka + ks * 32) >> 4) & 0x3FFF),
-                     idesc, ks > 0);
+        for (int ks = 0; ks < 4; ++ks)   // 16 features per step; group ks / (4 / G) accumulates over its own steps
+          mma_f16_ts(tb + COL_S + b * 128 + (ks / (4 / G)) * KT, tb + COL_Q + ks * 8,
+                     dk + (uint64_t)(((ka + ks * 32) >> 4) & 0x3FFF), idesc, (ks % (4 / G)) > 0);
         mma_commit(bar(BAR_SFULL + b));
         mma_commit(bar(BAR_EMPTY + s));
       }
@@ -258,7 +264,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         tc_fence_after();
         const uint32_t va = smem_u32(vtile(s));
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
+        for (int ks = 0; ks < KT / 16; ++ks)
           mma_f16_ts(tb + COL_O, tb + COL_S + b * 128 + ks * 8, dmn + (uint64_t)(((va + ks * 2048) >> 4) & 0x3FFF),
                      idesc, (j > 0 || ks > 0) ? 1u : 0u);
         mma_commit(bar(BAR_PEMPTY + b));
@@ -291,8 +297,45 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       ok = wait_or_abort(bar(BAR_SFULL + b), (j / NBUF) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
+      const bool diag = (j >= ntiles - G);
+      if constexpr (G > 1) {
+        // this warp weighs keys [ch KT/2, ch KT/2 + KT/2) of the tile: one column run per group
+        constexpr int KH = KT / 2;
+        const int key0 = j * KT + ch * KH;
+        uint32_t y[G][KH], pk[KH / 2];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const uint32_t col = tmem_addr(tb, q4 * 32, COL_S + b * 128 + g * KT + ch * KH);
+          if constexpr (KH == 32) tmem_ld32(col, y[g]); else tmem_ld16(col, y[g]);
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) tmem_wait_ld(y[g]);
+#pragma unroll
+        for (int c = 0; c < KH; c += 2) {
+          float2 w = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            const float2 sv = make_float2(__uint_as_float(y[g][c]), __uint_as_float(y[g][c + 1]));
+            w = __ffma2_rn(sv, sv, w);
+          }
+          if (diag) {
+            if (key0 + c > qrow) w.x = 0.f;
+            if (key0 + c + 1 > qrow) w.y = 0.f;
+          }
+          pk[c / 2] = pack_bf16(w.x, w.y);
+        }
+        // the weights overwrite score columns [0, KT/2) of the buffer (group 0, read by the ch = 0 warp)
+        tc_fence_before();
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + (int)q4) : "memory");
+        tc_fence_after();
+        const uint32_t pcol = tmem_addr(tb, q4 * 32, COL_S + b * 128 + ch * (KH / 2));
+        if constexpr (KH == 32) tmem_st16(pcol, pk); else tmem_st8(pcol, pk);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_PFULL + b));
+        continue;
+      }
       const uint32_t scol = tmem_addr(tb, q4 * 32, COL_S + b * 128 + ch * 64);
-      const bool diag = (j == ntiles - 1);
       const int key0 = j * KTILE + ch * 64;
       uint32_t ya[32], yb[32], pk[32];
       auto weigh = [&](const uint32_t (&y)[32], int half) {
@@ -381,12 +424,12 @@ EncodeTiledFn encode_fn() {
 }
 
 // [BH][T][64] bf16 tensor, box = 64 columns x 128 rows x 1 head, 128B swizzle; rows beyond T read as zero.
-bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T) {
+bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T, int rows) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)BH};
   cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
-  cuuint32_t box[3] = {(cuuint32_t)D, (cuuint32_t)KTILE, 1};
+  cuuint32_t box[3] = {(cuuint32_t)D, (cuuint32_t)rows, 1};
   cuuint32_t es[3] = {1, 1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -411,18 +454,19 @@ void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchC
       static_cast<const __nv_bfloat16*>(p.k), static_cast<const __nv_bfloat16*>(p.v), vs, rscale, n_rows);
   note_launch(ctx);
   CUtensorMap tmQ, tmK, tmV;
-  if (!make_map(&tmQ, p.q, BH, p.T) || !make_map(&tmK, p.k, BH, p.T) || !make_map(&tmV, vs, BH, p.T)) {
+  const int kt = KTILE / p.groups;
+  if (!make_map(&tmQ, p.q, BH, p.T, QT) || !make_map(&tmK, p.k, BH, p.T, kt) || !make_map(&tmV, vs, BH, p.T, kt)) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-  if (cudaFuncSetAttribute(tc_quad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) !=
-      cudaSuccess) {
+  auto kern = p.groups == 1 ? tc_quad_kernel<1> : p.groups == 2 ? tc_quad_kernel<2> : tc_quad_kernel<4>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
     cudaGetLastError();
     ctx.status = KATA_ERR_CUDA;
     return;
   }
   QArgs a{static_cast<__nv_bfloat16*>(p.out), rscale, device_status, p.T};
-  tc_quad_kernel<<<dim3((p.T + QT - 1) / QT, BH), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
+  kern<<<dim3((p.T + QT - 1) / QT, BH), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
   note_launch(ctx);
 }
 

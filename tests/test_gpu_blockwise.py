@@ -28,7 +28,9 @@ def test_blockwise_forms(form, dtype, dk, dv, g):
     w = inputs.gaussian_workload(f"mg_{dtype}_{dk}_{dv}_{g}", dtype, 2, 2, 333, dk, dv, 64, 300 + dk + g)
     o = FORMS[form](*dev_tensors(w), feature_groups=g)
     torch.cuda.synchronize()
-    assert kb.kata_last_impl() == kb.KATA_IMPL_SIMT        # the blockwise map runs on the fp32 kernels
+    # the quadratic form has a tensor-core kernel for the blockwise map (bf16, d = 64); the rest is fp32 SIMT
+    tensor = form == "quadratic" and (dtype, dk, dv) == ("bf16", 64, 64)
+    assert kb.kata_last_impl() == (kb.KATA_IMPL_TENSOR if tensor else kb.KATA_IMPL_SIMT)
     gpu = to_numpy64(o)
     for b in range(w.B):
         for h in range(w.H):
@@ -38,6 +40,49 @@ def test_blockwise_forms(form, dtype, dk, dv, g):
     o1, o0 = FORMS[form](*dev_tensors(w), feature_groups=1), FORMS[form](*dev_tensors(w))
     torch.cuda.synchronize()
     assert torch.equal(o1, o0)
+
+
+@pytest.mark.parametrize("g", [2, 4])
+@pytest.mark.parametrize("T", [1, 31, 32, 33, 64, 65, 127, 128, 129, 257, 640])
+def test_blockwise_quadratic_tensor_tiles(g, T):
+    """Tensor-core quadratic kernel: key tiles of 128 / g keys, the last g of them masked on the diagonal."""
+    import torch
+    w = inputs.gaussian_workload(f"mg_tc_{T}", "bf16", 1, 2, T, 64, 64, 64, 500 + T + g)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    o = kb.kata_fwd_quadratic(*dev_tensors(w), feature_groups=g, device_status=st)
+    torch.cuda.synchronize()
+    assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR and int(st.item()) == 0
+    gpu = to_numpy64(o)
+    for h in range(w.H):
+        ref = ko.kata_quadratic(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h], f"psd_direct:g{g}")[0]
+        check(gpu[0, h], ref, "bf16", f"M{g} tensor quadratic T={T} head {h}")
+    # the fp32 SIMT kernel on the same inputs agrees to the bf16 tolerance
+    o2 = kb.kata_fwd_quadratic(*dev_tensors(w), feature_groups=g, impl=kb.KATA_IMPL_SIMT)
+    torch.cuda.synchronize()
+    assert kb.kata_last_impl() == kb.KATA_IMPL_SIMT
+    assert float((o.float() - o2.float()).abs().max()) <= 4e-2
+
+
+@pytest.mark.parametrize("g", [2, 4])
+def test_blockwise_quadratic_tensor_degenerate(g):
+    """Zero keys and queries: zero feature, output 0 where the normaliser is 0."""
+    T = 300
+    w = inputs.gaussian_workload("mg_tc_deg", "bf16", 1, 1, T, 64, 64, 64, 77 + g)
+    q, k, v = w.q_dev.copy(), w.k_dev.copy(), w.v_dev.copy()
+    for t in (0, 1, 31, 32, 127, 128, 299):
+        k[0, 0, t] = 0
+    for t in (0, 5, 64, 128, 256):
+        q[0, 0, t] = 0
+    # one key that lives in a single block of the split: its other blocks are zero vectors
+    k[0, 0, 40, 64 // g:] = 0
+    from helpers import to_torch
+    qr, kr, vr = (inputs.bf16_bits_to_f64(a[0, 0]) for a in (q, k, v))
+    ref = ko.kata_quadratic(qr, kr, vr, f"psd_direct:g{g}")[0]
+    o = kb.kata_fwd_quadratic(*(to_torch(a, "bf16") for a in (q, k, v)), feature_groups=g)
+    assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR
+    gpu = to_numpy64(o)
+    check(gpu[0, 0], ref, "bf16", f"M{g} degenerate")
+    assert np.all(gpu[0, 0, [0, 1, 5, 64, 128, 256]] == 0)
 
 
 @pytest.mark.parametrize("layout", ["psd_direct", "psd_packed"])
