@@ -72,6 +72,8 @@ int check_shape(int fn, int B, int H, int T, int d_k, int d_v, int C) {
 
 bool want_tensor(int fn, const Problem& p, const Opts& o) {
   const bool scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || (fn == KATA_FN_CHUNKED && o.inter_chunk == KATA_SCAN);
+  // the tensor-core kernel exports the final state for the plain feature only
+  if (p.groups != 1 && fn == KATA_FN_CHUNKED && o.s_pre != nullptr) return false;
   return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn, scan);
 }
 

@@ -5,9 +5,9 @@ namespace kata {
 
 bool tc_supported(const Problem& p, int fn, bool scan) {
   if (p.dtype != KATA_BF16 || p.d_k != 64 || p.d_v != 64 || p.feature_order != 2) return false;
-  (void)scan;
-  // blockwise map (g = 2, 4): the quadratic form only; the state forms run on the fp32 kernels
-  if (p.groups != 1) return fn == KATA_FN_QUADRATIC && (p.groups == 2 || p.groups == 4);
+  // blockwise map (g = 2, 4): the quadratic form and the one-pass chunked form; the scan forms run on the fp32 kernels
+  if (p.groups != 1)
+    return (fn == KATA_FN_QUADRATIC || (fn == KATA_FN_CHUNKED && !scan)) && (p.groups == 2 || p.groups == 4);
   return fn == KATA_FN_QUADRATIC || fn == KATA_FN_CHUNKED || fn == KATA_FN_CHUNK_STATE_SCAN;
 }
 

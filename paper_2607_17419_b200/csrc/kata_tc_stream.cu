@@ -71,6 +71,28 @@ constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
 static_assert(OFF_W + NWBUF * W_BYTES == OFF_ZERO && OFF_ZERO + 2048 == OFF_SP, "layout");
 
+// Blockwise map (Section 3.3) with G feature groups of 64 / G features: only the 16 x 16 state blocks whose a-block
+// and b-block lie in the same group exist.  b-block beta keeps the a-blocks first(beta) .. beta.
+template <int G>
+struct Geo {
+  static constexpr int BPG = 4 / G;                                       // b-blocks per feature group
+  __host__ __device__ static constexpr int first(int beta) { return beta / BPG * BPG; }
+  __host__ __device__ static constexpr int nblk(int beta) { return beta - first(beta) + 1; }
+  __host__ __device__ static constexpr uint32_t col_s(int beta) {         // first accumulator column of b-block beta
+    uint32_t c = 0;
+    for (int i = 0; i < beta; ++i) c += 16u * nblk(i);
+    return c;
+  }
+  static constexpr uint32_t Z = col_s(4);                                 // G = 1: 160, 2: 96, 4: 64
+  static constexpr uint32_t Y = Z + 64;
+  static constexpr uint32_t P = G == 1 ? 384u : Y + 160u;                 // scores of one intra-tile piece
+  static constexpr int NP = G == 4 ? 4 : 2;                               // intra-tile pieces of KH keys:
+  static constexpr int KH = CT / NP;                                      //   G x KH score columns (64, 128, 128)
+  static_assert(P + G * KH <= 448, "TMEM columns");
+};
+static_assert(Geo<1>::col_s(1) == 16 && Geo<1>::col_s(2) == 48 && Geo<1>::col_s(3) == 96 && Geo<1>::Z == COL_Z &&
+              Geo<1>::Y == COL_Y && Geo<1>::P == COL_P, "the plain feature keeps its layout");
+
 // Every barrier has waiters that consume each of its phases in order.
 enum {
   BAR_K_FULL = 0,     // [2] key tile landed
@@ -227,6 +249,7 @@ __device__ __noinline__ void export_state(uint32_t tb, uint32_t q4, int t, float
 }
 #endif
 
+template <int G>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const SArgs args) {
   extern __shared__ unsigned char smem_raw[];
@@ -241,6 +264,8 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   __shared__ int abort_s;
   volatile int* abort_flag = &abort_s;
 
+  using geo = Geo<G>;
+  constexpr uint32_t COL_Z = geo::Z, COL_Y = geo::Y, COL_P = geo::P;     // (the namespace constants are those of G = 1)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int slice = blockIdx.x, bh = blockIdx.y;
   const int v0 = slice * VS;
@@ -335,15 +360,19 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           const uint32_t wa = smem_u32(wbuf(wbi)), ka = smem_u32(ktile(s)) + sc * 2048;
           const uint64_t db = at(dB, ka);
           const uint32_t acc = (j > 0 || sc > 0) ? 1u : 0u;
+          // b-block beta: N = its a-blocks, the B operand starts at the first feature of its group (32 bytes per a-block)
           if (producer) {
-            mma_f16_ss(tb + COL_S + 96, at(dA, wa + 3 * 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64), acc);
+            mma_f16_ss(tb + COL_S + geo::col_s(3), at(dA, wa + 3 * 4096), db + 2 * geo::first(3),
+                       instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 16 * geo::nblk(3)), acc);
             // Z rows: 64 rows of this buffer, the other 64 rows of the tile read the zero atom (LBO reaches it)
             mma_f16_ss(tb + COL_Z, smem_desc(wa + 16384, smem_u32(base + OFF_ZERO) - (wa + 16384), 1024, kSwizzle128B), db,
                        instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64), acc);
           } else {
             mma_f16_ss(tb + COL_S + 0, at(dA, wa), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 16), acc);
-            mma_f16_ss(tb + COL_S + 16, at(dA, wa + 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 32), acc);
-            mma_f16_ss(tb + COL_S + 48, at(dA, wa + 2 * 4096), db, instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 48), acc);
+            mma_f16_ss(tb + COL_S + geo::col_s(1), at(dA, wa + 4096), db + 2 * geo::first(1),
+                       instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 16 * geo::nblk(1)), acc);
+            mma_f16_ss(tb + COL_S + geo::col_s(2), at(dA, wa + 2 * 4096), db + 2 * geo::first(2),
+                       instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 16 * geo::nblk(2)), acc);
           }
           mma_commit(bar(BAR_W_EMPTY + wbi));
           if (++wbi == NWBUF) { wbi = 0; wph ^= 1; }
@@ -373,8 +402,9 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           tc_fence_after();
           const uint32_t sbase = spa + (j & 1) * SP_BYTES + sp_block(p) * SP_BLOCK + sp_koff(p);
 #pragma unroll 1
-          for (int al = 0; al <= (p >> 1); ++al)
-            mma_f16_ts(tb + COL_Y + yb * 80, tb + COL_Q + al * 8, at(dS, sbase + al * 32), idR, al > 0);
+          for (int al = geo::first(p >> 1); al <= (p >> 1); ++al)
+            mma_f16_ts(tb + COL_Y + yb * 80, tb + COL_Q + al * 8, at(dS, sbase + (al - geo::first(p >> 1)) * 32), idR,
+                       al > geo::first(p >> 1));
           mma_commit(bar(BAR_Y_FULL + yb));
         }
         if (!ok) break;
@@ -384,7 +414,8 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   } else if (warp == WARP_I) {
     // =========================== intra-tile issuer: scores and [O | D] ===========================
     if (lane == 0) {
-      const uint32_t idQK = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 64);
+      constexpr int NP = geo::NP, KH = geo::KH;
+      const uint32_t idQK = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, KH);
       const uint32_t idPV = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 16);
       const uint64_t dK = smem_desc(0, 16, 1024, kSwizzle128B);
       for (int j = 0; j < nch && ok; ++j) {
@@ -396,25 +427,27 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (ok && j > 0) ok = wait_or_abort(bar(BAR_O_FULL), (j - 1) & 1, abort_flag);
         const uint32_t ka = smem_u32(ktile(s)), va = smem_u32(vptile(s));
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < NP; ++h) {
           if (!ok) break;
-          if (h == 1) ok = wait_or_abort(bar(BAR_PV0), j & 1, abort_flag);
+          // the weights of piece h - 1 alias the score columns: its apply MMAs must be through
+          if (h > 0) ok = wait_or_abort(bar(BAR_PV0), (j * (NP - 1) + h - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            mma_f16_ts(tb + COL_P, tb + COL_Q + ks * 8, at(dK, ka + h * 8192 + ks * 32), idQK, ks > 0);
+          for (int ks = 0; ks < 4; ++ks)   // 16 features per step; group ks / (4 / G) has its own KH score columns
+            mma_f16_ts(tb + COL_P + (ks / (4 / G)) * KH, tb + COL_Q + ks * 8, at(dK, ka + h * KH * 128 + ks * 32), idQK,
+                       (ks % (4 / G)) > 0);
           mma_commit(bar(BAR_S_FULL));
-          ok = wait_or_abort(bar(BAR_P_FULL), h, abort_flag);
+          ok = wait_or_abort(bar(BAR_P_FULL), h & 1, abort_flag);
           if (ok && h == 0 && j > 0) ok = wait_or_abort(bar(BAR_O_EMPTY), (j - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
+          for (int ks = 0; ks < KH / 16; ++ks)
             // MN-major, no swizzle: 8 keys x 16 bytes per core matrix, next 8 keys +128 (LBO), columns 8..15 +2048 (SBO)
-            mma_f16_ts(tb + COL_O, tb + COL_P + ks * 8, smem_desc(va + h * 1024 + ks * 256, 128, 2048, kSwizzleNone), idPV,
+            mma_f16_ts(tb + COL_O, tb + COL_P + ks * 8, smem_desc(va + h * KH * 16 + ks * 256, 128, 2048, kSwizzleNone), idPV,
                        (h > 0 || ks > 0) ? 1u : 0u);
-          if (h == 0) mma_commit(bar(BAR_PV0));
+          if (h < NP - 1) mma_commit(bar(BAR_PV0));
         }
         if (!ok) break;
         mma_commit(bar(BAR_O_FULL));
@@ -439,7 +472,62 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       tc_fence_after();
       unsigned char* sp = base + OFF_SP + ((jp + 1) & 1) * SP_BYTES;
       auto rowp = [&](int p) { return sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128; };
-      if (team == 1) {
+      if constexpr (G > 1) {
+        // b-blocks 0 and 2 are diagonal blocks only; b-block 1 is [a-block 0 doubled | diagonal] for G = 2, diagonal
+        // for G = 4; a Z row keeps the a-blocks of its group
+        if (team == 1) {
+          uint32_t e[16], c0[16];
+          tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + geo::col_s(2)), e);
+          tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 0), c0);
+          const int p2 = 4 + (bloc >> 3), p0 = bloc >> 3;
+          tmem_wait_ld(e);
+          tmem_wait_ld(c0);
+          tc_fence_before();
+          mbar_arrive(bar(BAR_SNAP_LD));
+          snap_store16(rowp(p2), sp_koff(p2) >> 4, vv, e, 1.f);
+          snap_store16(rowp(p0), sp_koff(p0) >> 4, vv, c0, 1.f);
+        } else {
+          uint32_t c1[16 * geo::nblk(1)];
+          const uint32_t col1 = tmem_addr(tb, q4 * 32, COL_S + 16);
+          if constexpr (geo::nblk(1) == 2) tmem_ld32(col1, c1); else tmem_ld16(col1, c1);
+          const int p1 = 2 + (bloc >> 3);
+          unsigned char* r1 = rowp(p1);
+          const uint32_t k1 = sp_koff(p1) >> 4;
+          auto store1 = [&]() {
+            if constexpr (geo::nblk(1) == 2) {
+              snap_store16(r1, k1, vv, c1, 2.f);
+              snap_store16(r1, k1 + 2, vv, c1 + 16, 1.f);
+            } else {
+              snap_store16(r1, k1, vv, c1, 1.f);
+            }
+          };
+          if (q4 < 2) {
+            // Z rows: lane = b; row 64 + (b % 8) of piece b / 8
+            uint32_t z0[32], z1[32];
+            tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z), z0);
+            tmem_wait_ld(c1);
+            store1();
+            tmem_ld32(tmem_addr(tb, q4 * 32, COL_Z + 32), z1);
+            tmem_wait_ld(z0);
+            tmem_wait_ld(z1);
+            tc_fence_before();
+            mbar_arrive(bar(BAR_SNAP_LD));
+            const int b = row_t, bz = b >> 4, fz = geo::first(bz), pz = b >> 3;
+            unsigned char* rowz = sp + sp_block(pz) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
+            const uint32_t cz = sp_koff(pz) >> 4;
+            const uint32_t rz = (uint32_t)(b & 7);
+#pragma unroll
+            for (int al = 0; al < 4; ++al)
+              if (al >= fz && al <= bz)
+                snap_store16(rowz, cz + 2 * (al - fz), rz, (al < 2 ? z0 : z1) + 16 * (al & 1), al < bz ? 2.f : 1.f);
+          } else {
+            tmem_wait_ld(c1);
+            tc_fence_before();
+            mbar_arrive(bar(BAR_SNAP_LD));
+            store1();
+          }
+        }
+      } else if (team == 1) {
         uint32_t e[32], f[16], c0[16];
         tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 48), e);
         tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + 80), f);
@@ -688,17 +776,34 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       unsigned char* sp = base + OFF_SP + ((j + 1) & 1) * SP_BYTES;
       const int p3 = 6 + (bloc >> 3);
       unsigned char* r3 = sp + sp_block(p3) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
-      uint32_t a0[32], a1[32];
-      tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 96), a0);
-      tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 128), a1);
-      tmem_wait_ld(a0);
-      tmem_wait_ld(a1);
-      tc_fence_before();
-      mbar_arrive(bar(BAR_SNAP_LD));
-      snap_store16(r3, 0, vv, a0, 2.f);
-      snap_store16(r3, 2, vv, a0 + 16, 2.f);
-      snap_store16(r3, 4, vv, a1, 2.f);
-      snap_store16(r3, 6, vv, a1 + 16, 1.f);
+      if constexpr (G == 1) {
+        uint32_t a0[32], a1[32];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 96), a0);
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + 128), a1);
+        tmem_wait_ld(a0);
+        tmem_wait_ld(a1);
+        tc_fence_before();
+        mbar_arrive(bar(BAR_SNAP_LD));
+        snap_store16(r3, 0, vv, a0, 2.f);
+        snap_store16(r3, 2, vv, a0 + 16, 2.f);
+        snap_store16(r3, 4, vv, a1, 2.f);
+        snap_store16(r3, 6, vv, a1 + 16, 1.f);
+      } else if constexpr (G == 2) {      // [a-block 2 doubled | diagonal]
+        uint32_t a0[32];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + geo::col_s(3)), a0);
+        tmem_wait_ld(a0);
+        tc_fence_before();
+        mbar_arrive(bar(BAR_SNAP_LD));
+        snap_store16(r3, 0, vv, a0, 2.f);
+        snap_store16(r3, 2, vv, a0 + 16, 1.f);
+      } else {                            // the diagonal block
+        uint32_t a0[16];
+        tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + geo::col_s(3)), a0);
+        tmem_wait_ld(a0);
+        tc_fence_before();
+        mbar_arrive(bar(BAR_SNAP_LD));
+        snap_store16(r3, 0, vv, a0, 1.f);
+      }
       fence_async_smem();
       mbar_arrive(bar(BAR_SNAP_ST));
     };
@@ -714,12 +819,12 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       // ---- weights P = (q.k)^2, causal, two halves of 64 keys ----
       if (j >= 0) {
 #pragma unroll 1
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < geo::NP; ++h) {
           // The copy of the state out of TMEM sits between two updates: serve it first when the update
           // completes while this warp waits for scores.
           ok = false;
           for (uint32_t i = 0; i < kSpinLimit; ++i) {
-            if (mbar_test_wait(bar(BAR_S_FULL), h)) { ok = true; break; }
+            if (mbar_test_wait(bar(BAR_S_FULL), h & 1)) { ok = true; break; }
             if (!snapped && mbar_test_wait(bar(BAR_U_DONE), j & 1)) { snapshot_share(j); snapped = true; }
             __nanosleep(64);
             if ((i & 1023u) == 1023u && *abort_flag) break;
@@ -727,7 +832,35 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (!ok) { *abort_flag = 1; break; }
           tc_fence_after();
           const uint32_t scol = tmem_addr(tb, q4 * 32, COL_P);
-          // 32 scores at a time; the bf16 weights go back over columns this thread has already read
+          if constexpr (G > 1) {
+            // 16 keys at a time: the weight of a key is the sum over the groups of its squared scores (group g in
+            // columns [g KH, g KH + KH)).  The bf16 weights of keys [16 i, 16 i + 16) go to columns [8 i, 8 i + 8),
+            // group-0 scores that this thread has read already.
+            constexpr int KH = geo::KH;
+#pragma unroll 1
+            for (int i = 0; i < KH / 16; ++i) {
+              float2 w[8];
+              uint32_t y[16], pk[8];
+#pragma unroll
+              for (int g = 0; g < G; ++g) {
+                tmem_ld16(scol + g * KH + 16 * i, y);
+                tmem_wait_ld(y);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const float2 sv = make_float2(__uint_as_float(y[2 * e]), __uint_as_float(y[2 * e + 1]));
+                  w[e] = g == 0 ? __fmul2_rn(sv, sv) : __ffma2_rn(sv, sv, w[e]);
+                }
+              }
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const int c = h * KH + 16 * i + 2 * e;
+                if (c > t) w[e].x = 0.f;
+                if (c + 1 > t) w[e].y = 0.f;
+                pk[e] = pack_bf16(w[e].x, w[e].y);
+              }
+              tmem_st8(scol + 8 * i, pk);
+            }
+          } else {
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             uint32_t y[32], pk[16];
@@ -743,6 +876,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
               pk[jj / 2] = pack_bf16(w.x, w.y);
             }
             tmem_st16(scol + half * 16, pk);
+          }
           }
           tmem_wait_st();
           tc_fence_before();
@@ -845,7 +979,12 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-  if (cudaFuncSetAttribute(tc_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
+#ifdef KATA_STREAM_EXPORT
+  auto kern = tc_stream_kernel<1>;       // the state export covers the plain feature
+#else
+  auto kern = p.groups == 1 ? tc_stream_kernel<1> : p.groups == 2 ? tc_stream_kernel<2> : tc_stream_kernel<4>;
+#endif
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
     cudaGetLastError();
     ctx.status = KATA_ERR_CUDA;
     return;
@@ -856,7 +995,7 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
 #else
   SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T};
 #endif
-  tc_stream_kernel<<<dim3(NSLICE, BH, 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, a);
+  kern<<<dim3(NSLICE, BH, 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, a);
   note_launch(ctx);
 }
 

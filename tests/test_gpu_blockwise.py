@@ -28,8 +28,8 @@ def test_blockwise_forms(form, dtype, dk, dv, g):
     w = inputs.gaussian_workload(f"mg_{dtype}_{dk}_{dv}_{g}", dtype, 2, 2, 333, dk, dv, 64, 300 + dk + g)
     o = FORMS[form](*dev_tensors(w), feature_groups=g)
     torch.cuda.synchronize()
-    # the quadratic form has a tensor-core kernel for the blockwise map (bf16, d = 64); the rest is fp32 SIMT
-    tensor = form == "quadratic" and (dtype, dk, dv) == ("bf16", 64, 64)
+    # the quadratic and the one-pass chunked form have tensor-core kernels for the blockwise map (bf16, d = 64)
+    tensor = form in ("quadratic", "chunked_seq") and (dtype, dk, dv) == ("bf16", 64, 64)
     assert kb.kata_last_impl() == (kb.KATA_IMPL_TENSOR if tensor else kb.KATA_IMPL_SIMT)
     gpu = to_numpy64(o)
     for b in range(w.B):
@@ -64,7 +64,24 @@ def test_blockwise_quadratic_tensor_tiles(g, T):
 
 
 @pytest.mark.parametrize("g", [2, 4])
-def test_blockwise_quadratic_tensor_degenerate(g):
+@pytest.mark.parametrize("T", [1, 15, 16, 17, 33, 64, 127, 128, 129, 255, 256, 257, 385, 640, 1100])
+def test_blockwise_chunked_tensor_tiles(g, T):
+    """Tensor-core one-pass chunked kernel with the state blocks of the g feature groups only."""
+    import torch
+    w = inputs.gaussian_workload(f"mg_tcs_{T}", "bf16", 1, 2, T, 64, 64, 64, 600 + T + g)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    o = kb.kata_fwd_chunked(*dev_tensors(w), feature_groups=g, device_status=st)
+    torch.cuda.synchronize()
+    assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR and int(st.item()) == 0
+    gpu = to_numpy64(o)
+    for h in range(w.H):
+        ref = ko.kata_quadratic(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h], f"psd_direct:g{g}")[0]
+        check(gpu[0, h], ref, "bf16", f"M{g} tensor chunked T={T} head {h}")
+
+
+@pytest.mark.parametrize("form", ["quadratic", "chunked_seq"])
+@pytest.mark.parametrize("g", [2, 4])
+def test_blockwise_tensor_degenerate(form, g):
     """Zero keys and queries: zero feature, output 0 where the normaliser is 0."""
     T = 300
     w = inputs.gaussian_workload("mg_tc_deg", "bf16", 1, 1, T, 64, 64, 64, 77 + g)
@@ -78,10 +95,10 @@ def test_blockwise_quadratic_tensor_degenerate(g):
     from helpers import to_torch
     qr, kr, vr = (inputs.bf16_bits_to_f64(a[0, 0]) for a in (q, k, v))
     ref = ko.kata_quadratic(qr, kr, vr, f"psd_direct:g{g}")[0]
-    o = kb.kata_fwd_quadratic(*(to_torch(a, "bf16") for a in (q, k, v)), feature_groups=g)
+    o = FORMS[form](*(to_torch(a, "bf16") for a in (q, k, v)), feature_groups=g)
     assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR
     gpu = to_numpy64(o)
-    check(gpu[0, 0], ref, "bf16", f"M{g} degenerate")
+    check(gpu[0, 0], ref, "bf16", f"M{g} degenerate/{form}")
     assert np.all(gpu[0, 0, [0, 1, 5, 64, 128, 256]] == 0)
 
 
@@ -135,4 +152,4 @@ def test_blockwise_argument_checks():
         kb.kata_fwd_quadratic(q, k, v, feature_groups=2, feature_order=1)
     wb = inputs.gaussian_workload("mg_args_bf16", "bf16", 1, 1, 64, 64, 64, 64, 1)
     with pytest.raises(kb.KataError):
-        kb.kata_fwd_chunked(*dev_tensors(wb), feature_groups=2, impl=kb.KATA_IMPL_TENSOR)
+        kb.kata_fwd_chunked(*dev_tensors(wb), feature_groups=2, inter_chunk=kb.KATA_SCAN, impl=kb.KATA_IMPL_TENSOR)
