@@ -372,6 +372,14 @@ def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
     res["quadratic_c2"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=fl / (ms * 1e-3) / 1e12,
                                frac_of_bf16_burst=fl / (ms * 1e-3) / 1e12 / peaks["bf16_burst"],
                                impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
+    # blockwise map (KATA-Mg): one-pass chunked form on the headline workload, quadratic form on config 2
+    for g in (2, 4):
+        ms = timed(lambda: kb.kata_fwd_chunked(q, k, v, out, feature_groups=g))
+        res[f"chunked_seq_M{g}"] = dict(ms=ms, tokens_per_s=T / (ms * 1e-3), launches=kb.kata_last_launch_count(),
+                                        impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
+        ms = timed(lambda: kb.kata_fwd_quadratic(q2, k2, v2, o2, feature_groups=g))
+        res[f"quadratic_c2_M{g}"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=fl / (ms * 1e-3) / 1e12,
+                                         impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
     # decode step: B=16, H=16, d=64, bf16 tokens, fp32 state in the direct layout (285 MB of state > L2);
     # HBM-bound: the state is read and written once per token
     Bd, Hd, d = 16, 16, 64

@@ -142,6 +142,27 @@ def test_blockwise_states_and_decode(layout, g):
         check(gdec[0, h], ref, "f32", f"M{g} decode after prefill/{layout}")
 
 
+@pytest.mark.parametrize("g", [2, 4])
+def test_blockwise_full_size_sampled_rows(g):
+    """The benchmark shapes: one-pass chunked form at T = 131072 (c4) and the quadratic form on c2, rows sampled
+    from the definition."""
+    import torch
+    from helpers import oracle_rows, sample_picks
+    feat = f"psd_direct:g{g}"
+    for w, form in ((inputs.config(4, 131072), "chunked_seq"), (inputs.config(2), "quadratic")):
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        o = FORMS[form](*dev_tensors(w), feature_groups=g, device_status=st)
+        torch.cuda.synchronize()
+        assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR and int(st.item()) == 0
+        gpu = to_numpy64(o)
+        assert np.all(np.isfinite(gpu))
+        picks = sample_picks(w, 128, 7 + g)
+        ref = oracle_rows(w, picks, feat)
+        got = np.stack([gpu[b, h, t] for b, h, t in picks])
+        check(got, ref, "bf16", f"M{g} {form} {w.name} sampled rows")
+        del o, gpu
+
+
 def test_blockwise_argument_checks():
     import torch
     w = inputs.gaussian_workload("mg_args", "f32", 1, 1, 64, 16, 16, 64, 1)
