@@ -73,7 +73,7 @@ enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2,
  *                 psi_Mg(u) = (u_1 u_1^T, ..., u_g u_g^T) of the normalised row cut into g blocks of d_k/g
  *                 entries ("KATA-Mg"), with <psi(q),psi(k)> = sum_a (q_a . k_a)^2.  The state layouts then hold
  *                 the g blocks one after the other: DIRECT n_psi = g (d_k/g)^2, PACKED n_psi = g m(m+1)/2 with
- *                 m = d_k/g.  Runs on the fp32 kernels.
+ *                 m = d_k/g.
  *  state_layout   layout of the exported prefix states for feature_order 2:
  *                 DIRECT  n_psi = d_k^2, row a*d_k+b holds the (a,b) entry of sum k_hat k_hat^T (x) v;
  *                 PACKED  n_psi = d_k(d_k+1)/2, upper triangle a<=b in row-major order, diagonal
@@ -98,6 +98,14 @@ enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2,
  *                 continues from (prefill -> decode).  Any other entry point: KATA_ERR_INVALID_ARG.
  *  device_status  optional device int, written only on a device-side timeout.
  *  stream         cudaStream_t as void* (null = the legacy default stream).
+ *  s_init, z_init optional device inputs (fp32), both null or both non-null; kata_fwd_chunked with inter_chunk =
+ *                 SEQUENTIAL and feature_order 2 only (anything else: KATA_ERR_INVALID_ARG).  The state before the
+ *                 first token, s_init [B,H,n_psi,d_v], z_init [B,H,n_psi] in state_layout: the call continues a
+ *                 sequence whose earlier tokens are summarised by that state (the recurrence "S_t = S_{t-1} +
+ *                 psi(k_t) v_t^T" started from S_0 = s_init instead of 0), so feeding a long sequence in pieces,
+ *                 each call's s_pre/z_pre being the next call's s_init/z_init, gives the outputs of the one long
+ *                 call.  s_init may equal s_pre (and z_init z_pre): the state is then advanced in place.  Read
+ *                 before anything is written.
  */
 typedef struct kata_opts {
   uint32_t struct_size;
@@ -114,6 +122,8 @@ typedef struct kata_opts {
   float* z_pre;
   int* device_status;
   void* stream;
+  const float* s_init;
+  const float* z_init;
 } kata_opts;
 
 /*

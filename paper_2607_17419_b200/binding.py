@@ -44,6 +44,8 @@ class KataOpts(ctypes.Structure):
         ("z_pre", ctypes.c_void_p),
         ("device_status", ctypes.c_void_p),
         ("stream", ctypes.c_void_p),
+        ("s_init", ctypes.c_void_p),
+        ("z_init", ctypes.c_void_p),
     ]
 
 
@@ -97,7 +99,7 @@ def make_opts(dtype: int, *, feature_order: int = 2, state_layout: int = KATA_LA
               inter_chunk: int = KATA_SEQUENTIAL, impl: int = KATA_IMPL_AUTO, scan_group: int = 0,
               feature_groups: int = 0,
               workspace: int = 0, workspace_bytes: int = 0, s_pre: int = 0, z_pre: int = 0,
-              device_status: int = 0, stream: int = 0) -> KataOpts:
+              device_status: int = 0, stream: int = 0, s_init: int = 0, z_init: int = 0) -> KataOpts:
     o = KataOpts()
     o.struct_size = ctypes.sizeof(KataOpts)
     o.dtype, o.feature_order, o.state_layout = dtype, feature_order, state_layout
@@ -106,6 +108,7 @@ def make_opts(dtype: int, *, feature_order: int = 2, state_layout: int = KATA_LA
     o.workspace, o.workspace_bytes = workspace or None, workspace_bytes
     o.s_pre, o.z_pre = s_pre or None, z_pre or None
     o.device_status, o.stream = device_status or None, stream or None
+    o.s_init, o.z_init = s_init or None, z_init or None
     return o
 
 
@@ -171,7 +174,7 @@ _default_ws = Workspace()
 
 
 def _call(fn: int, q, k, v, out, C: int, *, host_io: bool = False, workspace: Optional[Workspace] = None,
-          s_pre=None, z_pre=None, device_status=None, stream=None, **opt_kw):
+          s_pre=None, z_pre=None, s_init=None, z_init=None, device_status=None, stream=None, **opt_kw):
     import torch
     if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
         raise ValueError("q, k, v must be contiguous [B,H,T,d]")
@@ -185,6 +188,8 @@ def _call(fn: int, q, k, v, out, C: int, *, host_io: bool = False, workspace: Op
     opts = make_opts(_dtype_code(q), stream=stream,
                      s_pre=s_pre.data_ptr() if s_pre is not None else 0,
                      z_pre=z_pre.data_ptr() if z_pre is not None else 0,
+                     s_init=s_init.data_ptr() if s_init is not None else 0,
+                     z_init=z_init.data_ptr() if z_init is not None else 0,
                      device_status=device_status.data_ptr() if device_status is not None else 0, **opt_kw)
     need = kata_workspace_bytes(fn | (KATA_FN_HOST_IO if host_io else 0), B, H, T, d_k, d_v, C, opts)
     ws = workspace if workspace is not None else _default_ws
@@ -208,7 +213,8 @@ def kata_fwd_quadratic(q, k, v, out=None, C: int = 64, **kw):
 
 
 def kata_fwd_chunked(q, k, v, out=None, C: int = 64, **kw):
-    """Chunked-state forward; inter_chunk=KATA_SEQUENTIAL (default) or KATA_SCAN."""
+    """Chunked-state forward; inter_chunk=KATA_SEQUENTIAL (default) or KATA_SCAN.  In the sequential form
+    s_init/z_init give the state before the first token and s_pre/z_pre receive the state after the last."""
     return _call(KATA_FN_CHUNKED, q, k, v, out, C, **kw)
 
 

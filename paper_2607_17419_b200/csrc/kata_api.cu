@@ -27,6 +27,8 @@ struct Opts {
   size_t workspace_bytes;
   float* s_pre;
   float* z_pre;
+  const float* s_init;
+  const float* z_init;
   int* device_status;
   cudaStream_t stream;
 };
@@ -44,6 +46,8 @@ int read_opts(const kata_opts* o, Opts& out) {
   out.workspace_bytes = o->workspace_bytes;
   out.s_pre = o->s_pre;
   out.z_pre = o->z_pre;
+  out.s_init = o->s_init;
+  out.z_init = o->z_init;
   out.device_status = o->device_status;
   out.stream = static_cast<cudaStream_t>(o->stream);
   if (out.dtype != KATA_F32 && out.dtype != KATA_BF16) return KATA_ERR_INVALID_ARG;
@@ -72,8 +76,8 @@ int check_shape(int fn, int B, int H, int T, int d_k, int d_v, int C) {
 
 bool want_tensor(int fn, const Problem& p, const Opts& o) {
   const bool scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || (fn == KATA_FN_CHUNKED && o.inter_chunk == KATA_SCAN);
-  // the tensor-core kernel exports the final state for the plain feature only
-  if (p.groups != 1 && fn == KATA_FN_CHUNKED && o.s_pre != nullptr) return false;
+  // the tensor-core kernel imports and exports the state for the plain feature only
+  if (p.groups != 1 && fn == KATA_FN_CHUNKED && (o.s_pre != nullptr || o.s_init != nullptr)) return false;
   return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn, scan);
 }
 
@@ -187,6 +191,10 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   if (r.o.s_pre != nullptr && !(fn == KATA_FN_CHUNK_STATE_SCAN ||
                                 (fn == KATA_FN_CHUNKED && r.o.inter_chunk == KATA_SEQUENTIAL))) return KATA_ERR_INVALID_ARG;
   if (r.o.s_pre != nullptr && fn == KATA_FN_CHUNKED && r.o.feature_order != 2) return KATA_ERR_UNSUPPORTED_SHAPE;
+  // s_init/z_init: the state before the first token, sequential chunked forward only
+  if ((r.o.s_init == nullptr) != (r.o.z_init == nullptr)) return KATA_ERR_INVALID_ARG;
+  if (r.o.s_init != nullptr && !(fn == KATA_FN_CHUNKED && r.o.inter_chunk == KATA_SEQUENTIAL)) return KATA_ERR_INVALID_ARG;
+  if (r.o.s_init != nullptr && r.o.feature_order != 2) return KATA_ERR_UNSUPPORTED_SHAPE;
   r.p = Problem{q, k, v, out, B, H, T, d_k, d_v, r.o.dtype, r.o.feature_order, r.o.groups};
   r.tensor = want_tensor(fn, r.p, r.o);
   if (r.o.impl == KATA_IMPL_TENSOR && !r.tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
@@ -198,8 +206,8 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
     st = make_plan(fn, r.p, r.o, r.tensor, r.plan, r.state_elems);
     if (st != KATA_OK) return st;
     r.inner_bytes = inner_workspace(fn, r.plan, r.p, r.state_elems);
-    // final-state export of the fp32 path goes through one internal state per head
-    if (fn == KATA_FN_CHUNKED && r.o.s_pre != nullptr && !r.tensor)
+    // state import and final-state export of the fp32 path go through one internal state per head
+    if (fn == KATA_FN_CHUNKED && (r.o.s_pre != nullptr || r.o.s_init != nullptr) && !r.tensor)
       r.inner_bytes = align_up((size_t)B * H * r.state_elems * sizeof(float));
   }
   return KATA_OK;
@@ -213,9 +221,11 @@ int run_device(int fn, Prepared& r, void* ws) {
     else simt_quadratic(r.p, ctx);
   } else {
     const bool use_scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || r.plan.n_groups > 1;
-    if (r.tensor) tc_chunked(r.p, r.plan, use_scan, wsf, r.o.device_status, r.o.s_pre, r.o.z_pre, r.o.state_layout, ctx);
+    if (r.tensor)
+      tc_chunked(r.p, r.plan, use_scan, wsf, r.o.device_status, r.o.s_init, r.o.z_init, r.o.s_pre, r.o.z_pre,
+                 r.o.state_layout, ctx);
     else if (r.p.feature_order == 1) order1_chunked(r.p, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, ctx);
-    else simt_chunked(r.p, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, r.o.state_layout, ctx);
+    else simt_chunked(r.p, r.plan, use_scan, wsf, r.o.s_init, r.o.z_init, r.o.s_pre, r.o.z_pre, r.o.state_layout, ctx);
   }
   if (ctx.status == KATA_OK) {
     g_last_launches = ctx.launches;
@@ -231,6 +241,7 @@ int entry(int fn, const void* q, const void* k, const void* v, void* out, int B,
   if (st != KATA_OK) return st;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return KATA_ERR_ALIGNMENT;
   if (r.o.s_pre != nullptr && (!aligned16(r.o.s_pre) || !aligned16(r.o.z_pre))) return KATA_ERR_ALIGNMENT;
+  if (r.o.s_init != nullptr && (!aligned16(r.o.s_init) || !aligned16(r.o.z_init))) return KATA_ERR_ALIGNMENT;
   if (r.inner_bytes > 0) {
     if (r.o.workspace == nullptr || r.o.workspace_bytes < r.inner_bytes) return KATA_ERR_WORKSPACE_TOO_SMALL;
     if ((reinterpret_cast<uintptr_t>(r.o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;
@@ -270,7 +281,7 @@ int kata_decode_step(const void* q, const void* k, const void* v, void* out, flo
   if (B < 1 || H < 1 || d_k < 1 || d_v < 1) return KATA_ERR_INVALID_ARG;
   if ((long long)B * H > 65535) return KATA_ERR_UNSUPPORTED_SHAPE;
   if (!dim_ok(d_k) || !dim_ok(d_v)) return KATA_ERR_UNSUPPORTED_SHAPE;
-  if (o.s_pre != nullptr) return KATA_ERR_INVALID_ARG;
+  if (o.s_pre != nullptr || o.s_init != nullptr || o.z_init != nullptr) return KATA_ERR_INVALID_ARG;
   if (q == nullptr || k == nullptr || v == nullptr || out == nullptr || S == nullptr || Z == nullptr) return KATA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(S) || !aligned16(Z)) return KATA_ERR_ALIGNMENT;
   const int n_psi = decode_n_psi(d_k, o.state_layout, o.feature_order, o.groups);
@@ -295,6 +306,7 @@ int kata_fwd_host(int fn, const void* q_host, const void* k_host, const void* v_
   int st = prepare(fn, q_host, k_host, v_host, out_host, B, H, T, d_k, d_v, C, opts, true, r);
   if (st != KATA_OK) return st;
   if (r.o.s_pre != nullptr && (!aligned16(r.o.s_pre) || !aligned16(r.o.z_pre))) return KATA_ERR_ALIGNMENT;
+  if (r.o.s_init != nullptr && (!aligned16(r.o.s_init) || !aligned16(r.o.z_init))) return KATA_ERR_ALIGNMENT;
   const Staging s = staging_layout(r.p, r.inner_bytes);
   if (r.o.workspace == nullptr || r.o.workspace_bytes < s.total) return KATA_ERR_WORKSPACE_TOO_SMALL;
   if ((reinterpret_cast<uintptr_t>(r.o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;

@@ -66,8 +66,8 @@ int simt_chunked_slices(int d_k, int d_v);          // CTAs per (b,h,group)
 // (E a multiple of 4), ping-ponging between bufA (input) and bufB; returns the buffer holding the result.
 const float* scan_group_states(float* bufA, float* bufB, int BH, int n_groups, int g_used, size_t E,
                                LaunchCtx& ctx);
-void simt_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre,
-                  float* z_pre, int state_layout, LaunchCtx& ctx);
+void simt_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, const float* s_init,
+                  const float* z_init, float* s_pre, float* z_pre, int state_layout, LaunchCtx& ctx);
 
 // feature_order = 1: rows of q,k are the features (plain normalised linear attention, state d_k x d_v)
 size_t order1_state_elems(int d_k, int d_v);
@@ -86,11 +86,12 @@ bool tc_supported(const Problem& p, int fn, bool scan);
 size_t tc_quadratic_workspace_bytes(const Problem& p);
 void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx);
 void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx);
-void tc_chunked_stream_export(const Problem& p, int* device_status, float* s_final, float* z_final, int state_layout,
-                              LaunchCtx& ctx);
+void tc_chunked_stream_export(const Problem& p, int* device_status, const float* s_init, const float* z_init,
+                              float* s_final, float* z_final, int state_layout, LaunchCtx& ctx);
 size_t tc_chunked_state_elems();
 int tc_chunked_slices();
 void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, int* device_status,
-                float* s_final, float* z_final, int state_layout, LaunchCtx& ctx);
+                const float* s_init, const float* z_init, float* s_final, float* z_final, int state_layout,
+                LaunchCtx& ctx);
 
 }  // namespace kata

@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(NTHR) chunk_simt_kernel(const T* __restrict__ 
                                                            int n_groups,
                                                            const float* __restrict__ init_state,
                                                            float* __restrict__ final_state, int write_out,
-                                                           int groups) {
+                                                           int groups, int init_first) {
   using G = Cfg<D, DV>;
   constexpr int BLK = G::BLK, VS = G::VS, RS = G::RS;
   extern __shared__ __align__(16) float smem[];
@@ -109,8 +109,11 @@ __global__ void __launch_bounds__(NTHR) chunk_simt_kernel(const T* __restrict__ 
   float S[BLK][BLK][VS];
   float Z[BLK][BLK];
   const size_t slot = (size_t)G::NREG * NTHR;
-  if (init_state != nullptr && grp > 0) {
-    const float* src = init_state + ((bh * n_groups + (grp - 1)) * G::NSLICE + slice) * slot + tid;
+  // group grp starts from the state in slot grp - 1 (the prefix before it); with init_first the slots hold the
+  // states the groups start from, slot 0 being the state before the first token
+  const int src_grp = grp - 1 + init_first;
+  if (init_state != nullptr && src_grp >= 0) {
+    const float* src = init_state + ((bh * n_groups + src_grp) * G::NSLICE + slice) * slot + tid;
 #pragma unroll
     for (int i = 0; i < BLK; ++i)
 #pragma unroll
@@ -424,8 +427,49 @@ __global__ void export_final_kernel(const float* __restrict__ fin, float* __rest
   }
 }
 
+// The state before the first token, from the public layouts to the internal state [BH][NSLICE][slot] of a
+// whole-sequence pass (the inverse of export_final_kernel).
+template <int D, int DV>
+__global__ void import_initial_kernel(const float* __restrict__ s_in, const float* __restrict__ z_in,
+                                      float* __restrict__ dst, int layout, int groups) {
+  using G = Cfg<D, DV>;
+  constexpr int BLK = G::BLK, VS = G::VS;
+  const size_t bh = blockIdx.y;
+  const int m = D / groups;
+  const bool packed = layout == KATA_LAYOUT_PACKED;
+  const int per = packed ? m * (m + 1) / 2 : m * m;
+  const int n_psi = groups * per;
+  const size_t slot = (size_t)G::NREG * NTHR;
+  const float* sp = s_in + bh * (size_t)n_psi * DV;
+  const float* zp = z_in + bh * (size_t)n_psi;
+  const int total = G::NSLICE * G::NREG * NTHR;
+  for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x) {
+    const int tid = item % NTHR;
+    const int reg = (item / NTHR) % G::NREG;
+    const int slice = item / (NTHR * G::NREG);
+    const int cc = reg % (VS + 1), ij = reg / (VS + 1), i = ij / BLK, j = ij % BLK;
+    float val = 0.f;
+    if (tid < NPAIR) {
+      int A = 0, t = tid;
+      while (t >= NB - A) { t -= NB - A; ++A; }
+      const int Bq = A + t;
+      const int a = A * BLK + i, b = Bq * BLK + j;
+      const int lo = min(a, b), hi = max(a, b);
+      const int gb = lo / m;
+      if (hi / m == gb) {
+        const int la = lo - gb * m, lb = hi - gb * m;
+        const int row = gb * per + (packed ? la * m - la * (la - 1) / 2 + (lb - la) : la * m + lb);
+        const float scale = (packed && la != lb) ? 0.70710678118654752440f : 1.f;
+        val = scale * (cc < VS ? sp[(size_t)row * DV + slice * VS + cc] : zp[row]);
+      }
+    }
+    dst[(bh * G::NSLICE + slice) * slot + (size_t)reg * NTHR + tid] = val;
+  }
+}
+
 template <typename T, int D, int DV>
-void run(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre, float* z_pre,
+void run(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, const float* s_init, const float* z_init,
+         float* s_pre, float* z_pre,
          int state_layout, LaunchCtx& ctx) {
   using G = Cfg<D, DV>;
   auto kern = chunk_simt_kernel<T, D, DV>;
@@ -441,10 +485,16 @@ void run(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float
   T* o = static_cast<T*>(p.out);
   const int BH = p.B * p.H;
   if (!use_scan) {
-    // whole sequence in one pass; with s_pre/z_pre the state after the last token is exported
+    // whole sequence in one pass; with s_init/z_init it starts from that state, with s_pre/z_pre the state after
+    // the last token is exported (both through the one internal state per head in the workspace)
     float* fin = (s_pre != nullptr) ? ws : nullptr;
+    const float* ini = (s_init != nullptr) ? ws : nullptr;
+    if (ini != nullptr) {
+      import_initial_kernel<D, DV><<<dim3(16, BH), 256, 0, ctx.stream>>>(s_init, z_init, ws, state_layout, p.groups);
+      note_launch(ctx);
+    }
     kern<<<dim3(G::NSLICE, BH, 1), NTHR, smem, ctx.stream>>>(q, k, v, o, p.T, plan.n_chunks, plan.n_chunks,
-                                                            1, nullptr, fin, 1, p.groups);
+                                                            1, ini, fin, 1, p.groups, 1);
     note_launch(ctx);
     if (fin != nullptr) {
       export_final_kernel<D, DV><<<dim3(16, BH), 256, 0, ctx.stream>>>(fin, s_pre, z_pre, state_layout, p.groups);
@@ -460,14 +510,14 @@ void run(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float
   if (NG > 1) {
     // pass 1: local states of all groups but the last (its state is never read)
     kern<<<dim3(G::NSLICE, BH, NG - 1), NTHR, smem, ctx.stream>>>(q, k, v, o, p.T, plan.n_chunks,
-                                                                 plan.chunks_per_group, NG, nullptr, bufA, 0, p.groups);
+                                                                 plan.chunks_per_group, NG, nullptr, bufA, 0, p.groups, 0);
     note_launch(ctx);
     // pass 2: inclusive scan over the first NG-1 group states, ceil(log2(NG-1)) rounds
     incl = scan_group_states(bufA, bufB, BH, NG, NG - 1, E, ctx);
   }
   // pass 3: every group restarts from the prefix before it
   kern<<<dim3(G::NSLICE, BH, NG), NTHR, smem, ctx.stream>>>(q, k, v, o, p.T, plan.n_chunks,
-                                                           plan.chunks_per_group, NG, incl, nullptr, 1, p.groups);
+                                                           plan.chunks_per_group, NG, incl, nullptr, 1, p.groups, 0);
   note_launch(ctx);
   if (s_pre != nullptr && z_pre != nullptr) {
     export_states_kernel<D, DV><<<dim3(plan.n_chunks, BH), 256, 0, ctx.stream>>>(incl, s_pre, z_pre,
@@ -477,22 +527,24 @@ void run(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float
 }
 
 template <typename T, int D>
-void run_dv(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre, float* z_pre,
+void run_dv(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, const float* s_init, const float* z_init,
+            float* s_pre, float* z_pre,
             int layout, LaunchCtx& ctx) {
   switch (p.d_v) {
-    case 16: run<T, D, 16>(p, plan, use_scan, ws, s_pre, z_pre, layout, ctx); break;
-    case 32: run<T, D, 32>(p, plan, use_scan, ws, s_pre, z_pre, layout, ctx); break;
-    default: run<T, D, 64>(p, plan, use_scan, ws, s_pre, z_pre, layout, ctx); break;
+    case 16: run<T, D, 16>(p, plan, use_scan, ws, s_init, z_init, s_pre, z_pre, layout, ctx); break;
+    case 32: run<T, D, 32>(p, plan, use_scan, ws, s_init, z_init, s_pre, z_pre, layout, ctx); break;
+    default: run<T, D, 64>(p, plan, use_scan, ws, s_init, z_init, s_pre, z_pre, layout, ctx); break;
   }
 }
 
 template <typename T>
-void run_d(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre, float* z_pre,
+void run_d(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, const float* s_init, const float* z_init,
+           float* s_pre, float* z_pre,
            int layout, LaunchCtx& ctx) {
   switch (p.d_k) {
-    case 16: run_dv<T, 16>(p, plan, use_scan, ws, s_pre, z_pre, layout, ctx); break;
-    case 32: run_dv<T, 32>(p, plan, use_scan, ws, s_pre, z_pre, layout, ctx); break;
-    default: run_dv<T, 64>(p, plan, use_scan, ws, s_pre, z_pre, layout, ctx); break;
+    case 16: run_dv<T, 16>(p, plan, use_scan, ws, s_init, z_init, s_pre, z_pre, layout, ctx); break;
+    case 32: run_dv<T, 32>(p, plan, use_scan, ws, s_init, z_init, s_pre, z_pre, layout, ctx); break;
+    default: run_dv<T, 64>(p, plan, use_scan, ws, s_init, z_init, s_pre, z_pre, layout, ctx); break;
   }
 }
 
@@ -539,10 +591,10 @@ size_t simt_chunked_state_elems(int d_k, int d_v) {
   }
 }
 
-void simt_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre,
-                  float* z_pre, int state_layout, LaunchCtx& ctx) {
-  if (p.dtype == KATA_F32) run_d<float>(p, plan, use_scan, ws, s_pre, z_pre, state_layout, ctx);
-  else run_d<__nv_bfloat16>(p, plan, use_scan, ws, s_pre, z_pre, state_layout, ctx);
+void simt_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, const float* s_init,
+                  const float* z_init, float* s_pre, float* z_pre, int state_layout, LaunchCtx& ctx) {
+  if (p.dtype == KATA_F32) run_d<float>(p, plan, use_scan, ws, s_init, z_init, s_pre, z_pre, state_layout, ctx);
+  else run_d<__nv_bfloat16>(p, plan, use_scan, ws, s_init, z_init, s_pre, z_pre, state_layout, ctx);
 }
 
 }  // namespace kata

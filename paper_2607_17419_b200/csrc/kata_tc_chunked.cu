@@ -729,9 +729,11 @@ size_t tc_chunked_state_elems() { return (size_t)NSLICE * STATE_PER_SLICE; }
 int tc_chunked_slices() { return NSLICE; }
 
 void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, int* device_status,
-                float* s_final, float* z_final, int state_layout, LaunchCtx& ctx) {
+                const float* s_init, const float* z_init, float* s_final, float* z_final, int state_layout,
+                LaunchCtx& ctx) {
   if (!use_scan) {   // whole sequence in one pass: the token-major streaming kernel
-    if (s_final != nullptr) tc_chunked_stream_export(p, device_status, s_final, z_final, state_layout, ctx);
+    if (s_final != nullptr || s_init != nullptr)
+      tc_chunked_stream_export(p, device_status, s_init, z_init, s_final, z_final, state_layout, ctx);
     else tc_chunked_stream(p, device_status, ctx);
     return;
   }

@@ -17,8 +17,9 @@
 //   intra    P = (Q K^T)^2 masked causally, [O | D] += P [V' | 1/||k||^2]   as in the quadratic form
 //   out      (N_inter + O) / (D_inter + D)             (0 where the denominator is 0)
 // The query norm cancels and is never applied.
-// Compiled a second time with KATA_STREAM_EXPORT (kata_tc_stream_export.cu): the same kernel plus the export of
-// the state after the last token; kept as a separate build so that the plain kernel's code stays as it is.
+// Compiled a second time with KATA_STREAM_EXPORT (kata_tc_stream_export.cu): the same kernel plus the import of
+// a state before the first token and the export of the state after the last token; kept as a separate build so
+// that the plain kernel's code stays as it is.
 //
 // Warps (768 threads, 80 registers each): 0 TMA producer and update-MMA issuer (b-block 3, Z); 1 update-MMA
 // issuer (b-blocks 0-2); 2 read-MMA issuer; 3 intra-tile MMA issuer; 4-11 W builders in two teams (even / odd
@@ -128,8 +129,10 @@ struct SArgs {
   int Tlen;
 #ifdef KATA_STREAM_EXPORT
   int layout;          // KATA_LAYOUT_DIRECT / KATA_LAYOUT_PACKED
-  float* s_final;      // state after the last token, [BH][n_psi][64] in the public layout
+  float* s_final;      // state after the last token, [BH][n_psi][64] in the public layout (null: not exported)
   float* z_final;      // [BH][n_psi]
+  const float* s_init; // state before the first token, same layout (null: zero)
+  const float* z_init;
 #endif
 };
 
@@ -247,6 +250,69 @@ __device__ __noinline__ void export_state(uint32_t tb, uint32_t q4, int t, float
     }
   }
 }
+
+// The state before the first token, from the public layout into the TMEM accumulators (the inverse of
+// export_state; same thread <-> row mapping), and its bf16 snapshot into snapshot buffer 0, which the reads of
+// the first tile use.  One call per thread of the four auxiliary warps, before the pipeline starts.
+__device__ __noinline__ void import_state(uint32_t tb, unsigned char* sp, uint32_t q4, int t, const float* s_init,
+                                          const float* z_init, int layout, int bh, int v0) {
+  const bool packed = layout == KATA_LAYOUT_PACKED;
+  const int n_psi = packed ? D * (D + 1) / 2 : D * D;
+  const float* sf = s_init + (size_t)bh * n_psi * D + v0;
+  const float* zf = z_init + (size_t)bh * n_psi;
+  // entry (a, b) of the symmetric state: DIRECT row a D + b, PACKED the row of (min, max) with sqrt(2) taken out
+  auto srow = [&](int a, int b, float& scale) -> int {
+    if (!packed) { scale = 1.f; return a * D + b; }
+    const int lo = a < b ? a : b, hi = a < b ? b : a;
+    scale = lo == hi ? 1.f : 0.70710678118654752440f;
+    return lo * D - lo * (lo - 1) / 2 + (hi - lo);
+  };
+  const int bloc = t >> 3, vv = t & 7;
+  uint32_t scol = tmem_addr(tb, q4 * 32, COL_S);
+#pragma unroll 1
+  for (int be = 0; be < 4; ++be) {
+    const int b = 16 * be + bloc;
+    const int p = 2 * be + (bloc >> 3);
+    unsigned char* row = sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
+#pragma unroll 1
+    for (int al = 0; al <= be; ++al, scol += 16) {
+      uint32_t z[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        float scale;
+        const int r = srow(16 * al + i, b, scale);
+        z[i] = __float_as_uint(scale * sf[(size_t)r * D + vv]);
+      }
+      tmem_st16(scol, z);
+      snap_store16(row, (sp_koff(p) >> 4) + 2 * al, (uint32_t)vv, z, al < be ? 2.f : 1.f);
+    }
+  }
+  if (q4 < 2) {
+    const int b = t, bz = b >> 4, pz = b >> 3;
+    unsigned char* rowz = sp + sp_block(pz) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
+#pragma unroll 1
+    for (int al = 0; al < 4; ++al) {
+      uint32_t z[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        float scale;
+        const int r = srow(16 * al + i, b, scale);
+        z[i] = __float_as_uint(scale * zf[r]);
+      }
+      tmem_st16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
+      if (al <= bz) snap_store16(rowz, (sp_koff(pz) >> 4) + 2 * al, (uint32_t)(b & 7), z, al < bz ? 2.f : 1.f);
+    }
+  } else {
+    // lanes 64..127 of the Z accumulators: rows of the zero atom, kept at zero
+    uint32_t z[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) z[i] = 0u;
+#pragma unroll 1
+    for (int al = 0; al < 4; ++al) tmem_st16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
+  }
+  tmem_wait_st();
+  fence_async_smem();
+}
 #endif
 
 template <int G>
@@ -317,6 +383,18 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
   bool ok = true;
+#ifdef KATA_STREAM_EXPORT
+  const bool resume = args.s_init != nullptr;       // accumulators and snapshot 0 start from the given state
+  if (resume) {
+    if (warp >= WARP_AUX0)
+      import_state(tb, base + OFF_SP, warp & 3, (warp & 3) * 32 + lane, args.s_init, args.z_init, args.layout, bh, v0);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+  }
+#else
+  constexpr bool resume = false;
+#endif
 
   if (warp == WARP_UB || warp == WARP_U) {
     // =========================== update issuers: S += W^T K ===========================
@@ -359,7 +437,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           tc_fence_after();
           const uint32_t wa = smem_u32(wbuf(wbi)), ka = smem_u32(ktile(s)) + sc * 2048;
           const uint64_t db = at(dB, ka);
-          const uint32_t acc = (j > 0 || sc > 0) ? 1u : 0u;
+          const uint32_t acc = (resume || j > 0 || sc > 0) ? 1u : 0u;
           // b-block beta: N = its a-blocks, the B operand starts at the first feature of its group (32 bytes per a-block)
           if (producer) {
             mma_f16_ss(tb + COL_S + geo::col_s(3), at(dA, wa + 3 * 4096), db + 2 * geo::first(3),
@@ -914,7 +992,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // ---- the state after the last token, from the accumulators to the public layout ----
     if (ok) {
       ok = wait_or_abort(bar(BAR_U_DONE), (nch - 1) & 1, abort_flag);
-      if (ok) export_state(tb, q4, t, args.s_final, args.z_final, args.layout, bh, v0, slice);
+      if (ok && args.s_final != nullptr) export_state(tb, q4, t, args.s_final, args.z_final, args.layout, bh, v0, slice);
     }
 #endif
   }
@@ -968,8 +1046,8 @@ bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T) {
 }  // namespace
 
 #ifdef KATA_STREAM_EXPORT
-void tc_chunked_stream_export(const Problem& p, int* device_status, float* s_final, float* z_final, int state_layout,
-                              LaunchCtx& ctx) {
+void tc_chunked_stream_export(const Problem& p, int* device_status, const float* s_init, const float* z_init,
+                              float* s_final, float* z_final, int state_layout, LaunchCtx& ctx) {
 #else
 void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
 #endif
@@ -991,7 +1069,7 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
   }
 #ifdef KATA_STREAM_EXPORT
   SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T, state_layout,
-          s_final, z_final};
+          s_final, z_final, s_init, z_init};
 #else
   SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T};
 #endif

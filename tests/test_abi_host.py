@@ -39,8 +39,9 @@ def test_version_and_status_strings(L):
 
 
 def test_opts_struct_layout():
-    assert ctypes.sizeof(kb.KataOpts) == 80
+    assert ctypes.sizeof(kb.KataOpts) == 96
     assert kb.KataOpts.workspace.offset == 32 and kb.KataOpts.stream.offset == 72
+    assert kb.KataOpts.s_init.offset == 80 and kb.KataOpts.z_init.offset == 88
 
 
 def call(L, fn, q=256, k=512, v=768, out=1024, B=1, H=1, T=64, d_k=64, d_v=64, C=64, opts=None):
@@ -83,8 +84,21 @@ def test_invalid_arguments(L, fn):
         assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192, feature_order=1)) == SHAPE
         assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096)) == INV
         assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192)) == WS          # fp32 path: one internal state per head
+        # initial state: the same rules
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_init=4096)) == INV
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, z_init=4096)) == INV
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_init=4096, z_init=8192, inter_chunk=kb.KATA_SCAN)) == INV
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_init=4096, z_init=8192, feature_order=1)) == SHAPE
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_init=4096, z_init=8192)) == WS
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_BF16, s_init=4096 + 4, z_init=8192)) == ALIGN
+        # the tensor-core path takes the state without a workspace; the blockwise map goes through the fp32 path
+        o = kb.make_opts(kb.KATA_BF16, s_init=4096, z_init=8192)
+        assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 1, 64, 64, 64, 64, o) == 0
+        o = kb.make_opts(kb.KATA_BF16, s_init=4096, z_init=8192, feature_groups=2)
+        assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 1, 64, 64, 64, 64, o) > 0
     else:
         assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192)) == INV
+        assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_init=4096, z_init=8192)) == INV
 
 
 def test_scan_workspace_and_plan(L):
