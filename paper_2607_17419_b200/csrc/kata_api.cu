@@ -3,6 +3,8 @@
 // every entry point are in include/kata.h.
 #include <cstring>
 
+#include <cmath>
+
 #include "kata_common.cuh"
 
 namespace kata {
@@ -69,7 +71,7 @@ int check_shape(int fn, int B, int H, int T, int d_k, int d_v, int C) {
   if (!dim_ok(d_k) || !dim_ok(d_v)) return KATA_ERR_UNSUPPORTED_SHAPE;
   if (fn != KATA_FN_QUADRATIC) {
     if (C < 1) return KATA_ERR_INVALID_ARG;
-    if (C != kChunk) return KATA_ERR_UNSUPPORTED_SHAPE;
+    if (C != kChunk && C != 2 * kChunk) return KATA_ERR_UNSUPPORTED_SHAPE;   // C = 128: see prepare()
   }
   return KATA_OK;
 }
@@ -82,10 +84,44 @@ bool want_tensor(int fn, const Problem& p, const Opts& o) {
 }
 
 // How the chunk axis is cut into scan groups, and how many floats one group state takes.
-int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, ScanPlan& plan, size_t& state_elems) {
-  plan.n_chunks = (p.T + kChunk - 1) / kChunk;
+int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanPlan& plan, size_t& state_elems) {
+  plan.n_chunks = (p.T + C - 1) / C;
   const int NC = plan.n_chunks;
   const int BH = p.B * p.H;
+  if (tensor && p.feature_order == 1) {
+    // first-order tensor-core kernel: groups of whole 128-token tiles, reduce-then-scan over the groups whatever
+    // the entry point (any grouping of the chunk axis gives the same result up to fp32 re-association)
+    state_elems = tc_order1_state_elems();
+    const int cpt = tc_order1_tile() / C;                 // chunks per tile: 2 or 1
+    int G;
+    if (fn == KATA_FN_CHUNKED && o.inter_chunk == KATA_SEQUENTIAL) {
+      G = NC;
+    } else if (o.scan_group > 0) {
+      G = (o.scan_group + cpt - 1) / cpt * cpt;
+    } else {
+      // Grouped (reduce, scan, restart: 1.5x the HBM traffic, three or more launches) or one pass per head,
+      // whichever the cost model says is faster.  Measured on B200: a CTA walks its tiles at about 1.3 us per
+      // tile (1.75 us for both passes of a group), the kernel streams about 6 GB/ms, the extra launches cost
+      // about 60 us.
+      const double n_tiles = (double)((p.T + tc_order1_tile() - 1) / tc_order1_tile());
+      const double hbm_us = (double)BH * n_tiles * 65536.0 / 6.0e6;
+      const double one_pass = fmax(hbm_us, ceil(BH / 148.0) * n_tiles * 1.3);
+      int ng = (4 * 148 + BH - 1) / BH;                    // about four groups per SM over the run of the kernel
+      if (ng < 2) ng = 2;
+      G = (NC + ng - 1) / ng;
+      if (G < 2 * cpt) G = 2 * cpt;                        // at least two tiles per group
+      G = (G + cpt - 1) / cpt * cpt;
+      if (G > NC) G = NC;
+      const double groups = ceil((double)NC / G), tiles_per_group = (double)G / cpt;
+      const double grouped = fmax(1.5 * hbm_us, ceil(BH * groups / 148.0) * tiles_per_group * 1.75) + 60.0;
+      if (one_pass <= grouped) G = NC;
+    }
+    if (G > NC) G = NC;
+    plan.chunks_per_group = G;
+    plan.n_groups = (NC + G - 1) / G;
+    plan.rounds = plan.n_groups > 2 ? ceil_log2(plan.n_groups - 1) : 0;
+    return KATA_OK;
+  }
   int slices;
   if (tensor) {
     state_elems = tc_chunked_state_elems();
@@ -178,6 +214,7 @@ struct Prepared {
   size_t state_elems;
   size_t inner_bytes;
   bool tensor;
+  int C;
 };
 
 int prepare(int fn, const void* q, const void* k, const void* v, void* out, int B, int H, int T, int d_k,
@@ -198,12 +235,15 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   r.p = Problem{q, k, v, out, B, H, T, d_k, d_v, r.o.dtype, r.o.feature_order, r.o.groups};
   r.tensor = want_tensor(fn, r.p, r.o);
   if (r.o.impl == KATA_IMPL_TENSOR && !r.tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
-  r.plan = ScanPlan{(T + kChunk - 1) / kChunk, 0, 1, 0};
+  r.C = fn == KATA_FN_QUADRATIC ? kChunk : C;
+  r.plan = ScanPlan{(T + r.C - 1) / r.C, 0, 1, 0};
   r.state_elems = 0;
   r.inner_bytes = (fn == KATA_FN_QUADRATIC && r.tensor) ? tc_quadratic_workspace_bytes(r.p) : 0;
   if (fn != KATA_FN_QUADRATIC) {
     if (r.tensor && r.o.s_pre != nullptr && fn == KATA_FN_CHUNK_STATE_SCAN) r.tensor = false;   // per-chunk export: SIMT pipeline
-    st = make_plan(fn, r.p, r.o, r.tensor, r.plan, r.state_elems);
+    // C = 128 (the chunk size of the paper's scan benchmark) exists on the first-order tensor-core path only
+    if (r.C != kChunk && !(r.tensor && r.p.feature_order == 1)) return KATA_ERR_UNSUPPORTED_SHAPE;
+    st = make_plan(fn, r.p, r.o, r.tensor, r.C, r.plan, r.state_elems);
     if (st != KATA_OK) return st;
     r.inner_bytes = inner_workspace(fn, r.plan, r.p, r.state_elems);
     // state import and final-state export of the fp32 path go through one internal state per head
@@ -221,7 +261,9 @@ int run_device(int fn, Prepared& r, void* ws) {
     else simt_quadratic(r.p, ctx);
   } else {
     const bool use_scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || r.plan.n_groups > 1;
-    if (r.tensor)
+    if (r.tensor && r.p.feature_order == 1)
+      tc_order1(r.p, r.plan, use_scan, r.C, wsf, r.o.device_status, ctx);
+    else if (r.tensor)
       tc_chunked(r.p, r.plan, use_scan, wsf, r.o.device_status, r.o.s_init, r.o.z_init, r.o.s_pre, r.o.z_pre,
                  r.o.state_layout, ctx);
     else if (r.p.feature_order == 1) order1_chunked(r.p, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, ctx);

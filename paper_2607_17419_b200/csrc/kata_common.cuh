@@ -94,4 +94,10 @@ void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws
                 const float* s_init, const float* z_init, float* s_final, float* z_final, int state_layout,
                 LaunchCtx& ctx);
 
+// First-order feature on the tensor cores (bf16, d_k = d_v = 64): groups of whole 128-token tiles
+size_t tc_order1_state_elems();
+int tc_order1_tile();
+void tc_order1(const Problem& p, const ScanPlan& plan, bool use_scan, int C, float* ws, int* device_status,
+               LaunchCtx& ctx);
+
 }  // namespace kata

@@ -4,7 +4,10 @@
 namespace kata {
 
 bool tc_supported(const Problem& p, int fn, bool scan) {
-  if (p.dtype != KATA_BF16 || p.d_k != 64 || p.d_v != 64 || p.feature_order != 2) return false;
+  if (p.dtype != KATA_BF16 || p.d_k != 64 || p.d_v != 64) return false;
+  // first-order feature: the chunked and scan forms (the quadratic form stays on the fp32 kernel)
+  if (p.feature_order == 1) return fn == KATA_FN_CHUNKED || fn == KATA_FN_CHUNK_STATE_SCAN;
+  if (p.feature_order != 2) return false;
   // blockwise map (g = 2, 4): the quadratic form and the one-pass chunked form; the scan forms run on the fp32 kernels
   if (p.groups != 1)
     return (fn == KATA_FN_QUADRATIC || (fn == KATA_FN_CHUNKED && !scan)) && (p.groups == 2 || p.groups == 4);
