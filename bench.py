@@ -340,6 +340,43 @@ def run_decode(args):
                           gbs=nbytes / (ms * 1e-3) / 1e9)))
 
 
+def order1_inputs(B, T, dev, seed=11):
+    """Non-negative first-order features (|N(0,1)|-like: uniform here, the kernel's speed does not depend on the
+    values), H = 16, d = 64, bf16: the shapes of the paper's scan benchmark."""
+    import torch
+    g = torch.Generator(device=dev).manual_seed(seed)
+    return tuple(torch.rand(B, 16, T, 64, device=dev, generator=g).to(torch.bfloat16) for _ in range(3))
+
+
+def run_order1(args):
+    """Profiler case of the first-order tensor-core kernel: B=16, H=16, T=8192, C=128 (inputs 805 MB > L2, 256
+    CTAs), one kernel per step in the sequential form, three passes with --mode scan; short line."""
+    import torch
+    from paper_2607_17419_b200 import binding as kb, build as kbuild
+    kbuild.build()
+    torch.cuda.set_device(0)
+    B, T = 16, 8192
+    q, k, v = order1_inputs(B, T, torch.device("cuda", 0))
+    out = torch.empty_like(v)
+    kw = dict(feature_order=1, C=128)
+    if args.mode == "scan":
+        kw.update(inter_chunk=kb.KATA_SCAN, scan_group=8)
+    for _ in range(args.warmup):
+        kb.kata_fwd_chunked(q, k, v, out, **kw)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        kb.kata_fwd_chunked(q, k, v, out, **kw)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    nbytes = B * 16 * T * 512
+    print(json.dumps(dict(case="order1", B=B, T=T, ms_per_step=ms, tokens_per_s=B * T / (ms * 1e-3),
+                          algorithmic_bytes=nbytes, gbs=nbytes / (ms * 1e-3) / 1e9, launches=kb.kata_last_launch_count(),
+                          impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")))
+
+
 def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
     """Separately timed secondary figures: scan forms on the same workload, quadratic form on config 2."""
     import numpy as np
@@ -380,6 +417,19 @@ def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
         ms = timed(lambda: kb.kata_fwd_quadratic(q2, k2, v2, o2, feature_groups=g))
         res[f"quadratic_c2_M{g}"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=fl / (ms * 1e-3) / 1e12,
                                          impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
+    # first-order feature (rows of q, k as features; matched d x d state, C = 128): shapes of the paper's scan
+    # benchmark; HBM-bound, 512 algorithmic bytes per token and head (q, k, v read, o written)
+    for Bo, To in ((1, 8192), (1, 131072), (4, 32768), (16, 8192), (32, 32768)):
+        qo, ko_, vo = order1_inputs(Bo, To, dev)
+        oo = torch.empty_like(vo)
+        nb = Bo * 16 * To * 512
+        for name, fn in (("seq", lambda: kb.kata_fwd_chunked(qo, ko_, vo, oo, feature_order=1, C=128)),
+                         ("scan", lambda: kb.kata_chunk_state_scan(qo, ko_, vo, oo, feature_order=1, C=128))):
+            ms = timed(fn)
+            res[f"order1_{name}_B{Bo}_T{To}"] = dict(ms=ms, tokens_per_s=Bo * To / (ms * 1e-3), gbs=nb / (ms * 1e-3) / 1e9,
+                                                     frac_of_hbm=nb / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                                     launches=kb.kata_last_launch_count())
+        del qo, ko_, vo, oo
     # decode step: B=16, H=16, d=64, bf16 tokens, fp32 state in the direct layout (285 MB of state > L2);
     # HBM-bound: the state is read and written once per token
     Bd, Hd, d = 16, 16, 64
@@ -405,14 +455,17 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="sequential", choices=["sequential", "scan"])
     ap.add_argument("--no-extra", dest="extra", action="store_false")
-    ap.add_argument("--case", default="full", choices=["full", "small", "decode"],
-                    help="small: the same kernel on T=32768 only; decode: the decode step only (both for profiler "
-                         "captures; they print a short line)")
+    ap.add_argument("--case", default="full", choices=["full", "small", "decode", "order1"],
+                    help="small: the same kernel on T=32768 only; decode: the decode step only; order1: the "
+                         "first-order tensor-core kernel on B=16, T=8192 (all for profiler captures; they print a "
+                         "short line)")
     args = ap.parse_args()
     if args.case == "small":
         run_small(args)
     elif args.case == "decode":
         run_decode(args)
+    elif args.case == "order1":
+        run_order1(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
