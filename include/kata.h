@@ -23,9 +23,10 @@
  *   - The caller owns every buffer.  The library allocates nothing, frees nothing and never
  *     synchronises; all work is enqueued on opts->stream.  q,k,v are read-only; out and the
  *     workspace are fully overwritten (no pre-zeroing needed).
- *   - Supported shapes: d_k, d_v in {16,32,64}; C = 64 (the chunked/scan forms); T >= 1
- *     (any; the last chunk is zero-padded as in Algorithm 1 and truncated on output);
- *     B,H >= 1.  The tensor-core (tcgen05) kernels cover bf16 with d_k = d_v = 64; everything
+ *   - Supported shapes: d_k, d_v in {16,32,64}; C = 64 (the chunked/scan forms), and C = 128 for
+ *     feature_order 1 with bf16, d_k = d_v = 64 (the chunk size of the paper's scan benchmark; tensor-core
+ *     path, no s_pre/z_pre); T >= 1 (any; the last chunk is zero-padded as in Algorithm 1 and truncated on
+ *     output); B,H >= 1.  The tensor-core (tcgen05) kernels cover bf16 with d_k = d_v = 64; everything
  *     else runs on the fp32 SIMT kernels.
  *   - Return value: KATA_OK (0) or a negative kata_status.  Errors detectable on the host
  *     launch nothing.  No exceptions, no abort, no device trap.  A bounded device-side wait
@@ -87,7 +88,10 @@ enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2,
  *  impl           AUTO picks the tensor-core kernels where they exist; SIMT / TENSOR force one
  *                 (TENSOR returns KATA_ERR_UNSUPPORTED_SHAPE where it does not exist).
  *  scan_group     chunks per scan group; 0 = library's choice (kata_chunk_state_scan: 1, i.e.
- *                 the paper's per-chunk pipeline, whenever s_pre/z_pre are requested).
+ *                 the paper's per-chunk pipeline, whenever s_pre/z_pre are requested).  The first-order
+ *                 tensor-core path works in tiles of 128 tokens: it rounds the group up to whole tiles, and its
+ *                 own choice may be a single group (one pass per head) when the heads alone fill the GPU;
+ *                 kata_scan_plan reports what will run.
  *  workspace      device scratch of at least kata_workspace_bytes(...) bytes, 256-byte aligned;
  *                 may be null when that size is 0.
  *  s_pre, z_pre   optional device outputs (fp32), both null or both non-null.
