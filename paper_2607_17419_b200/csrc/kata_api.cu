@@ -146,6 +146,13 @@ int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanP
       if (ng > NC) ng = NC;
       G = (NC + ng - 1) / ng;
     }
+  } else if (tensor && o.s_pre == nullptr && o.scan_group == 0) {
+    // tensor-core pipeline without the per-chunk export: the grouping of the scan form of kata_fwd_chunked
+    // (a group state is 0.9 MB per head here, so few large groups)
+    int ng = (2 * 148 + slices * BH - 1) / (slices * BH);
+    if (ng < 2) ng = 2;
+    if (ng > NC) ng = NC;
+    G = (NC + ng - 1) / ng;
   } else {
     if (o.s_pre != nullptr && o.scan_group > 1) return KATA_ERR_INVALID_ARG;
     if (o.s_pre != nullptr) {
@@ -159,6 +166,12 @@ int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanP
       while (G < NC && 2.0 * BH * ((NC + G - 1) / G) * (double)state_elems * 4.0 > cap) G *= 2;
       if (G > NC) G = NC;
     }
+  }
+  // the tensor-core kernel works in tiles of 128 tokens: groups of whole tiles
+  if (tensor && G < NC) {
+    const int cpt = tc_stream_tile() / kChunk;
+    G = (G + cpt - 1) / cpt * cpt;
+    if (G > NC) G = NC;
   }
   plan.chunks_per_group = G;
   plan.n_groups = (NC + G - 1) / G;

@@ -86,8 +86,24 @@ bool tc_supported(const Problem& p, int fn, bool scan);
 size_t tc_quadratic_workspace_bytes(const Problem& p);
 void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx);
 void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx);
-void tc_chunked_stream_export(const Problem& p, int* device_status, const float* s_init, const float* z_init,
-                              float* s_final, float* z_final, int state_layout, LaunchCtx& ctx);
+// State hand-off and groups of tiles for the second build of the streaming kernel (zero-initialise, then set).
+struct StreamIO {
+  const float* s_init;         // state before the first token in the public layout (null: zero)
+  const float* z_init;
+  float* s_final;              // state after the last token in the public layout (null: not exported)
+  float* z_final;
+  int layout;                  // KATA_LAYOUT_DIRECT / KATA_LAYOUT_PACKED
+  const float* init_compact;   // [BH][n_groups][state]: group g starts from slot g - 1 (null: zero)
+  float* final_compact;        // [BH][n_groups][state]: what a group leaves behind (null: not kept)
+  int write_out;               // 0: state only
+  int tiles_per_group;         // used when n_groups > 0
+  int n_groups;                // 0: the whole sequence is one group
+  int launch_groups;           // groups launched (0: n_groups)
+};
+void tc_chunked_stream_export(const Problem& p, int* device_status, const StreamIO& io, LaunchCtx& ctx);
+size_t tc_stream_state_elems();
+int tc_stream_slices();
+int tc_stream_tile();
 size_t tc_chunked_state_elems();
 int tc_chunked_slices();
 void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, int* device_status,

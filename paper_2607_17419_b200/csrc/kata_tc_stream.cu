@@ -133,6 +133,12 @@ struct SArgs {
   float* z_final;      // [BH][n_psi]
   const float* s_init; // state before the first token, same layout (null: zero)
   const float* z_init;
+  // groups of tiles (reduce-then-scan over the chunk axis): grid z = group
+  const float* init_compact;   // [BH][n_groups][8 slices][224 columns][128 lanes]: group g starts from slot g - 1
+  float* final_compact;        // same shape: the state a group leaves behind (null: not kept)
+  int write_out;               // 0: state only (no queries, no output)
+  int tiles_per_group;
+  int n_groups;
 #endif
 };
 
@@ -251,15 +257,29 @@ __device__ __noinline__ void export_state(uint32_t tb, uint32_t q4, int t, float
   }
 }
 
-// The state before the first token, from the public layout into the TMEM accumulators (the inverse of
-// export_state; same thread <-> row mapping), and its bf16 snapshot into snapshot buffer 0, which the reads of
-// the first tile use.  One call per thread of the four auxiliary warps, before the pipeline starts.
+// The accumulators as they are (224 columns x 128 lanes, column-major) for the scan over groups of tiles.
+__device__ __noinline__ void export_compact(uint32_t tb, uint32_t q4, int t, float* dst) {
+  tc_fence_after();
+#pragma unroll 1
+  for (int c = 0; c < 224; c += 16) {
+    uint32_t z[16];
+    tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + c), z);
+    tmem_wait_ld(z);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) dst[(size_t)(c + i) * 128 + t] = __uint_as_float(z[i]);
+  }
+}
+
+// The state before the first token, from the public layout (or, with comp, from the column-major copy of the
+// accumulators that export_compact writes) into the TMEM accumulators (the inverse of export_state; same thread
+// <-> row mapping), and its bf16 snapshot into snapshot buffer 0, which the reads of the first tile use.  One
+// call per thread of the four auxiliary warps, before the pipeline starts.
 __device__ __noinline__ void import_state(uint32_t tb, unsigned char* sp, uint32_t q4, int t, const float* s_init,
-                                          const float* z_init, int layout, int bh, int v0) {
+                                          const float* z_init, int layout, int bh, int v0, const float* comp) {
   const bool packed = layout == KATA_LAYOUT_PACKED;
   const int n_psi = packed ? D * (D + 1) / 2 : D * D;
-  const float* sf = s_init + (size_t)bh * n_psi * D + v0;
-  const float* zf = z_init + (size_t)bh * n_psi;
+  const float* sf = comp ? nullptr : s_init + (size_t)bh * n_psi * D + v0;
+  const float* zf = comp ? nullptr : z_init + (size_t)bh * n_psi;
   // entry (a, b) of the symmetric state: DIRECT row a D + b, PACKED the row of (min, max) with sqrt(2) taken out
   auto srow = [&](int a, int b, float& scale) -> int {
     if (!packed) { scale = 1.f; return a * D + b; }
@@ -269,19 +289,24 @@ __device__ __noinline__ void import_state(uint32_t tb, unsigned char* sp, uint32
   };
   const int bloc = t >> 3, vv = t & 7;
   uint32_t scol = tmem_addr(tb, q4 * 32, COL_S);
+  int col = 0;
 #pragma unroll 1
   for (int be = 0; be < 4; ++be) {
     const int b = 16 * be + bloc;
     const int p = 2 * be + (bloc >> 3);
     unsigned char* row = sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
 #pragma unroll 1
-    for (int al = 0; al <= be; ++al, scol += 16) {
+    for (int al = 0; al <= be; ++al, scol += 16, col += 16) {
       uint32_t z[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
-        float scale;
-        const int r = srow(16 * al + i, b, scale);
-        z[i] = __float_as_uint(scale * sf[(size_t)r * D + vv]);
+        if (comp != nullptr) {
+          z[i] = __float_as_uint(comp[(size_t)(col + i) * 128 + t]);
+        } else {
+          float scale;
+          const int r = srow(16 * al + i, b, scale);
+          z[i] = __float_as_uint(scale * sf[(size_t)r * D + vv]);
+        }
       }
       tmem_st16(scol, z);
       snap_store16(row, (sp_koff(p) >> 4) + 2 * al, (uint32_t)vv, z, al < be ? 2.f : 1.f);
@@ -295,9 +320,13 @@ __device__ __noinline__ void import_state(uint32_t tb, unsigned char* sp, uint32
       uint32_t z[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
-        float scale;
-        const int r = srow(16 * al + i, b, scale);
-        z[i] = __float_as_uint(scale * zf[r]);
+        if (comp != nullptr) {
+          z[i] = __float_as_uint(comp[(size_t)(COL_Z + 16 * al + i) * 128 + t]);
+        } else {
+          float scale;
+          const int r = srow(16 * al + i, b, scale);
+          z[i] = __float_as_uint(scale * zf[r]);
+        }
       }
       tmem_st16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
       if (al <= bz) snap_store16(rowz, (sp_koff(pz) >> 4) + 2 * al, (uint32_t)(b & 7), z, al < bz ? 2.f : 1.f);
@@ -335,13 +364,29 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int slice = blockIdx.x, bh = blockIdx.y;
   const int v0 = slice * VS;
+#ifdef KATA_STREAM_EXPORT
+  // a group of tiles of the sequence (grid z); wo = false: only the state of the group is computed
+  const int grp = blockIdx.z;
+  const int t0 = grp * args.tiles_per_group;
+  const int nch = min((args.Tlen + CT - 1) / CT, t0 + args.tiles_per_group) - t0;
+  if (nch <= 0) return;
+  const bool wo = args.write_out != 0;
+  const size_t comp_elems = (size_t)224 * 128;
+  const float* comp_in = (args.init_compact != nullptr && grp > 0)
+      ? args.init_compact + ((((size_t)bh * args.n_groups + (grp - 1)) * NSLICE + slice) * comp_elems) : nullptr;
+  float* comp_out = args.final_compact != nullptr
+      ? args.final_compact + ((((size_t)bh * args.n_groups + grp) * NSLICE + slice) * comp_elems) : nullptr;
+#else
+  constexpr int t0 = 0;
+  constexpr bool wo = true;
   const int nch = (args.Tlen + CT - 1) / CT;
+#endif
 
   if (tid == 0) {
     abort_s = 0;
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(BAR_K_FULL + s), 1);
-      mbar_init(bar(BAR_K_EMPTY + s), 3);
+      mbar_init(bar(BAR_K_EMPTY + s), wo ? 3 : 2);
       mbar_init(bar(BAR_PREP + s), 128);
       mbar_init(bar(BAR_Y_FULL + s), 1);
       mbar_init(bar(BAR_Y_EMPTY + s), 128);
@@ -384,10 +429,11 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const uint32_t tb = tmem_base_s;
   bool ok = true;
 #ifdef KATA_STREAM_EXPORT
-  const bool resume = args.s_init != nullptr;       // accumulators and snapshot 0 start from the given state
+  const bool resume = args.s_init != nullptr || comp_in != nullptr;   // accumulators and snapshot 0 start from a given state
   if (resume) {
     if (warp >= WARP_AUX0)
-      import_state(tb, base + OFF_SP, warp & 3, (warp & 3) * 32 + lane, args.s_init, args.z_init, args.layout, bh, v0);
+      import_state(tb, base + OFF_SP, warp & 3, (warp & 3) * 32 + lane, args.s_init, args.z_init, args.layout, bh, v0,
+                   comp_in);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -410,24 +456,24 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int s = j & 1;
         if (!wait_or_abort(bar(BAR_K_EMPTY + s), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
         mbar_arrive_expect_tx(bar(BAR_K_FULL + s), 16384);
-        tma_load_3d(ktile(s), &tmK, bar(BAR_K_FULL + s), 0, j * CT, bh);
+        tma_load_3d(ktile(s), &tmK, bar(BAR_K_FULL + s), 0, (t0 + j) * CT, bh);
         return true;
       };
       auto load_q = [&](int j) -> bool {     // one staging buffer: free once the previous tile was copied to TMEM
         if (!wait_or_abort(bar(BAR_QS_EMPTY), (j & 1) ^ 1, abort_flag)) return false;
         mbar_arrive_expect_tx(bar(BAR_Q_FULL), 16384);
-        tma_load_3d(qtile, &tmQ, bar(BAR_Q_FULL), 0, j * CT, bh);
+        tma_load_3d(qtile, &tmQ, bar(BAR_Q_FULL), 0, (t0 + j) * CT, bh);
         return true;
       };
       if (producer) {
-        ok = load_k(0) && load_q(0);
+        ok = load_k(0) && (!wo || load_q(0));
         if (ok && nch > 1) ok = load_k(1);
       }
       uint32_t wbi = 0, wph = 0;             // W buffer of the step and the parity of its phase
       for (int j = 0; j < nch && ok; ++j) {
         const int s = j & 1;
         ok = wait_or_abort(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag);
-        if (ok && j > 0) ok = wait_or_abort(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
+        if (ok && wo && j > 0) ok = wait_or_abort(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
         // the key stage of tile j - 1 is free once that tile's consumers are through: refill it with tile j + 1
         if (ok && producer && j > 0 && j + 1 < nch) ok = load_k(j + 1);
 #pragma unroll 1
@@ -456,15 +502,17 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (++wbi == NWBUF) { wbi = 0; wph ^= 1; }
         }
         if (!ok) break;
-        mma_commit(bar(BAR_U_DONE));
+        // state-only pass: nobody looks at the state between the tiles, one commit after the last update (a parity
+        // wait cannot tell phases two apart)
+        if (wo || j + 1 == nch) mma_commit(bar(BAR_U_DONE));
         mma_commit(bar(BAR_K_EMPTY + s));
         // the query staging buffer is free once tile j was copied to TMEM (at the end of tile j - 1)
-        if (producer && j + 1 < nch) ok = load_q(j + 1);
+        if (producer && wo && j + 1 < nch) ok = load_q(j + 1);
       }
     }
   } else if (warp == WARP_R) {
     // =========================== read issuer: Y = Q S'^T, 8 pieces ===========================
-    if (lane == 0) {
+    if (lane == 0 && wo) {
       const uint32_t idR = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 80);
       const uint64_t dS = smem_desc(0, 16, 1024, kSwizzle128B);
       const uint32_t spa = smem_u32(base + OFF_SP);
@@ -491,7 +539,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
   } else if (warp == WARP_I) {
     // =========================== intra-tile issuer: scores and [O | D] ===========================
-    if (lane == 0) {
+    if (lane == 0 && wo) {
       constexpr int NP = geo::NP, KH = geo::KH;
       const uint32_t idQK = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, KH);
       const uint32_t idPV = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 16);
@@ -666,7 +714,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
            wait_or_abort(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
       // team 1 copies its share of the state after tile j - 1 before its first step of tile j, team 0 after
       // its first step: either way right when the update of tile j - 1 completes
-      if (ok && team == 1 && j > 0) ok = snapshot_share(j - 1);
+      if (ok && wo && team == 1 && j > 0) ok = snapshot_share(j - 1);
 #pragma unroll 1
       for (int sc = team; sc < 8 && ok; sc += 2) {
         const int t = sc * 16 + tk;
@@ -700,7 +748,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         // this team's next step is two steps on: two buffers further in the ring of three
         wbi += 2;
         if (wbi >= NWBUF) { wbi -= NWBUF; wph ^= 1; }
-        if (sc == 0 && j > 0) ok = snapshot_share(j - 1);
+        if (wo && sc == 0 && j > 0) ok = snapshot_share(j - 1);
       }
     }
   } else if (warp < WARP_AUX0) {
@@ -712,7 +760,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int t = q4 * 32 + lane;
     float* part = reinterpret_cast<float*>(base + OFF_PART);
     const uint32_t ycol = tmem_addr(tb, q4 * 32, COL_Y + team * 80);
-    for (int j = 0; j < nch && ok; ++j) {
+    for (int j = 0; j < nch && ok && wo; ++j) {
       ok = wait_or_abort(bar(BAR_QT_FULL), j & 1, abort_flag);    // the multipliers come from the TMEM copy of the query tile
       if (!ok) break;
       tc_fence_after();
@@ -797,7 +845,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       mbar_arrive(bar(BAR_O_EMPTY));
       const float den = accz + __uint_as_float(o[8]);
       const float inv = den > 0.f ? 1.f / den : 0.f;
-      const int tok = j * CT + t;
+      const int tok = (t0 + j) * CT + t;
       if (tok < args.Tlen) {
         uint4 pkt;
         pkt.x = pack_bf16((acc[0].x + __uint_as_float(o[0])) * inv, (acc[0].y + __uint_as_float(o[1])) * inv);
@@ -812,7 +860,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const uint32_t q4 = warp & 3;
     const int t = q4 * 32 + lane;       // token of the tile, and TMEM lane
     auto load_v = [&](int j) -> uint4 {
-      const int tok = j * CT + t;
+      const int tok = (t0 + j) * CT + t;
       if (j < nch && tok < args.Tlen)
         return *reinterpret_cast<const uint4*>(args.v + ((size_t)bh * args.Tlen + tok) * D + v0);
       return make_uint4(0u, 0u, 0u, 0u);
@@ -886,7 +934,14 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       mbar_arrive(bar(BAR_SNAP_ST));
     };
     uint4 vnext = load_v(0);
-    for (int j = -1; j < nch && ok; ++j) {
+    if (!wo) {
+      // state-only pass: key scales and v' of every tile, nothing else
+      for (int j = 0; j < nch && ok; ++j) {
+        ok = prep(j, vnext);
+        vnext = load_v(j + 1);
+      }
+    }
+    for (int j = -1; j < nch && ok && wo; ++j) {
       // ---- scales of the next tile, so that its W rows can be built during this tile's update ----
       if (j + 1 < nch) {
         ok = prep(j + 1, vnext);
@@ -989,10 +1044,11 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     }
 #ifdef KATA_STREAM_EXPORT
-    // ---- the state after the last token, from the accumulators to the public layout ----
+    // ---- the state after the last token, from the accumulators to the public layout or as it is ----
     if (ok) {
-      ok = wait_or_abort(bar(BAR_U_DONE), (nch - 1) & 1, abort_flag);
+      ok = wait_or_abort(bar(BAR_U_DONE), wo ? (nch - 1) & 1 : 0, abort_flag);
       if (ok && args.s_final != nullptr) export_state(tb, q4, t, args.s_final, args.z_final, args.layout, bh, v0, slice);
+      if (ok && comp_out != nullptr) export_compact(tb, q4, t, comp_out);
     }
 #endif
   }
@@ -1046,8 +1102,11 @@ bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T) {
 }  // namespace
 
 #ifdef KATA_STREAM_EXPORT
-void tc_chunked_stream_export(const Problem& p, int* device_status, const float* s_init, const float* z_init,
-                              float* s_final, float* z_final, int state_layout, LaunchCtx& ctx) {
+size_t tc_stream_state_elems() { return (size_t)NSLICE * 224 * 128; }
+int tc_stream_slices() { return NSLICE; }
+int tc_stream_tile() { return CT; }
+
+void tc_chunked_stream_export(const Problem& p, int* device_status, const StreamIO& io, LaunchCtx& ctx) {
 #else
 void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
 #endif
@@ -1058,7 +1117,7 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
     return;
   }
 #ifdef KATA_STREAM_EXPORT
-  auto kern = tc_stream_kernel<1>;       // the state export covers the plain feature
+  auto kern = tc_stream_kernel<1>;       // state import / export and groups cover the plain feature
 #else
   auto kern = p.groups == 1 ? tc_stream_kernel<1> : p.groups == 2 ? tc_stream_kernel<2> : tc_stream_kernel<4>;
 #endif
@@ -1068,12 +1127,17 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
     return;
   }
 #ifdef KATA_STREAM_EXPORT
-  SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T, state_layout,
-          s_final, z_final, s_init, z_init};
+  const int n_tiles = (p.T + CT - 1) / CT;
+  const int n_groups = io.n_groups > 0 ? io.n_groups : 1;
+  SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T, io.layout,
+          io.s_final, io.z_final, io.s_init, io.z_init, io.init_compact, io.final_compact, io.write_out,
+          io.n_groups > 0 ? io.tiles_per_group : n_tiles, n_groups};
+  const int launch_groups = io.launch_groups > 0 ? io.launch_groups : n_groups;
+  kern<<<dim3(NSLICE, BH, launch_groups), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, a);
 #else
   SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T};
-#endif
   kern<<<dim3(NSLICE, BH, 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, a);
+#endif
   note_launch(ctx);
 }
 
