@@ -30,6 +30,8 @@ Forms, all of which must agree to rounding:
                    chunk-local states, exclusive prefix (running sum or
                    log-depth doubling), chunk output
   gate_decomposition   Proposition 1 (output-level gating)
+  kata_quadratic_bwd   gradients of the definition with respect to q, k, v (chain rule
+                   through o = N/D, the weights and the normalisation)
 
 feature="identity" treats the rows of q,k as already-mapped features (the
 setting the scan appendix analyses): no normalisation, no lift.
@@ -207,6 +209,53 @@ def kata_recurrent(q, k, v, feature: str = "psd_direct"):
         if den != 0:
             o[t] = (fq[t] @ S) / den
     return o
+
+
+# ---------------------------------------------------------------------------
+# backward of the definition (vector-Jacobian product)
+# ---------------------------------------------------------------------------
+
+def kata_quadratic_bwd(q, k, v, dout, feature: str = "psd_direct"):
+    """Gradients of L = sum(dout * o) for o = kata_quadratic(q, k, v, feature)[0], by the chain rule through the
+    definition in the order it is written: o = N / D, N = W V, D = W 1, W = tril(<psi(q_hat), psi(k_hat)>),
+    x_hat = x / ||x||.  Returns (dq, dk, dv).  Rows with D = 0 have o = 0 identically in a neighbourhood of
+    the inputs that keeps D = 0 and contribute nothing; a zero row of q or k has a zero feature and gets a zero
+    gradient (the reading of the forward: the feature of a zero row is the constant 0)."""
+    q = np.asarray(q, np.float64)
+    k = np.asarray(k, np.float64)
+    v = np.asarray(v, np.float64)
+    dout = np.asarray(dout, np.float64)
+    base, g = split_feature(feature)
+    W = causal_weights(q, k, feature)
+    D = W.sum(axis=1)
+    o = _safe_div(W @ v, D)
+    live = D != 0
+    invD = np.zeros_like(D)
+    invD[live] = 1.0 / D[live]
+    # o_t = sum_i W_ti v_i / D_t:  dL/dW_ti = dout_t . (v_i - o_t) / D_t  (i <= t),  dL/dv_i = sum_t (W_ti / D_t) dout_t
+    G = np.tril((dout @ v.T - np.sum(dout * o, axis=1)[:, None]) * invD[:, None])
+    dv = (W * invD[:, None]).T @ dout
+    if base == "identity":
+        return G @ k, G.T @ q, dv          # W_ti = q_t . k_i
+    qh, kh = normalize_rows(q), normalize_rows(k)
+    d = q.shape[1]
+    m = d // g
+    dqh, dkh = np.zeros_like(q), np.zeros_like(k)
+    for a in range(g):                      # W_ti = sum_a (qh_t,a . kh_i,a)^2
+        sl = slice(a * m, (a + 1) * m)
+        E = 2.0 * G * (qh[:, sl] @ kh[:, sl].T)
+        dqh[:, sl] = E @ kh[:, sl]
+        dkh[:, sl] = E.T @ qh[:, sl]
+
+    def through_normalisation(x, xh, dxh):  # x_hat = x/||x||:  dx = (dx_hat - x_hat (x_hat . dx_hat)) / ||x||
+        n = np.sqrt(np.sum(x * x, axis=1))
+        out = np.zeros_like(x)
+        nz = n > 0
+        proj = dxh - xh * np.sum(xh * dxh, axis=1, keepdims=True)
+        out[nz] = proj[nz] / n[nz, None]
+        return out
+
+    return through_normalisation(q, qh, dqh), through_normalisation(k, kh, dkh), dv
 
 
 def kata_decode_step(S, Z, q, k, v, feature: str = "psd_direct"):

@@ -475,3 +475,80 @@ def test_blockwise_feature_sizes_and_kernel():
         ko.apply_feature(q, "psd_direct:g3")
     with pytest.raises(ValueError):
         ko.apply_feature(q, "identity:g2")
+
+
+# ---------------------------------------------------------------------------
+# backward of the definition
+# ---------------------------------------------------------------------------
+
+def _loss(q, k, v, dout, feature):
+    return float(np.sum(dout * ko.kata_quadratic(q, k, v, feature)[0]))
+
+
+@pytest.mark.parametrize("feature", ["psd_direct", "psd_direct:g2", "psd_packed:g4", "identity"])
+def test_backward_matches_central_differences(feature):
+    """Every entry of dq, dk, dv against (L(x + h e) - L(x - h e)) / 2h of the forward definition."""
+    r = np.random.default_rng(71)
+    T, d, dv = 9, 8, 5
+    q, k, v, dout = r.normal(size=(T, d)), r.normal(size=(T, d)), r.normal(size=(T, dv)), r.normal(size=(T, dv))
+    if feature == "identity":
+        q, k = np.abs(q) + 0.1, np.abs(k) + 0.1          # keep the normaliser away from 0
+    dq, dk, dvv = ko.kata_quadratic_bwd(q, k, v, dout, feature)
+    h = 1e-6
+    for name, x, grad in (("q", q, dq), ("k", k, dk), ("v", v, dvv)):
+        num = np.zeros_like(x)
+        for idx in np.ndindex(*x.shape):
+            old = x[idx]
+            x[idx] = old + h
+            lp = _loss(q, k, v, dout, feature)
+            x[idx] = old - h
+            lm = _loss(q, k, v, dout, feature)
+            x[idx] = old
+            num[idx] = (lp - lm) / (2 * h)
+        assert np.max(np.abs(num - grad)) <= 2e-7 * max(1.0, np.abs(grad).max()), name
+
+
+def test_backward_invariants():
+    r = np.random.default_rng(72)
+    T, d, dv = 40, 16, 12
+    q, k, v, dout = r.normal(size=(T, d)), r.normal(size=(T, d)), r.normal(size=(T, dv)), r.normal(size=(T, dv))
+    for feature in ("psd_direct", "psd_direct:g2", "psd_direct:g4"):
+        dq, dk, dvv = ko.kata_quadratic_bwd(q, k, v, dout, feature)
+        # o does not change when a query or a key row is rescaled (degree 0): Euler's relation per row
+        assert np.max(np.abs(np.sum(dq * q, axis=1))) <= 1e-12
+        assert np.max(np.abs(np.sum(dk * k, axis=1))) <= 1e-12
+        # adding one vector c to every value row adds c to every output row: sum_i dv_i = sum_t dout_t
+        assert np.max(np.abs(dvv.sum(axis=0) - dout.sum(axis=0))) <= 1e-12
+        # packed and direct coordinates are the same function of q, k
+        dq2, dk2, dv2 = ko.kata_quadratic_bwd(q, k, v, dout, feature.replace("direct", "packed"))
+        assert np.max(np.abs(dq - dq2)) <= 1e-13 and np.max(np.abs(dk - dk2)) <= 1e-13 and np.max(np.abs(dvv - dv2)) <= 1e-13
+    # first-order feature: degree 0 in the common scale of ALL keys only (one relation in total)
+    qp, kp = np.abs(q) + 0.1, np.abs(k) + 0.1
+    dq, dk, dvv = ko.kata_quadratic_bwd(qp, kp, v, dout, "identity")
+    assert abs(np.sum(dk * kp)) <= 1e-10 and np.max(np.abs(np.sum(dq * qp, axis=1))) <= 1e-10
+    # token 0 sees only itself: o_0 = v_0 whatever q_0, k_0 are
+    dq, dk, dvv = ko.kata_quadratic_bwd(q[:1], k[:1], v[:1], dout[:1])
+    assert np.max(np.abs(dq)) <= 1e-12 and np.max(np.abs(dk)) <= 1e-12 and np.allclose(dvv, dout[:1])
+
+
+def test_backward_zero_rows_and_dead_denominators():
+    r = np.random.default_rng(73)
+    T, d, dv = 12, 8, 4
+    q, k, v, dout = r.normal(size=(T, d)), r.normal(size=(T, d)), r.normal(size=(T, dv)), r.normal(size=(T, dv))
+    k[0] = 0
+    k[1] = 0            # rows 0, 1 have D = 0
+    k[5] = 0
+    q[7] = 0
+    dq, dk, dvv = ko.kata_quadratic_bwd(q, k, v, dout)
+    assert np.all(np.isfinite(dq)) and np.all(np.isfinite(dk)) and np.all(np.isfinite(dvv))
+    assert np.all(dk[[0, 1, 5]] == 0) and np.all(dq[[0, 1, 7]] == 0) and np.all(dvv[[0, 1, 5]] == 0)
+    # rows 0, 1 are dead as keys (zero feature) and as queries (D = 0): the rest is the problem without them
+    keep = list(range(2, T))
+    dq2, dk2, dv2 = ko.kata_quadratic_bwd(q[keep], k[keep], v[keep], dout[keep])
+    assert np.allclose(dq[keep], dq2, atol=1e-13) and np.allclose(dk[keep], dk2, atol=1e-13)
+    assert np.allclose(dvv[keep], dv2, atol=1e-13)
+    # a key with a zero feature carries zero weight: its value row does not matter to anything
+    v2 = v.copy()
+    v2[5] += 100.0
+    dq3, dk3, dv3 = ko.kata_quadratic_bwd(q, k, v2, dout)
+    assert np.allclose(dq3, dq, atol=1e-12) and np.allclose(dk3, dk, atol=1e-12) and np.allclose(dv3, dvv, atol=1e-12)
