@@ -60,7 +60,8 @@ enum { KATA_F32 = 0, KATA_BF16 = 1 };                 /* kata_opts.dtype        
 enum { KATA_LAYOUT_DIRECT = 0, KATA_LAYOUT_PACKED = 1 }; /* kata_opts.state_layout */
 enum { KATA_SEQUENTIAL = 0, KATA_SCAN = 1 };          /* kata_opts.inter_chunk    */
 enum { KATA_IMPL_AUTO = 0, KATA_IMPL_SIMT = 1, KATA_IMPL_TENSOR = 2 }; /* kata_opts.impl */
-enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2, KATA_FN_DECODE_STEP = 3 };
+enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2, KATA_FN_DECODE_STEP = 3,
+       KATA_FN_BWD_QUADRATIC = 4 };
 
 /*
  * Options (plain data; zero-initialise, then set struct_size = sizeof(kata_opts)).
@@ -178,6 +179,21 @@ int kata_chunk_state_scan(const void* q, const void* k, const void* v, void* out
  */
 int kata_decode_step(const void* q, const void* k, const void* v, void* out, float* S, float* Z,
                      int B, int H, int d_k, int d_v, const kata_opts* opts);
+
+/*
+ * Backward of the forward pass: given dout = dL/dout [B,H,T,d_v], writes dq, dk [B,H,T,d_k] and dv [B,H,T,d_v]
+ * (element type opts->dtype, device pointers, 16-byte aligned, fully overwritten), the gradients of
+ * L = sum(dout * out) through out_t = sum_{i<=t} w_ti v_i / sum_{i<=t} w_ti, the weights w_ti and the l2
+ * normalisation of the rows (chain rule through the definition; the forms of the forward are one function, so
+ * this is the backward of all of them).  Evaluated tile by tile like kata_fwd_quadratic: the forward is
+ * recomputed (no saved activations are needed), O(T^2) work, fp32 arithmetic, every sum in a fixed order
+ * (bit-reproducible).  Rows whose normaliser is 0 (out = 0) and zero rows of q or k get zero gradients.
+ * feature_order, feature_groups as in the forward; inter_chunk, scan_group, state_layout are ignored;
+ * s_pre/z_pre/s_init/z_init must be null; impl = KATA_IMPL_TENSOR returns KATA_ERR_UNSUPPORTED_SHAPE (fp32 kernels
+ * only).  Workspace: kata_workspace_bytes(KATA_FN_BWD_QUADRATIC, B, H, T, d_k, d_v, 0, opts) (two floats per row).
+ */
+int kata_bwd_quadratic(const void* q, const void* k, const void* v, const void* dout, void* dq, void* dk, void* dv,
+                       int B, int H, int T, int d_k, int d_v, const kata_opts* opts);
 
 /*
  * Same computation as entry point `fn` (a KATA_FN_* value) but q,k,v,out are HOST pointers

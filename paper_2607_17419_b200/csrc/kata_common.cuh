@@ -69,6 +69,10 @@ const float* scan_group_states(float* bufA, float* bufB, int BH, int n_groups, i
 void simt_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, const float* s_init,
                   const float* z_init, float* s_pre, float* z_pre, int state_layout, LaunchCtx& ctx);
 
+// Backward of the quadratic form (fp32 arithmetic; any supported shape and element type)
+size_t simt_bwd_workspace_elems(int BH, int T);
+void simt_bwd_quadratic(const Problem& p, const void* dout, void* dq, void* dk, void* dv, float* stats, LaunchCtx& ctx);
+
 // feature_order = 1: rows of q,k are the features (plain normalised linear attention, state d_k x d_v)
 size_t order1_state_elems(int d_k, int d_v);
 void order1_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre,

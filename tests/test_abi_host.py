@@ -158,3 +158,20 @@ def test_decode_step_argument_checks(L):
     o = kb.make_opts(kb.KATA_F32, feature_order=1)
     assert kb.kata_workspace_bytes(kb.KATA_FN_DECODE_STEP, 1, 1, 1, 16, 16, 0, o) == 256   # 17 floats, rounded up
     assert kb.decode_n_psi(64) == 4096 and kb.decode_n_psi(64, 2, kb.KATA_LAYOUT_PACKED) == 2080 and kb.decode_n_psi(64, 1) == 64
+
+
+def test_backward_argument_checks(L):
+    INV, SHAPE, ALIGN, WS = -1, -2, -3, -4
+    def bwd(q=4096, k=4096, v=4096, dout=4096, dq=4096, dk=4096, dv=4096, B=2, H=2, T=100, d_k=64, d_v=64, opts=None):
+        o = opts if opts is not None else kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 30)
+        return L.kata_bwd_quadratic(q, k, v, dout, dq, dk, dv, B, H, T, d_k, d_v, ctypes.byref(o))
+
+    assert bwd(q=0) == INV and bwd(dout=0) == INV and bwd(dv=0) == INV and bwd(T=0) == INV
+    assert bwd(d_k=48) == SHAPE and bwd(d_v=8) == SHAPE
+    assert bwd(dq=4100) == ALIGN
+    assert bwd(opts=kb.make_opts(kb.KATA_F32)) == WS
+    assert bwd(opts=kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 30, impl=kb.KATA_IMPL_TENSOR)) == SHAPE
+    assert bwd(opts=kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 30, feature_groups=3)) == INV
+    assert bwd(opts=kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 30, s_pre=4096, z_pre=8192)) == INV
+    o = kb.make_opts(kb.KATA_BF16)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 64, 64, 0, o) == (2 * 3 * 100 * 2 * 4 + 255) // 256 * 256
