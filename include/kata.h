@@ -189,8 +189,9 @@ int kata_decode_step(const void* q, const void* k, const void* v, void* out, flo
  * recomputed (no saved activations are needed), O(T^2) work, fp32 arithmetic, every sum in a fixed order
  * (bit-reproducible).  Rows whose normaliser is 0 (out = 0) and zero rows of q or k get zero gradients.
  * feature_order, feature_groups as in the forward; inter_chunk, scan_group, state_layout are ignored;
- * s_pre/z_pre/s_init/z_init must be null; impl = KATA_IMPL_TENSOR returns KATA_ERR_UNSUPPORTED_SHAPE (fp32 kernels
- * only).  Workspace: kata_workspace_bytes(KATA_FN_BWD_QUADRATIC, B, H, T, d_k, d_v, 0, opts) (two floats per row).
+ * s_pre/z_pre/s_init/z_init must be null.  Tensor-core kernels for bf16, d_k = d_v = 64, feature_groups 1 (the
+ * weights P and E pass through bf16 there, as P does in the forward); fp32 kernels for everything else.
+ * Workspace: kata_workspace_bytes(KATA_FN_BWD_QUADRATIC, B, H, T, d_k, d_v, 0, opts).
  */
 int kata_bwd_quadratic(const void* q, const void* k, const void* v, const void* dout, void* dq, void* dk, void* dv,
                        int B, int H, int T, int d_k, int d_v, const kata_opts* opts);

@@ -83,6 +83,12 @@ bool want_tensor(int fn, const Problem& p, const Opts& o) {
   return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn, scan);
 }
 
+// The tensor-core backward covers bf16, d_k = d_v = 64, the full rank-one feature.
+bool bwd_tensor(const Problem& p, const Opts& o) {
+  return o.impl != KATA_IMPL_SIMT && p.dtype == KATA_BF16 && p.d_k == 64 && p.d_v == 64 && p.feature_order == 2 &&
+         p.groups == 1;
+}
+
 // How the chunk axis is cut into scan groups, and how many floats one group state takes.
 int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanPlan& plan, size_t& state_elems) {
   plan.n_chunks = (p.T + C - 1) / C;
@@ -364,23 +370,25 @@ int kata_bwd_quadratic(const void* q, const void* k, const void* v, const void* 
   if ((long long)B * H > 65535) return KATA_ERR_UNSUPPORTED_SHAPE;
   if (!dim_ok(d_k) || !dim_ok(d_v)) return KATA_ERR_UNSUPPORTED_SHAPE;
   if (o.s_pre != nullptr || o.s_init != nullptr || o.z_init != nullptr) return KATA_ERR_INVALID_ARG;
-  if (o.impl == KATA_IMPL_TENSOR) return KATA_ERR_UNSUPPORTED_SHAPE;
+  const Problem p{q, k, v, nullptr, B, H, T, d_k, d_v, o.dtype, o.feature_order, o.groups};
+  const bool tensor = bwd_tensor(p, o);
+  if (o.impl == KATA_IMPL_TENSOR && !tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
   if (q == nullptr || k == nullptr || v == nullptr || dout == nullptr || dq == nullptr || dk == nullptr || dv == nullptr)
     return KATA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) ||
       !aligned16(dv))
     return KATA_ERR_ALIGNMENT;
-  const size_t need = align_up(simt_bwd_workspace_elems(B * H, T) * sizeof(float));
+  const size_t need = tensor ? align_up(tc_bwd_workspace_bytes(p)) : align_up(simt_bwd_workspace_elems(B * H, T) * sizeof(float));
   if (o.workspace == nullptr || o.workspace_bytes < need) return KATA_ERR_WORKSPACE_TOO_SMALL;
   if ((reinterpret_cast<uintptr_t>(o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;
   st = check_arch();
   if (st != KATA_OK) return st;
   LaunchCtx ctx{o.stream, 0, KATA_OK};
-  const Problem p{q, k, v, nullptr, B, H, T, d_k, d_v, o.dtype, o.feature_order, o.groups};
-  simt_bwd_quadratic(p, dout, dq, dk, dv, static_cast<float*>(o.workspace), ctx);
+  if (tensor) tc_bwd_quadratic(p, dout, dq, dk, dv, o.workspace, o.device_status, ctx);
+  else simt_bwd_quadratic(p, dout, dq, dk, dv, static_cast<float*>(o.workspace), ctx);
   if (ctx.status == KATA_OK) {
     g_last_launches = ctx.launches;
-    g_last_impl = KATA_IMPL_SIMT;
+    g_last_impl = tensor ? KATA_IMPL_TENSOR : KATA_IMPL_SIMT;
   }
   return ctx.status;
 }
@@ -427,6 +435,8 @@ size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C
   if (fn == KATA_FN_BWD_QUADRATIC) {    // C is ignored
     Opts o;
     if (host_io || read_opts(opts, o) != KATA_OK || B < 1 || H < 1 || T < 1 || !dim_ok(d_k) || !dim_ok(d_v)) return 0;
+    const Problem p{nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, o.dtype, o.feature_order, o.groups};
+    if (bwd_tensor(p, o)) return align_up(tc_bwd_workspace_bytes(p));
     return align_up(simt_bwd_workspace_elems(B * H, T) * sizeof(float));
   }
   if (fn == KATA_FN_DECODE_STEP) {      // T and C are ignored

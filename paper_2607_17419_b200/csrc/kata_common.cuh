@@ -73,6 +73,11 @@ void simt_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* 
 size_t simt_bwd_workspace_elems(int BH, int T);
 void simt_bwd_quadratic(const Problem& p, const void* dout, void* dq, void* dk, void* dv, float* stats, LaunchCtx& ctx);
 
+// Backward of the quadratic form on the tensor cores (bf16, d_k = d_v = 64, full rank-one feature)
+size_t tc_bwd_workspace_bytes(const Problem& p);
+void tc_bwd_quadratic(const Problem& p, const void* dout, void* dq, void* dk, void* dv, void* workspace, int* device_status,
+                      LaunchCtx& ctx);
+
 // feature_order = 1: rows of q,k are the features (plain normalised linear attention, state d_k x d_v)
 size_t order1_state_elems(int d_k, int d_v);
 void order1_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws, float* s_pre,

@@ -1,0 +1,541 @@
+// Backward of the quadratic form on the Blackwell tensor cores: bf16, d_k = d_v = 64, full rank-one feature.
+//
+// With s_ti = q_t . k_i, r_i = 1/||k_i||^2, a_ti = r_i s_ti^2 (i <= t), D_t = sum_i a_ti, o_t = sum_i a_ti v_i / D_t:
+//   c_ti = dout_t . v_i,   g_ti = (c_ti - dout_t . o_t) / D_t,   e_ti = 2 g_ti s_ti,   p_ti = s_ti^2 / D_t
+//   dq_t = sum_i e_ti k'_i                       (k' = r k, written by the pre-pass)
+//   dv_i = r_i sum_t p_ti dout_t
+//   dk_i = r_i (u_i - r_i (k_i . u_i) k_i),  u_i = sum_t e_ti q_t      (the second term is the derivative of r_i; it
+//                                                                       makes dk_i orthogonal to k_i: o has degree 0 in k_i)
+// A pre-pass writes k' and r; then one kernel in two modes, both with a fixed tile of 128 rows on the TMEM lanes and
+// tiles of 64 rows streamed past it:
+//   MODE_DQ   fixed = 128 queries (Q, dout), streamed = keys (K, V, K', r), twice:  S = Q K^T, C = dout V^T (SS MMAs,
+//             N = 64); in the first sweep the weight warps sum D_t = sum_i r_i s^2 and sum_i r_i s^2 c in fp32 (the
+//             same weights in both, so dout_t . o_t is consistent with c: their difference is what the gradient is
+//             made of) and leave (1/D_t, dout_t . o_t) in the workspace; in the second sweep they form E, and
+//             dq += E K' (A = E from TMEM)
+//   MODE_DKV  fixed = 128 keys (K, V), streamed = queries (Q, dout, their scalars):  S^T = K Q^T, C^T = V dout^T,
+//             the weight warps form P^T and E^T with the scalars of the columns, then dv~ += P^T dout, u += E^T Q
+//             (B = the streamed tiles read MN-major), and the epilogue applies r_i and the projection.
+// No atomics, every sum in a fixed order.  Warps (384 threads): 0 TMA producer, 1 score-MMA issuer, 2 output-MMA
+// issuer, 4-11 weights and epilogue.  All waits are bounded.
+#include <cuda.h>
+
+#include "kata_common.cuh"
+#include "kata_umma.cuh"
+
+namespace kata {
+namespace {
+
+using namespace umma;
+
+constexpr int D = 64;
+constexpr int MT = 128;          // rows of the fixed tile (TMEM lanes)
+constexpr int NT = 64;           // rows of a streamed tile
+constexpr int NSTAGE = 4;
+constexpr int NBUF = 3;
+constexpr int NTHREADS = 384;
+constexpr int WARP_BLD0 = 4;
+enum { MODE_DQ = 0, MODE_DKV = 1 };
+
+constexpr uint32_t COL_B = 0;      // 3 x 128 fp32: [S | C] of a streamed tile; the bf16 weights overwrite columns
+                                   // [0,32) of each half
+constexpr uint32_t COL_ACC = 384;  // 2 x 64 fp32 accumulators
+constexpr uint32_t TMEM_COLS = 512;
+
+constexpr uint32_t OFF_X1 = 0;                     // fixed tiles: 128 x 64 bf16, 128B swizzle
+constexpr uint32_t OFF_X2 = 16384;
+constexpr uint32_t OFF_ST = 32768;                 // stages: two streamed tiles of 8 KB, then K' (MODE_DQ)
+constexpr uint32_t STAGE_BYTES = 24576;
+constexpr uint32_t OFF_SC = OFF_ST + NSTAGE * STAGE_BYTES;   // per stage 512 bytes of scalars of the 64 streamed rows:
+                                                             // r_i (MODE_DQ) or (1/D_t, dout_t . o_t) (MODE_DKV)
+constexpr uint32_t OFF_PART = OFF_SC + NSTAGE * 512;         // 2 x 128 float2: the column halves of a row meet here
+constexpr uint32_t OFF_BAR = OFF_PART + 2048;
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
+constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
+static_assert(SMEM_ALLOC > 116 * 1024, "one CTA per SM is assumed (the CTA allocates all of TMEM)");
+
+// Every barrier has waiters that consume each of its phases in order; a producer of a phase always depends on the
+// waiter's progress (no barrier can complete two phases ahead of a waiter).
+enum {
+  BAR_XFULL = 0,     // fixed tiles landed
+  BAR_FULL = 1,      // [4] streamed tiles landed (TMA bytes + 32 producer lanes)
+  BAR_EMPTY = 5,     // [4] stage free: both issuers' commits
+  BAR_SFULL = 9,     // [3] scores in TMEM
+  BAR_PFULL = 12,    // [3] weights stored (256 threads)
+  BAR_PEMPTY = 15,   // [3] weights consumed: the buffer may take new scores
+  BAR_ODONE = 18,
+  BAR_DRAIN = 19,
+  BAR_COUNT = 20
+};
+
+struct BArgs {
+  __nv_bfloat16* out0;       // MODE_DQ: dq;  MODE_DKV: dk
+  __nv_bfloat16* out1;       // MODE_DKV: dv
+  float* stats;              // [BH][T][2]: 1 / D_t, dout_t . o_t (written by MODE_DQ, read by MODE_DKV)
+  const float* rk;           // [BH][T]: 1 / ||k_i||^2
+  int* device_status;
+  int Tlen;
+};
+
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u32 i;\n\t"
+      "mov.u32 i, 0;\n\t"
+      "KATA_WAIT_%=:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra KATA_DONE_%=;\n\t"
+      "add.u32 i, i, 1;\n\t"
+      "setp.lt.u32 q, i, %3;\n\t"
+      "@q bra KATA_WAIT_%=;\n\t"
+      "KATA_DONE_%=:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSpinLimit)
+      : "memory");
+  if (ok == 0) *abort_flag = 1;
+  return ok != 0;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ uint64_t at(uint64_t desc, uint32_t saddr) { return desc + (uint64_t)((saddr >> 4) & 0x3FFF); }
+
+template <int MODE>
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CUtensorMap tmX2,
+              const __grid_constant__ CUtensorMap tmY1, const __grid_constant__ CUtensorMap tmY2,
+              const __grid_constant__ CUtensorMap tmY3, const BArgs args) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  auto bar = [&](int i) { return reinterpret_cast<uint64_t*>(base + OFF_BAR) + i; };
+  auto y1 = [&](int s) { return base + OFF_ST + s * STAGE_BYTES; };
+  auto y2 = [&](int s) { return base + OFF_ST + s * STAGE_BYTES + 8192; };
+  auto y3 = [&](int s) { return base + OFF_ST + s * STAGE_BYTES + 16384; };
+  auto sc = [&](int s) { return base + OFF_SC + s * 512; };
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bh = blockIdx.y;
+  const int n_stream = (args.Tlen + NT - 1) / NT;                 // streamed tiles of the whole sequence
+  // MODE_DQ: heaviest (last) query tiles first, keys 0 .. m0 + 127;  MODE_DKV: key tile blockIdx.x (the first are
+  // the heaviest), queries m0 .. T - 1
+  const int mtile = MODE == MODE_DQ ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
+  const int m0 = mtile * MT;
+  const int jbeg = MODE == MODE_DQ ? 0 : 2 * mtile;
+  const int jend = MODE == MODE_DQ ? min(n_stream, 2 * mtile + 2) : n_stream;
+  const int ntiles = jend - jbeg;
+  const int nsteps = MODE == MODE_DQ ? 2 * ntiles : ntiles;       // MODE_DQ streams the keys twice
+
+  if (tid == 0) {
+    abort_s = 0;
+    mbar_init(bar(BAR_XFULL), 1);
+    for (int i = 0; i < NSTAGE; ++i) {
+      mbar_init(bar(BAR_FULL + i), 1 + 32);
+      mbar_init(bar(BAR_EMPTY + i), 2);
+    }
+    for (int i = 0; i < NBUF; ++i) {
+      mbar_init(bar(BAR_SFULL + i), 1);
+      mbar_init(bar(BAR_PFULL + i), 256);
+      mbar_init(bar(BAR_PEMPTY + i), 1);
+    }
+    mbar_init(bar(BAR_ODONE), 1);
+    mbar_init(bar(BAR_DRAIN), 2);
+    fence_mbar_init();
+    tma_prefetch_desc(&tmX1);
+    tma_prefetch_desc(&tmX2);
+    tma_prefetch_desc(&tmY1);
+    tma_prefetch_desc(&tmY2);
+    if (MODE == MODE_DQ) tma_prefetch_desc(&tmY3);
+  }
+  if (warp == 0) {
+    tmem_alloc(&tmem_base_s, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tb = tmem_base_s;
+  bool ok = true;
+
+  if (warp == 0) {
+    // =========================== TMA producer (+ the scalars of the streamed queries) ===========================
+    if (lane == 0) {
+      mbar_arrive_expect_tx(bar(BAR_XFULL), 32768);
+      tma_load_3d(base + OFF_X1, &tmX1, bar(BAR_XFULL), 0, m0, bh);
+      tma_load_3d(base + OFF_X2, &tmX2, bar(BAR_XFULL), 0, m0, bh);
+    }
+    for (int j = 0; j < nsteps && ok; ++j) {
+      const int s = j % NSTAGE;
+      const int n0 = (jbeg + j % ntiles) * NT;
+      ok = wait_or_abort(bar(BAR_EMPTY + s), ((j / NSTAGE) & 1) ^ 1, abort_flag);
+      if (!ok) break;
+      if (lane == 0) {
+        mbar_arrive_expect_tx(bar(BAR_FULL + s), MODE == MODE_DQ ? 24576u : 16384u);
+        tma_load_3d(y1(s), &tmY1, bar(BAR_FULL + s), 0, n0, bh);
+        tma_load_3d(y2(s), &tmY2, bar(BAR_FULL + s), 0, n0, bh);
+        if (MODE == MODE_DQ) tma_load_3d(y3(s), &tmY3, bar(BAR_FULL + s), 0, n0, bh);
+      }
+      const int t = n0 + 2 * lane;                       // two streamed rows per lane
+      if (MODE == MODE_DKV) {
+        // (1 / D_t, dout_t . o_t) of the 64 streamed queries
+        float4 st = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* src = args.stats + ((size_t)bh * args.Tlen + t) * 2;
+        if (t < args.Tlen) { st.x = src[0]; st.y = src[1]; }
+        if (t + 1 < args.Tlen) { st.z = src[2]; st.w = src[3]; }
+        *reinterpret_cast<float4*>(sc(s) + lane * 16) = st;
+      } else {
+        // r_i of the 64 streamed keys
+        float2 r2 = make_float2(0.f, 0.f);
+        const float* src = args.rk + (size_t)bh * args.Tlen + t;
+        if (t < args.Tlen) r2.x = src[0];
+        if (t + 1 < args.Tlen) r2.y = src[1];
+        *reinterpret_cast<float2*>(sc(s) + lane * 8) = r2;
+      }
+      mbar_arrive(bar(BAR_FULL + s));
+    }
+  } else if (warp == 1) {
+    // =========================== score MMA issuer: [S | C] ===========================
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 64);
+      const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
+      const uint32_t x1 = smem_u32(base + OFF_X1), x2 = smem_u32(base + OFF_X2);
+      ok = wait_or_abort(bar(BAR_XFULL), 0, abort_flag);
+      for (int j = 0; j < nsteps && ok; ++j) {
+        const int s = j % NSTAGE, b = j % NBUF;
+        ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
+             wait_or_abort(bar(BAR_PEMPTY + b), ((j / NBUF) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a1 = smem_u32(y1(s)), a2 = smem_u32(y2(s));
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          mma_f16_ss(tb + COL_B + b * 128, at(dk, x1 + ks * 32), at(dk, a1 + ks * 32), idesc, ks > 0);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          mma_f16_ss(tb + COL_B + b * 128 + 64, at(dk, x2 + ks * 32), at(dk, a2 + ks * 32), idesc, ks > 0);
+        mma_commit(bar(BAR_SFULL + b));
+        mma_commit(bar(BAR_EMPTY + s));
+      }
+    }
+  } else if (warp == 2) {
+    // =========================== output MMA issuer ===========================
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 64);     // A tmem, B MN-major
+      // MN-major, 128B swizzle: 8 streamed rows x 64 columns per 1 KB atom (SBO); 16 rows per MMA
+      const uint64_t dmn = smem_desc(0, 8192, 1024, kSwizzle128B);
+      for (int j = 0; j < nsteps && ok; ++j) {
+        const int s = j % NSTAGE, b = j % NBUF;
+        ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
+             wait_or_abort(bar(BAR_PFULL + b), (j / NBUF) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        if (MODE == MODE_DQ) {
+          if (j >= ntiles) {      // the first sweep only sums the row scalars: nothing to multiply
+            const uint32_t kp = smem_u32(y3(s));
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              mma_f16_ts(tb + COL_ACC, tb + COL_B + b * 128 + ks * 8, at(dmn, kp + ks * 2048), idesc,
+                         (j > ntiles || ks > 0) ? 1u : 0u);
+          }
+        } else {
+          const uint32_t qa = smem_u32(y1(s)), ga = smem_u32(y2(s));
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)      // dv~ += P^T dout
+            mma_f16_ts(tb + COL_ACC, tb + COL_B + b * 128 + ks * 8, at(dmn, ga + ks * 2048), idesc, (j > 0 || ks > 0) ? 1u : 0u);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)      // u += E^T Q
+            mma_f16_ts(tb + COL_ACC + 64, tb + COL_B + b * 128 + 64 + ks * 8, at(dmn, qa + ks * 2048), idesc,
+                       (j > 0 || ks > 0) ? 1u : 0u);
+        }
+        mma_commit(bar(BAR_PEMPTY + b));
+        mma_commit(bar(BAR_EMPTY + s));
+      }
+      if (ok) mma_commit(bar(BAR_ODONE));
+    }
+  } else if (warp >= WARP_BLD0) {
+    // =========================== weights and epilogue (256 threads) ===========================
+    const uint32_t q4 = warp & 3;
+    const int ch = (warp - WARP_BLD0) >> 2;      // column half: streamed rows [32 ch, 32 ch + 32) of the tile
+    const int rowl = q4 * 32 + lane;             // row of the fixed tile (= TMEM lane)
+    const int grow = m0 + rowl;
+    float inv_row = 0.f, del_row = 0.f;          // MODE_DQ: the scalars of this query (1 / D_t, dout_t . o_t)
+    float sum_d = 0.f, sum_m = 0.f;              // MODE_DQ, first sweep: this warp's share of D_t and of sum a c
+    float2* part = reinterpret_cast<float2*>(base + OFF_PART);
+    for (int j = 0; j < nsteps && ok; ++j) {
+      const int s = j % NSTAGE, b = j % NBUF;
+      const int n0 = (jbeg + j % ntiles) * NT + ch * 32;   // first streamed row of this warp's columns
+      if (MODE == MODE_DQ && j == ntiles) {
+        // between the sweeps: the two column halves of a row meet, the scalars go to registers and to the workspace
+        part[ch * MT + rowl] = make_float2(sum_d, sum_m);
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + (int)q4) : "memory");
+        const float2 other = part[(1 - ch) * MT + rowl];
+        const float dt = ch == 0 ? sum_d + other.x : other.x + sum_d;      // fixed order of the halves
+        const float mt = ch == 0 ? sum_m + other.y : other.y + sum_m;
+        inv_row = dt > 0.f ? 1.f / dt : 0.f;
+        del_row = mt * inv_row;
+        if (ch == 0 && grow < args.Tlen)
+          *reinterpret_cast<float2*>(args.stats + ((size_t)bh * args.Tlen + grow) * 2) = make_float2(inv_row, del_row);
+      }
+      ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&     // the column scalars are in the stage
+           wait_or_abort(bar(BAR_SFULL + b), (j / NBUF) & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t scol = tmem_addr(tb, q4 * 32, COL_B + b * 128 + ch * 32);
+      uint32_t sv[32], cv[32], pe[16], pp[16];
+      tmem_ld32(scol, sv);
+      tmem_ld32(scol + 64, cv);
+      tmem_wait_ld(sv);
+      tmem_wait_ld(cv);
+      if (MODE == MODE_DQ && j < ntiles) {
+        // first sweep: a = r_i s^2 for the keys n <= this query; D_t += a, sum += a c
+        const float2* cs = reinterpret_cast<const float2*>(sc(s) + ch * 128);
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const float2 r2 = cs[c / 2];
+          const float s0 = __uint_as_float(sv[c]), s1 = __uint_as_float(sv[c + 1]);
+          const float a0 = (n0 + c <= grow) ? s0 * s0 * r2.x : 0.f;
+          const float a1 = (n0 + c + 1 <= grow) ? s1 * s1 * r2.y : 0.f;
+          sum_d += a0;
+          sum_d += a1;
+          sum_m = fmaf(a0, __uint_as_float(cv[c]), sum_m);
+          sum_m = fmaf(a1, __uint_as_float(cv[c + 1]), sum_m);
+        }
+        // nothing is stored; the buffer is handed on as it is
+        tc_fence_before();
+        mbar_arrive(bar(BAR_PFULL + b));
+        continue;
+      }
+      if (MODE == MODE_DQ) {
+        // e = 2 (c - dout.o) / D * s, keys n <= this query
+        const float f = 2.f * inv_row;
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const float s0 = __uint_as_float(sv[c]), s1 = __uint_as_float(sv[c + 1]);
+          float e0 = (__uint_as_float(cv[c]) - del_row) * f * s0;
+          float e1 = (__uint_as_float(cv[c + 1]) - del_row) * f * s1;
+          if (n0 + c > grow) e0 = 0.f;
+          if (n0 + c + 1 > grow) e1 = 0.f;
+          pe[c / 2] = pack_bf16(e0, e1);
+        }
+      } else {
+        // p = s^2 / D_t, e = 2 (c - dout_t.o_t) / D_t * s with the scalars of the columns (queries t >= this key)
+        const float4* cs = reinterpret_cast<const float4*>(sc(s) + ch * 256);
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const float4 st = cs[c / 2];                       // (1/D, dout.o) of queries n0 + c, n0 + c + 1
+          const float s0 = __uint_as_float(sv[c]), s1 = __uint_as_float(sv[c + 1]);
+          float p0 = s0 * s0 * st.x, p1 = s1 * s1 * st.z;
+          float e0 = (__uint_as_float(cv[c]) - st.y) * (2.f * st.x) * s0;
+          float e1 = (__uint_as_float(cv[c + 1]) - st.w) * (2.f * st.z) * s1;
+          if (n0 + c < grow) { p0 = 0.f; e0 = 0.f; }
+          if (n0 + c + 1 < grow) { p1 = 0.f; e1 = 0.f; }
+          pp[c / 2] = pack_bf16(p0, p1);
+          pe[c / 2] = pack_bf16(e0, e1);
+        }
+      }
+      // the weights overwrite score columns [0,32) of each half, which the column-half-0 warp of this quadrant
+      // reads: both warps of the quadrant must have their scores in registers first
+      tc_fence_before();
+      asm volatile("bar.sync %0, 64;" ::"r"(1 + (int)q4) : "memory");
+      tc_fence_after();
+      if (MODE == MODE_DQ) {
+        tmem_st16(tmem_addr(tb, q4 * 32, COL_B + b * 128 + ch * 16), pe);
+      } else {
+        tmem_st16(tmem_addr(tb, q4 * 32, COL_B + b * 128 + ch * 16), pp);
+        tmem_st16(tmem_addr(tb, q4 * 32, COL_B + b * 128 + 64 + ch * 16), pe);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(BAR_PFULL + b));
+    }
+    // ---- epilogue ----
+    if (ok) ok = wait_or_abort(bar(BAR_ODONE), 0, abort_flag);
+    if (ok) {
+      tc_fence_after();
+      uint32_t a0[32];
+      tmem_ld32(tmem_addr(tb, q4 * 32, COL_ACC + ch * 32), a0);
+      tmem_wait_ld(a0);
+      auto store32 = [&](__nv_bfloat16* dst, const float (&x)[32]) {
+#pragma unroll
+        for (int c = 0; c < 32; c += 8) {
+          uint4 pkt;
+          pkt.x = pack_bf16(x[c], x[c + 1]);
+          pkt.y = pack_bf16(x[c + 2], x[c + 3]);
+          pkt.z = pack_bf16(x[c + 4], x[c + 5]);
+          pkt.w = pack_bf16(x[c + 6], x[c + 7]);
+          *reinterpret_cast<uint4*>(dst + c) = pkt;
+        }
+      };
+      float x[32];
+      if (MODE == MODE_DQ) {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) x[c] = __uint_as_float(a0[c]);
+        if (grow < args.Tlen) store32(args.out0 + ((size_t)bh * args.Tlen + grow) * D + ch * 32, x);
+      } else {
+        uint32_t u[32];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_ACC + 64 + ch * 32), u);
+        tmem_wait_ld(u);
+        // this key's row (32 of its 64 entries), its share of ||k||^2 and of k . u; the halves meet in shared memory
+        float kf[32];
+        float n2 = 0.f, dot = 0.f;
+#pragma unroll
+        for (int cix = 0; cix < 4; ++cix) {
+          const uint4 raw = *reinterpret_cast<const uint4*>(base + OFF_X1 + sw128_offset(rowl, ch * 4 + cix));
+          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            kf[8 * cix + 2 * e] = __uint_as_float(w[e] << 16);
+            kf[8 * cix + 2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+          }
+        }
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          n2 = fmaf(kf[c], kf[c], n2);
+          dot = fmaf(kf[c], __uint_as_float(u[c]), dot);
+        }
+        part[ch * MT + rowl] = make_float2(n2, dot);
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + (int)q4) : "memory");
+        const float2 other = part[(1 - ch) * MT + rowl];
+        // fixed order of the two halves
+        const float n2t = ch == 0 ? n2 + other.x : other.x + n2;
+        const float dott = ch == 0 ? dot + other.y : other.y + dot;
+        const float r = inv_or_zero(n2t);
+        const float proj = r * dott;
+        if (grow < args.Tlen) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) x[c] = r * (__uint_as_float(u[c]) - proj * kf[c]);
+          store32(args.out0 + ((size_t)bh * args.Tlen + grow) * D + ch * 32, x);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) x[c] = r * __uint_as_float(a0[c]);
+          store32(args.out1 + ((size_t)bh * args.Tlen + grow) * D + ch * 32, x);
+        }
+      }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  if (!ok && args.device_status != nullptr) atomicExch(args.device_status, (int)KATA_ERR_DEVICE_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if ((warp == 1 || warp == 2) && lane == 0) {
+    mma_commit(bar(BAR_DRAIN));
+    mbar_wait(bar(BAR_DRAIN), 0);
+  }
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tb, TMEM_COLS);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// [BH][T][64] bf16 tensor, box = 64 columns x rows x 1 head, 128B swizzle; rows beyond T read as zero.
+bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T, int rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)BH};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
+  cuuint32_t box[3] = {(cuuint32_t)D, (cuuint32_t)rows, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+size_t align256(size_t n) { return (n + 255) / 256 * 256; }
+
+// Pre-pass: one warp per 4 key rows (8 lanes x 16 bytes per row).  k' = k / ||k||^2 (bf16), r = 1 / ||k||^2 (fp32).
+__global__ void __launch_bounds__(256) bwd_prescale_kernel(const __nv_bfloat16* __restrict__ k, __nv_bfloat16* __restrict__ ks,
+                                                           float* __restrict__ rk, size_t n_rows) {
+  const size_t row = (size_t)blockIdx.x * 32 + (threadIdx.x >> 3);
+  const int part = threadIdx.x & 7;
+  if (row >= n_rows) return;
+  const uint4 kraw = *reinterpret_cast<const uint4*>(k + row * D + part * 8);
+  const uint32_t kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
+  float ss = 0.f;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float lo = __uint_as_float(kw[e] << 16), hi = __uint_as_float(kw[e] & 0xFFFF0000u);
+    ss = fmaf(lo, lo, ss);
+    ss = fmaf(hi, hi, ss);
+  }
+  ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+  ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+  ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+  const float r = inv_or_zero(ss);
+  uint4 kc;
+  kc.x = pack_bf16(__uint_as_float(kw[0] << 16) * r, __uint_as_float(kw[0] & 0xFFFF0000u) * r);
+  kc.y = pack_bf16(__uint_as_float(kw[1] << 16) * r, __uint_as_float(kw[1] & 0xFFFF0000u) * r);
+  kc.z = pack_bf16(__uint_as_float(kw[2] << 16) * r, __uint_as_float(kw[2] & 0xFFFF0000u) * r);
+  kc.w = pack_bf16(__uint_as_float(kw[3] << 16) * r, __uint_as_float(kw[3] & 0xFFFF0000u) * r);
+  *reinterpret_cast<uint4*>(ks + row * D + part * 8) = kc;
+  if (part == 0) rk[row] = r;
+}
+
+}  // namespace
+
+// workspace: K' [BH][T][64] bf16, r [BH][T] fp32, the row scalars [BH][T][2] fp32
+size_t tc_bwd_workspace_bytes(const Problem& p) {
+  const size_t rows = (size_t)p.B * p.H * p.T;
+  return align256(rows * D * 2) + align256(rows * sizeof(float)) + align256(rows * 2 * sizeof(float));
+}
+
+void tc_bwd_quadratic(const Problem& p, const void* dout, void* dq, void* dk, void* dv, void* workspace, int* device_status,
+                      LaunchCtx& ctx) {
+  const int BH = p.B * p.H;
+  const size_t rows = (size_t)BH * p.T;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  __nv_bfloat16* ks = reinterpret_cast<__nv_bfloat16*>(ws);
+  float* rk = reinterpret_cast<float*>(ws + align256(rows * D * 2));
+  float* stats = reinterpret_cast<float*>(ws + align256(rows * D * 2) + align256(rows * sizeof(float)));
+  bwd_prescale_kernel<<<(unsigned)((rows + 31) / 32), 256, 0, ctx.stream>>>(static_cast<const __nv_bfloat16*>(p.k), ks, rk, rows);
+  note_launch(ctx);
+  CUtensorMap q128, g128, k128, v128, q64, g64, k64, v64, ks64;
+  if (!make_map(&q128, p.q, BH, p.T, MT) || !make_map(&g128, dout, BH, p.T, MT) || !make_map(&k128, p.k, BH, p.T, MT) ||
+      !make_map(&v128, p.v, BH, p.T, MT) || !make_map(&q64, p.q, BH, p.T, NT) || !make_map(&g64, dout, BH, p.T, NT) ||
+      !make_map(&k64, p.k, BH, p.T, NT) || !make_map(&v64, p.v, BH, p.T, NT) || !make_map(&ks64, ks, BH, p.T, NT)) {
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  auto kq = tc_bwd_kernel<MODE_DQ>;
+  auto kkv = tc_bwd_kernel<MODE_DKV>;
+  if (cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+      cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
+    cudaGetLastError();
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  const dim3 grid((p.T + MT - 1) / MT, BH);
+  // dq and the row scalars, then dk and dv (which read the scalars)
+  BArgs a{static_cast<__nv_bfloat16*>(dq), nullptr, stats, rk, device_status, p.T};
+  kq<<<grid, NTHREADS, SMEM_ALLOC, ctx.stream>>>(q128, g128, k64, v64, ks64, a);
+  note_launch(ctx);
+  BArgs b{static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), stats, rk, device_status, p.T};
+  kkv<<<grid, NTHREADS, SMEM_ALLOC, ctx.stream>>>(k128, v128, q64, g64, q64, b);
+  note_launch(ctx);
+}
+
+}  // namespace kata

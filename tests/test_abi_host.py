@@ -173,5 +173,12 @@ def test_backward_argument_checks(L):
     assert bwd(opts=kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 30, impl=kb.KATA_IMPL_TENSOR)) == SHAPE
     assert bwd(opts=kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 30, feature_groups=3)) == INV
     assert bwd(opts=kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 30, s_pre=4096, z_pre=8192)) == INV
+    up = lambda n: (n + 255) // 256 * 256
+    rows = 2 * 3 * 100
+    # fp32 kernels: two floats per row; tensor-core kernels (bf16, d = 64): k' (bf16), r and the two row scalars (fp32)
+    o = kb.make_opts(kb.KATA_F32)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 64, 64, 0, o) == up(rows * 2 * 4)
     o = kb.make_opts(kb.KATA_BF16)
-    assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 64, 64, 0, o) == (2 * 3 * 100 * 2 * 4 + 255) // 256 * 256
+    assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 64, 64, 0, o) == up(rows * 128) + up(rows * 4) + up(rows * 8)
+    o = kb.make_opts(kb.KATA_BF16, feature_groups=2)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 64, 64, 0, o) == up(rows * 2 * 4)

@@ -30,9 +30,15 @@ def check_grads(w, feature, seed=5, **kw):
     import torch
     q, k, v = dev_tensors(w)
     g_dev, g_ref = dout_for(w, seed)
-    dq, dk, dv = kb.kata_bwd_quadratic(q, k, v, g_dev, **kw)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dq, dk, dv = kb.kata_bwd_quadratic(q, k, v, g_dev, device_status=st, **kw)
     torch.cuda.synchronize()
-    assert kb.kata_last_impl() == kb.KATA_IMPL_SIMT and kb.kata_last_launch_count() == 2
+    assert int(st.item()) == 0
+    # tensor-core kernels for bf16, d = 64, the full rank-one feature (pre-pass, dq with the row scalars, dk/dv)
+    tensor = (w.dtype == "bf16" and w.d_k == 64 and w.d_v == 64 and feature == "psd_direct"
+              and kw.get("impl", kb.KATA_IMPL_AUTO) != kb.KATA_IMPL_SIMT)
+    assert kb.kata_last_impl() == (kb.KATA_IMPL_TENSOR if tensor else kb.KATA_IMPL_SIMT)
+    assert kb.kata_last_launch_count() == (3 if tensor else 2)
     tol = TOL[w.dtype]
     for b in range(w.B):
         for h in range(w.H):
@@ -51,6 +57,33 @@ def check_grads(w, feature, seed=5, **kw):
 def test_backward_psd(dtype, dk, dv, T):
     w = inputs.gaussian_workload(f"bwd_{dtype}_{dk}_{dv}_{T}", dtype, 1, 2, T, dk, dv, 64, 800 + T + dk)
     check_grads(w, "psd_direct")
+
+
+@pytest.mark.parametrize("T", [1, 2, 63, 64, 65, 127, 128, 129, 191, 192, 193, 257, 600])
+def test_backward_tensor_tile_boundaries(T):
+    """Tensor-core kernels: fixed tiles of 128 rows, streamed tiles of 64; and the fp32 kernels on the same inputs."""
+    w = inputs.gaussian_workload(f"bwd_tc_{T}", "bf16", 1, 2, T, 64, 64, 64, 860 + T)
+    a = check_grads(w, "psd_direct")
+    b = check_grads(w, "psd_direct", impl=kb.KATA_IMPL_SIMT)
+    for x, y in zip(a, b):
+        assert float((x.float() - y.float()).abs().max()) <= 4e-2 * max(1.0, float(y.float().abs().max()))
+
+
+def test_backward_tensor_zero_rows():
+    import torch
+    T = 300
+    w = inputs.gaussian_workload("bwd_tc_zero", "bf16", 1, 1, T, 64, 64, 64, 870)
+    for t in (0, 1, 64, 127, 128, 200):
+        w.k_dev[0, 0, t] = 0
+        w.k_ref[0, 0, t] = 0
+    for t in (0, 5, 128, 256):
+        w.q_dev[0, 0, t] = 0
+        w.q_ref[0, 0, t] = 0
+    dq, dk, dv = check_grads(w, "psd_direct")
+    assert torch.all(dk[0, 0, [0, 1, 64, 127, 128, 200]] == 0) and torch.all(dv[0, 0, [0, 1, 64, 127, 128, 200]] == 0)
+    assert torch.all(dq[0, 0, [0, 1, 5, 128, 256]] == 0)
+    dq2, dk2, dv2 = check_grads(w, "psd_direct")
+    assert torch.equal(dq, dq2) and torch.equal(dk, dk2) and torch.equal(dv, dv2)      # fixed summation order
 
 
 @pytest.mark.parametrize("g", [2, 4])
@@ -103,6 +136,6 @@ def test_backward_argument_checks():
     w = inputs.gaussian_workload("bwd_args", "bf16", 1, 1, 64, 64, 64, 64, 1)
     q, k, v = dev_tensors(w)
     with pytest.raises(kb.KataError):
-        kb.kata_bwd_quadratic(q, k, v, v, impl=kb.KATA_IMPL_TENSOR)
+        kb.kata_bwd_quadratic(q, k, v, v, impl=kb.KATA_IMPL_TENSOR, feature_groups=2)    # fp32 kernels only
     with pytest.raises(kb.KataError):
         kb.kata_bwd_quadratic(q, k, v, v, feature_groups=3)
