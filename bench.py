@@ -377,6 +377,33 @@ def run_order1(args):
                           impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")))
 
 
+def run_bwd(args):
+    """Profiler case of the backward pass: config 2 (B=4, H=16, T=4096, d=64, bf16; inputs 134 MB > L2); short line."""
+    import numpy as np
+    import torch
+    from paper_2607_17419_b200 import binding as kb, build as kbuild, inputs
+    kbuild.build()
+    torch.cuda.set_device(0)
+    w = inputs.config(2)
+    q, k, v = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda() for a in (w.q_dev, w.k_dev, w.v_dev))
+    g = torch.randn(v.shape, device="cuda", generator=torch.Generator(device="cuda").manual_seed(7)).to(torch.bfloat16)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    for _ in range(args.warmup):
+        kb.kata_bwd_quadratic(q, k, v, g, dq, dk, dv)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        kb.kata_bwd_quadratic(q, k, v, g, dq, dk, dv)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    fl = quadratic_flops(w.B, w.H, w.T) / 256.0 * 640.0
+    print(json.dumps(dict(case="bwd", ms_per_step=ms, tokens_per_s=w.B * w.T / (ms * 1e-3), tflops=fl / (ms * 1e-3) / 1e12,
+                          launches=kb.kata_last_launch_count(),
+                          impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")))
+
+
 def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
     """Separately timed secondary figures: scan forms on the same workload, quadratic form on config 2."""
     import numpy as np
@@ -417,6 +444,16 @@ def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
         ms = timed(lambda: kb.kata_fwd_quadratic(q2, k2, v2, o2, feature_groups=g))
         res[f"quadratic_c2_M{g}"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=fl / (ms * 1e-3) / 1e12,
                                          impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
+    # backward of the quadratic form on config 2 (tensor-core kernels; recomputation, 5 matrix products of
+    # 2 * 64 flops per causal pair = 640 algorithmic flops per pair)
+    g2 = torch.randn(v2.shape, device=dev, generator=torch.Generator(device=dev).manual_seed(7)).to(torch.bfloat16)
+    dq2, dk2, dv2 = torch.empty_like(q2), torch.empty_like(k2), torch.empty_like(v2)
+    ms = timed(lambda: kb.kata_bwd_quadratic(q2, k2, v2, g2, dq2, dk2, dv2))
+    flb = fl / 256.0 * 640.0
+    res["bwd_quadratic_c2"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=flb / (ms * 1e-3) / 1e12,
+                                   frac_of_bf16_burst=flb / (ms * 1e-3) / 1e12 / peaks["bf16_burst"],
+                                   launches=kb.kata_last_launch_count(),
+                                   impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
     # first-order feature (rows of q, k as features; matched d x d state, C = 128): shapes of the paper's scan
     # benchmark; HBM-bound, 512 algorithmic bytes per token and head (q, k, v read, o written)
     for Bo, To in ((1, 8192), (1, 131072), (4, 32768), (16, 8192), (32, 32768)):
@@ -455,7 +492,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="sequential", choices=["sequential", "scan"])
     ap.add_argument("--no-extra", dest="extra", action="store_false")
-    ap.add_argument("--case", default="full", choices=["full", "small", "decode", "order1"],
+    ap.add_argument("--case", default="full", choices=["full", "small", "decode", "order1", "bwd"],
                     help="small: the same kernel on T=32768 only; decode: the decode step only; order1: the "
                          "first-order tensor-core kernel on B=16, T=8192 (all for profiler captures; they print a "
                          "short line)")
@@ -466,6 +503,8 @@ def main():
         run_decode(args)
     elif args.case == "order1":
         run_order1(args)
+    elif args.case == "bwd":
+        run_bwd(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -139,3 +139,22 @@ def test_backward_argument_checks():
         kb.kata_bwd_quadratic(q, k, v, v, impl=kb.KATA_IMPL_TENSOR, feature_groups=2)    # fp32 kernels only
     with pytest.raises(kb.KataError):
         kb.kata_bwd_quadratic(q, k, v, v, feature_groups=3)
+
+
+def test_backward_config2_full_size_heads():
+    """The benchmark shape (B=4, H=16, T=4096, d=64, bf16): every row of two heads against the oracle."""
+    import torch
+    w = inputs.config(2)
+    q, k, v = dev_tensors(w)
+    g_dev, g_ref = dout_for(w, 11)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dq, dk, dv = kb.kata_bwd_quadratic(q, k, v, g_dev, device_status=st)
+    torch.cuda.synchronize()
+    assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR and int(st.item()) == 0
+    for b, h in ((0, 0), (3, 15)):
+        rq, rk, rv = ko.kata_quadratic_bwd(w.q_ref[b, h], w.k_ref[b, h], w.v_ref[b, h], g_ref[b, h])
+        for name, got, ref in (("dq", dq, rq), ("dk", dk, rk), ("dv", dv, rv)):
+            gg = to_numpy64(got[b, h])
+            assert np.all(np.isfinite(gg))
+            err = np.max(np.abs(gg - ref))
+            assert err <= 2e-2 * max(1.0, np.abs(ref).max()), f"{name} ({b},{h}): {err:.3e}"
