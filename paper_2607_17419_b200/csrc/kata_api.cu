@@ -268,6 +268,10 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
     // state import and final-state export of the fp32 path go through one internal state per head
     if (fn == KATA_FN_CHUNKED && (r.o.s_pre != nullptr || r.o.s_init != nullptr) && !r.tensor)
       r.inner_bytes = align_up((size_t)B * H * r.state_elems * sizeof(float));
+    // tensor-core path, state advanced in place: every value slice of a head reads the normaliser state and one of
+    // them writes it, so the kernel reads a copy of z_init
+    if (fn == KATA_FN_CHUNKED && r.tensor && r.o.z_init != nullptr && r.o.z_init == r.o.z_pre)
+      r.inner_bytes = align_up((size_t)B * H * decode_n_psi(d_k, r.o.state_layout, 2, 1) * sizeof(float));
   }
   return KATA_OK;
 }
@@ -280,11 +284,21 @@ int run_device(int fn, Prepared& r, void* ws) {
     else simt_quadratic(r.p, ctx);
   } else {
     const bool use_scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || r.plan.n_groups > 1;
-    if (r.tensor && r.p.feature_order == 1)
+    if (r.tensor && r.p.feature_order == 1) {
       tc_order1(r.p, r.plan, use_scan, r.C, wsf, r.o.device_status, ctx);
-    else if (r.tensor)
-      tc_chunked(r.p, r.plan, use_scan, wsf, r.o.device_status, r.o.s_init, r.o.z_init, r.o.s_pre, r.o.z_pre,
+    } else if (r.tensor) {
+      const float* z_init = r.o.z_init;
+      if (fn == KATA_FN_CHUNKED && z_init != nullptr && z_init == r.o.z_pre) {
+        const size_t nb = (size_t)r.p.B * r.p.H * decode_n_psi(r.p.d_k, r.o.state_layout, 2, 1) * sizeof(float);
+        if (cudaMemcpyAsync(wsf, z_init, nb, cudaMemcpyDeviceToDevice, r.o.stream) != cudaSuccess) {
+          cudaGetLastError();
+          return KATA_ERR_CUDA;
+        }
+        z_init = wsf;
+      }
+      tc_chunked(r.p, r.plan, use_scan, wsf, r.o.device_status, r.o.s_init, z_init, r.o.s_pre, r.o.z_pre,
                  r.o.state_layout, ctx);
+    }
     else if (r.p.feature_order == 1) order1_chunked(r.p, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, ctx);
     else simt_chunked(r.p, r.plan, use_scan, wsf, r.o.s_init, r.o.z_init, r.o.s_pre, r.o.z_pre, r.o.state_layout, ctx);
   }

@@ -124,3 +124,18 @@ def test_resume_argument_checks():
         kb.kata_chunk_state_scan(q, k, v, s_init=S, z_init=Z)
     with pytest.raises(kb.KataError):
         kb.kata_fwd_chunked(q, k, v, s_init=S, z_init=Z, feature_order=1)
+
+
+def test_resume_in_place_many_heads():
+    """More CTAs than SMs (64 heads x 8 value slices): the slices of a head start at different times, and the
+    state advanced in place must still be read before it is written."""
+    import torch
+    w = inputs.gaussian_workload("resume_many", "bf16", 4, 16, 384, 64, 64, 64, 59)
+    a = run_pieces(w, (128, 256), "psd_direct", in_place=False)
+    b = run_pieces(w, (128, 256), "psd_direct", in_place=True)
+    assert a[3] == b[3] == {kb.KATA_IMPL_TENSOR}
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
+    gpu = to_numpy64(b[0])
+    for bb, h in ((0, 0), (3, 15)):
+        ref = ko.kata_quadratic(w.q_ref[bb, h], w.k_ref[bb, h], w.v_ref[bb, h])[0]
+        check(gpu[bb, h], ref, "bf16", f"in place, many heads ({bb},{h})")
