@@ -377,6 +377,32 @@ def run_order1(args):
                           impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")))
 
 
+def run_quadratic(args):
+    """Profiler case of the quadratic forward: config 2 (B=4, H=16, T=4096, d=64, bf16; inputs 134 MB > L2); short line."""
+    import numpy as np
+    import torch
+    from paper_2607_17419_b200 import binding as kb, build as kbuild, inputs
+    kbuild.build()
+    torch.cuda.set_device(0)
+    w = inputs.config(2)
+    q, k, v = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda() for a in (w.q_dev, w.k_dev, w.v_dev))
+    out = torch.empty_like(v)
+    for _ in range(args.warmup):
+        kb.kata_fwd_quadratic(q, k, v, out)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        kb.kata_fwd_quadratic(q, k, v, out)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    fl = quadratic_flops(w.B, w.H, w.T)
+    print(json.dumps(dict(case="quadratic", ms_per_step=ms, tokens_per_s=w.B * w.T / (ms * 1e-3), tflops=fl / (ms * 1e-3) / 1e12,
+                          launches=kb.kata_last_launch_count(),
+                          impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")))
+
+
 def run_bwd(args):
     """Profiler case of the backward pass: config 2 (B=4, H=16, T=4096, d=64, bf16; inputs 134 MB > L2); short line."""
     import numpy as np
@@ -492,7 +518,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="sequential", choices=["sequential", "scan"])
     ap.add_argument("--no-extra", dest="extra", action="store_false")
-    ap.add_argument("--case", default="full", choices=["full", "small", "decode", "order1", "bwd"],
+    ap.add_argument("--case", default="full", choices=["full", "small", "decode", "order1", "bwd", "quadratic"],
                     help="small: the same kernel on T=32768 only; decode: the decode step only; order1: the "
                          "first-order tensor-core kernel on B=16, T=8192 (all for profiler captures; they print a "
                          "short line)")
@@ -505,6 +531,8 @@ def main():
         run_order1(args)
     elif args.case == "bwd":
         run_bwd(args)
+    elif args.case == "quadratic":
+        run_quadratic(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
