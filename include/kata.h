@@ -26,8 +26,10 @@
  *   - Supported shapes: d_k, d_v in {16,32,64}; C = 64 (the chunked/scan forms), and C = 128 for
  *     feature_order 1 with bf16, d_k = d_v = 64 (the chunk size of the paper's scan benchmark; tensor-core
  *     path, no s_pre/z_pre); T >= 1 (any; the last chunk is zero-padded as in Algorithm 1 and truncated on
- *     output); B,H >= 1.  The tensor-core (tcgen05) kernels cover bf16 with d_k = d_v = 64; everything
- *     else runs on the fp32 SIMT kernels.
+ *     output); B,H >= 1.  The tensor-core (tcgen05) kernels cover bf16 with d_k = d_v = 64; narrower bf16
+ *     rows are zero-padded to 64 entries in the workspace and run on the same kernels (the result is the same
+ *     function: dot products and norms do not change) unless feature_groups > 1 or a state is handed over, whose
+ *     layouts depend on the true width; everything else runs on the fp32 SIMT kernels.
  *   - Return value: KATA_OK (0) or a negative kata_status.  Errors detectable on the host
  *     launch nothing.  No exceptions, no abort, no device trap.  A bounded device-side wait
  *     that expires writes KATA_ERR_DEVICE_TIMEOUT to *opts->device_status (if non-null),

@@ -234,7 +234,40 @@ struct Prepared {
   size_t inner_bytes;
   bool tensor;
   int C;
+  bool pad;             // bf16 rows narrower than 64 are zero-padded to 64 so that the tensor-core kernels apply
+  size_t pad_bytes;     // one padded tensor [B*H*T][64] bf16 (q, k, v, out: four of them at the start of the scratch)
 };
+
+// Zero-padding the rows of q, k, v to 64 entries changes neither the dot products nor the norms, and the padded
+// value columns give output columns that are dropped: the same function, computed by the d = 64 kernels.
+__global__ void pad_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t rows, int d) {
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // one 16-byte chunk of a padded row
+  if (idx >= rows * 8) return;
+  const size_t row = idx >> 3;
+  const int c = (int)(idx & 7);
+  uint4 x = make_uint4(0u, 0u, 0u, 0u);
+  if (c * 8 < d) x = *reinterpret_cast<const uint4*>(src + row * d + c * 8);
+  *reinterpret_cast<uint4*>(dst + row * 64 + c * 8) = x;
+}
+
+__global__ void unpad_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t rows, int d) {
+  const int cpr = d / 8;                                                  // 16-byte chunks per output row
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * cpr) return;
+  const size_t row = idx / cpr;
+  const int c = (int)(idx % cpr);
+  *reinterpret_cast<uint4*>(dst + row * d + c * 8) = *reinterpret_cast<const uint4*>(src + row * 64 + c * 8);
+}
+
+// The problem the kernels see: the caller's, or its copy with rows padded to 64 entries.
+Problem kernel_problem(const Prepared& r) {
+  Problem pp = r.p;
+  if (r.pad) {
+    pp.d_k = 64;
+    pp.d_v = 64;
+  }
+  return pp;
+}
 
 int prepare(int fn, const void* q, const void* k, const void* v, void* out, int B, int H, int T, int d_k,
             int d_v, int C, const kata_opts* opts, bool need_ptrs, Prepared& r) {
@@ -252,19 +285,29 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   if (r.o.s_init != nullptr && !(fn == KATA_FN_CHUNKED && r.o.inter_chunk == KATA_SEQUENTIAL)) return KATA_ERR_INVALID_ARG;
   if (r.o.s_init != nullptr && r.o.feature_order != 2) return KATA_ERR_UNSUPPORTED_SHAPE;
   r.p = Problem{q, k, v, out, B, H, T, d_k, d_v, r.o.dtype, r.o.feature_order, r.o.groups};
-  r.tensor = want_tensor(fn, r.p, r.o);
+  // bf16 rows narrower than 64: zero-pad to 64 and use the tensor-core kernels (plain feature, no state hand-off:
+  // the state layouts and the feature blocks depend on the true width)
+  r.pad = r.o.impl != KATA_IMPL_SIMT && r.o.dtype == KATA_BF16 && (d_k < 64 || d_v < 64) && r.o.groups == 1 &&
+          r.o.s_pre == nullptr && r.o.s_init == nullptr;
+  r.pad_bytes = 0;
+  if (r.pad) {
+    r.pad = want_tensor(fn, kernel_problem(r), r.o);
+    if (r.pad) r.pad_bytes = align_up((size_t)B * H * T * 64 * 2);
+  }
+  const Problem kp = kernel_problem(r);
+  r.tensor = want_tensor(fn, kp, r.o);
   if (r.o.impl == KATA_IMPL_TENSOR && !r.tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
   r.C = fn == KATA_FN_QUADRATIC ? kChunk : C;
   r.plan = ScanPlan{(T + r.C - 1) / r.C, 0, 1, 0};
   r.state_elems = 0;
-  r.inner_bytes = (fn == KATA_FN_QUADRATIC && r.tensor) ? tc_quadratic_workspace_bytes(r.p) : 0;
+  r.inner_bytes = (fn == KATA_FN_QUADRATIC && r.tensor) ? tc_quadratic_workspace_bytes(kp) : 0;
   if (fn != KATA_FN_QUADRATIC) {
     if (r.tensor && r.o.s_pre != nullptr && fn == KATA_FN_CHUNK_STATE_SCAN) r.tensor = false;   // per-chunk export: SIMT pipeline
     // C = 128 (the chunk size of the paper's scan benchmark) exists on the first-order tensor-core path only
     if (r.C != kChunk && !(r.tensor && r.p.feature_order == 1)) return KATA_ERR_UNSUPPORTED_SHAPE;
-    st = make_plan(fn, r.p, r.o, r.tensor, r.C, r.plan, r.state_elems);
+    st = make_plan(fn, kp, r.o, r.tensor, r.C, r.plan, r.state_elems);
     if (st != KATA_OK) return st;
-    r.inner_bytes = inner_workspace(fn, r.plan, r.p, r.state_elems);
+    r.inner_bytes = inner_workspace(fn, r.plan, kp, r.state_elems);
     // state import and final-state export of the fp32 path go through one internal state per head
     if (fn == KATA_FN_CHUNKED && (r.o.s_pre != nullptr || r.o.s_init != nullptr) && !r.tensor)
       r.inner_bytes = align_up((size_t)B * H * r.state_elems * sizeof(float));
@@ -273,19 +316,41 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
     if (fn == KATA_FN_CHUNKED && r.tensor && r.o.z_init != nullptr && r.o.z_init == r.o.z_pre)
       r.inner_bytes = align_up((size_t)B * H * decode_n_psi(d_k, r.o.state_layout, 2, 1) * sizeof(float));
   }
+  r.inner_bytes += 4 * r.pad_bytes;
   return KATA_OK;
 }
 
 int run_device(int fn, Prepared& r, void* ws) {
   LaunchCtx ctx{r.o.stream, 0, KATA_OK};
+  Problem P = kernel_problem(r);
+  if (r.pad) {
+    // [q | k | v | out] padded to 64 columns at the start of the scratch, the kernels' own scratch after them
+    unsigned char* w8 = static_cast<unsigned char*>(ws);
+    __nv_bfloat16* pq = reinterpret_cast<__nv_bfloat16*>(w8);
+    __nv_bfloat16* pk = reinterpret_cast<__nv_bfloat16*>(w8 + r.pad_bytes);
+    __nv_bfloat16* pv = reinterpret_cast<__nv_bfloat16*>(w8 + 2 * r.pad_bytes);
+    const size_t rows = (size_t)P.B * P.H * P.T;
+    const unsigned blocks = (unsigned)((rows * 8 + 255) / 256);
+    pad_rows_kernel<<<blocks, 256, 0, r.o.stream>>>(static_cast<const __nv_bfloat16*>(r.p.q), pq, rows, r.p.d_k);
+    note_launch(ctx);
+    pad_rows_kernel<<<blocks, 256, 0, r.o.stream>>>(static_cast<const __nv_bfloat16*>(r.p.k), pk, rows, r.p.d_k);
+    note_launch(ctx);
+    pad_rows_kernel<<<blocks, 256, 0, r.o.stream>>>(static_cast<const __nv_bfloat16*>(r.p.v), pv, rows, r.p.d_v);
+    note_launch(ctx);
+    P.q = pq;
+    P.k = pk;
+    P.v = pv;
+    P.out = w8 + 3 * r.pad_bytes;
+    ws = w8 + 4 * r.pad_bytes;
+  }
   float* wsf = static_cast<float*>(ws);
   if (fn == KATA_FN_QUADRATIC) {
-    if (r.tensor) tc_quadratic(r.p, ws, r.o.device_status, ctx);
-    else simt_quadratic(r.p, ctx);
+    if (r.tensor) tc_quadratic(P, ws, r.o.device_status, ctx);
+    else simt_quadratic(P, ctx);
   } else {
     const bool use_scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || r.plan.n_groups > 1;
-    if (r.tensor && r.p.feature_order == 1) {
-      tc_order1(r.p, r.plan, use_scan, r.C, wsf, r.o.device_status, ctx);
+    if (r.tensor && P.feature_order == 1) {
+      tc_order1(P, r.plan, use_scan, r.C, wsf, r.o.device_status, ctx);
     } else if (r.tensor) {
       const float* z_init = r.o.z_init;
       if (fn == KATA_FN_CHUNKED && z_init != nullptr && z_init == r.o.z_pre) {
@@ -296,11 +361,18 @@ int run_device(int fn, Prepared& r, void* ws) {
         }
         z_init = wsf;
       }
-      tc_chunked(r.p, r.plan, use_scan, wsf, r.o.device_status, r.o.s_init, z_init, r.o.s_pre, r.o.z_pre,
+      tc_chunked(P, r.plan, use_scan, wsf, r.o.device_status, r.o.s_init, z_init, r.o.s_pre, r.o.z_pre,
                  r.o.state_layout, ctx);
     }
-    else if (r.p.feature_order == 1) order1_chunked(r.p, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, ctx);
-    else simt_chunked(r.p, r.plan, use_scan, wsf, r.o.s_init, r.o.z_init, r.o.s_pre, r.o.z_pre, r.o.state_layout, ctx);
+    else if (r.p.feature_order == 1) order1_chunked(P, r.plan, use_scan, wsf, r.o.s_pre, r.o.z_pre, ctx);
+    else simt_chunked(P, r.plan, use_scan, wsf, r.o.s_init, r.o.z_init, r.o.s_pre, r.o.z_pre, r.o.state_layout, ctx);
+  }
+  if (r.pad && ctx.status == KATA_OK) {
+    const size_t rows = (size_t)P.B * P.H * P.T;
+    const unsigned blocks = (unsigned)((rows * (r.p.d_v / 8) + 255) / 256);
+    unpad_rows_kernel<<<blocks, 256, 0, r.o.stream>>>(static_cast<const __nv_bfloat16*>(P.out),
+                                                      static_cast<__nv_bfloat16*>(r.p.out), rows, r.p.d_v);
+    note_launch(ctx);
   }
   if (ctx.status == KATA_OK) {
     g_last_launches = ctx.launches;
