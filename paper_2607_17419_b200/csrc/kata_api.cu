@@ -83,10 +83,23 @@ bool want_tensor(int fn, const Problem& p, const Opts& o) {
   return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn, scan);
 }
 
-// The tensor-core backward covers bf16, d_k = d_v = 64, the full rank-one feature.
+// The tensor-core backward covers bf16 and the full rank-one feature: d_k = d_v = 64, narrower rows zero-padded.
 bool bwd_tensor(const Problem& p, const Opts& o) {
-  return o.impl != KATA_IMPL_SIMT && p.dtype == KATA_BF16 && p.d_k == 64 && p.d_v == 64 && p.feature_order == 2 &&
-         p.groups == 1;
+  return o.impl != KATA_IMPL_SIMT && p.dtype == KATA_BF16 && p.feature_order == 2 && p.groups == 1;
+}
+
+// Scratch of the backward: the fp32 kernels' row scalars, or the tensor-core kernels' scratch behind seven padded
+// tensors (q, k, v, dout, dq, dk, dv) when the rows are narrower than 64.
+size_t bwd_workspace(const Problem& p, const Opts& o, size_t* pad_bytes) {
+  *pad_bytes = 0;
+  if (!bwd_tensor(p, o)) return align_up(simt_bwd_workspace_elems(p.B * p.H, p.T) * sizeof(float));
+  Problem pp = p;
+  if (p.d_k < 64 || p.d_v < 64) {
+    *pad_bytes = align_up((size_t)p.B * p.H * p.T * 64 * 2);
+    pp.d_k = 64;
+    pp.d_v = 64;
+  }
+  return 7 * *pad_bytes + align_up(tc_bwd_workspace_bytes(pp));
 }
 
 // How the chunk axis is cut into scan groups, and how many floats one group state takes.
@@ -464,14 +477,44 @@ int kata_bwd_quadratic(const void* q, const void* k, const void* v, const void* 
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) ||
       !aligned16(dv))
     return KATA_ERR_ALIGNMENT;
-  const size_t need = tensor ? align_up(tc_bwd_workspace_bytes(p)) : align_up(simt_bwd_workspace_elems(B * H, T) * sizeof(float));
+  size_t pad_bytes = 0;
+  const size_t need = bwd_workspace(p, o, &pad_bytes);
   if (o.workspace == nullptr || o.workspace_bytes < need) return KATA_ERR_WORKSPACE_TOO_SMALL;
   if ((reinterpret_cast<uintptr_t>(o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;
   st = check_arch();
   if (st != KATA_OK) return st;
   LaunchCtx ctx{o.stream, 0, KATA_OK};
-  if (tensor) tc_bwd_quadratic(p, dout, dq, dk, dv, o.workspace, o.device_status, ctx);
-  else simt_bwd_quadratic(p, dout, dq, dk, dv, static_cast<float*>(o.workspace), ctx);
+  if (tensor && pad_bytes > 0) {
+    // rows zero-padded to 64 entries: the padded columns of dq, dk, dv come out zero and are dropped
+    unsigned char* w8 = static_cast<unsigned char*>(o.workspace);
+    auto buf = [&](int i) { return reinterpret_cast<__nv_bfloat16*>(w8 + (size_t)i * pad_bytes); };
+    const size_t rows = (size_t)B * H * T;
+    const unsigned blocks = (unsigned)((rows * 8 + 255) / 256);
+    const void* src[4] = {q, k, v, dout};
+    const int width[4] = {d_k, d_k, d_v, d_v};
+    for (int i = 0; i < 4; ++i) {
+      pad_rows_kernel<<<blocks, 256, 0, o.stream>>>(static_cast<const __nv_bfloat16*>(src[i]), buf(i), rows, width[i]);
+      note_launch(ctx);
+    }
+    Problem pp = p;
+    pp.q = buf(0);
+    pp.k = buf(1);
+    pp.v = buf(2);
+    pp.d_k = 64;
+    pp.d_v = 64;
+    tc_bwd_quadratic(pp, buf(3), buf(4), buf(5), buf(6), w8 + 7 * pad_bytes, o.device_status, ctx);
+    void* dst[3] = {dq, dk, dv};
+    const int wout[3] = {d_k, d_k, d_v};
+    for (int i = 0; i < 3 && ctx.status == KATA_OK; ++i) {
+      const unsigned ub = (unsigned)((rows * (wout[i] / 8) + 255) / 256);
+      unpad_rows_kernel<<<ub, 256, 0, o.stream>>>(buf(4 + i), static_cast<__nv_bfloat16*>(dst[i]), rows, wout[i]);
+      note_launch(ctx);
+    }
+  } else if (tensor) {
+    tc_bwd_quadratic(p, dout, dq, dk, dv, o.workspace, o.device_status, ctx);
+  } else {
+    simt_bwd_quadratic(p, dout, dq, dk, dv, static_cast<float*>(o.workspace), ctx);
+  }
   if (ctx.status == KATA_OK) {
     g_last_launches = ctx.launches;
     g_last_impl = tensor ? KATA_IMPL_TENSOR : KATA_IMPL_SIMT;
@@ -522,8 +565,8 @@ size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C
     Opts o;
     if (host_io || read_opts(opts, o) != KATA_OK || B < 1 || H < 1 || T < 1 || !dim_ok(d_k) || !dim_ok(d_v)) return 0;
     const Problem p{nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, o.dtype, o.feature_order, o.groups};
-    if (bwd_tensor(p, o)) return align_up(tc_bwd_workspace_bytes(p));
-    return align_up(simt_bwd_workspace_elems(B * H, T) * sizeof(float));
+    size_t pad_bytes = 0;
+    return bwd_workspace(p, o, &pad_bytes);
   }
   if (fn == KATA_FN_DECODE_STEP) {      // T and C are ignored
     Opts o;
