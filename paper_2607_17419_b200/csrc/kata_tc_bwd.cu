@@ -21,6 +21,7 @@
 #include <cuda.h>
 
 #include "kata_common.cuh"
+#include "kata_tmap.cuh"
 #include "kata_umma.cuh"
 
 namespace kata {
@@ -76,36 +77,6 @@ struct BArgs {
   int* device_status;
   int Tlen;
 };
-
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p, q;\n\t"
-      ".reg .u32 i;\n\t"
-      "mov.u32 i, 0;\n\t"
-      "KATA_WAIT_%=:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "@p bra KATA_DONE_%=;\n\t"
-      "add.u32 i, i, 1;\n\t"
-      "setp.lt.u32 q, i, %3;\n\t"
-      "@q bra KATA_WAIT_%=;\n\t"
-      "KATA_DONE_%=:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t"
-      "}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(kSpinLimit)
-      : "memory");
-  if (ok == 0) *abort_flag = 1;
-  return ok != 0;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
-__device__ __forceinline__ uint64_t at(uint64_t desc, uint32_t saddr) { return desc + (uint64_t)((saddr >> 4) & 0x3FFF); }
 
 template <int MODE>
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -446,36 +417,6 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
   if (warp == 0) tmem_dealloc(tb, TMEM_COLS);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) {
-      cudaGetLastError();
-      return nullptr;
-    }
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
-// [BH][T][64] bf16 tensor, box = 64 columns x rows x 1 head, 128B swizzle; rows beyond T read as zero.
-bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T, int rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
-  cuuint32_t box[3] = {(cuuint32_t)D, (cuuint32_t)rows, 1};
-  cuuint32_t es[3] = {1, 1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 size_t align256(size_t n) { return (n + 255) / 256 * 256; }
 
 // Pre-pass: one warp per 4 key rows (8 lanes x 16 bytes per row).  k' = k / ||k||^2 (bf16), r = 1 / ||k||^2 (fp32).
@@ -525,9 +466,9 @@ void tc_bwd_quadratic(const Problem& p, const void* dout, void* dq, void* dk, vo
   bwd_prescale_kernel<<<(unsigned)((rows + 31) / 32), 256, 0, ctx.stream>>>(static_cast<const __nv_bfloat16*>(p.k), ks, rk, rows);
   note_launch(ctx);
   CUtensorMap q128, g128, k128, v128, q64, g64, k64, v64, ks64;
-  if (!make_map(&q128, p.q, BH, p.T, MT) || !make_map(&g128, dout, BH, p.T, MT) || !make_map(&k128, p.k, BH, p.T, MT) ||
-      !make_map(&v128, p.v, BH, p.T, MT) || !make_map(&q64, p.q, BH, p.T, NT) || !make_map(&g64, dout, BH, p.T, NT) ||
-      !make_map(&k64, p.k, BH, p.T, NT) || !make_map(&v64, p.v, BH, p.T, NT) || !make_map(&ks64, ks, BH, p.T, NT)) {
+  if (!make_tile_map(&q128, p.q, BH, p.T, MT) || !make_tile_map(&g128, dout, BH, p.T, MT) || !make_tile_map(&k128, p.k, BH, p.T, MT) ||
+      !make_tile_map(&v128, p.v, BH, p.T, MT) || !make_tile_map(&q64, p.q, BH, p.T, NT) || !make_tile_map(&g64, dout, BH, p.T, NT) ||
+      !make_tile_map(&k64, p.k, BH, p.T, NT) || !make_tile_map(&v64, p.v, BH, p.T, NT) || !make_tile_map(&ks64, ks, BH, p.T, NT)) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }

@@ -21,6 +21,7 @@
 #include <cuda.h>
 
 #include "kata_common.cuh"
+#include "kata_tmap.cuh"
 #include "kata_umma.cuh"
 
 namespace kata {
@@ -69,37 +70,6 @@ struct QArgs {
   int* device_status;
   int Tlen;
 };
-
-// Bounded wait, as few instructions per poll as possible (the polling warps share the issue slots with the warps
-// that work): try_wait, exit branch, counter, loop branch.  A wait that gives up raises the abort flag; the other
-// waiters give up on their own limits.
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p, q;\n\t"
-      ".reg .u32 i;\n\t"
-      "mov.u32 i, 0;\n\t"
-      "KATA_WAIT_%=:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "@p bra KATA_DONE_%=;\n\t"
-      "add.u32 i, i, 1;\n\t"
-      "setp.lt.u32 q, i, %3;\n\t"
-      "@q bra KATA_WAIT_%=;\n\t"
-      "KATA_DONE_%=:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t"
-      "}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(kSpinLimit)
-      : "memory");
-  if (ok == 0) *abort_flag = 1;
-  return ok != 0;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
 
 // Pre-pass: one warp per 4 key rows (8 lanes x 16 bytes per row).  V' = v / ||k||^2, r = 1 / ||k||^2.
 __global__ void __launch_bounds__(256) quad_prescale_kernel(const __nv_bfloat16* __restrict__ k,
@@ -406,36 +376,6 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   if (warp == 0) tmem_dealloc(tb, TMEM_COLS);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) {
-      cudaGetLastError();
-      return nullptr;
-    }
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
-// [BH][T][64] bf16 tensor, box = 64 columns x 128 rows x 1 head, 128B swizzle; rows beyond T read as zero.
-bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T, int rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
-  cuuint32_t box[3] = {(cuuint32_t)D, (cuuint32_t)rows, 1};
-  cuuint32_t es[3] = {1, 1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 // workspace: V' [BH][T][64] bf16, then r [BH][T] bf16
@@ -455,7 +395,7 @@ void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchC
   note_launch(ctx);
   CUtensorMap tmQ, tmK, tmV;
   const int kt = KTILE / p.groups;
-  if (!make_map(&tmQ, p.q, BH, p.T, QT) || !make_map(&tmK, p.k, BH, p.T, kt) || !make_map(&tmV, vs, BH, p.T, kt)) {
+  if (!make_tile_map(&tmQ, p.q, BH, p.T, QT) || !make_tile_map(&tmK, p.k, BH, p.T, kt) || !make_tile_map(&tmV, vs, BH, p.T, kt)) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }

@@ -31,6 +31,7 @@
 #include <cuda.h>
 
 #include "kata_common.cuh"
+#include "kata_tmap.cuh"
 #include "kata_umma.cuh"
 
 namespace kata {
@@ -142,46 +143,13 @@ struct SArgs {
 #endif
 };
 
-// Bounded wait, as few instructions per poll as possible (24 warps poll most of the time and share the issue
-// slots with the warps that work): try_wait, exit branch, counter, loop branch.  A wait that gives up raises the
-// abort flag; the other waiters give up on their own limits.
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p, q;\n\t"
-      ".reg .u32 i;\n\t"
-      "mov.u32 i, 0;\n\t"
-      "KATA_WAIT_%=:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "@p bra KATA_DONE_%=;\n\t"
-      "add.u32 i, i, 1;\n\t"
-      "setp.lt.u32 q, i, %3;\n\t"
-      "@q bra KATA_WAIT_%=;\n\t"
-      "KATA_DONE_%=:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t"
-      "}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(kSpinLimit)
-      : "memory");
-  if (ok == 0) *abort_flag = 1;
-  return ok != 0;
-}
-
 __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
   const __nv_bfloat162 r = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
   return *reinterpret_cast<const uint32_t*>(&r);
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
-
-__device__ __forceinline__ uint64_t at(uint64_t desc, uint32_t saddr) { return desc + (uint64_t)((saddr >> 4) & 0x3FFF); }
 
 // Rounds 16 fp32 accumulator columns (scaled by sc) to bf16 and stores them as the 16-byte chunks c and c + 1 of a
 // 128-byte snapshot row (128B swizzle: chunk index xor row-in-atom rx).
@@ -1069,36 +1037,6 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) {
-      cudaGetLastError();
-      return nullptr;
-    }
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
-// [BH][T][64] bf16 tensor, box = 64 features x 128 tokens x 1 head, 128B swizzle; rows beyond T read as zero.
-bool make_map(CUtensorMap* tm, const void* ptr, int BH, int T) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
-  cuuint32_t box[3] = {(cuuint32_t)D, (cuuint32_t)CT, 1};
-  cuuint32_t es[3] = {1, 1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 #ifdef KATA_STREAM_EXPORT
@@ -1112,7 +1050,7 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
 #endif
   const int BH = p.B * p.H;
   CUtensorMap tmQ, tmK;
-  if (!make_map(&tmQ, p.q, BH, p.T) || !make_map(&tmK, p.k, BH, p.T)) {
+  if (!make_tile_map(&tmQ, p.q, BH, p.T, CT) || !make_tile_map(&tmK, p.k, BH, p.T, CT)) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }

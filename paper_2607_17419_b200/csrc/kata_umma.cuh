@@ -278,5 +278,42 @@ __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t chunk16)
   return row * 128u + ((chunk16 ^ (row & 7u)) << 4);
 }
 
+// ---------------------------------------------------------------------------------------------
+// helpers shared by the tensor-core kernels
+// ---------------------------------------------------------------------------------------------
+// Bounded wait, as few instructions per poll as possible (24 warps poll most of the time and share the issue
+// slots with the warps that work): try_wait, exit branch, counter, loop branch.  A wait that gives up raises the
+// abort flag; the other waiters give up on their own limits.
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u32 i;\n\t"
+      "mov.u32 i, 0;\n\t"
+      "KATA_WAIT_%=:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra KATA_DONE_%=;\n\t"
+      "add.u32 i, i, 1;\n\t"
+      "setp.lt.u32 q, i, %3;\n\t"
+      "@q bra KATA_WAIT_%=;\n\t"
+      "KATA_DONE_%=:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSpinLimit)
+      : "memory");
+  if (ok == 0) *abort_flag = 1;
+  return ok != 0;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// A descriptor with its start-address field set to a shared-memory address (the field is 14 bits of address >> 4).
+__device__ __forceinline__ uint64_t at(uint64_t desc, uint32_t saddr) { return desc + (uint64_t)((saddr >> 4) & 0x3FFF); }
+
 }  // namespace umma
 }  // namespace kata
