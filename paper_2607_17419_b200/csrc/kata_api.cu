@@ -78,8 +78,9 @@ int check_shape(int fn, int B, int H, int T, int d_k, int d_v, int C) {
 
 bool want_tensor(int fn, const Problem& p, const Opts& o) {
   const bool scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || (fn == KATA_FN_CHUNKED && o.inter_chunk == KATA_SCAN);
-  // the tensor-core kernel imports and exports the state for the plain feature only
-  if (p.groups != 1 && fn == KATA_FN_CHUNKED && (o.s_pre != nullptr || o.s_init != nullptr)) return false;
+  // the tensor-core kernel imports and exports the state, and runs groups of tiles, for the plain feature only
+  if (p.groups != 1 && fn != KATA_FN_QUADRATIC && (o.s_pre != nullptr || o.s_init != nullptr)) return false;
+  if (p.groups != 1 && scan && o.scan_group > 0) return false;
   return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn, scan);
 }
 
@@ -139,6 +140,15 @@ int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanP
     plan.chunks_per_group = G;
     plan.n_groups = (NC + G - 1) / G;
     plan.rounds = plan.n_groups > 2 ? ceil_log2(plan.n_groups - 1) : 0;
+    return KATA_OK;
+  }
+  if (tensor && p.groups != 1) {
+    // blockwise map on the tensor cores: one pass per head whatever the entry point (a single group is a valid
+    // grouping; the grouped passes exist for the plain feature only)
+    state_elems = 0;
+    plan.chunks_per_group = NC;
+    plan.n_groups = 1;
+    plan.rounds = 0;
     return KATA_OK;
   }
   int slices;

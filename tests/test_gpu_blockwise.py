@@ -28,8 +28,9 @@ def test_blockwise_forms(form, dtype, dk, dv, g):
     w = inputs.gaussian_workload(f"mg_{dtype}_{dk}_{dv}_{g}", dtype, 2, 2, 333, dk, dv, 64, 300 + dk + g)
     o = FORMS[form](*dev_tensors(w), feature_groups=g)
     torch.cuda.synchronize()
-    # the quadratic and the one-pass chunked form have tensor-core kernels for the blockwise map (bf16, d = 64)
-    tensor = form in ("quadratic", "chunked_seq") and (dtype, dk, dv) == ("bf16", 64, 64)
+    # tensor-core kernels for the blockwise map (bf16, d = 64): the quadratic form and the chunked form in one pass
+    # per head, which is also what the scan forms are planned as when the grouping is left to the library
+    tensor = (dtype, dk, dv) == ("bf16", 64, 64)
     assert kb.kata_last_impl() == (kb.KATA_IMPL_TENSOR if tensor else kb.KATA_IMPL_SIMT)
     gpu = to_numpy64(o)
     for b in range(w.B):
@@ -163,6 +164,20 @@ def test_blockwise_full_size_sampled_rows(g):
         del o, gpu
 
 
+def test_blockwise_explicit_grouping_runs_on_the_fp32_kernels():
+    import torch
+    w = inputs.gaussian_workload("mg_grouped", "bf16", 1, 2, 700, 64, 64, 64, 77)
+    o = kb.kata_chunk_state_scan(*dev_tensors(w), feature_groups=2, scan_group=3)
+    torch.cuda.synchronize()
+    assert kb.kata_last_impl() == kb.KATA_IMPL_SIMT
+    gpu = to_numpy64(o)
+    for h in range(w.H):
+        ref = ko.kata_quadratic(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h], "psd_direct:g2")[0]
+        check(gpu[0, h], ref, "bf16", f"M2 explicit grouping head {h}")
+    assert kb.kata_scan_plan(kb.KATA_FN_CHUNK_STATE_SCAN, 1, 2, 700, 64, 64, 64,
+                             kb.make_opts(kb.KATA_BF16, feature_groups=2))[0] == 1          # the library's own plan
+
+
 def test_blockwise_argument_checks():
     import torch
     w = inputs.gaussian_workload("mg_args", "f32", 1, 1, 64, 16, 16, 64, 1)
@@ -173,4 +188,5 @@ def test_blockwise_argument_checks():
         kb.kata_fwd_quadratic(q, k, v, feature_groups=2, feature_order=1)
     wb = inputs.gaussian_workload("mg_args_bf16", "bf16", 1, 1, 64, 64, 64, 64, 1)
     with pytest.raises(kb.KataError):
-        kb.kata_fwd_chunked(*dev_tensors(wb), feature_groups=2, inter_chunk=kb.KATA_SCAN, impl=kb.KATA_IMPL_TENSOR)
+        kb.kata_fwd_chunked(*dev_tensors(wb), feature_groups=2, inter_chunk=kb.KATA_SCAN, scan_group=4,
+                            impl=kb.KATA_IMPL_TENSOR)          # an explicit grouping of the blockwise map: fp32 kernels
