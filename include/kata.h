@@ -193,9 +193,9 @@ int kata_decode_step(const void* q, const void* k, const void* v, void* out, flo
  * recomputed (no saved activations are needed), O(T^2) work, fp32 arithmetic, every sum in a fixed order
  * (bit-reproducible).  Rows whose normaliser is 0 (out = 0) and zero rows of q or k get zero gradients.
  * feature_order, feature_groups as in the forward; inter_chunk, scan_group, state_layout are ignored;
- * s_pre/z_pre/s_init/z_init must be null.  Tensor-core kernels for bf16, feature_order 2, feature_groups 1 (rows
- * narrower than 64 zero-padded in the workspace; the weights P and E pass through bf16 there, as P does in the
- * forward); fp32 kernels for everything else.
+ * s_pre/z_pre/s_init/z_init must be null.  Tensor-core kernels for bf16 and feature_order 2: feature_groups 1 with
+ * d_k = d_v = 64 or narrower rows zero-padded in the workspace, feature_groups 2 or 4 with d_k = d_v = 64 (the
+ * weights P and E pass through bf16 there, as P does in the forward); fp32 kernels for everything else.
  * Workspace: kata_workspace_bytes(KATA_FN_BWD_QUADRATIC, B, H, T, d_k, d_v, 0, opts).
  */
 int kata_bwd_quadratic(const void* q, const void* k, const void* v, const void* dout, void* dq, void* dk, void* dv,

@@ -84,9 +84,12 @@ bool want_tensor(int fn, const Problem& p, const Opts& o) {
   return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn, scan);
 }
 
-// The tensor-core backward covers bf16 and the full rank-one feature: d_k = d_v = 64, narrower rows zero-padded.
+// The tensor-core backward covers bf16: the full rank-one feature with d_k = d_v = 64 or narrower rows zero-padded,
+// and the blockwise map (g = 2, 4) at d_k = d_v = 64.
 bool bwd_tensor(const Problem& p, const Opts& o) {
-  return o.impl != KATA_IMPL_SIMT && p.dtype == KATA_BF16 && p.feature_order == 2 && p.groups == 1;
+  if (o.impl == KATA_IMPL_SIMT || p.dtype != KATA_BF16 || p.feature_order != 2) return false;
+  // feature blocks depend on the true width: no padding there
+  return p.groups == 1 || ((p.groups == 2 || p.groups == 4) && p.d_k == 64 && p.d_v == 64);
 }
 
 // Scratch of the backward: the fp32 kernels' row scalars, or the tensor-core kernels' scratch behind seven padded

@@ -33,13 +33,14 @@ constexpr int D = 64;
 constexpr int MT = 128;          // rows of the fixed tile (TMEM lanes)
 constexpr int NT = 64;           // rows of a streamed tile
 constexpr int NSTAGE = 4;
-constexpr int NBUF = 3;
+constexpr int NBUF_MAX = 3;
 constexpr int NTHREADS = 384;
 constexpr int WARP_BLD0 = 4;
 enum { MODE_DQ = 0, MODE_DKV = 1 };
 
-constexpr uint32_t COL_B = 0;      // 3 x 128 fp32: [S | C] of a streamed tile; the bf16 weights overwrite columns
-                                   // [0,32) of each half
+constexpr uint32_t COL_B = 0;      // score buffers of (G + 1) x 64 fp32 columns: [S_0 | .. | S_{G-1} | C] of a streamed tile
+                                   // (G feature groups; three buffers for G = 1, two for G = 2, one for G = 4); the
+                                   // bf16 weights overwrite columns [0,32) of each block
 constexpr uint32_t COL_ACC = 384;  // 2 x 64 fp32 accumulators
 constexpr uint32_t TMEM_COLS = 512;
 
@@ -78,7 +79,9 @@ struct BArgs {
   int Tlen;
 };
 
-template <int MODE>
+// G feature groups of the blockwise map: s_g = q_g . k_g per group, a = r sum_g s_g^2, e_g = 2 g s_g; dq and u are
+// formed group by group (N = 64 / G columns of the accumulator, the B operand offset into the 128-byte rows).
+template <int MODE, int G>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CUtensorMap tmX2,
               const __grid_constant__ CUtensorMap tmY1, const __grid_constant__ CUtensorMap tmY2,
@@ -94,6 +97,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
   __shared__ int abort_s;
   volatile int* abort_flag = &abort_s;
 
+  constexpr int NBUF = G == 1 ? 3 : G == 2 ? 2 : 1;
+  constexpr uint32_t BW = (G + 1) * 64;            // columns of a score buffer
+  constexpr uint32_t CB = G * 64;                  // its C block
+  constexpr int MG = D / G;                        // features per group
+  static_assert(NBUF * BW <= COL_ACC, "TMEM columns");
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bh = blockIdx.y;
   const int n_stream = (args.Tlen + NT - 1) / NT;                 // streamed tiles of the whole sequence
@@ -113,7 +121,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
       mbar_init(bar(BAR_FULL + i), 1 + 32);
       mbar_init(bar(BAR_EMPTY + i), 2);
     }
-    for (int i = 0; i < NBUF; ++i) {
+    for (int i = 0; i < NBUF_MAX; ++i) {
       mbar_init(bar(BAR_SFULL + i), 1);
       mbar_init(bar(BAR_PFULL + i), 256);
       mbar_init(bar(BAR_PEMPTY + i), 1);
@@ -188,11 +196,12 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
         tc_fence_after();
         const uint32_t a1 = smem_u32(y1(s)), a2 = smem_u32(y2(s));
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          mma_f16_ss(tb + COL_B + b * 128, at(dk, x1 + ks * 32), at(dk, a1 + ks * 32), idesc, ks > 0);
+        for (int ks = 0; ks < 4; ++ks)      // 16 features per step; group ks / (4 / G) has its own 64 score columns
+          mma_f16_ss(tb + COL_B + b * BW + (ks / (4 / G)) * 64, at(dk, x1 + ks * 32), at(dk, a1 + ks * 32), idesc,
+                     (ks % (4 / G)) > 0);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          mma_f16_ss(tb + COL_B + b * 128 + 64, at(dk, x2 + ks * 32), at(dk, a2 + ks * 32), idesc, ks > 0);
+          mma_f16_ss(tb + COL_B + b * BW + CB, at(dk, x2 + ks * 32), at(dk, a2 + ks * 32), idesc, ks > 0);
         mma_commit(bar(BAR_SFULL + b));
         mma_commit(bar(BAR_EMPTY + s));
       }
@@ -209,23 +218,31 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
              wait_or_abort(bar(BAR_PFULL + b), (j / NBUF) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
+        // group g: N = 64 / G accumulator columns, the B operand starts 2 * 64 / G bytes further into the rows
+        const uint32_t idg = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, MG);
         if (MODE == MODE_DQ) {
           if (j >= ntiles) {      // the first sweep only sums the row scalars: nothing to multiply
             const uint32_t kp = smem_u32(y3(s));
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              mma_f16_ts(tb + COL_ACC, tb + COL_B + b * 128 + ks * 8, at(dmn, kp + ks * 2048), idesc,
-                         (j > ntiles || ks > 0) ? 1u : 0u);
+            for (int g = 0; g < G; ++g)
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks)
+                mma_f16_ts(tb + COL_ACC + g * MG, tb + COL_B + b * BW + g * 64 + ks * 8,
+                           at(dmn, kp + ks * 2048 + g * MG * 2), idg, (j > ntiles || ks > 0) ? 1u : 0u);
           }
         } else {
           const uint32_t qa = smem_u32(y1(s)), ga = smem_u32(y2(s));
+          // P^T sits over the first score block for G = 1 and over the C block otherwise; E_g^T over the other / its own
+          const uint32_t pcol = G == 1 ? 0u : CB;
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)      // dv~ += P^T dout
-            mma_f16_ts(tb + COL_ACC, tb + COL_B + b * 128 + ks * 8, at(dmn, ga + ks * 2048), idesc, (j > 0 || ks > 0) ? 1u : 0u);
+            mma_f16_ts(tb + COL_ACC, tb + COL_B + b * BW + pcol + ks * 8, at(dmn, ga + ks * 2048), idesc, (j > 0 || ks > 0) ? 1u : 0u);
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)      // u += E^T Q
-            mma_f16_ts(tb + COL_ACC + 64, tb + COL_B + b * 128 + 64 + ks * 8, at(dmn, qa + ks * 2048), idesc,
-                       (j > 0 || ks > 0) ? 1u : 0u);
+          for (int g = 0; g < G; ++g)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)    // u_g += E_g^T Q_g
+              mma_f16_ts(tb + COL_ACC + 64 + g * MG, tb + COL_B + b * BW + (G == 1 ? 64u : (uint32_t)g * 64u) + ks * 8,
+                         at(dmn, qa + ks * 2048 + g * MG * 2), idg, (j > 0 || ks > 0) ? 1u : 0u);
         }
         mma_commit(bar(BAR_PEMPTY + b));
         mma_commit(bar(BAR_EMPTY + s));
@@ -260,6 +277,85 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
            wait_or_abort(bar(BAR_SFULL + b), (j / NBUF) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
+      if constexpr (G > 1) {
+        // one block of 64 score columns per group, then the C block; this warp's 32 columns of each
+        const uint32_t bcol = tmem_addr(tb, q4 * 32, COL_B + b * BW + ch * 32);
+        uint32_t cvg[32], sg[32], pk[16];
+        tmem_ld32(bcol + CB, cvg);
+        tmem_wait_ld(cvg);
+        const bool first = MODE == MODE_DQ && j < ntiles;
+        const bool diag = MODE == MODE_DQ ? (n0 + 31 > m0) : (n0 < m0 + MT - 1);
+        auto dead = [&](int c) { return MODE == MODE_DQ ? (n0 + c > grow) : (n0 + c < grow); };
+        float2 cf[16], ss[16];
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const float2 c2 = make_float2(__uint_as_float(cvg[c]), __uint_as_float(cvg[c + 1]));
+          if (MODE == MODE_DQ) {
+            // second sweep: 2 (c - dout.o) / D; first sweep: c as it is
+            cf[c / 2] = first ? c2 : __fmul2_rn(__fadd2_rn(c2, make_float2(-del_row, -del_row)), make_float2(2.f * inv_row, 2.f * inv_row));
+          } else {
+            const float4 st = reinterpret_cast<const float4*>(sc(s) + ch * 256)[c / 2];
+            cf[c / 2] = __fmul2_rn(__fadd2_rn(c2, make_float2(-st.y, -st.w)), make_float2(2.f * st.x, 2.f * st.z));
+          }
+          if (diag && !first) {
+            if (dead(c)) cf[c / 2].x = 0.f;
+            if (dead(c + 1)) cf[c / 2].y = 0.f;
+          }
+          ss[c / 2] = make_float2(0.f, 0.f);
+        }
+#pragma unroll 1
+        for (int g = 0; g < G; ++g) {
+          tmem_ld32(bcol + g * 64, sg);
+          tmem_wait_ld(sg);
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            const float2 s2 = make_float2(__uint_as_float(sg[c]), __uint_as_float(sg[c + 1]));
+            ss[c / 2] = __ffma2_rn(s2, s2, ss[c / 2]);
+            const float2 e2 = __fmul2_rn(cf[c / 2], s2);
+            pk[c / 2] = pack_bf16(e2.x, e2.y);
+          }
+          if (first) continue;
+          // E_g goes over columns [0,32) of its own block, which the column-half-0 warp reads
+          tc_fence_before();
+          asm volatile("bar.sync %0, 64;" ::"r"(1 + (int)q4) : "memory");
+          tc_fence_after();
+          tmem_st16(tmem_addr(tb, q4 * 32, COL_B + b * BW + g * 64 + ch * 16), pk);
+        }
+        if (first) {
+          // a = r_i sum_g s_g^2 for the keys n <= this query; D_t += a, sum += a c
+          const float2* cs = reinterpret_cast<const float2*>(sc(s) + ch * 128);
+          float2 d2 = make_float2(0.f, 0.f), m2 = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            float2 a2 = __fmul2_rn(ss[c / 2], cs[c / 2]);
+            if (diag) {
+              if (dead(c)) a2.x = 0.f;
+              if (dead(c + 1)) a2.y = 0.f;
+            }
+            d2 = __fadd2_rn(d2, a2);
+            m2 = __ffma2_rn(a2, cf[c / 2], m2);
+          }
+          sum_d += d2.x + d2.y;
+          sum_m += m2.x + m2.y;
+        } else if (MODE == MODE_DKV) {
+          // P^T = sum_g s_g^2 / D_t over the C block (both warps of the quadrant hold its scores since the first sync)
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            const float4 st = reinterpret_cast<const float4*>(sc(s) + ch * 256)[c / 2];
+            float2 p2 = __fmul2_rn(ss[c / 2], make_float2(st.x, st.z));
+            if (diag) {
+              if (dead(c)) p2.x = 0.f;
+              if (dead(c + 1)) p2.y = 0.f;
+            }
+            pk[c / 2] = pack_bf16(p2.x, p2.y);
+          }
+          tmem_st16(tmem_addr(tb, q4 * 32, COL_B + b * BW + CB + ch * 16), pk);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_PFULL + b));
+        continue;
+      }
       const uint32_t scol = tmem_addr(tb, q4 * 32, COL_B + b * 128 + ch * 32);
       uint32_t sv[32], cv[32], pe[16], pp[16];
       tmem_ld32(scol, sv);
@@ -472,8 +568,8 @@ void tc_bwd_quadratic(const Problem& p, const void* dout, void* dq, void* dk, vo
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-  auto kq = tc_bwd_kernel<MODE_DQ>;
-  auto kkv = tc_bwd_kernel<MODE_DKV>;
+  auto kq = p.groups == 1 ? tc_bwd_kernel<MODE_DQ, 1> : p.groups == 2 ? tc_bwd_kernel<MODE_DQ, 2> : tc_bwd_kernel<MODE_DQ, 4>;
+  auto kkv = p.groups == 1 ? tc_bwd_kernel<MODE_DKV, 1> : p.groups == 2 ? tc_bwd_kernel<MODE_DKV, 2> : tc_bwd_kernel<MODE_DKV, 4>;
   if (cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
       cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
     cudaGetLastError();

@@ -180,8 +180,9 @@ def test_backward_argument_checks(L):
     assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 64, 64, 0, o) == up(rows * 2 * 4)
     o = kb.make_opts(kb.KATA_BF16)
     assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 64, 64, 0, o) == up(rows * 128) + up(rows * 4) + up(rows * 8)
-    o = kb.make_opts(kb.KATA_BF16, feature_groups=2)
-    assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 64, 64, 0, o) == up(rows * 2 * 4)
+    o = kb.make_opts(kb.KATA_BF16, feature_groups=2)          # blockwise map at d = 64: tensor-core kernels too
+    assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 64, 64, 0, o) == up(rows * 128) + up(rows * 4) + up(rows * 8)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 32, 32, 0, o) == up(rows * 2 * 4)     # narrower: fp32 kernels
     # narrower bf16 rows: seven padded tensors in front of the tensor-core scratch
     o = kb.make_opts(kb.KATA_BF16)
     assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 32, 16, 0, o) == \

@@ -36,7 +36,8 @@ def check_grads(w, feature, seed=5, **kw):
     assert int(st.item()) == 0
     # tensor-core kernels for bf16 and the full rank-one feature (pre-pass, dq with the row scalars, dk/dv); rows
     # narrower than 64 are zero-padded (four copies in, three out)
-    tensor = (w.dtype == "bf16" and feature == "psd_direct" and kw.get("impl", kb.KATA_IMPL_AUTO) != kb.KATA_IMPL_SIMT)
+    tensor = (w.dtype == "bf16" and kw.get("impl", kb.KATA_IMPL_AUTO) != kb.KATA_IMPL_SIMT and
+              (feature == "psd_direct" or (feature.startswith("psd_direct:g") and w.d_k == 64 and w.d_v == 64)))
     padded = tensor and (w.d_k < 64 or w.d_v < 64)
     assert kb.kata_last_impl() == (kb.KATA_IMPL_TENSOR if tensor else kb.KATA_IMPL_SIMT)
     assert kb.kata_last_launch_count() == (10 if padded else 3 if tensor else 2)
@@ -85,6 +86,17 @@ def test_backward_tensor_zero_rows():
     assert torch.all(dq[0, 0, [0, 1, 5, 128, 256]] == 0)
     dq2, dk2, dv2 = check_grads(w, "psd_direct")
     assert torch.equal(dq, dq2) and torch.equal(dk, dk2) and torch.equal(dv, dv2)      # fixed summation order
+
+
+@pytest.mark.parametrize("g", [2, 4])
+@pytest.mark.parametrize("T", [1, 63, 64, 65, 128, 129, 200, 257, 600])
+def test_backward_blockwise_tensor_tile_boundaries(g, T):
+    """Blockwise map on the tensor-core backward kernels (bf16, d = 64), and the fp32 kernels on the same inputs."""
+    w = inputs.gaussian_workload(f"bwd_tc_mg_{T}", "bf16", 1, 2, T, 64, 64, 64, 880 + T + g)
+    a = check_grads(w, f"psd_direct:g{g}", feature_groups=g)
+    b = check_grads(w, f"psd_direct:g{g}", feature_groups=g, impl=kb.KATA_IMPL_SIMT)
+    for x, y in zip(a, b):
+        assert float((x.float() - y.float()).abs().max()) <= 4e-2 * max(1.0, float(y.float().abs().max()))
 
 
 @pytest.mark.parametrize("g", [2, 4])
@@ -137,7 +149,7 @@ def test_backward_argument_checks():
     w = inputs.gaussian_workload("bwd_args", "bf16", 1, 1, 64, 64, 64, 64, 1)
     q, k, v = dev_tensors(w)
     with pytest.raises(kb.KataError):
-        kb.kata_bwd_quadratic(q, k, v, v, impl=kb.KATA_IMPL_TENSOR, feature_groups=2)    # fp32 kernels only
+        kb.kata_bwd_quadratic(q, k, v, v, impl=kb.KATA_IMPL_TENSOR, feature_order=1)     # fp32 kernels only
     with pytest.raises(kb.KataError):
         kb.kata_bwd_quadratic(q, k, v, v, feature_groups=3)
 
