@@ -480,6 +480,10 @@ def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
                                    frac_of_bf16_burst=flb / (ms * 1e-3) / 1e12 / peaks["bf16_burst"],
                                    launches=kb.kata_last_launch_count(),
                                    impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
+    ms = timed(lambda: kb.kata_bwd_quadratic(q2, k2, v2, g2, dq2, dk2, dv2, feature_groups=2))
+    res["bwd_quadratic_c2_M2"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=flb / (ms * 1e-3) / 1e12,
+                                      launches=kb.kata_last_launch_count(),
+                                      impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
     # first-order feature (rows of q, k as features; matched d x d state, C = 128): shapes of the paper's scan
     # benchmark; HBM-bound, 512 algorithmic bytes per token and head (q, k, v read, o written)
     for Bo, To in ((1, 8192), (1, 131072), (4, 32768), (16, 8192), (32, 32768)):

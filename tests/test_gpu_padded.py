@@ -69,3 +69,20 @@ def test_padding_is_not_used_where_the_width_matters():
     assert kb.kata_last_impl() == kb.KATA_IMPL_SIMT
     with pytest.raises(kb.KataError):
         kb.kata_fwd_quadratic(q, k, v, feature_groups=2, impl=kb.KATA_IMPL_TENSOR)
+
+
+def test_padded_host_io_entry_matches_device_entry():
+    """Host buffers in, host buffer out, rows padded inside the workspace: the same bits as the device entry."""
+    import torch
+    w = inputs.gaussian_workload("pad_host", "bf16", 2, 2, 300, 32, 16, 64, 61)
+    q, k, v = dev_tensors(w)
+    for fn, call in ((kb.KATA_FN_QUADRATIC, kb.kata_fwd_quadratic), (kb.KATA_FN_CHUNKED, kb.kata_fwd_chunked),
+                     (kb.KATA_FN_CHUNK_STATE_SCAN, kb.kata_chunk_state_scan)):
+        ref = call(q, k, v)
+        assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR
+        hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+        ho = torch.empty_like(hv).pin_memory()
+        kb.kata_fwd_host(fn, hq, hk, hv, ho)
+        torch.cuda.synchronize()
+        assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR
+        assert torch.equal(ho, ref.cpu())
