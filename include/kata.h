@@ -77,9 +77,7 @@ enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2,
  *                 psi_Mg(u) = (u_1 u_1^T, ..., u_g u_g^T) of the normalised row cut into g blocks of d_k/g
  *                 entries ("KATA-Mg"), with <psi(q),psi(k)> = sum_a (q_a . k_a)^2.  The state layouts then hold
  *                 the g blocks one after the other: DIRECT n_psi = g (d_k/g)^2, PACKED n_psi = g m(m+1)/2 with
- *                 m = d_k/g.  On the tensor-core path (bf16, d_k = d_v = 64) the scan forms of the blockwise map
- *                 run as a single group unless scan_group is given (then, and for any state hand-off, the fp32
- *                 kernels run).
+ *                 m = d_k/g.
  *  state_layout   layout of the exported prefix states for feature_order 2:
  *                 DIRECT  n_psi = d_k^2, row a*d_k+b holds the (a,b) entry of sum k_hat k_hat^T (x) v;
  *                 PACKED  n_psi = d_k(d_k+1)/2, upper triangle a<=b in row-major order, diagonal

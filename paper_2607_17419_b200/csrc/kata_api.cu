@@ -78,9 +78,6 @@ int check_shape(int fn, int B, int H, int T, int d_k, int d_v, int C) {
 
 bool want_tensor(int fn, const Problem& p, const Opts& o) {
   const bool scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || (fn == KATA_FN_CHUNKED && o.inter_chunk == KATA_SCAN);
-  // the tensor-core kernel imports and exports the state, and runs groups of tiles, for the plain feature only
-  if (p.groups != 1 && fn != KATA_FN_QUADRATIC && (o.s_pre != nullptr || o.s_init != nullptr)) return false;
-  if (p.groups != 1 && scan && o.scan_group > 0) return false;
   return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn, scan);
 }
 
@@ -143,15 +140,6 @@ int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanP
     plan.chunks_per_group = G;
     plan.n_groups = (NC + G - 1) / G;
     plan.rounds = plan.n_groups > 2 ? ceil_log2(plan.n_groups - 1) : 0;
-    return KATA_OK;
-  }
-  if (tensor && p.groups != 1) {
-    // blockwise map on the tensor cores: one pass per head whatever the entry point (a single group is a valid
-    // grouping; the grouped passes exist for the plain feature only)
-    state_elems = 0;
-    plan.chunks_per_group = NC;
-    plan.n_groups = 1;
-    plan.rounds = 0;
     return KATA_OK;
   }
   int slices;
@@ -340,7 +328,7 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
     // tensor-core path, state advanced in place: every value slice of a head reads the normaliser state and one of
     // them writes it, so the kernel reads a copy of z_init
     if (fn == KATA_FN_CHUNKED && r.tensor && r.o.z_init != nullptr && r.o.z_init == r.o.z_pre)
-      r.inner_bytes = align_up((size_t)B * H * decode_n_psi(d_k, r.o.state_layout, 2, 1) * sizeof(float));
+      r.inner_bytes = align_up((size_t)B * H * decode_n_psi(d_k, r.o.state_layout, 2, r.o.groups) * sizeof(float));
   }
   r.inner_bytes += 4 * r.pad_bytes;
   return KATA_OK;
@@ -380,7 +368,7 @@ int run_device(int fn, Prepared& r, void* ws) {
     } else if (r.tensor) {
       const float* z_init = r.o.z_init;
       if (fn == KATA_FN_CHUNKED && z_init != nullptr && z_init == r.o.z_pre) {
-        const size_t nb = (size_t)r.p.B * r.p.H * decode_n_psi(r.p.d_k, r.o.state_layout, 2, 1) * sizeof(float);
+        const size_t nb = (size_t)r.p.B * r.p.H * decode_n_psi(r.p.d_k, r.o.state_layout, 2, r.o.groups) * sizeof(float);
         if (cudaMemcpyAsync(wsf, z_init, nb, cudaMemcpyDeviceToDevice, r.o.stream) != cudaSuccess) {
           cudaGetLastError();
           return KATA_ERR_CUDA;

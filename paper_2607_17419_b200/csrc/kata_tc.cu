@@ -8,8 +8,7 @@ bool tc_supported(const Problem& p, int fn, bool scan) {
   // first-order feature: the chunked and scan forms (the quadratic form stays on the fp32 kernel)
   if (p.feature_order == 1) return fn == KATA_FN_CHUNKED || fn == KATA_FN_CHUNK_STATE_SCAN;
   if (p.feature_order != 2) return false;
-  // blockwise map (g = 2, 4): the quadratic form and the chunked form in one pass per head (the scan forms, when
-  // the grouping is left to the library, are planned as a single group; an explicit grouping runs on the fp32 kernels)
+  // blockwise map (g = 2, 4): the same kernels with the state blocks of the feature groups only
   (void)scan;
   if (p.groups != 1)
     return (fn == KATA_FN_QUADRATIC || fn == KATA_FN_CHUNKED || fn == KATA_FN_CHUNK_STATE_SCAN) &&

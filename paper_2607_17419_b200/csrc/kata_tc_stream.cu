@@ -171,22 +171,33 @@ __device__ __forceinline__ uint32_t sp_block(int p) { return (0x43102210u >> (4 
 __device__ __forceinline__ uint32_t sp_koff(int p) { return p == 3 ? 64u : (p == 4 || p == 5) ? 32u : 0u; }
 
 #ifdef KATA_STREAM_EXPORT
+// Row of entry (a, b) of the exported state (a, b in the same feature group): the g blocks follow one another, each
+// the direct m x m layout or the packed upper triangle (rows of la <= lb, off-diagonal entries times sqrt(2)).
+template <int G>
+__device__ __forceinline__ int state_row(int a, int b, bool packed) {
+  constexpr int m = D / G;
+  const int gb = a / m, la = a - gb * m, lb = b - gb * m;
+  return packed ? gb * (m * (m + 1) / 2) + la * m - la * (la - 1) / 2 + (lb - la) : gb * m * m + la * m + lb;
+}
+
 // The state after the last token, from the TMEM accumulators to the public layout (one call per thread of the
 // four auxiliary warps; kept out of line so that it does not weigh on the register allocation of the main loop).
+template <int G>
 __device__ __noinline__ void export_state(uint32_t tb, uint32_t q4, int t, float* s_final, float* z_final, int layout,
                                           int bh, int v0, int slice) {
+  using geo = Geo<G>;
   tc_fence_after();
   const bool packed = layout == KATA_LAYOUT_PACKED;
-  const int n_psi = packed ? D * (D + 1) / 2 : D * D;
+  constexpr int m = D / G;
+  const int n_psi = G * (packed ? m * (m + 1) / 2 : m * m);
   float* sf = s_final + (size_t)bh * n_psi * D + v0;
-  auto prow = [&](int a, int b) { return a * D - a * (a - 1) / 2 + (b - a); };   // packed row of a <= b
   const int vv = t & 7;
   uint32_t scol = tmem_addr(tb, q4 * 32, COL_S);
 #pragma unroll 1
   for (int be = 0; be < 4; ++be) {
     const int b = 16 * be + (t >> 3);
 #pragma unroll 1
-    for (int al = 0; al <= be; ++al, scol += 16) {
+    for (int al = geo::first(be); al <= be; ++al, scol += 16) {
       uint32_t z[16];
       tmem_ld16(scol, z);
       tmem_wait_ld(z);
@@ -195,41 +206,43 @@ __device__ __noinline__ void export_state(uint32_t tb, uint32_t q4, int t, float
         const int a = 16 * al + i;
         const float val = __uint_as_float(z[i]);
         if (packed) {
-          if (a <= b) sf[(size_t)prow(a, b) * D + vv] = (a == b) ? val : val * 1.41421356237309504880f;
+          if (a <= b) sf[(size_t)state_row<G>(a, b, true) * D + vv] = (a == b) ? val : val * 1.41421356237309504880f;
         } else {
-          sf[(size_t)(a * D + b) * D + vv] = val;
-          if (al < be) sf[(size_t)(b * D + a) * D + vv] = val;     // the dropped half of the symmetric state
+          sf[(size_t)state_row<G>(a, b, false) * D + vv] = val;
+          if (al < be) sf[(size_t)state_row<G>(b, a, false) * D + vv] = val;     // the dropped half of the symmetric state
         }
       }
     }
   }
   if (slice == 0 && q4 < 2) {
     float* zf = z_final + (size_t)bh * n_psi;
-    const int b = t;
+    const int b = t, bz = b >> 4, fz = geo::first(bz);
 #pragma unroll 1
-    for (int al = 0; al < 4; ++al) {
+    for (int al = 0; al < 4; ++al) {      // the load is warp-wide: every lane walks all four a-blocks
       uint32_t z[16];
-      tmem_ld16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
+      tmem_ld16(tmem_addr(tb, q4 * 32, geo::Z + 16 * al), z);
       tmem_wait_ld(z);
+      if (al < fz || al >= fz + geo::BPG) continue;      // a-block outside the feature group of this lane's b
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const int a = 16 * al + i;
         const float val = __uint_as_float(z[i]);
         if (packed) {
-          if (a <= b) zf[prow(a, b)] = (a == b) ? val : val * 1.41421356237309504880f;
+          if (a <= b) zf[state_row<G>(a, b, true)] = (a == b) ? val : val * 1.41421356237309504880f;
         } else {
-          zf[a * D + b] = val;
+          zf[state_row<G>(a, b, false)] = val;
         }
       }
     }
   }
 }
 
-// The accumulators as they are (224 columns x 128 lanes, column-major) for the scan over groups of tiles.
+// The accumulators as they are (up to 224 columns x 128 lanes, column-major) for the scan over groups of tiles.
+template <int G>
 __device__ __noinline__ void export_compact(uint32_t tb, uint32_t q4, int t, float* dst) {
   tc_fence_after();
 #pragma unroll 1
-  for (int c = 0; c < 224; c += 16) {
+  for (int c = 0; c < (int)Geo<G>::Z + 64; c += 16) {
     uint32_t z[16];
     tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + c), z);
     tmem_wait_ld(z);
@@ -242,18 +255,21 @@ __device__ __noinline__ void export_compact(uint32_t tb, uint32_t q4, int t, flo
 // accumulators that export_compact writes) into the TMEM accumulators (the inverse of export_state; same thread
 // <-> row mapping), and its bf16 snapshot into snapshot buffer 0, which the reads of the first tile use.  One
 // call per thread of the four auxiliary warps, before the pipeline starts.
+template <int G>
 __device__ __noinline__ void import_state(uint32_t tb, unsigned char* sp, uint32_t q4, int t, const float* s_init,
                                           const float* z_init, int layout, int bh, int v0, const float* comp) {
+  using geo = Geo<G>;
   const bool packed = layout == KATA_LAYOUT_PACKED;
-  const int n_psi = packed ? D * (D + 1) / 2 : D * D;
+  constexpr int m = D / G;
+  const int n_psi = G * (packed ? m * (m + 1) / 2 : m * m);
   const float* sf = comp ? nullptr : s_init + (size_t)bh * n_psi * D + v0;
   const float* zf = comp ? nullptr : z_init + (size_t)bh * n_psi;
-  // entry (a, b) of the symmetric state: DIRECT row a D + b, PACKED the row of (min, max) with sqrt(2) taken out
+  // entry (a, b) of the symmetric state: DIRECT its own row, PACKED the row of (min, max) with sqrt(2) taken out
   auto srow = [&](int a, int b, float& scale) -> int {
-    if (!packed) { scale = 1.f; return a * D + b; }
+    if (!packed) { scale = 1.f; return state_row<G>(a, b, false); }
     const int lo = a < b ? a : b, hi = a < b ? b : a;
     scale = lo == hi ? 1.f : 0.70710678118654752440f;
-    return lo * D - lo * (lo - 1) / 2 + (hi - lo);
+    return state_row<G>(lo, hi, true);
   };
   const int bloc = t >> 3, vv = t & 7;
   uint32_t scol = tmem_addr(tb, q4 * 32, COL_S);
@@ -264,7 +280,7 @@ __device__ __noinline__ void import_state(uint32_t tb, unsigned char* sp, uint32
     const int p = 2 * be + (bloc >> 3);
     unsigned char* row = sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128;
 #pragma unroll 1
-    for (int al = 0; al <= be; ++al, scol += 16, col += 16) {
+    for (int al = geo::first(be); al <= be; ++al, scol += 16, col += 16) {
       uint32_t z[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
@@ -277,27 +293,30 @@ __device__ __noinline__ void import_state(uint32_t tb, unsigned char* sp, uint32
         }
       }
       tmem_st16(scol, z);
-      snap_store16(row, (sp_koff(p) >> 4) + 2 * al, (uint32_t)vv, z, al < be ? 2.f : 1.f);
+      snap_store16(row, (sp_koff(p) >> 4) + 2 * (al - geo::first(be)), (uint32_t)vv, z, al < be ? 2.f : 1.f);
     }
   }
   if (q4 < 2) {
-    const int b = t, bz = b >> 4, pz = b >> 3;
+    const int b = t, bz = b >> 4, fz = geo::first(bz), pz = b >> 3;
     unsigned char* rowz = sp + sp_block(pz) * SP_BLOCK + 8 * 1024 + (b & 7) * 128;
 #pragma unroll 1
     for (int al = 0; al < 4; ++al) {
+      const bool same = al >= fz && al < fz + geo::BPG;      // a-block in the feature group of b
       uint32_t z[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         if (comp != nullptr) {
-          z[i] = __float_as_uint(comp[(size_t)(COL_Z + 16 * al + i) * 128 + t]);
-        } else {
+          z[i] = __float_as_uint(comp[(size_t)(geo::Z + 16 * al + i) * 128 + t]);
+        } else if (same) {
           float scale;
           const int r = srow(16 * al + i, b, scale);
           z[i] = __float_as_uint(scale * zf[r]);
+        } else {
+          z[i] = 0u;
         }
       }
-      tmem_st16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
-      if (al <= bz) snap_store16(rowz, (sp_koff(pz) >> 4) + 2 * al, (uint32_t)(b & 7), z, al < bz ? 2.f : 1.f);
+      tmem_st16(tmem_addr(tb, q4 * 32, geo::Z + 16 * al), z);
+      if (al >= fz && al <= bz) snap_store16(rowz, (sp_koff(pz) >> 4) + 2 * (al - fz), (uint32_t)(b & 7), z, al < bz ? 2.f : 1.f);
     }
   } else {
     // lanes 64..127 of the Z accumulators: rows of the zero atom, kept at zero
@@ -305,7 +324,7 @@ __device__ __noinline__ void import_state(uint32_t tb, unsigned char* sp, uint32
 #pragma unroll
     for (int i = 0; i < 16; ++i) z[i] = 0u;
 #pragma unroll 1
-    for (int al = 0; al < 4; ++al) tmem_st16(tmem_addr(tb, q4 * 32, COL_Z + 16 * al), z);
+    for (int al = 0; al < 4; ++al) tmem_st16(tmem_addr(tb, q4 * 32, geo::Z + 16 * al), z);
   }
   tmem_wait_st();
   fence_async_smem();
@@ -400,7 +419,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const bool resume = args.s_init != nullptr || comp_in != nullptr;   // accumulators and snapshot 0 start from a given state
   if (resume) {
     if (warp >= WARP_AUX0)
-      import_state(tb, base + OFF_SP, warp & 3, (warp & 3) * 32 + lane, args.s_init, args.z_init, args.layout, bh, v0,
+      import_state<G>(tb, base + OFF_SP, warp & 3, (warp & 3) * 32 + lane, args.s_init, args.z_init, args.layout, bh, v0,
                    comp_in);
     tc_fence_before();
     __syncthreads();
@@ -1015,8 +1034,8 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // ---- the state after the last token, from the accumulators to the public layout or as it is ----
     if (ok) {
       ok = wait_or_abort(bar(BAR_U_DONE), wo ? (nch - 1) & 1 : 0, abort_flag);
-      if (ok && args.s_final != nullptr) export_state(tb, q4, t, args.s_final, args.z_final, args.layout, bh, v0, slice);
-      if (ok && comp_out != nullptr) export_compact(tb, q4, t, comp_out);
+      if (ok && args.s_final != nullptr) export_state<G>(tb, q4, t, args.s_final, args.z_final, args.layout, bh, v0, slice);
+      if (ok && comp_out != nullptr) export_compact<G>(tb, q4, t, comp_out);
     }
 #endif
   }
@@ -1054,11 +1073,7 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-#ifdef KATA_STREAM_EXPORT
-  auto kern = tc_stream_kernel<1>;       // state import / export and groups cover the plain feature
-#else
   auto kern = p.groups == 1 ? tc_stream_kernel<1> : p.groups == 2 ? tc_stream_kernel<2> : tc_stream_kernel<4>;
-#endif
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
     cudaGetLastError();
     ctx.status = KATA_ERR_CUDA;

@@ -91,11 +91,16 @@ def test_invalid_arguments(L, fn):
         assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_init=4096, z_init=8192, feature_order=1)) == SHAPE
         assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_init=4096, z_init=8192)) == WS
         assert call(L, fn, opts=kb.make_opts(kb.KATA_BF16, s_init=4096 + 4, z_init=8192)) == ALIGN
-        # the tensor-core path takes the state without a workspace; the blockwise map goes through the fp32 path
+        # the tensor-core path takes the state without a workspace (unless it is advanced in place: a copy of the
+        # normaliser state); narrower rows with a state go through the fp32 path
         o = kb.make_opts(kb.KATA_BF16, s_init=4096, z_init=8192)
         assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 1, 64, 64, 64, 64, o) == 0
         o = kb.make_opts(kb.KATA_BF16, s_init=4096, z_init=8192, feature_groups=2)
-        assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 1, 64, 64, 64, 64, o) > 0
+        assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 1, 64, 64, 64, 64, o) == 0
+        o = kb.make_opts(kb.KATA_BF16, s_init=4096, z_init=8192, s_pre=4096, z_pre=8192, feature_groups=2)
+        assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 1, 64, 64, 64, 64, o) == 2 * 32 * 32 * 4
+        o = kb.make_opts(kb.KATA_BF16, s_init=4096, z_init=8192)
+        assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 1, 64, 32, 32, 64, o) > 0
     else:
         assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_pre=4096, z_pre=8192)) == INV
         assert call(L, fn, opts=kb.make_opts(kb.KATA_F32, s_init=4096, z_init=8192)) == INV

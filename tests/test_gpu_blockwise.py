@@ -28,8 +28,7 @@ def test_blockwise_forms(form, dtype, dk, dv, g):
     w = inputs.gaussian_workload(f"mg_{dtype}_{dk}_{dv}_{g}", dtype, 2, 2, 333, dk, dv, 64, 300 + dk + g)
     o = FORMS[form](*dev_tensors(w), feature_groups=g)
     torch.cuda.synchronize()
-    # tensor-core kernels for the blockwise map (bf16, d = 64): the quadratic form and the chunked form in one pass
-    # per head, which is also what the scan forms are planned as when the grouping is left to the library
+    # tensor-core kernels for the blockwise map (bf16, d = 64), every form
     tensor = (dtype, dk, dv) == ("bf16", 64, 64)
     assert kb.kata_last_impl() == (kb.KATA_IMPL_TENSOR if tensor else kb.KATA_IMPL_SIMT)
     gpu = to_numpy64(o)
@@ -164,18 +163,56 @@ def test_blockwise_full_size_sampled_rows(g):
         del o, gpu
 
 
-def test_blockwise_explicit_grouping_runs_on_the_fp32_kernels():
+@pytest.mark.parametrize("g", [2, 4])
+@pytest.mark.parametrize("scan_group", [0, 2, 3, 8])
+def test_blockwise_groupings_tensor(g, scan_group):
+    """Scan forms of the blockwise map on the tensor-core kernels: groups of tiles, restart from the scanned prefix."""
     import torch
-    w = inputs.gaussian_workload("mg_grouped", "bf16", 1, 2, 700, 64, 64, 64, 77)
-    o = kb.kata_chunk_state_scan(*dev_tensors(w), feature_groups=2, scan_group=3)
+    w = inputs.gaussian_workload("mg_grouped", "bf16", 1, 2, 1100, 64, 64, 64, 77 + g)
+    for form in ("chunked_scan", "state_scan"):
+        o = FORMS[form](*dev_tensors(w), feature_groups=g, scan_group=scan_group)
+        torch.cuda.synchronize()
+        assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR
+        gpu = to_numpy64(o)
+        for h in range(w.H):
+            ref = ko.kata_quadratic(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h], f"psd_direct:g{g}")[0]
+            check(gpu[0, h], ref, "bf16", f"M{g} {form} scan_group={scan_group} head {h}")
+
+
+@pytest.mark.parametrize("layout", ["psd_direct", "psd_packed"])
+@pytest.mark.parametrize("g", [2, 4])
+def test_blockwise_state_hand_off_tensor(layout, g):
+    """Final state, restart from it (in pieces, in place) and decode steps, bf16 d = 64 on the tensor-core kernel."""
+    import torch
+    B, H, T, d = 1, 2, 420, 64
+    w = inputs.gaussian_workload("mg_state_tc", "bf16", B, H, T, d, d, 64, 460 + g)
+    q, k, v = dev_tensors(w)
+    code = kb.KATA_LAYOUT_PACKED if layout == "psd_packed" else kb.KATA_LAYOUT_DIRECT
+    feat = f"{layout}:g{g}"
+    n = kb.decode_n_psi(d, 2, code, g)
+    S = torch.zeros(B, H, n, d, device="cuda")
+    Z = torch.zeros(B, H, n, device="cuda")
+    outs = []
+    cuts = [0, 130, 257, 400]
+    for i in range(3):
+        a, b = cuts[i], cuts[i + 1]
+        kw = dict(s_pre=S, z_pre=Z, state_layout=code, feature_groups=g)
+        if i > 0:
+            kw.update(s_init=S, z_init=Z)                      # advanced in place
+        outs.append(kb.kata_fwd_chunked(q[:, :, a:b].contiguous(), k[:, :, a:b].contiguous(), v[:, :, a:b].contiguous(), **kw))
+        assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR
+    for t in range(400, T):
+        outs.append(kb.kata_decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(), S, Z,
+                                        state_layout=code, feature_groups=g).unsqueeze(2))
     torch.cuda.synchronize()
-    assert kb.kata_last_impl() == kb.KATA_IMPL_SIMT
-    gpu = to_numpy64(o)
-    for h in range(w.H):
-        ref = ko.kata_quadratic(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h], "psd_direct:g2")[0]
-        check(gpu[0, h], ref, "bf16", f"M2 explicit grouping head {h}")
-    assert kb.kata_scan_plan(kb.KATA_FN_CHUNK_STATE_SCAN, 1, 2, 700, 64, 64, 64,
-                             kb.make_opts(kb.KATA_BF16, feature_groups=2))[0] == 1          # the library's own plan
+    gpu = to_numpy64(torch.cat(outs, dim=2))
+    for h in range(H):
+        ref = ko.kata_quadratic(w.q_ref[0, h], w.k_ref[0, h], w.v_ref[0, h], feat)[0]
+        check(gpu[0, h], ref, "bf16", f"M{g} hand-off/{layout} head {h}")
+        fk = ko.apply_feature(w.k_ref[0, h], feat)
+        Sr, Zr = fk.T @ w.v_ref[0, h], fk.sum(axis=0)
+        assert np.max(np.abs(to_numpy64(S[0, h]) - Sr)) <= 2e-2 * max(1.0, np.abs(Sr).max())
+        assert np.max(np.abs(to_numpy64(Z[0, h]) - Zr)) <= 2e-2 * max(1.0, np.abs(Zr).max())
 
 
 def test_blockwise_argument_checks():
@@ -188,5 +225,5 @@ def test_blockwise_argument_checks():
         kb.kata_fwd_quadratic(q, k, v, feature_groups=2, feature_order=1)
     wb = inputs.gaussian_workload("mg_args_bf16", "bf16", 1, 1, 64, 64, 64, 64, 1)
     with pytest.raises(kb.KataError):
-        kb.kata_fwd_chunked(*dev_tensors(wb), feature_groups=2, inter_chunk=kb.KATA_SCAN, scan_group=4,
-                            impl=kb.KATA_IMPL_TENSOR)          # an explicit grouping of the blockwise map: fp32 kernels
+        wn = inputs.gaussian_workload("mg_args_narrow", "bf16", 1, 1, 64, 32, 32, 64, 1)
+        kb.kata_fwd_chunked(*dev_tensors(wn), feature_groups=2, impl=kb.KATA_IMPL_TENSOR)   # blocks of a narrower row: fp32 kernels

@@ -75,7 +75,7 @@ def test_resume_tensor_in_place_and_simt_agree(in_place):
 
 
 @pytest.mark.parametrize("dtype,dk,dv,g", [("f32", 16, 16, 0), ("f32", 32, 64, 0), ("f32", 64, 32, 0), ("f32", 32, 16, 2),
-                                           ("f32", 64, 16, 4), ("bf16", 32, 32, 0), ("bf16", 64, 64, 2)])
+                                           ("f32", 64, 16, 4), ("bf16", 32, 32, 0), ("bf16", 32, 64, 2)])
 @pytest.mark.parametrize("layout", ["psd_direct", "psd_packed"])
 def test_resume_simt(dtype, dk, dv, g, layout):
     """fp32 kernels (every shape; the blockwise map hands its state over through them)."""
