@@ -103,6 +103,34 @@ size_t bwd_workspace(const Problem& p, const Opts& o, size_t* pad_bytes) {
   return 7 * *pad_bytes + align_up(tc_bwd_workspace_bytes(pp));
 }
 
+// Chunks per group of the scan forms on the SIMT kernels: enough groups for about two CTAs per SM, at least two.
+int simt_scan_group(int BH, int slices, int NC) {
+  int ng = (2 * 148 + slices * BH - 1) / (slices * BH);
+  if (ng < 2) ng = 2;
+  if (ng > NC) ng = NC;
+  return (NC + ng - 1) / ng;
+}
+
+// Chunks per group of the scan forms on the tensor-core kernel.  One CTA per SM and per (head, value slice, group):
+// the first pass runs groups 0 .. ng-2 in its state-only build (about 2.8 us a tile), the last pass runs all ng
+// groups (about 4.4 us a tile), each in whole waves of 148 CTAs; a group state costs four transfers of 115 KB per
+// CTA.  The smallest modelled time over ng = 2 .. 32 decides.
+int tensor_scan_group(int BH, int slices, int NC) {
+  const int cpt = tc_stream_tile() / kChunk;
+  const int tiles = (NC + cpt - 1) / cpt;
+  if (tiles < 2) return NC;
+  const double c = (double)slices * BH;
+  int best = 2;
+  double best_us = 0.0;
+  for (int ng = 2; ng <= 32 && ng <= tiles; ++ng) {
+    const double tpg = (double)((tiles + ng - 1) / ng);
+    const double us = ceil((ng - 1) * c / 148.0) * tpg * 2.8 + ceil(ng * c / 148.0) * tpg * 4.4 + ng * c * 0.115;
+    if (ng == 2 || us < best_us) { best = ng; best_us = us; }
+  }
+  const int G = (tiles + best - 1) / best * cpt;
+  return G < NC ? G : NC;
+}
+
 // How the chunk axis is cut into scan groups, and how many floats one group state takes.
 int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanPlan& plan, size_t& state_elems) {
   plan.n_chunks = (p.T + C - 1) / C;
@@ -160,19 +188,11 @@ int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanP
     } else if (o.scan_group > 0) {
       G = o.scan_group < NC ? o.scan_group : NC;
     } else {
-      // enough groups for about two CTAs per SM, at least two groups
-      int ng = (2 * 148 + slices * BH - 1) / (slices * BH);
-      if (ng < 2) ng = 2;
-      if (ng > NC) ng = NC;
-      G = (NC + ng - 1) / ng;
+      G = tensor ? tensor_scan_group(BH, slices, NC) : simt_scan_group(BH, slices, NC);
     }
   } else if (tensor && o.s_pre == nullptr && o.scan_group == 0) {
     // tensor-core pipeline without the per-chunk export: the grouping of the scan form of kata_fwd_chunked
-    // (a group state is 0.9 MB per head here, so few large groups)
-    int ng = (2 * 148 + slices * BH - 1) / (slices * BH);
-    if (ng < 2) ng = 2;
-    if (ng > NC) ng = NC;
-    G = (NC + ng - 1) / ng;
+    G = tensor_scan_group(BH, slices, NC);
   } else {
     if (o.s_pre != nullptr && o.scan_group > 1) return KATA_ERR_INVALID_ARG;
     if (o.s_pre != nullptr) {

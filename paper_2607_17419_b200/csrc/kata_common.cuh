@@ -109,7 +109,9 @@ struct StreamIO {
   int n_groups;                // 0: the whole sequence is one group
   int launch_groups;           // groups launched (0: n_groups)
 };
-void tc_chunked_stream_export(const Problem& p, int* device_status, const StreamIO& io, LaunchCtx& ctx);
+void tc_chunked_stream_export(const Problem& p, int* device_status, const StreamIO& io, LaunchCtx& ctx);    // public state I/O
+void tc_chunked_stream_restart(const Problem& p, int* device_status, const StreamIO& io, LaunchCtx& ctx);   // groups from init_compact
+void tc_chunked_stream_state(const Problem& p, int* device_status, const StreamIO& io, LaunchCtx& ctx);     // groups to final_compact
 size_t tc_stream_state_elems();
 int tc_stream_slices();
 int tc_stream_tile();

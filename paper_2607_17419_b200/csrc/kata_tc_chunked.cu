@@ -42,7 +42,7 @@ void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws
   io.final_compact = bufA;
   io.write_out = 0;
   io.launch_groups = NG - 1;
-  tc_chunked_stream_export(p, device_status, io, ctx);
+  tc_chunked_stream_state(p, device_status, io, ctx);
   // pass 2
   const float* incl = scan_group_states(bufA, bufB, BH, NG, NG - 1, E, ctx);
   // pass 3
@@ -50,7 +50,7 @@ void tc_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* ws
   io.final_compact = nullptr;
   io.write_out = 1;
   io.launch_groups = NG;
-  tc_chunked_stream_export(p, device_status, io, ctx);
+  tc_chunked_stream_restart(p, device_status, io, ctx);
 }
 
 }  // namespace kata

@@ -17,9 +17,12 @@
 //   intra    P = (Q K^T)^2 masked causally, [O | D] += P [V' | 1/||k||^2]   as in the quadratic form
 //   out      (N_inter + O) / (D_inter + D)             (0 where the denominator is 0)
 // The query norm cancels and is never applied.
-// Compiled a second time with KATA_STREAM_EXPORT (kata_tc_stream_export.cu): the same kernel plus the import of
-// a state before the first token and the export of the state after the last token; kept as a separate build so
-// that the plain kernel's code stays as it is.
+// Compiled three more times with KATA_STREAM_EXPORT and KATA_STREAM_MODE set (kept as separate builds so that the
+// plain kernel's code stays as it is, and each build carries only what it needs):
+//   mode 1 (kata_tc_stream_export.cu)   state before the first token / after the last token in the public layouts
+//   mode 2 (kata_tc_stream_restart.cu)  a group of tiles restarted from a scanned prefix state (pass 3 of the scan forms)
+//   mode 3 (kata_tc_stream_state.cu)    state only: what a group of tiles adds to the state (pass 1); no queries, no
+//                                       reads, no intra tile, and a third key stage in the space they leave
 //
 // Warps (768 threads, 80 registers each): 0 TMA producer and update-MMA issuer (b-block 3, Z); 1 update-MMA
 // issuer (b-blocks 0-2); 2 read-MMA issuer; 3 intra-tile MMA issuer; 4-11 W builders in two teams (even / odd
@@ -69,7 +72,7 @@ constexpr uint32_t SP_BYTES = 5 * SP_BLOCK;
 constexpr uint32_t OFF_R2 = 217088;       // 2 stages x 128 x (bf16 1/||k||^2 twice)
 constexpr uint32_t OFF_PART = 218112;     // 9 x 128 fp32: partial sums of the second reader team
 constexpr uint32_t OFF_BAR = 222720;
-constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 320;     // BAR_COUNT barriers and three more of the state-only build
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
 static_assert(OFF_W + NWBUF * W_BYTES == OFF_ZERO && OFF_ZERO + 2048 == OFF_SP, "layout");
 
@@ -339,9 +342,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   auto bar = [&](int i) { return reinterpret_cast<uint64_t*>(base + OFF_BAR) + i; };
   unsigned char* const qtile = base + OFF_Q;
   auto ktile = [&](int s) { return base + OFF_K + s * 16384; };
-  auto vptile = [&](int s) { return base + OFF_VP + s * 4096; };
   auto wbuf = [&](int b) { return base + OFF_W + b * W_BYTES; };
-  auto r2pair = [&](int s) { return reinterpret_cast<uint32_t*>(base + OFF_R2) + s * CT; };
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
   volatile int* abort_flag = &abort_s;
@@ -357,16 +358,43 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int t0 = grp * args.tiles_per_group;
   const int nch = min((args.Tlen + CT - 1) / CT, t0 + args.tiles_per_group) - t0;
   if (nch <= 0) return;
-  const bool wo = args.write_out != 0;
+  constexpr bool wo = KATA_STREAM_MODE != 3;
+#if KATA_STREAM_MODE != 1
   const size_t comp_elems = (size_t)224 * 128;
+#endif
+#if KATA_STREAM_MODE == 2
   const float* comp_in = (args.init_compact != nullptr && grp > 0)
       ? args.init_compact + ((((size_t)bh * args.n_groups + (grp - 1)) * NSLICE + slice) * comp_elems) : nullptr;
-  float* comp_out = args.final_compact != nullptr
-      ? args.final_compact + ((((size_t)bh * args.n_groups + grp) * NSLICE + slice) * comp_elems) : nullptr;
+#endif
+#if KATA_STREAM_MODE == 3
+  float* comp_out = args.final_compact + ((((size_t)bh * args.n_groups + grp) * NSLICE + slice) * comp_elems);
+#endif
 #else
   constexpr int t0 = 0;
   constexpr bool wo = true;
   const int nch = (args.Tlen + CT - 1) / CT;
+#endif
+#if defined(KATA_STREAM_EXPORT) && KATA_STREAM_MODE == 3
+  // The state-only build has the query and snapshot areas to spare: a third key stage (tile, scales, barriers), so
+  // that a key tile is requested two tiles ahead (with two stages the chain stage free -> TMA -> key scales ->
+  // first W step is as long as the tile itself).
+  constexpr int NKS = 3;
+  auto kst = [&](int j) { return j % 3; };
+  auto kph = [&](int j) { return (uint32_t)((j / 3) & 1); };
+  auto kfull = [&](int s) { return s < 2 ? bar(BAR_K_FULL + s) : bar(BAR_COUNT); };
+  auto kempty = [&](int s) { return s < 2 ? bar(BAR_K_EMPTY + s) : bar(BAR_COUNT + 1); };
+  auto kprep = [&](int s) { return s < 2 ? bar(BAR_PREP + s) : bar(BAR_COUNT + 2); };
+  auto vptile = [&](int s) { return s < 2 ? base + OFF_VP + s * 4096 : base + OFF_SP; };
+  auto r2pair = [&](int s) { return s < 2 ? reinterpret_cast<uint32_t*>(base + OFF_R2) + s * CT : reinterpret_cast<uint32_t*>(base + OFF_SP + 4096); };
+#else
+  constexpr int NKS = 2;
+  auto kst = [&](int j) { return j & 1; };
+  auto kph = [&](int j) { return (uint32_t)((j >> 1) & 1); };
+  auto kfull = [&](int s) { return bar(BAR_K_FULL + s); };
+  auto kempty = [&](int s) { return bar(BAR_K_EMPTY + s); };
+  auto kprep = [&](int s) { return bar(BAR_PREP + s); };
+  auto vptile = [&](int s) { return base + OFF_VP + s * 4096; };
+  auto r2pair = [&](int s) { return reinterpret_cast<uint32_t*>(base + OFF_R2) + s * CT; };
 #endif
 
   if (tid == 0) {
@@ -377,6 +405,11 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       mbar_init(bar(BAR_PREP + s), 128);
       mbar_init(bar(BAR_Y_FULL + s), 1);
       mbar_init(bar(BAR_Y_EMPTY + s), 128);
+    }
+    if (NKS == 3) {
+      mbar_init(kfull(2), 1);
+      mbar_init(kempty(2), 2);
+      mbar_init(kprep(2), 128);
     }
     for (int s = 0; s < NWBUF; ++s) {
       mbar_init(bar(BAR_W_FULL + s), 128);
@@ -415,8 +448,14 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
   bool ok = true;
-#ifdef KATA_STREAM_EXPORT
-  const bool resume = args.s_init != nullptr || comp_in != nullptr;   // accumulators and snapshot 0 start from a given state
+#if defined(KATA_STREAM_EXPORT) && KATA_STREAM_MODE != 3
+  // accumulators and snapshot 0 start from a given state: the public one (mode 1) or a scanned prefix (mode 2)
+#if KATA_STREAM_MODE == 1
+  const bool resume = args.s_init != nullptr;
+  const float* comp_in = nullptr;
+#else
+  const bool resume = comp_in != nullptr;
+#endif
   if (resume) {
     if (warp >= WARP_AUX0)
       import_state<G>(tb, base + OFF_SP, warp & 3, (warp & 3) * 32 + lane, args.s_init, args.z_init, args.layout, bh, v0,
@@ -440,10 +479,10 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const uint64_t dB = smem_desc(0, 16384, 1024, kSwizzle128B);
       const bool producer = (warp == WARP_UB);
       auto load_k = [&](int j) -> bool {
-        const int s = j & 1;
-        if (!wait_or_abort(bar(BAR_K_EMPTY + s), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
-        mbar_arrive_expect_tx(bar(BAR_K_FULL + s), 16384);
-        tma_load_3d(ktile(s), &tmK, bar(BAR_K_FULL + s), 0, (t0 + j) * CT, bh);
+        const int s = kst(j);
+        if (!wait_or_abort(kempty(s), kph(j) ^ 1, abort_flag)) return false;
+        mbar_arrive_expect_tx(kfull(s), 16384);
+        tma_load_3d(ktile(s), &tmK, kfull(s), 0, (t0 + j) * CT, bh);
         return true;
       };
       auto load_q = [&](int j) -> bool {     // one staging buffer: free once the previous tile was copied to TMEM
@@ -455,14 +494,16 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (producer) {
         ok = load_k(0) && (!wo || load_q(0));
         if (ok && nch > 1) ok = load_k(1);
+        if (ok && NKS == 3 && nch > 2) ok = load_k(2);
       }
       uint32_t wbi = 0, wph = 0;             // W buffer of the step and the parity of its phase
       for (int j = 0; j < nch && ok; ++j) {
-        const int s = j & 1;
-        ok = wait_or_abort(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag);
+        const int s = kst(j);
+        ok = wait_or_abort(kfull(s), kph(j), abort_flag);
         if (ok && wo && j > 0) ok = wait_or_abort(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
-        // the key stage of tile j - 1 is free once that tile's consumers are through: refill it with tile j + 1
-        if (ok && producer && j > 0 && j + 1 < nch) ok = load_k(j + 1);
+        // the key stage of tile j - 1 is free once that tile's consumers are through: refill it (with tile j + 1;
+        // with tile j + 2 where there are three stages)
+        if (ok && producer && j > 0 && j + NKS - 1 < nch) ok = load_k(j + NKS - 1);
 #pragma unroll 1
         for (int sc = 0; sc < 8 && ok; ++sc) {
           ok = wait_or_abort(bar(BAR_W_FULL + wbi), wph, abort_flag);
@@ -492,7 +533,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         // state-only pass: nobody looks at the state between the tiles, one commit after the last update (a parity
         // wait cannot tell phases two apart)
         if (wo || j + 1 == nch) mma_commit(bar(BAR_U_DONE));
-        mma_commit(bar(BAR_K_EMPTY + s));
+        mma_commit(kempty(s));
         // the query staging buffer is free once tile j was copied to TMEM (at the end of tile j - 1)
         if (producer && wo && j + 1 < nch) ok = load_q(j + 1);
       }
@@ -696,9 +737,8 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       return true;
     };
     for (int j = 0; j < nch && ok; ++j) {
-      const int s = j & 1;
-      ok = wait_or_abort(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag) &&
-           wait_or_abort(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
+      const int s = kst(j);
+      ok = wait_or_abort(kfull(s), kph(j), abort_flag) && wait_or_abort(kprep(s), kph(j), abort_flag);
       // team 1 copies its share of the state after tile j - 1 before its first step of tile j, team 0 after
       // its first step: either way right when the update of tile j - 1 completes
       if (ok && wo && team == 1 && j > 0) ok = snapshot_share(j - 1);
@@ -854,8 +894,8 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     };
     // key scales and v' of tile j (the value slice was fetched one tile earlier)
     auto prep = [&](int j, const uint4& vraw) -> bool {
-      const int s = j & 1;
-      if (!wait_or_abort(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag)) return false;
+      const int s = kst(j);
+      if (!wait_or_abort(kfull(s), kph(j), abort_flag)) return false;
       float ss = 0.f;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
@@ -878,7 +918,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       *reinterpret_cast<uint4*>(vptile(s) + 2048 + t * 16) = make_uint4(rb & 0xFFFFu, 0u, 0u, 0u);
       r2pair(s)[t] = rb;
       fence_async_smem();
-      mbar_arrive(bar(BAR_PREP + s));
+      mbar_arrive(kprep(s));
       return true;
     };
     // this warp's share of the snapshot of the state after tile j (b-block 3; the other blocks and Z: warps 4-11);
@@ -1030,12 +1070,17 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         mbar_arrive(bar(BAR_QT_FULL));
       }
     }
-#ifdef KATA_STREAM_EXPORT
-    // ---- the state after the last token, from the accumulators to the public layout or as it is ----
+#if defined(KATA_STREAM_EXPORT) && KATA_STREAM_MODE == 1
+    // ---- the state after the last token, from the accumulators to the public layout ----
+    if (ok && args.s_final != nullptr) {
+      ok = wait_or_abort(bar(BAR_U_DONE), (nch - 1) & 1, abort_flag);
+      if (ok) export_state<G>(tb, q4, t, args.s_final, args.z_final, args.layout, bh, v0, slice);
+    }
+#elif defined(KATA_STREAM_EXPORT) && KATA_STREAM_MODE == 3
+    // ---- what the group adds to the state: the accumulators as they are (the one commit of this build's updates) ----
     if (ok) {
-      ok = wait_or_abort(bar(BAR_U_DONE), wo ? (nch - 1) & 1 : 0, abort_flag);
-      if (ok && args.s_final != nullptr) export_state<G>(tb, q4, t, args.s_final, args.z_final, args.layout, bh, v0, slice);
-      if (ok && comp_out != nullptr) export_compact<G>(tb, q4, t, comp_out);
+      ok = wait_or_abort(bar(BAR_U_DONE), 0, abort_flag);
+      if (ok) export_compact<G>(tb, q4, t, comp_out);
     }
 #endif
   }
@@ -1058,12 +1103,16 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 }  // namespace
 
-#ifdef KATA_STREAM_EXPORT
+#if defined(KATA_STREAM_EXPORT) && KATA_STREAM_MODE == 1
 size_t tc_stream_state_elems() { return (size_t)NSLICE * 224 * 128; }
 int tc_stream_slices() { return NSLICE; }
 int tc_stream_tile() { return CT; }
 
 void tc_chunked_stream_export(const Problem& p, int* device_status, const StreamIO& io, LaunchCtx& ctx) {
+#elif defined(KATA_STREAM_EXPORT) && KATA_STREAM_MODE == 2
+void tc_chunked_stream_restart(const Problem& p, int* device_status, const StreamIO& io, LaunchCtx& ctx) {
+#elif defined(KATA_STREAM_EXPORT) && KATA_STREAM_MODE == 3
+void tc_chunked_stream_state(const Problem& p, int* device_status, const StreamIO& io, LaunchCtx& ctx) {
 #else
 void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
 #endif
