@@ -454,6 +454,14 @@ def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
                      ("chunk_state_scan", lambda: kb.kata_chunk_state_scan(q, k, v, out))):
         ms = timed(fn)
         res[name] = dict(ms=ms, tokens_per_s=T / (ms * 1e-3), launches=kb.kata_last_launch_count())
+    # one batch element, four of the sixteen heads of the same workload: 32 CTAs on the sequential walk, where
+    # the scan form (and inter_chunk = AUTO, which picks it here) fills the GPU with groups of tiles
+    q4, k4, v4, o4 = (a[:, :4] for a in (q, k, v, out))
+    q4, k4, v4, o4 = q4.contiguous(), k4.contiguous(), v4.contiguous(), o4.contiguous()
+    for name, mode in (("seq", kb.KATA_SEQUENTIAL), ("scan", kb.KATA_SCAN), ("auto", kb.KATA_INTER_AUTO)):
+        ms = timed(lambda: kb.kata_fwd_chunked(q4, k4, v4, o4, inter_chunk=mode))
+        res[f"chunked_{name}_H4"] = dict(ms=ms, tokens_per_s=T / (ms * 1e-3), launches=kb.kata_last_launch_count())
+    del q4, k4, v4, o4
     w2 = inputs.config(2)
     q2, k2, v2 = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).to(dev) for a in (w2.q_dev, w2.k_dev, w2.v_dev))
     o2 = torch.empty_like(v2)

@@ -60,7 +60,7 @@ typedef enum kata_status {
 
 enum { KATA_F32 = 0, KATA_BF16 = 1 };                 /* kata_opts.dtype          */
 enum { KATA_LAYOUT_DIRECT = 0, KATA_LAYOUT_PACKED = 1 }; /* kata_opts.state_layout */
-enum { KATA_SEQUENTIAL = 0, KATA_SCAN = 1 };          /* kata_opts.inter_chunk    */
+enum { KATA_SEQUENTIAL = 0, KATA_SCAN = 1, KATA_INTER_AUTO = 2 };   /* kata_opts.inter_chunk */
 enum { KATA_IMPL_AUTO = 0, KATA_IMPL_SIMT = 1, KATA_IMPL_TENSOR = 2 }; /* kata_opts.impl */
 enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2, KATA_FN_DECODE_STEP = 3,
        KATA_FN_BWD_QUADRATIC = 4 };
@@ -87,7 +87,13 @@ enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2,
  *  inter_chunk    kata_fwd_chunked only: SEQUENTIAL walks the chunks of a head in order
  *                 (Algorithm 1); SCAN splits the chunk axis into groups, reduces each group,
  *                 runs a log-depth exclusive scan over the group states and finishes every
- *                 group in parallel (section "Tree-scan inter-chunk reduction").
+ *                 group in parallel (section "Tree-scan inter-chunk reduction").  INTER_AUTO lets the
+ *                 library choose: SCAN where the heads alone leave most of the GPU idle and the
+ *                 sequence is long enough for the scan form's extra pass to pay (a model of the
+ *                 tensor-core kernel's time in whole waves of CTAs decides); SEQUENTIAL otherwise,
+ *                 on the fp32 kernels, for feature_order 1 (whose tensor-core path makes this choice
+ *                 by itself) and whenever a state is handed in or out.  Both forms give the same
+ *                 result up to the rounding order of the state sums.
  *  impl           AUTO picks the tensor-core kernels where they exist; SIMT / TENSOR force one
  *                 (TENSOR returns KATA_ERR_UNSUPPORTED_SHAPE where it does not exist).
  *  scan_group     chunks per scan group; 0 = library's choice (kata_chunk_state_scan: 1, i.e.

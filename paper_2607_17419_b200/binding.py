@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(HERE, "libkata.so")
 
 KATA_F32, KATA_BF16 = 0, 1
 KATA_LAYOUT_DIRECT, KATA_LAYOUT_PACKED = 0, 1
-KATA_SEQUENTIAL, KATA_SCAN = 0, 1
+KATA_SEQUENTIAL, KATA_SCAN, KATA_INTER_AUTO = 0, 1, 2
 KATA_IMPL_AUTO, KATA_IMPL_SIMT, KATA_IMPL_TENSOR = 0, 1, 2
 KATA_FN_QUADRATIC, KATA_FN_CHUNKED, KATA_FN_CHUNK_STATE_SCAN, KATA_FN_DECODE_STEP = 0, 1, 2, 3
 KATA_FN_BWD_QUADRATIC = 4
@@ -216,7 +216,7 @@ def kata_fwd_quadratic(q, k, v, out=None, C: int = 64, **kw):
 
 
 def kata_fwd_chunked(q, k, v, out=None, C: int = 64, **kw):
-    """Chunked-state forward; inter_chunk=KATA_SEQUENTIAL (default) or KATA_SCAN.  In the sequential form
+    """Chunked-state forward; inter_chunk=KATA_SEQUENTIAL (default), KATA_SCAN or KATA_INTER_AUTO.  In the sequential form
     s_init/z_init give the state before the first token and s_pre/z_pre receive the state after the last."""
     return _call(KATA_FN_CHUNKED, q, k, v, out, C, **kw)
 

@@ -55,7 +55,7 @@ int read_opts(const kata_opts* o, Opts& out) {
   if (out.dtype != KATA_F32 && out.dtype != KATA_BF16) return KATA_ERR_INVALID_ARG;
   if (out.feature_order != 1 && out.feature_order != 2) return KATA_ERR_INVALID_ARG;
   if (out.state_layout != KATA_LAYOUT_DIRECT && out.state_layout != KATA_LAYOUT_PACKED) return KATA_ERR_INVALID_ARG;
-  if (out.inter_chunk != KATA_SEQUENTIAL && out.inter_chunk != KATA_SCAN) return KATA_ERR_INVALID_ARG;
+  if (out.inter_chunk < KATA_SEQUENTIAL || out.inter_chunk > KATA_INTER_AUTO) return KATA_ERR_INVALID_ARG;
   if (out.impl < KATA_IMPL_AUTO || out.impl > KATA_IMPL_TENSOR) return KATA_ERR_INVALID_ARG;
   if (out.scan_group < 0) return KATA_ERR_INVALID_ARG;
   if (out.groups != 1 && out.groups != 2 && out.groups != 4) return KATA_ERR_INVALID_ARG;
@@ -115,9 +115,10 @@ int simt_scan_group(int BH, int slices, int NC) {
 // the first pass runs groups 0 .. ng-2 in its state-only build (about 2.8 us a tile), the last pass runs all ng
 // groups (about 4.4 us a tile), each in whole waves of 148 CTAs; a group state costs four transfers of 115 KB per
 // CTA.  The smallest modelled time over ng = 2 .. 32 decides.
-int tensor_scan_group(int BH, int slices, int NC) {
+int tensor_scan_group(int BH, int slices, int NC, double* model_us = nullptr) {
   const int cpt = tc_stream_tile() / kChunk;
   const int tiles = (NC + cpt - 1) / cpt;
+  if (model_us) *model_us = 1e30;
   if (tiles < 2) return NC;
   const double c = (double)slices * BH;
   int best = 2;
@@ -127,8 +128,21 @@ int tensor_scan_group(int BH, int slices, int NC) {
     const double us = ceil((ng - 1) * c / 148.0) * tpg * 2.8 + ceil(ng * c / 148.0) * tpg * 4.4 + ng * c * 0.115;
     if (ng == 2 || us < best_us) { best = ng; best_us = us; }
   }
+  if (model_us) *model_us = best_us + 20.0;   // two more launches
   const int G = (tiles + best - 1) / best * cpt;
   return G < NC ? G : NC;
+}
+
+// inter_chunk = AUTO on the tensor-core kernel: the scan form where its modelled time is below nine tenths of the
+// sequential walk's (whole waves of one CTA per head and value slice, 4.4 us a tile).
+bool tensor_scan_pays(int BH, int NC) {
+  const int cpt = tc_stream_tile() / kChunk;
+  const int tiles = (NC + cpt - 1) / cpt;
+  const int slices = tc_chunked_slices();
+  double scan_us;
+  tensor_scan_group(BH, slices, NC, &scan_us);
+  const double seq_us = ceil((double)slices * BH / 148.0) * tiles * 4.4;
+  return scan_us < 0.9 * seq_us;
 }
 
 // How the chunk axis is cut into scan groups, and how many floats one group state takes.
@@ -310,6 +324,10 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   st = check_shape(fn, B, H, T, d_k, d_v, C);
   if (st != KATA_OK) return st;
   if (need_ptrs && (q == nullptr || k == nullptr || v == nullptr || out == nullptr)) return KATA_ERR_INVALID_ARG;
+  // inter_chunk = AUTO stays open only where both forms exist and no state is handed over; decided below
+  if (r.o.inter_chunk == KATA_INTER_AUTO &&
+      (fn != KATA_FN_CHUNKED || r.o.s_pre != nullptr || r.o.s_init != nullptr || r.o.feature_order != 2))
+    r.o.inter_chunk = KATA_SEQUENTIAL;
   // s_pre/z_pre: prefix chunk states of the scan pipeline, or the final state of the sequential chunked forward
   if (r.o.s_pre != nullptr && !(fn == KATA_FN_CHUNK_STATE_SCAN ||
                                 (fn == KATA_FN_CHUNKED && r.o.inter_chunk == KATA_SEQUENTIAL))) return KATA_ERR_INVALID_ARG;
@@ -329,6 +347,13 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
     if (r.pad) r.pad_bytes = align_up((size_t)B * H * T * 64 * 2);
   }
   const Problem kp = kernel_problem(r);
+  if (r.o.inter_chunk == KATA_INTER_AUTO) {
+    Opts scan = r.o;
+    scan.inter_chunk = KATA_SCAN;
+    r.o.inter_chunk = KATA_SEQUENTIAL;
+    if (C == kChunk && want_tensor(fn, kp, r.o) && want_tensor(fn, kp, scan) && tensor_scan_pays(B * H, (T + C - 1) / C))
+      r.o.inter_chunk = KATA_SCAN;
+  }
   r.tensor = want_tensor(fn, kp, r.o);
   if (r.o.impl == KATA_IMPL_TENSOR && !r.tensor) return KATA_ERR_UNSUPPORTED_SHAPE;
   r.C = fn == KATA_FN_QUADRATIC ? kChunk : C;

@@ -130,6 +130,32 @@ def test_scan_workspace_and_plan(L):
     assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 1, 1, 64, 48, 64, 64, o) == 0      # invalid -> 0
 
 
+def test_inter_chunk_auto_and_tensor_groups(L):
+    """inter_chunk = AUTO: the scan form only where few heads leave the GPU idle on a long sequence, never with a
+    state hand-off, never on the fp32 kernels; the tensor-core scan form's own grouping fills whole waves."""
+    auto = kb.make_opts(kb.KATA_BF16, inter_chunk=kb.KATA_INTER_AUTO)
+    plan = lambda B, H, T, o: kb.kata_scan_plan(kb.KATA_FN_CHUNKED, B, H, T, 64, 64, 64, o)
+    assert plan(8, 16, 4096, auto)[0] == 1                    # 1024 CTAs: sequential
+    assert plan(1, 16, 131072, auto)[0] == 1                  # 128 CTAs already fill 148 SMs
+    ng, g, rounds = plan(1, 1, 131072, auto)                  # 8 CTAs per group: 18 groups make one wave of 144
+    assert (ng, g) == (18, 114) and rounds == 5
+    assert plan(1, 4, 131072, auto)[0] > 1
+    assert plan(1, 1, 256, auto)[0] == 1                      # two tiles: nothing to gain
+    auto32 = kb.make_opts(kb.KATA_F32, inter_chunk=kb.KATA_INTER_AUTO)
+    assert plan(1, 1, 131072, auto32)[0] == 1
+    hand = kb.make_opts(kb.KATA_BF16, inter_chunk=kb.KATA_INTER_AUTO, s_pre=4096, z_pre=8192)
+    assert plan(1, 1, 131072, hand)[0] == 1
+    bad = kb.make_opts(kb.KATA_BF16, inter_chunk=3)
+    with pytest.raises(kb.KataError):
+        plan(1, 1, 1024, bad)
+    # explicit scan form on the tensor cores: groups of whole 128-token tiles, the last pass in whole waves
+    scan = kb.make_opts(kb.KATA_BF16, inter_chunk=kb.KATA_SCAN)
+    ng, g, _ = plan(1, 16, 131072, scan)
+    assert (ng, g) == (2, 1024)
+    ng, g, _ = plan(1, 4, 131072, scan)
+    assert g % 2 == 0 and (ng - 1) * g < 2048 <= ng * g
+
+
 def test_no_oracle_in_product_path():
     """The package must not import or reference the oracle."""
     pkg = os.path.join(ROOT, "paper_2607_17419_b200")

@@ -95,6 +95,27 @@ def test_scan_group_sizes_agree():
             check(g[b, h], r, "bf16", f"scan_group={sg}")
 
 
+def test_inter_chunk_auto_takes_the_scan_form_for_one_long_head():
+    """One head of 6000 tokens: AUTO runs the grouped passes and equals the oracle; sixteen such
+    heads fill the GPU and stay on the single sequential pass."""
+    import torch
+    w = inputs.gaussian_workload("auto_scan", "bf16", 1, 1, 6000, 64, 64, 64, 21)
+    q, k, v = dev_tensors(w)
+    o = kb.kata_fwd_chunked(q, k, v, inter_chunk=kb.KATA_INTER_AUTO)
+    torch.cuda.synchronize()
+    # 16 groups of 3 tiles: the state-only pass, four scan rounds, the restarted pass
+    assert kb.kata_last_launch_count() == 6 and kb.kata_last_impl() == 2
+    for (b, h), r in oracle_full(w).items():
+        check(to_numpy64(o)[b, h], r, "bf16", "auto -> scan")
+    w = inputs.gaussian_workload("auto_seq", "bf16", 1, 16, 1000, 64, 64, 64, 22)
+    q, k, v = dev_tensors(w)
+    o = kb.kata_fwd_chunked(q, k, v, inter_chunk=kb.KATA_INTER_AUTO)
+    torch.cuda.synchronize()
+    assert kb.kata_last_launch_count() == 1
+    for (b, h), r in oracle_full(w, heads=[(0, 3)]).items():
+        check(to_numpy64(o)[b, h], r, "bf16", "auto -> sequential")
+
+
 def test_degenerate_rows():
     """Zero keys/queries and D = 0 rows give 0, never NaN (reading: readout defined only for D > 0)."""
     import torch
