@@ -430,6 +430,32 @@ def run_bwd(args):
                           impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")))
 
 
+def run_scan(args):
+    """Profiler case of the scan form of the chunked forward: config 4 at T = 32768 (B=1, H=16, d=64, bf16), two
+    groups of 128 tiles: a state-only pass over the first group, then both groups restarted; short line."""
+    import numpy as np
+    import torch
+    from paper_2607_17419_b200 import binding as kb, build as kbuild, inputs
+    kbuild.build()
+    torch.cuda.set_device(0)
+    w = inputs.config(4, 32768)
+    q, k, v = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda() for a in (w.q_dev, w.k_dev, w.v_dev))
+    out = torch.empty_like(v)
+    for _ in range(args.warmup):
+        kb.kata_fwd_chunked(q, k, v, out, inter_chunk=kb.KATA_SCAN)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        kb.kata_fwd_chunked(q, k, v, out, inter_chunk=kb.KATA_SCAN)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    print(json.dumps(dict(case="scan", ms_per_step=ms, tokens_per_s=w.B * w.T / (ms * 1e-3),
+                          launches=kb.kata_last_launch_count(),
+                          impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")))
+
+
 def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
     """Separately timed secondary figures: scan forms on the same workload, quadratic form on config 2."""
     import numpy as np
@@ -530,7 +556,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="sequential", choices=["sequential", "scan"])
     ap.add_argument("--no-extra", dest="extra", action="store_false")
-    ap.add_argument("--case", default="full", choices=["full", "small", "decode", "order1", "bwd", "quadratic"],
+    ap.add_argument("--case", default="full", choices=["full", "small", "decode", "order1", "bwd", "quadratic", "scan"],
                     help="small: the same kernel on T=32768 only; decode: the decode step only; order1: the "
                          "first-order tensor-core kernel on B=16, T=8192 (all for profiler captures; they print a "
                          "short line)")
@@ -545,6 +571,8 @@ def main():
         run_bwd(args)
     elif args.case == "quadratic":
         run_quadratic(args)
+    elif args.case == "scan":
+        run_scan(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
