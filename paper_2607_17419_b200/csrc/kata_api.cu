@@ -2,6 +2,7 @@
 // dispatch to the SIMT (fp32) or tensor-core (tcgen05) kernels.  Declarations and the contract of
 // every entry point are in include/kata.h.
 #include <cstring>
+#include <mutex>
 
 #include <cmath>
 
@@ -457,6 +458,138 @@ int entry(int fn, const void* q, const void* k, const void* v, void* out, int B,
   return run_device(fn, r, r.o.workspace);
 }
 
+// ---- host buffers, long sequences: copies and kernels overlapped piece by piece ----
+// The sequential chunked forward can be fed in pieces of the token axis (the state after a piece is the state before
+// the next).  The host-buffer entry uses that on the tensor-core path: while piece i is computed, piece i + 1 is on
+// its way to the device and the output of piece i - 1 on its way back, on two internal streams.  The pieces are
+// tensors of their own on the device ([B,H,T_piece,d], two sets of buffers); the host tensors are read and written
+// with pitched copies.
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, in_done[2] = {nullptr, nullptr}, comp_done[2] = {nullptr, nullptr},
+              out_done[2] = {nullptr, nullptr};
+};
+std::mutex g_pipe_mutex;
+HostPipe g_pipe[64];                        // one per device ordinal, created on first use, kept for the process
+
+bool host_pipe_get(HostPipe*& hp) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  HostPipe& h = g_pipe[dev];
+  if (!h.ready) {
+    bool ok = cudaStreamCreateWithFlags(&h.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&h.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&h.start, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+      ok = cudaEventCreateWithFlags(&h.in_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&h.comp_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&h.out_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      return false;
+    }
+    h.ready = true;
+  }
+  hp = &h;
+  return true;
+}
+
+struct PipePlan {
+  int pieces, piece_T;
+  size_t tensor_bytes;       // one piece of q, k, v or out on the device
+  size_t s_bytes, z_bytes;   // the state handed from piece to piece (fp32, DIRECT layout)
+  size_t inner_bytes;        // scratch of one piece's call
+  size_t total;
+};
+
+// Pieces of at least 8192 tokens, at most eight of them, whole 128-token tiles; bf16 d_k = d_v = 64 tensor-core path of
+// the sequential form with no state asked for or given by the caller.
+bool host_pipe_plan(int fn, const Prepared& r, const kata_opts* opts, int C, PipePlan& pp) {
+  const Problem& p = r.p;
+  if (fn != KATA_FN_CHUNKED || !r.tensor || r.pad || r.o.inter_chunk != KATA_SEQUENTIAL || p.feature_order != 2) return false;
+  if (r.o.s_pre != nullptr || r.o.s_init != nullptr || p.dtype != KATA_BF16 || p.d_k != 64 || p.d_v != 64) return false;
+  if (p.T < 4 * 8192) return false;
+  pp.pieces = p.T / 8192 < 8 ? p.T / 8192 : 8;
+  pp.piece_T = ((p.T + pp.pieces - 1) / pp.pieces + 127) / 128 * 128;
+  pp.pieces = (p.T + pp.piece_T - 1) / pp.piece_T;
+  pp.tensor_bytes = align_up((size_t)p.B * p.H * pp.piece_T * 64 * 2);
+  const size_t n_psi = (size_t)decode_n_psi(p.d_k, KATA_LAYOUT_DIRECT, 2, p.groups);
+  pp.s_bytes = align_up((size_t)p.B * p.H * n_psi * p.d_v * sizeof(float));
+  pp.z_bytes = align_up((size_t)p.B * p.H * n_psi * sizeof(float));
+  kata_opts po = *opts;
+  po.state_layout = KATA_LAYOUT_DIRECT;
+  po.s_init = po.s_pre = reinterpret_cast<float*>(kAlign);       // any non-null, aligned value: sizes only
+  po.z_init = po.z_pre = reinterpret_cast<float*>(kAlign);
+  pp.inner_bytes = align_up(kata_workspace_bytes(KATA_FN_CHUNKED, p.B, p.H, pp.piece_T, p.d_k, p.d_v, C, &po));
+  pp.total = 8 * pp.tensor_bytes + pp.s_bytes + pp.z_bytes + pp.inner_bytes;
+  return pp.total <= r.o.workspace_bytes;
+}
+
+int host_pipelined(const Prepared& r, const PipePlan& pp, const void* q_host, const void* k_host, const void* v_host,
+                   void* out_host, int C, const kata_opts* opts) {
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  HostPipe* hp = nullptr;
+  if (!host_pipe_get(hp)) return KATA_ERR_CUDA;
+  const Problem& p = r.p;
+  cudaStream_t main = r.o.stream;
+  char* ws = static_cast<char*>(r.o.workspace);
+  auto in_buf = [&](int b, int which) { return ws + (size_t)(b * 3 + which) * pp.tensor_bytes; };
+  auto out_buf = [&](int b) { return ws + (size_t)(6 + b) * pp.tensor_bytes; };
+  float* S = reinterpret_cast<float*>(ws + 8 * pp.tensor_bytes);
+  float* Z = reinterpret_cast<float*>(ws + 8 * pp.tensor_bytes + pp.s_bytes);
+  char* inner = ws + 8 * pp.tensor_bytes + pp.s_bytes + pp.z_bytes;
+  const size_t row = 64 * 2, host_pitch = (size_t)p.T * row;
+  const int heads = p.B * p.H;
+  bool ok = cudaEventRecord(hp->start, main) == cudaSuccess &&
+            cudaStreamWaitEvent(hp->in, hp->start, 0) == cudaSuccess &&
+            cudaStreamWaitEvent(hp->out, hp->start, 0) == cudaSuccess;
+  int launches = 0;
+  for (int i = 0; i < pp.pieces && ok; ++i) {
+    const int b = i & 1;
+    const int t0 = i * pp.piece_T;
+    const int len = p.T - t0 < pp.piece_T ? p.T - t0 : pp.piece_T;
+    const size_t width = (size_t)len * row;
+    // inputs of piece i: their buffers were last read by the kernels of piece i - 2
+    if (i >= 2) ok = cudaStreamWaitEvent(hp->in, hp->comp_done[b], 0) == cudaSuccess;
+    const void* src[3] = {q_host, k_host, v_host};
+    for (int w = 0; w < 3 && ok; ++w)
+      ok = cudaMemcpy2DAsync(in_buf(b, w), width, static_cast<const char*>(src[w]) + (size_t)t0 * row, host_pitch, width,
+                             heads, cudaMemcpyHostToDevice, hp->in) == cudaSuccess;
+    ok = ok && cudaEventRecord(hp->in_done[b], hp->in) == cudaSuccess &&
+         cudaStreamWaitEvent(main, hp->in_done[b], 0) == cudaSuccess;
+    // the output buffer of piece i was last drained by the copy of piece i - 2
+    if (ok && i >= 2) ok = cudaStreamWaitEvent(main, hp->out_done[b], 0) == cudaSuccess;
+    if (!ok) break;
+    kata_opts po = *opts;
+    po.state_layout = KATA_LAYOUT_DIRECT;
+    po.workspace = inner;
+    po.workspace_bytes = pp.inner_bytes;
+    po.s_init = i > 0 ? S : nullptr;
+    po.z_init = i > 0 ? Z : nullptr;
+    po.s_pre = i + 1 < pp.pieces ? S : nullptr;
+    po.z_pre = i + 1 < pp.pieces ? Z : nullptr;
+    const int st = entry(KATA_FN_CHUNKED, in_buf(b, 0), in_buf(b, 1), in_buf(b, 2), out_buf(b), p.B, p.H, len, p.d_k,
+                         p.d_v, C, &po);
+    if (st != KATA_OK) return st;
+    launches += g_last_launches;
+    ok = cudaEventRecord(hp->comp_done[b], main) == cudaSuccess &&
+         cudaStreamWaitEvent(hp->out, hp->comp_done[b], 0) == cudaSuccess &&
+         cudaMemcpy2DAsync(static_cast<char*>(out_host) + (size_t)t0 * row, host_pitch, out_buf(b), width, width, heads,
+                           cudaMemcpyDeviceToHost, hp->out) == cudaSuccess &&
+         cudaEventRecord(hp->out_done[b], hp->out) == cudaSuccess;
+  }
+  // the caller's stream ends behind the last copies back (the last two pieces cover both event slots)
+  ok = ok && cudaStreamWaitEvent(main, hp->out_done[0], 0) == cudaSuccess &&
+       cudaStreamWaitEvent(main, hp->out_done[1], 0) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return KATA_ERR_CUDA;
+  }
+  g_last_launches = launches;
+  return KATA_OK;
+}
+
 }  // namespace
 }  // namespace kata
 
@@ -580,6 +713,8 @@ int kata_fwd_host(int fn, const void* q_host, const void* k_host, const void* v_
   if ((reinterpret_cast<uintptr_t>(r.o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;
   st = check_arch();
   if (st != KATA_OK) return st;
+  PipePlan pp;
+  if (host_pipe_plan(fn, r, opts, C, pp)) return host_pipelined(r, pp, q_host, k_host, v_host, out_host, C, opts);
   char* ws = static_cast<char*>(r.o.workspace);
   const size_t eb = elem_bytes(r.p.dtype);
   const size_t nqk = (size_t)B * H * T * d_k * eb, nv = (size_t)B * H * T * d_v * eb;

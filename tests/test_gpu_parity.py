@@ -164,6 +164,30 @@ def test_host_io_entry_matches_device_entry():
     check(to_numpy64(ho2)[0, 0], oracle_full(w, heads=[(0, 0)])[(0, 0)], "bf16", "host scan")
 
 
+@pytest.mark.parametrize("B,H,T,groups", [(1, 2, 33000, 0), (2, 1, 40000, 2), (1, 1, 70001, 0)])
+def test_host_io_long_sequence_in_pieces(B, H, T, groups):
+    """Long sequences through the host-buffer entry are copied and computed piece by piece (state handed from
+    piece to piece, copies overlapped with the kernels): the result equals the device entry's within the bf16
+    tolerance and the oracle on sampled rows; the ragged last piece and a second call on the same buffers too."""
+    import torch
+    w = inputs.gaussian_workload("hostpipe", "bf16", B, H, T, 64, 64, 64, 31 + T)
+    q, k, v = dev_tensors(w)
+    ref = to_numpy64(kb.kata_fwd_chunked(q, k, v, feature_groups=groups))
+    hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+    ho = torch.empty_like(hv).pin_memory()
+    for rep in range(2):
+        ho.zero_()
+        kb.kata_fwd_host(kb.KATA_FN_CHUNKED, hq, hk, hv, ho, feature_groups=groups)
+        torch.cuda.synchronize()
+        assert kb.kata_last_launch_count() >= 4          # one kernel (and a state copy) per piece
+        g = to_numpy64(ho)
+        assert elem_err(g, ref) <= TOL["bf16"] and row_err(g, ref) <= TOL["bf16"]
+    picks = sample_picks(w, 96, T) + [(B - 1, H - 1, T - 1), (0, 0, 0)]
+    feature = "psd_direct" if groups == 0 else f"psd_direct:g{groups}"
+    got = np.stack([g[b, h, t] for b, h, t in picks])
+    check(got, oracle_rows(w, picks, feature), "bf16", "host pieces, sampled rows")
+
+
 # ---------------------------------------------------------------------------
 # first-order features (rows used as they are), nonnegative inputs so that D > 0
 # ---------------------------------------------------------------------------
