@@ -55,6 +55,9 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_update_kernel(const T* __r
   __shared__ float kh[64], qs[64], red[DEC_THREADS / 32][DV + 1];
   const int bh = blockIdx.y, slab = blockIdx.x, n_slabs = gridDim.x;
   const int tid = threadIdx.x;
+  // Launched with programmatic stream serialisation: the CTAs may be resident before the kernel ahead in the stream
+  // (the producer of q, k, v, or the previous step's finish kernel, which still reads `part`) has ended.
+  cudaGridDependencySynchronize();
   // k_hat = k / ||k|| (zero row -> zero feature); the query norm cancels in the readout and is not applied
   if (tid < 64) {
     float kv = tid < d_k ? to_f32<T>(k[(size_t)bh * d_k + tid]) : 0.f;
@@ -169,6 +172,9 @@ __global__ void decode_finish_kernel(const float* __restrict__ part, const T* __
     w += (order == 1) ? qk : qk * qk;
   }
   if (order != 1) w *= inv_or_zero(kk);     // raw q: the query norm cancels in the ratio
+  // Launched with programmatic stream serialisation: everything above ran while the update kernel was still
+  // streaming the state; its partial sums are visible from here on.
+  cudaGridDependencySynchronize();
   if (c >= DV) return;
   float num = 0.f, den = 0.f;
   for (int s = 0; s < n_slabs; ++s) {
@@ -184,12 +190,35 @@ template <typename T, int DV>
 void launch(const void* q, const void* k, const void* v, void* out, float* S, float* Z, float* part, int BH, int d_k,
             int n_psi, int layout, int order, int groups, LaunchCtx& ctx) {
   const int n_slabs = decode_slabs(n_psi);
-  decode_update_kernel<T, DV><<<dim3(n_slabs, BH), DEC_THREADS, 0, ctx.stream>>>(
-      static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), S, Z, part, d_k, n_psi, layout, order, groups);
-  note_launch(ctx);
-  decode_finish_kernel<T, DV><<<BH, 64, 0, ctx.stream>>>(part, static_cast<const T*>(q), static_cast<const T*>(k),
-                                                         static_cast<const T*>(v), static_cast<T*>(out), n_slabs, d_k, order, groups);
-  note_launch(ctx);
+  // both kernels may become resident before the kernel ahead of them has ended (each waits inside: the update kernel
+  // at its top, the finish kernel after its own prologue)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_slabs, BH);
+  cfg.blockDim = dim3(DEC_THREADS);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = ctx.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const float* part_c = part;
+  const T *qc = static_cast<const T*>(q), *kc = static_cast<const T*>(k), *vc = static_cast<const T*>(v);
+  T* oc = static_cast<T*>(out);
+  if (cudaLaunchKernelEx(&cfg, decode_update_kernel<T, DV>, qc, kc, vc, S, Z, part, d_k, n_psi, layout, order, groups) != cudaSuccess) {
+    cudaGetLastError();
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  ++ctx.launches;
+  cfg.gridDim = dim3(BH);
+  cfg.blockDim = dim3(64);
+  if (cudaLaunchKernelEx(&cfg, decode_finish_kernel<T, DV>, part_c, qc, kc, vc, oc, n_slabs, d_k, order, groups) != cudaSuccess) {
+    cudaGetLastError();
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  ++ctx.launches;
 }
 
 }  // namespace
