@@ -316,6 +316,7 @@ __global__ void __launch_bounds__(NTHR) chunk_simt_kernel(const T* __restrict__ 
 __global__ void scan_round_kernel(const float4* __restrict__ src, float4* __restrict__ dst, size_t e4,
                                   int n_groups, int g_used, int stride) {
   const int bh = blockIdx.y;
+  cudaGridDependencySynchronize();      // a programmatic dependent launch: resident while the kernel ahead drains
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)g_used * e4;
        i += (size_t)gridDim.x * blockDim.x) {
     const int g = (int)(i / e4);
@@ -566,10 +567,22 @@ const float* scan_group_states(float* bufA, float* bufB, int BH, int n_groups, i
   for (int stride = 1; stride < g_used; stride <<= 1) {
     const size_t work = (size_t)g_used * e4;
     const int blocks = (int)((work + 255) / 256 > 4096 ? 4096 : (work + 255) / 256);
-    scan_round_kernel<<<dim3(blocks, BH), 256, 0, ctx.stream>>>(reinterpret_cast<const float4*>(src),
-                                                                reinterpret_cast<float4*>(dst), e4, n_groups,
-                                                                g_used, stride);
-    note_launch(ctx);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks, BH);
+    cfg.blockDim = dim3(256);
+    cfg.stream = ctx.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, scan_round_kernel, reinterpret_cast<const float4*>(src), reinterpret_cast<float4*>(dst),
+                           e4, n_groups, g_used, stride) != cudaSuccess) {
+      cudaGetLastError();
+      ctx.status = KATA_ERR_CUDA;
+      return src;
+    }
+    ++ctx.launches;
     float* t = src; src = dst; dst = t;
   }
   return src;

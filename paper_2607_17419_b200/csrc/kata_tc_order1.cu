@@ -159,6 +159,10 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
   bool ok = true;
+  // Everything above touched only this CTA's shared memory and TMEM.  As a programmatic dependent launch (the
+  // restart pass behind the scan rounds) the CTA got here while the kernel ahead was still draining; its results
+  // (the prefix states) are visible from here on.  A no-op in an ordinary launch.
+  cudaGridDependencySynchronize();
 
   if (resume) {
     // the state before the first tile: into the accumulators and, as bf16, into snapshot 0
@@ -437,8 +441,28 @@ void tc_order1(const Problem& p, const ScanPlan& plan, bool use_scan, int C, flo
   a.init_state = incl;
   a.final_state = nullptr;
   a.write_out = 1;
-  tc_order1_kernel<<<dim3(BH, NG), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
-  note_launch(ctx);
+  if (NG > 1) {
+    // behind the scan rounds: resident, with its prologue done, while the last round drains
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(BH, NG);
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = SMEM_ALLOC;
+    cfg.stream = ctx.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, tc_order1_kernel, tmQ, tmK, tmV, a) != cudaSuccess) {
+      cudaGetLastError();
+      ctx.status = KATA_ERR_CUDA;
+      return;
+    }
+    ++ctx.launches;
+  } else {
+    tc_order1_kernel<<<dim3(BH, NG), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
+    note_launch(ctx);
+  }
 }
 
 }  // namespace kata
