@@ -167,6 +167,9 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       mbar_arrive_expect_tx(bar(BAR_QFULL), 16384);
       tma_load_3d(base + OFF_Q, &tmQ, bar(BAR_QFULL), 0, q0, bh);
     }
+    // The kernel is a programmatic dependent launch behind the pre-pass: up to here (and in every other warp) only
+    // q, k and on-chip memory were touched; the scaled values and r are the pre-pass's, visible from here on.
+    cudaGridDependencySynchronize();
     const __nv_bfloat16* rs = args.rscale + (size_t)bh * args.Tlen;
     // r of this lane's 4 keys of a tile, fetched one tile ahead (the global-load latency stays off the ring)
     auto load_r = [&](int j, unsigned short (&rv)[KPL]) {
@@ -406,8 +409,22 @@ void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchC
     return;
   }
   QArgs a{static_cast<__nv_bfloat16*>(p.out), rscale, device_status, p.T};
-  kern<<<dim3((p.T + QT - 1) / QT, BH), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
-  note_launch(ctx);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((p.T + QT - 1) / QT, BH);
+  cfg.blockDim = dim3(NTHREADS);
+  cfg.dynamicSmemBytes = SMEM_ALLOC;
+  cfg.stream = ctx.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, tmQ, tmK, tmV, a) != cudaSuccess) {
+    cudaGetLastError();
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  ++ctx.launches;
 }
 
 }  // namespace kata
