@@ -260,6 +260,15 @@ int kata_chunk_state_scan_static(const void* q, const void* k, const void* v, vo
  */
 size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
 
+/*
+ * Pieces of the token axis kata_fwd_host(fn, ...) would work in for these sizes and options, given a workspace of
+ * kata_workspace_bytes(fn | KATA_FN_HOST_IO, ...) bytes: 1 = copy in, run, copy back; more = the overlapped
+ * piecewise route described at kata_fwd_host; *piece_tokens (may be null) receives the length of a piece.
+ * Returns a KATA_ERR_* value for invalid arguments.  For reporting and tests.
+ */
+int kata_host_plan(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts, int* pieces,
+                   int* piece_tokens);
+
 /* Number of scan groups / chunks per group the library would use (for reporting and tests). */
 int kata_scan_plan(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts,
                    int* n_groups, int* chunks_per_group, int* scan_rounds);

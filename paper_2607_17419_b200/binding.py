@@ -24,7 +24,7 @@ KATA_FN_HOST_IO = 0x100
 
 EXPORTS = ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan", "kata_chunk_state_scan_static",
            "kata_fwd_host", "kata_decode_step", "kata_bwd_quadratic",
-           "kata_workspace_bytes", "kata_scan_plan", "kata_last_launch_count", "kata_last_impl",
+           "kata_workspace_bytes", "kata_scan_plan", "kata_host_plan", "kata_last_launch_count", "kata_last_impl",
            "kata_status_string",
            "kata_version")
 
@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
     L.kata_workspace_bytes.restype = ctypes.c_size_t
     L.kata_scan_plan.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(KataOpts)] + [ctypes.POINTER(i)] * 3
     L.kata_scan_plan.restype = i
+    L.kata_host_plan.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(KataOpts)] + [ctypes.POINTER(i)] * 2
+    L.kata_host_plan.restype = i
     L.kata_last_launch_count.argtypes = []
     L.kata_last_launch_count.restype = i
     L.kata_last_impl.argtypes = []
@@ -127,6 +129,15 @@ def kata_scan_plan(fn: int, B, H, T, d_k, d_v, C, opts: KataOpts):
     if st != 0:
         raise KataError(st, "kata_scan_plan")
     return a.value, b.value, c.value
+
+
+def kata_host_plan(fn: int, B, H, T, d_k, d_v, C, opts: KataOpts):
+    """(pieces, tokens per piece) the host-buffer entry would work in."""
+    a, b = ctypes.c_int(), ctypes.c_int()
+    st = lib().kata_host_plan(fn, B, H, T, d_k, d_v, C, ctypes.byref(opts), ctypes.byref(a), ctypes.byref(b))
+    if st != 0:
+        raise KataError(st, "kata_host_plan")
+    return a.value, b.value
 
 
 def kata_last_launch_count() -> int:

@@ -772,6 +772,21 @@ int kata_scan_plan(int fn, int B, int H, int T, int d_k, int d_v, int C, const k
   return KATA_OK;
 }
 
+int kata_host_plan(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts, int* pieces,
+                   int* piece_tokens) {
+  Prepared r;
+  fn &= ~KATA_FN_HOST_IO;
+  const int st = prepare(fn, nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, C, opts, false, r);
+  if (st != KATA_OK) return st;
+  // as if the caller had passed the workspace the host entry asks for
+  r.o.workspace_bytes = staging_layout(r.p, r.inner_bytes).total;
+  PipePlan pp;
+  const bool piecewise = host_pipe_plan(fn, r, opts, C, pp);
+  if (pieces) *pieces = piecewise ? pp.pieces : 1;
+  if (piece_tokens) *piece_tokens = piecewise ? pp.piece_T : T;
+  return KATA_OK;
+}
+
 int kata_last_launch_count(void) { return g_last_launches; }
 
 int kata_last_impl(void) { return g_last_impl; }

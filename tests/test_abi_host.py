@@ -156,6 +156,30 @@ def test_inter_chunk_auto_and_tensor_groups(L):
     assert g % 2 == 0 and (ng - 1) * g < 2048 <= ng * g
 
 
+def test_host_entry_piece_plan(L):
+    """The host-buffer entry works piece by piece only on long sequences of the sequential chunked form on the
+    tensor-core path: at least four pieces of at least 8192 tokens, at most eight, whole 128-token tiles."""
+    o = kb.make_opts(kb.KATA_BF16)
+    plan = lambda fn, B, H, T, opts=o, d=64: kb.kata_host_plan(fn, B, H, T, d, d, 64, opts)
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072) == (8, 16384)
+    assert plan(kb.KATA_FN_CHUNKED, 1, 2, 32768) == (4, 8192)
+    pieces, tokens = plan(kb.KATA_FN_CHUNKED, 1, 1, 70001)
+    assert tokens % 128 == 0 and (pieces - 1) * tokens < 70001 <= pieces * tokens and pieces == 8
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 32767) == (1, 32767)                  # too short
+    assert plan(kb.KATA_FN_QUADRATIC, 1, 16, 65536) == (1, 65536)                # needs every key
+    assert plan(kb.KATA_FN_CHUNK_STATE_SCAN, 1, 16, 131072) == (1, 131072)
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, inter_chunk=kb.KATA_SCAN)) == (1, 131072)
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_F32)) == (1, 131072)      # fp32 kernels
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, impl=kb.KATA_IMPL_SIMT)) == (1, 131072)
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, feature_order=1)) == (1, 131072)
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, o, d=32) == (1, 131072)       # padded rows
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, feature_groups=2)) == (8, 16384)
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, s_pre=4096, z_pre=8192)) == (1, 131072)
+    # the pieces fit the workspace the host entry asks for anyway
+    with pytest.raises(kb.KataError):
+        plan(kb.KATA_FN_CHUNKED, 0, 16, 131072)
+
+
 def test_no_oracle_in_product_path():
     """The package must not import or reference the oracle."""
     pkg = os.path.join(ROOT, "paper_2607_17419_b200")
