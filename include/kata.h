@@ -211,7 +211,7 @@ int kata_bwd_quadratic(const void* q, const void* k, const void* v, const void* 
  * the kernels run, and out is copied back, all enqueued on opts->stream; the caller synchronises
  * the stream before reading out.  Workspace: kata_workspace_bytes(fn | KATA_FN_HOST_IO, ...).
  * Long sequences (kata_fwd_chunked, inter_chunk = SEQUENTIAL, bf16, d_k = d_v = 64, feature_order 2, T >= 32768,
- * no state pointers in opts) are processed in up to eight pieces of the token axis: the copy in of the next piece
+ * no state pointers in opts) are processed in up to sixteen pieces of the token axis: the copy in of the next piece
  * and the copy back of the previous one run on two streams owned by the library while the current piece is
  * computed, each piece starting from the state the previous one left ("Linear attention as a recurrence").  The
  * caller's stream waits for all of it, so the contract above is unchanged, and so is the result (bit-identical to

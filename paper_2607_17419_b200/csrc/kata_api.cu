@@ -503,14 +503,14 @@ struct PipePlan {
   size_t total;
 };
 
-// Pieces of at least 8192 tokens, at most eight of them, whole 128-token tiles; bf16 d_k = d_v = 64 tensor-core path of
+// Pieces of at least 8192 tokens, at most sixteen of them, whole 128-token tiles; bf16 d_k = d_v = 64 tensor-core path of
 // the sequential form with no state asked for or given by the caller.
 bool host_pipe_plan(int fn, const Prepared& r, const kata_opts* opts, int C, PipePlan& pp) {
   const Problem& p = r.p;
   if (fn != KATA_FN_CHUNKED || !r.tensor || r.pad || r.o.inter_chunk != KATA_SEQUENTIAL || p.feature_order != 2) return false;
   if (r.o.s_pre != nullptr || r.o.s_init != nullptr || p.dtype != KATA_BF16 || p.d_k != 64 || p.d_v != 64) return false;
   if (p.T < 4 * 8192) return false;
-  pp.pieces = p.T / 8192 < 8 ? p.T / 8192 : 8;
+  pp.pieces = p.T / 8192 < 16 ? p.T / 8192 : 16;
   pp.piece_T = ((p.T + pp.pieces - 1) / pp.pieces + 127) / 128 * 128;
   pp.pieces = (p.T + pp.piece_T - 1) / pp.piece_T;
   pp.tensor_bytes = align_up((size_t)p.B * p.H * pp.piece_T * 64 * 2);

@@ -158,10 +158,10 @@ def test_inter_chunk_auto_and_tensor_groups(L):
 
 def test_host_entry_piece_plan(L):
     """The host-buffer entry works piece by piece only on long sequences of the sequential chunked form on the
-    tensor-core path: at least four pieces of at least 8192 tokens, at most eight, whole 128-token tiles."""
+    tensor-core path: at least four pieces of at least 8192 tokens, at most sixteen, whole 128-token tiles."""
     o = kb.make_opts(kb.KATA_BF16)
     plan = lambda fn, B, H, T, opts=o, d=64: kb.kata_host_plan(fn, B, H, T, d, d, 64, opts)
-    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072) == (8, 16384)
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072) == (16, 8192)
     assert plan(kb.KATA_FN_CHUNKED, 1, 2, 32768) == (4, 8192)
     pieces, tokens = plan(kb.KATA_FN_CHUNKED, 1, 1, 70001)
     assert tokens % 128 == 0 and (pieces - 1) * tokens < 70001 <= pieces * tokens and pieces == 8
@@ -173,7 +173,7 @@ def test_host_entry_piece_plan(L):
     assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, impl=kb.KATA_IMPL_SIMT)) == (1, 131072)
     assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, feature_order=1)) == (1, 131072)
     assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, o, d=32) == (1, 131072)       # padded rows
-    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, feature_groups=2)) == (8, 16384)
+    assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, feature_groups=2)) == (16, 8192)
     assert plan(kb.KATA_FN_CHUNKED, 1, 16, 131072, kb.make_opts(kb.KATA_BF16, s_pre=4096, z_pre=8192)) == (1, 131072)
     # the pieces fit the workspace the host entry asks for anyway
     with pytest.raises(kb.KataError):
