@@ -455,6 +455,9 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const float* comp_in = nullptr;
 #else
   const bool resume = comp_in != nullptr;
+  // This build is launched as a programmatic dependent launch behind the scan rounds: up to here the CTA touched
+  // only its own shared memory and TMEM; the prefix states are visible from here on.
+  cudaGridDependencySynchronize();
 #endif
   if (resume) {
     if (warp >= WARP_AUX0)
@@ -1135,7 +1138,27 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx) {
           io.s_final, io.z_final, io.s_init, io.z_init, io.init_compact, io.final_compact, io.write_out,
           io.n_groups > 0 ? io.tiles_per_group : n_tiles, n_groups};
   const int launch_groups = io.launch_groups > 0 ? io.launch_groups : n_groups;
+#if KATA_STREAM_MODE == 2
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(NSLICE, BH, launch_groups);
+  cfg.blockDim = dim3(NTHREADS);
+  cfg.dynamicSmemBytes = SMEM_ALLOC;
+  cfg.stream = ctx.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, tmQ, tmK, a) != cudaSuccess) {
+    cudaGetLastError();
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  ++ctx.launches;
+  return;
+#else
   kern<<<dim3(NSLICE, BH, launch_groups), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, a);
+#endif
 #else
   SArgs a{static_cast<const __nv_bfloat16*>(p.v), static_cast<__nv_bfloat16*>(p.out), device_status, p.T};
   kern<<<dim3(NSLICE, BH, 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, a);
