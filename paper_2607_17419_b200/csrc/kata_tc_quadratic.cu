@@ -32,7 +32,7 @@ using namespace umma;
 constexpr int D = 64;
 constexpr int QT = 128;          // queries per CTA
 constexpr int KTILE = 128;       // keys per tile
-constexpr int NSTAGE = 3;        // shared-memory stages of (K, V', r) tiles
+constexpr int NSTAGE = 4;        // shared-memory stages of (K, V', r) tiles
 constexpr int NBUF = 3;          // TMEM score / weight buffers
 constexpr int NTHREADS = 384;
 constexpr int WARP_BLD0 = 4;
@@ -55,13 +55,13 @@ enum {
   BAR_QFULL = 0,     // query tile landed in shared memory
   BAR_QTMEM = 1,     // query tile copied to TMEM (256 builders)
   BAR_FULL = 2,      // [3] K and V' tiles landed and the scale column written (TMA bytes + 32 producer lanes)
-  BAR_EMPTY = 5,     // [3] stage free: both issuers' commits
-  BAR_SFULL = 8,     // [3] scores in TMEM
-  BAR_PFULL = 11,    // [3] weights stored (256 builders)
-  BAR_PEMPTY = 14,   // [3] weights consumed by the apply MMA: the buffer may take new scores
-  BAR_ODONE = 17,
-  BAR_DRAIN = 18,
-  BAR_COUNT = 19
+  BAR_EMPTY = 6,     // [3] stage free: both issuers' commits
+  BAR_SFULL = 10,     // [3] scores in TMEM
+  BAR_PFULL = 13,    // [3] weights stored (256 builders)
+  BAR_PEMPTY = 16,   // [3] weights consumed by the apply MMA: the buffer may take new scores
+  BAR_ODONE = 19,
+  BAR_DRAIN = 20,
+  BAR_COUNT = 21
 };
 
 struct QArgs {
