@@ -483,13 +483,13 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const bool producer = (warp == WARP_UB);
       auto load_k = [&](int j) -> bool {
         const int s = kst(j);
-        if (!wait_or_abort(kempty(s), kph(j) ^ 1, abort_flag)) return false;
+        if (!wait_or_abort_counted(kempty(s), kph(j) ^ 1, abort_flag)) return false;
         mbar_arrive_expect_tx(kfull(s), 16384);
         tma_load_3d(ktile(s), &tmK, kfull(s), 0, (t0 + j) * CT, bh);
         return true;
       };
       auto load_q = [&](int j) -> bool {     // one staging buffer: free once the previous tile was copied to TMEM
-        if (!wait_or_abort(bar(BAR_QS_EMPTY), (j & 1) ^ 1, abort_flag)) return false;
+        if (!wait_or_abort_counted(bar(BAR_QS_EMPTY), (j & 1) ^ 1, abort_flag)) return false;
         mbar_arrive_expect_tx(bar(BAR_Q_FULL), 16384);
         tma_load_3d(qtile, &tmQ, bar(BAR_Q_FULL), 0, (t0 + j) * CT, bh);
         return true;
@@ -502,14 +502,14 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       uint32_t wbi = 0, wph = 0;             // W buffer of the step and the parity of its phase
       for (int j = 0; j < nch && ok; ++j) {
         const int s = kst(j);
-        ok = wait_or_abort(kfull(s), kph(j), abort_flag);
-        if (ok && wo && j > 0) ok = wait_or_abort(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
+        ok = wait_or_abort_counted(kfull(s), kph(j), abort_flag);
+        if (ok && wo && j > 0) ok = wait_or_abort_counted(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
         // the key stage of tile j - 1 is free once that tile's consumers are through: refill it (with tile j + 1;
         // with tile j + 2 where there are three stages)
         if (ok && producer && j > 0 && j + NKS - 1 < nch) ok = load_k(j + NKS - 1);
 #pragma unroll 1
         for (int sc = 0; sc < 8 && ok; ++sc) {
-          ok = wait_or_abort(bar(BAR_W_FULL + wbi), wph, abort_flag);
+          ok = wait_or_abort_counted(bar(BAR_W_FULL + wbi), wph, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint32_t wa = smem_u32(wbuf(wbi)), ka = smem_u32(ktile(s)) + sc * 2048;
@@ -548,13 +548,13 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const uint64_t dS = smem_desc(0, 16, 1024, kSwizzle128B);
       const uint32_t spa = smem_u32(base + OFF_SP);
       for (int j = 0; j < nch && ok; ++j) {
-        ok = wait_or_abort(bar(BAR_QT_FULL), j & 1, abort_flag);
-        if (ok && j > 0) ok = wait_or_abort(bar(BAR_SNAP_ST), (j - 1) & 1, abort_flag);
+        ok = wait_or_abort_counted(bar(BAR_QT_FULL), j & 1, abort_flag);
+        if (ok && j > 0) ok = wait_or_abort_counted(bar(BAR_SNAP_ST), (j - 1) & 1, abort_flag);
 #pragma unroll 1
         for (int p = 0; p < 8; ++p) {
           if (!ok) break;
           const int g = 8 * j + p, yb = g & 1;
-          ok = wait_or_abort(bar(BAR_Y_EMPTY + yb), ((g >> 1) & 1) ^ 1, abort_flag);
+          ok = wait_or_abort_counted(bar(BAR_Y_EMPTY + yb), ((g >> 1) & 1) ^ 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sbase = spa + (j & 1) * SP_BYTES + sp_block(p) * SP_BLOCK + sp_koff(p);
@@ -577,17 +577,17 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const uint64_t dK = smem_desc(0, 16, 1024, kSwizzle128B);
       for (int j = 0; j < nch && ok; ++j) {
         const int s = j & 1;
-        ok = wait_or_abort(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_QT_FULL), j & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
+        ok = wait_or_abort_counted(bar(BAR_K_FULL + s), (j >> 1) & 1, abort_flag) &&
+             wait_or_abort_counted(bar(BAR_QT_FULL), j & 1, abort_flag) &&
+             wait_or_abort_counted(bar(BAR_PREP + s), (j >> 1) & 1, abort_flag);
         // the weights of the previous tile's second half are read by its last apply MMAs
-        if (ok && j > 0) ok = wait_or_abort(bar(BAR_O_FULL), (j - 1) & 1, abort_flag);
+        if (ok && j > 0) ok = wait_or_abort_counted(bar(BAR_O_FULL), (j - 1) & 1, abort_flag);
         const uint32_t ka = smem_u32(ktile(s)), va = smem_u32(vptile(s));
 #pragma unroll
         for (int h = 0; h < NP; ++h) {
           if (!ok) break;
           // the weights of piece h - 1 alias the score columns: its apply MMAs must be through
-          if (h > 0) ok = wait_or_abort(bar(BAR_PV0), (j * (NP - 1) + h - 1) & 1, abort_flag);
+          if (h > 0) ok = wait_or_abort_counted(bar(BAR_PV0), (j * (NP - 1) + h - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
@@ -595,8 +595,8 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             mma_f16_ts(tb + COL_P + (ks / (4 / G)) * KH, tb + COL_Q + ks * 8, at(dK, ka + h * KH * 128 + ks * 32), idQK,
                        (ks % (4 / G)) > 0);
           mma_commit(bar(BAR_S_FULL));
-          ok = wait_or_abort(bar(BAR_P_FULL), h & 1, abort_flag);
-          if (ok && h == 0 && j > 0) ok = wait_or_abort(bar(BAR_O_EMPTY), (j - 1) & 1, abort_flag);
+          ok = wait_or_abort_counted(bar(BAR_P_FULL), h & 1, abort_flag);
+          if (ok && h == 0 && j > 0) ok = wait_or_abort_counted(bar(BAR_O_EMPTY), (j - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
@@ -625,7 +625,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // The buffer written was read by the reads of tile jp - 1.  They are complete: warps 20-23 wait for them
     // before they scale tile jp + 1, and the callers have waited for those scales (BAR_PREP).
     auto snapshot_share = [&](int jp) -> bool {
-      if (!wait_or_abort(bar(BAR_U_DONE), jp & 1, abort_flag)) return false;
+      if (!wait_or_abort_counted(bar(BAR_U_DONE), jp & 1, abort_flag)) return false;
       tc_fence_after();
       unsigned char* sp = base + OFF_SP + ((jp + 1) & 1) * SP_BYTES;
       auto rowp = [&](int p) { return sp + sp_block(p) * SP_BLOCK + (bloc & 7) * 1024 + vv * 128; };
@@ -741,7 +741,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     };
     for (int j = 0; j < nch && ok; ++j) {
       const int s = kst(j);
-      ok = wait_or_abort(kfull(s), kph(j), abort_flag) && wait_or_abort(kprep(s), kph(j), abort_flag);
+      ok = wait_or_abort_counted(kfull(s), kph(j), abort_flag) && wait_or_abort_counted(kprep(s), kph(j), abort_flag);
       // team 1 copies its share of the state after tile j - 1 before its first step of tile j, team 0 after
       // its first step: either way right when the update of tile j - 1 completes
       if (ok && wo && team == 1 && j > 0) ok = snapshot_share(j - 1);
@@ -752,7 +752,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint4 vp = *reinterpret_cast<const uint4*>(vptile(s) + t * 16);
         const uint32_t rr = r2pair(s)[t];
         const uint32_t kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
-        ok = wait_or_abort(bar(BAR_W_EMPTY + wbi), wph ^ 1, abort_flag);
+        ok = wait_or_abort_counted(bar(BAR_W_EMPTY + wbi), wph ^ 1, abort_flag);
         if (!ok) break;
         unsigned char* wrow = wbuf(wbi) + (tk >> 3) * 1024 + (tk & 7) * 128;
 #pragma unroll
@@ -791,7 +791,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     float* part = reinterpret_cast<float*>(base + OFF_PART);
     const uint32_t ycol = tmem_addr(tb, q4 * 32, COL_Y + team * 80);
     for (int j = 0; j < nch && ok && wo; ++j) {
-      ok = wait_or_abort(bar(BAR_QT_FULL), j & 1, abort_flag);    // the multipliers come from the TMEM copy of the query tile
+      ok = wait_or_abort_counted(bar(BAR_QT_FULL), j & 1, abort_flag);    // the multipliers come from the TMEM copy of the query tile
       if (!ok) break;
       tc_fence_after();
       float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
@@ -807,7 +807,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           tc_fence_before();
           mbar_arrive(bar(BAR_Q_FREE));
         }
-        ok = wait_or_abort(bar(BAR_Y_FULL + team), (g >> 1) & 1, abort_flag);
+        ok = wait_or_abort_counted(bar(BAR_Y_FULL + team), (g >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         uint32_t y0[16], y1[16], y2[16];
@@ -847,7 +847,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
       if (!ok) break;
       if (team == 1) {
-        ok = wait_or_abort(bar(BAR_PART_EMPTY), (j & 1) ^ 1, abort_flag);
+        ok = wait_or_abort_counted(bar(BAR_PART_EMPTY), (j & 1) ^ 1, abort_flag);
         if (!ok) break;
         part[0 * CT + t] = acc[0].x; part[1 * CT + t] = acc[0].y;
         part[2 * CT + t] = acc[1].x; part[3 * CT + t] = acc[1].y;
@@ -857,7 +857,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         mbar_arrive(bar(BAR_PART_FULL));
         continue;
       }
-      ok = wait_or_abort(bar(BAR_PART_FULL), j & 1, abort_flag);
+      ok = wait_or_abort_counted(bar(BAR_PART_FULL), j & 1, abort_flag);
       if (!ok) break;
       acc[0].x += part[0 * CT + t]; acc[0].y += part[1 * CT + t];
       acc[1].x += part[2 * CT + t]; acc[1].y += part[3 * CT + t];
@@ -865,7 +865,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       acc[3].x += part[6 * CT + t]; acc[3].y += part[7 * CT + t];
       accz += part[8 * CT + t];
       mbar_arrive(bar(BAR_PART_EMPTY));
-      ok = wait_or_abort(bar(BAR_O_FULL), j & 1, abort_flag);
+      ok = wait_or_abort_counted(bar(BAR_O_FULL), j & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       uint32_t o[16];
@@ -898,7 +898,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // key scales and v' of tile j (the value slice was fetched one tile earlier)
     auto prep = [&](int j, const uint4& vraw) -> bool {
       const int s = kst(j);
-      if (!wait_or_abort(kfull(s), kph(j), abort_flag)) return false;
+      if (!wait_or_abort_counted(kfull(s), kph(j), abort_flag)) return false;
       float ss = 0.f;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
@@ -1049,15 +1049,15 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
       if (j + 1 >= nch) break;
       if (!snapped) {
-        ok = wait_or_abort(bar(BAR_U_DONE), j & 1, abort_flag);
+        ok = wait_or_abort_counted(bar(BAR_U_DONE), j & 1, abort_flag);
         if (!ok) break;
         snapshot_share(j);
       }
       // ---- query tile j + 1 to TMEM, once the reads of tile j are complete, the readers hold their multipliers
       //      (the scores of tile j are complete: see above) and the tile has landed ----
       {
-        if (j >= 0) ok = wait_or_abort(bar(BAR_R_DONE), j & 1, abort_flag) && wait_or_abort(bar(BAR_Q_FREE), j & 1, abort_flag);
-        if (ok) ok = wait_or_abort(bar(BAR_Q_FULL), (j + 1) & 1, abort_flag);
+        if (j >= 0) ok = wait_or_abort_counted(bar(BAR_R_DONE), j & 1, abort_flag) && wait_or_abort_counted(bar(BAR_Q_FREE), j & 1, abort_flag);
+        if (ok) ok = wait_or_abort_counted(bar(BAR_Q_FULL), (j + 1) & 1, abort_flag);
         if (!ok) break;
         uint32_t qw[32];
 #pragma unroll
@@ -1076,13 +1076,13 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #if defined(KATA_STREAM_EXPORT) && KATA_STREAM_MODE == 1
     // ---- the state after the last token, from the accumulators to the public layout ----
     if (ok && args.s_final != nullptr) {
-      ok = wait_or_abort(bar(BAR_U_DONE), (nch - 1) & 1, abort_flag);
+      ok = wait_or_abort_counted(bar(BAR_U_DONE), (nch - 1) & 1, abort_flag);
       if (ok) export_state<G>(tb, q4, t, args.s_final, args.z_final, args.layout, bh, v0, slice);
     }
 #elif defined(KATA_STREAM_EXPORT) && KATA_STREAM_MODE == 3
     // ---- what the group adds to the state: the accumulators as they are (the one commit of this build's updates) ----
     if (ok) {
-      ok = wait_or_abort(bar(BAR_U_DONE), 0, abort_flag);
+      ok = wait_or_abort_counted(bar(BAR_U_DONE), 0, abort_flag);
       if (ok) export_compact<G>(tb, q4, t, comp_out);
     }
 #endif

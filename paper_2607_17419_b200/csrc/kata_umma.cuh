@@ -2,8 +2,8 @@
 // waits, TMEM allocation and access (tcgen05.alloc/ld/st), tcgen05.mma issue and commit, shared
 // memory matrix descriptors and the instruction descriptor, and TMA tile loads.
 //
-// Every wait is bounded: after `kSpinLimit` polls a wait gives up and returns false; the caller
-// records KATA_ERR_DEVICE_TIMEOUT and winds down (frees TMEM, returns).  Nothing here traps.
+// Every wait is bounded (by time in `wait_or_abort`, by `kSpinLimit` polls elsewhere): a wait that gives up returns
+// false; the caller records KATA_ERR_DEVICE_TIMEOUT and winds down (frees TMEM, returns).  Nothing here traps.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -281,23 +281,56 @@ __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t chunk16)
 // ---------------------------------------------------------------------------------------------
 // helpers shared by the tensor-core kernels
 // ---------------------------------------------------------------------------------------------
-// Bounded wait, as few instructions per poll as possible (24 warps poll most of the time and share the issue
-// slots with the warps that work): try_wait, exit branch, counter, loop branch.  A wait that gives up raises the
+// Bounded wait.  The try_wait carries a suspend-time hint: the waiting warp sleeps in the barrier unit until the
+// phase completes (or the hint runs out) instead of coming back to poll, so the two dozen warps that wait most of
+// the time take hardly any issue slots or shared-memory bandwidth from the warps that work.  The bound is on time:
+// after the first failed try the clock is read, and a wait that has lasted kWaitLimitNs gives up and raises the
 // abort flag; the other waiters give up on their own limits.
+constexpr uint32_t kSuspendHintNs = 10000000u;      // upper bound the hardware may cut short
+constexpr uint32_t kWaitLimitNs = 100000000u;       // 0.1 s (the low word of the timer wraps every 4.3 s)
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u32 t0, t1;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "@p bra KATA_DONE_%=;\n\t"
+      "mov.u32 t0, %%globaltimer_lo;\n\t"
+      "KATA_WAIT_%=:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "@p bra KATA_DONE_%=;\n\t"
+      "mov.u32 t1, %%globaltimer_lo;\n\t"
+      "sub.u32 t1, t1, t0;\n\t"
+      "setp.lt.u32 q, t1, %4;\n\t"
+      "@q bra KATA_WAIT_%=;\n\t"
+      "KATA_DONE_%=:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs), "r"(kWaitLimitNs)
+      : "memory");
+  if (ok == 0) *abort_flag = 1;
+  return ok != 0;
+}
+
+// The same wait bounded by a poll count (one register less, one instruction less per poll; for the kernel that runs
+// at its register cap).  With a hint of 1 us a wait gives up after at most kSpinLimit x 1 us = 4 s, and no sooner
+// than kSpinLimit polls take where the hardware cuts the suspension short (0.1 s).
+__device__ __forceinline__ bool wait_or_abort_counted(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   uint32_t ok;
   asm volatile(
       "{\n\t"
       ".reg .pred p, q;\n\t"
       ".reg .u32 i;\n\t"
       "mov.u32 i, 0;\n\t"
-      "KATA_WAIT_%=:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "@p bra KATA_DONE_%=;\n\t"
+      "KATA_WAITC_%=:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 1000;\n\t"
+      "@p bra KATA_DONEC_%=;\n\t"
       "add.u32 i, i, 1;\n\t"
       "setp.lt.u32 q, i, %3;\n\t"
-      "@q bra KATA_WAIT_%=;\n\t"
-      "KATA_DONE_%=:\n\t"
+      "@q bra KATA_WAITC_%=;\n\t"
+      "KATA_DONEC_%=:\n\t"
       "selp.u32 %0, 1, 0, p;\n\t"
       "}"
       : "=r"(ok)
