@@ -19,6 +19,7 @@
 // No atomics, every sum in a fixed order.  Warps (384 threads): 0 TMA producer, 1 score-MMA issuer, 2 output-MMA
 // issuer, 4-11 weights and epilogue.  All waits are bounded.
 #include <cuda.h>
+#include <type_traits>
 
 #include "kata_common.cuh"
 #include "kata_tmap.cuh"
@@ -367,17 +368,21 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
         const float2* cs = reinterpret_cast<const float2*>(sc(s) + ch * 128);
         const bool diag = n0 + 31 > m0;                 // some key of these columns lies after some query of the tile
         float2 d2 = make_float2(0.f, 0.f), m2 = make_float2(0.f, 0.f);
+        // two copies of the loop, chosen once per tile: the causal test exists on diagonal tiles only
+        auto sums = [&](auto masked) {
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float2 s2 = make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1]));
-          float2 a2 = __fmul2_rn(__fmul2_rn(s2, s2), cs[c / 2]);
-          if (diag) {
-            if (n0 + c > grow) a2.x = 0.f;
-            if (n0 + c + 1 > grow) a2.y = 0.f;
+          for (int c = 0; c < 32; c += 2) {
+            const float2 s2 = make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1]));
+            float2 a2 = __fmul2_rn(__fmul2_rn(s2, s2), cs[c / 2]);
+            if constexpr (decltype(masked)::value) {
+              if (n0 + c > grow) a2.x = 0.f;
+              if (n0 + c + 1 > grow) a2.y = 0.f;
+            }
+            d2 = __fadd2_rn(d2, a2);
+            m2 = __ffma2_rn(a2, make_float2(__uint_as_float(cv[c]), __uint_as_float(cv[c + 1])), m2);
           }
-          d2 = __fadd2_rn(d2, a2);
-          m2 = __ffma2_rn(a2, make_float2(__uint_as_float(cv[c]), __uint_as_float(cv[c + 1])), m2);
-        }
+        };
+        if (diag) sums(std::true_type{}); else sums(std::false_type{});
         sum_d += d2.x + d2.y;
         sum_m += m2.x + m2.y;
         // nothing is stored; the buffer is handed on as it is
@@ -389,36 +394,42 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
         // e = 2 (c - dout.o) / D * s, keys n <= this query
         const float2 f2 = make_float2(2.f * inv_row, 2.f * inv_row), nd2 = make_float2(-del_row, -del_row);
         const bool diag = n0 + 31 > m0;
+        auto weigh = [&](auto masked) {
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float2 s2 = make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1]));
-          const float2 c2 = make_float2(__uint_as_float(cv[c]), __uint_as_float(cv[c + 1]));
-          float2 e2 = __fmul2_rn(__fmul2_rn(__fadd2_rn(c2, nd2), f2), s2);
-          if (diag) {
-            if (n0 + c > grow) e2.x = 0.f;
-            if (n0 + c + 1 > grow) e2.y = 0.f;
+          for (int c = 0; c < 32; c += 2) {
+            const float2 s2 = make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1]));
+            const float2 c2 = make_float2(__uint_as_float(cv[c]), __uint_as_float(cv[c + 1]));
+            float2 e2 = __fmul2_rn(__fmul2_rn(__fadd2_rn(c2, nd2), f2), s2);
+            if constexpr (decltype(masked)::value) {
+              if (n0 + c > grow) e2.x = 0.f;
+              if (n0 + c + 1 > grow) e2.y = 0.f;
+            }
+            pe[c / 2] = pack_bf16(e2.x, e2.y);
           }
-          pe[c / 2] = pack_bf16(e2.x, e2.y);
-        }
+        };
+        if (diag) weigh(std::true_type{}); else weigh(std::false_type{});
       } else {
         // p = s^2 / D_t, e = 2 (c - dout_t.o_t) / D_t * s with the scalars of the columns (queries t >= this key)
         const float4* cs = reinterpret_cast<const float4*>(sc(s) + ch * 256);
         const bool diag = n0 < m0 + MT - 1;             // some query of these columns lies before some key of the tile
+        auto weigh = [&](auto masked) {
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float4 st = cs[c / 2];                       // (1/D, dout.o) of queries n0 + c, n0 + c + 1
-          const float2 s2 = make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1]));
-          const float2 c2 = make_float2(__uint_as_float(cv[c]), __uint_as_float(cv[c + 1]));
-          const float2 t2 = __fmul2_rn(s2, make_float2(st.x, st.z));                    // s / D
-          float2 p2 = __fmul2_rn(t2, s2);                                               // s^2 / D
-          float2 e2 = __fmul2_rn(__fadd2_rn(c2, make_float2(-st.y, -st.w)), __fadd2_rn(t2, t2));
-          if (diag) {
-            if (n0 + c < grow) { p2.x = 0.f; e2.x = 0.f; }
-            if (n0 + c + 1 < grow) { p2.y = 0.f; e2.y = 0.f; }
+          for (int c = 0; c < 32; c += 2) {
+            const float4 st = cs[c / 2];                       // (1/D, dout.o) of queries n0 + c, n0 + c + 1
+            const float2 s2 = make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1]));
+            const float2 c2 = make_float2(__uint_as_float(cv[c]), __uint_as_float(cv[c + 1]));
+            const float2 t2 = __fmul2_rn(s2, make_float2(st.x, st.z));                    // s / D
+            float2 p2 = __fmul2_rn(t2, s2);                                               // s^2 / D
+            float2 e2 = __fmul2_rn(__fadd2_rn(c2, make_float2(-st.y, -st.w)), __fadd2_rn(t2, t2));
+            if constexpr (decltype(masked)::value) {
+              if (n0 + c < grow) { p2.x = 0.f; e2.x = 0.f; }
+              if (n0 + c + 1 < grow) { p2.y = 0.f; e2.y = 0.f; }
+            }
+            pp[c / 2] = pack_bf16(p2.x, p2.y);
+            pe[c / 2] = pack_bf16(e2.x, e2.y);
           }
-          pp[c / 2] = pack_bf16(p2.x, p2.y);
-          pe[c / 2] = pack_bf16(e2.x, e2.y);
-        }
+        };
+        if (diag) weigh(std::true_type{}); else weigh(std::false_type{});
       }
       // the weights overwrite score columns [0,32) of each half, which the column-half-0 warp of this quadrant
       // reads: both warps of the quadrant must have their scores in registers first

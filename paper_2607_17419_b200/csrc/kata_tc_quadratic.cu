@@ -19,6 +19,7 @@
 // issuer, 2 apply-MMA issuer, 3 idle, 4-11 weight builders (TMEM lane quadrant = warp % 4, column half =
 // (warp - 4) / 4).  All waits are bounded.
 #include <cuda.h>
+#include <type_traits>
 
 #include "kata_common.cuh"
 #include "kata_tmap.cuh"
@@ -283,20 +284,24 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
 #pragma unroll
         for (int g = 0; g < G; ++g) tmem_wait_ld(y[g]);
+        // two copies of the loop, chosen once per tile: the causal test exists on the diagonal tiles only
+        auto weigh_g = [&](auto masked) {
 #pragma unroll
-        for (int c = 0; c < KH; c += 2) {
-          float2 w = make_float2(0.f, 0.f);
+          for (int c = 0; c < KH; c += 2) {
+            float2 w = make_float2(0.f, 0.f);
 #pragma unroll
-          for (int g = 0; g < G; ++g) {
-            const float2 sv = make_float2(__uint_as_float(y[g][c]), __uint_as_float(y[g][c + 1]));
-            w = __ffma2_rn(sv, sv, w);
+            for (int g = 0; g < G; ++g) {
+              const float2 sv = make_float2(__uint_as_float(y[g][c]), __uint_as_float(y[g][c + 1]));
+              w = __ffma2_rn(sv, sv, w);
+            }
+            if constexpr (decltype(masked)::value) {
+              if (key0 + c > qrow) w.x = 0.f;
+              if (key0 + c + 1 > qrow) w.y = 0.f;
+            }
+            pk[c / 2] = pack_bf16(w.x, w.y);
           }
-          if (diag) {
-            if (key0 + c > qrow) w.x = 0.f;
-            if (key0 + c + 1 > qrow) w.y = 0.f;
-          }
-          pk[c / 2] = pack_bf16(w.x, w.y);
-        }
+        };
+        if (diag) weigh_g(std::true_type{}); else weigh_g(std::false_type{});
         // the weights overwrite score columns [0, KT/2) of the buffer (group 0, read by the ch = 0 warp)
         tc_fence_before();
         asm volatile("bar.sync %0, 64;" ::"r"(1 + (int)q4) : "memory");
@@ -311,13 +316,14 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const uint32_t scol = tmem_addr(tb, q4 * 32, COL_S + b * 128 + ch * 64);
       const int key0 = j * KTILE + ch * 64;
       uint32_t ya[32], yb[32], pk[32];
-      auto weigh = [&](const uint32_t (&y)[32], int half) {
+      // two copies of the loop, chosen once per tile: the causal test exists on the diagonal tile only
+      auto weigh = [&](const uint32_t (&y)[32], int half, auto masked) {
 #pragma unroll
         for (int jj = 0; jj < 32; jj += 2) {
           const int c = half * 32 + jj;
           const float2 sv = make_float2(__uint_as_float(y[jj]), __uint_as_float(y[jj + 1]));
           float2 w = __fmul2_rn(sv, sv);
-          if (diag) {
+          if constexpr (decltype(masked)::value) {
             if (key0 + c > qrow) w.x = 0.f;
             if (key0 + c + 1 > qrow) w.y = 0.f;
           }
@@ -327,9 +333,15 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       tmem_ld32(scol, ya);
       tmem_wait_ld(ya);
       tmem_ld32(scol + 32, yb);
-      weigh(ya, 0);
-      tmem_wait_ld(yb);
-      weigh(yb, 1);
+      if (diag) {
+        weigh(ya, 0, std::true_type{});
+        tmem_wait_ld(yb);
+        weigh(yb, 1, std::true_type{});
+      } else {
+        weigh(ya, 0, std::false_type{});
+        tmem_wait_ld(yb);
+        weigh(yb, 1, std::false_type{});
+      }
       // the weights overwrite score columns [0,64) of the buffer, which the column-half-0 warp of this
       // quadrant reads: both warps of the quadrant must have their scores in registers first
       tc_fence_before();
