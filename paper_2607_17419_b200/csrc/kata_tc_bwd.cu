@@ -288,22 +288,26 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
         const bool diag = MODE == MODE_DQ ? (n0 + 31 > m0) : (n0 < m0 + MT - 1);
         auto dead = [&](int c) { return MODE == MODE_DQ ? (n0 + c > grow) : (n0 + c < grow); };
         float2 cf[16], ss[16];
+        // two copies of each loop with a causal test, chosen once per tile: the test exists on diagonal tiles only
+        auto factors = [&](auto masked) {
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float2 c2 = make_float2(__uint_as_float(cvg[c]), __uint_as_float(cvg[c + 1]));
-          if (MODE == MODE_DQ) {
-            // second sweep: 2 (c - dout.o) / D; first sweep: c as it is
-            cf[c / 2] = first ? c2 : __fmul2_rn(__fadd2_rn(c2, make_float2(-del_row, -del_row)), make_float2(2.f * inv_row, 2.f * inv_row));
-          } else {
-            const float4 st = reinterpret_cast<const float4*>(sc(s) + ch * 256)[c / 2];
-            cf[c / 2] = __fmul2_rn(__fadd2_rn(c2, make_float2(-st.y, -st.w)), make_float2(2.f * st.x, 2.f * st.z));
+          for (int c = 0; c < 32; c += 2) {
+            const float2 c2 = make_float2(__uint_as_float(cvg[c]), __uint_as_float(cvg[c + 1]));
+            if (MODE == MODE_DQ) {
+              // second sweep: 2 (c - dout.o) / D; first sweep: c as it is
+              cf[c / 2] = first ? c2 : __fmul2_rn(__fadd2_rn(c2, make_float2(-del_row, -del_row)), make_float2(2.f * inv_row, 2.f * inv_row));
+            } else {
+              const float4 st = reinterpret_cast<const float4*>(sc(s) + ch * 256)[c / 2];
+              cf[c / 2] = __fmul2_rn(__fadd2_rn(c2, make_float2(-st.y, -st.w)), make_float2(2.f * st.x, 2.f * st.z));
+            }
+            if constexpr (decltype(masked)::value) {
+              if (dead(c)) cf[c / 2].x = 0.f;
+              if (dead(c + 1)) cf[c / 2].y = 0.f;
+            }
+            ss[c / 2] = make_float2(0.f, 0.f);
           }
-          if (diag && !first) {
-            if (dead(c)) cf[c / 2].x = 0.f;
-            if (dead(c + 1)) cf[c / 2].y = 0.f;
-          }
-          ss[c / 2] = make_float2(0.f, 0.f);
-        }
+        };
+        if (diag && !first) factors(std::true_type{}); else factors(std::false_type{});
 #pragma unroll 1
         for (int g = 0; g < G; ++g) {
           tmem_ld32(bcol + g * 64, sg);
@@ -326,30 +330,36 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
           // a = r_i sum_g s_g^2 for the keys n <= this query; D_t += a, sum += a c
           const float2* cs = reinterpret_cast<const float2*>(sc(s) + ch * 128);
           float2 d2 = make_float2(0.f, 0.f), m2 = make_float2(0.f, 0.f);
+          auto sums = [&](auto masked) {
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) {
-            float2 a2 = __fmul2_rn(ss[c / 2], cs[c / 2]);
-            if (diag) {
-              if (dead(c)) a2.x = 0.f;
-              if (dead(c + 1)) a2.y = 0.f;
+            for (int c = 0; c < 32; c += 2) {
+              float2 a2 = __fmul2_rn(ss[c / 2], cs[c / 2]);
+              if constexpr (decltype(masked)::value) {
+                if (dead(c)) a2.x = 0.f;
+                if (dead(c + 1)) a2.y = 0.f;
+              }
+              d2 = __fadd2_rn(d2, a2);
+              m2 = __ffma2_rn(a2, cf[c / 2], m2);
             }
-            d2 = __fadd2_rn(d2, a2);
-            m2 = __ffma2_rn(a2, cf[c / 2], m2);
-          }
+          };
+          if (diag) sums(std::true_type{}); else sums(std::false_type{});
           sum_d += d2.x + d2.y;
           sum_m += m2.x + m2.y;
         } else if (MODE == MODE_DKV) {
           // P^T = sum_g s_g^2 / D_t over the C block (both warps of the quadrant hold its scores since the first sync)
+          auto weights = [&](auto masked) {
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) {
-            const float4 st = reinterpret_cast<const float4*>(sc(s) + ch * 256)[c / 2];
-            float2 p2 = __fmul2_rn(ss[c / 2], make_float2(st.x, st.z));
-            if (diag) {
-              if (dead(c)) p2.x = 0.f;
-              if (dead(c + 1)) p2.y = 0.f;
+            for (int c = 0; c < 32; c += 2) {
+              const float4 st = reinterpret_cast<const float4*>(sc(s) + ch * 256)[c / 2];
+              float2 p2 = __fmul2_rn(ss[c / 2], make_float2(st.x, st.z));
+              if constexpr (decltype(masked)::value) {
+                if (dead(c)) p2.x = 0.f;
+                if (dead(c + 1)) p2.y = 0.f;
+              }
+              pk[c / 2] = pack_bf16(p2.x, p2.y);
             }
-            pk[c / 2] = pack_bf16(p2.x, p2.y);
-          }
+          };
+          if (diag) weights(std::true_type{}); else weights(std::false_type{});
           tmem_st16(tmem_addr(tb, q4 * 32, COL_B + b * BW + CB + ch * 16), pk);
         }
         tmem_wait_st();
