@@ -1,6 +1,7 @@
 // C ABI of the KATA forward library: argument validation, scan planning, workspace carve-up and
 // dispatch to the SIMT (fp32) or tensor-core (tcgen05) kernels.  Declarations and the contract of
 // every entry point are in include/kata.h.
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -260,6 +261,16 @@ Staging staging_layout(const Problem& p, size_t inner_bytes) {
   return s;
 }
 
+// Diagnostic override: KATA_CHUNKED_KERNEL=stream in the environment keeps the sequential chunked form on the
+// value-sliced streaming kernel (for A/B timing); read once.
+bool stream_kernel_forced() {
+  static const bool forced = []() {
+    const char* e = getenv("KATA_CHUNKED_KERNEL");
+    return e != nullptr && strcmp(e, "stream") == 0;
+  }();
+  return forced;
+}
+
 int check_arch() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) {
@@ -283,6 +294,7 @@ struct Prepared {
   size_t inner_bytes;
   bool tensor;
   int C;
+  bool split;           // sequential chunked form on the feature-split kernel (needs scratch for the links of a head)
   bool pad;             // bf16 rows narrower than 64 are zero-padded to 64 so that the tensor-core kernels apply
   size_t pad_bytes;     // one padded tensor [B*H*T][64] bf16 (q, k, v, out: four of them at the start of the scratch)
 };
@@ -360,6 +372,7 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
   r.C = fn == KATA_FN_QUADRATIC ? kChunk : C;
   r.plan = ScanPlan{(T + r.C - 1) / r.C, 0, 1, 0};
   r.state_elems = 0;
+  r.split = false;
   r.inner_bytes = (fn == KATA_FN_QUADRATIC && r.tensor) ? tc_quadratic_workspace_bytes(kp) : 0;
   if (fn != KATA_FN_QUADRATIC) {
     if (r.tensor && r.o.s_pre != nullptr && fn == KATA_FN_CHUNK_STATE_SCAN) r.tensor = false;   // per-chunk export: SIMT pipeline
@@ -368,6 +381,10 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
     st = make_plan(fn, kp, r.o, r.tensor, r.C, r.plan, r.state_elems);
     if (st != KATA_OK) return st;
     r.inner_bytes = inner_workspace(fn, r.plan, kp, r.state_elems);
+    // one pass over the whole sequence, no state handed in or out: the feature-split kernel
+    r.split = fn == KATA_FN_CHUNKED && r.tensor && r.plan.n_groups == 1 && r.o.s_pre == nullptr && r.o.s_init == nullptr &&
+              tc_split_supported(kp) && !stream_kernel_forced();
+    if (r.split) r.inner_bytes = align_up(tc_split_workspace_bytes(kp));
     // state import and final-state export of the fp32 path go through one internal state per head
     if (fn == KATA_FN_CHUNKED && (r.o.s_pre != nullptr || r.o.s_init != nullptr) && !r.tensor)
       r.inner_bytes = align_up((size_t)B * H * r.state_elems * sizeof(float));
@@ -411,6 +428,8 @@ int run_device(int fn, Prepared& r, void* ws) {
     const bool use_scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || r.plan.n_groups > 1;
     if (r.tensor && P.feature_order == 1) {
       tc_order1(P, r.plan, use_scan, r.C, wsf, r.o.device_status, ctx);
+    } else if (r.split) {
+      tc_chunked_split(P, ws, r.o.device_status, ctx);
     } else if (r.tensor) {
       const float* z_init = r.o.z_init;
       if (fn == KATA_FN_CHUNKED && z_init != nullptr && z_init == r.o.z_pre) {

@@ -95,6 +95,10 @@ bool tc_supported(const Problem& p, int fn, bool scan);
 size_t tc_quadratic_workspace_bytes(const Problem& p);
 void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx);
 void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx);
+// Sequential chunked form with the feature axis of the state split over the CTAs of a head (kata_tc_split.cu)
+bool tc_split_supported(const Problem& p);
+size_t tc_split_workspace_bytes(const Problem& p);
+void tc_chunked_split(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx);
 // State hand-off and groups of tiles for the second build of the streaming kernel (zero-initialise, then set).
 struct StreamIO {
   const float* s_init;         // state before the first token in the public layout (null: zero)

@@ -1,0 +1,808 @@
+// Chunked (linear-state) KATA forward on the Blackwell tensor cores with the FEATURE axis of the state split over
+// the CTAs of a head (bf16, d_k = d_v = 64, sequential inter-chunk recurrence, whole sequence in one pass).
+//
+// Algorithm 1 / section "Chunkwise forward", with the rank-one lift psi(u) = u u^T written as 8 x 8 blocks: the 64
+// features of a row are cut into 8 runs of 8, and a "block pair" (g, h), g <= h, is the 64 products
+// u[8g+i] u[8h+j].  <psi(q), psi(k)> = (q.k)^2 = sum over the 36 block pairs of w_gh <Q_gh, K_gh> with w = 1 on
+// the diagonal pairs (which hold both (i,j) and (j,i)) and w = 2 off it.  One CTA owns 4 block pairs = 256 state
+// rows (two M = 128 accumulator tiles S[m], 80 fp32 TMEM columns each: 64 value columns, the normaliser column,
+// padding); nine CTAs make a head.  With k' scale r = 1/||k||^2 folded into the values (V' = r V) and the
+// normaliser carried as column 64 of every B operand, per tile of 128 tokens a CTA does
+//   update   S[m] += Psi(K)_m^T [V' | r]      A = the products, built by token threads in shared memory (MN-major),
+//                                             B = the TMA-loaded value tile scaled in place, N = 80
+//   snapshot B_m = bf16(S[m])                 TMEM -> shared memory, the B operand of the next tile's read
+//   read     ACC  = Psi(Q)_m [S | Z]_m        A = the weighted query products in TMEM, N = 80
+//   intra    ACC += P_c [V' | r]_c            P_c = (Q K_c^T)^2 masked causally for the 16 keys c of the tile this
+//                                             CTA owns (the eight 16-key runs of a tile go to eight of the CTAs)
+// ACC is this CTA's share of [N | D] of the tile's 128 queries; the shares are summed
+//   (a) inside a thread-block cluster through distributed shared memory (every CTA owns 128 / CS query rows), then
+//   (b) from cluster to cluster ("links" of a head) through fp32 scratch in global memory: a link adds what the
+//       link before it left (release/acquire progress counters; a link never waits for a later one), and the last
+//       link applies the gate/normalise step out = N / D (0 where D = 0) and writes the output.
+// The query norm cancels between N and D and is never applied.
+//
+// Why links: a head needs nine CTAs (36 block pairs / 4), and 16 clusters of 8 or 9 CTAs do not fit the GPCs of a
+// B200 at once.  Clusters of 4 do: a head is one single CTA (link 0, its own launch) and two clusters of 4.
+//
+// Warps (896 threads): 0 TMA producer, 1 update issuer, 2 read issuer, 3 score issuer; 4-11 key teams (team m
+// builds the products of accumulator tile m; both scale the values); 12-15 query team; 16-23 state teams
+// (TMEM -> bf16 snapshot); 24-27 weights, share exchange, owner sums and output.  Every wait is bounded.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cstdlib>
+
+#include "kata_common.cuh"
+#include "kata_tmap.cuh"
+#include "kata_umma.cuh"
+
+namespace kata {
+namespace {
+
+using namespace umma;
+
+constexpr int D = 64;
+constexpr int CT = 128;            // tokens per tile
+constexpr int NBP = 4;             // block pairs per CTA
+constexpr int NTHREADS = 896;
+constexpr int W_TMA = 0, W_U = 1, W_R = 2, W_I = 3, W_K0 = 4, W_Q0 = 12, W_S0 = 16, W_E0 = 24;
+constexpr int MAX_CTAS = 12;       // CTAs of a head over all links
+
+// ---- TMEM columns ----
+constexpr uint32_t COL_S = 0;      // 2 x 80: state tiles (lanes = state rows)
+constexpr uint32_t COL_PSIQ = 160; // 128: weighted query products as bf16 pairs (lanes = tokens), 32 per block pair
+constexpr uint32_t COL_ACC = 288;  // 2 x 80: this CTA's share of [N | D] (lanes = tokens)
+constexpr uint32_t COL_SC = 448;   // 16 fp32 scores
+constexpr uint32_t COL_P = 464;    // 2 x 8: bf16 weights
+constexpr uint32_t TMEM_COLS = 512;
+
+// ---- shared memory (1024-byte aligned tiles of 128-byte rows, 128B swizzle) ----
+constexpr uint32_t OFF_PSIK = 0;        // 4 block pairs x [128 tokens][64 products]
+constexpr uint32_t OFF_KRAW = 65536;    // key tile
+constexpr uint32_t OFF_QRAW = 81920;    // query tile
+constexpr uint32_t OFF_VP = 98304;      // 2 x value tile (scaled in place)
+constexpr uint32_t OFF_SNAP = 131072;   // 2 x [128 state rows][64 values] bf16
+constexpr uint32_t OFF_COL64 = 163840;  // column 64 of the four B operands above: 32 bytes of every row each
+constexpr uint32_t OFF_RECV = 180224;   // 128 rows x 68 floats: shares received for the rows this CTA owns
+constexpr uint32_t RECV_ROW = 272;
+constexpr uint32_t OFF_BAR = OFF_RECV + 128 * RECV_ROW;
+constexpr uint32_t OFF_MISC = OFF_BAR + 512;
+constexpr uint32_t OFF_SINK = OFF_MISC + 64;   // one word per thread: see consume_before_arrive
+constexpr uint32_t SMEM_BYTES = OFF_SINK + NTHREADS * 4;
+constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
+static_assert(SMEM_ALLOC <= 232448, "shared memory");
+
+// Every barrier has waiters that consume each of its phases in order.
+enum {
+  B_K_FULL = 0,      // key tile landed
+  B_K_EMPTY = 1,     // ... and read by the 256 key threads
+  B_Q_FULL = 2,
+  B_Q_EMPTY = 3,     // ... by the 128 query threads
+  B_V_FULL = 4,      // [2] value tile landed
+  B_VP_READY = 6,    // [2] values scaled, column 64 written (256 key threads)
+  B_VP_EMPTY = 8,    // [2] update and intra MMAs of the tile complete
+  B_PSIK_FULL = 10,  // [2] products of accumulator tile m built (128 threads)
+  B_U_DONE = 12,     // [2] update of accumulator tile m complete
+  B_S_FREE = 14,     // [2] accumulator tile m copied out of TMEM (128 threads)
+  B_SNAP_FULL = 16,  // [2] snapshot m stored (128 threads)
+  B_R_DONE = 18,     // [2] read MMAs of half m complete
+  B_PSIQ_FULL = 20,  // [2] query products of half m stored (128 threads)
+  B_SC_FULL = 22,    // scores in TMEM
+  B_P_FULL = 23,     // [2] weights stored in buffer tile & 1 (128 threads)
+  B_ACC_FULL = 25,   // [2]
+  B_ACC_EMPTY = 27,  // [2] (128 threads)
+  B_RECV_FULL = 29,  // 128 arrivals from the CTAs of the cluster
+  B_RECV_EMPTY = 30, // [4] the owner with that rank has summed what this CTA sent
+  B_DRAIN = 34,
+  B_K_USED = 35,     // the score MMAs that read the key tile are complete (commit only)
+  B_Q_USED = 36,     // ... the query tile
+  B_COUNT = 37
+};
+
+struct BlockPairs {
+  unsigned char g[MAX_CTAS * NBP], h[MAX_CTAS * NBP], w[MAX_CTAS * NBP];   // w = 0: unused slot
+};
+
+struct SplitArgs {
+  __nv_bfloat16* out;
+  float* scrN;            // [links - 1][BH][Tpad][64]
+  float* scrD;            // [links - 1][BH][Tpad]
+  unsigned* progress;     // [links][BH][4]: tiles completed by each owner of a link
+  int* device_status;
+  int T, ntiles, BH;
+  int n_links;            // links of a head over all launches
+  int link0, cta0;        // first link / first CTA (within the head) of this launch
+  int ctas;               // CTAs of a head in this launch (a multiple of the cluster size)
+  int cs_prev;            // cluster size of the launch before (owners of link0 - 1)
+  int trigger;            // 1: let the next launch in the stream start at once
+  BlockPairs bp;
+};
+
+// ---- cluster helpers ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t raddr, float a, float b, float c, float d) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(raddr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void arrive_remote(uint32_t rbar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(rbar) : "memory");
+}
+// Bounded wait whose acquire covers writes made by other CTAs of the cluster before their arrival.
+__device__ __forceinline__ bool wait_cluster_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u32 t0, t1;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "@p bra KATA_CDONE_%=;\n\t"
+      "mov.u32 t0, %%globaltimer_lo;\n\t"
+      "KATA_CWAIT_%=:\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "@p bra KATA_CDONE_%=;\n\t"
+      "mov.u32 t1, %%globaltimer_lo;\n\t"
+      "sub.u32 t1, t1, t0;\n\t"
+      "setp.lt.u32 q, t1, %4;\n\t"
+      "@q bra KATA_CWAIT_%=;\n\t"
+      "KATA_CDONE_%=:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs), "r"(kWaitLimitNs)
+      : "memory");
+  if (ok == 0) *abort_flag = 1;
+  return ok != 0;
+}
+// Bounded wait for a progress counter in global memory (written with release by another CTA).
+__device__ __forceinline__ bool wait_progress(const unsigned* p, unsigned want, volatile int* abort_flag) {
+  unsigned v, t0, t1;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  if (v >= want) return true;
+  asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t0));
+  for (;;) {
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    if (v >= want) return true;
+    asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t1));
+    if (*abort_flag != 0 || t1 - t0 > 10u * kWaitLimitNs) {   // a producer that is not resident yet may take long
+      *abort_flag = 1;
+      return false;
+    }
+    __nanosleep(200);
+  }
+}
+
+// Shared-memory accesses of buffers that other agents refill (TMA, MMA operands, other CTAs): by address in the shared
+// window and volatile.  A plain load may be executed again later by the assembler instead of keeping its value in a
+// register (seen here: key runs re-read after the arrival that hands the tile back to the TMA producer, i.e. from the
+// next tile), and a generic-address load is not ordered with that arrival either.
+__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
+  uint4 r;
+  asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(saddr) : "memory");
+  return r;
+}
+__device__ __forceinline__ float4 lds128f(uint32_t saddr) {
+  float4 r;
+  asm volatile("ld.volatile.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(saddr) : "memory");
+  return r;
+}
+__device__ __forceinline__ float lds32f(uint32_t saddr) {
+  float r;
+  asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(r) : "r"(saddr) : "memory");
+  return r;
+}
+__device__ __forceinline__ void sts128(uint32_t saddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.volatile.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void sts16(uint32_t saddr, unsigned short v) {
+  asm volatile("st.volatile.shared.u16 [%0], %1;" ::"r"(saddr), "h"(v) : "memory");
+}
+
+// Values loaded from a buffer are kept in registers across the arrival that hands the buffer back to its producer.
+// Neither the assembler nor the hardware makes that arrival wait for loads whose results nobody has used yet (seen
+// here: key runs that came from the NEXT tile, the refill having overtaken the load), so the loaded words are folded
+// into one word that is stored before the arrival: the store cannot issue until every load has returned.
+template <int N>
+__device__ __forceinline__ void consume_before_arrive(uint32_t sink_addr, const uint32_t (&w)[N]) {
+  uint32_t x = w[0];
+#pragma unroll
+  for (int i = 1; i < N; ++i) x ^= w[i];
+  asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(sink_addr), "r"(x) : "memory");
+}
+
+// 64 products a[i] b[j] (i, j < 8) of two runs of 8 bf16 (4 words each), scaled by the bf16 pair `wgt`, as 8 chunks of
+// 8 bf16 (chunk i = a[i] * b[0..7]).  One rounding per product (the scale is 0, 1 or 2).
+__device__ __forceinline__ void products8x8(const uint32_t (&a)[4], const uint32_t (&b)[4], uint32_t wgt, uint32_t (&out)[32]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t ai = __byte_perm(a[i >> 1], 0u, (i & 1) ? 0x3232 : 0x1010);   // a[i] in both halves
+    __nv_bfloat162 s = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&ai), *reinterpret_cast<const __nv_bfloat162*>(&wgt));
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      __nv_bfloat162 pr = __hmul2(s, *reinterpret_cast<const __nv_bfloat162*>(&b[c]));
+      out[i * 4 + c] = *reinterpret_cast<uint32_t*>(&pr);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ SplitArgs args) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  auto bar = [&](int i) { return reinterpret_cast<uint64_t*>(base + OFF_BAR) + i; };
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(base + OFF_MISC);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base + OFF_MISC + 4);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t CS = cluster_nctarank(), rank = cluster_ctarank();
+  const int bh = blockIdx.x / args.ctas;
+  const int cta_launch = blockIdx.x % args.ctas;              // CTA of the head within this launch
+  const int cta_head = args.cta0 + cta_launch;                // ... within the head
+  const int link = args.link0 + cta_launch / (int)CS;
+  const bool last_link = link == args.n_links - 1;
+  const int ntiles = args.ntiles;
+  const int chunk = cta_head - 1;                             // 16-key run of every tile this CTA weighs (link 0: none)
+  const bool has_intra = chunk >= 0 && chunk < 8;
+  const int RPO = CT / (int)CS;                               // query rows of a tile this CTA owns
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    mbar_init(bar(B_K_FULL), 1);
+    mbar_init(bar(B_K_EMPTY), 256);
+    mbar_init(bar(B_K_USED), 1);
+    mbar_init(bar(B_Q_USED), 1);
+    mbar_init(bar(B_Q_FULL), 1);
+    mbar_init(bar(B_Q_EMPTY), 128);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(B_V_FULL + i), 1);
+      mbar_init(bar(B_VP_READY + i), 256);
+      mbar_init(bar(B_VP_EMPTY + i), 2);
+      mbar_init(bar(B_PSIK_FULL + i), 128);
+      mbar_init(bar(B_U_DONE + i), 1);
+      mbar_init(bar(B_S_FREE + i), 128);
+      mbar_init(bar(B_SNAP_FULL + i), 128);
+      mbar_init(bar(B_R_DONE + i), 1);
+      mbar_init(bar(B_PSIQ_FULL + i), 128);
+      mbar_init(bar(B_ACC_FULL + i), 1);
+      mbar_init(bar(B_ACC_EMPTY + i), 128);
+    }
+    mbar_init(bar(B_SC_FULL), 1);
+    mbar_init(bar(B_P_FULL), 128);
+    mbar_init(bar(B_P_FULL + 1), 128);
+    mbar_init(bar(B_RECV_FULL), 128);
+    for (int i = 0; i < 4; ++i) mbar_init(bar(B_RECV_EMPTY + i), 1);
+    mbar_init(bar(B_DRAIN), 3);
+    fence_mbar_init();
+    tma_prefetch_desc(&tmQ);
+    tma_prefetch_desc(&tmK);
+    tma_prefetch_desc(&tmV);
+  }
+  // column 64 of the B operands: zero except one bf16 per row and operand
+  const uint32_t sbase = smem_u32(base);
+  for (int i = tid; i < 1024; i += NTHREADS) sts128(sbase + OFF_COL64 + i * 16, 0u, 0u, 0u, 0u);
+  fence_async_smem();
+  if (warp == 0) {
+    tmem_alloc(tmem_base_s, TMEM_COLS);
+    tmem_relinquish();
+  }
+  if (args.trigger) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                 // every CTA's barriers exist before anything arrives on them from outside
+  tc_fence_after();
+  const uint32_t tb = *tmem_base_s;
+  bool ok = true;
+
+  if (warp == W_TMA) {
+    // =========================== TMA producer ===========================
+    if (lane == 0) {
+      for (int j = 0; j < ntiles && ok; ++j) {
+        const int b = j & 1;
+        if (j >= 1) ok = wait_or_abort(bar(B_K_EMPTY), (j - 1) & 1, abort_flag) && wait_or_abort(bar(B_K_USED), (j - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar(B_K_FULL), 16384);
+        tma_load_3d(base + OFF_KRAW, &tmK, bar(B_K_FULL), 0, j * CT, bh);
+        if (j >= 2) ok = wait_or_abort(bar(B_VP_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar(B_V_FULL + b), 16384);
+        tma_load_3d(base + OFF_VP + b * 16384, &tmV, bar(B_V_FULL + b), 0, j * CT, bh);
+        if (j >= 1) ok = wait_or_abort(bar(B_Q_EMPTY), (j - 1) & 1, abort_flag) && wait_or_abort(bar(B_Q_USED), (j - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar(B_Q_FULL), 16384);
+        tma_load_3d(base + OFF_QRAW, &tmQ, bar(B_Q_FULL), 0, j * CT, bh);
+      }
+    }
+  } else if (warp == W_U) {
+    // =========================== update issuer: S[m] += Psi(K)_m^T [V' | r] ===========================
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 80);
+      const uint64_t da = smem_desc(0, 16384, 1024, kSwizzle128B);      // second run of 64 state rows: next block pair
+      for (int j = 0; j < ntiles && ok; ++j) {
+        const int b = j & 1;
+        const uint32_t vp = smem_u32(base + OFF_VP + b * 16384);
+        const uint64_t db = smem_desc(0, smem_u32(base + OFF_COL64) + 32 * b - vp, 1024, kSwizzle128B);
+        for (int m = 0; m < 2 && ok; ++m) {
+          ok = wait_or_abort(bar(B_PSIK_FULL + m), j & 1, abort_flag);
+          if (ok && m == 0) ok = wait_or_abort(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
+          if (ok && j >= 1) ok = wait_or_abort(bar(B_S_FREE + m), (j - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t pa = smem_u32(base + OFF_PSIK + m * 32768);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+            mma_f16_ss(tb + COL_S + m * 80, at(da, pa + ks * 2048), at(db, vp + ks * 2048), idesc, (j > 0 || ks > 0) ? 1u : 0u);
+          mma_commit(bar(B_U_DONE + m));
+        }
+        if (ok) mma_commit(bar(B_VP_EMPTY + b));
+      }
+    }
+  } else if (warp == W_R) {
+    // =========================== read issuer: ACC = Psi(Q) [S | Z] (+ the intra-tile apply) ===========================
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);
+      for (int j = 0; j < ntiles && ok; ++j) {
+        const int b = j & 1;
+        if (j >= 2) ok = wait_or_abort(bar(B_ACC_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
+        for (int m = 0; m < 2 && ok; ++m) {
+          ok = wait_or_abort(bar(B_PSIQ_FULL + m), j & 1, abort_flag);
+          if (ok && j >= 1) ok = wait_or_abort(bar(B_SNAP_FULL + m), (j - 1) & 1, abort_flag);
+          if (!ok) break;
+          if (j >= 1) {
+            tc_fence_after();
+            const uint32_t sn = smem_u32(base + OFF_SNAP + m * 16384);
+            const uint64_t db = smem_desc(0, smem_u32(base + OFF_COL64) + 32 * (2 + m) - sn, 1024, kSwizzle128B);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+              mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_PSIQ + m * 64 + ks * 8, at(db, sn + ks * 2048), idesc,
+                         (m > 0 || ks > 0) ? 1u : 0u);
+          }
+          mma_commit(bar(B_R_DONE + m));
+        }
+        if (!ok) break;
+        if (has_intra) {
+          ok = wait_or_abort(bar(B_P_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t vp = smem_u32(base + OFF_VP + b * 16384);
+          const uint64_t db = smem_desc(0, smem_u32(base + OFF_COL64) + 32 * b - vp, 1024, kSwizzle128B);
+          mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_P + b * 8, at(db, vp + chunk * 2048), idesc, j >= 1 ? 1u : 0u);
+        }
+        mma_commit(bar(B_ACC_FULL + b));
+        mma_commit(bar(B_VP_EMPTY + b));
+      }
+    }
+  } else if (warp == W_I) {
+    // =========================== score issuer: Q K_c^T for this CTA's 16 keys ===========================
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 16);
+      const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
+      const uint32_t qa = smem_u32(base + OFF_QRAW), ka = smem_u32(base + OFF_KRAW) + (has_intra ? chunk : 0) * 2048;
+      for (int j = 0; j < ntiles && ok; ++j) {
+        ok = wait_or_abort(bar(B_K_FULL), j & 1, abort_flag) && wait_or_abort(bar(B_Q_FULL), j & 1, abort_flag);
+        if (ok && has_intra && j >= 1) ok = wait_or_abort(bar(B_P_FULL + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag);   // scores read
+        if (!ok) break;
+        if (has_intra) {
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            mma_f16_ss(tb + COL_SC, at(dk, qa + ks * 32), at(dk, ka + ks * 32), idesc, ks > 0 ? 1u : 0u);
+          mma_commit(bar(B_SC_FULL));
+        }
+        mma_commit(bar(B_K_USED));
+        mma_commit(bar(B_Q_USED));
+      }
+    }
+  } else if (warp < W_Q0) {
+    // =========================== key teams (thread = token, team m = accumulator tile m) ===========================
+    const int m = (warp - W_K0) >> 2;
+    const int t = ((warp - W_K0) & 3) * 32 + lane;
+    int pg[2], ph[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      pg[e] = args.bp.g[cta_head * NBP + 2 * m + e];
+      ph[e] = args.bp.h[cta_head * NBP + 2 * m + e];
+    }
+    const uint32_t kraw = sbase + OFF_KRAW;
+    for (int j = 0; j < ntiles && ok; ++j) {
+      const int b = j & 1;
+      ok = wait_or_abort(bar(B_K_FULL), j & 1, abort_flag);
+      if (!ok) break;
+      float ss = 0.f;
+      uint32_t ga[2][4], gb[2][4];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 raw = lds128(kraw + sw128_offset(t, c));
+        const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float lo = __uint_as_float(w4[e] << 16), hi = __uint_as_float(w4[e] & 0xFFFF0000u);
+          ss = fmaf(lo, lo, ss);
+          ss = fmaf(hi, hi, ss);
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const uint4 ra = lds128(kraw + sw128_offset(t, pg[e]));
+        const uint4 rb = lds128(kraw + sw128_offset(t, ph[e]));
+        ga[e][0] = ra.x; ga[e][1] = ra.y; ga[e][2] = ra.z; ga[e][3] = ra.w;
+        gb[e][0] = rb.x; gb[e][1] = rb.y; gb[e][2] = rb.z; gb[e][3] = rb.w;
+      }
+      {
+        const uint32_t held[16] = {ga[0][0], ga[0][1], ga[0][2], ga[0][3], gb[0][0], gb[0][1], gb[0][2], gb[0][3],
+                                   ga[1][0], ga[1][1], ga[1][2], ga[1][3], gb[1][0], gb[1][1], gb[1][2], gb[1][3]};
+        consume_before_arrive(sbase + OFF_SINK + tid * 4, held);
+      }
+      mbar_arrive(bar(B_K_EMPTY));
+      const float r = inv_or_zero(ss);
+      // values of this token scaled in place: team m takes 32 of the 64 columns; team 0 writes column 64
+      ok = wait_or_abort(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag);
+      if (!ok) break;
+      const uint32_t vp = sbase + OFF_VP + b * 16384;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const uint32_t p4 = vp + sw128_offset(t, 4 * m + c);
+        uint4 x = lds128(p4);
+        x.x = pack_bf16(__uint_as_float(x.x << 16) * r, __uint_as_float(x.x & 0xFFFF0000u) * r);
+        x.y = pack_bf16(__uint_as_float(x.y << 16) * r, __uint_as_float(x.y & 0xFFFF0000u) * r);
+        x.z = pack_bf16(__uint_as_float(x.z << 16) * r, __uint_as_float(x.z & 0xFFFF0000u) * r);
+        x.w = pack_bf16(__uint_as_float(x.w << 16) * r, __uint_as_float(x.w & 0xFFFF0000u) * r);
+        sts128(p4, x.x, x.y, x.z, x.w);
+      }
+      if (m == 0) sts16(sbase + OFF_COL64 + sw128_offset(t, 2 * b), __bfloat16_as_ushort(__float2bfloat16_rn(r)));
+      fence_async_smem();
+      mbar_arrive(bar(B_VP_READY + b));
+      // products of the two block pairs of accumulator tile m
+      if (j >= 1) ok = wait_or_abort(bar(B_U_DONE + m), (j - 1) & 1, abort_flag);
+      if (!ok) break;
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        uint32_t pr[32];
+        products8x8(ga[e], gb[e], 0x3F803F80u, pr);
+        const uint32_t dst = sbase + OFF_PSIK + (2 * m + e) * 16384;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sts128(dst + sw128_offset(t, i), pr[4 * i], pr[4 * i + 1], pr[4 * i + 2], pr[4 * i + 3]);
+      }
+      fence_async_smem();
+      mbar_arrive(bar(B_PSIK_FULL + m));
+    }
+  } else if (warp < W_S0) {
+    // =========================== query team (thread = token) ===========================
+    const uint32_t q4 = warp & 3;
+    const int t = q4 * 32 + lane;
+    int pg[NBP], ph[NBP];
+    uint32_t pw[NBP];
+#pragma unroll
+    for (int e = 0; e < NBP; ++e) {
+      pg[e] = args.bp.g[cta_head * NBP + e];
+      ph[e] = args.bp.h[cta_head * NBP + e];
+      const int w = args.bp.w[cta_head * NBP + e];
+      pw[e] = w == 0 ? 0u : w == 1 ? 0x3F803F80u : 0x40004000u;
+    }
+    const uint32_t qraw = sbase + OFF_QRAW;
+    for (int j = 0; j < ntiles && ok; ++j) {
+      ok = wait_or_abort(bar(B_Q_FULL), j & 1, abort_flag);
+      if (!ok) break;
+      uint32_t ga[NBP][4], gb[NBP][4];
+#pragma unroll
+      for (int e = 0; e < NBP; ++e) {
+        const uint4 ra = lds128(qraw + sw128_offset(t, pg[e]));
+        const uint4 rb = lds128(qraw + sw128_offset(t, ph[e]));
+        ga[e][0] = ra.x; ga[e][1] = ra.y; ga[e][2] = ra.z; ga[e][3] = ra.w;
+        gb[e][0] = rb.x; gb[e][1] = rb.y; gb[e][2] = rb.z; gb[e][3] = rb.w;
+      }
+      {
+        uint32_t held[8 * NBP];
+#pragma unroll
+        for (int e = 0; e < NBP; ++e)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            held[8 * e + i] = ga[e][i];
+            held[8 * e + 4 + i] = gb[e][i];
+          }
+        consume_before_arrive(sbase + OFF_SINK + tid * 4, held);
+      }
+      mbar_arrive(bar(B_Q_EMPTY));
+#pragma unroll
+      for (int m = 0; m < 2; ++m) {
+        if (j >= 1) ok = ok && wait_or_abort(bar(B_R_DONE + m), (j - 1) & 1, abort_flag);
+        if (ok) {
+          tc_fence_after();
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            uint32_t pr[32];
+            products8x8(ga[2 * m + e], gb[2 * m + e], pw[2 * m + e], pr);
+            tmem_st32(tmem_addr(tb, q4 * 32, COL_PSIQ + (2 * m + e) * 32), pr);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar(B_PSIQ_FULL + m));
+        }
+      }
+      if (!ok) break;
+    }
+  } else if (warp < W_E0) {
+    // =========================== state teams (thread = state row of accumulator tile m) ===========================
+    const int m = (warp - W_S0) >> 2;
+    const uint32_t q4 = warp & 3;
+    const int f = q4 * 32 + lane;
+    const uint32_t snap = sbase + OFF_SNAP + m * 16384;
+    for (int j = 0; j + 1 < ntiles && ok; ++j) {
+      ok = wait_or_abort(bar(B_U_DONE + m), j & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t pk[32], zc[4];
+      {
+        uint32_t y[32];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + m * 80), y);
+        tmem_wait_ld(y);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) pk[c] = pack_bf16(__uint_as_float(y[2 * c]), __uint_as_float(y[2 * c + 1]));
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + m * 80 + 32), y);
+        tmem_ld4(tmem_addr(tb, q4 * 32, COL_S + m * 80 + 64), zc);
+        tmem_wait_ld(y);
+        tmem_wait_ld(zc);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) pk[16 + c] = pack_bf16(__uint_as_float(y[2 * c]), __uint_as_float(y[2 * c + 1]));
+      }
+      tc_fence_before();
+      mbar_arrive(bar(B_S_FREE + m));
+      // the read of tile j (which uses the snapshot after tile j - 1) must be complete
+      ok = wait_or_abort(bar(B_R_DONE + m), j & 1, abort_flag);
+      if (!ok) break;
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        sts128(snap + sw128_offset(f, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+      sts16(sbase + OFF_COL64 + sw128_offset(f, 2 * (2 + m)), __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(zc[0]))));
+      fence_async_smem();
+      mbar_arrive(bar(B_SNAP_FULL + m));
+    }
+  } else {
+    // =========================== weights, share exchange, owner sums, output (thread = token) ===========================
+    const uint32_t q4 = warp & 3;
+    const int t = q4 * 32 + lane;
+    const int et = tid - W_E0 * 32;                            // 0..127
+    const uint32_t owner = (uint32_t)(t / RPO);
+    const uint32_t recv_remote = map_to_rank(smem_u32(base + OFF_RECV + (rank * RPO + (t % RPO)) * RECV_ROW), owner);
+    const uint32_t full_remote = map_to_rank(smem_u32(bar(B_RECV_FULL)), owner);
+    const size_t tpad = (size_t)ntiles * CT;
+    const float* inN = link > 0 ? args.scrN + ((size_t)(link - 1) * args.BH + bh) * tpad * 64 : nullptr;
+    const float* inD = link > 0 ? args.scrD + ((size_t)(link - 1) * args.BH + bh) * tpad : nullptr;
+    float* outN = !last_link ? args.scrN + ((size_t)link * args.BH + bh) * tpad * 64 : nullptr;
+    float* outD = !last_link ? args.scrD + ((size_t)link * args.BH + bh) * tpad : nullptr;
+    // owners of the link before: the rows this CTA owns lie inside the rows of one of them
+    const int cs_in = link > args.link0 ? (int)CS : args.cs_prev;
+    const unsigned* prog_in = link > 0 ? args.progress + ((size_t)(link - 1) * args.BH + bh) * 4 + (rank * RPO) / (CT / cs_in) : nullptr;
+    unsigned* prog_out = args.progress + ((size_t)link * args.BH + bh) * 4 + rank;
+    __nv_bfloat16* outp = args.out + (size_t)bh * args.T * D;
+
+    for (int it = 0; it < ntiles + 2 && ok; ++it) {
+      // ---- (1) weights of tile `it`: P = (Q K_c^T)^2, causal inside the tile ----
+      if (it < ntiles && has_intra) {
+        ok = wait_or_abort(bar(B_SC_FULL), it & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t y[16], pk[8];
+        tmem_ld16(tmem_addr(tb, q4 * 32, COL_SC), y);
+        tmem_wait_ld(y);
+#pragma unroll
+        for (int c = 0; c < 16; c += 2) {
+          float a = __uint_as_float(y[c]), bq = __uint_as_float(y[c + 1]);
+          a = (chunk * 16 + c <= t) ? a * a : 0.f;
+          bq = (chunk * 16 + c + 1 <= t) ? bq * bq : 0.f;
+          pk[c >> 1] = pack_bf16(a, bq);
+        }
+        tmem_st8(tmem_addr(tb, q4 * 32, COL_P + (it & 1) * 8), pk);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(B_P_FULL + (it & 1)));
+      }
+      // ---- (3) owner: sum the shares of tile it - 2, add the link before, hand on or write the output ----
+      if (it >= 2) {
+        const int j = it - 2;
+        ok = wait_cluster_or_abort(bar(B_RECV_FULL), j & 1, abort_flag);
+        if (ok && prog_in != nullptr) ok = wait_progress(prog_in, (unsigned)(j + 1), abort_flag);
+        if (!ok) break;
+        for (int item = et; item < RPO * 4; item += 128) {
+          const int row = item >> 2, qu = item & 3;            // row among the owned rows, 16 of the 64 columns
+          float acc[16], dsum = 0.f;
+#pragma unroll
+          for (int c = 0; c < 16; ++c) acc[c] = 0.f;
+          for (uint32_t s = 0; s < CS; ++s) {
+            const uint32_t src = sbase + OFF_RECV + (s * RPO + row) * RECV_ROW;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const float4 x = lds128f(src + qu * 64 + c * 16);
+              acc[4 * c] += x.x; acc[4 * c + 1] += x.y; acc[4 * c + 2] += x.z; acc[4 * c + 3] += x.w;
+            }
+            if (qu == 0) dsum += lds32f(src + 256);
+          }
+          const size_t grow = (size_t)j * CT + rank * RPO + row;      // token of the head
+          if (inN != nullptr) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const float4 x = *reinterpret_cast<const float4*>(inN + grow * 64 + qu * 16 + c * 4);
+              acc[4 * c] += x.x; acc[4 * c + 1] += x.y; acc[4 * c + 2] += x.z; acc[4 * c + 3] += x.w;
+            }
+            if (qu == 0) dsum += inD[grow];
+          }
+          if (!last_link) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              *reinterpret_cast<float4*>(outN + grow * 64 + qu * 16 + c * 4) = make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+            if (qu == 0) outD[grow] = dsum;
+          } else {
+            // the four threads of a row are neighbours in a warp: the denominator comes from the first of them
+            const float den = __shfl_sync(0xffffffffu, dsum, lane & ~3);
+            const float inv = den > 0.f ? 1.f / den : 0.f;
+            if (grow < (size_t)args.T) {
+              uint4 o0, o1;
+              o0.x = pack_bf16(acc[0] * inv, acc[1] * inv);   o0.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+              o0.z = pack_bf16(acc[4] * inv, acc[5] * inv);   o0.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+              o1.x = pack_bf16(acc[8] * inv, acc[9] * inv);   o1.y = pack_bf16(acc[10] * inv, acc[11] * inv);
+              o1.z = pack_bf16(acc[12] * inv, acc[13] * inv); o1.w = pack_bf16(acc[14] * inv, acc[15] * inv);
+              uint4* dst = reinterpret_cast<uint4*>(outp + grow * D + qu * 16);
+              dst[0] = o0;
+              dst[1] = o1;
+            }
+          }
+        }
+        if (!last_link) __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et < (int)CS) arrive_remote(map_to_rank(smem_u32(bar(B_RECV_EMPTY + rank)), (uint32_t)et));
+        if (et == 0 && !last_link) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(prog_out), "r"((unsigned)(j + 1)) : "memory");
+      }
+      // ---- (2) send this CTA's share of tile it - 1 to the owners of its rows ----
+      if (it >= 1 && it <= ntiles) {
+        const int j = it - 1, b = j & 1;
+        ok = wait_or_abort(bar(B_ACC_FULL + b), (j >> 1) & 1, abort_flag);
+        if (ok && j >= 1) ok = wait_cluster_or_abort(bar(B_RECV_EMPTY + owner), (j - 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const bool valid = has_intra || j >= 1;                  // nothing was accumulated otherwise
+        uint32_t y[32], dn[4];
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_ACC + b * 80), y);
+        tmem_wait_ld(y);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          st_cluster_v4(recv_remote + c * 16, valid ? __uint_as_float(y[4 * c]) : 0.f, valid ? __uint_as_float(y[4 * c + 1]) : 0.f,
+                        valid ? __uint_as_float(y[4 * c + 2]) : 0.f, valid ? __uint_as_float(y[4 * c + 3]) : 0.f);
+        tmem_ld32(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + 32), y);
+        tmem_ld4(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + 64), dn);
+        tmem_wait_ld(y);
+        tmem_wait_ld(dn);
+        tc_fence_before();
+        mbar_arrive(bar(B_ACC_EMPTY + b));
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          st_cluster_v4(recv_remote + 128 + c * 16, valid ? __uint_as_float(y[4 * c]) : 0.f, valid ? __uint_as_float(y[4 * c + 1]) : 0.f,
+                        valid ? __uint_as_float(y[4 * c + 2]) : 0.f, valid ? __uint_as_float(y[4 * c + 3]) : 0.f);
+        st_cluster_v4(recv_remote + 256, valid ? __uint_as_float(dn[0]) : 0.f, 0.f, 0.f, 0.f);
+        arrive_remote(full_remote);
+      }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  if (!ok && args.device_status != nullptr) atomicExch(args.device_status, (int)KATA_ERR_DEVICE_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp >= W_U && warp <= W_I && lane == 0) {
+    mma_commit(bar(B_DRAIN));
+    mbar_wait(bar(B_DRAIN), 0);
+  }
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tb, TMEM_COLS);
+  cluster_sync_all();                 // no CTA leaves while others may still write into its shared memory
+}
+
+// The 36 block pairs (g <= h) of the rank-one lift in the order they are dealt out, four to a CTA.
+void fill_block_pairs(BlockPairs& bp, int* n_ctas) {
+  int n = 0;
+  for (int g = 0; g < 8; ++g)
+    for (int h = g; h < 8; ++h) {
+      bp.g[n] = (unsigned char)g;
+      bp.h[n] = (unsigned char)h;
+      bp.w[n] = (unsigned char)(g == h ? 1 : 2);
+      ++n;
+    }
+  *n_ctas = (n + NBP - 1) / NBP;
+  for (; n < MAX_CTAS * NBP; ++n) bp.g[n] = bp.h[n] = bp.w[n] = 0;
+}
+
+constexpr int kLinks = 3;              // a single CTA, then two clusters of four
+
+}  // namespace
+
+size_t tc_split_workspace_bytes(const Problem& p) {
+  const size_t BH = (size_t)p.B * p.H, tpad = (size_t)((p.T + CT - 1) / CT) * CT;
+  return (kLinks - 1) * BH * tpad * 65 * sizeof(float) + ((kLinks * BH * 4 * sizeof(unsigned) + 255) / 256) * 256;
+}
+
+// True where 2 BH clusters of four CTAs of this kernel can be resident next to BH single CTAs is not required for
+// correctness (a link only ever waits for the link before it, which is launched or scheduled first).
+bool tc_split_supported(const Problem& p) {
+  return p.dtype == KATA_BF16 && p.d_k == 64 && p.d_v == 64 && p.feature_order == 2 && p.groups == 1;
+}
+
+void tc_chunked_split(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx) {
+  const int BH = p.B * p.H;
+  const int ntiles = (p.T + CT - 1) / CT;
+  const size_t tpad = (size_t)ntiles * CT;
+  CUtensorMap tmQ, tmK, tmV;
+  if (!make_tile_map(&tmQ, p.q, BH, p.T, CT) || !make_tile_map(&tmK, p.k, BH, p.T, CT) || !make_tile_map(&tmV, p.v, BH, p.T, CT)) {
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  if (cudaFuncSetAttribute(tc_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
+    cudaGetLastError();
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  unsigned char* w8 = static_cast<unsigned char*>(workspace);
+  const size_t prog_bytes = ((kLinks * (size_t)BH * 4 * sizeof(unsigned) + 255) / 256) * 256;
+  SplitArgs a{};
+  a.out = static_cast<__nv_bfloat16*>(p.out);
+  a.progress = reinterpret_cast<unsigned*>(w8);
+  a.scrN = reinterpret_cast<float*>(w8 + prog_bytes);
+  a.scrD = a.scrN + (size_t)(kLinks - 1) * BH * tpad * 64;
+  a.device_status = device_status;
+  a.T = p.T;
+  a.ntiles = ntiles;
+  a.BH = BH;
+  a.n_links = kLinks;
+  int n_ctas = 0;
+  fill_block_pairs(a.bp, &n_ctas);
+  if (cudaMemsetAsync(a.progress, 0, prog_bytes, ctx.stream) != cudaSuccess) {
+    cudaGetLastError();
+    ctx.status = KATA_ERR_CUDA;
+    return;
+  }
+  // launch 1: link 0, one CTA per head; launch 2: links 1 and 2, two clusters of four per head, allowed to start
+  // while launch 1 runs (it consumes what launch 1 produces tile by tile)
+  for (int launch = 0; launch < 2; ++launch) {
+    const int cs = launch == 0 ? 1 : 4;
+    a.link0 = launch == 0 ? 0 : 1;
+    a.cta0 = launch == 0 ? 0 : 1;
+    a.ctas = launch == 0 ? 1 : 8;
+    a.cs_prev = 1;
+    a.trigger = launch == 0 ? 1 : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(BH * a.ctas));
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = SMEM_ALLOC;
+    cfg.stream = ctx.stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = launch == 0 ? 1 : 2;
+    if (cudaLaunchKernelEx(&cfg, tc_split_kernel, tmQ, tmK, tmV, a) != cudaSuccess) {
+      cudaGetLastError();
+      ctx.status = KATA_ERR_CUDA;
+      return;
+    }
+    ++ctx.launches;
+  }
+}
+
+}  // namespace kata
