@@ -9,7 +9,7 @@
 // padding); nine CTAs make a head.  With k' scale r = 1/||k||^2 folded into the values (V' = r V) and the
 // normaliser carried as column 64 of every B operand, per tile of 128 tokens a CTA does
 //   update   S[m] += Psi(K)_m^T [V' | r]      A = the products, built by token threads in shared memory (MN-major),
-//                                             B = the TMA-loaded value tile scaled in place, N = 80
+//                                             B = the TMA-loaded tile of scaled values, N = 80
 //   snapshot B_m = bf16(S[m])                 TMEM -> shared memory, the B operand of the next tile's read
 //   read     ACC  = Psi(Q)_m [S | Z]_m        A = the weighted query products in TMEM, N = 80
 //   intra    ACC += P_c [V' | r]_c            P_c = (Q K_c^T)^2 masked causally for the 16 keys c of the tile this
@@ -24,9 +24,12 @@
 // Why links: a head needs nine CTAs (36 block pairs / 4), and 16 clusters of 8 or 9 CTAs do not fit the GPCs of a
 // B200 at once.  Clusters of 4 do: a head is one single CTA (link 0, its own launch) and two clusters of 4.
 //
-// Warps (896 threads): 0 TMA producer, 1 update issuer, 2 read issuer, 3 score issuer; 4-11 key teams (team m
-// builds the products of accumulator tile m; both scale the values); 12-15 query team; 16-23 state teams
-// (TMEM -> bf16 snapshot); 24-27 weights, share exchange, owner sums and output.  Every wait is bounded.
+// A light pre-pass writes V' = r V and r (bf16) once per head, so that the nine CTAs of a head load the scaled values
+// with TMA as they are.
+// Warps (896 threads): 0 TMA producer, 1 update issuer, 2 read issuer, 3 score issuer; 4-11 key teams (team m builds
+// the products of accumulator tile m; team 0 also places r); 12-15 query team; 16-19 state team (TMEM -> bf16
+// snapshot, both accumulator tiles in turn); 20-23 intra-tile weights and the exchange of shares; 24-27 owner sums,
+// link hand-off and output.  Every wait is bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cstdlib>
@@ -44,7 +47,7 @@ constexpr int D = 64;
 constexpr int CT = 128;            // tokens per tile
 constexpr int NBP = 4;             // block pairs per CTA
 constexpr int NTHREADS = 896;
-constexpr int W_TMA = 0, W_U = 1, W_R = 2, W_I = 3, W_K0 = 4, W_Q0 = 12, W_S0 = 16, W_E0 = 24;
+constexpr int W_TMA = 0, W_U = 1, W_R = 2, W_I = 3, W_K0 = 4, W_Q0 = 12, W_S0 = 16, W_E0 = 20, W_O0 = 24;
 constexpr int MAX_CTAS = 12;       // CTAs of a head over all links
 
 // ---- TMEM columns ----
@@ -67,7 +70,8 @@ constexpr uint32_t RECV_ROW = 272;
 constexpr uint32_t OFF_BAR = OFF_RECV + 128 * RECV_ROW;
 constexpr uint32_t OFF_MISC = OFF_BAR + 512;
 constexpr uint32_t OFF_SINK = OFF_MISC + 64;   // one word per thread: see consume_before_arrive
-constexpr uint32_t SMEM_BYTES = OFF_SINK + NTHREADS * 4;
+constexpr uint32_t OFF_QSTASH = OFF_SINK + NTHREADS * 4;   // 4 x 2 KB: query runs of the last two block pairs
+constexpr uint32_t SMEM_BYTES = OFF_QSTASH + 8192;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
 static_assert(SMEM_ALLOC <= 232448, "shared memory");
 
@@ -78,7 +82,7 @@ enum {
   B_Q_FULL = 2,
   B_Q_EMPTY = 3,     // ... by the 128 query threads
   B_V_FULL = 4,      // [2] value tile landed
-  B_VP_READY = 6,    // [2] values scaled, column 64 written (256 key threads)
+  B_VP_READY = 6,    // [2] column 64 of the value operand written (128 threads of key team 0)
   B_VP_EMPTY = 8,    // [2] update and intra MMAs of the tile complete
   B_PSIK_FULL = 10,  // [2] products of accumulator tile m built (128 threads)
   B_U_DONE = 12,     // [2] update of accumulator tile m complete
@@ -114,6 +118,7 @@ struct SplitArgs {
   int ctas;               // CTAs of a head in this launch (a multiple of the cluster size)
   int cs_prev;            // cluster size of the launch before (owners of link0 - 1)
   int trigger;            // 1: let the next launch in the stream start at once
+  const __nv_bfloat16* rscale;   // [BH][T] bf16: 1 / ||k||^2 (pre-pass)
   BlockPairs bp;
 };
 
@@ -226,11 +231,13 @@ __device__ __forceinline__ void consume_before_arrive(uint32_t sink_addr, const 
 
 // 64 products a[i] b[j] (i, j < 8) of two runs of 8 bf16 (4 words each), scaled by the bf16 pair `wgt`, as 8 chunks of
 // 8 bf16 (chunk i = a[i] * b[0..7]).  One rounding per product (the scale is 0, 1 or 2).
+template <bool SCALED>
 __device__ __forceinline__ void products8x8(const uint32_t (&a)[4], const uint32_t (&b)[4], uint32_t wgt, uint32_t (&out)[32]) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const uint32_t ai = __byte_perm(a[i >> 1], 0u, (i & 1) ? 0x3232 : 0x1010);   // a[i] in both halves
-    __nv_bfloat162 s = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&ai), *reinterpret_cast<const __nv_bfloat162*>(&wgt));
+    __nv_bfloat162 s = *reinterpret_cast<const __nv_bfloat162*>(&ai);
+    if (SCALED) s = __hmul2(s, *reinterpret_cast<const __nv_bfloat162*>(&wgt));
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       __nv_bfloat162 pr = __hmul2(s, *reinterpret_cast<const __nv_bfloat162*>(&b[c]));
@@ -239,6 +246,38 @@ __device__ __forceinline__ void products8x8(const uint32_t (&a)[4], const uint32
   }
 }
 
+// Pre-pass: V' = v / ||k||^2 (bf16) and r = 1 / ||k||^2 (bf16), so that the key scale is applied once per head and not
+// once in each of the nine CTAs of a head.  One warp per 4 key rows (8 lanes x 16 bytes per row).
+__global__ void __launch_bounds__(256) split_prescale_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+                                                             __nv_bfloat16* __restrict__ vs, __nv_bfloat16* __restrict__ rscale,
+                                                             size_t n_rows) {
+  const size_t row = (size_t)blockIdx.x * 32 + (threadIdx.x >> 3);
+  const int part = threadIdx.x & 7;
+  if (row >= n_rows) return;
+  const uint4 kraw = *reinterpret_cast<const uint4*>(k + row * D + part * 8);
+  const uint32_t kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
+  float ss = 0.f;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float lo = __uint_as_float(kw[e] << 16), hi = __uint_as_float(kw[e] & 0xFFFF0000u);
+    ss = fmaf(lo, lo, ss);
+    ss = fmaf(hi, hi, ss);
+  }
+  ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+  ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+  ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+  const float r2 = inv_or_zero(ss);
+  const uint4 vraw = *reinterpret_cast<const uint4*>(v + row * D + part * 8);
+  uint4 sc;
+  sc.x = pack_bf16(__uint_as_float(vraw.x << 16) * r2, __uint_as_float(vraw.x & 0xFFFF0000u) * r2);
+  sc.y = pack_bf16(__uint_as_float(vraw.y << 16) * r2, __uint_as_float(vraw.y & 0xFFFF0000u) * r2);
+  sc.z = pack_bf16(__uint_as_float(vraw.z << 16) * r2, __uint_as_float(vraw.z & 0xFFFF0000u) * r2);
+  sc.w = pack_bf16(__uint_as_float(vraw.w << 16) * r2, __uint_as_float(vraw.w & 0xFFFF0000u) * r2);
+  *reinterpret_cast<uint4*>(vs + row * D + part * 8) = sc;
+  if (part == 0) rscale[row] = __float2bfloat16_rn(r2);
+}
+
+template <int CS>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ SplitArgs args) {
@@ -249,16 +288,16 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base + OFF_MISC + 4);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t CS = cluster_nctarank(), rank = cluster_ctarank();
+  const uint32_t rank = CS == 1 ? 0u : cluster_ctarank();
   const int bh = blockIdx.x / args.ctas;
   const int cta_launch = blockIdx.x % args.ctas;              // CTA of the head within this launch
   const int cta_head = args.cta0 + cta_launch;                // ... within the head
-  const int link = args.link0 + cta_launch / (int)CS;
+  const int link = args.link0 + cta_launch / CS;
   const bool last_link = link == args.n_links - 1;
   const int ntiles = args.ntiles;
   const int chunk = cta_head - 1;                             // 16-key run of every tile this CTA weighs (link 0: none)
   const bool has_intra = chunk >= 0 && chunk < 8;
-  const int RPO = CT / (int)CS;                               // query rows of a tile this CTA owns
+  constexpr int RPO = CT / CS;                                // query rows of a tile this CTA owns
 
   if (tid == 0) {
     *abort_flag = 0;
@@ -270,7 +309,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     mbar_init(bar(B_Q_EMPTY), 128);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(B_V_FULL + i), 1);
-      mbar_init(bar(B_VP_READY + i), 256);
+      mbar_init(bar(B_VP_READY + i), 128);
       mbar_init(bar(B_VP_EMPTY + i), 2);
       mbar_init(bar(B_PSIK_FULL + i), 128);
       mbar_init(bar(B_U_DONE + i), 1);
@@ -338,7 +377,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint64_t db = smem_desc(0, smem_u32(base + OFF_COL64) + 32 * b - vp, 1024, kSwizzle128B);
         for (int m = 0; m < 2 && ok; ++m) {
           ok = wait_or_abort(bar(B_PSIK_FULL + m), j & 1, abort_flag);
-          if (ok && m == 0) ok = wait_or_abort(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
+          if (ok && m == 0) ok = wait_or_abort(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
           if (ok && j >= 1) ok = wait_or_abort(bar(B_S_FREE + m), (j - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
@@ -375,7 +414,8 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         if (!ok) break;
         if (has_intra) {
-          ok = wait_or_abort(bar(B_P_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
+          ok = wait_or_abort(bar(B_P_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag) &&
+               wait_or_abort(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint32_t vp = smem_u32(base + OFF_VP + b * 16384);
@@ -408,7 +448,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
     }
   } else if (warp < W_Q0) {
-    // =========================== key teams (thread = token, team m = accumulator tile m) ===========================
+    // =========================== key teams (thread = token; team m = accumulator tile m) ===========================
     const int m = (warp - W_K0) >> 2;
     const int t = ((warp - W_K0) & 3) * 32 + lane;
     int pg[2], ph[2];
@@ -418,23 +458,24 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       ph[e] = args.bp.h[cta_head * NBP + 2 * m + e];
     }
     const uint32_t kraw = sbase + OFF_KRAW;
+    const unsigned short* rs = reinterpret_cast<const unsigned short*>(args.rscale) + (size_t)bh * args.T;
+    unsigned short r_next = (m == 0 && t < args.T) ? rs[t] : (unsigned short)0;
     for (int j = 0; j < ntiles && ok; ++j) {
       const int b = j & 1;
+      // team 0: column 64 of the value operand (r of this token), once the tile two back is done with its copy
+      if (m == 0) {
+        const unsigned short r_now = r_next;
+        const int tn = (j + 1) * CT + t;
+        r_next = (j + 1 < ntiles && tn < args.T) ? rs[tn] : (unsigned short)0;
+        if (j >= 2) ok = wait_or_abort(bar(B_VP_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        sts16(sbase + OFF_COL64 + sw128_offset(t, 2 * b), r_now);
+        fence_async_smem();
+        mbar_arrive(bar(B_VP_READY + b));
+      }
       ok = wait_or_abort(bar(B_K_FULL), j & 1, abort_flag);
       if (!ok) break;
-      float ss = 0.f;
       uint32_t ga[2][4], gb[2][4];
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const uint4 raw = lds128(kraw + sw128_offset(t, c));
-        const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float lo = __uint_as_float(w4[e] << 16), hi = __uint_as_float(w4[e] & 0xFFFF0000u);
-          ss = fmaf(lo, lo, ss);
-          ss = fmaf(hi, hi, ss);
-        }
-      }
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         const uint4 ra = lds128(kraw + sw128_offset(t, pg[e]));
@@ -448,31 +489,13 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         consume_before_arrive(sbase + OFF_SINK + tid * 4, held);
       }
       mbar_arrive(bar(B_K_EMPTY));
-      const float r = inv_or_zero(ss);
-      // values of this token scaled in place: team m takes 32 of the 64 columns; team 0 writes column 64
-      ok = wait_or_abort(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag);
-      if (!ok) break;
-      const uint32_t vp = sbase + OFF_VP + b * 16384;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const uint32_t p4 = vp + sw128_offset(t, 4 * m + c);
-        uint4 x = lds128(p4);
-        x.x = pack_bf16(__uint_as_float(x.x << 16) * r, __uint_as_float(x.x & 0xFFFF0000u) * r);
-        x.y = pack_bf16(__uint_as_float(x.y << 16) * r, __uint_as_float(x.y & 0xFFFF0000u) * r);
-        x.z = pack_bf16(__uint_as_float(x.z << 16) * r, __uint_as_float(x.z & 0xFFFF0000u) * r);
-        x.w = pack_bf16(__uint_as_float(x.w << 16) * r, __uint_as_float(x.w & 0xFFFF0000u) * r);
-        sts128(p4, x.x, x.y, x.z, x.w);
-      }
-      if (m == 0) sts16(sbase + OFF_COL64 + sw128_offset(t, 2 * b), __bfloat16_as_ushort(__float2bfloat16_rn(r)));
-      fence_async_smem();
-      mbar_arrive(bar(B_VP_READY + b));
       // products of the two block pairs of accumulator tile m
       if (j >= 1) ok = wait_or_abort(bar(B_U_DONE + m), (j - 1) & 1, abort_flag);
       if (!ok) break;
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         uint32_t pr[32];
-        products8x8(ga[e], gb[e], 0x3F803F80u, pr);
+        products8x8<false>(ga[e], gb[e], 0u, pr);
         const uint32_t dst = sbase + OFF_PSIK + (2 * m + e) * 16384;
 #pragma unroll
         for (int i = 0; i < 8; ++i) sts128(dst + sw128_offset(t, i), pr[4 * i], pr[4 * i + 1], pr[4 * i + 2], pr[4 * i + 3]);
@@ -494,38 +517,47 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       pw[e] = w == 0 ? 0u : w == 1 ? 0x3F803F80u : 0x40004000u;
     }
     const uint32_t qraw = sbase + OFF_QRAW;
+    const uint32_t stash = sbase + OFF_QSTASH + (tid - W_Q0 * 32) * 16;   // 4 runs of 16 bytes, 2 KB apart (conflict-free)
     for (int j = 0; j < ntiles && ok; ++j) {
       ok = wait_or_abort(bar(B_Q_FULL), j & 1, abort_flag);
       if (!ok) break;
-      uint32_t ga[NBP][4], gb[NBP][4];
+      // the runs of the first two block pairs stay in registers, those of the last two wait in a private stash
+      uint32_t ga[2][4], gb[2][4];
 #pragma unroll
-      for (int e = 0; e < NBP; ++e) {
+      for (int e = 0; e < 2; ++e) {
         const uint4 ra = lds128(qraw + sw128_offset(t, pg[e]));
         const uint4 rb = lds128(qraw + sw128_offset(t, ph[e]));
         ga[e][0] = ra.x; ga[e][1] = ra.y; ga[e][2] = ra.z; ga[e][3] = ra.w;
         gb[e][0] = rb.x; gb[e][1] = rb.y; gb[e][2] = rb.z; gb[e][3] = rb.w;
+        const uint4 sa = lds128(qraw + sw128_offset(t, pg[2 + e]));
+        const uint4 sb = lds128(qraw + sw128_offset(t, ph[2 + e]));
+        sts128(stash + (2 * e) * 2048, sa.x, sa.y, sa.z, sa.w);
+        sts128(stash + (2 * e + 1) * 2048, sb.x, sb.y, sb.z, sb.w);
       }
       {
-        uint32_t held[8 * NBP];
-#pragma unroll
-        for (int e = 0; e < NBP; ++e)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            held[8 * e + i] = ga[e][i];
-            held[8 * e + 4 + i] = gb[e][i];
-          }
+        const uint32_t held[16] = {ga[0][0], ga[0][1], ga[0][2], ga[0][3], gb[0][0], gb[0][1], gb[0][2], gb[0][3],
+                                   ga[1][0], ga[1][1], ga[1][2], ga[1][3], gb[1][0], gb[1][1], gb[1][2], gb[1][3]};
         consume_before_arrive(sbase + OFF_SINK + tid * 4, held);
       }
       mbar_arrive(bar(B_Q_EMPTY));
 #pragma unroll
       for (int m = 0; m < 2; ++m) {
+        if (m == 1) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const uint4 ra = lds128(stash + (2 * e) * 2048);
+            const uint4 rb = lds128(stash + (2 * e + 1) * 2048);
+            ga[e][0] = ra.x; ga[e][1] = ra.y; ga[e][2] = ra.z; ga[e][3] = ra.w;
+            gb[e][0] = rb.x; gb[e][1] = rb.y; gb[e][2] = rb.z; gb[e][3] = rb.w;
+          }
+        }
         if (j >= 1) ok = ok && wait_or_abort(bar(B_R_DONE + m), (j - 1) & 1, abort_flag);
         if (ok) {
           tc_fence_after();
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
             uint32_t pr[32];
-            products8x8(ga[2 * m + e], gb[2 * m + e], pw[2 * m + e], pr);
+            products8x8<true>(ga[e], gb[e], pw[2 * m + e], pr);
             tmem_st32(tmem_addr(tb, q4 * 32, COL_PSIQ + (2 * m + e) * 32), pr);
           }
           tmem_wait_st();
@@ -536,62 +568,49 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (!ok) break;
     }
   } else if (warp < W_E0) {
-    // =========================== state teams (thread = state row of accumulator tile m) ===========================
-    const int m = (warp - W_S0) >> 2;
+    // =========================== state team (thread = state row; both accumulator tiles in turn) ===========================
     const uint32_t q4 = warp & 3;
     const int f = q4 * 32 + lane;
-    const uint32_t snap = sbase + OFF_SNAP + m * 16384;
     for (int j = 0; j + 1 < ntiles && ok; ++j) {
-      ok = wait_or_abort(bar(B_U_DONE + m), j & 1, abort_flag);
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t pk[32], zc[4];
-      {
-        uint32_t y[32];
-        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + m * 80), y);
-        tmem_wait_ld(y);
+#pragma unroll 1
+      for (int m = 0; m < 2 && ok; ++m) {
+        ok = wait_or_abort(bar(B_U_DONE + m), j & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t pk[32], zc[4];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) pk[c] = pack_bf16(__uint_as_float(y[2 * c]), __uint_as_float(y[2 * c + 1]));
-        tmem_ld32(tmem_addr(tb, q4 * 32, COL_S + m * 80 + 32), y);
-        tmem_ld4(tmem_addr(tb, q4 * 32, COL_S + m * 80 + 64), zc);
-        tmem_wait_ld(y);
+        for (int h = 0; h < 4; ++h) {
+          uint32_t y[16];
+          tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + m * 80 + h * 16), y);
+          if (h == 3) tmem_ld4(tmem_addr(tb, q4 * 32, COL_S + m * 80 + 64), zc);
+          tmem_wait_ld(y);
+#pragma unroll
+          for (int c = 0; c < 8; ++c) pk[h * 8 + c] = pack_bf16(__uint_as_float(y[2 * c]), __uint_as_float(y[2 * c + 1]));
+        }
         tmem_wait_ld(zc);
+        tc_fence_before();
+        mbar_arrive(bar(B_S_FREE + m));
+        // the read of tile j (which uses the snapshot after tile j - 1) must be complete
+        ok = wait_or_abort(bar(B_R_DONE + m), j & 1, abort_flag);
+        if (!ok) break;
+        const uint32_t snap = sbase + OFF_SNAP + m * 16384;
 #pragma unroll
-        for (int c = 0; c < 16; ++c) pk[16 + c] = pack_bf16(__uint_as_float(y[2 * c]), __uint_as_float(y[2 * c + 1]));
+        for (int c = 0; c < 8; ++c) sts128(snap + sw128_offset(f, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        sts16(sbase + OFF_COL64 + sw128_offset(f, 2 * (2 + m)), __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(zc[0]))));
+        fence_async_smem();
+        mbar_arrive(bar(B_SNAP_FULL + m));
       }
-      tc_fence_before();
-      mbar_arrive(bar(B_S_FREE + m));
-      // the read of tile j (which uses the snapshot after tile j - 1) must be complete
-      ok = wait_or_abort(bar(B_R_DONE + m), j & 1, abort_flag);
-      if (!ok) break;
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        sts128(snap + sw128_offset(f, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-      sts16(sbase + OFF_COL64 + sw128_offset(f, 2 * (2 + m)), __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(zc[0]))));
-      fence_async_smem();
-      mbar_arrive(bar(B_SNAP_FULL + m));
     }
-  } else {
-    // =========================== weights, share exchange, owner sums, output (thread = token) ===========================
+  } else if (warp < W_O0) {
+    // =========================== intra-tile weights and the exchange of shares (thread = token) ===========================
     const uint32_t q4 = warp & 3;
     const int t = q4 * 32 + lane;
-    const int et = tid - W_E0 * 32;                            // 0..127
     const uint32_t owner = (uint32_t)(t / RPO);
-    const uint32_t recv_remote = map_to_rank(smem_u32(base + OFF_RECV + (rank * RPO + (t % RPO)) * RECV_ROW), owner);
-    const uint32_t full_remote = map_to_rank(smem_u32(bar(B_RECV_FULL)), owner);
-    const size_t tpad = (size_t)ntiles * CT;
-    const float* inN = link > 0 ? args.scrN + ((size_t)(link - 1) * args.BH + bh) * tpad * 64 : nullptr;
-    const float* inD = link > 0 ? args.scrD + ((size_t)(link - 1) * args.BH + bh) * tpad : nullptr;
-    float* outN = !last_link ? args.scrN + ((size_t)link * args.BH + bh) * tpad * 64 : nullptr;
-    float* outD = !last_link ? args.scrD + ((size_t)link * args.BH + bh) * tpad : nullptr;
-    // owners of the link before: the rows this CTA owns lie inside the rows of one of them
-    const int cs_in = link > args.link0 ? (int)CS : args.cs_prev;
-    const unsigned* prog_in = link > 0 ? args.progress + ((size_t)(link - 1) * args.BH + bh) * 4 + (rank * RPO) / (CT / cs_in) : nullptr;
-    unsigned* prog_out = args.progress + ((size_t)link * args.BH + bh) * 4 + rank;
-    __nv_bfloat16* outp = args.out + (size_t)bh * args.T * D;
-
-    for (int it = 0; it < ntiles + 2 && ok; ++it) {
-      // ---- (1) weights of tile `it`: P = (Q K_c^T)^2, causal inside the tile ----
+    const uint32_t recv_local = sbase + OFF_RECV + (rank * RPO + (t % RPO)) * RECV_ROW;
+    const uint32_t recv_remote = CS == 1 ? recv_local : map_to_rank(recv_local, owner);
+    const uint32_t full_remote = CS == 1 ? smem_u32(bar(B_RECV_FULL)) : map_to_rank(smem_u32(bar(B_RECV_FULL)), owner);
+    for (int it = 0; it <= ntiles && ok; ++it) {
+      // ---- weights of tile `it`: P = (Q K_c^T)^2, causal inside the tile ----
       if (it < ntiles && has_intra) {
         ok = wait_or_abort(bar(B_SC_FULL), it & 1, abort_flag);
         if (!ok) break;
@@ -611,28 +630,90 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tc_fence_before();
         mbar_arrive(bar(B_P_FULL + (it & 1)));
       }
-      // ---- (3) owner: sum the shares of tile it - 2, add the link before, hand on or write the output ----
-      if (it >= 2) {
-        const int j = it - 2;
-        ok = wait_cluster_or_abort(bar(B_RECV_FULL), j & 1, abort_flag);
-        if (ok && prog_in != nullptr) ok = wait_progress(prog_in, (unsigned)(j + 1), abort_flag);
+      // ---- this CTA's share of tile it - 1 goes to the owners of its rows ----
+      if (it >= 1) {
+        const int j = it - 1, b = j & 1;
+        ok = wait_or_abort(bar(B_ACC_FULL + b), (j >> 1) & 1, abort_flag);
+        if (ok && j >= 1) ok = wait_cluster_or_abort(bar(B_RECV_EMPTY + owner), (j - 1) & 1, abort_flag);
         if (!ok) break;
-        for (int item = et; item < RPO * 4; item += 128) {
-          const int row = item >> 2, qu = item & 3;            // row among the owned rows, 16 of the 64 columns
-          float acc[16], dsum = 0.f;
+        tc_fence_after();
+        const bool valid = has_intra || j >= 1;                  // nothing was accumulated otherwise
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+          uint32_t y[32];
+          tmem_ld32(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + h * 32), y);
+          tmem_wait_ld(y);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) acc[c] = 0.f;
-          for (uint32_t s = 0; s < CS; ++s) {
-            const uint32_t src = sbase + OFF_RECV + (s * RPO + row) * RECV_ROW;
+          for (int c = 0; c < 8; ++c)
+            st_cluster_v4(recv_remote + h * 128 + c * 16, valid ? __uint_as_float(y[4 * c]) : 0.f, valid ? __uint_as_float(y[4 * c + 1]) : 0.f,
+                          valid ? __uint_as_float(y[4 * c + 2]) : 0.f, valid ? __uint_as_float(y[4 * c + 3]) : 0.f);
+        }
+        uint32_t dn[4];
+        tmem_ld4(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + 64), dn);
+        tmem_wait_ld(dn);
+        tc_fence_before();
+        mbar_arrive(bar(B_ACC_EMPTY + b));
+        st_cluster_v4(recv_remote + 256, valid ? __uint_as_float(dn[0]) : 0.f, 0.f, 0.f, 0.f);
+        if (CS == 1) mbar_arrive(bar(B_RECV_FULL)); else arrive_remote(full_remote);
+      }
+    }
+  } else {
+    // =========================== owner: sums of the shares, link hand-off, output ===========================
+    const int et = tid - W_O0 * 32;                            // 0..127
+    const size_t tpad = (size_t)ntiles * CT;
+    const float* inN = link > 0 ? args.scrN + ((size_t)(link - 1) * args.BH + bh) * tpad * 64 : nullptr;
+    const float* inD = link > 0 ? args.scrD + ((size_t)(link - 1) * args.BH + bh) * tpad : nullptr;
+    float* outN = !last_link ? args.scrN + ((size_t)link * args.BH + bh) * tpad * 64 : nullptr;
+    float* outD = !last_link ? args.scrD + ((size_t)link * args.BH + bh) * tpad : nullptr;
+    // owners of the link before: the rows this CTA owns lie inside the rows of one of them
+    const int cs_in = link > args.link0 ? CS : args.cs_prev;
+    const unsigned* prog_in = link > 0 ? args.progress + ((size_t)(link - 1) * args.BH + bh) * 4 + (rank * RPO) / (CT / cs_in) : nullptr;
+    unsigned* prog_out = args.progress + ((size_t)link * args.BH + bh) * 4 + rank;
+    __nv_bfloat16* outp = args.out + (size_t)bh * args.T * D;
+    constexpr int N_ITEMS = RPO * 4 / 128;                     // (row, 16 columns) items per thread: 1 (clusters of 4) or 4
+    // what the link before left for the first item of the next tile, fetched one tile ahead
+    float4 pre[4];
+    float pre_d = 0.f;
+    auto prefetch = [&](int j) {
+      const int row = et >> 2, qu = et & 3;
+      const size_t grow = (size_t)j * CT + rank * RPO + row;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) pre[c] = *reinterpret_cast<const float4*>(inN + grow * 64 + qu * 16 + c * 4);
+      if (qu == 0) pre_d = inD[grow];
+    };
+    if (inN != nullptr && ntiles > 0) {
+      ok = wait_progress(prog_in, 1u, abort_flag);
+      if (ok) prefetch(0);
+    }
+    for (int j = 0; j < ntiles && ok; ++j) {
+      ok = wait_cluster_or_abort(bar(B_RECV_FULL), j & 1, abort_flag);
+      if (!ok) break;
+#pragma unroll 1
+      for (int k = 0; k < N_ITEMS; ++k) {
+        const int item = et + k * 128;
+        const int row = item >> 2, qu = item & 3;              // row among the owned rows, 16 of the 64 columns
+        float acc[16], dsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) acc[c] = 0.f;
+#pragma unroll
+        for (int s = 0; s < CS; ++s) {
+          const uint32_t src = sbase + OFF_RECV + (s * RPO + row) * RECV_ROW;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const float4 x = lds128f(src + qu * 64 + c * 16);
+            acc[4 * c] += x.x; acc[4 * c + 1] += x.y; acc[4 * c + 2] += x.z; acc[4 * c + 3] += x.w;
+          }
+          if (qu == 0) dsum += lds32f(src + 256);
+        }
+        const size_t grow = (size_t)j * CT + rank * RPO + row;      // token of the head
+        if (inN != nullptr) {
+          if (k == 0) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-              const float4 x = lds128f(src + qu * 64 + c * 16);
-              acc[4 * c] += x.x; acc[4 * c + 1] += x.y; acc[4 * c + 2] += x.z; acc[4 * c + 3] += x.w;
+              acc[4 * c] += pre[c].x; acc[4 * c + 1] += pre[c].y; acc[4 * c + 2] += pre[c].z; acc[4 * c + 3] += pre[c].w;
             }
-            if (qu == 0) dsum += lds32f(src + 256);
-          }
-          const size_t grow = (size_t)j * CT + rank * RPO + row;      // token of the head
-          if (inN != nullptr) {
+            if (qu == 0) dsum += pre_d;
+          } else {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               const float4 x = *reinterpret_cast<const float4*>(inN + grow * 64 + qu * 16 + c * 4);
@@ -640,59 +721,42 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
             if (qu == 0) dsum += inD[grow];
           }
-          if (!last_link) {
+        }
+        if (!last_link) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-              *reinterpret_cast<float4*>(outN + grow * 64 + qu * 16 + c * 4) = make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
-            if (qu == 0) outD[grow] = dsum;
-          } else {
-            // the four threads of a row are neighbours in a warp: the denominator comes from the first of them
-            const float den = __shfl_sync(0xffffffffu, dsum, lane & ~3);
-            const float inv = den > 0.f ? 1.f / den : 0.f;
-            if (grow < (size_t)args.T) {
-              uint4 o0, o1;
-              o0.x = pack_bf16(acc[0] * inv, acc[1] * inv);   o0.y = pack_bf16(acc[2] * inv, acc[3] * inv);
-              o0.z = pack_bf16(acc[4] * inv, acc[5] * inv);   o0.w = pack_bf16(acc[6] * inv, acc[7] * inv);
-              o1.x = pack_bf16(acc[8] * inv, acc[9] * inv);   o1.y = pack_bf16(acc[10] * inv, acc[11] * inv);
-              o1.z = pack_bf16(acc[12] * inv, acc[13] * inv); o1.w = pack_bf16(acc[14] * inv, acc[15] * inv);
-              uint4* dst = reinterpret_cast<uint4*>(outp + grow * D + qu * 16);
-              dst[0] = o0;
-              dst[1] = o1;
-            }
+          for (int c = 0; c < 4; ++c)
+            *reinterpret_cast<float4*>(outN + grow * 64 + qu * 16 + c * 4) = make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+          if (qu == 0) outD[grow] = dsum;
+        } else {
+          // the four threads of a row are neighbours in a warp: the denominator comes from the first of them
+          const float den = __shfl_sync(0xffffffffu, dsum, lane & ~3);
+          const float inv = den > 0.f ? 1.f / den : 0.f;
+          if (grow < (size_t)args.T) {
+            uint4 o0, o1;
+            o0.x = pack_bf16(acc[0] * inv, acc[1] * inv);   o0.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+            o0.z = pack_bf16(acc[4] * inv, acc[5] * inv);   o0.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+            o1.x = pack_bf16(acc[8] * inv, acc[9] * inv);   o1.y = pack_bf16(acc[10] * inv, acc[11] * inv);
+            o1.z = pack_bf16(acc[12] * inv, acc[13] * inv); o1.w = pack_bf16(acc[14] * inv, acc[15] * inv);
+            uint4* dst = reinterpret_cast<uint4*>(outp + grow * D + qu * 16);
+            dst[0] = o0;
+            dst[1] = o1;
           }
         }
-        if (!last_link) __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (et < (int)CS) arrive_remote(map_to_rank(smem_u32(bar(B_RECV_EMPTY + rank)), (uint32_t)et));
-        if (et == 0 && !last_link) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(prog_out), "r"((unsigned)(j + 1)) : "memory");
       }
-      // ---- (2) send this CTA's share of tile it - 1 to the owners of its rows ----
-      if (it >= 1 && it <= ntiles) {
-        const int j = it - 1, b = j & 1;
-        ok = wait_or_abort(bar(B_ACC_FULL + b), (j >> 1) & 1, abort_flag);
-        if (ok && j >= 1) ok = wait_cluster_or_abort(bar(B_RECV_EMPTY + owner), (j - 1) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const bool valid = has_intra || j >= 1;                  // nothing was accumulated otherwise
-        uint32_t y[32], dn[4];
-        tmem_ld32(tmem_addr(tb, q4 * 32, COL_ACC + b * 80), y);
-        tmem_wait_ld(y);
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-          st_cluster_v4(recv_remote + c * 16, valid ? __uint_as_float(y[4 * c]) : 0.f, valid ? __uint_as_float(y[4 * c + 1]) : 0.f,
-                        valid ? __uint_as_float(y[4 * c + 2]) : 0.f, valid ? __uint_as_float(y[4 * c + 3]) : 0.f);
-        tmem_ld32(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + 32), y);
-        tmem_ld4(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + 64), dn);
-        tmem_wait_ld(y);
-        tmem_wait_ld(dn);
-        tc_fence_before();
-        mbar_arrive(bar(B_ACC_EMPTY + b));
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-          st_cluster_v4(recv_remote + 128 + c * 16, valid ? __uint_as_float(y[4 * c]) : 0.f, valid ? __uint_as_float(y[4 * c + 1]) : 0.f,
-                        valid ? __uint_as_float(y[4 * c + 2]) : 0.f, valid ? __uint_as_float(y[4 * c + 3]) : 0.f);
-        st_cluster_v4(recv_remote + 256, valid ? __uint_as_float(dn[0]) : 0.f, 0.f, 0.f, 0.f);
-        arrive_remote(full_remote);
+      // every thread of the team has read its shares (and written its rows): the senders may refill the buffer,
+      // and one thread publishes the tile to the next link (its release covers the team's writes, which the
+      // barrier orders before it)
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (et < CS) {
+        if (CS == 1) mbar_arrive(bar(B_RECV_EMPTY)); else arrive_remote(map_to_rank(smem_u32(bar(B_RECV_EMPTY + rank)), (uint32_t)et));
+      }
+      if (et == 0 && !last_link) {
+        __threadfence();
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(prog_out), "r"((unsigned)(j + 1)) : "memory");
+      }
+      if (inN != nullptr && j + 1 < ntiles) {
+        ok = wait_progress(prog_in, (unsigned)(j + 2), abort_flag);
+        if (ok) prefetch(j + 1);
       }
     }
   }
@@ -729,13 +793,15 @@ constexpr int kLinks = 3;              // a single CTA, then two clusters of fou
 
 }  // namespace
 
+static size_t al256(size_t x) { return (x + 255) / 256 * 256; }
+
+// workspace: progress counters | V' [BH][T][64] bf16 | r [BH][T] bf16 | N scratch [links - 1][BH][Tpad][64] fp32 | D scratch
 size_t tc_split_workspace_bytes(const Problem& p) {
   const size_t BH = (size_t)p.B * p.H, tpad = (size_t)((p.T + CT - 1) / CT) * CT;
-  return (kLinks - 1) * BH * tpad * 65 * sizeof(float) + ((kLinks * BH * 4 * sizeof(unsigned) + 255) / 256) * 256;
+  return al256(kLinks * BH * 4 * sizeof(unsigned)) + al256(BH * p.T * D * 2) + al256(BH * p.T * 2) +
+         (kLinks - 1) * BH * tpad * 65 * sizeof(float);
 }
 
-// True where 2 BH clusters of four CTAs of this kernel can be resident next to BH single CTAs is not required for
-// correctness (a link only ever waits for the link before it, which is launched or scheduled first).
 bool tc_split_supported(const Problem& p) {
   return p.dtype == KATA_BF16 && p.d_k == 64 && p.d_v == 64 && p.feature_order == 2 && p.groups == 1;
 }
@@ -744,23 +810,28 @@ void tc_chunked_split(const Problem& p, void* workspace, int* device_status, Lau
   const int BH = p.B * p.H;
   const int ntiles = (p.T + CT - 1) / CT;
   const size_t tpad = (size_t)ntiles * CT;
+  unsigned char* w8 = static_cast<unsigned char*>(workspace);
+  const size_t prog_bytes = al256(kLinks * (size_t)BH * 4 * sizeof(unsigned));
+  __nv_bfloat16* vs = reinterpret_cast<__nv_bfloat16*>(w8 + prog_bytes);
+  __nv_bfloat16* rscale = reinterpret_cast<__nv_bfloat16*>(w8 + prog_bytes + al256((size_t)BH * p.T * D * 2));
+  float* scr = reinterpret_cast<float*>(w8 + prog_bytes + al256((size_t)BH * p.T * D * 2) + al256((size_t)BH * p.T * 2));
   CUtensorMap tmQ, tmK, tmV;
-  if (!make_tile_map(&tmQ, p.q, BH, p.T, CT) || !make_tile_map(&tmK, p.k, BH, p.T, CT) || !make_tile_map(&tmV, p.v, BH, p.T, CT)) {
+  if (!make_tile_map(&tmQ, p.q, BH, p.T, CT) || !make_tile_map(&tmK, p.k, BH, p.T, CT) || !make_tile_map(&tmV, vs, BH, p.T, CT)) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-  if (cudaFuncSetAttribute(tc_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
+  if (cudaFuncSetAttribute(tc_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_split_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
     cudaGetLastError();
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-  unsigned char* w8 = static_cast<unsigned char*>(workspace);
-  const size_t prog_bytes = ((kLinks * (size_t)BH * 4 * sizeof(unsigned) + 255) / 256) * 256;
   SplitArgs a{};
   a.out = static_cast<__nv_bfloat16*>(p.out);
   a.progress = reinterpret_cast<unsigned*>(w8);
-  a.scrN = reinterpret_cast<float*>(w8 + prog_bytes);
-  a.scrD = a.scrN + (size_t)(kLinks - 1) * BH * tpad * 64;
+  a.scrN = scr;
+  a.scrD = scr + (size_t)(kLinks - 1) * BH * tpad * 64;
+  a.rscale = rscale;
   a.device_status = device_status;
   a.T = p.T;
   a.ntiles = ntiles;
@@ -773,6 +844,10 @@ void tc_chunked_split(const Problem& p, void* workspace, int* device_status, Lau
     ctx.status = KATA_ERR_CUDA;
     return;
   }
+  const size_t n_rows = (size_t)BH * p.T;
+  split_prescale_kernel<<<(unsigned)((n_rows + 31) / 32), 256, 0, ctx.stream>>>(
+      static_cast<const __nv_bfloat16*>(p.k), static_cast<const __nv_bfloat16*>(p.v), vs, rscale, n_rows);
+  note_launch(ctx);
   // launch 1: link 0, one CTA per head; launch 2: links 1 and 2, two clusters of four per head, allowed to start
   // while launch 1 runs (it consumes what launch 1 produces tile by tile)
   for (int launch = 0; launch < 2; ++launch) {
@@ -796,7 +871,9 @@ void tc_chunked_split(const Problem& p, void* workspace, int* device_status, Lau
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = launch == 0 ? 1 : 2;
-    if (cudaLaunchKernelEx(&cfg, tc_split_kernel, tmQ, tmK, tmV, a) != cudaSuccess) {
+    const cudaError_t err = launch == 0 ? cudaLaunchKernelEx(&cfg, tc_split_kernel<1>, tmQ, tmK, tmV, a)
+                                        : cudaLaunchKernelEx(&cfg, tc_split_kernel<4>, tmQ, tmK, tmV, a);
+    if (err != cudaSuccess) {
       cudaGetLastError();
       ctx.status = KATA_ERR_CUDA;
       return;
