@@ -49,6 +49,7 @@ constexpr int NBP = 4;             // block pairs per CTA
 constexpr int NTHREADS = 896;
 constexpr int W_TMA = 0, W_U = 1, W_R = 2, W_I = 3, W_K0 = 4, W_Q0 = 12, W_S0 = 16, W_E0 = 20, W_O0 = 24;
 constexpr int MAX_CTAS = 12;       // CTAs of a head over all links
+constexpr int kPublish = 8;        // tiles between two publications of a link's progress
 
 // ---- TMEM columns ----
 constexpr uint32_t COL_S = 0;      // 2 x 80: state tiles (lanes = state rows)
@@ -147,28 +148,26 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t raddr, float a, float b, 
 __device__ __forceinline__ void arrive_remote(uint32_t rbar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(rbar) : "memory");
 }
-// Bounded wait whose acquire covers writes made by other CTAs of the cluster before their arrival.
+// Bounded wait whose acquire covers writes made by other CTAs of the cluster before their arrival.  Bounded by a
+// poll count (hint 1 us per poll): reading the global timer after a failed first try costs more than most waits last.
 __device__ __forceinline__ bool wait_cluster_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   uint32_t ok;
   asm volatile(
       "{\n\t"
       ".reg .pred p, q;\n\t"
-      ".reg .u32 t0, t1;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "@p bra KATA_CDONE_%=;\n\t"
-      "mov.u32 t0, %%globaltimer_lo;\n\t"
+      ".reg .u32 i;\n\t"
+      "mov.u32 i, 0;\n\t"
       "KATA_CWAIT_%=:\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, 1000;\n\t"
       "@p bra KATA_CDONE_%=;\n\t"
-      "mov.u32 t1, %%globaltimer_lo;\n\t"
-      "sub.u32 t1, t1, t0;\n\t"
-      "setp.lt.u32 q, t1, %4;\n\t"
+      "add.u32 i, i, 1;\n\t"
+      "setp.lt.u32 q, i, %3;\n\t"
       "@q bra KATA_CWAIT_%=;\n\t"
       "KATA_CDONE_%=:\n\t"
       "selp.u32 %0, 1, 0, p;\n\t"
       "}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs), "r"(kWaitLimitNs)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSpinLimit)
       : "memory");
   if (ok == 0) *abort_flag = 1;
   return ok != 0;
@@ -192,29 +191,28 @@ __device__ __forceinline__ bool wait_progress(const unsigned* p, unsigned want, 
 }
 
 // Shared-memory accesses of buffers that other agents refill (TMA, MMA operands, other CTAs): by address in the shared
-// window and volatile.  A plain load may be executed again later by the assembler instead of keeping its value in a
-// register (seen here: key runs re-read after the arrival that hands the tile back to the TMA producer, i.e. from the
-// next tile), and a generic-address load is not ordered with that arrival either.
+// window (a generic-address load is not ordered with the mbarrier arrival that hands the buffer back).  Not volatile:
+// a volatile shared access costs a round trip each (measured: ten times the time of the same code with weak accesses).
 __device__ __forceinline__ uint4 lds128(uint32_t saddr) {
   uint4 r;
-  asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(saddr) : "memory");
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(saddr) : "memory");
   return r;
 }
 __device__ __forceinline__ float4 lds128f(uint32_t saddr) {
   float4 r;
-  asm volatile("ld.volatile.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(saddr) : "memory");
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(saddr) : "memory");
   return r;
 }
 __device__ __forceinline__ float lds32f(uint32_t saddr) {
   float r;
-  asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(r) : "r"(saddr) : "memory");
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(r) : "r"(saddr) : "memory");
   return r;
 }
 __device__ __forceinline__ void sts128(uint32_t saddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.volatile.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ void sts16(uint32_t saddr, unsigned short v) {
-  asm volatile("st.volatile.shared.u16 [%0], %1;" ::"r"(saddr), "h"(v) : "memory");
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(saddr), "h"(v) : "memory");
 }
 
 // Values loaded from a buffer are kept in registers across the arrival that hands the buffer back to its producer.
@@ -226,8 +224,14 @@ __device__ __forceinline__ void consume_before_arrive(uint32_t sink_addr, const 
   uint32_t x = w[0];
 #pragma unroll
   for (int i = 1; i < N; ++i) x ^= w[i];
-  asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(sink_addr), "r"(x) : "memory");
+  asm volatile("st.shared.u32 [%0], %1;" ::"r"(sink_addr), "r"(x) : "memory");
 }
+
+// Register budget per warp group (the kernel is launched with 72 registers per thread for 896 threads): the four
+// issuer warps and the key teams give registers up, the teams that hold tiles of TMEM in registers take them.
+template <int N> __device__ __forceinline__ void regs_release() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void regs_take() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+static_assert(128 * 40 + 256 * 56 + 512 * 88 <= 896 * 72, "register budget");
 
 // 64 products a[i] b[j] (i, j < 8) of two runs of 8 bf16 (4 words each), scaled by the bf16 pair `wgt`, as 8 chunks of
 // 8 bf16 (chunk i = a[i] * b[0..7]).  One rounding per product (the scale is 0, 1 or 2).
@@ -347,20 +351,22 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t tb = *tmem_base_s;
   bool ok = true;
 
+  if (warp < W_K0) {
+  regs_release<40>();
   if (warp == W_TMA) {
     // =========================== TMA producer ===========================
     if (lane == 0) {
       for (int j = 0; j < ntiles && ok; ++j) {
         const int b = j & 1;
-        if (j >= 1) ok = wait_or_abort(bar(B_K_EMPTY), (j - 1) & 1, abort_flag) && wait_or_abort(bar(B_K_USED), (j - 1) & 1, abort_flag);
+        if (j >= 1) ok = wait_or_abort_counted(bar(B_K_EMPTY), (j - 1) & 1, abort_flag) && wait_or_abort_counted(bar(B_K_USED), (j - 1) & 1, abort_flag);
         if (!ok) break;
         mbar_arrive_expect_tx(bar(B_K_FULL), 16384);
         tma_load_3d(base + OFF_KRAW, &tmK, bar(B_K_FULL), 0, j * CT, bh);
-        if (j >= 2) ok = wait_or_abort(bar(B_VP_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
+        if (j >= 2) ok = wait_or_abort_counted(bar(B_VP_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
         if (!ok) break;
         mbar_arrive_expect_tx(bar(B_V_FULL + b), 16384);
         tma_load_3d(base + OFF_VP + b * 16384, &tmV, bar(B_V_FULL + b), 0, j * CT, bh);
-        if (j >= 1) ok = wait_or_abort(bar(B_Q_EMPTY), (j - 1) & 1, abort_flag) && wait_or_abort(bar(B_Q_USED), (j - 1) & 1, abort_flag);
+        if (j >= 1) ok = wait_or_abort_counted(bar(B_Q_EMPTY), (j - 1) & 1, abort_flag) && wait_or_abort_counted(bar(B_Q_USED), (j - 1) & 1, abort_flag);
         if (!ok) break;
         mbar_arrive_expect_tx(bar(B_Q_FULL), 16384);
         tma_load_3d(base + OFF_QRAW, &tmQ, bar(B_Q_FULL), 0, j * CT, bh);
@@ -376,9 +382,9 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint32_t vp = smem_u32(base + OFF_VP + b * 16384);
         const uint64_t db = smem_desc(0, smem_u32(base + OFF_COL64) + 32 * b - vp, 1024, kSwizzle128B);
         for (int m = 0; m < 2 && ok; ++m) {
-          ok = wait_or_abort(bar(B_PSIK_FULL + m), j & 1, abort_flag);
-          if (ok && m == 0) ok = wait_or_abort(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
-          if (ok && j >= 1) ok = wait_or_abort(bar(B_S_FREE + m), (j - 1) & 1, abort_flag);
+          ok = wait_or_abort_counted(bar(B_PSIK_FULL + m), j & 1, abort_flag);
+          if (ok && m == 0) ok = wait_or_abort_counted(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort_counted(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
+          if (ok && j >= 1) ok = wait_or_abort_counted(bar(B_S_FREE + m), (j - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint32_t pa = smem_u32(base + OFF_PSIK + m * 32768);
@@ -396,10 +402,10 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);
       for (int j = 0; j < ntiles && ok; ++j) {
         const int b = j & 1;
-        if (j >= 2) ok = wait_or_abort(bar(B_ACC_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
+        if (j >= 2) ok = wait_or_abort_counted(bar(B_ACC_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
         for (int m = 0; m < 2 && ok; ++m) {
-          ok = wait_or_abort(bar(B_PSIQ_FULL + m), j & 1, abort_flag);
-          if (ok && j >= 1) ok = wait_or_abort(bar(B_SNAP_FULL + m), (j - 1) & 1, abort_flag);
+          ok = wait_or_abort_counted(bar(B_PSIQ_FULL + m), j & 1, abort_flag);
+          if (ok && j >= 1) ok = wait_or_abort_counted(bar(B_SNAP_FULL + m), (j - 1) & 1, abort_flag);
           if (!ok) break;
           if (j >= 1) {
             tc_fence_after();
@@ -414,8 +420,8 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         if (!ok) break;
         if (has_intra) {
-          ok = wait_or_abort(bar(B_P_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag) &&
-               wait_or_abort(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
+          ok = wait_or_abort_counted(bar(B_P_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort_counted(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag) &&
+               wait_or_abort_counted(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint32_t vp = smem_u32(base + OFF_VP + b * 16384);
@@ -433,8 +439,8 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
       const uint32_t qa = smem_u32(base + OFF_QRAW), ka = smem_u32(base + OFF_KRAW) + (has_intra ? chunk : 0) * 2048;
       for (int j = 0; j < ntiles && ok; ++j) {
-        ok = wait_or_abort(bar(B_K_FULL), j & 1, abort_flag) && wait_or_abort(bar(B_Q_FULL), j & 1, abort_flag);
-        if (ok && has_intra && j >= 1) ok = wait_or_abort(bar(B_P_FULL + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag);   // scores read
+        ok = wait_or_abort_counted(bar(B_K_FULL), j & 1, abort_flag) && wait_or_abort_counted(bar(B_Q_FULL), j & 1, abort_flag);
+        if (ok && has_intra && j >= 1) ok = wait_or_abort_counted(bar(B_P_FULL + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag);   // scores read
         if (!ok) break;
         if (has_intra) {
           tc_fence_after();
@@ -447,7 +453,9 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mma_commit(bar(B_Q_USED));
       }
     }
+  }
   } else if (warp < W_Q0) {
+    regs_release<56>();
     // =========================== key teams (thread = token; team m = accumulator tile m) ===========================
     const int m = (warp - W_K0) >> 2;
     const int t = ((warp - W_K0) & 3) * 32 + lane;
@@ -467,13 +475,13 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const unsigned short r_now = r_next;
         const int tn = (j + 1) * CT + t;
         r_next = (j + 1 < ntiles && tn < args.T) ? rs[tn] : (unsigned short)0;
-        if (j >= 2) ok = wait_or_abort(bar(B_VP_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
+        if (j >= 2) ok = wait_or_abort_counted(bar(B_VP_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
         if (!ok) break;
         sts16(sbase + OFF_COL64 + sw128_offset(t, 2 * b), r_now);
         fence_async_smem();
         mbar_arrive(bar(B_VP_READY + b));
       }
-      ok = wait_or_abort(bar(B_K_FULL), j & 1, abort_flag);
+      ok = wait_or_abort_counted(bar(B_K_FULL), j & 1, abort_flag);
       if (!ok) break;
       uint32_t ga[2][4], gb[2][4];
 #pragma unroll
@@ -490,7 +498,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       mbar_arrive(bar(B_K_EMPTY));
       // products of the two block pairs of accumulator tile m
-      if (j >= 1) ok = wait_or_abort(bar(B_U_DONE + m), (j - 1) & 1, abort_flag);
+      if (j >= 1) ok = wait_or_abort_counted(bar(B_U_DONE + m), (j - 1) & 1, abort_flag);
       if (!ok) break;
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
@@ -504,6 +512,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       mbar_arrive(bar(B_PSIK_FULL + m));
     }
   } else if (warp < W_S0) {
+    regs_take<88>();
     // =========================== query team (thread = token) ===========================
     const uint32_t q4 = warp & 3;
     const int t = q4 * 32 + lane;
@@ -519,7 +528,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t qraw = sbase + OFF_QRAW;
     const uint32_t stash = sbase + OFF_QSTASH + (tid - W_Q0 * 32) * 16;   // 4 runs of 16 bytes, 2 KB apart (conflict-free)
     for (int j = 0; j < ntiles && ok; ++j) {
-      ok = wait_or_abort(bar(B_Q_FULL), j & 1, abort_flag);
+      ok = wait_or_abort_counted(bar(B_Q_FULL), j & 1, abort_flag);
       if (!ok) break;
       // the runs of the first two block pairs stay in registers, those of the last two wait in a private stash
       uint32_t ga[2][4], gb[2][4];
@@ -551,7 +560,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             gb[e][0] = rb.x; gb[e][1] = rb.y; gb[e][2] = rb.z; gb[e][3] = rb.w;
           }
         }
-        if (j >= 1) ok = ok && wait_or_abort(bar(B_R_DONE + m), (j - 1) & 1, abort_flag);
+        if (j >= 1) ok = ok && wait_or_abort_counted(bar(B_R_DONE + m), (j - 1) & 1, abort_flag);
         if (ok) {
           tc_fence_after();
 #pragma unroll
@@ -568,13 +577,14 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (!ok) break;
     }
   } else if (warp < W_E0) {
+    regs_take<88>();
     // =========================== state team (thread = state row; both accumulator tiles in turn) ===========================
     const uint32_t q4 = warp & 3;
     const int f = q4 * 32 + lane;
     for (int j = 0; j + 1 < ntiles && ok; ++j) {
 #pragma unroll 1
       for (int m = 0; m < 2 && ok; ++m) {
-        ok = wait_or_abort(bar(B_U_DONE + m), j & 1, abort_flag);
+        ok = wait_or_abort_counted(bar(B_U_DONE + m), j & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         uint32_t pk[32], zc[4];
@@ -591,7 +601,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tc_fence_before();
         mbar_arrive(bar(B_S_FREE + m));
         // the read of tile j (which uses the snapshot after tile j - 1) must be complete
-        ok = wait_or_abort(bar(B_R_DONE + m), j & 1, abort_flag);
+        ok = wait_or_abort_counted(bar(B_R_DONE + m), j & 1, abort_flag);
         if (!ok) break;
         const uint32_t snap = sbase + OFF_SNAP + m * 16384;
 #pragma unroll
@@ -602,6 +612,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
     }
   } else if (warp < W_O0) {
+    regs_take<88>();
     // =========================== intra-tile weights and the exchange of shares (thread = token) ===========================
     const uint32_t q4 = warp & 3;
     const int t = q4 * 32 + lane;
@@ -612,7 +623,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     for (int it = 0; it <= ntiles && ok; ++it) {
       // ---- weights of tile `it`: P = (Q K_c^T)^2, causal inside the tile ----
       if (it < ntiles && has_intra) {
-        ok = wait_or_abort(bar(B_SC_FULL), it & 1, abort_flag);
+        ok = wait_or_abort_counted(bar(B_SC_FULL), it & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         uint32_t y[16], pk[8];
@@ -633,7 +644,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // ---- this CTA's share of tile it - 1 goes to the owners of its rows ----
       if (it >= 1) {
         const int j = it - 1, b = j & 1;
-        ok = wait_or_abort(bar(B_ACC_FULL + b), (j >> 1) & 1, abort_flag);
+        ok = wait_or_abort_counted(bar(B_ACC_FULL + b), (j >> 1) & 1, abort_flag);
         if (ok && j >= 1) ok = wait_cluster_or_abort(bar(B_RECV_EMPTY + owner), (j - 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -658,6 +669,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
     }
   } else {
+    regs_take<88>();
     // =========================== owner: sums of the shares, link hand-off, output ===========================
     const int et = tid - W_O0 * 32;                            // 0..127
     const size_t tpad = (size_t)ntiles * CT;
@@ -750,10 +762,10 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (et < CS) {
         if (CS == 1) mbar_arrive(bar(B_RECV_EMPTY)); else arrive_remote(map_to_rank(smem_u32(bar(B_RECV_EMPTY + rank)), (uint32_t)et));
       }
-      if (et == 0 && !last_link) {
-        __threadfence();
+      // (every kPublish tiles and at the end: a release at GPU scope waits for the whole team's stores to land,
+      // thousands of cycles, and the next link is content to run a few tiles behind)
+      if (et == 0 && !last_link && (((j + 1) % kPublish) == 0 || j + 1 == ntiles))
         asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(prog_out), "r"((unsigned)(j + 1)) : "memory");
-      }
       if (inN != nullptr && j + 1 < ntiles) {
         ok = wait_progress(prog_in, (unsigned)(j + 2), abort_flag);
         if (ok) prefetch(j + 1);
