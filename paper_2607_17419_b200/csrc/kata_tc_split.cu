@@ -56,7 +56,7 @@ constexpr uint32_t COL_S = 0;      // 2 x 80: state tiles (lanes = state rows)
 constexpr uint32_t COL_PSIQ = 160; // 128: weighted query products as bf16 pairs (lanes = tokens), 32 per block pair
 constexpr uint32_t COL_ACC = 288;  // 2 x 80: this CTA's share of [N | D] (lanes = tokens)
 constexpr uint32_t COL_SC = 448;   // 16 fp32 scores
-constexpr uint32_t COL_P = 464;    // 2 x 8: bf16 weights
+constexpr uint32_t COL_P = 464;    // 8: bf16 weights
 constexpr uint32_t TMEM_COLS = 512;
 
 // ---- shared memory (1024-byte aligned tiles of 128-byte rows, 128B swizzle) ----
@@ -70,38 +70,23 @@ constexpr uint32_t OFF_RECV = 180224;   // 128 rows x 68 floats: shares received
 constexpr uint32_t RECV_ROW = 272;
 constexpr uint32_t OFF_BAR = OFF_RECV + 128 * RECV_ROW;
 constexpr uint32_t OFF_MISC = OFF_BAR + 512;
-constexpr uint32_t OFF_SINK = OFF_MISC + 64;   // one word per thread: see consume_before_arrive
-constexpr uint32_t OFF_QSTASH = OFF_SINK + NTHREADS * 4;   // 4 x 2 KB: query runs of the last two block pairs
-constexpr uint32_t SMEM_BYTES = OFF_QSTASH + 8192;
+constexpr uint32_t SMEM_BYTES = OFF_MISC + 64;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
 static_assert(SMEM_ALLOC <= 232448, "shared memory");
 
 // Every barrier has waiters that consume each of its phases in order.
 enum {
   B_K_FULL = 0,      // key tile landed
-  B_K_EMPTY = 1,     // ... and read by the 256 key threads
-  B_Q_FULL = 2,
-  B_Q_EMPTY = 3,     // ... by the 128 query threads
-  B_V_FULL = 4,      // [2] value tile landed
-  B_VP_READY = 6,    // [2] column 64 of the value operand written (128 threads of key team 0)
-  B_VP_EMPTY = 8,    // [2] update and intra MMAs of the tile complete
-  B_PSIK_FULL = 10,  // [2] products of accumulator tile m built (128 threads)
-  B_U_DONE = 12,     // [2] update of accumulator tile m complete
-  B_S_FREE = 14,     // [2] accumulator tile m copied out of TMEM (128 threads)
-  B_SNAP_FULL = 16,  // [2] snapshot m stored (128 threads)
-  B_R_DONE = 18,     // [2] read MMAs of half m complete
-  B_PSIQ_FULL = 20,  // [2] query products of half m stored (128 threads)
-  B_SC_FULL = 22,    // scores in TMEM
-  B_P_FULL = 23,     // [2] weights stored in buffer tile & 1 (128 threads)
-  B_ACC_FULL = 25,   // [2]
-  B_ACC_EMPTY = 27,  // [2] (128 threads)
-  B_RECV_FULL = 29,  // 128 arrivals from the CTAs of the cluster
-  B_RECV_EMPTY = 30, // [4] the owner with that rank has summed what this CTA sent
-  B_DRAIN = 34,
-  B_K_USED = 35,     // the score MMAs that read the key tile are complete (commit only)
-  B_Q_USED = 36,     // ... the query tile
-  B_COUNT = 37
+  B_Q_FULL = 1,      // query tile landed
+  B_V_FULL = 2,      // [2] tile of scaled values landed
+  B_SC_FULL = 4,     // intra-tile scores in TMEM
+  B_MMA_DONE = 5,    // update, read and apply MMAs of a tile complete (two commits)
+  B_RECV_FULL = 6,   // every share of the rows this CTA owns has arrived (transaction bytes; armed by the owner team)
+  B_RECV_EMPTY = 7,  // [4] the owner with that rank has summed what this CTA sent
+  B_DRAIN = 11,
+  B_COUNT = 12
 };
+
 
 struct BlockPairs {
   unsigned char g[MAX_CTAS * NBP], h[MAX_CTAS * NBP], w[MAX_CTAS * NBP];   // w = 0: unused slot
@@ -281,6 +266,29 @@ __global__ void __launch_bounds__(256) split_prescale_kernel(const __nv_bfloat16
   if (part == 0) rscale[row] = __float2bfloat16_rn(r2);
 }
 
+// Asynchronous store of 16 bytes into the shared memory of a CTA of the cluster; the bytes count towards the
+// transaction count of the mbarrier `rbar` of that CTA (no arrival of its own).
+__device__ __forceinline__ void st_async_v4(uint32_t raddr, uint32_t rbar, float a, float b, float c, float d) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(raddr), "f"(a),
+               "f"(b), "f"(c), "f"(d), "r"(rbar)
+               : "memory");
+}
+
+// The kernel walks the tiles in lockstep.  Tile j is two phases:
+//   A  everything the MMAs of the tile read is put in place: key products (key teams), weighted query products
+//      (query team), the snapshot of the state after tile j - 1 (state team), the intra-tile weights (score MMA
+//      first, then the exchange team); one named barrier (kBarA) ends the phase;
+//   B  the update, read and apply MMAs of the tile are issued back to back (two issuing threads) and commit to
+//      one mbarrier (B_MMA_DONE), which every team waits for before it touches its buffers again.  Under phase B
+//      the exchange team sends the shares of tile j - 1, the owner team sums those of tile j - 2, and the TMA
+//      producer fetches the keys and queries of tile j + 1 (buffers free since phase A) and the values of tile
+//      j + 2.
+// Two synchronisations per tile instead of a web of point-to-point hand-offs: every hand-off between warps costs
+// several hundred cycles from arrival to the waiter's next instruction, and a pipeline whose every buffer is single
+// (shared memory and TMEM are full) turns each of them into a round trip.
+constexpr int kBarA = 2;
+constexpr int kBarAThreads = 32 * W_O0;     // every warp but the owner team
+
 template <int CS>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -302,32 +310,17 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int chunk = cta_head - 1;                             // 16-key run of every tile this CTA weighs (link 0: none)
   const bool has_intra = chunk >= 0 && chunk < 8;
   constexpr int RPO = CT / CS;                                // query rows of a tile this CTA owns
+  constexpr uint32_t RECV_BYTES = 128 * RECV_ROW;             // what the owner receives per tile
 
   if (tid == 0) {
     *abort_flag = 0;
     mbar_init(bar(B_K_FULL), 1);
-    mbar_init(bar(B_K_EMPTY), 256);
-    mbar_init(bar(B_K_USED), 1);
-    mbar_init(bar(B_Q_USED), 1);
     mbar_init(bar(B_Q_FULL), 1);
-    mbar_init(bar(B_Q_EMPTY), 128);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(B_V_FULL + i), 1);
-      mbar_init(bar(B_VP_READY + i), 128);
-      mbar_init(bar(B_VP_EMPTY + i), 2);
-      mbar_init(bar(B_PSIK_FULL + i), 128);
-      mbar_init(bar(B_U_DONE + i), 1);
-      mbar_init(bar(B_S_FREE + i), 128);
-      mbar_init(bar(B_SNAP_FULL + i), 128);
-      mbar_init(bar(B_R_DONE + i), 1);
-      mbar_init(bar(B_PSIQ_FULL + i), 128);
-      mbar_init(bar(B_ACC_FULL + i), 1);
-      mbar_init(bar(B_ACC_EMPTY + i), 128);
-    }
+    mbar_init(bar(B_V_FULL), 1);
+    mbar_init(bar(B_V_FULL + 1), 1);
     mbar_init(bar(B_SC_FULL), 1);
-    mbar_init(bar(B_P_FULL), 128);
-    mbar_init(bar(B_P_FULL + 1), 128);
-    mbar_init(bar(B_RECV_FULL), 128);
+    mbar_init(bar(B_MMA_DONE), 2);
+    mbar_init(bar(B_RECV_FULL), 1);
     for (int i = 0; i < 4; ++i) mbar_init(bar(B_RECV_EMPTY + i), 1);
     mbar_init(bar(B_DRAIN), 3);
     fence_mbar_init();
@@ -350,110 +343,129 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   tc_fence_after();
   const uint32_t tb = *tmem_base_s;
   bool ok = true;
+  // the wait that opens tile j for every team: the MMAs of tile j - 1 are complete
+  auto mma_done = [&](int j) { return j == 0 ? true : wait_or_abort_counted(bar(B_MMA_DONE), (j - 1) & 1, abort_flag); };
+  // end of phase A.  A team that gave up keeps arriving, so that nobody is left waiting at the named barrier.
+  auto phase_a_done = [&]() { asm volatile("bar.sync %0, %1;" ::"n"(kBarA), "n"(kBarAThreads) : "memory"); };
 
   if (warp < W_K0) {
-  regs_release<40>();
-  if (warp == W_TMA) {
-    // =========================== TMA producer ===========================
-    if (lane == 0) {
-      for (int j = 0; j < ntiles && ok; ++j) {
+    regs_release<40>();
+    if (warp == W_TMA) {
+      // =========================== TMA producer ===========================
+      for (int j = 0; j < ntiles; ++j) {
         const int b = j & 1;
-        if (j >= 1) ok = wait_or_abort_counted(bar(B_K_EMPTY), (j - 1) & 1, abort_flag) && wait_or_abort_counted(bar(B_K_USED), (j - 1) & 1, abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar(B_K_FULL), 16384);
-        tma_load_3d(base + OFF_KRAW, &tmK, bar(B_K_FULL), 0, j * CT, bh);
-        if (j >= 2) ok = wait_or_abort_counted(bar(B_VP_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar(B_V_FULL + b), 16384);
-        tma_load_3d(base + OFF_VP + b * 16384, &tmV, bar(B_V_FULL + b), 0, j * CT, bh);
-        if (j >= 1) ok = wait_or_abort_counted(bar(B_Q_EMPTY), (j - 1) & 1, abort_flag) && wait_or_abort_counted(bar(B_Q_USED), (j - 1) & 1, abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar(B_Q_FULL), 16384);
-        tma_load_3d(base + OFF_QRAW, &tmQ, bar(B_Q_FULL), 0, j * CT, bh);
+        if (lane == 0 && ok) {
+          if (j == 0) {
+            mbar_arrive_expect_tx(bar(B_K_FULL), 16384);
+            tma_load_3d(base + OFF_KRAW, &tmK, bar(B_K_FULL), 0, 0, bh);
+            mbar_arrive_expect_tx(bar(B_Q_FULL), 16384);
+            tma_load_3d(base + OFF_QRAW, &tmQ, bar(B_Q_FULL), 0, 0, bh);
+            mbar_arrive_expect_tx(bar(B_V_FULL), 16384);
+            tma_load_3d(base + OFF_VP, &tmV, bar(B_V_FULL), 0, 0, bh);
+            if (ntiles > 1) {
+              mbar_arrive_expect_tx(bar(B_V_FULL + 1), 16384);
+              tma_load_3d(base + OFF_VP + 16384, &tmV, bar(B_V_FULL + 1), 0, CT, bh);
+            }
+          }
+          // tiles three ahead into L2, so that the loads below find them there
+          if (j + 3 < ntiles) {
+            asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(&tmK), "r"(0), "r"((j + 3) * CT), "r"(bh) : "memory");
+            asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(&tmQ), "r"(0), "r"((j + 3) * CT), "r"(bh) : "memory");
+            asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(&tmV), "r"(0), "r"((j + 3) * CT), "r"(bh) : "memory");
+          }
+        }
+        phase_a_done();                 // keys and queries of tile j have been read (teams) and multiplied (score MMA)
+        if (lane == 0 && ok && j + 1 < ntiles) {
+          mbar_arrive_expect_tx(bar(B_K_FULL), 16384);
+          tma_load_3d(base + OFF_KRAW, &tmK, bar(B_K_FULL), 0, (j + 1) * CT, bh);
+          mbar_arrive_expect_tx(bar(B_Q_FULL), 16384);
+          tma_load_3d(base + OFF_QRAW, &tmQ, bar(B_Q_FULL), 0, (j + 1) * CT, bh);
+        }
+        if (j + 2 < ntiles) {
+          ok = ok && mma_done(j + 1);   // the MMAs of tile j are done with the value tile
+          if (lane == 0 && ok) {
+            mbar_arrive_expect_tx(bar(B_V_FULL + b), 16384);
+            tma_load_3d(base + OFF_VP + b * 16384, &tmV, bar(B_V_FULL + b), 0, (j + 2) * CT, bh);
+          }
+        }
       }
-    }
-  } else if (warp == W_U) {
-    // =========================== update issuer: S[m] += Psi(K)_m^T [V' | r] ===========================
-    if (lane == 0) {
+    } else if (warp == W_U) {
+      // =========================== update issuer: S[m] += Psi(K)_m^T [V' | r] ===========================
       const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 80);
       const uint64_t da = smem_desc(0, 16384, 1024, kSwizzle128B);      // second run of 64 state rows: next block pair
-      for (int j = 0; j < ntiles && ok; ++j) {
+      for (int j = 0; j < ntiles; ++j) {
         const int b = j & 1;
-        const uint32_t vp = smem_u32(base + OFF_VP + b * 16384);
-        const uint64_t db = smem_desc(0, smem_u32(base + OFF_COL64) + 32 * b - vp, 1024, kSwizzle128B);
-        for (int m = 0; m < 2 && ok; ++m) {
-          ok = wait_or_abort_counted(bar(B_PSIK_FULL + m), j & 1, abort_flag);
-          if (ok && m == 0) ok = wait_or_abort_counted(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort_counted(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
-          if (ok && j >= 1) ok = wait_or_abort_counted(bar(B_S_FREE + m), (j - 1) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t pa = smem_u32(base + OFF_PSIK + m * 32768);
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            mma_f16_ss(tb + COL_S + m * 80, at(da, pa + ks * 2048), at(db, vp + ks * 2048), idesc, (j > 0 || ks > 0) ? 1u : 0u);
-          mma_commit(bar(B_U_DONE + m));
-        }
-        if (ok) mma_commit(bar(B_VP_EMPTY + b));
-      }
-    }
-  } else if (warp == W_R) {
-    // =========================== read issuer: ACC = Psi(Q) [S | Z] (+ the intra-tile apply) ===========================
-    if (lane == 0) {
-      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);
-      for (int j = 0; j < ntiles && ok; ++j) {
-        const int b = j & 1;
-        if (j >= 2) ok = wait_or_abort_counted(bar(B_ACC_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
-        for (int m = 0; m < 2 && ok; ++m) {
-          ok = wait_or_abort_counted(bar(B_PSIQ_FULL + m), j & 1, abort_flag);
-          if (ok && j >= 1) ok = wait_or_abort_counted(bar(B_SNAP_FULL + m), (j - 1) & 1, abort_flag);
-          if (!ok) break;
-          if (j >= 1) {
+        phase_a_done();
+        ok = ok && wait_or_abort_counted(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag);
+        if (lane == 0) {
+          if (ok) {
             tc_fence_after();
-            const uint32_t sn = smem_u32(base + OFF_SNAP + m * 16384);
-            const uint64_t db = smem_desc(0, smem_u32(base + OFF_COL64) + 32 * (2 + m) - sn, 1024, kSwizzle128B);
+            const uint32_t vp = sbase + OFF_VP + b * 16384;
+            const uint64_t db = smem_desc(0, sbase + OFF_COL64 + 32 * b - vp, 1024, kSwizzle128B);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-              mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_PSIQ + m * 64 + ks * 8, at(db, sn + ks * 2048), idesc,
-                         (m > 0 || ks > 0) ? 1u : 0u);
+            for (int m = 0; m < 2; ++m) {
+              const uint32_t pa = sbase + OFF_PSIK + m * 32768;
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks)
+                mma_f16_ss(tb + COL_S + m * 80, at(da, pa + ks * 2048), at(db, vp + ks * 2048), idesc, (j > 0 || ks > 0) ? 1u : 0u);
+            }
           }
-          mma_commit(bar(B_R_DONE + m));
+          mma_commit(bar(B_MMA_DONE));
         }
-        if (!ok) break;
-        if (has_intra) {
-          ok = wait_or_abort_counted(bar(B_P_FULL + b), (j >> 1) & 1, abort_flag) && wait_or_abort_counted(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag) &&
-               wait_or_abort_counted(bar(B_VP_READY + b), (j >> 1) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t vp = smem_u32(base + OFF_VP + b * 16384);
-          const uint64_t db = smem_desc(0, smem_u32(base + OFF_COL64) + 32 * b - vp, 1024, kSwizzle128B);
-          mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_P + b * 8, at(db, vp + chunk * 2048), idesc, j >= 1 ? 1u : 0u);
-        }
-        mma_commit(bar(B_ACC_FULL + b));
-        mma_commit(bar(B_VP_EMPTY + b));
+        __syncwarp();
       }
-    }
-  } else if (warp == W_I) {
-    // =========================== score issuer: Q K_c^T for this CTA's 16 keys ===========================
-    if (lane == 0) {
+    } else if (warp == W_R) {
+      // =========================== read issuer: ACC = Psi(Q) [S | Z] + P_c [V' | r]_c ===========================
+      const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);
+      for (int j = 0; j < ntiles; ++j) {
+        const int b = j & 1;
+        phase_a_done();
+        if (has_intra) ok = ok && wait_or_abort_counted(bar(B_V_FULL + b), (j >> 1) & 1, abort_flag);
+        if (lane == 0) {
+          if (ok) {
+            tc_fence_after();
+            if (j >= 1) {
+#pragma unroll
+              for (int m = 0; m < 2; ++m) {
+                const uint32_t sn = sbase + OFF_SNAP + m * 16384;
+                const uint64_t db = smem_desc(0, sbase + OFF_COL64 + 32 * (2 + m) - sn, 1024, kSwizzle128B);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                  mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_PSIQ + m * 64 + ks * 8, at(db, sn + ks * 2048), idesc, (m > 0 || ks > 0) ? 1u : 0u);
+              }
+            }
+            if (has_intra) {
+              const uint32_t vp = sbase + OFF_VP + b * 16384;
+              const uint64_t db = smem_desc(0, sbase + OFF_COL64 + 32 * b - vp, 1024, kSwizzle128B);
+              mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_P, at(db, vp + chunk * 2048), idesc, j >= 1 ? 1u : 0u);
+            }
+          }
+          mma_commit(bar(B_MMA_DONE));
+        }
+        __syncwarp();
+      }
+    } else {
+      // =========================== score issuer: Q K_c^T for this CTA's 16 keys (opens phase A) ===========================
       const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 16);
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
-      const uint32_t qa = smem_u32(base + OFF_QRAW), ka = smem_u32(base + OFF_KRAW) + (has_intra ? chunk : 0) * 2048;
-      for (int j = 0; j < ntiles && ok; ++j) {
-        ok = wait_or_abort_counted(bar(B_K_FULL), j & 1, abort_flag) && wait_or_abort_counted(bar(B_Q_FULL), j & 1, abort_flag);
-        if (ok && has_intra && j >= 1) ok = wait_or_abort_counted(bar(B_P_FULL + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag);   // scores read
-        if (!ok) break;
+      const uint32_t qa = sbase + OFF_QRAW, ka = sbase + OFF_KRAW + (has_intra ? chunk : 0) * 2048;
+      for (int j = 0; j < ntiles; ++j) {
         if (has_intra) {
-          tc_fence_after();
+          ok = ok && mma_done(j);       // the apply MMA of tile j - 1 has read the weights; their columns may be rewritten
+          ok = ok && wait_or_abort_counted(bar(B_K_FULL), j & 1, abort_flag) && wait_or_abort_counted(bar(B_Q_FULL), j & 1, abort_flag);
+          if (lane == 0) {
+            if (ok) {
+              tc_fence_after();
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            mma_f16_ss(tb + COL_SC, at(dk, qa + ks * 32), at(dk, ka + ks * 32), idesc, ks > 0 ? 1u : 0u);
-          mma_commit(bar(B_SC_FULL));
+              for (int ks = 0; ks < 4; ++ks) mma_f16_ss(tb + COL_SC, at(dk, qa + ks * 32), at(dk, ka + ks * 32), idesc, ks > 0 ? 1u : 0u);
+            }
+            mma_commit(bar(B_SC_FULL));
+          }
+          __syncwarp();
         }
-        mma_commit(bar(B_K_USED));
-        mma_commit(bar(B_Q_USED));
+        phase_a_done();
       }
     }
-  }
   } else if (warp < W_Q0) {
     regs_release<56>();
     // =========================== key teams (thread = token; team m = accumulator tile m) ===========================
@@ -468,48 +480,30 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t kraw = sbase + OFF_KRAW;
     const unsigned short* rs = reinterpret_cast<const unsigned short*>(args.rscale) + (size_t)bh * args.T;
     unsigned short r_next = (m == 0 && t < args.T) ? rs[t] : (unsigned short)0;
-    for (int j = 0; j < ntiles && ok; ++j) {
+    for (int j = 0; j < ntiles; ++j) {
       const int b = j & 1;
-      // team 0: column 64 of the value operand (r of this token), once the tile two back is done with its copy
-      if (m == 0) {
-        const unsigned short r_now = r_next;
-        const int tn = (j + 1) * CT + t;
-        r_next = (j + 1 < ntiles && tn < args.T) ? rs[tn] : (unsigned short)0;
-        if (j >= 2) ok = wait_or_abort_counted(bar(B_VP_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
-        if (!ok) break;
-        sts16(sbase + OFF_COL64 + sw128_offset(t, 2 * b), r_now);
+      ok = ok && mma_done(j);           // the update of tile j - 1 has read the products (and column 64 of its values)
+      ok = ok && wait_or_abort_counted(bar(B_K_FULL), j & 1, abort_flag);
+      if (ok) {
+        if (m == 0) {                   // column 64 of the value operand: r of this token
+          sts16(sbase + OFF_COL64 + sw128_offset(t, 2 * b), r_next);
+          const int tn = (j + 1) * CT + t;
+          r_next = (j + 1 < ntiles && tn < args.T) ? rs[tn] : (unsigned short)0;
+        }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const uint4 ra = lds128(kraw + sw128_offset(t, pg[e]));
+          const uint4 rb = lds128(kraw + sw128_offset(t, ph[e]));
+          const uint32_t ga[4] = {ra.x, ra.y, ra.z, ra.w}, gb[4] = {rb.x, rb.y, rb.z, rb.w};
+          uint32_t pr[32];
+          products8x8<false>(ga, gb, 0u, pr);
+          const uint32_t dst = sbase + OFF_PSIK + (2 * m + e) * 16384;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) sts128(dst + sw128_offset(t, i), pr[4 * i], pr[4 * i + 1], pr[4 * i + 2], pr[4 * i + 3]);
+        }
         fence_async_smem();
-        mbar_arrive(bar(B_VP_READY + b));
       }
-      ok = wait_or_abort_counted(bar(B_K_FULL), j & 1, abort_flag);
-      if (!ok) break;
-      uint32_t ga[2][4], gb[2][4];
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const uint4 ra = lds128(kraw + sw128_offset(t, pg[e]));
-        const uint4 rb = lds128(kraw + sw128_offset(t, ph[e]));
-        ga[e][0] = ra.x; ga[e][1] = ra.y; ga[e][2] = ra.z; ga[e][3] = ra.w;
-        gb[e][0] = rb.x; gb[e][1] = rb.y; gb[e][2] = rb.z; gb[e][3] = rb.w;
-      }
-      {
-        const uint32_t held[16] = {ga[0][0], ga[0][1], ga[0][2], ga[0][3], gb[0][0], gb[0][1], gb[0][2], gb[0][3],
-                                   ga[1][0], ga[1][1], ga[1][2], ga[1][3], gb[1][0], gb[1][1], gb[1][2], gb[1][3]};
-        consume_before_arrive(sbase + OFF_SINK + tid * 4, held);
-      }
-      mbar_arrive(bar(B_K_EMPTY));
-      // products of the two block pairs of accumulator tile m
-      if (j >= 1) ok = wait_or_abort_counted(bar(B_U_DONE + m), (j - 1) & 1, abort_flag);
-      if (!ok) break;
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        uint32_t pr[32];
-        products8x8<false>(ga[e], gb[e], 0u, pr);
-        const uint32_t dst = sbase + OFF_PSIK + (2 * m + e) * 16384;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) sts128(dst + sw128_offset(t, i), pr[4 * i], pr[4 * i + 1], pr[4 * i + 2], pr[4 * i + 3]);
-      }
-      fence_async_smem();
-      mbar_arrive(bar(B_PSIK_FULL + m));
+      phase_a_done();
     }
   } else if (warp < W_S0) {
     regs_take<88>();
@@ -526,90 +520,56 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       pw[e] = w == 0 ? 0u : w == 1 ? 0x3F803F80u : 0x40004000u;
     }
     const uint32_t qraw = sbase + OFF_QRAW;
-    const uint32_t stash = sbase + OFF_QSTASH + (tid - W_Q0 * 32) * 16;   // 4 runs of 16 bytes, 2 KB apart (conflict-free)
-    for (int j = 0; j < ntiles && ok; ++j) {
-      ok = wait_or_abort_counted(bar(B_Q_FULL), j & 1, abort_flag);
-      if (!ok) break;
-      // the runs of the first two block pairs stay in registers, those of the last two wait in a private stash
-      uint32_t ga[2][4], gb[2][4];
+    for (int j = 0; j < ntiles; ++j) {
+      ok = ok && mma_done(j);           // the read of tile j - 1 has used the products
+      ok = ok && wait_or_abort_counted(bar(B_Q_FULL), j & 1, abort_flag);
+      if (ok) {
+        tc_fence_after();
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const uint4 ra = lds128(qraw + sw128_offset(t, pg[e]));
-        const uint4 rb = lds128(qraw + sw128_offset(t, ph[e]));
-        ga[e][0] = ra.x; ga[e][1] = ra.y; ga[e][2] = ra.z; ga[e][3] = ra.w;
-        gb[e][0] = rb.x; gb[e][1] = rb.y; gb[e][2] = rb.z; gb[e][3] = rb.w;
-        const uint4 sa = lds128(qraw + sw128_offset(t, pg[2 + e]));
-        const uint4 sb = lds128(qraw + sw128_offset(t, ph[2 + e]));
-        sts128(stash + (2 * e) * 2048, sa.x, sa.y, sa.z, sa.w);
-        sts128(stash + (2 * e + 1) * 2048, sb.x, sb.y, sb.z, sb.w);
-      }
-      {
-        const uint32_t held[16] = {ga[0][0], ga[0][1], ga[0][2], ga[0][3], gb[0][0], gb[0][1], gb[0][2], gb[0][3],
-                                   ga[1][0], ga[1][1], ga[1][2], ga[1][3], gb[1][0], gb[1][1], gb[1][2], gb[1][3]};
-        consume_before_arrive(sbase + OFF_SINK + tid * 4, held);
-      }
-      mbar_arrive(bar(B_Q_EMPTY));
-#pragma unroll
-      for (int m = 0; m < 2; ++m) {
-        if (m == 1) {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const uint4 ra = lds128(stash + (2 * e) * 2048);
-            const uint4 rb = lds128(stash + (2 * e + 1) * 2048);
-            ga[e][0] = ra.x; ga[e][1] = ra.y; ga[e][2] = ra.z; ga[e][3] = ra.w;
-            gb[e][0] = rb.x; gb[e][1] = rb.y; gb[e][2] = rb.z; gb[e][3] = rb.w;
-          }
+        for (int e = 0; e < NBP; ++e) {
+          const uint4 ra = lds128(qraw + sw128_offset(t, pg[e]));
+          const uint4 rb = lds128(qraw + sw128_offset(t, ph[e]));
+          const uint32_t ga[4] = {ra.x, ra.y, ra.z, ra.w}, gb[4] = {rb.x, rb.y, rb.z, rb.w};
+          uint32_t pr[32];
+          products8x8<true>(ga, gb, pw[e], pr);
+          tmem_st32(tmem_addr(tb, q4 * 32, COL_PSIQ + e * 32), pr);
         }
-        if (j >= 1) ok = ok && wait_or_abort_counted(bar(B_R_DONE + m), (j - 1) & 1, abort_flag);
-        if (ok) {
-          tc_fence_after();
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            uint32_t pr[32];
-            products8x8<true>(ga[e], gb[e], pw[2 * m + e], pr);
-            tmem_st32(tmem_addr(tb, q4 * 32, COL_PSIQ + (2 * m + e) * 32), pr);
-          }
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(bar(B_PSIQ_FULL + m));
-        }
+        tmem_wait_st();
+        tc_fence_before();
       }
-      if (!ok) break;
+      phase_a_done();
     }
   } else if (warp < W_E0) {
     regs_take<88>();
-    // =========================== state team (thread = state row; both accumulator tiles in turn) ===========================
+    // =========================== state team (thread = state row of both accumulator tiles) ===========================
     const uint32_t q4 = warp & 3;
     const int f = q4 * 32 + lane;
-    for (int j = 0; j + 1 < ntiles && ok; ++j) {
-#pragma unroll 1
-      for (int m = 0; m < 2 && ok; ++m) {
-        ok = wait_or_abort_counted(bar(B_U_DONE + m), j & 1, abort_flag);
-        if (!ok) break;
+    for (int j = 0; j < ntiles; ++j) {
+      ok = ok && mma_done(j);           // the update of tile j - 1 is complete, and so is the read that used the old snapshot
+      if (ok && j >= 1) {
         tc_fence_after();
-        uint32_t pk[32], zc[4];
 #pragma unroll
-        for (int h = 0; h < 4; ++h) {
-          uint32_t y[16];
-          tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + m * 80 + h * 16), y);
-          if (h == 3) tmem_ld4(tmem_addr(tb, q4 * 32, COL_S + m * 80 + 64), zc);
-          tmem_wait_ld(y);
+        for (int m = 0; m < 2; ++m) {
+          uint32_t pk[32], zc[4];
 #pragma unroll
-          for (int c = 0; c < 8; ++c) pk[h * 8 + c] = pack_bf16(__uint_as_float(y[2 * c]), __uint_as_float(y[2 * c + 1]));
+          for (int h = 0; h < 4; ++h) {
+            uint32_t y[16];
+            tmem_ld16(tmem_addr(tb, q4 * 32, COL_S + m * 80 + h * 16), y);
+            if (h == 3) tmem_ld4(tmem_addr(tb, q4 * 32, COL_S + m * 80 + 64), zc);
+            tmem_wait_ld(y);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) pk[h * 8 + c] = pack_bf16(__uint_as_float(y[2 * c]), __uint_as_float(y[2 * c + 1]));
+          }
+          tmem_wait_ld(zc);
+          const uint32_t snap = sbase + OFF_SNAP + m * 16384;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) sts128(snap + sw128_offset(f, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+          sts16(sbase + OFF_COL64 + sw128_offset(f, 2 * (2 + m)), __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(zc[0]))));
         }
-        tmem_wait_ld(zc);
         tc_fence_before();
-        mbar_arrive(bar(B_S_FREE + m));
-        // the read of tile j (which uses the snapshot after tile j - 1) must be complete
-        ok = wait_or_abort_counted(bar(B_R_DONE + m), j & 1, abort_flag);
-        if (!ok) break;
-        const uint32_t snap = sbase + OFF_SNAP + m * 16384;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) sts128(snap + sw128_offset(f, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-        sts16(sbase + OFF_COL64 + sw128_offset(f, 2 * (2 + m)), __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(zc[0]))));
         fence_async_smem();
-        mbar_arrive(bar(B_SNAP_FULL + m));
       }
+      phase_a_done();
     }
   } else if (warp < W_O0) {
     regs_take<88>();
@@ -618,54 +578,57 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int t = q4 * 32 + lane;
     const uint32_t owner = (uint32_t)(t / RPO);
     const uint32_t recv_local = sbase + OFF_RECV + (rank * RPO + (t % RPO)) * RECV_ROW;
-    const uint32_t recv_remote = CS == 1 ? recv_local : map_to_rank(recv_local, owner);
-    const uint32_t full_remote = CS == 1 ? smem_u32(bar(B_RECV_FULL)) : map_to_rank(smem_u32(bar(B_RECV_FULL)), owner);
-    for (int it = 0; it <= ntiles && ok; ++it) {
-      // ---- weights of tile `it`: P = (Q K_c^T)^2, causal inside the tile ----
-      if (it < ntiles && has_intra) {
-        ok = wait_or_abort_counted(bar(B_SC_FULL), it & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t y[16], pk[8];
-        tmem_ld16(tmem_addr(tb, q4 * 32, COL_SC), y);
-        tmem_wait_ld(y);
+    const uint32_t recv_remote = map_to_rank(recv_local, owner);
+    const uint32_t full_remote = map_to_rank(smem_u32(bar(B_RECV_FULL)), owner);
+    for (int j = 0; j <= ntiles; ++j) {
+      ok = ok && mma_done(j);           // observed here, like every team, before the tile's named barrier
+      // ---- phase A of tile j: weights P = (Q K_c^T)^2, causal inside the tile ----
+      if (j < ntiles) {
+        if (has_intra) {
+          ok = ok && wait_or_abort_counted(bar(B_SC_FULL), j & 1, abort_flag);
+          if (ok) {
+            tc_fence_after();
+            uint32_t y[16], pk[8];
+            tmem_ld16(tmem_addr(tb, q4 * 32, COL_SC), y);
+            tmem_wait_ld(y);
 #pragma unroll
-        for (int c = 0; c < 16; c += 2) {
-          float a = __uint_as_float(y[c]), bq = __uint_as_float(y[c + 1]);
-          a = (chunk * 16 + c <= t) ? a * a : 0.f;
-          bq = (chunk * 16 + c + 1 <= t) ? bq * bq : 0.f;
-          pk[c >> 1] = pack_bf16(a, bq);
+            for (int c = 0; c < 16; c += 2) {
+              float a = __uint_as_float(y[c]), bq = __uint_as_float(y[c + 1]);
+              a = (chunk * 16 + c <= t) ? a * a : 0.f;
+              bq = (chunk * 16 + c + 1 <= t) ? bq * bq : 0.f;
+              pk[c >> 1] = pack_bf16(a, bq);
+            }
+            tmem_st8(tmem_addr(tb, q4 * 32, COL_P), pk);
+            tmem_wait_st();
+            tc_fence_before();
+          }
         }
-        tmem_st8(tmem_addr(tb, q4 * 32, COL_P + (it & 1) * 8), pk);
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar(B_P_FULL + (it & 1)));
+        phase_a_done();
       }
-      // ---- this CTA's share of tile it - 1 goes to the owners of its rows ----
-      if (it >= 1) {
-        const int j = it - 1, b = j & 1;
-        ok = wait_or_abort_counted(bar(B_ACC_FULL + b), (j >> 1) & 1, abort_flag);
-        if (ok && j >= 1) ok = wait_cluster_or_abort(bar(B_RECV_EMPTY + owner), (j - 1) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const bool valid = has_intra || j >= 1;                  // nothing was accumulated otherwise
+      // ---- under phase B of tile j: this CTA's share of tile j - 1 goes to the owners of its rows ----
+      if (j >= 1) {
+        const int jj = j - 1, b = jj & 1;
+        if (ok && jj >= 1) ok = wait_cluster_or_abort(bar(B_RECV_EMPTY + owner), (jj - 1) & 1, abort_flag);
+        if (ok) {
+          tc_fence_after();
+          const bool valid = has_intra || jj >= 1;               // nothing was accumulated otherwise
 #pragma unroll 1
-        for (int h = 0; h < 2; ++h) {
-          uint32_t y[32];
-          tmem_ld32(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + h * 32), y);
-          tmem_wait_ld(y);
+          for (int h = 0; h < 2; ++h) {
+            uint32_t y[32];
+            tmem_ld32(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + h * 32), y);
+            tmem_wait_ld(y);
 #pragma unroll
-          for (int c = 0; c < 8; ++c)
-            st_cluster_v4(recv_remote + h * 128 + c * 16, valid ? __uint_as_float(y[4 * c]) : 0.f, valid ? __uint_as_float(y[4 * c + 1]) : 0.f,
-                          valid ? __uint_as_float(y[4 * c + 2]) : 0.f, valid ? __uint_as_float(y[4 * c + 3]) : 0.f);
+            for (int c = 0; c < 8; ++c)
+              st_async_v4(recv_remote + h * 128 + c * 16, full_remote, valid ? __uint_as_float(y[4 * c]) : 0.f,
+                          valid ? __uint_as_float(y[4 * c + 1]) : 0.f, valid ? __uint_as_float(y[4 * c + 2]) : 0.f,
+                          valid ? __uint_as_float(y[4 * c + 3]) : 0.f);
+          }
+          uint32_t dn[4];
+          tmem_ld4(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + 64), dn);
+          tmem_wait_ld(dn);
+          tc_fence_before();
+          st_async_v4(recv_remote + 256, full_remote, valid ? __uint_as_float(dn[0]) : 0.f, 0.f, 0.f, 0.f);
         }
-        uint32_t dn[4];
-        tmem_ld4(tmem_addr(tb, q4 * 32, COL_ACC + b * 80 + 64), dn);
-        tmem_wait_ld(dn);
-        tc_fence_before();
-        mbar_arrive(bar(B_ACC_EMPTY + b));
-        st_cluster_v4(recv_remote + 256, valid ? __uint_as_float(dn[0]) : 0.f, 0.f, 0.f, 0.f);
-        if (CS == 1) mbar_arrive(bar(B_RECV_FULL)); else arrive_remote(full_remote);
       }
     }
   } else {
@@ -693,6 +656,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       for (int c = 0; c < 4; ++c) pre[c] = *reinterpret_cast<const float4*>(inN + grow * 64 + qu * 16 + c * 4);
       if (qu == 0) pre_d = inD[grow];
     };
+    if (et == 0 && ntiles > 0) mbar_arrive_expect_tx(bar(B_RECV_FULL), RECV_BYTES);
     if (inN != nullptr && ntiles > 0) {
       ok = wait_progress(prog_in, 1u, abort_flag);
       if (ok) prefetch(0);
@@ -755,15 +719,14 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
       }
-      // every thread of the team has read its shares (and written its rows): the senders may refill the buffer,
-      // and one thread publishes the tile to the next link (its release covers the team's writes, which the
-      // barrier orders before it)
+      // every thread of the team has read its shares (and written its rows): the buffer is armed for the next tile
+      // and handed back to the senders, and one thread publishes the tile to the next link (its release covers
+      // the team's writes, which the barrier orders before it; every kPublish tiles and at the end: a release at
+      // GPU scope waits for the whole team's stores to land, and the next link is content to run a few tiles behind)
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (et < CS) {
-        if (CS == 1) mbar_arrive(bar(B_RECV_EMPTY)); else arrive_remote(map_to_rank(smem_u32(bar(B_RECV_EMPTY + rank)), (uint32_t)et));
-      }
-      // (every kPublish tiles and at the end: a release at GPU scope waits for the whole team's stores to land,
-      // thousands of cycles, and the next link is content to run a few tiles behind)
+      if (et == 0 && j + 1 < ntiles) mbar_arrive_expect_tx(bar(B_RECV_FULL), RECV_BYTES);
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (et < CS) arrive_remote(map_to_rank(smem_u32(bar(B_RECV_EMPTY + rank)), (uint32_t)et));
       if (et == 0 && !last_link && (((j + 1) % kPublish) == 0 || j + 1 == ntiles))
         asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(prog_out), "r"((unsigned)(j + 1)) : "memory");
       if (inN != nullptr && j + 1 < ntiles) {
