@@ -21,6 +21,7 @@ KATA_IMPL_AUTO, KATA_IMPL_SIMT, KATA_IMPL_TENSOR = 0, 1, 2
 KATA_FN_QUADRATIC, KATA_FN_CHUNKED, KATA_FN_CHUNK_STATE_SCAN, KATA_FN_DECODE_STEP = 0, 1, 2, 3
 KATA_FN_BWD_QUADRATIC = 4
 KATA_FN_HOST_IO = 0x100
+KATA_OK, KATA_ERR_INVALID_ARG, KATA_ERR_WORKSPACE_TOO_SMALL, KATA_ERR_DEVICE_TIMEOUT = 0, -1, -4, -7
 
 EXPORTS = ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan", "kata_chunk_state_scan_static",
            "kata_fwd_host", "kata_decode_step", "kata_bwd_quadratic",
@@ -92,6 +93,8 @@ def lib() -> ctypes.CDLL:
     L.kata_status_string.restype = ctypes.c_char_p
     L.kata_version.argtypes = []
     L.kata_version.restype = i
+    L.kata_selftest_wait_timeout.argtypes = [ptr, ptr, ctypes.c_uint, ptr]
+    L.kata_selftest_wait_timeout.restype = i
     _lib = L
     return L
 
@@ -138,6 +141,18 @@ def kata_host_plan(fn: int, B, H, T, d_k, d_v, C, opts: KataOpts):
     if st != 0:
         raise KataError(st, "kata_host_plan")
     return a.value, b.value
+
+
+def kata_selftest_wait_timeout(device_status, report, max_polls: int = 1000, stream=None) -> int:
+    """Test hook (csrc/kata_selftest.h): one warp runs both bounded waits on a barrier nobody arrives at.
+
+    `device_status` is an int32 CUDA tensor of one element (or None), `report` one of three.  Returns the status code.
+    """
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    return int(lib().kata_selftest_wait_timeout(device_status.data_ptr() if device_status is not None else None,
+                                                report.data_ptr() if report is not None else None, max_polls, stream))
 
 
 def kata_last_launch_count() -> int:

@@ -317,7 +317,7 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
 // The same wait bounded by a poll count (one register less, one instruction less per poll; for the kernel that runs
 // at its register cap).  With a hint of 1 us a wait gives up after at most kSpinLimit x 1 us = 4 s, and no sooner
 // than kSpinLimit polls take where the hardware cuts the suspension short (0.1 s).
-__device__ __forceinline__ bool wait_or_abort_counted(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool wait_or_abort_polls(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t max_polls) {
   uint32_t ok;
   asm volatile(
       "{\n\t"
@@ -334,10 +334,13 @@ __device__ __forceinline__ bool wait_or_abort_counted(uint64_t* bar, uint32_t pa
       "selp.u32 %0, 1, 0, p;\n\t"
       "}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(kSpinLimit)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(max_polls)
       : "memory");
   if (ok == 0) *abort_flag = 1;
   return ok != 0;
+}
+__device__ __forceinline__ bool wait_or_abort_counted(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  return wait_or_abort_polls(bar, parity, abort_flag, kSpinLimit);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {

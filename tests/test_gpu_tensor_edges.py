@@ -83,3 +83,23 @@ def test_nonnegative_values_stay_in_hull(form):
     assert np.all(g <= vmax + slack) and np.all(g >= vmin - slack)
     for (b, h), r in oracle_full(w).items():
         check(g[b, h], r, "bf16", f"hull/{form}")
+
+
+def test_bounded_waits_time_out_cleanly_and_the_stream_stays_usable():
+    """The error contract of the tensor-core kernels (`KATA_ERR_DEVICE_TIMEOUT` in `*device_status`): a wait that
+    nothing satisfies gives up on its own limit, the kernel writes the status and returns, and the next call on the
+    same stream is correct.  Run on a test-only kernel of one warp (no TMEM, MMA or TMA in flight)."""
+    import torch
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rep = torch.full((3,), -1, dtype=torch.int32, device="cuda")
+    assert kb.kata_selftest_wait_timeout(st, rep, max_polls=2000) == kb.KATA_OK
+    torch.cuda.synchronize()
+    assert int(st.item()) == kb.KATA_ERR_DEVICE_TIMEOUT
+    assert rep.tolist() == [1, 1, 1], "both waits gave up and raised the abort flag"
+    assert kb.kata_selftest_wait_timeout(st, rep, max_polls=0) == kb.KATA_ERR_INVALID_ARG
+    # the next ordinary call on the same stream
+    w = inputs.gaussian_workload("after_timeout", "bf16", 1, 2, 300, 64, 64, 64, 4242)
+    for form in FORMS:
+        g = run(form, *dev_tensors(w))
+        for (b, h), r in oracle_full(w).items():
+            check(g[b, h], r, "bf16", f"after a timed-out launch/{form} head ({b},{h})")
