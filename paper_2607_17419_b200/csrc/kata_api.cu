@@ -114,9 +114,13 @@ int simt_scan_group(int BH, int slices, int NC) {
 }
 
 // Chunks per group of the scan forms on the tensor-core kernel.  One CTA per SM and per (head, value slice, group):
-// the first pass runs groups 0 .. ng-2 in its state-only build (about 2.8 us a tile), the last pass runs all ng
-// groups (about 4.4 us a tile), each in whole waves of 148 CTAs; a group state costs four transfers of 115 KB per
-// CTA.  The smallest modelled time over ng = 2 .. 32 decides.
+// the first pass runs groups 0 .. ng-2 in its state-only build, the last pass runs all ng groups, each in whole waves
+// of 148 CTAs; a group state costs four transfers of 115 KB per CTA.  The smallest modelled time over ng = 2 .. 32
+// decides.  The constants are fitted to measured times of the scan form on one batch element of 131072 tokens, 1024
+// tiles (ms measured / modelled; heads x groups): 1 x 8: 0.89 / 0.92, 1 x 16: 0.50 / 0.48, 1 x 32: 0.54 / 0.49,
+// 4 x 2: 3.40 / 3.69, 4 x 4: 1.82 / 1.85, 4 x 8: 1.79 / 1.87, 16 x 2: 5.64 / 5.95, 16 x 4: 6.21 / 6.68.
+constexpr double kStateTileUs = 2.8, kFullTileUs = 4.4, kGroupStateUs = 0.115, kTwoLaunchesUs = 20.0;
+double scan_pass_us(double ctas, double tiles_per_group, double tile_us) { return ceil(ctas / 148.0) * tiles_per_group * tile_us; }
 int tensor_scan_group(int BH, int slices, int NC, double* model_us = nullptr) {
   const int cpt = tc_stream_tile() / kChunk;
   const int tiles = (NC + cpt - 1) / cpt;
@@ -127,10 +131,10 @@ int tensor_scan_group(int BH, int slices, int NC, double* model_us = nullptr) {
   double best_us = 0.0;
   for (int ng = 2; ng <= 32 && ng <= tiles; ++ng) {
     const double tpg = (double)((tiles + ng - 1) / ng);
-    const double us = ceil((ng - 1) * c / 148.0) * tpg * 2.8 + ceil(ng * c / 148.0) * tpg * 4.4 + ng * c * 0.115;
+    const double us = scan_pass_us((ng - 1) * c, tpg, kStateTileUs) + scan_pass_us(ng * c, tpg, kFullTileUs) + ng * c * kGroupStateUs;
     if (ng == 2 || us < best_us) { best = ng; best_us = us; }
   }
-  if (model_us) *model_us = best_us + 20.0;   // two more launches
+  if (model_us) *model_us = best_us + kTwoLaunchesUs;
   const int G = (tiles + best - 1) / best * cpt;
   return G < NC ? G : NC;
 }
@@ -146,7 +150,7 @@ bool tensor_scan_pays(int BH, int NC, bool split) {
   double scan_us;
   tensor_scan_group(BH, slices, NC, &scan_us);
   const double seq_us = split ? ceil(9.0 * BH / 148.0) * tiles * (9 * BH >= 74 ? 3.3 : 2.6) + 10.0
-                              : ceil((double)slices * BH / 148.0) * tiles * 4.4;
+                              : scan_pass_us((double)slices * BH, tiles, kFullTileUs);
   return scan_us < 0.9 * seq_us;
 }
 

@@ -112,7 +112,12 @@ def test_scan_workspace_and_plan(L):
     assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 4, 16, 4096, 64, 64, 64, o) == 4 * 16 * 4096 * (64 + 1) * 2
     o32 = kb.make_opts(kb.KATA_F32)
     assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 4, 16, 4096, 64, 64, 64, o32) == 0
-    assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 8, 16, 4096, 64, 64, 64, o) == 0   # sequential
+    # sequential walk of the feature-split kernel: tile counters and the ticket, the scaled values and key scales of
+    # the pre-pass, nine shares of 17 KB per head and tile of 128 tokens
+    al = lambda x: (x + 255) // 256 * 256
+    BH, T, nt = 8 * 16, 4096, 32
+    assert kb.kata_workspace_bytes(kb.KATA_FN_CHUNKED, 8, 16, 4096, 64, 64, 64, o) == \
+        al((BH * nt + 1) * 4) + al(BH * T * 64 * 2) + al(BH * T * 2) + al(BH * 9 * nt * (128 * 128 + 128 * 8))
     assert kb.kata_scan_plan(kb.KATA_FN_CHUNKED, 8, 16, 4096, 64, 64, 64, o)[0] == 1
     o = kb.make_opts(kb.KATA_BF16, inter_chunk=kb.KATA_SCAN, scan_group=16, impl=kb.KATA_IMPL_SIMT)
     ng, g, rounds = kb.kata_scan_plan(kb.KATA_FN_CHUNKED, 1, 16, 8192, 64, 64, 64, o)

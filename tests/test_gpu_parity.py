@@ -103,8 +103,10 @@ def test_inter_chunk_auto_takes_the_scan_form_for_one_long_head():
     q, k, v = dev_tensors(w)
     o = kb.kata_fwd_chunked(q, k, v, inter_chunk=kb.KATA_INTER_AUTO)
     torch.cuda.synchronize()
-    # 16 groups of 3 tiles: the state-only pass, four scan rounds, the restarted pass
-    assert kb.kata_last_launch_count() == 6 and kb.kata_last_impl() == 2
+    # groups of a few tiles: the state-only pass, the scan rounds, the restarted pass
+    ng, _, rounds = kb.kata_scan_plan(kb.KATA_FN_CHUNKED, 1, 1, 6000, 64, 64, 64, kb.make_opts(kb.KATA_BF16, inter_chunk=kb.KATA_INTER_AUTO))
+    assert ng >= 8 and rounds >= 3
+    assert kb.kata_last_launch_count() == 2 + rounds and kb.kata_last_impl() == 2
     for (b, h), r in oracle_full(w).items():
         check(to_numpy64(o)[b, h], r, "bf16", "auto -> scan")
     w = inputs.gaussian_workload("auto_seq", "bf16", 1, 16, 1000, 64, 64, 64, 22)
@@ -239,6 +241,30 @@ def test_config5_recall_full():
     g = full_check(w, "chunked_seq")
     gq = run_form("quadratic", w)
     assert elem_err(gq, g) <= TOL["bf16"]
+
+
+def test_config4_scan_forms_in_sixteen_groups():
+    """Config 4 at T = 131072 with the chunk axis cut into 16 groups of 128 chunks: the state-only pass, four rounds
+    of the Hillis-Steele scan over the group states (section "Tree-scan inter-chunk reduction", appendix
+    "Associative-scan kernel"), the restarted pass.  Both scan entry points against the definition on sampled rows
+    and against the sequential walk on every element."""
+    T = 131072
+    w = inputs.config(4, T)
+    sg = (T // 64) // 16
+    for fn, mode in ((kb.KATA_FN_CHUNKED, kb.KATA_SCAN), (kb.KATA_FN_CHUNK_STATE_SCAN, kb.KATA_SEQUENTIAL)):
+        ng, cpg, rounds = kb.kata_scan_plan(fn, w.B, w.H, T, 64, 64, 64, kb.make_opts(kb.KATA_BF16, inter_chunk=mode, scan_group=sg))
+        assert ng == 16 and cpg == sg and rounds == 4
+    seq = run_form("chunked_seq", w)
+    picks = sample_picks(w, 192, 777)
+    ref = oracle_rows(w, picks)
+    for form in ("chunked_scan", "state_scan"):
+        g = run_form(form, w, scan_group=sg)
+        assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR
+        assert kb.kata_last_launch_count() >= 2 + 4, "state-only pass, four scan rounds, restarted pass"
+        assert np.all(np.isfinite(g))
+        assert elem_err(g, seq) <= TOL["bf16"] and row_err(g, seq) <= TOL["bf16"], form
+        got = np.stack([g[b, h, t] for b, h, t in picks])
+        check(got, ref, "bf16", f"c4 T={T} {form} in 16 groups, sampled rows")
 
 
 @pytest.mark.parametrize("T", [8192, 32768, 131072])
