@@ -63,7 +63,7 @@ enum { KATA_LAYOUT_DIRECT = 0, KATA_LAYOUT_PACKED = 1 }; /* kata_opts.state_layo
 enum { KATA_SEQUENTIAL = 0, KATA_SCAN = 1, KATA_INTER_AUTO = 2 };   /* kata_opts.inter_chunk */
 enum { KATA_IMPL_AUTO = 0, KATA_IMPL_SIMT = 1, KATA_IMPL_TENSOR = 2 }; /* kata_opts.impl */
 enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2, KATA_FN_DECODE_STEP = 3,
-       KATA_FN_BWD_QUADRATIC = 4 };
+       KATA_FN_BWD_QUADRATIC = 4, KATA_FN_BWD_CHUNKED = 5 };
 
 /*
  * Options (plain data; zero-initialise, then set struct_size = sizeof(kata_opts)).
@@ -204,6 +204,23 @@ int kata_decode_step(const void* q, const void* k, const void* v, void* out, flo
  */
 int kata_bwd_quadratic(const void* q, const void* k, const void* v, const void* dout, void* dq, void* dk, void* dv,
                        int B, int H, int T, int d_k, int d_v, const kata_opts* opts);
+
+/*
+ * The same gradients as kata_bwd_quadratic in O(T) work: the two-pass linear-state backward of the table
+ * "Training-step latency versus sequence length".  A forward sweep over the chunks carries the state of the forward
+ * pass (S = sum psi(k_hat) v^T, Z = sum psi(k_hat)), recomputes out_t and its normaliser and produces dq; a reverse
+ * sweep carries the state sum psi(q_hat_t) [dout_t / D_t, (dout_t . out_t) / D_t] of the tokens behind and produces dk
+ * and dv; the terms inside a chunk come from its C x C causal scores.  Arguments, layouts and error values as for
+ * kata_bwd_quadratic; C must be 64.  fp32 arithmetic on plain FMAs for both element types (bf16 tensors are widened on
+ * load and rounded once on store), every sum in a fixed order (bit-reproducible).  Supported: feature_order 2,
+ * feature_groups 1, d_k in {16, 32, 64}, d_v a multiple of 8 up to 64 (KATA_ERR_UNSUPPORTED_SHAPE otherwise,
+ * also for opts->impl = KATA_IMPL_TENSOR); inter_chunk, scan_group, state_layout are ignored; s_pre/z_pre/s_init/
+ * z_init must be null.  Rows whose normaliser is 0 and zero rows of q or k get zero gradients.
+ * Workspace: kata_workspace_bytes(KATA_FN_BWD_CHUNKED, B, H, T, d_k, d_v, 64, opts) bytes, about
+ * 4 (2 d_k + d_v + (d_v / 8)(d_k + 1) + 2) bytes per token and head (2.9 KB at d_k = d_v = 64).
+ */
+int kata_bwd_chunked(const void* q, const void* k, const void* v, const void* dout, void* dq, void* dk, void* dv,
+                     int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
 
 /*
  * Same computation as entry point `fn` (a KATA_FN_* value) but q,k,v,out are HOST pointers

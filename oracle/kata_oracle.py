@@ -32,6 +32,7 @@ Forms, all of which must agree to rounding:
   gate_decomposition   Proposition 1 (output-level gating)
   kata_quadratic_bwd   gradients of the definition with respect to q, k, v (chain rule
                    through o = N/D, the weights and the normalisation)
+  kata_bwd_rows    the same gradients for selected tokens only (long sequences)
 
 feature="identity" treats the rows of q,k as already-mapped features (the
 setting the scan appendix analyses): no normalisation, no lift.
@@ -256,6 +257,56 @@ def kata_quadratic_bwd(q, k, v, dout, feature: str = "psd_direct"):
         return out
 
     return through_normalisation(q, qh, dqh), through_normalisation(k, kh, dkh), dv
+
+
+def kata_bwd_rows(q, k, v, dout, rows_q, rows_k, C: int = 256):
+    """Rows of the gradients of `kata_quadratic_bwd` (feature 'psd_direct') for long sequences: dq for the tokens in
+    rows_q, dk and dv for the tokens in rows_k.  o_t and D_t of every token come from Algorithm 1 (chunk equations,
+    one chunk of features at a time); each requested row is then the sum the chain rule states, written out over
+    all the tokens it couples to:
+        u_t = dout_t / D_t,  c_t = (dout_t . o_t) / D_t,  s_ti = q_hat_t . k_hat_i,
+        dq_hat_t = 2 sum_{i<=t} s_ti (u_t . v_i - c_t) k_hat_i,
+        dk_hat_i = 2 sum_{t>=i} s_ti (u_t . v_i - c_t) q_hat_t,   dv_i = sum_{t>=i} s_ti^2 u_t,
+        dx = (dx_hat - x_hat (x_hat . dx_hat)) / ||x||.
+    Returns (dq [len(rows_q), d], dk [len(rows_k), d], dv [len(rows_k), d_v])."""
+    q = np.asarray(q, np.float64)
+    k = np.asarray(k, np.float64)
+    v = np.asarray(v, np.float64)
+    dout = np.asarray(dout, np.float64)
+    T, d = q.shape
+    qh, kh = normalize_rows(q), normalize_rows(k)
+    o = np.zeros_like(v)
+    D = np.zeros(T)
+    S = np.zeros((d * d, v.shape[1]))
+    Z = np.zeros(d * d)
+    for t0 in range(0, T, C):
+        sl = slice(t0, min(T, t0 + C))
+        FQ, FK = psi_direct(qh[sl]), psi_direct(kh[sl])
+        o[sl], _, D[sl] = chunk_output(FQ, FK, v[sl], S, Z)
+        S = S + FK.T @ v[sl]
+        Z = Z + FK.sum(axis=0)
+    invD = np.zeros(T)
+    invD[D != 0] = 1.0 / D[D != 0]
+    u = dout * invD[:, None]
+    c = np.sum(dout * o, axis=1) * invD
+
+    def through_normalisation(x, xh, dxh):
+        n = math.sqrt(float(np.sum(x * x)))
+        return (dxh - xh * np.dot(xh, dxh)) / n if n > 0 else np.zeros_like(x)
+
+    dq = np.zeros((len(rows_q), d))
+    for j, t in enumerate(rows_q):
+        s = kh[:t + 1] @ qh[t]
+        e = v[:t + 1] @ u[t] - c[t]
+        dq[j] = through_normalisation(q[t], qh[t], 2.0 * (s * e) @ kh[:t + 1])
+    dk = np.zeros((len(rows_k), d))
+    dv = np.zeros((len(rows_k), v.shape[1]))
+    for j, i in enumerate(rows_k):
+        s = qh[i:] @ kh[i]
+        e = u[i:] @ v[i] - c[i:]
+        dk[j] = through_normalisation(k[i], kh[i], 2.0 * (s * e) @ qh[i:])
+        dv[j] = (s * s) @ u[i:]
+    return dq, dk, dv
 
 
 def kata_decode_step(S, Z, q, k, v, feature: str = "psd_direct"):

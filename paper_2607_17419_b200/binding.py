@@ -20,11 +20,12 @@ KATA_SEQUENTIAL, KATA_SCAN, KATA_INTER_AUTO = 0, 1, 2
 KATA_IMPL_AUTO, KATA_IMPL_SIMT, KATA_IMPL_TENSOR = 0, 1, 2
 KATA_FN_QUADRATIC, KATA_FN_CHUNKED, KATA_FN_CHUNK_STATE_SCAN, KATA_FN_DECODE_STEP = 0, 1, 2, 3
 KATA_FN_BWD_QUADRATIC = 4
+KATA_FN_BWD_CHUNKED = 5
 KATA_FN_HOST_IO = 0x100
 KATA_OK, KATA_ERR_INVALID_ARG, KATA_ERR_WORKSPACE_TOO_SMALL, KATA_ERR_DEVICE_TIMEOUT = 0, -1, -4, -7
 
 EXPORTS = ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan", "kata_chunk_state_scan_static",
-           "kata_fwd_host", "kata_decode_step", "kata_bwd_quadratic",
+           "kata_fwd_host", "kata_decode_step", "kata_bwd_quadratic", "kata_bwd_chunked",
            "kata_workspace_bytes", "kata_scan_plan", "kata_host_plan", "kata_last_launch_count", "kata_last_impl",
            "kata_status_string",
            "kata_version")
@@ -79,6 +80,8 @@ def lib() -> ctypes.CDLL:
     L.kata_decode_step.restype = i
     L.kata_bwd_quadratic.argtypes = [ptr] * 7 + [i] * 5 + [ctypes.POINTER(KataOpts)]
     L.kata_bwd_quadratic.restype = i
+    L.kata_bwd_chunked.argtypes = [ptr] * 7 + [i] * 6 + [ctypes.POINTER(KataOpts)]
+    L.kata_bwd_chunked.restype = i
     L.kata_workspace_bytes.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(KataOpts)]
     L.kata_workspace_bytes.restype = ctypes.c_size_t
     L.kata_scan_plan.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(KataOpts)] + [ctypes.POINTER(i)] * 3
@@ -319,6 +322,32 @@ def kata_bwd_quadratic(q, k, v, dout, dq=None, dk=None, dv=None, *, workspace: O
                                   dk.data_ptr(), dv.data_ptr(), B, H, T, d_k, d_v, ctypes.byref(opts))
     if st != 0:
         raise KataError(st, "kata_bwd_quadratic")
+    return dq, dk, dv
+
+
+def kata_bwd_chunked(q, k, v, dout, dq=None, dk=None, dv=None, C: int = 64, *, workspace: Optional[Workspace] = None,
+                     stream=None, **opt_kw):
+    """The same gradients as ``kata_bwd_quadratic`` by the O(T) two-pass linear-state backward.  Returns (dq, dk, dv)
+    in the dtype of the inputs."""
+    import torch
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and dout.is_contiguous()):
+        raise ValueError("q, k, v, dout must be contiguous [B,H,T,d]")
+    B, H, T, d_k = q.shape
+    d_v = v.shape[-1]
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    opts = make_opts(_dtype_code(q), stream=stream, **opt_kw)
+    need = kata_workspace_bytes(KATA_FN_BWD_CHUNKED, B, H, T, d_k, d_v, C, opts)
+    ws = workspace if workspace is not None else _default_ws
+    ptr, size = ws.get(need, q.device)
+    opts.workspace, opts.workspace_bytes = ptr or None, size
+    st = lib().kata_bwd_chunked(q.data_ptr(), k.data_ptr(), v.data_ptr(), dout.data_ptr(), dq.data_ptr(),
+                                dk.data_ptr(), dv.data_ptr(), B, H, T, d_k, d_v, C, ctypes.byref(opts))
+    if st != 0:
+        raise KataError(st, "kata_bwd_chunked")
     return dq, dk, dv
 
 

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkata.so")
-SOURCES = ["kata_api.cu", "kata_simt_quadratic.cu", "kata_simt_bwd.cu", "kata_simt_chunked.cu", "kata_simt_order1.cu", "kata_tc.cu", "kata_tc_chunked.cu",
+SOURCES = ["kata_api.cu", "kata_simt_quadratic.cu", "kata_simt_bwd.cu", "kata_simt_bwd_chunked.cu", "kata_simt_chunked.cu", "kata_simt_order1.cu", "kata_tc.cu", "kata_tc_chunked.cu",
     "kata_tc_stream.cu", "kata_tc_split.cu", "kata_tc_stream_export.cu", "kata_tc_stream_restart.cu", "kata_tc_stream_state.cu", "kata_tc_quadratic.cu", "kata_tc_bwd.cu", "kata_tc_order1.cu", "kata_decode.cu", "kata_static.cu", "kata_selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]

@@ -765,9 +765,45 @@ int kata_fwd_host(int fn, const void* q_host, const void* k_host, const void* v_
   return KATA_OK;
 }
 
+int kata_bwd_chunked(const void* q, const void* k, const void* v, const void* dout, void* dq, void* dk, void* dv,
+                     int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts) {
+  Opts o;
+  int st = read_opts(opts, o);
+  if (st != KATA_OK) return st;
+  if (B < 1 || H < 1 || T < 1 || d_k < 1 || d_v < 1) return KATA_ERR_INVALID_ARG;
+  if (o.s_pre != nullptr || o.s_init != nullptr || o.z_init != nullptr) return KATA_ERR_INVALID_ARG;
+  const Problem p{q, k, v, nullptr, B, H, T, d_k, d_v, o.dtype, o.feature_order, o.groups};
+  if (C != kChunk || !simt_bwd_chunked_supported(p) || o.impl == KATA_IMPL_TENSOR) return KATA_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)B * H * (d_v / 8) > 2147483647LL) return KATA_ERR_UNSUPPORTED_SHAPE;
+  if (q == nullptr || k == nullptr || v == nullptr || dout == nullptr || dq == nullptr || dk == nullptr || dv == nullptr)
+    return KATA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) ||
+      !aligned16(dv))
+    return KATA_ERR_ALIGNMENT;
+  const size_t need = align_up(simt_bwd_chunked_workspace_elems(p) * sizeof(float));
+  if (o.workspace == nullptr || o.workspace_bytes < need) return KATA_ERR_WORKSPACE_TOO_SMALL;
+  if ((reinterpret_cast<uintptr_t>(o.workspace) & (kAlign - 1)) != 0) return KATA_ERR_ALIGNMENT;
+  st = check_arch();
+  if (st != KATA_OK) return st;
+  LaunchCtx ctx{o.stream, 0, KATA_OK};
+  simt_bwd_chunked(p, dout, dq, dk, dv, static_cast<float*>(o.workspace), ctx);
+  if (ctx.status == KATA_OK) {
+    g_last_launches = ctx.launches;
+    g_last_impl = KATA_IMPL_SIMT;
+  }
+  return ctx.status;
+}
+
 size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts) {
   const bool host_io = (fn & KATA_FN_HOST_IO) != 0;
   fn &= ~KATA_FN_HOST_IO;
+  if (fn == KATA_FN_BWD_CHUNKED) {
+    Opts o;
+    if (host_io || read_opts(opts, o) != KATA_OK || B < 1 || H < 1 || T < 1 || C != kChunk) return 0;
+    const Problem p{nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, o.dtype, o.feature_order, o.groups};
+    if (!simt_bwd_chunked_supported(p)) return 0;
+    return align_up(simt_bwd_chunked_workspace_elems(p) * sizeof(float));
+  }
   if (fn == KATA_FN_BWD_QUADRATIC) {    // C is ignored
     Opts o;
     if (host_io || read_opts(opts, o) != KATA_OK || B < 1 || H < 1 || T < 1 || !dim_ok(d_k) || !dim_ok(d_v)) return 0;

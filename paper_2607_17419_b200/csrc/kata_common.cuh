@@ -72,6 +72,9 @@ void simt_chunked(const Problem& p, const ScanPlan& plan, bool use_scan, float* 
 // Backward of the quadratic form (fp32 arithmetic; any supported shape and element type)
 size_t simt_bwd_workspace_elems(int BH, int T);
 void simt_bwd_quadratic(const Problem& p, const void* dout, void* dq, void* dk, void* dv, float* stats, LaunchCtx& ctx);
+bool simt_bwd_chunked_supported(const Problem& p);
+size_t simt_bwd_chunked_workspace_elems(const Problem& p);
+void simt_bwd_chunked(const Problem& p, const void* dout, void* dq, void* dk, void* dv, float* ws, LaunchCtx& ctx);
 
 // Backward of the quadratic form on the tensor cores (bf16, d_k = d_v = 64, full rank-one feature)
 size_t tc_bwd_workspace_bytes(const Problem& p);

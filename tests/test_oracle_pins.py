@@ -552,3 +552,35 @@ def test_backward_zero_rows_and_dead_denominators():
     v2[5] += 100.0
     dq3, dk3, dv3 = ko.kata_quadratic_bwd(q, k, v2, dout)
     assert np.allclose(dq3, dq, atol=1e-12) and np.allclose(dk3, dk, atol=1e-12) and np.allclose(dv3, dvv, atol=1e-12)
+
+
+def test_backward_rows_equal_the_backward_of_the_definition():
+    """`kata_bwd_rows` (the long-sequence helper: forward by the chunk equations, then each requested row as the sum
+    the chain rule states) against `kata_quadratic_bwd` on every row of a short sequence, including a zero key row,
+    a zero query row and a ragged last chunk; and against central differences of the definition for one row."""
+    rng = np.random.default_rng(77)
+    T, d, dv = 150, 8, 5
+    q, k, v, dout = (rng.standard_normal((T, n)) for n in (d, d, dv, dv))
+    k[3] = 0.0
+    q[10] = 0.0
+    rq, rk, rv = ko.kata_quadratic_bwd(q, k, v, dout)
+    rows = list(range(T))
+    for C in (64, 256, 7):
+        dq, dk, dvv = ko.kata_bwd_rows(q, k, v, dout, rows, rows, C=C)
+        for got, ref in ((dq, rq), (dk, rk), (dvv, rv)):
+            assert np.max(np.abs(got - ref)) <= 1e-10 * max(1.0, np.abs(ref).max())
+    # a subset in arbitrary order
+    sel = [149, 0, 64, 63, 3]
+    dq, dk, dvv = ko.kata_bwd_rows(q, k, v, dout, sel, sel[::-1])
+    assert np.allclose(dq, rq[sel], atol=1e-10) and np.allclose(dk, rk[sel[::-1]], atol=1e-10)
+    assert np.allclose(dvv, rv[sel[::-1]], atol=1e-10)
+    # central differences of L = sum(dout * o) in k[40]
+    L = lambda kk: float(np.sum(dout * ko.kata_quadratic(q, kk, v)[0]))
+    eps = 1e-6
+    num = np.zeros(d)
+    for a in range(d):
+        kp, km = k.copy(), k.copy()
+        kp[40, a] += eps
+        km[40, a] -= eps
+        num[a] = (L(kp) - L(km)) / (2 * eps)
+    assert np.allclose(ko.kata_bwd_rows(q, k, v, dout, [], [40])[1][0], num, rtol=1e-5, atol=1e-7)
