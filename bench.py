@@ -567,6 +567,23 @@ def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
     res["bwd_quadratic_c2_M2"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=flb / (ms * 1e-3) / 1e12,
                                       launches=kb.kata_last_launch_count(),
                                       impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
+    # O(T) two-pass backward against the quadratic-form backward on one batch element of 16 heads (the first T tokens
+    # of the headline workload): where the linear-state form takes over
+    gfull = torch.randn(v.shape, device=dev, generator=torch.Generator(device=dev).manual_seed(9)).to(torch.bfloat16)
+    cross = None
+    for Tb in (4096, 16384, 65536, T):
+        qb, kb_, vb, gb = (a[:, :, :Tb].contiguous() for a in (q, k, v, gfull))
+        dqb, dkb, dvb = torch.empty_like(qb), torch.empty_like(kb_), torch.empty_like(vb)
+        ms_c = timed(lambda: kb.kata_bwd_chunked(qb, kb_, vb, gb, dqb, dkb, dvb), reps=3, warm=1)
+        lc = kb.kata_last_launch_count()
+        ms_q = timed(lambda: kb.kata_bwd_quadratic(qb, kb_, vb, gb, dqb, dkb, dvb), reps=3, warm=1)
+        res[f"bwd_chunked_H16_T{Tb}"] = dict(ms=ms_c, tokens_per_s=Tb / (ms_c * 1e-3), launches=lc, impl="simt",
+                                             bwd_quadratic_ms=ms_q, speedup_over_quadratic=ms_q / ms_c)
+        if cross is None and ms_c < ms_q:
+            cross = Tb
+        del qb, kb_, vb, gb, dqb, dkb, dvb
+    res["bwd_chunked_crossover"] = dict(first_T_where_chunked_is_faster=cross, shapes="B=1 H=16 d=64 bf16, T in 4096, 16384, 65536, 131072")
+    del gfull
     # first-order feature (rows of q, k as features; matched d x d state, C = 128): shapes of the paper's scan
     # benchmark; HBM-bound, 512 algorithmic bytes per token and head (q, k, v read, o written)
     for Bo, To in ((1, 8192), (1, 131072), (4, 32768), (16, 8192), (32, 32768)):
