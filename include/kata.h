@@ -19,10 +19,19 @@
  *   - q, k: [B,H,T,d_k]; v, out: [B,H,T,d_v]; row-major, contiguous, 16-byte aligned,
  *     DEVICE pointers (except in kata_fwd_host), element type opts->dtype (fp32 or bf16).
  *   - All accumulation, the running state (S,Z) and the normaliser are fp32; out is rounded
- *     to the element type (round-to-nearest-even).
- *   - The caller owns every buffer.  The library allocates nothing, frees nothing and never
+ *     to the element type (round-to-nearest-even).  On the bf16 tensor-core kernels the OPERANDS of the matrix
+ *     products are bf16: the chunked forms read the running state through a bf16 copy taken once per tile of 128
+ *     tokens (S and Z are accumulated in fp32, but psi(q)^T S and psi(q)^T Z see them rounded), the intra-tile
+ *     weights (q.k)^2 are rounded to bf16 before they multiply the values, and the key scale 1/||k||^2 and the scaled
+ *     values v/||k||^2 are rounded separately.  The convex weights of the output gate therefore sum to 1 only to
+ *     about 2^-8, and a normaliser that is tiny against its terms (a query nearly orthogonal to every key before it)
+ *     can come out <= 0 from the rounded operands, in which case out = 0 as for an exact zero.  All of it stays
+ *     inside the 2e-2 tolerance of the bf16 tests.
+ *   - The caller owns every buffer.  The library allocates no device or host memory, frees nothing and never
  *     synchronises; all work is enqueued on opts->stream.  q,k,v are read-only; out and the
- *     workspace are fully overwritten (no pre-zeroing needed).
+ *     workspace are fully overwritten (no pre-zeroing needed).  One exception to "allocates nothing":
+ *     kata_fwd_host on its piecewise route creates, once per device and for the life of the process, two CUDA
+ *     streams and seven events, and takes a process-wide mutex for the duration of the call (see there).
  *   - Supported shapes: d_k, d_v in {16,32,64}; C = 64 (the chunked/scan forms), and C = 128 for
  *     feature_order 1 with bf16, d_k = d_v = 64 (the chunk size of the paper's scan benchmark; tensor-core
  *     path, no s_pre/z_pre); T >= 1 (any; the last chunk is zero-padded as in Algorithm 1 and truncated on
@@ -33,7 +42,11 @@
  *   - Return value: KATA_OK (0) or a negative kata_status.  Errors detectable on the host
  *     launch nothing.  No exceptions, no abort, no device trap.  A bounded device-side wait
  *     that expires writes KATA_ERR_DEVICE_TIMEOUT to *opts->device_status (if non-null),
- *     visible after the caller synchronises the stream; the kernel still terminates.
+ *     visible after the caller synchronises the stream; the kernel still terminates.  How long a launch
+ *     that has stalled takes to end: the waits of its warps run out side by side and a warp enters no further
+ *     wait once one has failed, so it is one limit, not their sum -- 0.1 s on the streaming, quadratic, backward
+ *     and first-order kernels (a limit on time), and on the feature-split chunked kernel 4 M polls of at most 1 us
+ *     each (between 0.1 s and 4 s) plus at most 2 s for a CTA that waits for the other CTAs of its head.
  */
 #ifndef KATA_H_
 #define KATA_H_
@@ -71,8 +84,8 @@ enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2,
  *  dtype          element type of q,k,v,out.
  *  feature_order  2: rank-one PSD lift of the normalised rows (default when 0 is passed).
  *                 1: rows of q,k are already-mapped features used as they are (no
- *                    normalisation, no lift; state d_k x d_v) -- the setting of the paper's
- *                    associative-scan appendix ("already-feature-mapped inputs").
+ *                    normalisation, no lift; state d_k x d_v) -- the setting analysed in the appendix
+ *                    "Associative-scan kernel", where the feature map has been applied beforehand.
  *  feature_groups 0 or 1: the full rank-one lift.  g = 2 or 4 (feature_order 2 only): the blockwise PSD map
  *                 psi_Mg(u) = (u_1 u_1^T, ..., u_g u_g^T) of the normalised row cut into g blocks of d_k/g
  *                 entries ("KATA-Mg"), with <psi(q),psi(k)> = sum_a (q_a . k_a)^2.  The state layouts then hold
@@ -156,7 +169,11 @@ int kata_fwd_quadratic(const void* q, const void* k, const void* v, void* out,
  *   D = Psi(Q_[c]) Z_[c] + P 1,  O_[c] = diag(D)^-1 N
  * (section "Chunkwise forward").  O(T) work, fp32 state.  opts->inter_chunk selects how
  * the inter-chunk recurrence is traversed; both give the same result up to fp32
- * re-association.  Workspace: kata_workspace_bytes(KATA_FN_CHUNKED, ...).
+ * re-association.  Workspace: kata_workspace_bytes(KATA_FN_CHUNKED, ...); the sequential walk on the tensor-core
+ * path (bf16, d_k = d_v = 64, feature_order 2, feature_groups 1, no state pointers) splits the state of a head over
+ * nine CTAs and needs about 1.36 KB per token and head there (scaled values, key scales, the CTAs' shares of the
+ * output and a counter per tile); the environment variable KATA_CHUNKED_KERNEL=stream selects the one-CTA-per-value-
+ * slice streaming kernel instead (no workspace; for comparisons).
  */
 int kata_fwd_chunked(const void* q, const void* k, const void* v, void* out,
                      int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
@@ -231,9 +248,12 @@ int kata_bwd_chunked(const void* q, const void* k, const void* v, const void* do
  * no state pointers in opts) are processed in up to sixteen pieces of the token axis: the copy in of the next piece
  * and the copy back of the previous one run on two streams owned by the library while the current piece is
  * computed, each piece starting from the state the previous one left ("Linear attention as a recurrence").  The
- * caller's stream waits for all of it, so the contract above is unchanged, and so is the result (bit-identical to
- * the one-pass call).  Calls that take this route are serialised inside the library; host memory that is not
- * pinned makes the copies synchronous.
+ * caller's stream waits for all of it -- also when a piece fails: the error is returned only after the caller's
+ * stream has been made to wait for every copy already queued on the library's streams -- so the contract above is
+ * unchanged.  The result is the same function as the one-pass call; the pieces run on the streaming kernel, which
+ * rounds at other places than the feature-split kernel of the one-pass call (both inside the bf16 tolerance).
+ * This route creates two streams and seven events per device on first use and keeps them; calls that take it are
+ * serialised inside the library by a process-wide mutex; host memory that is not pinned makes the copies synchronous.
  * The paper has no counterpart; this is the end-to-end path measured by the benchmark.
  */
 #define KATA_FN_HOST_IO 0x100
@@ -257,7 +277,9 @@ int kata_fwd_host(int fn, const void* q_host, const void* k_host, const void* v_
  *    (KATA_ERR_INVALID_ARG otherwise); if opts->scan_group is 0 the library picks the smallest
  *    power-of-two group size whose scratch fits the array.
  *  - If the scratch needed exceeds KATA_STATIC_SCRATCH_BYTES (large B*H with a small scan_group, or
- *    simply too many heads), nothing is launched and KATA_ERR_WORKSPACE_TOO_SMALL is returned.
+ *    simply too many heads), nothing is launched and KATA_ERR_WORKSPACE_TOO_SMALL is returned.  bf16 rows narrower
+ *    than 64 entries take the zero-padded route of the tensor-core kernels, whose padded copies of q, k, v and out
+ *    (4 * B*H*T * 128 bytes) must fit the array as well: about 65 thousand tokens over all heads.
  *  - The call allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine.
  *  - The first call on each device looks up the device address of the array (one
  *    cudaGetSymbolAddress, with that device current).  Make that first call outside any stream

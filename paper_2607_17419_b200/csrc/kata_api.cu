@@ -79,8 +79,7 @@ int check_shape(int fn, int B, int H, int T, int d_k, int d_v, int C) {
 }
 
 bool want_tensor(int fn, const Problem& p, const Opts& o) {
-  const bool scan = (fn == KATA_FN_CHUNK_STATE_SCAN) || (fn == KATA_FN_CHUNKED && o.inter_chunk == KATA_SCAN);
-  return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn, scan);
+  return o.impl != KATA_IMPL_SIMT && tc_supported(p, fn);
 }
 
 // The tensor-core backward covers bf16: the full rank-one feature with d_k = d_v = 64 or narrower rows zero-padded,
@@ -571,6 +570,19 @@ int host_pipelined(const Prepared& r, const PipePlan& pp, const void* q_host, co
             cudaStreamWaitEvent(hp->in, hp->start, 0) == cudaSuccess &&
             cudaStreamWaitEvent(hp->out, hp->start, 0) == cudaSuccess;
   int launches = 0;
+  int status = KATA_OK;
+  // On every way out the caller's stream is made to wait for whatever is queued on the library's two streams: the
+  // caller may reuse its buffers once its own stream is idle, whether the call succeeded or not.
+  auto join = [&]() {
+    bool j = cudaEventRecord(hp->in_done[0], hp->in) == cudaSuccess && cudaStreamWaitEvent(main, hp->in_done[0], 0) == cudaSuccess;
+    j = (cudaEventRecord(hp->out_done[0], hp->out) == cudaSuccess && cudaStreamWaitEvent(main, hp->out_done[0], 0) == cudaSuccess) && j;
+    if (!j) {           // last resort: the event calls themselves fail
+      cudaGetLastError();
+      cudaStreamSynchronize(hp->in);
+      cudaStreamSynchronize(hp->out);
+      cudaGetLastError();
+    }
+  };
   for (int i = 0; i < pp.pieces && ok; ++i) {
     const int b = i & 1;
     const int t0 = i * pp.piece_T;
@@ -597,7 +609,10 @@ int host_pipelined(const Prepared& r, const PipePlan& pp, const void* q_host, co
     po.z_pre = i + 1 < pp.pieces ? Z : nullptr;
     const int st = entry(KATA_FN_CHUNKED, in_buf(b, 0), in_buf(b, 1), in_buf(b, 2), out_buf(b), p.B, p.H, len, p.d_k,
                          p.d_v, C, &po);
-    if (st != KATA_OK) return st;
+    if (st != KATA_OK) {
+      status = st;
+      break;
+    }
     launches += g_last_launches;
     ok = cudaEventRecord(hp->comp_done[b], main) == cudaSuccess &&
          cudaStreamWaitEvent(hp->out, hp->comp_done[b], 0) == cudaSuccess &&
@@ -606,13 +621,14 @@ int host_pipelined(const Prepared& r, const PipePlan& pp, const void* q_host, co
          cudaEventRecord(hp->out_done[b], hp->out) == cudaSuccess;
   }
   // the caller's stream ends behind the last copies back (the last two pieces cover both event slots)
-  ok = ok && cudaStreamWaitEvent(main, hp->out_done[0], 0) == cudaSuccess &&
+  ok = ok && status == KATA_OK && cudaStreamWaitEvent(main, hp->out_done[0], 0) == cudaSuccess &&
        cudaStreamWaitEvent(main, hp->out_done[1], 0) == cudaSuccess;
+  g_last_launches = launches;
   if (!ok) {
     cudaGetLastError();
-    return KATA_ERR_CUDA;
+    join();
+    return status != KATA_OK ? status : KATA_ERR_CUDA;
   }
-  g_last_launches = launches;
   return KATA_OK;
 }
 

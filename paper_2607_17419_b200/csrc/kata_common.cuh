@@ -94,7 +94,7 @@ void decode_step(const void* q, const void* k, const void* v, void* out, float* 
                  int d_k, int d_v, int dtype, int layout, int order, int groups, LaunchCtx& ctx);
 
 // Tensor-core kernels (tcgen05/TMEM; bf16, d_k = d_v = 64)
-bool tc_supported(const Problem& p, int fn, bool scan);
+bool tc_supported(const Problem& p, int fn);
 size_t tc_quadratic_workspace_bytes(const Problem& p);
 void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx);
 void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx);

@@ -59,8 +59,18 @@ extern "C" int kata_chunk_state_scan_static(const void* q, const void* k, const 
       if (need <= (size_t)KATA_STATIC_SCRATCH_BYTES || g >= n_chunks) break;
     }
   }
-  // (invalid sizes give need == 0 and are reported by the pipeline entry point below)
+  // Validation first, with the codes of kata_chunk_state_scan: arguments it rejects (and the few it accepts without
+  // scratch) give need == 0 and go straight to it, before the array or the device is looked at.
+  if (need == 0) return kata_chunk_state_scan(q, k, v, out, B, H, T, d_k, d_v, C, &o);
   if (need > (size_t)KATA_STATIC_SCRATCH_BYTES) return KATA_ERR_WORKSPACE_TOO_SMALL;
+  {
+    int dev = -1, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return KATA_ERR_CUDA;
+    }
+    if (major != 10) return KATA_ERR_ARCH;
+  }
   void* scratch = nullptr;
   const int st = scratch_for_current_device(&scratch);
   if (st != KATA_OK) return st;

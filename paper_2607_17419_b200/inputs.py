@@ -169,6 +169,22 @@ def recall_workload(name: str, dtype: str, B: int, H: int, T: int, d_k: int, d_v
     return _finish(name, dtype, B, H, T, d_k, d_v, C, seed, q, k, v)
 
 
+def near_orthogonal_workload(name: str, dtype: str, B: int, H: int, T: int, d_k: int, d_v: int, C: int, seed: int,
+                             span: int = 48, every: int = 97, eps: float = 0.125) -> Workload:
+    """Gaussian rows whose keys live in the first ``span`` coordinates; every ``every``-th query ("probe" rows
+    t = every - 1, 2 every - 1, ...) has its part inside that span scaled by ``eps`` (a power of two), so that it is
+    nearly orthogonal to every key up to and including its own: small normaliser, output still of order one."""
+    q = normal(seed, 0, B * H * T * d_k).reshape(B, H, T, d_k)
+    k = normal(seed, 1, B * H * T * d_k).reshape(B, H, T, d_k)
+    v = normal(seed, 2, B * H * T * d_v)
+    k[..., span:] = 0.0
+    probes = np.arange(every - 1, T, every)
+    if dtype == "bf16":                      # scale the rounded values, so that the scaling is exact
+        q = bf16_bits_to_f64(f32_to_bf16_bits(q.astype(np.float32)).reshape(q.shape))
+    q[:, :, probes, :span] *= eps
+    return _finish(name, dtype, B, H, T, d_k, d_v, C, seed, q.reshape(-1), k.reshape(-1), v)
+
+
 def nonnegative_workload(name: str, dtype: str, B: int, H: int, T: int, d_k: int, d_v: int,
                          C: int, seed: int) -> Workload:
     """|N(0,1)| features for q,k (already-mapped first-order features), N(0,1) values."""

@@ -103,3 +103,24 @@ def test_bounded_waits_time_out_cleanly_and_the_stream_stays_usable():
         g = run(form, *dev_tensors(w))
         for (b, h), r in oracle_full(w).items():
             check(g[b, h], r, "bf16", f"after a timed-out launch/{form} head ({b},{h})")
+
+
+@pytest.mark.parametrize("form", list(FORMS))
+def test_queries_nearly_orthogonal_to_every_key(form):
+    """Small normalisers: probe queries whose cosine to every key (their own included) is about a tenth of a
+    typical one, so the normaliser is about a hundredth of its usual size while the output stays of order one.  The
+    kernels read the state and the weights through bf16 operands; the output must still match the definition, and
+    it must not have fallen into the `normaliser <= 0 -> out = 0` branch."""
+    T, every = 1500, 97
+    w = inputs.near_orthogonal_workload("near_orth", "bf16", 1, 2, T, 64, 64, 64, 606, every=every)
+    probes = np.arange(every - 1, T, every)
+    ref = oracle_full(w)
+    D = {bh: ko.kata_quadratic(w.q_ref[bh], w.k_ref[bh], w.v_ref[bh])[2] for bh in ref}
+    g = run(form, *dev_tensors(w))
+    for (b, h), r in ref.items():
+        d = D[(b, h)]
+        others = np.setdiff1d(np.arange(200, T), probes)
+        assert np.median(d[probes[2:]] / (probes[2:] + 1)) < 0.1 * np.median(d[others] / (others + 1)), "the probes are not small"
+        check(g[b, h], r, "bf16", f"near-orthogonal/{form} head ({b},{h})")
+        check(g[b, h][probes], r[probes], "bf16", f"near-orthogonal/{form} probe rows, head ({b},{h})")
+        assert np.all(np.abs(g[b, h][probes]).max(axis=1) > 0), "a probe row came out as 0: its normaliser was lost"

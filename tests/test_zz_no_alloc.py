@@ -15,7 +15,7 @@ from paper_2607_17419_b200 import binding as kb
 from paper_2607_17419_b200 import build as kbuild
 from paper_2607_17419_b200 import inputs
 
-from helpers import TOL, dev_tensors, elem_err, row_err, to_numpy64
+from helpers import TOL, check, dev_tensors, elem_err, oracle_full, row_err, to_numpy64
 
 pytestmark = pytest.mark.gpu
 
@@ -37,13 +37,21 @@ def test_static_scratch_matches_workspace_entry_point(dtype, B, H, T, d):
     ref = kb.kata_chunk_state_scan(q, k, v)
     torch.cuda.synchronize()
     r = to_numpy64(ref)
-    for attempt in range(2):                      # two calls in a row share the one scratch array
-        out = torch.full_like(v, float("nan"))
+    oracle = oracle_full(w)
+    outs = [torch.full_like(v, float("nan")) for _ in range(3)]
+    free = []
+    for attempt, out in enumerate(outs):          # calls in a row share the one scratch array
         assert call_static(q, k, v, out, B, H, T, d) == 0
         torch.cuda.synchronize()
+        free.append(torch.cuda.mem_get_info()[0])
+    # the central claim: no device memory is taken by the second and later calls (the first may load the module)
+    assert free[1] == free[2], free
+    for attempt, out in enumerate(outs):
         g = to_numpy64(out)
         assert np.all(np.isfinite(g)), attempt
         assert elem_err(g, r) <= TOL[dtype] and row_err(g, r) <= TOL[dtype], attempt
+        for (b, h), ref_bh in oracle.items():     # and against the definition, not only against its sibling
+            check(g[b, h], ref_bh, dtype, f"static entry, call {attempt}, head ({b},{h})")
     # a different problem in between, then the first one again
     w2 = inputs.gaussian_workload("noalloc2", dtype, 1, 3, 1111, d, d, 64, 32)
     q2, k2, v2 = dev_tensors(w2)
@@ -70,6 +78,9 @@ def test_static_scratch_rejects_what_does_not_fit():
     assert call_static(q, k, v, out, 8, 16, 1 << 17, 64, scan_group=1) == -4
     # state export is not offered by this entry point
     assert call_static(q, k, v, out, 1, 2, 256, 64, s_pre=4096, z_pre=8192) == -1
+    # invalid arguments come back with the codes of kata_chunk_state_scan, before the scratch is looked up
+    assert call_static(q, k, v, out, 1, 2, 0, 64) == -1          # T = 0
+    assert call_static(q, k, v, out, 1, 2, 256, 48) == -2         # unsupported row width
     # and a normal call still works afterwards
     assert call_static(q, k, v, out, 1, 2, 256, 64) == 0
     torch.cuda.synchronize()
