@@ -142,13 +142,13 @@ int tensor_scan_group(int BH, int slices, int NC, double* model_us = nullptr) {
 // sequential walk's.  The sequential walk is the feature-split kernel where it applies (nine CTAs per head in whole
 // waves of 148, about 3.3 us a tile of 128 tokens with the GPU full and 2.6 us with a few heads), else the streaming
 // kernel (one CTA per head and value slice, 4.4 us a tile).
-bool tensor_scan_pays(int BH, int NC, bool split) {
+bool tensor_scan_pays(int BH, int NC, int split_ctas) {   // split_ctas: CTAs per head of the feature-split kernel, 0 = not used
   const int cpt = tc_stream_tile() / kChunk;
   const int tiles = (NC + cpt - 1) / cpt;
   const int slices = tc_chunked_slices();
   double scan_us;
   tensor_scan_group(BH, slices, NC, &scan_us);
-  const double seq_us = split ? ceil(9.0 * BH / 148.0) * tiles * (9 * BH >= 74 ? 3.3 : 2.6) + 10.0
+  const double seq_us = split_ctas > 0 ? ceil((double)split_ctas * BH / 148.0) * tiles * (split_ctas * BH >= 74 ? 3.3 : 2.6) + 10.0
                               : scan_pass_us((double)slices * BH, tiles, kFullTileUs);
   return scan_us < 0.9 * seq_us;
 }
@@ -370,7 +370,7 @@ int prepare(int fn, const void* q, const void* k, const void* v, void* out, int 
     Opts scan = r.o;
     scan.inter_chunk = KATA_SCAN;
     r.o.inter_chunk = KATA_SEQUENTIAL;
-    if (C == kChunk && want_tensor(fn, kp, r.o) && want_tensor(fn, kp, scan) && tensor_scan_pays(B * H, (T + C - 1) / C, r.o.s_init == nullptr && tc_split_supported(kp) && !stream_kernel_forced()))
+    if (C == kChunk && want_tensor(fn, kp, r.o) && want_tensor(fn, kp, scan) && tensor_scan_pays(B * H, (T + C - 1) / C, (r.o.s_init == nullptr && tc_split_supported(kp) && !stream_kernel_forced()) ? tc_split_ctas_per_head(kp) : 0))
       r.o.inter_chunk = KATA_SCAN;
   }
   r.tensor = want_tensor(fn, kp, r.o);

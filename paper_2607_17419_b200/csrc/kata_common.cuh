@@ -101,6 +101,7 @@ void tc_chunked_stream(const Problem& p, int* device_status, LaunchCtx& ctx);
 // Sequential chunked form with the feature axis of the state split over the CTAs of a head (kata_tc_split.cu)
 bool tc_split_supported(const Problem& p);
 size_t tc_split_workspace_bytes(const Problem& p);
+int tc_split_ctas_per_head(const Problem& p);
 void tc_chunked_split(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx);
 // State hand-off and groups of tiles for the second build of the streaming kernel (zero-initialise, then set).
 struct StreamIO {

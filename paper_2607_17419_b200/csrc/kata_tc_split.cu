@@ -58,19 +58,20 @@ using namespace umma;
 
 constexpr int D = 64;
 constexpr int CT = 128;            // tokens per tile
-constexpr int NBP = 4;             // block pairs per CTA
-constexpr int NCTA = 9;            // CTAs of a head: 36 block pairs / 4
+// CTAs of a head (template parameter NCTA): 36 block pairs / 4 (full lift), 20 / 4 or 20 / 2 (two feature groups), 12 / 2 (four)
+constexpr int BP_MAX = 40;
 constexpr int NTHREADS = 896;
 constexpr int kPrefetchTiles = 4;    // tiles between a tile's L2 prefetch and its load
-constexpr int kRowsPerCta = 15;     // query rows of a tile one CTA finishes (9 x 15 >= 128)
+constexpr int kRowSlots = 15;        // query rows of a tile the combine team finishes per pass (8 threads each)
 constexpr int W_TMA = 0, W_U = 1, W_R = 2, W_I = 3, W_K0 = 4, W_Q0 = 12, W_S0 = 16, W_E0 = 20, W_O0 = 24;
 
-// ---- TMEM columns ----
-constexpr uint32_t COL_S = 0;      // 2 x 80: state tiles (lanes = state rows)
-constexpr uint32_t COL_PSIQ = 160; // 128: weighted query products as bf16 pairs (lanes = tokens), 32 per block pair
-constexpr uint32_t COL_ACC = 288;  // 2 x 80: this CTA's share of [N | D] (lanes = tokens)
-constexpr uint32_t COL_SC = 448;   // 2 x 16 fp32 scores (tile & 1)
-constexpr uint32_t COL_P = 480;    // 8: bf16 weights
+// ---- TMEM columns; NM = accumulator tiles (of 128 state rows = 2 block pairs) per CTA ----
+constexpr uint32_t COL_S = 0;      // NM x 80: state tiles (lanes = state rows)
+constexpr uint32_t COL_ACC = 288;  // 2 x 80: this CTA's share of [N | D] (lanes = tokens), double-buffered
+// weighted query products as bf16 pairs (lanes = tokens), 32 columns per block pair
+template <int NM> struct Cols { static constexpr uint32_t PSIQ = NM == 2 ? 160u : 208u, SC = NM == 2 ? 448u : 80u; };
+// fp32 scores, 16 columns per (key run, feature group); the bf16 weights of a run overwrite the start of its scores
+// (at most 4 (run, group) tiles = 64 columns with two accumulator tiles, 8 = 128 columns with one)
 constexpr uint32_t TMEM_COLS = 512;
 
 // ---- shared memory (1024-byte aligned tiles of 128-byte rows, 128B swizzle) ----
@@ -100,24 +101,27 @@ enum {
   B_ACC_FREE = 11,   // [2] ... and has been copied out of it (128 threads of the share team)
   B_STG_FULL = 13,   // [2] the share of a tile is staged (128 threads of the share team); one barrier per store thread
   B_STG_FREE = 15,   // the bulk store has read the staging tile
-  B_DRAIN = 16,
-  B_COUNT = 17
+  B_A_DONE = 16,     // phase A of a tile is complete (16 warps)
+  B_DRAIN = 17,
+  B_COUNT = 18
 };
 static_assert(B_COUNT * 8 <= 256, "barrier block");
-constexpr int kBarA = 2;                    // named barrier that ends phase A
-constexpr int kBarAThreads = 32 * 20;       // TMA producer, the three MMA issuers, key, query and state teams
+constexpr int kBarA = 2;                    // named barrier that ends phase A (full lift)
+constexpr int kBarAThreads = 32 * 19;       // TMA producer, update and read issuers, key, query and state teams
 
 struct BlockPairs {
-  unsigned char g[NCTA * NBP], h[NCTA * NBP], w[NCTA * NBP];
+  unsigned char g[BP_MAX], h[BP_MAX], w[BP_MAX];
 };
 
 struct SplitArgs {
   __nv_bfloat16* out;
   const __nv_bfloat16* rscale;   // [BH][T] bf16: 1 / ||k||^2 (pre-pass)
-  unsigned char* share;          // [BH][NCTA][ntiles] blocks: [128 rows][64 fp16 numerators / scale, 16-byte pieces swizzled by row] | [128][normaliser, scale] fp32
+  unsigned char* share;          // [BH][ncta][ntiles] blocks: [128 rows][64 fp16 numerators / scale, 16-byte pieces swizzled by row] | [128][normaliser, scale] fp32
   unsigned* counter;             // [BH][ntiles]: CTAs of the head that have written their share of the tile
   int* device_status;
   int T, ntiles;
+  int ncta;                      // CTAs per head
+  int groups;                    // feature groups of the blockwise map (1 = the full lift)
   long long* prof;               // profiling build only: [CTA][5 teams][8] cycle counts
   BlockPairs bp;
 };
@@ -208,6 +212,7 @@ __global__ void __launch_bounds__(256) split_prescale_kernel(const __nv_bfloat16
   if (part == 0) rscale[row] = __float2bfloat16_rn(r2);
 }
 
+template <int NM, int G, int NCTA>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ SplitArgs args) {
@@ -235,6 +240,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     mbar_init(bar(B_MMA_DONE), 2);
     mbar_init(bar(B_STG_FREE), 1);
+    mbar_init(bar(B_A_DONE), 16);
     mbar_init(bar(B_DRAIN), 2);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
@@ -257,10 +263,22 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   // the other eight CTAs of its head, and with tickets those are running or next in line whatever order the blocks
   // are dispatched in.
   const unsigned ticket = *ticket_s;
-  const int bh = (int)(ticket / NCTA);
-  const int cta_head = (int)(ticket % NCTA);                  // CTA of the head
-  const int chunk = cta_head;                                 // 16-key run of every tile this CTA weighs (CTA 8: none)
-  const bool has_intra = chunk < 8;
+  constexpr int NBP = 2 * NM;                                 // block pairs of this CTA
+  constexpr uint32_t COL_PSIQ = Cols<NM>::PSIQ, COL_SC = Cols<NM>::SC;
+  constexpr int ncta = NCTA;
+  constexpr int MAXRUN = NCTA < 8 ? 2 : 1;                     // key runs a CTA can have
+  // With one run and one group the scores are double-buffered and the weights have columns of their own, so that the
+  // scores of a tile can be issued as soon as its keys and queries have landed; otherwise one buffer, the weights
+  // over the start of the scores, and the score MMAs wait for the apply MMA of the tile before.
+  constexpr bool SC2 = MAXRUN == 1 && G == 1;
+  constexpr int kRowsPerCta = (CT + NCTA - 1) / NCTA;          // query rows of a tile this CTA finishes
+  constexpr uint32_t COL_P = 480;
+  const int bh = (int)(ticket / ncta);
+  const int cta_head = (int)(ticket % ncta);                  // CTA of the head
+  // The eight 16-key runs of a tile are dealt round-robin to the CTAs of the head: run cta_head, and run
+  // cta_head + ncta where that is still below 8 (heads of fewer than eight CTAs).
+  const int nrun = (cta_head < 8 ? 1 : 0) + (cta_head + ncta < 8 ? 1 : 0);
+  const bool has_intra = nrun > 0;
   bool ok = true;
 #if KATA_SPLIT_PROF
   long long pacc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, plast = clock64();
@@ -275,14 +293,31 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   auto wwait = [&](int b, uint32_t parity) { return wait_or_abort_counted(bar(b), parity, abort_flag); };
   // the wait that opens tile j + 1 for every team: the MMAs of tile j are complete
   auto mma_done = [&](int j) { return j < 0 ? true : wwait(B_MMA_DONE, j & 1); };
-  // end of phase A.  A team that gave up keeps arriving, so that nobody is left waiting at the named barrier.
-  auto phase_a_done = [&]() { asm volatile("bar.sync %0, %1;" ::"n"(kBarA), "n"(kBarAThreads) : "memory"); };
+  // End of phase A.  Two forms, chosen by measurement (c4, ms: full lift 3.34 / 3.73, two groups 3.63 / 2.99, four
+  // groups 3.05 / 3.03): a named barrier that the issuers, the TMA producer and the sixteen warps of the key, query
+  // and state teams all wait at, or an mbarrier on which the teams only arrive (and go on to wait for the MMAs) and
+  // for which only the issuers and the producer wait.  A team that gave up keeps arriving in both.
+  constexpr bool kArriveOnly = G != 1;
+  constexpr bool kRollIssue = G != 1;
+  auto phase_a_arrive = [&]() {
+    if (kArriveOnly) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_A_DONE));
+    } else {
+      asm volatile("bar.sync %0, %1;" ::"n"(kBarA), "n"(kBarAThreads) : "memory");
+    }
+  };
+  auto phase_a_wait = [&](int j) {
+    if (kArriveOnly) return wwait(B_A_DONE, j & 1);
+    asm volatile("bar.sync %0, %1;" ::"n"(kBarA), "n"(kBarAThreads) : "memory");
+    return true;
+  };
   // A staged share goes to global memory as one bulk copy, issued by one thread; once the copy of the tile before is
   // complete that tile is published (a counter per head and tile, released at GPU scope).  The release waits for
   // memory operations of the whole SM that are in flight, the loads of the combine team among them; the share team
   // only ever waits for a copy to have read the staging tile.
   auto store_thread = [&]() {
-    unsigned char* mine = args.share + ((size_t)bh * NCTA + cta_head) * ntiles * kShareBytes;
+    unsigned char* mine = args.share + ((size_t)bh * ncta + cta_head) * ntiles * kShareBytes;
     unsigned* cnt = args.counter + (size_t)bh * ntiles;
     int prev = -1;
     for (int j = 0; j < ntiles; ++j) {
@@ -328,7 +363,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int j = 2; j < 2 + kPrefetchTiles; ++j) prefetch(j);
       }
       for (int j = 0; j < ntiles; ++j) {
-        phase_a_done();                 // keys and queries of tile j have been read (teams) and multiplied (score MMA)
+        ok = ok && phase_a_wait(j);                 // keys and queries of tile j have been read (teams) and multiplied (score MMA)
         if (j + 2 < ntiles) {
           if (lane == 0 && ok) {
             load(B_K_FULL, OFF_KRAW, &tmK, j + 2);
@@ -348,7 +383,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const int b = j & 1;
         ok = ok && wwait(B_V_FULL + b, (j >> 1) & 1);
         TICK(0);
-        phase_a_done();
+        ok = ok && phase_a_wait(j);
         TICK(1);
         if (lane == 0) {
           if (ok) {
@@ -356,45 +391,61 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const uint32_t vp = sbase + OFF_VP + b * 16384;
             const uint64_t dbv = smem_desc(0, sbase + OFF_COL64 + 32 * b - vp, 1024, kSwizzle128B);
 #pragma unroll
-            for (int m = 0; m < 2; ++m) {
+            for (int m = 0; m < NM; ++m) {
               const uint32_t pa = sbase + OFF_PSIK + m * 32768;
+              // (whether these loops are unrolled changes how the update and the read chains interleave in the pipe:
+              // c4, ms, unrolled / rolled: full lift 3.35 / 3.70, two groups 3.90 / 2.99, four groups 3.08 / 3.03)
+              if (kRollIssue) {
+#pragma unroll 1
+                for (int ks = 0; ks < 8; ++ks)
+                  mma_f16_ss(tb + COL_S + m * 80, at(da, pa + ks * 2048), at(dbv, vp + ks * 2048), idesc_u, (j > 0 || ks > 0) ? 1u : 0u);
+              } else {
 #pragma unroll
-              for (int ks = 0; ks < 8; ++ks)
-                mma_f16_ss(tb + COL_S + m * 80, at(da, pa + ks * 2048), at(dbv, vp + ks * 2048), idesc_u, (j > 0 || ks > 0) ? 1u : 0u);
+                for (int ks = 0; ks < 8; ++ks)
+                  mma_f16_ss(tb + COL_S + m * 80, at(da, pa + ks * 2048), at(dbv, vp + ks * 2048), idesc_u, (j > 0 || ks > 0) ? 1u : 0u);
+              }
             }
           }
           mma_commit(bar(B_MMA_DONE));
         }
         __syncwarp();
         TICK(2);
-        TICK(3);
       }
       TOCK(0);
     } else if (warp == W_R) {
-      // =========================== read issuer: ACC = Psi(Q) [S | Z] + P_c [V' | r]_c ===========================
+      // =========================== read issuer: ACC = Psi(Q) [S | Z] + sum over this CTA's key runs c of P_c [V' | r]_c ===========================
       const uint32_t idesc_r = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);
       for (int j = 0; j < ntiles; ++j) {
         const int b = j & 1;
         if (has_intra) ok = ok && wwait(B_V_FULL + b, (j >> 1) & 1);
         if (j >= 2) ok = ok && wwait(B_ACC_FREE + b, ((j >> 1) - 1) & 1);          // share of tile j - 2 copied out
-        phase_a_done();
+        ok = ok && phase_a_wait(j);
         if (lane == 0) {
           if (ok) {
             tc_fence_after();
             if (j >= 1) {
 #pragma unroll
-              for (int m = 0; m < 2; ++m) {
+              for (int m = 0; m < NM; ++m) {
                 const uint32_t sn = sbase + OFF_SNAP + m * 16384;
                 const uint64_t db = smem_desc(0, sbase + OFF_COL64 + 32 * (2 + m) - sn, 1024, kSwizzle128B);
+                if (kRollIssue) {
+#pragma unroll 1
+                  for (int ks = 0; ks < 8; ++ks)
+                    mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_PSIQ + m * 64 + ks * 8, at(db, sn + ks * 2048), idesc_r, (m > 0 || ks > 0) ? 1u : 0u);
+                } else {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                  mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_PSIQ + m * 64 + ks * 8, at(db, sn + ks * 2048), idesc_r, (m > 0 || ks > 0) ? 1u : 0u);
+                  for (int ks = 0; ks < 8; ++ks)
+                    mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_PSIQ + m * 64 + ks * 8, at(db, sn + ks * 2048), idesc_r, (m > 0 || ks > 0) ? 1u : 0u);
+                }
               }
             }
             if (has_intra) {
               const uint32_t vp = sbase + OFF_VP + b * 16384;
               const uint64_t dbv = smem_desc(0, sbase + OFF_COL64 + 32 * b - vp, 1024, kSwizzle128B);
-              mma_f16_ts(tb + COL_ACC + b * 80, tb + COL_P, at(dbv, vp + chunk * 2048), idesc_r, j >= 1 ? 1u : 0u);
+#pragma unroll
+              for (int r = 0; r < MAXRUN; ++r)   // the weights of run r sit at the start of its scores
+                if (r < nrun) mma_f16_ts(tb + COL_ACC + b * 80, SC2 ? tb + COL_P : tb + COL_SC + r * G * 16, at(dbv, vp + (cta_head + r * ncta) * 2048), idesc_r,
+                           (j >= 1 || r > 0) ? 1u : 0u);
             }
           }
           mma_commit(bar(B_ACC_FULL + b));
@@ -403,38 +454,47 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         __syncwarp();
       }
     } else {
-      // =========================== score issuer: Q K_c^T for this CTA's 16 keys (opens phase A) ===========================
+      // =========================== score issuer: Q_g K_c,g^T per feature group g for this CTA's key runs c (opens phase A) ===========================
       const uint32_t idesc_s = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 16);
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
       for (int j = 0; j < ntiles; ++j) {
         if (has_intra) {
           const int s = j & 1;
-          const uint32_t qa = sbase + OFF_QRAW + s * 16384, ka = sbase + OFF_KRAW + s * 16384 + chunk * 2048;
-          ok = ok && mma_done(j - 1);   // the apply MMA of tile j - 1 has read the weights; their columns may be rewritten
+          const uint32_t qa = sbase + OFF_QRAW + s * 16384;
+          if (!SC2) ok = ok && mma_done(j - 1);   // the apply MMA of tile j - 1 has read the weights; their columns take the scores
           ok = ok && wwait(B_K_FULL + s, (j >> 1) & 1) && wwait(B_Q_FULL + s, (j >> 1) & 1);
           if (lane == 0) {
             if (ok) {
               tc_fence_after();
+              // per key run and feature group: the 64 / G features of the group in steps of 16
+              constexpr int ksg = 4 / G;
 #pragma unroll
-              for (int ks = 0; ks < 4; ++ks) mma_f16_ss(tb + COL_SC + 16 * s, at(dk, qa + ks * 32), at(dk, ka + ks * 32), idesc_s, ks > 0 ? 1u : 0u);
+              for (int r = 0; r < MAXRUN; ++r) {
+                if (r < nrun) {
+                  const uint32_t ka = sbase + OFF_KRAW + s * 16384 + (cta_head + r * ncta) * 2048;
+#pragma unroll
+                  for (int ks = 0; ks < 4; ++ks)
+                    mma_f16_ss(tb + COL_SC + (SC2 ? s : r * G + ks / ksg) * 16, at(dk, qa + ks * 32), at(dk, ka + ks * 32), idesc_s, (ks % ksg) > 0 ? 1u : 0u);
+                }
+              }
             }
             mma_commit(bar(B_SC_FULL + s));
           }
           __syncwarp();
         }
-        phase_a_done();
+
       }
     }
   } else if (warp < W_Q0) {
     regs_release<56>();
-    // =========================== key teams (thread = token; team m = accumulator tile m) ===========================
-    const int m = (warp - W_K0) >> 2;
+    // =========================== key teams (thread = token; a team of four warps builds NM of the block pairs) ===========================
+    const int m = (warp - W_K0) >> 2;   // team: with two accumulator tiles, tile m; with one, its block pair m
     const int t = ((warp - W_K0) & 3) * 32 + lane;
-    int pg[2], ph[2];
+    int pg[NM], ph[NM];
 #pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      pg[e] = args.bp.g[cta_head * NBP + 2 * m + e];
-      ph[e] = args.bp.h[cta_head * NBP + 2 * m + e];
+    for (int e = 0; e < NM; ++e) {
+      pg[e] = args.bp.g[cta_head * NBP + NM * m + e];
+      ph[e] = args.bp.h[cta_head * NBP + NM * m + e];
     }
     const unsigned short* rs = reinterpret_cast<const unsigned short*>(args.rscale) + (size_t)bh * args.T;
     unsigned short r_next = (m == 0 && t < args.T) ? rs[t] : (unsigned short)0;
@@ -452,20 +512,20 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           r_next = (j + 1 < ntiles && tn < args.T) ? rs[tn] : (unsigned short)0;
         }
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
+        for (int e = 0; e < NM; ++e) {
           const uint4 ra = lds128(kraw + sw128_offset(t, pg[e]));
           const uint4 rb = lds128(kraw + sw128_offset(t, ph[e]));
           const uint32_t ga[4] = {ra.x, ra.y, ra.z, ra.w}, gb[4] = {rb.x, rb.y, rb.z, rb.w};
           uint32_t pr[32];
           products8x8<false>(ga, gb, 0u, pr);
-          const uint32_t dst = sbase + OFF_PSIK + (2 * m + e) * 16384;
+          const uint32_t dst = sbase + OFF_PSIK + (NM * m + e) * 16384;
 #pragma unroll
           for (int i = 0; i < 8; ++i) sts128(dst + sw128_offset(t, i), pr[4 * i], pr[4 * i + 1], pr[4 * i + 2], pr[4 * i + 3]);
         }
         fence_async_smem();
       }
       TICK(2);
-      phase_a_done();
+      phase_a_arrive();
       TICK(3);
     }
     if (warp == W_K0) TOCK(1);
@@ -502,28 +562,37 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
       }
       TICK(2);
-      if (has_intra) {                  // weights P = (Q K_c^T)^2, causal inside the tile
+      if (has_intra) {                  // weights P_c = sum_g (Q_g K_c,g^T)^2, causal inside the tile
         ok = ok && wwait(B_SC_FULL + b, (j >> 1) & 1);
         TICK(3);
         if (ok) {
           tc_fence_after();
-          uint32_t y[16], pk[8];
-          tmem_ld16(tmem_addr(tb, q4 * 32, COL_SC + 16 * b), y);
-          tmem_wait_ld(y);
 #pragma unroll
-          for (int c = 0; c < 16; c += 2) {
-            float a = __uint_as_float(y[c]), bq = __uint_as_float(y[c + 1]);
-            a = (chunk * 16 + c <= t) ? a * a : 0.f;
-            bq = (chunk * 16 + c + 1 <= t) ? bq * bq : 0.f;
-            pk[c >> 1] = pack_bf16(a, bq);
+          for (int r = 0; r < MAXRUN; ++r) {        // w = sum over the feature groups of (q_g . k_g)^2, masked
+            if (r >= nrun) break;
+            float w[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) w[c] = 0.f;
+#pragma unroll
+            for (int a = 0; a < G; ++a) {
+              uint32_t y[16];
+              tmem_ld16(tmem_addr(tb, q4 * 32, COL_SC + (SC2 ? b : r * G + a) * 16), y);
+              tmem_wait_ld(y);
+#pragma unroll
+              for (int c = 0; c < 16; ++c) w[c] = fmaf(__uint_as_float(y[c]), __uint_as_float(y[c]), w[c]);
+            }
+            const int key0 = (cta_head + r * ncta) * 16;
+            uint32_t pk[8];
+#pragma unroll
+            for (int c = 0; c < 16; c += 2) pk[c >> 1] = pack_bf16(key0 + c <= t ? w[c] : 0.f, key0 + c + 1 <= t ? w[c + 1] : 0.f);
+            tmem_st8(tmem_addr(tb, q4 * 32, SC2 ? COL_P : COL_SC + r * G * 16), pk);   // (over the scores just read, unless the weights have their own columns)
           }
-          tmem_st8(tmem_addr(tb, q4 * 32, COL_P), pk);
         }
       }
       tmem_wait_st();
       tc_fence_before();
       TICK(4);
-      phase_a_done();
+      phase_a_arrive();
       TICK(5);
     }
     if (warp == W_Q0) TOCK(2);
@@ -538,7 +607,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (ok && j >= 1) {
         tc_fence_after();
 #pragma unroll
-        for (int m = 0; m < 2; ++m) {
+        for (int m = 0; m < NM; ++m) {
           uint32_t pk[32], zc[4];
 #pragma unroll
           for (int h = 0; h < 4; ++h) {
@@ -559,7 +628,7 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         fence_async_smem();
       }
       TICK(1);
-      phase_a_done();
+      phase_a_arrive();
       TICK(2);
     }
     if (warp == W_S0) TOCK(3);
@@ -623,49 +692,57 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     // one, so that a tile costs one trip to L2.
     const int et = tid - W_O0 * 32;
     const int r_in = et >> 3, piece = et & 7;
-    const int trow = cta_head * kRowsPerCta + r_in;               // query row of the tile
-    const bool active = r_in < kRowsPerCta && trow < CT;
     __nv_bfloat16* outp = args.out + (size_t)bh * args.T * D;
     const unsigned* cnt = args.counter + (size_t)bh * ntiles;
     if (et == 127) {
       store_thread();
-    } else if (active) {
+    } else if (r_in < kRowSlots) {
       unsigned have = 0;                                          // shares of tile j seen so far
-      const size_t in_tile = (size_t)trow * 128 + ((piece ^ (trow & 7)) * 16);
       for (int j = 0; j < ntiles; ++j) {
-        if (have < NCTA) ok = wait_count_global(cnt + j, NCTA, abort_flag);
+        if (have < (unsigned)ncta) ok = wait_count_global(cnt + j, (unsigned)ncta, abort_flag);
         if (!ok) break;
-        have = NCTA;
+        have = (unsigned)ncta;
         if (j + 1 < ntiles) asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(have) : "l"(cnt + j + 1) : "memory");
-        const size_t row = (size_t)j * CT + trow;
-        uint4 pk[NCTA];
-        float2 ds[NCTA];
 #pragma unroll
-        for (int s = 0; s < NCTA; ++s) {
-          const unsigned char* blk = args.share + (((size_t)bh * NCTA + s) * ntiles + j) * kShareBytes;
-          pk[s] = __ldcg(reinterpret_cast<const uint4*>(blk + in_tile));
-          ds[s] = __ldcg(reinterpret_cast<const float2*>(blk + 16384 + trow * 8));
-        }
-        float acc[8], den = 0.f;
+        for (int r0 = 0; r0 < kRowsPerCta; r0 += kRowSlots) {     // this CTA's rows of the tile, kRowSlots at a time
+          const int r_cta = r0 + r_in;
+          const int trow = cta_head * kRowsPerCta + r_cta;        // query row of the tile
+          if (r_cta >= kRowsPerCta || trow >= CT) continue;
+          const size_t in_tile = (size_t)trow * 128 + ((piece ^ (trow & 7)) * 16);
+          const size_t row = (size_t)j * CT + trow;
+          uint4 pk[NCTA];
+          float2 ds[NCTA];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) acc[c] = 0.f;
-#pragma unroll
-        for (int s = 0; s < NCTA; ++s) {
-          den += ds[s].x;
-          const uint32_t w4[4] = {pk[s].x, pk[s].y, pk[s].z, pk[s].w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float2 f2 = __half22float2(*reinterpret_cast<const __half2*>(&w4[e]));
-            acc[2 * e] = fmaf(f2.x, ds[s].y, acc[2 * e]);
-            acc[2 * e + 1] = fmaf(f2.y, ds[s].y, acc[2 * e + 1]);
+          for (int s = 0; s < NCTA; ++s) {
+            {
+              const unsigned char* blk = args.share + (((size_t)bh * ncta + s) * ntiles + j) * kShareBytes;
+              pk[s] = __ldcg(reinterpret_cast<const uint4*>(blk + in_tile));
+              ds[s] = __ldcg(reinterpret_cast<const float2*>(blk + 16384 + trow * 8));
+            }
           }
-        }
-        const float inv = den > 0.f ? 1.f / den : 0.f;
-        if (row < (size_t)args.T) {
-          uint4 o;
-          o.x = pack_bf16(acc[0] * inv, acc[1] * inv); o.y = pack_bf16(acc[2] * inv, acc[3] * inv);
-          o.z = pack_bf16(acc[4] * inv, acc[5] * inv); o.w = pack_bf16(acc[6] * inv, acc[7] * inv);
-          reinterpret_cast<uint4*>(outp + row * D)[piece] = o;
+          float acc[8], den = 0.f;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+#pragma unroll
+          for (int s = 0; s < NCTA; ++s) {
+            {
+              den += ds[s].x;
+              const uint32_t w4[4] = {pk[s].x, pk[s].y, pk[s].z, pk[s].w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float2 f2 = __half22float2(*reinterpret_cast<const __half2*>(&w4[e]));
+                acc[2 * e] = fmaf(f2.x, ds[s].y, acc[2 * e]);
+                acc[2 * e + 1] = fmaf(f2.y, ds[s].y, acc[2 * e + 1]);
+              }
+            }
+          }
+          const float inv = den > 0.f ? 1.f / den : 0.f;
+          if (row < (size_t)args.T) {
+            uint4 o;
+            o.x = pack_bf16(acc[0] * inv, acc[1] * inv); o.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+            o.z = pack_bf16(acc[4] * inv, acc[5] * inv); o.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+            reinterpret_cast<uint4*>(outp + row * D)[piece] = o;
+          }
         }
       }
     }
@@ -684,36 +761,56 @@ tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (warp == 0) tmem_dealloc(tb, TMEM_COLS);
 }
 
-// The 36 block pairs (g <= h) of the rank-one lift in the order they are dealt out, four to a CTA.
-void fill_block_pairs(BlockPairs& bp) {
+// The block pairs (g <= h) the state holds, in the order they are dealt out to the CTAs of a head: all 36 for the
+// full lift, those inside a feature group for the blockwise map (runs of 8 features, 8 / groups runs per group).
+int fill_block_pairs(BlockPairs& bp, int groups) {
+  const int per = 8 / groups;
   int n = 0;
   for (int g = 0; g < 8; ++g)
     for (int h = g; h < 8; ++h) {
+      if (g / per != h / per) continue;
       bp.g[n] = (unsigned char)g;
       bp.h[n] = (unsigned char)h;
       bp.w[n] = (unsigned char)(g == h ? 1 : 2);
       ++n;
     }
+  return n;
+}
+
+// How a head is cut: CTAs per head and accumulator tiles (of two block pairs) per CTA.  The full lift: 36 pairs, nine
+// CTAs of four.  Two feature groups: 20 pairs, ten CTAs of two while ten per head fit the GPU in one wave, else five of
+// four.  Four groups: 12 pairs, six CTAs of two.
+struct SplitPlan {
+  int ncta, nm;
+};
+SplitPlan split_plan(int groups, size_t BH) {
+  if (groups == 1) return {9, 2};
+  if (groups == 2) return 10 * BH <= 148 ? SplitPlan{10, 1} : SplitPlan{5, 2};
+  return {6, 1};
 }
 
 size_t al256(size_t x) { return (x + 255) / 256 * 256; }
 
 }  // namespace
 
-// workspace: counters [BH][ntiles] | V' [BH][T][64] bf16 | r [BH][T] bf16 | share numerators | share normalisers and scales
+// workspace: counters [BH][ntiles] + ticket | V' [BH][T][64] bf16 | r [BH][T] bf16 | shares [BH][ncta][ntiles][17 KB]
 size_t tc_split_workspace_bytes(const Problem& p) {
-  const size_t BH = (size_t)p.B * p.H, nt = (size_t)(p.T + CT - 1) / CT, tpad = nt * CT;
-  return al256((BH * nt + 1) * sizeof(unsigned)) + al256(BH * p.T * D * 2) + al256(BH * p.T * 2) + al256(BH * NCTA * nt * kShareBytes) + (KATA_SPLIT_PROF ? al256(BH * NCTA * 5 * 8 * 8) : 0);
+  const size_t BH = (size_t)p.B * p.H, nt = (size_t)(p.T + CT - 1) / CT;
+  const size_t ncta = (size_t)split_plan(p.groups, BH).ncta;
+  return al256((BH * nt + 1) * sizeof(unsigned)) + al256(BH * p.T * D * 2) + al256(BH * p.T * 2) + al256(BH * ncta * nt * kShareBytes) +
+         (KATA_SPLIT_PROF ? al256(BH * ncta * 5 * 8 * 8) : 0);
 }
 
+int tc_split_ctas_per_head(const Problem& p) { return split_plan(p.groups, (size_t)p.B * p.H).ncta; }
+
 bool tc_split_supported(const Problem& p) {
-  return p.dtype == KATA_BF16 && p.d_k == 64 && p.d_v == 64 && p.feature_order == 2 && p.groups == 1;
+  return p.dtype == KATA_BF16 && p.d_k == 64 && p.d_v == 64 && p.feature_order == 2 && (p.groups == 1 || p.groups == 2 || p.groups == 4);
 }
 
 void tc_chunked_split(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx) {
   const size_t BH = (size_t)p.B * p.H;
   const int ntiles = (p.T + CT - 1) / CT;
-  const size_t tpad = (size_t)ntiles * CT;
+  const SplitPlan plan = split_plan(p.groups, BH);
   unsigned char* w8 = static_cast<unsigned char*>(workspace);
   const size_t cnt_bytes = al256((BH * ntiles + 1) * sizeof(unsigned));   // + the ticket counter
   __nv_bfloat16* vs = reinterpret_cast<__nv_bfloat16*>(w8 + cnt_bytes);
@@ -724,7 +821,8 @@ void tc_chunked_split(const Problem& p, void* workspace, int* device_status, Lau
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-  if (cudaFuncSetAttribute(tc_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
+  auto kern = p.groups == 1 ? tc_split_kernel<2, 1, 9> : p.groups == 4 ? tc_split_kernel<1, 4, 6> : plan.nm == 1 ? tc_split_kernel<1, 2, 10> : tc_split_kernel<2, 2, 5>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess) {
     cudaGetLastError();
     ctx.status = KATA_ERR_CUDA;
     return;
@@ -734,11 +832,16 @@ void tc_chunked_split(const Problem& p, void* workspace, int* device_status, Lau
   a.rscale = rscale;
   a.counter = reinterpret_cast<unsigned*>(w8);
   a.share = sh;
-  a.prof = reinterpret_cast<long long*>(sh + al256(BH * NCTA * (size_t)ntiles * kShareBytes));
+  a.prof = reinterpret_cast<long long*>(sh + al256(BH * plan.ncta * (size_t)ntiles * kShareBytes));
   a.device_status = device_status;
   a.T = p.T;
   a.ntiles = ntiles;
-  fill_block_pairs(a.bp);
+  a.ncta = plan.ncta;
+  a.groups = p.groups;
+  if (fill_block_pairs(a.bp, p.groups) != plan.ncta * 2 * plan.nm) {
+    ctx.status = KATA_ERR_UNSUPPORTED_SHAPE;
+    return;
+  }
   if (cudaMemsetAsync(a.counter, 0, cnt_bytes, ctx.stream) != cudaSuccess) {
     cudaGetLastError();
     ctx.status = KATA_ERR_CUDA;
@@ -748,7 +851,7 @@ void tc_chunked_split(const Problem& p, void* workspace, int* device_status, Lau
   split_prescale_kernel<<<(unsigned)((n_rows + 31) / 32), 256, 0, ctx.stream>>>(
       static_cast<const __nv_bfloat16*>(p.k), static_cast<const __nv_bfloat16*>(p.v), vs, rscale, n_rows);
   note_launch(ctx);
-  tc_split_kernel<<<(unsigned)(BH * NCTA), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
+  kern<<<(unsigned)(BH * plan.ncta), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
   note_launch(ctx);
 }
 
