@@ -170,8 +170,8 @@ int kata_fwd_quadratic(const void* q, const void* k, const void* v, void* out,
  * (section "Chunkwise forward").  O(T) work, fp32 state.  opts->inter_chunk selects how
  * the inter-chunk recurrence is traversed; both give the same result up to fp32
  * re-association.  Workspace: kata_workspace_bytes(KATA_FN_CHUNKED, ...); the sequential walk on the tensor-core
- * path (bf16, d_k = d_v = 64, feature_order 2, feature_groups 1, no state pointers) splits the state of a head over
- * nine CTAs and needs about 1.36 KB per token and head there (scaled values, key scales, the CTAs' shares of the
+ * path (bf16, d_k = d_v = 64, feature_order 2, no state pointers) splits the state of a head over
+ * nine CTAs (five, six or ten with feature_groups 2 or 4) and needs about 0.15 KB per token, head and CTA there (scaled values, key scales, the CTAs' shares of the
  * output and a counter per tile); the environment variable KATA_CHUNKED_KERNEL=stream selects the one-CTA-per-value-
  * slice streaming kernel instead (no workspace; for comparisons).
  */

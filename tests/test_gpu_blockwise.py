@@ -79,6 +79,30 @@ def test_blockwise_chunked_tensor_tiles(g, T):
         check(gpu[0, h], ref, "bf16", f"M{g} tensor chunked T={T} head {h}")
 
 
+@pytest.mark.parametrize("g,B,H,T", [(2, 1, 3, 1000), (2, 2, 16, 700), (2, 1, 14, 515), (4, 1, 2, 1300), (4, 3, 9, 520),
+                                     (4, 2, 16, 900)])
+def test_blockwise_chunked_head_layouts(g, B, H, T):
+    """The feature-split kernel with the blockwise map: block pairs inside a feature group only, dealt to ten CTAs of
+    two per head while ten per head fit the GPU in one wave (g = 2, B*H <= 14), to five of four beyond, to six of two
+    for g = 4; CTAs of the five- and six-CTA layouts weigh two 16-key runs of a tile.  Several tiles, a ragged tail,
+    grids of one and of several waves; and the same result run after run."""
+    import torch
+    w = inputs.gaussian_workload(f"mg_split_{g}_{B}_{H}_{T}", "bf16", B, H, T, 64, 64, 64, 4100 + T + g)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    o = kb.kata_fwd_chunked(*dev_tensors(w), feature_groups=g, device_status=st)
+    torch.cuda.synchronize()
+    assert kb.kata_last_impl() == kb.KATA_IMPL_TENSOR and int(st.item()) == 0
+    assert kb.kata_last_launch_count() == 2, "the key-scale pre-pass and the feature-split kernel"
+    o2 = kb.kata_fwd_chunked(*dev_tensors(w), feature_groups=g)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o2)
+    gpu = to_numpy64(o)
+    for b in range(B):
+        for h in range(0, H, max(1, H // 3)):
+            ref = ko.kata_quadratic(w.q_ref[b, h], w.k_ref[b, h], w.v_ref[b, h], f"psd_direct:g{g}")[0]
+            check(gpu[b, h], ref, "bf16", f"M{g} feature-split B{B} H{H} T={T} head ({b},{h})")
+
+
 @pytest.mark.parametrize("form", ["quadratic", "chunked_seq"])
 @pytest.mark.parametrize("g", [2, 4])
 def test_blockwise_tensor_degenerate(form, g):
