@@ -3,9 +3,11 @@
 // Pre-pass (one light kernel per call): V'[i] = v_i / ||k_i||^2 (bf16) and r[i] = 1 / ||k_i||^2 (bf16) into
 // the workspace, so that the key scale never touches the 128 x 128 weight tiles.
 //
-// Main kernel: one CTA = one head x one tile of 128 queries; it walks the key tiles j <= i of 128 keys:
-//   scores   S = Q K_j^T            tcgen05 kind::f16; A = the query tile, copied once into TMEM; B = the
-//                                   TMA-loaded 128B-swizzled key tile; fp32 result in one of three TMEM buffers
+// Main kernel: persistent, one CTA per SM.  A work item = one head x one tile of 128 queries; the items are ordered
+// heaviest first (latest query tiles first) and dealt round-robin to the CTAs, which walk the key tiles j <= i of
+// 128 keys of each of their items:
+//   scores   S = Q K_j^T            tcgen05 kind::f16; A = the query tile and B = the key tile, both TMA-loaded
+//                                   128B-swizzled tiles in shared memory; fp32 result in one of three TMEM buffers
 //   weights  P = S^2 (causal mask   packed fp32x2 multiplies on the TMEM read-back, rounded to bf16 and stored
 //            on the diagonal tile)  back over the first 64 columns of the same buffer
 //   apply    [O | D] += P [V' | r]  tcgen05 kind::f16, A = P from TMEM, B = the V' tile plus one extra column
@@ -14,6 +16,10 @@
 //   epilogue out = O / D (0 where D = 0)      the gate/normalise step of the readout
 // There is no running maximum and no rescaling: the weights are polynomial.  The query norm cancels between
 // numerator and denominator and is never applied.  The d^2-wide feature state is never formed.
+// Nothing is set up per item: TMEM and the barriers are the CTA's, the stage and buffer rings run on across items
+// (every role counts tiles cumulatively), the query tile is double-buffered, and the producer and the score MMAs
+// run ahead into the next item while the builders finish the current one; only [O | D] is handed over (the apply
+// MMAs of the next item wait until the epilogue has read it).
 //
 // Warps (384 threads): 0 TMA producer (its lanes also place r into the extra column group), 1 score-MMA
 // issuer, 2 apply-MMA issuer, 3 idle, 4-11 weight builders (TMEM lane quadrant = warp % 4, column half =
@@ -40,12 +46,11 @@ constexpr int WARP_BLD0 = 4;
 
 constexpr uint32_t COL_S = 0;    // 3 x 128 fp32 score buffers; the bf16 weights overwrite columns [0,64) of a buffer
 constexpr uint32_t COL_O = 384;  // 80 fp32 accumulators: 64 outputs, column 64 = normaliser
-constexpr uint32_t COL_Q = 464;  // 32: the query tile as bf16 pairs (A operand of the score MMA)
 constexpr uint32_t TMEM_COLS = 512;
 
-constexpr uint32_t OFF_Q = 0;                       // 128 x 64 bf16, 128B swizzle (staging for the TMEM copy)
+constexpr uint32_t OFF_Q = 0;                       // 2 x (128 x 64 bf16, 128B swizzle): the query tiles of this and the next work item
 constexpr uint32_t STAGE_BYTES = 49152;             // K tile 16 KB, V' tile 16 KB, scale-column tile 16 KB
-constexpr uint32_t OFF_KV = 16384;                  // NSTAGE stages
+constexpr uint32_t OFF_KV = 32768;                  // NSTAGE stages
 constexpr uint32_t OFF_BAR = OFF_KV + NSTAGE * STAGE_BYTES;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
@@ -53,16 +58,17 @@ static_assert(SMEM_ALLOC > 116 * 1024, "one CTA per SM is assumed (the CTA alloc
 
 // Every barrier has waiters that consume each of its phases in order (no waiter skips a phase).
 enum {
-  BAR_QFULL = 0,     // query tile landed in shared memory
-  BAR_QTMEM = 1,     // query tile copied to TMEM (256 builders)
-  BAR_FULL = 2,      // [3] K and V' tiles landed and the scale column written (TMA bytes + 32 producer lanes)
-  BAR_EMPTY = 6,     // [3] stage free: both issuers' commits
-  BAR_SFULL = 10,     // [3] scores in TMEM
+  BAR_QFULL = 0,     // [2] query tile of a work item landed in shared memory
+  BAR_FULL = 2,      // [4] K and V' tiles landed and the scale column written (TMA bytes + 32 producer lanes)
+  BAR_EMPTY = 6,     // [4] stage free: both issuers' commits
+  BAR_SFULL = 10,    // [3] scores in TMEM
   BAR_PFULL = 13,    // [3] weights stored (256 builders)
   BAR_PEMPTY = 16,   // [3] weights consumed by the apply MMA: the buffer may take new scores
-  BAR_ODONE = 19,
+  BAR_ODONE = 19,    // the apply MMAs of a work item are complete: [O | D] is final
   BAR_DRAIN = 20,
-  BAR_COUNT = 21
+  BAR_QEMPTY = 21,   // [2] the score MMAs of a work item are complete: its query tile may be replaced
+  BAR_OFREE = 23,    // [O | D] of a work item has been read (256 builders): the next item may overwrite it
+  BAR_COUNT = 24
 };
 
 struct QArgs {
@@ -70,6 +76,7 @@ struct QArgs {
   const __nv_bfloat16* rscale;   // [BH][T] bf16: 1 / ||k||^2
   int* device_status;
   int Tlen;
+  int BH, n_qtiles;              // work items: (head, tile of 128 queries), heaviest tiles first
 };
 
 // Pre-pass: one warp per 4 key rows (8 lanes x 16 bytes per row).  V' = v / ||k||^2, r = 1 / ||k||^2.
@@ -121,17 +128,20 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   volatile int* abort_flag = &abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int qtile = gridDim.x - 1 - blockIdx.x;   // heaviest tiles first
-  const int bh = blockIdx.y;
-  const int q0 = qtile * QT;
   constexpr int KT = KTILE / G;                   // keys per tile
   constexpr int KPL = KT / 32;                    // keys per producer lane
-  const int ntiles = (qtile + 1) * G;             // key tiles covering keys 0 .. q0 + 127
+  const int n_items = args.BH * args.n_qtiles;
+  // work item id -> (head, query tile): the latest query tiles (the most key tiles) come first
+  auto item_qtile = [&](int id) { return args.n_qtiles - 1 - id / args.BH; };
+  auto item_bh = [&](int id) { return id % args.BH; };
 
   if (tid == 0) {
     abort_s = 0;
-    mbar_init(bar(BAR_QFULL), 1);
-    mbar_init(bar(BAR_QTMEM), 256);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BAR_QFULL + i), 1);
+      mbar_init(bar(BAR_QEMPTY + i), 1);
+    }
+    mbar_init(bar(BAR_OFREE), 256);
     for (int i = 0; i < NSTAGE; ++i) {
       mbar_init(bar(BAR_FULL + i), 1 + 32);
       mbar_init(bar(BAR_EMPTY + i), 2);
@@ -164,64 +174,78 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
   if (warp == 0) {
     // =========================== TMA producer (+ scale column) ===========================
-    if (lane == 0) {
-      mbar_arrive_expect_tx(bar(BAR_QFULL), 16384);
-      tma_load_3d(base + OFF_Q, &tmQ, bar(BAR_QFULL), 0, q0, bh);
-    }
-    // The kernel is a programmatic dependent launch behind the pre-pass: up to here (and in every other warp) only
-    // q, k and on-chip memory were touched; the scaled values and r are the pre-pass's, visible from here on.
+    // The kernel is a programmatic dependent launch behind the pre-pass: the scaled values and r are the pre-pass's,
+    // visible from here on (only this warp reads them).
     cudaGridDependencySynchronize();
-    const __nv_bfloat16* rs = args.rscale + (size_t)bh * args.Tlen;
-    // r of this lane's 4 keys of a tile, fetched one tile ahead (the global-load latency stays off the ring)
-    auto load_r = [&](int j, unsigned short (&rv)[KPL]) {
-#pragma unroll
-      for (int e = 0; e < KPL; ++e) {
-        const int key = j * KT + lane * KPL + e;
-        rv[e] = (j < ntiles && key < args.Tlen) ? __bfloat16_as_ushort(rs[key]) : (unsigned short)0;
-      }
-    };
-    unsigned short rv[KPL];
-    load_r(0, rv);
-    for (int j = 0; j < ntiles && ok; ++j) {
-      const int s = j % NSTAGE;
-      unsigned short rn[KPL];
-      load_r(j + 1, rn);
-      ok = wait_or_abort(bar(BAR_EMPTY + s), ((j / NSTAGE) & 1) ^ 1, abort_flag);
+    uint32_t it = 0;                                   // key tiles loaded so far, over all items
+    int n = 0;
+    for (int id = blockIdx.x; id < n_items && ok; id += gridDim.x, ++n) {
+      const int qtile = item_qtile(id), bh = item_bh(id), ntiles = (qtile + 1) * G, qb = n & 1;
+      ok = wait_or_abort(bar(BAR_QEMPTY + qb), ((n >> 1) & 1) ^ 1, abort_flag);
       if (!ok) break;
       if (lane == 0) {
-        mbar_arrive_expect_tx(bar(BAR_FULL + s), 2 * KT * 128);   // K and V' tiles
-        tma_load_3d(ktile(s), &tmK, bar(BAR_FULL + s), 0, j * KT, bh);
-        tma_load_3d(vtile(s), &tmV, bar(BAR_FULL + s), 0, j * KT, bh);
+        mbar_arrive_expect_tx(bar(BAR_QFULL + qb), 16384);
+        tma_load_3d(base + OFF_Q + qb * 16384, &tmQ, bar(BAR_QFULL + qb), 0, qtile * QT, bh);
       }
-      // column 64 of the B operand: r for the keys of the tile (element 0 of chunk 0 of each key row)
-      unsigned char* rt = rtile(s);
+      const __nv_bfloat16* rs = args.rscale + (size_t)bh * args.Tlen;
+      // r of this lane's keys of a tile, fetched one tile ahead (the global-load latency stays off the ring)
+      auto load_r = [&](int j, unsigned short (&rv)[KPL]) {
 #pragma unroll
-      for (int e = 0; e < KPL; ++e) {
-        *reinterpret_cast<uint16_t*>(rt + sw128_offset(lane * KPL + e, 0)) = rv[e];
-        rv[e] = rn[e];
+        for (int e = 0; e < KPL; ++e) {
+          const int key = j * KT + lane * KPL + e;
+          rv[e] = (j < ntiles && key < args.Tlen) ? __bfloat16_as_ushort(rs[key]) : (unsigned short)0;
+        }
+      };
+      unsigned short rv[KPL];
+      load_r(0, rv);
+      for (int j = 0; j < ntiles && ok; ++j, ++it) {
+        const int s = it % NSTAGE;
+        unsigned short rn[KPL];
+        load_r(j + 1, rn);
+        ok = wait_or_abort(bar(BAR_EMPTY + s), ((it / NSTAGE) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(bar(BAR_FULL + s), 2 * KT * 128);   // K and V' tiles
+          tma_load_3d(ktile(s), &tmK, bar(BAR_FULL + s), 0, j * KT, bh);
+          tma_load_3d(vtile(s), &tmV, bar(BAR_FULL + s), 0, j * KT, bh);
+        }
+        // column 64 of the B operand: r for the keys of the tile (element 0 of chunk 0 of each key row)
+        unsigned char* rt = rtile(s);
+#pragma unroll
+        for (int e = 0; e < KPL; ++e) {
+          *reinterpret_cast<uint16_t*>(rt + sw128_offset(lane * KPL + e, 0)) = rv[e];
+          rv[e] = rn[e];
+        }
+        fence_async_smem();
+        mbar_arrive(bar(BAR_FULL + s));
       }
-      fence_async_smem();
-      mbar_arrive(bar(BAR_FULL + s));
     }
   } else if (warp == 1) {
     // =========================== score MMA issuer: S = Q K^T ===========================
     if (lane == 0) {
       const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, KT);
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
-      ok = wait_or_abort(bar(BAR_QTMEM), 0, abort_flag);
-      for (int j = 0; j < ntiles && ok; ++j) {
-        const int s = j % NSTAGE, b = j % NBUF;
-        ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_PEMPTY + b), ((j / NBUF) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t ka = smem_u32(ktile(s));
+      uint32_t it = 0;
+      int n = 0;
+      for (int id = blockIdx.x; id < n_items && ok; id += gridDim.x, ++n) {
+        const int ntiles = (item_qtile(id) + 1) * G, qb = n & 1;
+        ok = wait_or_abort(bar(BAR_QFULL + qb), (n >> 1) & 1, abort_flag);
+        const uint32_t qa = smem_u32(base + OFF_Q + qb * 16384);
+        for (int j = 0; j < ntiles && ok; ++j, ++it) {
+          const int s = it % NSTAGE, b = it % NBUF;
+          ok = wait_or_abort(bar(BAR_FULL + s), (it / NSTAGE) & 1, abort_flag) &&
+               wait_or_abort(bar(BAR_PEMPTY + b), ((it / NBUF) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t ka = smem_u32(ktile(s));
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)   // 16 features per step; group ks / (4 / G) accumulates over its own steps
-          mma_f16_ts(tb + COL_S + b * 128 + (ks / (4 / G)) * KT, tb + COL_Q + ks * 8,
-                     dk + (uint64_t)(((ka + ks * 32) >> 4) & 0x3FFF), idesc, (ks % (4 / G)) > 0);
-        mma_commit(bar(BAR_SFULL + b));
-        mma_commit(bar(BAR_EMPTY + s));
+          for (int ks = 0; ks < 4; ++ks)   // 16 features per step; group ks / (4 / G) accumulates over its own steps
+            mma_f16_ss(tb + COL_S + b * 128 + (ks / (4 / G)) * KT, dk + (uint64_t)(((qa + ks * 32) >> 4) & 0x3FFF),
+                       dk + (uint64_t)(((ka + ks * 32) >> 4) & 0x3FFF), idesc, (ks % (4 / G)) > 0);
+          mma_commit(bar(BAR_SFULL + b));
+          mma_commit(bar(BAR_EMPTY + s));
+        }
+        mma_commit(bar(BAR_QEMPTY + qb));   // (also after a failed wait: the producer is not left waiting)
       }
     }
   } else if (warp == 2) {
@@ -230,45 +254,41 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const uint32_t idesc = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);     // A tmem, B MN-major, N = 64 + 16
       // MN-major, 128B swizzle: 8 key rows per 1024-byte atom (SBO), second group of 64 columns 16 KB on (LBO)
       const uint64_t dmn = smem_desc(0, 16384, 1024, kSwizzle128B);
-      for (int j = 0; j < ntiles && ok; ++j) {
-        const int s = j % NSTAGE, b = j % NBUF;
-        ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_PFULL + b), (j / NBUF) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t va = smem_u32(vtile(s));
+      uint32_t it = 0;
+      int n = 0;
+      for (int id = blockIdx.x; id < n_items && ok; id += gridDim.x, ++n) {
+        const int ntiles = (item_qtile(id) + 1) * G;
+        if (n > 0) ok = wait_or_abort(bar(BAR_OFREE), (n - 1) & 1, abort_flag);   // the epilogue of the item before has read [O | D]
+        for (int j = 0; j < ntiles && ok; ++j, ++it) {
+          const int s = it % NSTAGE, b = it % NBUF;
+          ok = wait_or_abort(bar(BAR_FULL + s), (it / NSTAGE) & 1, abort_flag) &&
+               wait_or_abort(bar(BAR_PFULL + b), (it / NBUF) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t va = smem_u32(vtile(s));
 #pragma unroll
-        for (int ks = 0; ks < KT / 16; ++ks)
-          mma_f16_ts(tb + COL_O, tb + COL_S + b * 128 + ks * 8, dmn + (uint64_t)(((va + ks * 2048) >> 4) & 0x3FFF),
-                     idesc, (j > 0 || ks > 0) ? 1u : 0u);
-        mma_commit(bar(BAR_PEMPTY + b));
-        mma_commit(bar(BAR_EMPTY + s));
+          for (int ks = 0; ks < KT / 16; ++ks)
+            mma_f16_ts(tb + COL_O, tb + COL_S + b * 128 + ks * 8, dmn + (uint64_t)(((va + ks * 2048) >> 4) & 0x3FFF),
+                       idesc, (j > 0 || ks > 0) ? 1u : 0u);
+          mma_commit(bar(BAR_PEMPTY + b));
+          mma_commit(bar(BAR_EMPTY + s));
+        }
+        mma_commit(bar(BAR_ODONE));
       }
-      if (ok) mma_commit(bar(BAR_ODONE));
     }
   } else if (warp >= WARP_BLD0) {
     // =========================== weight builders (256 threads) ===========================
     const uint32_t q4 = warp & 3;
     const int ch = (warp - WARP_BLD0) >> 2;      // column half: keys [64 ch, 64 ch + 64) of the tile
     const int rowl = q4 * 32 + lane;             // query row inside the tile (= TMEM lane)
-    const int qrow = q0 + rowl;
-    // the query tile goes to TMEM once: this thread copies features [32 ch, 32 ch + 32) of its row
-    ok = wait_or_abort(bar(BAR_QFULL), 0, abort_flag);
-    if (ok) {
-      uint32_t qw[16];
-#pragma unroll
-      for (int cix = 0; cix < 4; ++cix) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(base + OFF_Q + sw128_offset(rowl, ch * 4 + cix));
-        qw[4 * cix] = raw.x; qw[4 * cix + 1] = raw.y; qw[4 * cix + 2] = raw.z; qw[4 * cix + 3] = raw.w;
-      }
-      tmem_st16(tmem_addr(tb, q4 * 32, COL_Q + ch * 16), qw);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar(BAR_QTMEM));
-    }
-    for (int j = 0; j < ntiles && ok; ++j) {
-      const int b = j % NBUF;
-      ok = wait_or_abort(bar(BAR_SFULL + b), (j / NBUF) & 1, abort_flag);
+    uint32_t it = 0;                             // key tiles weighed so far, over all items
+    int n = 0;
+    for (int id = blockIdx.x; id < n_items && ok; id += gridDim.x, ++n) {
+    const int qtile = item_qtile(id), bh = item_bh(id), ntiles = (qtile + 1) * G;
+    const int qrow = qtile * QT + rowl;
+    for (int j = 0; j < ntiles && ok; ++j, ++it) {
+      const int b = it % NBUF;
+      ok = wait_or_abort(bar(BAR_SFULL + b), (it / NBUF) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       const bool diag = (j >= ntiles - G);
@@ -353,7 +373,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       mbar_arrive(bar(BAR_PFULL + b));
     }
     // ---- epilogue: out = O / D ----
-    if (ok) ok = wait_or_abort(bar(BAR_ODONE), 0, abort_flag);
+    if (ok) ok = wait_or_abort(bar(BAR_ODONE), n & 1, abort_flag);
     if (ok) {
       tc_fence_after();
       uint32_t o[32], dn[16];
@@ -361,6 +381,8 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       tmem_ld16(tmem_addr(tb, q4 * 32, COL_O + 64), dn);
       tmem_wait_ld(o);
       tmem_wait_ld(dn);
+      tc_fence_before();
+      mbar_arrive(bar(BAR_OFREE));               // the apply MMAs of the next item may overwrite [O | D]
       const float den = __uint_as_float(dn[0]);
       const float inv = den > 0.f ? 1.f / den : 0.f;
       if (qrow < args.Tlen) {
@@ -376,6 +398,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
       }
     }
+    }   // work items
   }
 
   // ---------------- teardown ----------------
@@ -420,9 +443,16 @@ void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchC
     ctx.status = KATA_ERR_CUDA;
     return;
   }
-  QArgs a{static_cast<__nv_bfloat16*>(p.out), rscale, device_status, p.T};
+  const int n_qtiles = (p.T + QT - 1) / QT;
+  QArgs a{static_cast<__nv_bfloat16*>(p.out), rscale, device_status, p.T, BH, n_qtiles};
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    sms = 148;
+  }
+  const long long n_items = (long long)BH * n_qtiles;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((p.T + QT - 1) / QT, BH);
+  cfg.gridDim = dim3((unsigned)(n_items < sms ? n_items : sms));   // persistent: one CTA per SM, items dealt round-robin
   cfg.blockDim = dim3(NTHREADS);
   cfg.dynamicSmemBytes = SMEM_ALLOC;
   cfg.stream = ctx.stream;
