@@ -134,6 +134,9 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   // work item id -> (head, query tile): the latest query tiles (the most key tiles) come first
   auto item_qtile = [&](int id) { return args.n_qtiles - 1 - id / args.BH; };
   auto item_bh = [&](int id) { return id % args.BH; };
+  // the n-th item of this CTA: rounds of gridDim.x items, dealt forwards and backwards in turn, so that the CTA that got
+  // the heaviest item of one round gets the lightest of the next
+  auto item_id = [&](int n) { return n * (int)gridDim.x + ((n & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x); };
 
   if (tid == 0) {
     abort_s = 0;
@@ -179,7 +182,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     cudaGridDependencySynchronize();
     uint32_t it = 0;                                   // key tiles loaded so far, over all items
     int n = 0;
-    for (int id = blockIdx.x; id < n_items && ok; id += gridDim.x, ++n) {
+    for (int id = item_id(n); id < n_items && ok; id = item_id(++n)) {
       const int qtile = item_qtile(id), bh = item_bh(id), ntiles = (qtile + 1) * G, qb = n & 1;
       ok = wait_or_abort(bar(BAR_QEMPTY + qb), ((n >> 1) & 1) ^ 1, abort_flag);
       if (!ok) break;
@@ -227,7 +230,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
       uint32_t it = 0;
       int n = 0;
-      for (int id = blockIdx.x; id < n_items && ok; id += gridDim.x, ++n) {
+      for (int id = item_id(n); id < n_items && ok; id = item_id(++n)) {
         const int ntiles = (item_qtile(id) + 1) * G, qb = n & 1;
         ok = wait_or_abort(bar(BAR_QFULL + qb), (n >> 1) & 1, abort_flag);
         const uint32_t qa = smem_u32(base + OFF_Q + qb * 16384);
@@ -256,7 +259,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const uint64_t dmn = smem_desc(0, 16384, 1024, kSwizzle128B);
       uint32_t it = 0;
       int n = 0;
-      for (int id = blockIdx.x; id < n_items && ok; id += gridDim.x, ++n) {
+      for (int id = item_id(n); id < n_items && ok; id = item_id(++n)) {
         const int ntiles = (item_qtile(id) + 1) * G;
         if (n > 0) ok = wait_or_abort(bar(BAR_OFREE), (n - 1) & 1, abort_flag);   // the epilogue of the item before has read [O | D]
         for (int j = 0; j < ntiles && ok; ++j, ++it) {
@@ -283,7 +286,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int rowl = q4 * 32 + lane;             // query row inside the tile (= TMEM lane)
     uint32_t it = 0;                             // key tiles weighed so far, over all items
     int n = 0;
-    for (int id = blockIdx.x; id < n_items && ok; id += gridDim.x, ++n) {
+    for (int id = item_id(n); id < n_items && ok; id = item_id(++n)) {
     const int qtile = item_qtile(id), bh = item_bh(id), ntiles = (qtile + 1) * G;
     const int qrow = qtile * QT + rowl;
     for (int j = 0; j < ntiles && ok; ++j, ++it) {
