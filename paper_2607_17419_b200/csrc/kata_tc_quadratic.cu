@@ -151,7 +151,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
     for (int i = 0; i < NBUF; ++i) {
       mbar_init(bar(BAR_SFULL + i), 1);
-      mbar_init(bar(BAR_PFULL + i), 256);
+      mbar_init(bar(BAR_PFULL + i), G == 1 ? 128 : 256);
       mbar_init(bar(BAR_PEMPTY + i), 1);
     }
     mbar_init(bar(BAR_ODONE), 1);
@@ -336,41 +336,45 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         mbar_arrive(bar(BAR_PFULL + b));
         continue;
       }
-      const uint32_t scol = tmem_addr(tb, q4 * 32, COL_S + b * 128 + ch * 64);
-      const int key0 = j * KTILE + ch * 64;
-      uint32_t ya[32], yb[32], pk[32];
+      // Full lift: the two groups of four warps take alternate tiles (both wait for every tile's scores, so that
+      // neither skips a phase of a barrier), and a warp weighs all 128 keys of its 32 query rows: while one group
+      // turns the scores of a tile into weights, the MMAs work for the other group's tile.
+      if ((it & 1u) != (uint32_t)ch) continue;
+      const uint32_t scol = tmem_addr(tb, q4 * 32, COL_S + b * 128);
+      const int key0 = j * KTILE;
+      uint32_t ya[32], yb[32], pk0[32], pk1[32];
       // two copies of the loop, chosen once per tile: the causal test exists on the diagonal tile only
-      auto weigh = [&](const uint32_t (&y)[32], int half, auto masked) {
+      auto weigh = [&](const uint32_t (&y)[32], uint32_t (&pk)[32], int col0, auto masked) {
 #pragma unroll
         for (int jj = 0; jj < 32; jj += 2) {
-          const int c = half * 32 + jj;
+          const int c = col0 + jj;
           const float2 sv = make_float2(__uint_as_float(y[jj]), __uint_as_float(y[jj + 1]));
           float2 w = __fmul2_rn(sv, sv);
           if constexpr (decltype(masked)::value) {
             if (key0 + c > qrow) w.x = 0.f;
             if (key0 + c + 1 > qrow) w.y = 0.f;
           }
-          pk[c / 2] = pack_bf16(w.x, w.y);
+          pk[(c & 63) / 2] = pack_bf16(w.x, w.y);
         }
       };
-      tmem_ld32(scol, ya);
-      tmem_wait_ld(ya);
-      tmem_ld32(scol + 32, yb);
-      if (diag) {
-        weigh(ya, 0, std::true_type{});
+      auto weigh_tile = [&](auto masked) {
+        tmem_ld32(scol, ya);
+        tmem_ld32(scol + 32, yb);
+        tmem_wait_ld(ya);
+        weigh(ya, pk0, 0, masked);
         tmem_wait_ld(yb);
-        weigh(yb, 1, std::true_type{});
-      } else {
-        weigh(ya, 0, std::false_type{});
+        weigh(yb, pk0, 32, masked);
+        tmem_ld32(scol + 64, ya);
+        tmem_ld32(scol + 96, yb);
+        tmem_wait_ld(ya);
+        weigh(ya, pk1, 64, masked);
         tmem_wait_ld(yb);
-        weigh(yb, 1, std::false_type{});
-      }
-      // the weights overwrite score columns [0,64) of the buffer, which the column-half-0 warp of this
-      // quadrant reads: both warps of the quadrant must have their scores in registers first
-      tc_fence_before();
-      asm volatile("bar.sync %0, 64;" ::"r"(1 + (int)q4) : "memory");
-      tc_fence_after();
-      tmem_st32(tmem_addr(tb, q4 * 32, COL_S + b * 128 + ch * 32), pk);
+        weigh(yb, pk1, 96, masked);
+      };
+      if (diag) weigh_tile(std::true_type{}); else weigh_tile(std::false_type{});
+      // the weights overwrite score columns [0,64) of the buffer: this warp's lanes only, all read above
+      tmem_st32(scol, pk0);
+      tmem_st32(scol + 32, pk1);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_PFULL + b));
