@@ -52,14 +52,15 @@ constexpr uint32_t OFF_Q = 0;                       // 2 x (128 x 64 bf16, 128B 
 constexpr uint32_t STAGE_BYTES = 49152;             // K tile 16 KB, V' tile 16 KB, scale-column tile 16 KB
 constexpr uint32_t OFF_KV = 32768;                  // NSTAGE stages
 constexpr uint32_t OFF_BAR = OFF_KV + NSTAGE * STAGE_BYTES;
-constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
+constexpr uint32_t OFF_RV = OFF_BAR + 256;          // NSTAGE x 128 bf16: 1 / ||k||^2 of the keys of a tile
+constexpr uint32_t SMEM_BYTES = OFF_RV + NSTAGE * 256;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;
 static_assert(SMEM_ALLOC > 116 * 1024, "one CTA per SM is assumed (the CTA allocates all of TMEM)");
 
 // Every barrier has waiters that consume each of its phases in order (no waiter skips a phase).
 enum {
   BAR_QFULL = 0,     // [2] query tile of a work item landed in shared memory
-  BAR_FULL = 2,      // [4] K and V' tiles landed and the scale column written (TMA bytes + 32 producer lanes)
+  BAR_FULL = 2,      // [4] K and V tiles landed (TMA bytes)
   BAR_EMPTY = 6,     // [4] stage free: both issuers' commits
   BAR_SFULL = 10,    // [3] scores in TMEM
   BAR_PFULL = 13,    // [3] weights stored (256 builders)
@@ -68,22 +69,13 @@ enum {
   BAR_DRAIN = 20,
   BAR_QEMPTY = 21,   // [2] the score MMAs of a work item are complete: its query tile may be replaced
   BAR_OFREE = 23,    // [O | D] of a work item has been read (256 builders): the next item may overwrite it
-  BAR_COUNT = 24
+  BAR_RFULL = 24,    // [4] the key scales of a tile are in shared memory (the scale warp)
+  BAR_COUNT = 28
 };
 
-struct QArgs {
-  __nv_bfloat16* out;
-  const __nv_bfloat16* rscale;   // [BH][T] bf16: 1 / ||k||^2
-  int* device_status;
-  int Tlen;
-  int BH, n_qtiles;              // work items: (head, tile of 128 queries), heaviest tiles first
-};
-
-// Pre-pass: one warp per 4 key rows (8 lanes x 16 bytes per row).  V' = v / ||k||^2, r = 1 / ||k||^2.
-__global__ void __launch_bounds__(256) quad_prescale_kernel(const __nv_bfloat16* __restrict__ k,
-                                                            const __nv_bfloat16* __restrict__ v,
-                                                            __nv_bfloat16* __restrict__ vs,
-                                                            __nv_bfloat16* __restrict__ rscale, size_t n_rows) {
+// Pre-pass: r = 1 / ||k||^2 per key row (0 for a zero row), one warp per 4 rows (8 lanes x 16 bytes per row).
+__global__ void __launch_bounds__(256) quad_rscale_kernel(const __nv_bfloat16* __restrict__ k, __nv_bfloat16* __restrict__ rscale,
+                                                          size_t n_rows) {
   const size_t row = (size_t)blockIdx.x * 32 + (threadIdx.x >> 3);
   const int part = threadIdx.x & 7;
   if (row >= n_rows) return;
@@ -99,16 +91,22 @@ __global__ void __launch_bounds__(256) quad_prescale_kernel(const __nv_bfloat16*
   ss += __shfl_xor_sync(0xffffffffu, ss, 1);
   ss += __shfl_xor_sync(0xffffffffu, ss, 2);
   ss += __shfl_xor_sync(0xffffffffu, ss, 4);
-  const float r2 = inv_or_zero(ss);
-  const uint4 vraw = *reinterpret_cast<const uint4*>(v + row * D + part * 8);
-  uint4 sc;
-  sc.x = pack_bf16(__uint_as_float(vraw.x << 16) * r2, __uint_as_float(vraw.x & 0xFFFF0000u) * r2);
-  sc.y = pack_bf16(__uint_as_float(vraw.y << 16) * r2, __uint_as_float(vraw.y & 0xFFFF0000u) * r2);
-  sc.z = pack_bf16(__uint_as_float(vraw.z << 16) * r2, __uint_as_float(vraw.z & 0xFFFF0000u) * r2);
-  sc.w = pack_bf16(__uint_as_float(vraw.w << 16) * r2, __uint_as_float(vraw.w & 0xFFFF0000u) * r2);
-  *reinterpret_cast<uint4*>(vs + row * D + part * 8) = sc;
-  if (part == 0) rscale[row] = __float2bfloat16_rn(r2);
+  if (part == 0) rscale[row] = __float2bfloat16_rn(inv_or_zero(ss));
 }
+
+// a pair of bf16 weights times the pair of key scales 1 / ||k||^2
+__device__ __forceinline__ uint32_t scale_pair(uint32_t w2, uint32_t r2) {
+  const __nv_bfloat162 p = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&w2), *reinterpret_cast<const __nv_bfloat162*>(&r2));
+  return *reinterpret_cast<const uint32_t*>(&p);
+}
+
+struct QArgs {
+  __nv_bfloat16* out;
+  const __nv_bfloat16* rscale;   // [BH][T] bf16: 1 / ||k||^2 (pre-pass)
+  int* device_status;
+  int Tlen;
+  int BH, n_qtiles;              // work items: (head, tile of 128 queries), heaviest tiles first
+};
 
 // G = feature groups of the blockwise map (Section 3.3): a key tile holds KT = 128 / G keys, and the 128 score
 // columns of a buffer hold the G per-group score blocks Q_a K_a^T side by side (group a in columns [a KT, a KT + KT));
@@ -146,7 +144,8 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
     mbar_init(bar(BAR_OFREE), 256);
     for (int i = 0; i < NSTAGE; ++i) {
-      mbar_init(bar(BAR_FULL + i), 1 + 32);
+      mbar_init(bar(BAR_FULL + i), 1);
+      mbar_init(bar(BAR_RFULL + i), 1);
       mbar_init(bar(BAR_EMPTY + i), 2);
     }
     for (int i = 0; i < NBUF; ++i) {
@@ -161,9 +160,13 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmV);
   }
-  // the scale-column tiles are zero except for one bf16 per key row, rewritten for every key tile
+  // column 64 of the B operand of the apply MMA is a column of ones (the normaliser is the row sum of the weights):
+  // the extra column-group tiles are zero except for one bf16 1.0 per key row, written once
   for (int i = tid; i < NSTAGE * 1024; i += NTHREADS)
     *reinterpret_cast<uint4*>(rtile(i >> 10) + (i & 1023) * 16) = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+  for (int i = tid; i < NSTAGE * 128; i += NTHREADS)
+    *reinterpret_cast<uint16_t*>(rtile(i >> 7) + sw128_offset(i & 127, 0)) = (uint16_t)0x3F80;
   fence_async_smem();
   if (warp == 0) {
     tmem_alloc(&tmem_base_s, TMEM_COLS);
@@ -176,10 +179,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   bool ok = true;
 
   if (warp == 0) {
-    // =========================== TMA producer (+ scale column) ===========================
-    // The kernel is a programmatic dependent launch behind the pre-pass: the scaled values and r are the pre-pass's,
-    // visible from here on (only this warp reads them).
-    cudaGridDependencySynchronize();
+    // =========================== TMA producer ===========================
     uint32_t it = 0;                                   // key tiles loaded so far, over all items
     int n = 0;
     for (int id = item_id(n); id < n_items && ok; id = item_id(++n)) {
@@ -190,37 +190,15 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         mbar_arrive_expect_tx(bar(BAR_QFULL + qb), 16384);
         tma_load_3d(base + OFF_Q + qb * 16384, &tmQ, bar(BAR_QFULL + qb), 0, qtile * QT, bh);
       }
-      const __nv_bfloat16* rs = args.rscale + (size_t)bh * args.Tlen;
-      // r of this lane's keys of a tile, fetched one tile ahead (the global-load latency stays off the ring)
-      auto load_r = [&](int j, unsigned short (&rv)[KPL]) {
-#pragma unroll
-        for (int e = 0; e < KPL; ++e) {
-          const int key = j * KT + lane * KPL + e;
-          rv[e] = (j < ntiles && key < args.Tlen) ? __bfloat16_as_ushort(rs[key]) : (unsigned short)0;
-        }
-      };
-      unsigned short rv[KPL];
-      load_r(0, rv);
       for (int j = 0; j < ntiles && ok; ++j, ++it) {
         const int s = it % NSTAGE;
-        unsigned short rn[KPL];
-        load_r(j + 1, rn);
         ok = wait_or_abort(bar(BAR_EMPTY + s), ((it / NSTAGE) & 1) ^ 1, abort_flag);
         if (!ok) break;
         if (lane == 0) {
-          mbar_arrive_expect_tx(bar(BAR_FULL + s), 2 * KT * 128);   // K and V' tiles
+          mbar_arrive_expect_tx(bar(BAR_FULL + s), 2 * KT * 128);   // K and V tiles
           tma_load_3d(ktile(s), &tmK, bar(BAR_FULL + s), 0, j * KT, bh);
           tma_load_3d(vtile(s), &tmV, bar(BAR_FULL + s), 0, j * KT, bh);
         }
-        // column 64 of the B operand: r for the keys of the tile (element 0 of chunk 0 of each key row)
-        unsigned char* rt = rtile(s);
-#pragma unroll
-        for (int e = 0; e < KPL; ++e) {
-          *reinterpret_cast<uint16_t*>(rt + sw128_offset(lane * KPL + e, 0)) = rv[e];
-          rv[e] = rn[e];
-        }
-        fence_async_smem();
-        mbar_arrive(bar(BAR_FULL + s));
       }
     }
   } else if (warp == 1) {
@@ -279,6 +257,41 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         mma_commit(bar(BAR_ODONE));
       }
     }
+  } else if (warp == 3) {
+    // =========================== scale warp: r = 1 / ||k||^2 of the keys of every tile, from the pre-pass to shared memory ===========================
+    // (the key scale multiplies the weights, so the values are used as they are; a zero key row has r = 0: zero
+    // feature).  The kernel is a programmatic dependent launch behind the pre-pass that computes r: this warp is the
+    // only one that reads it, everything else starts at once.
+    cudaGridDependencySynchronize();
+    uint32_t it = 0;
+    int n = 0;
+    for (int id = item_id(n); id < n_items && ok; id = item_id(++n)) {
+      const int ntiles = (item_qtile(id) + 1) * G;
+      const unsigned short* rs = reinterpret_cast<const unsigned short*>(args.rscale) + (size_t)item_bh(id) * args.Tlen;
+      auto load_r = [&](int j, unsigned short (&rv)[KPL]) {       // r of this lane's keys of tile j
+#pragma unroll
+        for (int e = 0; e < KPL; ++e) {
+          const int key = j * KT + lane * KPL + e;
+          rv[e] = (j < ntiles && key < args.Tlen) ? rs[key] : (unsigned short)0;
+        }
+      };
+      unsigned short rv[KPL];
+      load_r(0, rv);
+      for (int j = 0; j < ntiles && ok; ++j, ++it) {
+        const int s = it % NSTAGE;
+        unsigned short rn[KPL];
+        load_r(j + 1, rn);              // one tile ahead: the global-load latency stays off the ring
+        ok = wait_or_abort(bar(BAR_FULL + s), (it / NSTAGE) & 1, abort_flag);   // (the stage, and with it its r, has been let go of)
+        if (!ok) break;
+#pragma unroll
+        for (int e = 0; e < KPL; ++e) {
+          reinterpret_cast<unsigned short*>(base + OFF_RV + s * 256)[lane * KPL + e] = rv[e];
+          rv[e] = rn[e];
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_RFULL + s));
+      }
+    }
   } else if (warp >= WARP_BLD0) {
     // =========================== weight builders (256 threads) ===========================
     const uint32_t q4 = warp & 3;
@@ -300,6 +313,9 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         constexpr int KH = KT / 2;
         const int key0 = j * KT + ch * KH;
         uint32_t y[G][KH], pk[KH / 2];
+        ok = wait_or_abort(bar(BAR_RFULL + (it % NSTAGE)), (it / NSTAGE) & 1, abort_flag);
+        if (!ok) break;
+        const uint32_t* rw = reinterpret_cast<const uint32_t*>(base + OFF_RV + (it % NSTAGE) * 256) + ch * (KH / 2);   // r of this warp's keys, in pairs
 #pragma unroll
         for (int g = 0; g < G; ++g) {
           const uint32_t col = tmem_addr(tb, q4 * 32, COL_S + b * 128 + g * KT + ch * KH);
@@ -321,7 +337,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
               if (key0 + c > qrow) w.x = 0.f;
               if (key0 + c + 1 > qrow) w.y = 0.f;
             }
-            pk[c / 2] = pack_bf16(w.x, w.y);
+            pk[c / 2] = scale_pair(pack_bf16(w.x, w.y), rw[c / 2]);
           }
         };
         if (diag) weigh_g(std::true_type{}); else weigh_g(std::false_type{});
@@ -340,23 +356,33 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       // neither skips a phase of a barrier), and a warp weighs all 128 keys of its 32 query rows: while one group
       // turns the scores of a tile into weights, the MMAs work for the other group's tile.
       if ((it & 1u) != (uint32_t)ch) continue;
+      ok = wait_or_abort(bar(BAR_RFULL + (it % NSTAGE)), (it / NSTAGE) & 1, abort_flag);   // (a stage belongs to one group: NSTAGE is even)
+      if (!ok) break;
+      const uint4* rv4 = reinterpret_cast<const uint4*>(base + OFF_RV + (it % NSTAGE) * 256);   // r of the tile's 128 keys, 8 per load
       const uint32_t scol = tmem_addr(tb, q4 * 32, COL_S + b * 128);
       const int key0 = j * KTILE;
-      uint32_t ya[32], yb[32], pk0[32], pk1[32];
+      uint32_t ya[32], yb[32], pk0[32];
       // two copies of the loop, chosen once per tile: the causal test exists on the diagonal tile only
       auto weigh = [&](const uint32_t (&y)[32], uint32_t (&pk)[32], int col0, auto masked) {
 #pragma unroll
-        for (int jj = 0; jj < 32; jj += 2) {
-          const int c = col0 + jj;
-          const float2 sv = make_float2(__uint_as_float(y[jj]), __uint_as_float(y[jj + 1]));
-          float2 w = __fmul2_rn(sv, sv);
-          if constexpr (decltype(masked)::value) {
-            if (key0 + c > qrow) w.x = 0.f;
-            if (key0 + c + 1 > qrow) w.y = 0.f;
+        for (int i = 0; i < 4; ++i) {
+          const uint4 t4 = rv4[col0 / 8 + i];          // r of 8 keys
+          const uint32_t rr[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) {
+            const int jj = 8 * i + e, c = col0 + jj;
+            const float2 sv = make_float2(__uint_as_float(y[jj]), __uint_as_float(y[jj + 1]));
+            float2 w = __fmul2_rn(sv, sv);
+            if constexpr (decltype(masked)::value) {
+              if (key0 + c > qrow) w.x = 0.f;
+              if (key0 + c + 1 > qrow) w.y = 0.f;
+            }
+            pk[(c & 63) / 2] = scale_pair(pack_bf16(w.x, w.y), rr[e / 2]);
           }
-          pk[(c & 63) / 2] = pack_bf16(w.x, w.y);
         }
       };
+      // The weights overwrite score columns [0,64) of the buffer (this warp's lanes only): those of keys 0..63 once
+      // the scores of keys 0..63 are in registers, those of keys 64..127 after.
       auto weigh_tile = [&](auto masked) {
         tmem_ld32(scol, ya);
         tmem_ld32(scol + 32, yb);
@@ -366,15 +392,15 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         weigh(yb, pk0, 32, masked);
         tmem_ld32(scol + 64, ya);
         tmem_ld32(scol + 96, yb);
+        tmem_st32(scol, pk0);
         tmem_wait_ld(ya);
-        weigh(ya, pk1, 64, masked);
+        tmem_wait_st();                 // pk0 is reused
+        weigh(ya, pk0, 64, masked);
         tmem_wait_ld(yb);
-        weigh(yb, pk1, 96, masked);
+        weigh(yb, pk0, 96, masked);
+        tmem_st32(scol + 32, pk0);
       };
       if (diag) weigh_tile(std::true_type{}); else weigh_tile(std::false_type{});
-      // the weights overwrite score columns [0,64) of the buffer: this warp's lanes only, all read above
-      tmem_st32(scol, pk0);
-      tmem_st32(scol + 32, pk1);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_PFULL + b));
@@ -423,24 +449,18 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
 }  // namespace
 
-// workspace: V' [BH][T][64] bf16, then r [BH][T] bf16
-static size_t vs_bytes(const Problem& p) { return ((size_t)p.B * p.H * p.T * D * 2 + 255) / 256 * 256; }
-
-size_t tc_quadratic_workspace_bytes(const Problem& p) {
-  return vs_bytes(p) + ((size_t)p.B * p.H * p.T * 2 + 255) / 256 * 256;
-}
+// workspace: r [BH][T] bf16
+size_t tc_quadratic_workspace_bytes(const Problem& p) { return ((size_t)p.B * p.H * p.T * 2 + 255) / 256 * 256; }
 
 void tc_quadratic(const Problem& p, void* workspace, int* device_status, LaunchCtx& ctx) {
   const int BH = p.B * p.H;
-  __nv_bfloat16* vs = static_cast<__nv_bfloat16*>(workspace);
-  __nv_bfloat16* rscale = reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(workspace) + vs_bytes(p));
+  __nv_bfloat16* rscale = static_cast<__nv_bfloat16*>(workspace);
   const size_t n_rows = (size_t)BH * p.T;
-  quad_prescale_kernel<<<(unsigned)((n_rows + 31) / 32), 256, 0, ctx.stream>>>(
-      static_cast<const __nv_bfloat16*>(p.k), static_cast<const __nv_bfloat16*>(p.v), vs, rscale, n_rows);
+  quad_rscale_kernel<<<(unsigned)((n_rows + 31) / 32), 256, 0, ctx.stream>>>(static_cast<const __nv_bfloat16*>(p.k), rscale, n_rows);
   note_launch(ctx);
   CUtensorMap tmQ, tmK, tmV;
   const int kt = KTILE / p.groups;
-  if (!make_tile_map(&tmQ, p.q, BH, p.T, QT) || !make_tile_map(&tmK, p.k, BH, p.T, kt) || !make_tile_map(&tmV, vs, BH, p.T, kt)) {
+  if (!make_tile_map(&tmQ, p.q, BH, p.T, QT) || !make_tile_map(&tmK, p.k, BH, p.T, kt) || !make_tile_map(&tmV, p.v, BH, p.T, kt)) {
     ctx.status = KATA_ERR_CUDA;
     return;
   }

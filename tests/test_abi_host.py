@@ -108,8 +108,8 @@ def test_invalid_arguments(L, fn):
 
 def test_scan_workspace_and_plan(L):
     o = kb.make_opts(kb.KATA_BF16)
-    # tensor-core quadratic path: scaled values (bf16, size of v) + one bf16 scale per key
-    assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 4, 16, 4096, 64, 64, 64, o) == 4 * 16 * 4096 * (64 + 1) * 2
+    # tensor-core quadratic path: one bf16 scale per key (the values are used as they are)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 4, 16, 4096, 64, 64, 64, o) == 4 * 16 * 4096 * 2
     o32 = kb.make_opts(kb.KATA_F32)
     assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 4, 16, 4096, 64, 64, 64, o32) == 0
     # sequential walk of the feature-split kernel: tile counters and the ticket, the scaled values and key scales of
