@@ -22,8 +22,9 @@
  *     to the element type (round-to-nearest-even).  On the bf16 tensor-core kernels the OPERANDS of the matrix
  *     products are bf16: the chunked forms read the running state through a bf16 copy taken once per tile of 128
  *     tokens (S and Z are accumulated in fp32, but psi(q)^T S and psi(q)^T Z see them rounded), the intra-tile
- *     weights (q.k)^2 are rounded to bf16 before they multiply the values, and the key scale 1/||k||^2 and the scaled
- *     values v/||k||^2 are rounded separately.  The convex weights of the output gate therefore sum to 1 only to
+ *     weights (q.k)^2 are rounded to bf16 before they multiply the values, and the key scale 1/||k||^2 is rounded to
+ *     bf16 (the chunked forms multiply it into the values, v/||k||^2 rounded again; the quadratic form into the
+ *     weights, rounded again, whose row sum is then the normaliser).  The convex weights of the output gate therefore sum to 1 only to
  *     about 2^-8, and a normaliser that is tiny against its terms (a query nearly orthogonal to every key before it)
  *     can come out <= 0 from the rounded operands, in which case out = 0 as for an exact zero.  All of it stays
  *     inside the 2e-2 tolerance of the bf16 tests.
@@ -156,8 +157,8 @@ typedef struct kata_opts {
  * Quadratic ("flash-style") forward: the definition evaluated tile by tile, never forming
  * the d_k^2-wide state (section "Why the PSD feature keeps to O(T) or O(T^2)"; weights from
  * the rank-one lift identity <uu^T,vv^T>_F = (u^T v)^2).  O(T^2) work.  C is ignored.
- * Workspace: kata_workspace_bytes(KATA_FN_QUADRATIC, ...) -- the tensor-core path keeps the values scaled
- * by 1/||k||^2 there (about the size of v); the fp32 path needs none.
+ * Workspace: kata_workspace_bytes(KATA_FN_QUADRATIC, ...) -- the tensor-core path keeps the key scales
+ * 1/||k||^2 there (one bf16 per key and head); the fp32 path needs none.
  */
 int kata_fwd_quadratic(const void* q, const void* k, const void* v, void* out,
                        int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts);
