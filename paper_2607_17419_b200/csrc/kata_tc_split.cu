@@ -6,7 +6,7 @@
 // u[8g+i] u[8h+j].  <psi(q), psi(k)> = (q.k)^2 = sum over the 36 block pairs of w_gh <Q_gh, K_gh> with w = 1 on
 // the diagonal pairs (which hold both (i,j) and (j,i)) and w = 2 off it.  One CTA owns 4 block pairs = 256 state
 // rows (two M = 128 accumulator tiles S[m], 80 fp32 TMEM columns each: 64 value columns, the normaliser column,
-// padding); nine CTAs make a head and never talk to each other while they run.  With the key scale r = 1/||k||^2
+// padding); nine CTAs make a head; they meet only through the shares they publish.  With the key scale r = 1/||k||^2
 // folded into the values (V' = r V, written once per head by a light pre-pass) and the normaliser carried as column
 // 64 of every B operand, per tile of 128 tokens a CTA does
 //   update   S[m] += Psi(K)_m^T [V' | r]      A = the products, built by token threads in shared memory (MN-major),
@@ -35,6 +35,12 @@
 // hundred cycles from arrival to the waiter's next instruction, and a pipeline whose buffers are all single (shared
 // memory and TMEM are full) turns each of them into a round trip; a version of this kernel built that way spent
 // 5 k cycles per tile on synchronisation alone.
+//
+// Blockwise map (section "KATA-Mg", g = 2 or 4 feature groups): only the block pairs inside a group carry state (20
+// or 12 of the 36), the intra-tile weights are the sum over the groups of the squared per-group scores, and a head is
+// cut differently: the kernel is a template over (accumulator tiles per CTA, groups, CTAs per head) = (2, 1, 9) for
+// the full lift, (1, 2, 10) or (2, 2, 5) for two groups, (1, 4, 6) for four.  With fewer than eight CTAs per head a
+// CTA weighs two of the eight key runs of a tile.  Each CTA finishes ceil(128 / CTAs per head) query rows of a tile.
 //
 // Warps (896 threads): 0 TMA producer, 1 update issuer, 2 read issuer, 3 score issuer; 4-11 key teams (team m builds
 // the products of accumulator tile m; team 0 also places r); 12-15 query team; 16-19 state team; 20-23 share team;
