@@ -169,27 +169,27 @@ int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanP
     } else if (o.scan_group > 0) {
       G = (o.scan_group + cpt - 1) / cpt * cpt;
     } else {
-      // Grouped (reduce, scan, restart: 1.5x the HBM traffic, three or more launches) or one pass per head,
-      // whichever the cost model says is faster.  Measured on B200: a CTA walks its tiles at about 1.3 us per
-      // tile (1.75 us for both passes of a group), the kernel streams about 6 GB/ms, the extra launches cost
-      // about 60 us.
+      // One pass per head, or the groups of the single-launch scan (every group walked twice, the second time with
+      // its keys and values in L2 only where the groups of all CTAs fit there: up to 1.5x the HBM traffic),
+      // whichever the cost model says is faster.  Measured on B200: a CTA alone walks its tiles at about 1.25 us a
+      // tile in one pass and 2.15 us a tile for the two passes of a group, a group costs about 12 us on top (two
+      // pipeline ramps and the look-back), the kernel streams about 6 GB/ms.  Groups: one per CTA in one wave.
       const double n_tiles = (double)((p.T + tc_order1_tile() - 1) / tc_order1_tile());
       const double hbm_us = (double)BH * n_tiles * 65536.0 / 6.0e6;
-      const double one_pass = fmax(hbm_us, ceil(BH / 148.0) * n_tiles * 1.3);
-      int ng = (4 * 148 + BH - 1) / BH;                    // about four groups per SM over the run of the kernel
-      if (ng < 2) ng = 2;
-      G = (NC + ng - 1) / ng;
-      if (G < 2 * cpt) G = 2 * cpt;                        // at least two tiles per group
-      G = (G + cpt - 1) / cpt * cpt;
-      if (G > NC) G = NC;
-      const double groups = ceil((double)NC / G), tiles_per_group = (double)G / cpt;
-      const double grouped = fmax(1.5 * hbm_us, ceil(BH * groups / 148.0) * tiles_per_group * 1.75) + 60.0;
-      if (one_pass <= grouped) G = NC;
+      const double one_pass = fmax(hbm_us, ceil(BH / 148.0) * n_tiles * 1.25);
+      G = NC;
+      const int ng = 148 / BH;
+      if (ng >= 2 && n_tiles >= 2 * ng) {
+        const double tiles_per_group = ceil(n_tiles / ng);
+        const double grouped = fmax(1.5 * hbm_us, tiles_per_group * 2.15) + 12.0;
+        if (grouped < one_pass) G = (int)tiles_per_group * cpt;
+      }
     }
     if (G > NC) G = NC;
     plan.chunks_per_group = G;
     plan.n_groups = (NC + G - 1) / G;
-    plan.rounds = plan.n_groups > 2 ? ceil_log2(plan.n_groups - 1) : 0;
+    // the chained scan over the group states: one hop per anchor (every eighth group) instead of doubling rounds
+    plan.rounds = plan.n_groups > 1 ? (plan.n_groups - 2) / 8 + 1 : 0;
     return KATA_OK;
   }
   int slices;
@@ -244,7 +244,9 @@ int make_plan(int fn, const Problem& p, const Opts& o, bool tensor, int C, ScanP
 size_t inner_workspace(int fn, const ScanPlan& plan, const Problem& p, size_t state_elems) {
   if (fn == KATA_FN_QUADRATIC) return 0;
   if (fn == KATA_FN_CHUNKED && plan.n_groups == 1) return 0;
-  return 2 * align_up((size_t)p.B * p.H * plan.n_groups * state_elems * sizeof(float));
+  // the first-order kernels also keep one flag per group and a counter behind the two state buffers
+  const size_t flags = p.feature_order == 1 ? align_up(((size_t)p.B * p.H * plan.n_groups + 1) * sizeof(int)) : 0;
+  return 2 * align_up((size_t)p.B * p.H * plan.n_groups * state_elems * sizeof(float)) + flags;
 }
 
 size_t elem_bytes(int dtype) { return dtype == KATA_F32 ? 4 : 2; }

@@ -11,13 +11,18 @@
 //                                                  columns, the normaliser row, zero rows), B = the key tile;
 //                                                  fp32 accumulators stay in TMEM for the whole group
 //   out      O / D                                 (0 where D = 0)
-// With init_state the group starts from a given state, with final_state it leaves its state behind, with
-// write_out = 0 only the state is computed (keys and values are the only loads): these are the three passes of
-// the reduce-then-scan pipeline over groups of tiles.  HBM-bound: q, k, v in, o out, 512 bytes per token.
+// A head of many tiles and few heads: the chunk axis is cut into groups of tiles and the CTAs (one per SM) take
+// groups until none is left.  A group is walked twice.  Pass 0 builds the state of the group alone (keys and values
+// are the only loads) and publishes it; the look-back then adds up the states of the groups before it (a chained
+// scan over the group states: every eighth group is an anchor that publishes the sum of everything up to itself,
+// the others add the anchor and the groups after it, in order); pass 1 starts from that sum and writes the outputs,
+// with the keys and values of the group still in L2 where the groups are small.  One launch; the sum does not depend
+// on the order in which the CTAs run.  HBM-bound: q, k, v in, o out, 512 bytes per token.
 //
-// Warps (512 threads): 0 TMA producer; 1 issuer of the score and update MMAs; 2 issuer of the intra and inter
-// MMAs; 4-6 state snapshot (TMEM -> bf16 rows in shared memory, 32 rows each) and state import / export;
-// 8-15 weights and epilogue (two warps per lane quadrant, one per half of the columns).  All waits are bounded.
+// Warps (512 threads): 0 TMA producer; 1, 2, 3, 7 MMA issuers (scores, intra, update, inter: one thread gets an MMA
+// out about every hundred cycles whatever its size, so every group of MMAs has its own); 4-6 state snapshot (TMEM
+// -> bf16 rows in shared memory, 32 rows each) and state export; 4-7 state import; 8-15 weights and epilogue (two
+// warps per lane quadrant, one per half of the columns).  All waits are bounded.
 #include <cuda.h>
 
 #include "kata_common.cuh"
@@ -34,7 +39,7 @@ constexpr int CT = 128;            // tokens per tile
 constexpr int NTHREADS = 512;
 constexpr int NSTAGE = 3;
 constexpr int SROWS = 80;          // state rows kept: 64 value columns, the normaliser row, 15 zero rows
-constexpr int W_MMA_A = 1, W_MMA_B = 2, W_SNAP0 = 4, W_BLD0 = 8;
+constexpr int W_MMA_A = 1, W_MMA_B = 2, W_MMA_U = 3, W_SNAP0 = 4, W_MMA_R = 7, W_BLD0 = 8;
 
 constexpr uint32_t COL_S = 0;      // 64 fp32: [S | Z]^T, lanes = (v, z, 0..), columns = feature a
 constexpr uint32_t COL_P = 64;     // 2 x 128 fp32 scores; the bf16 weights overwrite columns [0,64) of a buffer
@@ -65,20 +70,53 @@ enum {
   BAR_SNAP_LD = 17,  // state copied out of TMEM (96 threads): the next update may run
   BAR_SNAP_ST = 18,  // [2] snapshot stored into buffer 0 / 1 (96 threads): the inter MMA that reads it may run
   BAR_DRAIN = 20,
-  BAR_COUNT = 21
+  BAR_R_DONE = 21,   // [2] inter-tile part of the result issued and complete: the intra MMAs may add to it
+  BAR_COUNT = 23
 };
 
 struct OArgs {
   __nv_bfloat16* out;
-  const float* init_state;   // [BH][n_groups][80][64]: group g starts from slot g - 1 (null: zero)
-  float* final_state;        // [BH][n_groups][80][64]: state of the group alone or continued (null: not kept)
   int* device_status;
   int Tlen;
   int n_tiles;
   int tiles_per_group;
   int n_groups;
-  int write_out;
+  // more than one group: group states [BH][n_groups][80][64] of the groups alone and of the anchor groups with
+  // everything before them, one flag per group, the ticket counter, B * H
+  float* local_state;
+  float* anchor_state;
+  int* flags;
+  unsigned* ticket;
+  int BH;
 };
+
+// Single-launch form: flag values of a group.  A group that gave up poisons its flag so that its successors give up
+// at once instead of waiting out their limits.
+constexpr int kFlagLocal = 1, kFlagAnchor = 2, kFlagPoison = 99;
+constexpr int kAnchorEvery = 8;
+
+// Bounded wait for a group's flag (2 s of wall time: the group may belong to a CTA that started a wave earlier).
+__device__ __forceinline__ bool wait_flag(const int* p, int want, volatile int* abort_flag) {
+  unsigned t0 = 0;
+  for (uint32_t i = 0;; ++i) {
+    int v;
+    unsigned t1;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    if (v == kFlagPoison) break;
+    if (v >= want) return true;
+    if (*abort_flag) return false;
+    asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t1));
+    if (i == 0) t0 = t1;
+    if (t1 - t0 > 2000000000u) break;
+    __nanosleep(64);
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void publish_flag(int* p, int v) {
+  __threadfence();
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 
 // One fp32 state row (64 features) as a bf16 row of a snapshot (128B swizzle: chunk index xor row-in-atom).
 __device__ __forceinline__ void snap_store_row(unsigned char* sp, int row, const uint32_t (&lo)[32], const uint32_t (&hi)[32]) {
@@ -110,36 +148,10 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   volatile int* abort_flag = &abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int bh = blockIdx.x, grp = blockIdx.y;
-  const int t_begin = grp * args.tiles_per_group;
-  const int n = min(args.n_tiles, t_begin + args.tiles_per_group) - t_begin;   // tiles of this group
-  if (n <= 0) return;
-  const bool wo = args.write_out != 0;
+  const bool fused = args.flags != nullptr;
   constexpr size_t E = (size_t)SROWS * D;
-  const float* init = (args.init_state != nullptr && grp > 0)
-                          ? args.init_state + ((size_t)bh * args.n_groups + (grp - 1)) * E : nullptr;
-  float* fin = args.final_state != nullptr ? args.final_state + ((size_t)bh * args.n_groups + grp) * E : nullptr;
-  const bool resume = init != nullptr;
-
   if (tid == 0) {
     abort_s = 0;
-    for (int i = 0; i < NSTAGE; ++i) {
-      mbar_init(bar(BAR_FULL + i), 1);
-      mbar_init(bar(BAR_EMPTY + i), wo ? 2 : 1);
-    }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(BAR_S_FULL + i), 1);
-      mbar_init(bar(BAR_P_FULL + i), 256);
-      mbar_init(bar(BAR_P_EMPTY + i), 1);
-      mbar_init(bar(BAR_O_FULL + i), 1);
-      mbar_init(bar(BAR_O_EMPTY + i), 256);
-    }
-    mbar_init(bar(BAR_U_DONE), 1);
-    mbar_init(bar(BAR_SNAP_LD), 96);
-    mbar_init(bar(BAR_SNAP_ST), 96);
-    mbar_init(bar(BAR_SNAP_ST + 1), 96);
-    mbar_init(bar(BAR_DRAIN), 2);
-    fence_mbar_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmV);
@@ -158,20 +170,103 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
+  // More than one group: the CTAs take groups until none is left.  Groups are dealt in the order in which they are
+  // asked for, earlier groups of every head first: the groups that a CTA waits for belong to CTAs that are working
+  // on them or are done with them, whatever the size of the grid.
+  __shared__ unsigned ticket_s;
+  bool bars_live = false, dead = false;
+  for (;;) {
+  int bh = blockIdx.x, grp = 0;
+  if (fused) {
+    __syncthreads();
+    if (tid == 0) ticket_s = atomicAdd(args.ticket, 1u);
+    __syncthreads();
+    if (ticket_s >= (unsigned)args.BH * (unsigned)args.n_groups) break;
+    grp = (int)(ticket_s / (unsigned)args.BH);
+    bh = (int)(ticket_s % (unsigned)args.BH);
+  }
+  const int t_begin = grp * args.tiles_per_group;
+  const int n = min(args.n_tiles, t_begin + args.tiles_per_group) - t_begin;   // tiles of this group
+  const size_t slot = (size_t)bh * args.n_groups + grp;
+  // Pass 0 builds the state of the group alone (keys and values only) and publishes it, pass 1 starts from the sum
+  // of the groups before it and writes the outputs; the last group of a head has no pass 0.
+  const int pass_first = fused && grp + 1 < args.n_groups ? 0 : 1;
+  for (int pass = pass_first; pass <= 1; ++pass) {
   bool ok = true;
-  // Everything above touched only this CTA's shared memory and TMEM.  As a programmatic dependent launch (the
-  // restart pass behind the scan rounds) the CTA got here while the kernel ahead was still draining; its results
-  // (the prefix states) are visible from here on.  A no-op in an ordinary launch.
-  cudaGridDependencySynchronize();
+  const bool wo = pass == 1;
+  float* fin = pass == 0 ? args.local_state + slot * E : nullptr;
+  const bool lookback = fused && pass == 1 && grp > 0;
+  const bool resume = lookback;
 
+  if (tid == 0) {
+    if (bars_live)
+      for (int i = 0; i < BAR_COUNT; ++i) mbar_inval(bar(i));
+    for (int i = 0; i < NSTAGE; ++i) {
+      mbar_init(bar(BAR_FULL + i), 1);
+      mbar_init(bar(BAR_EMPTY + i), wo ? 4 : 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BAR_S_FULL + i), 1);
+      mbar_init(bar(BAR_P_FULL + i), 256);
+      mbar_init(bar(BAR_P_EMPTY + i), 1);
+      mbar_init(bar(BAR_O_FULL + i), 1);
+      mbar_init(bar(BAR_O_EMPTY + i), 256);
+      mbar_init(bar(BAR_R_DONE + i), 1);
+    }
+    mbar_init(bar(BAR_U_DONE), 1);
+    mbar_init(bar(BAR_SNAP_LD), 96);
+    mbar_init(bar(BAR_SNAP_ST), 96);
+    mbar_init(bar(BAR_SNAP_ST + 1), 96);
+    mbar_init(bar(BAR_DRAIN), 4);
+    fence_mbar_init();
+  }
+  __syncthreads();
+
+  if (lookback) {
+    // Look-back: the nearest anchor group at or before grp - 1 holds the sum of everything up to itself (group 0 is
+    // its own anchor); the groups between it and this one are added in order, so the sum does not depend on who was
+    // first.  All threads take part (the loads of up to eight group states are in flight together); the sum goes
+    // through the first stage buffer, which is idle between the passes.  An anchor adds its own state for the groups
+    // behind it.
+    const int anchor = (grp - 1) / kAnchorEvery * kAnchorEvery;
+    const int cnt = grp - anchor;                                   // 1 .. 8
+    bool got = true;
+    for (int g2 = anchor; g2 < grp && got; ++g2)
+      got = wait_flag(args.flags + (slot - grp + g2), (g2 == anchor && anchor > 0) ? kFlagAnchor : kFlagLocal, abort_flag);
+    const bool publish = grp % kAnchorEvery == 0 && grp + 1 < args.n_groups;
+    float4* scratch = reinterpret_cast<float4*>(base);
+    if (got) {
+      for (int i = tid; i < (int)(E / 4); i += NTHREADS) {
+        float4 part[kAnchorEvery];
+#pragma unroll
+        for (int u = 0; u < kAnchorEvery; ++u)
+          if (u < cnt) {
+            const float* sb = (u == 0 && anchor > 0) ? args.anchor_state : args.local_state;
+            part[u] = __ldcg(reinterpret_cast<const float4*>(sb + (slot - grp + anchor + u) * E) + i);
+          }
+        float4 acc = part[0];
+#pragma unroll
+        for (int u = 1; u < kAnchorEvery; ++u)
+          if (u < cnt) { acc.x += part[u].x; acc.y += part[u].y; acc.z += part[u].z; acc.w += part[u].w; }
+        scratch[i] = acc;
+        if (publish) {
+          const float4 own = __ldcg(reinterpret_cast<const float4*>(args.local_state + slot * E) + i);
+          reinterpret_cast<float4*>(args.anchor_state + slot * E)[i] = make_float4(acc.x + own.x, acc.y + own.y, acc.z + own.z, acc.w + own.w);
+        }
+      }
+    }
+    fence_async_smem();   // the stage buffer goes back to the TMA
+    __syncthreads();
+    if (publish && tid == 0) publish_flag(args.flags + slot, *abort_flag ? kFlagPoison : kFlagAnchor);
+  }
   if (resume) {
     // the state before the first tile: into the accumulators and, as bf16, into snapshot 0
     if (warp >= W_SNAP0 && warp < W_SNAP0 + 4) {
       const uint32_t q4 = warp & 3;
       const int row = q4 * 32 + lane;
       uint32_t lo[32], hi[32];
-      if (row < SROWS) {
-        const float4* src = reinterpret_cast<const float4*>(init + (size_t)row * D);
+      if (row < SROWS && !*abort_flag) {
+        const float4* src = reinterpret_cast<const float4*>(base) + (size_t)row * (D / 4);
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           const float4 a = src[c], b = src[8 + c];
@@ -193,6 +288,7 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (*abort_flag) ok = false;
   }
 
   if (warp == 0) {
@@ -200,7 +296,7 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (lane == 0) {
       for (int j = 0; j < n && ok; ++j) {
         const int s = j % NSTAGE;
-        ok = wait_or_abort(bar(BAR_EMPTY + s), ((j / NSTAGE) & 1) ^ 1, abort_flag);
+        ok = wait_or_abort_counted(bar(BAR_EMPTY + s), ((j / NSTAGE) & 1) ^ 1, abort_flag);
         if (!ok) break;
         const int tok = (t_begin + j) * CT;
         mbar_arrive_expect_tx(bar(BAR_FULL + s), wo ? 49152u : 32768u);
@@ -210,30 +306,44 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     }
   } else if (warp == W_MMA_A) {
-    // =========================== scores P = Q K^T and the state update ===========================
-    if (lane == 0) {
+    // =========================== scores P = Q K^T ===========================
+    // Four issuer warps, one per MMA group of a tile: a thread gets an MMA out about every hundred cycles whatever
+    // its size, and the groups of a tile do not depend on one another.  Every lane waits, lane 0 issues (a warp of
+    // waiters is woken sooner than a single waiting lane).
+    if (wo) {
       const uint32_t idQK = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 128);
-      const uint32_t idU = instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64);     // A and B MN-major (token = K)
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
-      const uint32_t ones = smem_u32(base + OFF_ONES);
       for (int j = 0; j < n && ok; ++j) {
         const int s = j % NSTAGE, b = j & 1;
-        ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag);
+        ok = wait_or_abort_counted(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
+             wait_or_abort_counted(bar(BAR_P_EMPTY + b), ((j >> 1) & 1) ^ 1, abort_flag);
         if (!ok) break;
-        const uint32_t qa = smem_u32(qtile(s)), ka = smem_u32(ktile(s)), va = smem_u32(vtile(s));
-        if (wo) {
-          ok = wait_or_abort(bar(BAR_P_EMPTY + b), ((j >> 1) & 1) ^ 1, abort_flag);
-          if (!ok) break;
+        if (lane == 0) {
+          const uint32_t qa = smem_u32(qtile(s)), ka = smem_u32(ktile(s));
           tc_fence_after();
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
             mma_f16_ss(tb + COL_P + b * 128, at(dk, qa + ks * 32), at(dk, ka + ks * 32), idQK, ks > 0);
           mma_commit(bar(BAR_S_FULL + b));
+          mma_commit(bar(BAR_EMPTY + s));
         }
-        if (j + 1 < n || fin != nullptr) {
-          // the accumulators are free once the snapshot of the previous state has left TMEM
-          if (wo && j > 0) ok = wait_or_abort(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
-          if (!ok) break;
+        __syncwarp();
+      }
+    }
+  } else if (warp == W_MMA_U) {
+    // =========================== state update [S | Z]^T += [V | 1]^T K ===========================
+    const uint32_t idU = instr_desc(kFmtBF16, kFmtBF16, 1, 1, 128, 64);     // A and B MN-major (token = K)
+    const uint32_t ones = smem_u32(base + OFF_ONES);
+    for (int j = 0; j < n && ok; ++j) {
+      const int s = j % NSTAGE;
+      const bool upd = j + 1 < n || fin != nullptr;
+      ok = wait_or_abort_counted(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag);
+      // the accumulators are free once the snapshot of the previous state has left TMEM
+      if (ok && upd && wo && j > 0) ok = wait_or_abort_counted(bar(BAR_SNAP_LD), (j - 1) & 1, abort_flag);
+      if (!ok) break;
+      if (lane == 0) {
+        const uint32_t ka = smem_u32(ktile(s)), va = smem_u32(vtile(s));
+        if (upd) {
           tc_fence_after();
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
@@ -246,38 +356,58 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         mma_commit(bar(BAR_EMPTY + s));
       }
+      __syncwarp();
     }
-  } else if (warp == W_MMA_B) {
-    // =========================== [O | D] = P [V | 1] + Q [S | Z]^T ===========================
-    if (lane == 0 && wo) {
-      const uint32_t idPV = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);    // A tmem, B MN-major
+  } else if (warp == W_MMA_R) {
+    // =========================== inter-tile part [O | D] = Q [S | Z]^T (opens the accumulator of the tile) ===========================
+    if (wo) {
       const uint32_t idR = instr_desc(kFmtBF16, kFmtBF16, 0, 0, 128, 80);
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);
-      const uint32_t ones = smem_u32(base + OFF_ONES), spa = smem_u32(base + OFF_SP);
+      const uint32_t spa = smem_u32(base + OFF_SP);
       for (int j = 0; j < n && ok; ++j) {
         const int s = j % NSTAGE, b = j & 1;
-        ok = wait_or_abort(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_P_FULL + b), (j >> 1) & 1, abort_flag) &&
-             wait_or_abort(bar(BAR_O_EMPTY + b), ((j >> 1) & 1) ^ 1, abort_flag);
+        ok = wait_or_abort_counted(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
+             wait_or_abort_counted(bar(BAR_O_EMPTY + b), ((j >> 1) & 1) ^ 1, abort_flag);
+        // the snapshot after tile j - 1 went to buffer j & 1; it is that buffer's ((j - 1) / 2)-th
+        if (ok && j > 0) ok = wait_or_abort_counted(bar(BAR_SNAP_ST + (j & 1)), ((j - 1) >> 1) & 1, abort_flag);
         if (!ok) break;
-        tc_fence_after();
-        const uint32_t qa = smem_u32(qtile(s)), va = smem_u32(vtile(s));
+        if (lane == 0) {
+          if (resume || j > 0) {
+            const uint32_t qa = smem_u32(qtile(s));
+            tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          mma_f16_ts(tb + COL_O + b * 80, tb + COL_P + b * 128 + ks * 8,
-                     smem_desc(va + ks * 2048, ones - va, 1024, kSwizzle128B), idPV, ks > 0);
-        mma_commit(bar(BAR_P_EMPTY + b));
-        if (resume || j > 0) {
-          // the snapshot after tile j - 1 went to buffer j & 1; it is that buffer's ((j - 1) / 2)-th
-          if (j > 0) ok = wait_or_abort(bar(BAR_SNAP_ST + (j & 1)), ((j - 1) >> 1) & 1, abort_flag);
-          if (!ok) break;
+            for (int ks = 0; ks < 4; ++ks)
+              mma_f16_ss(tb + COL_O + b * 80, at(dk, qa + ks * 32), at(dk, spa + (j & 1) * SP_BYTES + ks * 32), idR, ks > 0);
+          }
+          mma_commit(bar(BAR_R_DONE + b));
+          mma_commit(bar(BAR_EMPTY + s));
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp == W_MMA_B) {
+    // =========================== intra-tile part [O | D] += P [V | 1] ===========================
+    if (wo) {
+      const uint32_t idPV = instr_desc(kFmtBF16, kFmtBF16, 0, 1, 128, 80);    // A tmem, B MN-major
+      const uint32_t ones = smem_u32(base + OFF_ONES);
+      for (int j = 0; j < n && ok; ++j) {
+        const int s = j % NSTAGE, b = j & 1;
+        ok = wait_or_abort_counted(bar(BAR_FULL + s), (j / NSTAGE) & 1, abort_flag) &&
+             wait_or_abort_counted(bar(BAR_P_FULL + b), (j >> 1) & 1, abort_flag) &&
+             wait_or_abort_counted(bar(BAR_R_DONE + b), (j >> 1) & 1, abort_flag);
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t va = smem_u32(vtile(s));
           tc_fence_after();
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            mma_f16_ss(tb + COL_O + b * 80, at(dk, qa + ks * 32), at(dk, spa + (j & 1) * SP_BYTES + ks * 32), idR, 1u);
+          for (int ks = 0; ks < 8; ++ks)
+            mma_f16_ts(tb + COL_O + b * 80, tb + COL_P + b * 128 + ks * 8,
+                       smem_desc(va + ks * 2048, ones - va, 1024, kSwizzle128B), idPV, (resume || j > 0 || ks > 0) ? 1u : 0u);
+          mma_commit(bar(BAR_P_EMPTY + b));
+          mma_commit(bar(BAR_O_FULL + b));
+          mma_commit(bar(BAR_EMPTY + s));
         }
-        mma_commit(bar(BAR_O_FULL + b));
-        mma_commit(bar(BAR_EMPTY + s));
+        __syncwarp();
       }
     }
   } else if (warp >= W_SNAP0 && warp < W_SNAP0 + 3) {
@@ -286,9 +416,9 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int row = q4 * 32 + lane;
     for (int j = wo ? 0 : n - 1; j < n && ok; ++j) {
       if (!(j + 1 < n || fin != nullptr)) break;          // the last update is skipped when nobody needs it
-      ok = wait_or_abort(bar(BAR_U_DONE), wo ? (j & 1) : 0, abort_flag);
+      ok = wait_or_abort_counted(bar(BAR_U_DONE), wo ? (j & 1) : 0, abort_flag);
       // the snapshot buffer written below was read by the inter MMA of tile j - 1
-      if (ok && wo && j > 0 && j + 1 < n) ok = wait_or_abort(bar(BAR_O_FULL + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag);
+      if (ok && wo && j > 0 && j + 1 < n) ok = wait_or_abort_counted(bar(BAR_O_FULL + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       uint32_t lo[32], hi[32];
@@ -319,6 +449,11 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
       }
     }
+    if (fused && pass == 0) {
+      // the group's own state is in place: tell the groups behind it
+      asm volatile("bar.sync 6, 96;" ::: "memory");
+      if (warp == W_SNAP0 && lane == 0) publish_flag(args.flags + slot, *abort_flag ? kFlagPoison : kFlagLocal);
+    }
   } else if (warp >= W_BLD0 && wo) {
     // =========================== weights and epilogue (256 threads) ===========================
     const uint32_t q4 = warp & 3;
@@ -326,7 +461,7 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int rowl = q4 * 32 + lane;             // token of the tile (= TMEM lane)
     auto epilogue = [&](int jj) -> bool {
       const int bb = jj & 1;
-      if (!wait_or_abort(bar(BAR_O_FULL + bb), (jj >> 1) & 1, abort_flag)) return false;
+      if (!wait_or_abort_counted(bar(BAR_O_FULL + bb), (jj >> 1) & 1, abort_flag)) return false;
       tc_fence_after();
       uint32_t o[32], dn[16];
       tmem_ld32(tmem_addr(tb, q4 * 32, COL_O + bb * 80 + ch * 32), o);
@@ -354,7 +489,7 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     };
     for (int j = 0; j < n && ok; ++j) {
       const int b = j & 1;
-      ok = wait_or_abort(bar(BAR_S_FULL + b), (j >> 1) & 1, abort_flag);
+      ok = wait_or_abort_counted(bar(BAR_S_FULL + b), (j >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       const uint32_t scol = tmem_addr(tb, q4 * 32, COL_P + b * 128 + ch * 64);
@@ -384,16 +519,25 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (ok) ok = epilogue(n - 1);
   }
 
-  // ---------------- teardown ----------------
+  // ---------------- end of the pass ----------------
   if (!ok && args.device_status != nullptr) atomicExch(args.device_status, (int)KATA_ERR_DEVICE_TIMEOUT);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if ((warp == W_MMA_A || warp == W_MMA_B) && lane == 0) {
+  if ((warp == W_MMA_A || warp == W_MMA_B || warp == W_MMA_U || warp == W_MMA_R) && lane == 0) {
     mma_commit(bar(BAR_DRAIN));
     mbar_wait(bar(BAR_DRAIN), 0);
   }
   __syncthreads();
+  bars_live = true;
+  if (*abort_flag) {
+    if (fused && tid == 0) publish_flag(args.flags + slot, kFlagPoison);
+    dead = true;
+    break;
+  }
+  }
+  if (!fused || dead) break;
+  }
   if (warp == 0) tmem_dealloc(tb, TMEM_COLS);
 }
 
@@ -427,42 +571,37 @@ void tc_order1(const Problem& p, const ScanPlan& plan, bool use_scan, int C, flo
   const size_t E = tc_order1_state_elems();
   float* bufA = ws;
   float* bufB = NG > 1 ? ws + (size_t)BH * NG * E : nullptr;
-  const float* incl = nullptr;
+  a.local_state = nullptr;
+  a.anchor_state = nullptr;
+  a.flags = nullptr;
+  a.ticket = nullptr;
+  a.BH = BH;
   if (NG > 1) {
-    // pass 1: local states of all groups but the last; pass 2: inclusive scan over them
-    a.init_state = nullptr;
-    a.final_state = bufA;
-    a.write_out = 0;
-    tc_order1_kernel<<<dim3(BH, NG - 1), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
-    note_launch(ctx);
-    incl = scan_group_states(bufA, bufB, BH, NG, NG - 1, E, ctx);
-  }
-  // pass 3: every group restarts from the prefix before it
-  a.init_state = incl;
-  a.final_state = nullptr;
-  a.write_out = 1;
-  if (NG > 1) {
-    // behind the scan rounds: resident, with its prologue done, while the last round drains
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(BH, NG);
-    cfg.blockDim = dim3(NTHREADS);
-    cfg.dynamicSmemBytes = SMEM_ALLOC;
-    cfg.stream = ctx.stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, tc_order1_kernel, tmQ, tmK, tmV, a) != cudaSuccess) {
+    // One launch: every CTA builds the state of its group alone, publishes it, adds up the groups before it (a chained
+    // scan with an anchor every eight groups) and walks its tiles again, now with the keys and values in L2.
+    int* flags = reinterpret_cast<int*>(ws + 2 * (size_t)BH * NG * E);
+    if (cudaMemsetAsync(flags, 0, ((size_t)BH * NG + 1) * sizeof(int), ctx.stream) != cudaSuccess) {
       cudaGetLastError();
       ctx.status = KATA_ERR_CUDA;
       return;
     }
-    ++ctx.launches;
-  } else {
-    tc_order1_kernel<<<dim3(BH, NG), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
+    a.local_state = bufA;
+    a.anchor_state = bufB;
+    a.flags = flags;
+    a.ticket = reinterpret_cast<unsigned*>(flags + (size_t)BH * NG);
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      cudaGetLastError();
+      sms = 148;
+    }
+    const unsigned total = (unsigned)BH * NG;
+    tc_order1_kernel<<<dim3(total < (unsigned)sms ? total : (unsigned)sms), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
     note_launch(ctx);
+    return;
   }
+  // one group: one CTA per head walks all its tiles
+  tc_order1_kernel<<<dim3(BH), NTHREADS, SMEM_ALLOC, ctx.stream>>>(tmQ, tmK, tmV, a);
+  note_launch(ctx);
 }
 
 }  // namespace kata
