@@ -382,7 +382,7 @@ def order1_inputs(B, T, dev, seed=11):
 
 def run_order1(args):
     """Profiler case of the first-order tensor-core kernel: B=16, H=16, T=8192, C=128 (inputs 805 MB > L2, 256
-    CTAs), one kernel per step in the sequential form, three passes with --mode scan; short line."""
+    CTAs), one kernel per step in both forms (--mode scan: eight groups per head, every group walked twice); short line."""
     import torch
     from paper_2607_17419_b200 import binding as kb, build as kbuild
     kbuild.build()

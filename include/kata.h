@@ -114,7 +114,13 @@ enum { KATA_FN_QUADRATIC = 0, KATA_FN_CHUNKED = 1, KATA_FN_CHUNK_STATE_SCAN = 2,
  *                 the paper's per-chunk pipeline, whenever s_pre/z_pre are requested).  The first-order
  *                 tensor-core path works in tiles of 128 tokens: it rounds the group up to whole tiles, and its
  *                 own choice may be a single group (one pass per head) when the heads alone fill the GPU;
- *                 kata_scan_plan reports what will run.
+ *                 kata_scan_plan reports what will run.  With more than one group it runs as ONE launch: the
+ *                 CTAs take groups in order, build the state of a group alone, publish it, add up the groups
+ *                 before it (a chained scan over the group states with an anchor every eighth group, summed in
+ *                 a fixed order: bit-reproducible) and walk the group again for the outputs; the scan_rounds
+ *                 that kata_scan_plan reports for this path are the anchor hops, not doubling rounds.  Its
+ *                 waits on other CTAs are bounded (2 s); a CTA that gives up marks its group so that the
+ *                 CTAs behind it give up at once.
  *  workspace      device scratch of at least kata_workspace_bytes(...) bytes, 256-byte aligned;
  *                 may be null when that size is 0.
  *  s_pre, z_pre   optional device outputs (fp32), both null or both non-null.
