@@ -36,7 +36,11 @@
  *   - Supported shapes: d_k, d_v in {16,32,64}; C = 64 (the chunked/scan forms), and C = 128 for
  *     feature_order 1 with bf16, d_k = d_v = 64 (the chunk size of the paper's scan benchmark; tensor-core
  *     path, no s_pre/z_pre); T >= 1 (any; the last chunk is zero-padded as in Algorithm 1 and truncated on
- *     output); B,H >= 1.  The tensor-core (tcgen05) kernels cover bf16 with d_k = d_v = 64; narrower bf16
+ *     output); B,H >= 1.  A kernel takes at most 65535 heads (B * H) at a time: kata_fwd_quadratic,
+ *     kata_fwd_chunked and kata_chunk_state_scan run more heads than that in slabs of 65535, one after the
+ *     other on the stream and in the same workspace (kata_workspace_bytes gives the largest slab's need), as
+ *     long as no state pointer is set; the other entry points, and these with state pointers, return
+ *     KATA_ERR_UNSUPPORTED_SHAPE beyond 65535 heads.  The tensor-core (tcgen05) kernels cover bf16 with d_k = d_v = 64; narrower bf16
  *     rows are zero-padded to 64 entries in the workspace and run on the same kernels (the result is the same
  *     function: dot products and norms do not change) unless feature_groups > 1 or a state is handed over, whose
  *     layouts depend on the true width; everything else runs on the fp32 SIMT kernels.

@@ -22,7 +22,7 @@ KATA_FN_QUADRATIC, KATA_FN_CHUNKED, KATA_FN_CHUNK_STATE_SCAN, KATA_FN_DECODE_STE
 KATA_FN_BWD_QUADRATIC = 4
 KATA_FN_BWD_CHUNKED = 5
 KATA_FN_HOST_IO = 0x100
-KATA_OK, KATA_ERR_INVALID_ARG, KATA_ERR_WORKSPACE_TOO_SMALL, KATA_ERR_DEVICE_TIMEOUT = 0, -1, -4, -7
+KATA_OK, KATA_ERR_INVALID_ARG, KATA_ERR_UNSUPPORTED_SHAPE, KATA_ERR_WORKSPACE_TOO_SMALL, KATA_ERR_DEVICE_TIMEOUT = 0, -1, -2, -4, -7
 
 EXPORTS = ("kata_fwd_quadratic", "kata_fwd_chunked", "kata_chunk_state_scan", "kata_chunk_state_scan_static",
            "kata_fwd_host", "kata_decode_step", "kata_bwd_quadratic", "kata_bwd_chunked",

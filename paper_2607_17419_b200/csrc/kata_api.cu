@@ -468,8 +468,33 @@ int run_device(int fn, Prepared& r, void* ws) {
   return ctx.status;
 }
 
+// The kernels put the head index on a grid axis that ends at 65535.  Heads are independent and lie one after the other
+// in [B,H,T,d] tensors, so the device entries of the forward take more heads than that in slabs of at most 65535, one
+// after the other on the caller's stream and in the same scratch (no state pointers: their layouts are per call).
+constexpr long long kMaxHeads = 65535;
+
 int entry(int fn, const void* q, const void* k, const void* v, void* out, int B, int H, int T, int d_k,
           int d_v, int C, const kata_opts* opts) {
+  if (B >= 1 && H >= 1 && (long long)B * H > kMaxHeads) {
+    Opts o;
+    int st = read_opts(opts, o);
+    if (st != KATA_OK) return st;
+    if (T < 1 || d_k < 1 || d_v < 1 || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return KATA_ERR_INVALID_ARG;
+    if (o.s_pre != nullptr || o.z_pre != nullptr || o.s_init != nullptr || o.z_init != nullptr) return KATA_ERR_UNSUPPORTED_SHAPE;
+    const size_t eb = elem_bytes(o.dtype);
+    const long long BH = (long long)B * H;
+    int launches = 0;
+    for (long long h0 = 0; h0 < BH; h0 += kMaxHeads) {
+      const int n = (int)(BH - h0 < kMaxHeads ? BH - h0 : kMaxHeads);
+      const size_t offk = (size_t)h0 * T * d_k * eb, offv = (size_t)h0 * T * d_v * eb;
+      st = entry(fn, static_cast<const char*>(q) + offk, static_cast<const char*>(k) + offk, static_cast<const char*>(v) + offv,
+                 static_cast<char*>(out) + offv, 1, n, T, d_k, d_v, C, opts);
+      if (st != KATA_OK) return st;
+      launches += g_last_launches;
+    }
+    g_last_launches = launches;
+    return KATA_OK;
+  }
   Prepared r;
   int st = prepare(fn, q, k, v, out, B, H, T, d_k, d_v, C, opts, true, r);
   if (st != KATA_OK) return st;
@@ -834,6 +859,13 @@ size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C
     if (host_io || read_opts(opts, o) != KATA_OK || B < 1 || H < 1 || !dim_ok(d_k) || !dim_ok(d_v)) return 0;
     return align_up(decode_workspace_elems(B * H, decode_n_psi(d_k, o.state_layout, o.feature_order, o.groups), d_v) * sizeof(float));
   }
+  if (!host_io && B >= 1 && H >= 1 && (long long)B * H > kMaxHeads) {
+    // the device entries work in slabs of heads: the scratch of the largest slab and of the last one
+    const long long BH = (long long)B * H, last = BH % kMaxHeads;
+    const size_t a = kata_workspace_bytes(fn, 1, (int)kMaxHeads, T, d_k, d_v, C, opts);
+    const size_t b = last > 0 ? kata_workspace_bytes(fn, 1, (int)last, T, d_k, d_v, C, opts) : 0;
+    return a > b ? a : b;
+  }
   Prepared r;
   if (prepare(fn, nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, C, opts, false, r) != KATA_OK) return 0;
   if (!host_io) return r.inner_bytes;
@@ -842,6 +874,7 @@ size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C
 
 int kata_scan_plan(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts, int* n_groups,
                    int* chunks_per_group, int* scan_rounds) {
+  if (B >= 1 && H >= 1 && (long long)B * H > kMaxHeads) { B = 1; H = (int)kMaxHeads; }   // the plan of a full slab of heads
   Prepared r;
   const int st = prepare(fn & ~KATA_FN_HOST_IO, nullptr, nullptr, nullptr, nullptr, B, H, T, d_k, d_v, C, opts,
                          false, r);

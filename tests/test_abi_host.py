@@ -247,3 +247,24 @@ def test_backward_argument_checks(L):
     o = kb.make_opts(kb.KATA_BF16)
     assert kb.kata_workspace_bytes(kb.KATA_FN_BWD_QUADRATIC, 2, 3, 100, 32, 16, 0, o) == \
         7 * up(rows * 128) + up(rows * 128) + up(rows * 4) + up(rows * 8)
+
+
+def test_more_heads_than_a_grid_axis(L):
+    """Beyond 65535 heads the forward device entries work in slabs: the scratch is the largest slab's, the plan a full
+    slab's; state pointers, the backward, the decode step and the host-buffer entry keep the limit."""
+    SHAPE, WS = -2, -4
+    o = kb.make_opts(kb.KATA_F32)
+    for fn in (kb.KATA_FN_CHUNKED, kb.KATA_FN_CHUNK_STATE_SCAN):
+        ws = lambda B, H, opts=o: kb.kata_workspace_bytes(fn, B, H, 300, 16, 16, 64, opts)
+        assert ws(65537, 1) == max(ws(1, 65535), ws(1, 2)) and ws(70000, 2) == max(ws(1, 65535), ws(1, 140000 % 65535))
+        assert kb.kata_scan_plan(fn, 65537, 1, 300, 16, 16, 64, o) == kb.kata_scan_plan(fn, 1, 65535, 300, 16, 16, 64, o)
+    assert kb.kata_workspace_bytes(kb.KATA_FN_QUADRATIC, 300, 300, 5, 16, 16, 64, o) == 0
+    # a slab's scratch is checked before anything is launched
+    need = kb.kata_workspace_bytes(kb.KATA_FN_CHUNK_STATE_SCAN, 65537, 1, 300, 16, 16, 64, o)
+    small = kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=need - 256)
+    assert call(L, "kata_chunk_state_scan", B=65537, T=300, d_k=16, d_v=16, opts=small) == WS
+    states = kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 40, s_init=4096, z_init=8192)
+    assert call(L, "kata_fwd_chunked", B=65537, T=300, d_k=16, d_v=16, opts=states) == SHAPE
+    ob = kb.make_opts(kb.KATA_F32, workspace=4096, workspace_bytes=1 << 40)
+    assert L.kata_bwd_quadratic(4096, 4096, 4096, 4096, 4096, 4096, 4096, 65537, 1, 8, 16, 16, ctypes.byref(ob)) == SHAPE
+    assert L.kata_decode_step(4096, 4096, 4096, 4096, 4096, 4096, 65537, 1, 16, 16, ctypes.byref(ob)) == SHAPE

@@ -291,3 +291,26 @@ def test_config4_long_context(T):
     lo, hi = np.minimum.accumulate(v, axis=2), np.maximum.accumulate(v, axis=2)
     slack = 2e-2 * np.maximum(1.0, np.abs(v).max())
     assert np.all(seq >= lo - slack) and np.all(seq <= hi + slack)
+
+
+def test_more_heads_than_one_grid_axis():
+    """65537 heads: a kernel takes at most 65535 at a time, the forward entries run the rest as a second slab on the
+    same stream and in the same scratch.  Heads on both sides of the cut against the definition; a call with state
+    pointers keeps the limit."""
+    import torch
+    B, H, T, d = 65537, 1, 3, 16
+    w = inputs.gaussian_workload("many_heads", "f32", B, H, T, d, d, 64, 91)
+    q, k, v = dev_tensors(w)
+    heads = [0, 1, 65533, 65534, 65535, 65536]
+    ref = {b: ko.kata_quadratic(w.q_ref[b, 0], w.k_ref[b, 0], w.v_ref[b, 0])[0] for b in heads}
+    for form in ("quadratic", "chunked_seq", "chunked_scan", "state_scan"):
+        g = run_form(form, w)
+        assert np.all(np.isfinite(g))
+        for b in heads:
+            check(g[b, 0], ref[b], "f32", f"{form}, head {b} of {B}")
+        assert kb.kata_last_launch_count() >= 2, "two slabs of heads"
+    S = torch.zeros(B, H, kb.decode_n_psi(d), d, device="cuda")
+    Z = torch.zeros(B, H, kb.decode_n_psi(d), device="cuda")
+    with pytest.raises(kb.KataError) as e:
+        kb.kata_fwd_chunked(q, k, v, s_init=S, z_init=Z)
+    assert e.value.status == kb.KATA_ERR_UNSUPPORTED_SHAPE
