@@ -30,7 +30,8 @@
  *     inside the 2e-2 tolerance of the bf16 tests.
  *   - The caller owns every buffer.  The library allocates no device or host memory, frees nothing and never
  *     synchronises; all work is enqueued on opts->stream.  q,k,v are read-only; out and the
- *     workspace are fully overwritten (no pre-zeroing needed).  One exception to "allocates nothing":
+ *     workspace are fully overwritten (no pre-zeroing needed).  A call on device pointers may therefore be
+ *     captured into a CUDA graph and replayed (same pointers, same workspace).  One exception to "allocates nothing":
  *     kata_fwd_host on its piecewise route creates, once per device and for the life of the process, two CUDA
  *     streams and seven events, and takes a process-wide mutex for the duration of the call (see there).
  *   - Supported shapes: d_k, d_v in {16,32,64}; C = 64 (the chunked/scan forms), and C = 128 for
