@@ -112,3 +112,30 @@ def test_scan_benchmark_shapes_sampled_rows(B, T):
         outs[form] = g
     assert np.max(np.abs(outs["chunked_scan"] - outs["chunked_seq"])) <= 2e-2
     assert np.max(np.abs(outs["state_scan"] - outs["chunked_seq"])) <= 2e-2
+
+
+@pytest.mark.parametrize("n_groups", [8, 9, 10, 16, 17, 18, 33])
+def test_anchor_boundaries_of_the_chained_scan(n_groups):
+    """Single-launch scan form with one tile per group: group counts on both sides of the anchors (every eighth
+    group publishes the sum of everything up to itself), a ragged last tile, more (group, head) tickets than SMs."""
+    T = 128 * n_groups - 5
+    w = inputs.nonnegative_workload(f"o1_anchor_{n_groups}", "bf16", 2, 3, T, 64, 64, 128, 900 + n_groups)
+    q, k, v = dev_tensors(w)
+    ng, cpg, hops = kb.kata_scan_plan(kb.KATA_FN_CHUNK_STATE_SCAN, 2, 3, T, 64, 64, 128,
+                                      kb.make_opts(kb.KATA_BF16, feature_order=1, scan_group=1))
+    assert (ng, cpg) == (n_groups, 1) and hops == (n_groups - 2) // 8 + 1
+    g = run("state_scan", q, k, v, C=128, scan_group=1)
+    assert kb.kata_last_launch_count() == 1
+    g2 = run("state_scan", q, k, v, C=128, scan_group=1)
+    assert np.array_equal(g, g2), "the sum over the group states has a fixed order"
+    for b in range(w.B):
+        for h in range(w.H):
+            check(g[b, h], reference(w, b, h), "bf16", f"order 1, {n_groups} groups ({b},{h})")
+
+
+def test_more_tickets_than_sms():
+    """32 heads x 12 groups = 384 (group, head) tickets for 148 persistent CTAs."""
+    w = inputs.nonnegative_workload("o1_tickets", "bf16", 2, 16, 3000, 64, 64, 128, 53)
+    g = run("state_scan", *dev_tensors(w), C=128, scan_group=2)
+    for b, h in ((0, 0), (0, 15), (1, 7), (1, 15)):
+        check(g[b, h], reference(w, b, h), "bf16", f"order 1, 384 tickets ({b},{h})")
