@@ -149,7 +149,8 @@ def kata_host_plan(fn: int, B, H, T, d_k, d_v, C, opts: KataOpts):
 def kata_selftest_wait_timeout(device_status, report, max_polls: int = 1000, stream=None) -> int:
     """Test hook (csrc/kata_selftest.h): one warp runs both bounded waits on a barrier nobody arrives at.
 
-    `device_status` is an int32 CUDA tensor of one element (or None), `report` one of three.  Returns the status code.
+    `device_status` is an int32 CUDA tensor of one element (or None), `report` one of eight (the last is the flag in
+    global memory that the flag wait is tried on: 0 on entry).  Returns the status code.
     """
     import torch
     if stream is None:

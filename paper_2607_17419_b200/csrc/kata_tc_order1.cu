@@ -90,33 +90,7 @@ struct OArgs {
   int BH;
 };
 
-// Single-launch form: flag values of a group.  A group that gave up poisons its flag so that its successors give up
-// at once instead of waiting out their limits.
-constexpr int kFlagLocal = 1, kFlagAnchor = 2, kFlagPoison = 99;
 constexpr int kAnchorEvery = 8;
-
-// Bounded wait for a group's flag (2 s of wall time: the group may belong to a CTA that started a wave earlier).
-__device__ __forceinline__ bool wait_flag(const int* p, int want, volatile int* abort_flag) {
-  unsigned t0 = 0;
-  for (uint32_t i = 0;; ++i) {
-    int v;
-    unsigned t1;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    if (v == kFlagPoison) break;
-    if (v >= want) return true;
-    if (*abort_flag) return false;
-    asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t1));
-    if (i == 0) t0 = t1;
-    if (t1 - t0 > 2000000000u) break;
-    __nanosleep(64);
-  }
-  *abort_flag = 1;
-  return false;
-}
-__device__ __forceinline__ void publish_flag(int* p, int v) {
-  __threadfence();
-  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 
 // One fp32 state row (64 features) as a bf16 row of a snapshot (128B swizzle: chunk index xor row-in-atom).
 __device__ __forceinline__ void snap_store_row(unsigned char* sp, int row, const uint32_t (&lo)[32], const uint32_t (&hi)[32]) {
@@ -232,7 +206,7 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int cnt = grp - anchor;                                   // 1 .. 8
     bool got = true;
     for (int g2 = anchor; g2 < grp && got; ++g2)
-      got = wait_flag(args.flags + (slot - grp + g2), (g2 == anchor && anchor > 0) ? kFlagAnchor : kFlagLocal, abort_flag);
+      got = wait_flag(args.flags + (slot - grp + g2), (g2 == anchor && anchor > 0) ? umma::kFlagAnchor : umma::kFlagLocal, abort_flag);
     const bool publish = grp % kAnchorEvery == 0 && grp + 1 < args.n_groups;
     float4* scratch = reinterpret_cast<float4*>(base);
     if (got) {
@@ -257,7 +231,7 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
     fence_async_smem();   // the stage buffer goes back to the TMA
     __syncthreads();
-    if (publish && tid == 0) publish_flag(args.flags + slot, *abort_flag ? kFlagPoison : kFlagAnchor);
+    if (publish && tid == 0) publish_flag(args.flags + slot, *abort_flag ? umma::kFlagPoison : umma::kFlagAnchor);
   }
   if (resume) {
     // the state before the first tile: into the accumulators and, as bf16, into snapshot 0
@@ -452,7 +426,7 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (fused && pass == 0) {
       // the group's own state is in place: tell the groups behind it
       asm volatile("bar.sync 6, 96;" ::: "memory");
-      if (warp == W_SNAP0 && lane == 0) publish_flag(args.flags + slot, *abort_flag ? kFlagPoison : kFlagLocal);
+      if (warp == W_SNAP0 && lane == 0) publish_flag(args.flags + slot, *abort_flag ? umma::kFlagPoison : umma::kFlagLocal);
     }
   } else if (warp >= W_BLD0 && wo) {
     // =========================== weights and epilogue (256 threads) ===========================
@@ -531,7 +505,7 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   __syncthreads();
   bars_live = true;
   if (*abort_flag) {
-    if (fused && tid == 0) publish_flag(args.flags + slot, kFlagPoison);
+    if (fused && tid == 0) publish_flag(args.flags + slot, umma::kFlagPoison);
     dead = true;
     break;
   }

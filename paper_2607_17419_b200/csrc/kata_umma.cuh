@@ -350,6 +350,33 @@ __device__ __forceinline__ bool wait_or_abort_counted(uint64_t* bar, uint32_t pa
   return wait_or_abort_polls(bar, parity, abort_flag, kSpinLimit);
 }
 
+// Flags that the CTAs of one launch publish for one another in global memory (the group states of the single-launch
+// first-order scan).  A CTA that gave up poisons its flag so that the CTAs waiting for it give up at once instead of
+// waiting out their limits.  The wait is bounded by wall time (default 2 s: the flag may belong to a CTA that started a
+// wave earlier); every thread that will read the published data waits for itself (its own acquire).
+constexpr int kFlagLocal = 1, kFlagAnchor = 2, kFlagPoison = 99;
+__device__ __forceinline__ bool wait_flag(const int* p, int want, volatile int* abort_flag, unsigned limit_ns = 2000000000u) {
+  unsigned t0 = 0;
+  for (uint32_t i = 0;; ++i) {
+    int v;
+    unsigned t1;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    if (v == kFlagPoison) break;
+    if (v >= want) return true;
+    if (*abort_flag) return false;
+    asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t1));
+    if (i == 0) t0 = t1;
+    if (t1 - t0 > limit_ns) break;
+    __nanosleep(64);
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void publish_flag(int* p, int v) {
+  __threadfence();
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);

@@ -91,11 +91,14 @@ def test_bounded_waits_time_out_cleanly_and_the_stream_stays_usable():
     same stream is correct.  Run on a test-only kernel of one warp (no TMEM, MMA or TMA in flight)."""
     import torch
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    rep = torch.full((3,), -1, dtype=torch.int32, device="cuda")
+    rep = torch.full((8,), -1, dtype=torch.int32, device="cuda")
+    rep[7] = 0                                               # the flag in global memory
     assert kb.kata_selftest_wait_timeout(st, rep, max_polls=2000) == kb.KATA_OK
     torch.cuda.synchronize()
     assert int(st.item()) == kb.KATA_ERR_DEVICE_TIMEOUT
-    assert rep.tolist() == [1, 1, 1], "both waits gave up and raised the abort flag"
+    assert rep.tolist()[:3] == [1, 1, 1], "both barrier waits gave up and raised the abort flag"
+    # the wait on a flag of another CTA: gives up when nobody sets it, returns when it is set, gives up at once on poison
+    assert rep.tolist()[3:7] == [1, 1, 1, 1]
     assert kb.kata_selftest_wait_timeout(st, rep, max_polls=0) == kb.KATA_ERR_INVALID_ARG
     # the next ordinary call on the same stream
     w = inputs.gaussian_workload("after_timeout", "bf16", 1, 2, 300, 64, 64, 64, 4242)
