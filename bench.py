@@ -549,10 +549,19 @@ def measure_extra(kb, inputs, dev, stream, q, k, v, out, peaks):
     for g in (2, 4):
         ms = timed(lambda: kb.kata_fwd_chunked(q, k, v, out, feature_groups=g))
         res[f"chunked_seq_M{g}"] = dict(ms=ms, tokens_per_s=T / (ms * 1e-3), launches=kb.kata_last_launch_count(),
+                                        ratio_to_M1=ms / res["chunked_seq"]["ms"],
                                         impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
         ms = timed(lambda: kb.kata_fwd_quadratic(q2, k2, v2, o2, feature_groups=g))
         res[f"quadratic_c2_M{g}"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), tflops=fl / (ms * 1e-3) / 1e12,
                                          impl="tensor" if kb.kata_last_impl() == kb.KATA_IMPL_TENSOR else "simt")
+    # the same forms on config 2 (64 heads x 4096 tokens), where the CTAs per head of a layout decide the number of
+    # waves of the grid: the blockwise maps against the full lift, with the ratio
+    ms1 = timed(lambda: kb.kata_fwd_chunked(q2, k2, v2, o2))
+    res["chunked_seq_c2"] = dict(ms=ms1, tokens_per_s=w2.B * w2.T / (ms1 * 1e-3), launches=kb.kata_last_launch_count())
+    for g in (2, 4):
+        ms = timed(lambda: kb.kata_fwd_chunked(q2, k2, v2, o2, feature_groups=g))
+        res[f"chunked_seq_c2_M{g}"] = dict(ms=ms, tokens_per_s=w2.B * w2.T / (ms * 1e-3), ratio_to_M1=ms / ms1,
+                                           launches=kb.kata_last_launch_count())
     # backward of the quadratic form on config 2 (tensor-core kernels; recomputation, 5 matrix products of
     # 2 * 64 flops per causal pair = 640 algorithmic flops per pair)
     g2 = torch.randn(v2.shape, device=dev, generator=torch.Generator(device=dev).manual_seed(7)).to(torch.bfloat16)
