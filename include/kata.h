@@ -195,7 +195,10 @@ int kata_fwd_chunked(const void* q, const void* k, const void* v, void* out,
  * S_loc = Psi(K_[c])^T V_[c], Z_loc = 1^T Psi(K_[c]) for all (b,h,c) in parallel; (ii) exclusive
  * prefix along the chunk axis in ceil(log2 N) rounds; (iii) chunk output from the prefix and
  * the local C x C causal term.  Writes out; if opts->s_pre/z_pre are set it also writes the
- * exclusive-prefix chunk states there (which forces scan_group = 1).
+ * exclusive-prefix chunk states there (which forces scan_group = 1).  With scan_group > 1 (or the library's choice)
+ * the stages work on groups of chunks, which the paper's associativity argument allows: the same result up to the
+ * rounding order of the state sums.  The first-order tensor-core path runs the three stages in one launch and its
+ * stage (ii) as a chained scan over the group states (see opts->scan_group).
  * Workspace: kata_workspace_bytes(KATA_FN_CHUNK_STATE_SCAN, ...).
  */
 int kata_chunk_state_scan(const void* q, const void* k, const void* v, void* out,
@@ -320,7 +323,9 @@ size_t kata_workspace_bytes(int fn, int B, int H, int T, int d_k, int d_v, int C
 int kata_host_plan(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts, int* pieces,
                    int* piece_tokens);
 
-/* Number of scan groups / chunks per group the library would use (for reporting and tests). */
+/* Number of scan groups, chunks per group and rounds of the scan over the group states (doubling rounds; anchor hops on
+ * the first-order tensor-core path) the library would use; beyond 65535 heads, those of a full slab of heads.  For
+ * reporting and tests. */
 int kata_scan_plan(int fn, int B, int H, int T, int d_k, int d_v, int C, const kata_opts* opts,
                    int* n_groups, int* chunks_per_group, int* scan_rounds);
 
