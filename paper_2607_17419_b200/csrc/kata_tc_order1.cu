@@ -173,6 +173,7 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const bool resume = lookback;
 
   if (tid == 0) {
+    // (one thread: initialising the barriers from as many threads at once gave barriers that did not work)
     if (bars_live)
       for (int i = 0; i < BAR_COUNT; ++i) mbar_inval(bar(i));
     for (int i = 0; i < NSTAGE; ++i) {
@@ -278,6 +279,11 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tma_load_3d(ktile(s), &tmK, bar(BAR_FULL + s), 0, tok, bh);
         tma_load_3d(vtile(s), &tmV, bar(BAR_FULL + s), 0, tok, bh);
       }
+      // The barriers are initialised again for the next pass, so no arrival may still be on its way when this pass
+      // ends: the last phases of the stage barriers, which no load waits for, are waited for here (a tcgen05.commit
+      // arrives some time after its MMAs; only a completed phase says that all its arrivals are in).
+      for (int j = (n > NSTAGE ? n - NSTAGE : 0); j < n && ok; ++j)      // the last tile of every stage that was used
+        ok = wait_or_abort_counted(bar(BAR_EMPTY + j % NSTAGE), (j / NSTAGE) & 1, abort_flag);
     }
   } else if (warp == W_MMA_A) {
     // =========================== scores P = Q K^T ===========================
@@ -303,6 +309,9 @@ tc_order1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         __syncwarp();
       }
+      // (as for the stage barriers: the weights barriers of the last two tiles, which no score MMA waits for)
+      for (int j = n; j < n + 2 && ok; ++j)
+        if (j >= 2) ok = wait_or_abort_counted(bar(BAR_P_EMPTY + (j & 1)), ((j >> 1) & 1) ^ 1, abort_flag);
     }
   } else if (warp == W_MMA_U) {
     // =========================== state update [S | Z]^T += [V | 1]^T K ===========================
